@@ -1,0 +1,213 @@
+/*
+ * gala.h -- C ABI of the B200 learner library for GALA-A2C
+ * (Gossip-based Actor-Learner Architectures, arXiv 1906.04585).
+ *
+ * The library holds N co-resident actor-learners ("agents") on one GPU and
+ * runs, per agent, the steps of Algorithm 1 after the environment
+ * interaction: network forward/backward over a rollout, n-step returns,
+ * advantages and the A2C objective, RMSProp, and the gossip average with the
+ * agent's in-peers.  Every step runs in CUDA kernels built for sm_100a; there
+ * is no CPU fallback.
+ *
+ * Conventions
+ *  - Every call returns 0 (GALA_OK) or a negative gala_status.  After a
+ *    failure, gala_last_error(ctx) returns a library-owned message that stays
+ *    valid until the next call on that context.
+ *  - The context owns parameters, optimiser state, snapshots, workspaces,
+ *    CUDA streams and events.  Rollout / observation / output buffers are
+ *    DEVICE pointers owned by the caller; they must stay valid until the
+ *    agent's stream has passed the call (gala_sync_agent, or gala_sync_all).
+ *    The only HOST pointers are the structs, gala_in_peers / gala_losses /
+ *    gala_stats outputs, and gala_get_state / gala_set_state buffers, which
+ *    may be host or device memory (the library asks the CUDA runtime which).
+ *  - Calls enqueue work and return; only the sync and get/set-state calls
+ *    wait.  One host thread per context.
+ *  - No kernel traps or spins without a bound.  A device-side wait that runs
+ *    out sets an error word that the next sync call reports as GALA_ECUDA.
+ *
+ * Flat parameter vector of one agent (x_i = (omega_i, theta_i), Sec. 3),
+ * float32, d entries, padded to d_padded:
+ *   conv net (Appendix C.2: 3 conv layers, one hidden layer, linear heads;
+ *   84x84x4 input, NHWC):
+ *     conv1.W[32][8][8][4]  conv1.b[32]      stride 4
+ *     conv2.W[64][4][4][32] conv2.b[64]      stride 2
+ *     conv3.W[64][3][3][64] conv3.b[64]      stride 1
+ *     fc.W[512][7][7][64]   fc.b[512]
+ *     pi.W[A][512] pi.b[A]  v.W[1][512] v.b[1]
+ *   MLP:  l1.W[H][obs_dim] l1.b[H]  l2.W[H][H] l2.b[H]
+ *         pi.W[A][H] pi.b[A]  v.W[1][H] v.b[1]
+ *   i.e. output-channel major, then (kh, kw, cin): the reduction index is the
+ *   fastest one.
+ */
+#ifndef GALA_H
+#define GALA_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gala_ctx gala_ctx; /* opaque */
+
+typedef enum {
+    GALA_OK = 0,
+    GALA_EINVAL = -1,   /* bad argument; nothing was enqueued */
+    GALA_ENOMEM = -2,   /* device or host allocation failed */
+    GALA_ECUDA = -3,    /* CUDA runtime error or device-side error word set */
+    GALA_ETIMEOUT = -4, /* a host wait with a deadline ran out */
+    GALA_ESTATE = -5    /* call not valid in the context's current state */
+} gala_status;
+
+typedef enum { GALA_NET_MLP = 0, GALA_NET_CONV = 1 } gala_net_kind;
+
+typedef struct {
+    int kind;       /* gala_net_kind */
+    int obs_dim;    /* MLP: observation length (float32). CONV: ignored (84x84x4 uint8) */
+    int hidden;     /* MLP: width of the two tanh layers. CONV: ignored (512) */
+    int n_actions;  /* 2..32 */
+    int gemm_dtype; /* 0 = fp32 FMA (MLP), 1 = bf16 operands, fp32 accumulate (CONV) */
+} gala_net_spec;
+
+typedef enum { GALA_TOPO_RING = 0, GALA_TOPO_EXP = 1, GALA_TOPO_COMPLETE = 2 } gala_topo_kind;
+
+/* Communication topology = the non-zero pattern of the mixing matrix P^(k)
+ * (Sec. 2 "Gossip algorithms", Sec. 3).  Non-zero weights are 1/(1+|N_in_i|)
+ * (footnote of Algorithm 1).
+ *   RING: directed ring v_0 -> v_1 -> ... -> v_{n-1} -> v_0 (Appendix C.2,
+ *         Fig. 5); in-peers of i are i-1 .. i-peers (mod n).
+ *   EXP:  time-varying exponential graph, L = ceil(log2 n): the j-th in-peer
+ *         of i at round k is i - 2^((peers*k + j) mod L) (mod n).
+ *   COMPLETE: reserved (not implemented; gala_create returns GALA_EINVAL). */
+typedef struct {
+    int kind;  /* gala_topo_kind */
+    int peers; /* in-peers per round: 1 or 2 */
+} gala_topology;
+
+/* Hyper-parameters (Table 2).  lr is used as given (the sqrt(#learners)
+ * scaling of Table 2 is the caller's). */
+typedef struct {
+    float lr;            /* 7e-4 */
+    float rms_alpha;     /* RMSProp decay, 0.99 */
+    float rms_eps;       /* added outside the square root */
+    float gamma;         /* discount, 0.99 */
+    float ent_coef;      /* eta of Eq. 3, 0.01 */
+    float vf_coef;       /* weight of the TD loss of Eq. 1, 0.5 */
+    float max_grad_norm; /* global-norm clip, 0.5; <= 0 switches it off */
+    int n_envs;          /* E: simulators per agent */
+    int n_steps;         /* T: rollout horizon (N in the paper) */
+    int staleness_tau;   /* reserved; must be < 0 (unbounded staleness) */
+    unsigned long long seed; /* initial parameters (library's own generator) */
+    int identical_init;  /* 1: all agents start from the same parameters (assumed by Prop. 1) */
+} gala_hparams;
+
+/* One agent's rollout {(s_t, a_t, r_t, s_{t+1})} (Algorithm 1, acting step). DEVICE pointers. */
+typedef struct {
+    const void* obs;            /* [T+1][E][84][84][4] uint8  or  [T+1][E][obs_dim] float32 */
+    const int* actions;         /* [T][E], each in [0, n_actions) */
+    const float* rewards;       /* [T][E] */
+    const unsigned char* dones; /* [T][E]; 1 = the episode ended at this step */
+} gala_rollout;
+
+/* Create n_agents agents (1..256).  Allocates everything; parameters are
+ * initialised from hp->seed (uniform +-1/sqrt(fan_in)), square-average state
+ * to 0, round counters to 0.  Uses the current CUDA device. */
+int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* net,
+                const gala_hparams* hp, gala_ctx** out);
+int gala_destroy(gala_ctx* ctx);
+
+/* Acting step of Algorithm 1: forward on E observations obs[E][...], softmax,
+ * inverse-CDF draw a = min{k : sum_{j<=k} pi_j > u} (clamped to A-1) from the
+ * caller's uniforms[E] in [0,1); writes actions[E] (int32), values[E].  All
+ * DEVICE pointers; actions or values may be NULL.  Uses the agent's forward
+ * workspace: do not interleave between gala_learn and its completion on
+ * another stream. */
+int gala_act(gala_ctx* ctx, int agent, const void* obs, const float* uniforms, int* actions,
+             float* values);
+
+/* Learner step of Algorithm 1 (returns, advantages, A2C gradient; Eqs. 1-4)
+ * on the agent's stream.  Leaves a pending gradient and its global norm.  If a
+ * gradient is already pending it is first applied without mixing (the
+ * no-gossip update of the appendix) and published. */
+int gala_learn(gala_ctx* ctx, int agent, const gala_rollout* rollout);
+
+/* Optimiser + gossip steps of Algorithm 1 on the agent's stream, one fused
+ * pass over the flat vector: RMSProp with the pending gradient (none
+ * pending: parameters unchanged), publish the result as the agent's newest
+ * snapshot (the non-blocking broadcast), and, if a snapshot newer than the
+ * one last consumed has COMPLETED for every in-peer of the agent's current
+ * round, replace the parameters by the equal-weight average (Eq. 6);
+ * otherwise keep the local result (Eq. 5).  Never waits for a peer. */
+int gala_gossip(gala_ctx* ctx, int agent);
+
+/* Deterministic synchronous round for all agents (Eq. 7 with zero delay):
+ * learn on rollouts[0..n_agents), then x_i <- (y_i + sum_{j in N_in_i(k)} y_j)/(1+p)
+ * with y the post-RMSProp parameters of the SAME round.  Runs on the
+ * context's main stream; waits for all agent streams first.  rollouts may be
+ * NULL: then the gradients currently stored (gala_set_grad) are used. */
+int gala_step_sync(gala_ctx* ctx, const gala_rollout* rollouts);
+
+/* Host waits.  timeout_ms < 0: no deadline.  GALA_ETIMEOUT if work is still
+ * running at the deadline (nothing is cancelled). */
+int gala_sync_agent(gala_ctx* ctx, int agent, int timeout_ms);
+int gala_sync_all(gala_ctx* ctx, int timeout_ms);
+
+/* Schedule query (host integers): in-peers of `agent` at round `round`.
+ * peers[] needs room for topo.peers entries. */
+int gala_in_peers(const gala_ctx* ctx, long long round, int agent, int* peers, int* n);
+
+/* State exchange (synchronises the agent first).  Any pointer may be NULL.
+ * Buffers hold d floats (not padded); host or device memory. */
+int gala_get_state(gala_ctx* ctx, int agent, float* params, float* sq_avg, float* grad,
+                   long long* round);
+int gala_set_state(gala_ctx* ctx, int agent, const float* params, const float* sq_avg,
+                   long long round);
+/* Store a gradient as the agent's pending gradient (for optimiser-only runs).
+ * clip_coef is the factor c applied to it (1 = none); < 0: compute it from
+ * max_grad_norm on the device. */
+int gala_set_grad(gala_ctx* ctx, int agent, const float* grad, float clip_coef);
+
+int gala_param_count(const gala_ctx* ctx, long long* d, long long* d_padded);
+/* out = {policy term, mean squared TD error, mean entropy, gradient norm} of the last learn. */
+int gala_losses(gala_ctx* ctx, int agent, float out[4]);
+/* out = {frames, rounds, mixes, skipped mixes, staleness sum, staleness max, published version, 0} */
+int gala_stats(gala_ctx* ctx, int agent, long long out[8]);
+/* Which snapshot versions the agent's last gala_gossip consumed: versions[j]
+ * for in-peer peers[j]; *mixed = 1 if the average was taken. */
+int gala_last_mix(gala_ctx* ctx, int agent, int* peers, long long* versions, int* n, int* mixed);
+/* Read snapshot `version` of an agent if it is still held (the two newest are). */
+int gala_get_snapshot(gala_ctx* ctx, int agent, long long version, float* out);
+/* Adopt a caller's CUDA stream (cudaStream_t) for the agent; NULL restores the library's. */
+int gala_set_stream(gala_ctx* ctx, int agent, void* cuda_stream);
+/* Copy intermediate tensors of the last learn/act of an agent for checks:
+ * what = 0 logits [B][A] f32, 1 values [B] f32, 2 returns [S], 3 advantages [S],
+ * 4 dlogits [S][A], 5 dvalues [S]; 10+l: output of trunk layer l as float32
+ * (B = (T+1)E rows).  out: host or device, `count` floats. */
+int gala_debug_read(gala_ctx* ctx, int agent, int what, float* out, long long count);
+/* Number of kernel launches issued by this context so far. */
+long long gala_launch_count(const gala_ctx* ctx);
+const char* gala_last_error(const gala_ctx* ctx);
+
+/* Stand-alone grouped GEMM on the tensor cores, exposed for validation:
+ * D[g] = op(A[g]) * op(B[g])^T, bf16 operands, fp32 accumulate, fp32 output
+ * D[g][M][N] row-major.  a_mn = 0: A stored [M][K] (K contiguous); 1: stored
+ * [K][M].  b_mn = 0: B stored [N][K]; 1: stored [K][N].  DEVICE pointers to
+ * bf16 (A, B) and float (D); K, M, N and the leading dimensions must keep
+ * rows 16-byte aligned (multiples of 8 elements).  split_k >= 1 splits the
+ * reduction and sums the partials in a fixed order.  Runs on `stream`
+ * (cudaStream_t, may be NULL) and returns after enqueueing. */
+int gala_gemm_bf16(const void* A, const void* B, float* D, int groups, int M, int N, int K,
+                   int a_mn, int b_mn, int split_k, void* stream);
+
+/* Stand-alone fused RMSProp + gossip pass over caller-owned arrays, exposed
+ * for the optimiser micro-benchmark and its parity test (Algorithm 1 optimiser
+ * and gossip steps; Eq. 7).  x, g, v: DEVICE float32 [n_agents][d_padded],
+ * updated in place (x, v).  Synchronous all-agent form: every agent takes its
+ * RMSProp step and all mix simultaneously with the in-peers of `round`.
+ * clip: DEVICE float[n_agents] or NULL (= 1).  d_padded % 4 == 0. */
+int gala_sweep_sync(float* x, const float* g, float* v, const float* clip, int n_agents,
+                    long long d_padded, const gala_topology* topo, long long round,
+                    const gala_hparams* hp, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GALA_H */

@@ -1,0 +1,973 @@
+// C ABI of the GALA learner library: context, topology schedule, per-agent streams and
+// double-buffered parameter snapshots, and the orchestration of Algorithm 1's learner,
+// optimiser and gossip steps out of the kernels in the other sources.
+#include <chrono>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <thread>
+
+#include "internal.h"
+
+using namespace gala;
+
+namespace {
+
+struct Agent {
+    cudaStream_t stream = nullptr, lib_stream = nullptr;
+    cudaEvent_t pub_event[2] = {nullptr, nullptr};  // completion of the sweep that wrote snapshot slot s
+    cudaEvent_t sweep_done = nullptr;               // completion of the agent's latest sweep
+    cudaEvent_t fence = nullptr;                    // scratch event for cross-stream ordering
+    long long version = 0;                          // newest snapshot version enqueued (0: none)
+    long long round = 0;                            // local iteration counter
+    bool pending = false;                           // a gradient waits for its optimiser step
+    std::vector<long long> consumed;                // newest version consumed from each agent
+    std::vector<int> slot_readers[2];               // agents whose sweeps read snapshot slot s
+    long long frames = 0, mixes = 0, skipped = 0, stale_sum = 0, stale_max = 0;
+    int last_n = 0, last_mixed = 0;
+    int last_peers[2] = {0, 0};
+    long long last_versions[2] = {0, 0};
+};
+
+struct Plan {  // one tensor-core product with its descriptors
+    GemmOperand A, B;
+    GemmArgs args;
+    long mask_stride = 0;
+};
+
+}  // namespace
+
+struct gala_ctx {
+    int n = 0;
+    gala_topology topo{};
+    gala_net_spec net{};
+    gala_hparams hp{};
+    long d = 0, d_pad = 0;
+    int T = 0, E = 0, A = 0, H = 0, obs_dim = 0;
+    long B = 0, S = 0;
+    bool conv = false;
+    ConvLayout cl{};
+    MlpLayout ml{};
+    std::vector<Agent> agents;
+    cudaStream_t main_stream = nullptr;
+    cudaEvent_t main_event = nullptr;
+    long long sync_round = 0;
+    long long launches = 0;
+    std::string err;
+    std::vector<void*> allocs;
+
+    float *x = nullptr, *g = nullptr, *v = nullptr, *snap = nullptr;
+    __nv_bfloat16* shadow = nullptr;
+    float *clip = nullptr, *norm = nullptr, *losses = nullptr;
+    double *norm_partial = nullptr, *colsum_partial = nullptr;
+    unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr;
+    int* error_word = nullptr;
+    float *logits = nullptr, *values = nullptr, *returns = nullptr, *adv = nullptr, *dlogits = nullptr,
+          *dvalues = nullptr;
+    // MLP workspaces
+    float *h1 = nullptr, *h2 = nullptr, *dpre1 = nullptr, *dpre2 = nullptr;
+    // conv workspaces (bf16)
+    __nv_bfloat16 *cols[3] = {nullptr, nullptr, nullptr}, *act[3] = {nullptr, nullptr, nullptr};
+    __nv_bfloat16 *hid = nullptr, *dh = nullptr, *dy[3] = {nullptr, nullptr, nullptr},
+                  *dcols[3] = {nullptr, nullptr, nullptr};
+    float* splitk_ws = nullptr;
+    long splitk_group_stride = 0;
+    int max_split = 32;
+    Plan fwd[3], fc_fwd, fc_wgrad, fc_dgrad, wgrad[3], dgrad[3];
+};
+
+namespace {
+
+int fail(gala_ctx* c, int code, const char* fmt, ...) {
+    if (c) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        c->err = buf;
+    }
+    return code;
+}
+#define CK(call)                                                                                       \
+    do {                                                                                               \
+        cudaError_t e__ = (call);                                                                      \
+        if (e__ != cudaSuccess)                                                                        \
+            return fail(c, e__ == cudaErrorMemoryAllocation ? GALA_ENOMEM : GALA_ECUDA, "%s: %s", #call, \
+                        cudaGetErrorString(e__));                                                      \
+    } while (0)
+#define LAUNCH(call)      \
+    do {                  \
+        CK(call);         \
+        c->launches++;    \
+    } while (0)
+
+template <typename Tp>
+int dev_alloc(gala_ctx* c, Tp** p, size_t count) {
+    void* q = nullptr;
+    size_t bytes = count * sizeof(Tp);
+    if (bytes == 0) bytes = 16;
+    cudaError_t e = cudaMalloc(&q, bytes);
+    if (e != cudaSuccess) return fail(c, GALA_ENOMEM, "cudaMalloc(%zu bytes): %s", bytes, cudaGetErrorString(e));
+    e = cudaMemset(q, 0, bytes);
+    if (e != cudaSuccess) return fail(c, GALA_ECUDA, "cudaMemset: %s", cudaGetErrorString(e));
+    c->allocs.push_back(q);
+    *p = reinterpret_cast<Tp*>(q);
+    return GALA_OK;
+}
+#define ALLOC(ptr, count)                       \
+    do {                                        \
+        int r__ = dev_alloc(c, &(ptr), (count)); \
+        if (r__ != GALA_OK) return r__;         \
+    } while (0)
+
+// ------------------------------------------------------------------ topology (integers only)
+// In-peers of `agent` at round `round`.
+//   ring: directed ring v_0 -> v_1 -> ... -> v_0, in-peers i-1 .. i-p (Appendix C.2, Fig. 5)
+//   exponential: L = ceil(log2 n); j-th in-peer is i - 2^((p*round + j) mod L)
+// Coinciding peers are kept as separate terms so the weights stay 1/(1+p).
+int topo_offsets(const gala_topology& t, int n, long long round, int* off) {
+    if (n <= 1) return 0;
+    if (t.kind == GALA_TOPO_RING) {
+        for (int j = 0; j < t.peers; j++) off[j] = (j + 1) % n;
+        return t.peers;
+    }
+    int L = 0;
+    while ((1LL << L) < n) L++;
+    if (L < 1) L = 1;
+    for (int j = 0; j < t.peers; j++) {
+        long long e = ((long long)t.peers * round + j) % L;
+        off[j] = (int)((1LL << e) % n);
+    }
+    return t.peers;
+}
+
+// ------------------------------------------------------------------ initial parameters
+// Counter-based generator: SplitMix64 finaliser applied to (seed, agent, index).
+inline uint64_t splitmix64(uint64_t z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+inline float uniform_pm1(uint64_t seed, uint64_t agent, uint64_t idx) {
+    uint64_t h = splitmix64(splitmix64(seed ^ (agent * 0xD1342543DE82EF95ull)) + idx);
+    return (float)((double)(h >> 11) * (1.0 / 9007199254740992.0) * 2.0 - 1.0);
+}
+void init_tensor(float* p, long off, long count, int fan_in, uint64_t seed, uint64_t agent) {
+    const float s = 1.0f / std::sqrt((float)fan_in);
+    for (long i = 0; i < count; i++) p[off + i] = s * uniform_pm1(seed, agent, (uint64_t)(off + i));
+}
+
+void fill_batch(PtrBatch& pb, const void* base, long stride_bytes, int agent0, int count) {
+    for (int i = 0; i < count; i++) pb.p[i] = reinterpret_cast<const char*>(base) + (long)(agent0 + i) * stride_bytes;
+}
+
+// ------------------------------------------------------------------ GEMM plans (conv net)
+int build_plans(gala_ctx* c) {
+    const int n = c->n;
+    const long B = c->B, S = c->S, dp = c->d_pad;
+    const int P[3] = {400, 81, 49};
+    auto zero_args = [&](Plan& p) {
+        memset(&p.args, 0, sizeof p.args);
+        p.args.groups = n; p.args.split_k = 1; p.args.scale = 1.0f; p.args.error_word = c->error_word;
+    };
+    bool ok = true;
+    for (int l = 0; l < 3; l++) {
+        const int KK = kConvKK[l], CO = kConvCout[l];
+        const int bn = CO;  // 32 or 64
+        // forward: patches [B*P][KK] x W[CO][KK]^T -> act[l] (bias, ReLU; conv1 also 1/255)
+        Plan& f = c->fwd[l];
+        zero_args(f);
+        ok &= make_operand(&f.A, c->cols[l], 0, (uint64_t)B * P[l], KK, n, KK, (uint64_t)B * P[l] * KK, 128);
+        ok &= make_operand(&f.B, c->shadow + c->cl.w[l], 0, CO, KK, n, KK, dp, bn);
+        f.args.M = (int)(B * P[l]); f.args.N = CO; f.args.K = KK; f.args.block_n = bn;
+        f.args.flags = EPI_OUT_BF16 | EPI_RELU;
+        f.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
+        f.args.bias = c->x + c->cl.b[l]; f.args.bias_group_stride = dp;
+        f.args.out = c->act[l]; f.args.out_group_stride = B * P[l] * CO; f.args.ldc = CO;
+        // weight gradient, transposed product: (patches^T [KK x S*P]) x (dY [S*P x CO]) stored at W[co][kk]
+        Plan& w = c->wgrad[l];
+        zero_args(w);
+        ok &= make_operand(&w.A, c->cols[l], 1, KK, (uint64_t)S * P[l], n, KK, (uint64_t)B * P[l] * KK, 128);
+        ok &= make_operand(&w.B, c->dy[l], 1, CO, (uint64_t)S * P[l], n, CO, (uint64_t)S * P[l] * CO, 64);
+        w.args.M = KK; w.args.N = CO; w.args.K = (int)(S * P[l]); w.args.block_n = 64;
+        w.args.flags = EPI_TRANSPOSE;
+        w.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
+        w.args.out = c->g + c->cl.w[l]; w.args.out_group_stride = dp; w.args.ldc = KK;
+        // data gradient (conv2, conv3): dY [S*P][CO] x W[CO][KK] -> patch gradients [S*P][KK]
+        if (l > 0) {
+            Plan& dg = c->dgrad[l];
+            zero_args(dg);
+            ok &= make_operand(&dg.A, c->dy[l], 0, (uint64_t)S * P[l], CO, n, CO, (uint64_t)S * P[l] * CO, 128);
+            ok &= make_operand(&dg.B, c->shadow + c->cl.w[l], 1, KK, CO, n, KK, dp, 128);
+            dg.args.M = (int)(S * P[l]); dg.args.N = KK; dg.args.K = CO; dg.args.block_n = 128;
+            dg.args.flags = EPI_OUT_BF16;
+            dg.args.out = c->dcols[l]; dg.args.out_group_stride = S * P[l] * KK; dg.args.ldc = KK;
+        }
+    }
+    {   // hidden layer forward: act3 [B][3136] x Wfc[512][3136]^T -> hid (bias, ReLU)
+        Plan& f = c->fc_fwd;
+        zero_args(f);
+        ok &= make_operand(&f.A, c->act[2], 0, B, kFeat, n, kFeat, (uint64_t)B * kFeat, 128);
+        ok &= make_operand(&f.B, c->shadow + c->cl.fcw, 0, kHidden, kFeat, n, kFeat, dp, 128);
+        f.args.M = (int)B; f.args.N = kHidden; f.args.K = kFeat; f.args.block_n = 128;
+        f.args.flags = EPI_OUT_BF16 | EPI_RELU;
+        f.args.bias = c->x + c->cl.fcb; f.args.bias_group_stride = dp;
+        f.args.out = c->hid; f.args.out_group_stride = B * kHidden; f.args.ldc = kHidden;
+        // weight gradient: dh^T [512 x S] x act3 [S x 3136] -> gW[512][3136]
+        Plan& w = c->fc_wgrad;
+        zero_args(w);
+        ok &= make_operand(&w.A, c->dh, 1, kHidden, S, n, kHidden, (uint64_t)S * kHidden, 128);
+        ok &= make_operand(&w.B, c->act[2], 1, kFeat, S, n, kFeat, (uint64_t)B * kFeat, 128);
+        w.args.M = kHidden; w.args.N = kFeat; w.args.K = (int)S; w.args.block_n = 128;
+        w.args.out = c->g + c->cl.fcw; w.args.out_group_stride = dp; w.args.ldc = kFeat;
+        // data gradient: dh [S][512] x Wfc [512][3136] -> dY3 [S][3136], masked by act3 > 0
+        Plan& dg = c->fc_dgrad;
+        zero_args(dg);
+        ok &= make_operand(&dg.A, c->dh, 0, S, kHidden, n, kHidden, (uint64_t)S * kHidden, 128);
+        ok &= make_operand(&dg.B, c->shadow + c->cl.fcw, 1, kFeat, kHidden, n, kFeat, dp, 128);
+        dg.args.M = (int)S; dg.args.N = kFeat; dg.args.K = kHidden; dg.args.block_n = 128;
+        dg.args.flags = EPI_OUT_BF16 | EPI_MASK;
+        dg.args.mask = c->act[2]; dg.args.mask_group_stride = B * kFeat;
+        dg.args.out = c->dy[2]; dg.args.out_group_stride = S * kFeat; dg.args.ldc = kFeat;
+    }
+    return ok ? GALA_OK : fail(c, GALA_ECUDA, "cuTensorMapEncodeTiled failed while building GEMM descriptors");
+}
+
+int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override, cudaStream_t st) {
+    GemmArgs a = p.args;
+    a.group0 = agent0; a.groups = groups;
+    if (m_override > 0) a.M = m_override;
+    const bool bf = a.flags & EPI_OUT_BF16;
+    a.out = reinterpret_cast<char*>(a.out) + (long)agent0 * a.out_group_stride * (bf ? 2 : 4);
+    if (a.mask) a.mask += (long)agent0 * a.mask_group_stride;
+    LAUNCH(launch_gemm(p.A, p.B, a, st));
+    return GALA_OK;
+}
+
+// weight-gradient product with the reduction split over CTAs and a fixed-order second stage
+int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t st) {
+    const int k_tiles = (p.args.K + 63) / 64;
+    const int tiles = ((p.args.M + 127) / 128) * ((p.args.N + p.args.block_n - 1) / p.args.block_n);
+    int split = (2 * 148) / (groups * tiles);
+    if (split > k_tiles / 4) split = k_tiles / 4;
+    if (split > c->max_split) split = c->max_split;
+    if (split < 1) split = 1;
+    if (split == 1) return run_plan(c, p, agent0, groups, 0, st);
+    GemmArgs a = p.args;
+    const long count = (long)p.args.M * p.args.N;
+    a.group0 = agent0; a.groups = groups; a.split_k = split;
+    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+    a.out_group_stride = c->splitk_group_stride;
+    a.out_split_stride = count;
+    LAUNCH(launch_gemm(p.A, p.B, a, st));
+    LAUNCH(launch_splitk_reduce(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
+                                reinterpret_cast<float*>(p.args.out) + (long)agent0 * p.args.out_group_stride, count,
+                                split, count, groups, c->splitk_group_stride, p.args.out_group_stride, st));
+    return GALA_OK;
+}
+
+// ------------------------------------------------------------------ forward / backward
+// Forward on `rows` observations per agent for agents [agent0, agent0+groups).
+int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, cudaStream_t st) {
+    const long dp = c->d_pad, B = c->B;
+    if (c->conv) {
+        const int P[3] = {400, 81, 49};
+        LAUNCH(launch_im2col_u8(obs, c->cols[0] + (long)agent0 * B * 400 * 256, B * 400 * 256, rows, groups, st));
+        for (int l = 0; l < 3; l++) {
+            int r = run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st);
+            if (r != GALA_OK) return r;
+            if (l < 2) {
+                const long as = B * P[l] * kConvCout[l], cs = B * P[l + 1] * kConvKK[l + 1];
+                LAUNCH(launch_im2col_bf16(c->act[l] + (long)agent0 * as, as, c->cols[l + 1] + (long)agent0 * cs, cs,
+                                          l + 1, rows, groups, st));
+            }
+        }
+        int r = run_plan(c, c->fc_fwd, agent0, groups, rows, st);
+        if (r != GALA_OK) return r;
+        HeadsArgs h{};
+        h.rows = rows; h.H = kHidden; h.A = c->A;
+        h.h = c->hid + (long)agent0 * B * kHidden; h.h_stride = B * kHidden; h.h_bf16 = 1;
+        h.params = c->x + (long)agent0 * dp; h.p_stride = dp;
+        h.piw = c->cl.piw; h.pib = c->cl.pib; h.vw = c->cl.vw; h.vb = c->cl.vb;
+        h.logits = c->logits + (long)agent0 * B * c->A; h.logits_stride = B * c->A;
+        h.values = c->values + (long)agent0 * B; h.values_stride = B;
+        LAUNCH(launch_heads_fwd(h, groups, st));
+    } else {
+        const int H = c->H;
+        DenseArgs a{};
+        a.rows = rows; a.in_dim = c->obs_dim; a.out_dim = H; a.act = 2;
+        a.in = obs; a.in_bf16 = 0;
+        a.W = c->x + (long)agent0 * dp + c->ml.w1; a.b = c->x + (long)agent0 * dp + c->ml.b1; a.w_stride = dp;
+        a.out = c->h1 + (long)agent0 * B * H; a.out_stride = B * H; a.out_bf16 = 0;
+        LAUNCH(launch_dense_fwd(a, groups, st));
+        DenseArgs b = a;
+        b.in_dim = H;
+        fill_batch(b.in, c->h1, B * H * 4, agent0, groups);
+        b.W = c->x + (long)agent0 * dp + c->ml.w2; b.b = c->x + (long)agent0 * dp + c->ml.b2;
+        b.out = c->h2 + (long)agent0 * B * H;
+        LAUNCH(launch_dense_fwd(b, groups, st));
+        HeadsArgs h{};
+        h.rows = rows; h.H = H; h.A = c->A;
+        h.h = c->h2 + (long)agent0 * B * H; h.h_stride = B * H; h.h_bf16 = 0;
+        h.params = c->x + (long)agent0 * dp; h.p_stride = dp;
+        h.piw = c->ml.piw; h.pib = c->ml.pib; h.vw = c->ml.vw; h.vb = c->ml.vb;
+        h.logits = c->logits + (long)agent0 * B * c->A; h.logits_stride = B * c->A;
+        h.values = c->values + (long)agent0 * B; h.values_stride = B;
+        LAUNCH(launch_heads_fwd(h, groups, st));
+    }
+    return GALA_OK;
+}
+
+int colsum(gala_ctx* c, const __nv_bfloat16* dy, long stride, long rows, int C, long grad_off, int agent0, int groups,
+           cudaStream_t st) {
+    LAUNCH(launch_colsum(dy + (long)agent0 * stride, stride, rows, C, c->g + (long)agent0 * c->d_pad + grad_off,
+                         c->d_pad, c->colsum_partial + (long)agent0 * kColsumChunks * 512, c->colsum_ticket + agent0,
+                         groups, st));
+    return GALA_OK;
+}
+
+// Learner step for agents [agent0, agent0+groups): forward, returns/advantages/objective,
+// backward into the flat gradient, global norm and clip coefficient.
+int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cudaStream_t st) {
+    const long dp = c->d_pad, B = c->B, S = c->S;
+    const int A = c->A;
+    PtrBatch obs{}, acts{}, rews{}, dns{};
+    for (int i = 0; i < groups; i++) {
+        obs.p[i] = ro[i].obs; acts.p[i] = ro[i].actions; rews.p[i] = ro[i].rewards; dns.p[i] = ro[i].dones;
+    }
+    int r = forward(c, agent0, groups, obs, (int)B, st);
+    if (r != GALA_OK) return r;
+    LossArgs la{};
+    la.T = c->T; la.E = c->E; la.A = A; la.B = B;
+    la.gamma = c->hp.gamma; la.ent_coef = c->hp.ent_coef; la.vf_coef = c->hp.vf_coef;
+    la.logits = c->logits + (long)agent0 * B * A; la.values = c->values + (long)agent0 * B;
+    la.actions = acts; la.rewards = rews; la.dones = dns;
+    la.returns = c->returns + (long)agent0 * S; la.adv = c->adv + (long)agent0 * S;
+    la.dlogits = c->dlogits + (long)agent0 * S * A; la.dvalues = c->dvalues + (long)agent0 * S;
+    la.losses = c->losses + (long)agent0 * 4;
+    LAUNCH(launch_a2c_loss(la, groups, st));
+
+    HeadsBwdArgs hb{};
+    hb.rows = (int)S; hb.A = A;
+    hb.params = c->x + (long)agent0 * dp; hb.p_stride = dp;
+    hb.dlogits = la.dlogits; hb.dlogits_stride = S * A;
+    hb.dvalues = la.dvalues; hb.dvalues_stride = S;
+    hb.grad = c->g + (long)agent0 * dp; hb.g_stride = dp;
+    if (c->conv) {
+        const int P[3] = {400, 81, 49};
+        hb.H = kHidden; hb.act = 1;
+        hb.h = c->hid + (long)agent0 * B * kHidden; hb.h_stride = B * kHidden; hb.h_bf16 = 1;
+        hb.piw = c->cl.piw; hb.pib = c->cl.pib; hb.vw = c->cl.vw; hb.vb = c->cl.vb;
+        hb.dpre = c->dh + (long)agent0 * S * kHidden; hb.dpre_stride = S * kHidden; hb.dpre_bf16 = 1;
+        LAUNCH(launch_heads_bwd(hb, groups, st));
+        c->launches++;  // two kernels
+        if ((r = colsum(c, c->dh, S * kHidden, S, kHidden, c->cl.fcb, agent0, groups, st)) != GALA_OK) return r;
+        if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, st)) != GALA_OK) return r;
+        if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
+        for (int l = 2; l >= 0; l--) {
+            const int CO = kConvCout[l];
+            if ((r = colsum(c, c->dy[l], S * P[l] * CO, S * P[l], CO, c->cl.b[l], agent0, groups, st)) != GALA_OK) return r;
+            if ((r = run_wgrad(c, c->wgrad[l], agent0, groups, st)) != GALA_OK) return r;
+            if (l > 0) {
+                if ((r = run_plan(c, c->dgrad[l], agent0, groups, 0, st)) != GALA_OK) return r;
+                const long ds = S * P[l] * kConvKK[l], as = B * P[l - 1] * kConvCout[l - 1],
+                           xs = S * P[l - 1] * kConvCout[l - 1];
+                LAUNCH(launch_col2im(c->dcols[l] + (long)agent0 * ds, ds, c->act[l - 1] + (long)agent0 * as, as,
+                                     c->dy[l - 1] + (long)agent0 * xs, xs, l, (int)S, groups, st));
+            }
+        }
+    } else {
+        const int H = c->H;
+        hb.H = H; hb.act = 2;
+        hb.h = c->h2 + (long)agent0 * B * H; hb.h_stride = B * H; hb.h_bf16 = 0;
+        hb.piw = c->ml.piw; hb.pib = c->ml.pib; hb.vw = c->ml.vw; hb.vb = c->ml.vb;
+        hb.dpre = c->dpre2 + (long)agent0 * S * H; hb.dpre_stride = S * H; hb.dpre_bf16 = 0;
+        LAUNCH(launch_heads_bwd(hb, groups, st));
+        c->launches++;
+        DenseBwdArgs d2{};
+        d2.rows = (int)S; d2.in_dim = H; d2.out_dim = H; d2.act_in = 2;
+        fill_batch(d2.in, c->h1, B * H * 4, agent0, groups);
+        d2.dpre = c->dpre2 + (long)agent0 * S * H; d2.dpre_stride = S * H;
+        d2.W = c->x + (long)agent0 * dp + c->ml.w2; d2.w_stride = dp;
+        d2.gW = c->g + (long)agent0 * dp + c->ml.w2; d2.gb = c->g + (long)agent0 * dp + c->ml.b2; d2.g_stride = dp;
+        d2.din = c->dpre1 + (long)agent0 * S * H; d2.din_stride = S * H;
+        LAUNCH(launch_dense_bwd(d2, groups, st));
+        c->launches++;
+        DenseBwdArgs d1{};
+        d1.rows = (int)S; d1.in_dim = c->obs_dim; d1.out_dim = H; d1.act_in = 0;
+        d1.in = obs;
+        d1.dpre = c->dpre1 + (long)agent0 * S * H; d1.dpre_stride = S * H;
+        d1.W = c->x + (long)agent0 * dp + c->ml.w1; d1.w_stride = dp;
+        d1.gW = c->g + (long)agent0 * dp + c->ml.w1; d1.gb = c->g + (long)agent0 * dp + c->ml.b1; d1.g_stride = dp;
+        d1.din = nullptr;
+        LAUNCH(launch_dense_bwd(d1, groups, st));
+    }
+    LAUNCH(launch_grad_norm(c->g, c->d, dp, agent0, groups, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
+                            c->norm, c->clip, st));
+    for (int i = 0; i < groups; i++) {
+        c->agents[agent0 + i].pending = true;
+        c->agents[agent0 + i].frames += S;
+    }
+    return GALA_OK;
+}
+
+// Newest snapshot version of agent j whose writing sweep has completed (0: none usable).
+long long usable_version(gala_ctx* c, int j) {
+    Agent& a = c->agents[j];
+    for (long long w = a.version; w > 0 && w >= a.version - 1; w--)
+        if (cudaEventQuery(a.pub_event[w & 1]) == cudaSuccess) return w;
+    return 0;
+}
+
+// Optimiser step + publication (+ conditional average) for one agent on its stream.
+int sweep_agent(gala_ctx* c, int i, bool try_mix) {
+    Agent& ag = c->agents[i];
+    const long dp = c->d_pad;
+    int off[2] = {0, 0};
+    int np = try_mix ? topo_offsets(c->topo, c->n, ag.round, off) : 0;
+    int peers[2] = {0, 0};
+    long long vers[2] = {0, 0};
+    bool fresh = np > 0;
+    for (int j = 0; j < np; j++) {
+        peers[j] = ((i - off[j]) % c->n + c->n) % c->n;
+        vers[j] = usable_version(c, peers[j]);
+        if (vers[j] <= ag.consumed[peers[j]]) fresh = false;
+    }
+    const long long w = ag.version + 1;
+    const int slot = (int)(w & 1);
+    // pairwise back-pressure: sweeps that still read the slot we are about to overwrite go first
+    for (int r : ag.slot_readers[slot]) CK(cudaStreamWaitEvent(ag.stream, c->agents[r].sweep_done, 0));
+    ag.slot_readers[slot].clear();
+    const float* p0 = nullptr;
+    const float* p1 = nullptr;
+    if (fresh) {
+        for (int j = 0; j < np; j++) {
+            Agent& pj = c->agents[peers[j]];
+            const float* ptr = c->snap + ((long)peers[j] * 2 + (vers[j] & 1)) * dp;
+            if (j == 0) p0 = ptr; else p1 = ptr;
+            pj.slot_readers[vers[j] & 1].push_back(i);
+            const long long stale = pj.version - vers[j];
+            ag.stale_sum += stale;
+            if (stale > ag.stale_max) ag.stale_max = stale;
+            ag.consumed[peers[j]] = vers[j];
+        }
+        ag.mixes++;
+    } else if (np > 0) {
+        ag.skipped++;
+    }
+    SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
+    LAUNCH(launch_sweep_agent(c->x + (long)i * dp, ag.pending ? c->g + (long)i * dp : nullptr, c->v + (long)i * dp,
+                              c->snap + ((long)i * 2 + slot) * dp, p0, p1, fresh ? np : 0, c->clip + i,
+                              c->conv ? c->shadow + (long)i * dp : nullptr, dp, hp, ag.stream));
+    CK(cudaEventRecord(ag.pub_event[slot], ag.stream));
+    CK(cudaEventRecord(ag.sweep_done, ag.stream));
+    ag.version = w;
+    ag.pending = false;
+    ag.last_n = np; ag.last_mixed = fresh ? 1 : 0;
+    for (int j = 0; j < 2; j++) { ag.last_peers[j] = peers[j]; ag.last_versions[j] = fresh ? vers[j] : 0; }
+    return GALA_OK;
+}
+
+int host_wait(gala_ctx* c, cudaStream_t st, int timeout_ms) {
+    if (timeout_ms < 0) {
+        CK(cudaStreamSynchronize(st));
+        return GALA_OK;
+    }
+    auto t0 = std::chrono::steady_clock::now();
+    for (;;) {
+        cudaError_t e = cudaStreamQuery(st);
+        if (e == cudaSuccess) return GALA_OK;
+        if (e != cudaErrorNotReady) return fail(c, GALA_ECUDA, "cudaStreamQuery: %s", cudaGetErrorString(e));
+        auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+        if (ms >= timeout_ms) return fail(c, GALA_ETIMEOUT, "work still running after %d ms", timeout_ms);
+        std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+}
+
+int check_error_word(gala_ctx* c) {
+    int w = 0;
+    CK(cudaMemcpy(&w, c->error_word, sizeof w, cudaMemcpyDeviceToHost));
+    if (w) {
+        int z = 0;
+        cudaMemcpy(c->error_word, &z, sizeof z, cudaMemcpyHostToDevice);
+        return fail(c, GALA_ECUDA, "a bounded device-side wait ran out (tensor-core pipeline)");
+    }
+    return GALA_OK;
+}
+
+bool valid_agent(const gala_ctx* c, int a) { return c && a >= 0 && a < c->n; }
+
+}  // namespace
+
+// ====================================================================== C ABI
+extern "C" {
+
+int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* net, const gala_hparams* hp,
+                gala_ctx** out) {
+    if (!out) return GALA_EINVAL;
+    *out = nullptr;
+    if (!topo || !net || !hp) return GALA_EINVAL;
+    if (n_agents < 1 || n_agents > 256) return GALA_EINVAL;
+    if (topo->kind != GALA_TOPO_RING && topo->kind != GALA_TOPO_EXP) return GALA_EINVAL;
+    if (topo->peers < 1 || topo->peers > 2) return GALA_EINVAL;
+    if (net->kind != GALA_NET_MLP && net->kind != GALA_NET_CONV) return GALA_EINVAL;
+    if (net->n_actions < 2 || net->n_actions > 32) return GALA_EINVAL;
+    if (hp->n_envs < 1 || hp->n_steps < 1 || hp->staleness_tau >= 0) return GALA_EINVAL;
+    if (!(hp->rms_eps > 0.0f) || !(hp->lr >= 0.0f) || hp->rms_alpha < 0.0f || hp->rms_alpha > 1.0f) return GALA_EINVAL;
+    if (net->kind == GALA_NET_MLP && (net->obs_dim < 1 || net->obs_dim > 4096 || net->hidden < 1 || net->hidden > 1024))
+        return GALA_EINVAL;
+    if (net->kind == GALA_NET_CONV && net->gemm_dtype != 1) return GALA_EINVAL;
+    if (net->kind == GALA_NET_MLP && net->gemm_dtype != 0) return GALA_EINVAL;
+
+    gala_ctx* c = new (std::nothrow) gala_ctx();
+    if (!c) return GALA_ENOMEM;
+    *out = c;  // handed out even on failure so that gala_last_error can explain; gala_destroy frees it
+    c->n = n_agents; c->topo = *topo; c->net = *net; c->hp = *hp;
+    c->conv = net->kind == GALA_NET_CONV;
+    c->T = hp->n_steps; c->E = hp->n_envs; c->A = net->n_actions;
+    c->B = (long)(c->T + 1) * c->E; c->S = (long)c->T * c->E;
+    const int A = c->A;
+    long off = 0;
+    if (c->conv) {
+        for (int l = 0; l < 3; l++) {
+            c->cl.w[l] = off; off += (long)kConvCout[l] * kConvKK[l];
+            c->cl.b[l] = off; off += kConvCout[l];
+        }
+        c->cl.fcw = off; off += (long)kHidden * kFeat;
+        c->cl.fcb = off; off += kHidden;
+        c->cl.piw = off; off += (long)A * kHidden;
+        c->cl.pib = off; off += A;
+        c->cl.vw = off; off += kHidden;
+        c->cl.vb = off; off += 1;
+        c->H = kHidden;
+    } else {
+        const int H = net->hidden, D = net->obs_dim;
+        c->H = H; c->obs_dim = D;
+        c->ml.w1 = off; off += (long)H * D;
+        c->ml.b1 = off; off += H;
+        c->ml.w2 = off; off += (long)H * H;
+        c->ml.b2 = off; off += H;
+        c->ml.piw = off; off += (long)A * H;
+        c->ml.pib = off; off += A;
+        c->ml.vw = off; off += H;
+        c->ml.vb = off; off += 1;
+    }
+    c->d = off;
+    c->d_pad = (off + 1023) / 1024 * 1024;
+    const long dp = c->d_pad, B = c->B, S = c->S;
+    const int n = c->n;
+
+    CK(cudaStreamCreateWithFlags(&c->main_stream, cudaStreamNonBlocking));
+    CK(cudaEventCreateWithFlags(&c->main_event, cudaEventDisableTiming));
+    c->agents.resize(n);
+    for (int i = 0; i < n; i++) {
+        Agent& a = c->agents[i];
+        CK(cudaStreamCreateWithFlags(&a.lib_stream, cudaStreamNonBlocking));
+        a.stream = a.lib_stream;
+        CK(cudaEventCreateWithFlags(&a.pub_event[0], cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&a.pub_event[1], cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&a.sweep_done, cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&a.fence, cudaEventDisableTiming));
+        a.consumed.assign(n, 0);
+    }
+    ALLOC(c->x, (size_t)n * dp); ALLOC(c->g, (size_t)n * dp); ALLOC(c->v, (size_t)n * dp);
+    ALLOC(c->snap, (size_t)n * 2 * dp);
+    ALLOC(c->clip, n); ALLOC(c->norm, n); ALLOC(c->losses, (size_t)n * 4);
+    ALLOC(c->norm_partial, (size_t)n * kNormChunks); ALLOC(c->norm_ticket, n);
+    ALLOC(c->error_word, 1);
+    ALLOC(c->logits, (size_t)n * B * A); ALLOC(c->values, (size_t)n * B);
+    ALLOC(c->returns, (size_t)n * S); ALLOC(c->adv, (size_t)n * S);
+    ALLOC(c->dlogits, (size_t)n * S * A); ALLOC(c->dvalues, (size_t)n * S);
+    {   // clip coefficients start at 1
+        std::vector<float> ones(n, 1.0f);
+        CK(cudaMemcpy(c->clip, ones.data(), n * sizeof(float), cudaMemcpyHostToDevice));
+    }
+    if (c->conv) {
+        const int P[3] = {400, 81, 49};
+        CK(gemm_init());
+        ALLOC(c->shadow, (size_t)n * dp);
+        ALLOC(c->colsum_partial, (size_t)n * kColsumChunks * 512); ALLOC(c->colsum_ticket, n);
+        for (int l = 0; l < 3; l++) {
+            ALLOC(c->cols[l], (size_t)n * B * P[l] * kConvKK[l]);
+            ALLOC(c->act[l], (size_t)n * B * P[l] * kConvCout[l]);
+            ALLOC(c->dy[l], (size_t)n * S * P[l] * kConvCout[l]);
+            if (l > 0) ALLOC(c->dcols[l], (size_t)n * S * P[l] * kConvKK[l]);
+        }
+        ALLOC(c->hid, (size_t)n * B * kHidden);
+        ALLOC(c->dh, (size_t)n * S * kHidden);
+        c->splitk_group_stride = (long)c->max_split * 64 * 576;
+        ALLOC(c->splitk_ws, (size_t)n * c->splitk_group_stride);
+        int r = build_plans(c);
+        if (r != GALA_OK) return r;
+    } else {
+        const int H = c->H;
+        ALLOC(c->h1, (size_t)n * B * H); ALLOC(c->h2, (size_t)n * B * H);
+        ALLOC(c->dpre1, (size_t)n * S * H); ALLOC(c->dpre2, (size_t)n * S * H);
+    }
+    // initial parameters: uniform(-1,1)/sqrt(fan_in), biases included
+    {
+        std::vector<float> host((size_t)dp, 0.0f);
+        for (int i = 0; i < n; i++) {
+            const uint64_t ag = hp->identical_init ? 0 : (uint64_t)i;
+            if (i == 0 || !hp->identical_init) {
+                if (c->conv) {
+                    for (int l = 0; l < 3; l++) {
+                        init_tensor(host.data(), c->cl.w[l], (long)kConvCout[l] * kConvKK[l], kConvKK[l], hp->seed, ag);
+                        init_tensor(host.data(), c->cl.b[l], kConvCout[l], kConvKK[l], hp->seed, ag);
+                    }
+                    init_tensor(host.data(), c->cl.fcw, (long)kHidden * kFeat, kFeat, hp->seed, ag);
+                    init_tensor(host.data(), c->cl.fcb, kHidden, kFeat, hp->seed, ag);
+                    init_tensor(host.data(), c->cl.piw, (long)A * kHidden, kHidden, hp->seed, ag);
+                    init_tensor(host.data(), c->cl.pib, A, kHidden, hp->seed, ag);
+                    init_tensor(host.data(), c->cl.vw, kHidden, kHidden, hp->seed, ag);
+                    init_tensor(host.data(), c->cl.vb, 1, kHidden, hp->seed, ag);
+                } else {
+                    const int H = c->H, D = c->obs_dim;
+                    init_tensor(host.data(), c->ml.w1, (long)H * D, D, hp->seed, ag);
+                    init_tensor(host.data(), c->ml.b1, H, D, hp->seed, ag);
+                    init_tensor(host.data(), c->ml.w2, (long)H * H, H, hp->seed, ag);
+                    init_tensor(host.data(), c->ml.b2, H, H, hp->seed, ag);
+                    init_tensor(host.data(), c->ml.piw, (long)A * H, H, hp->seed, ag);
+                    init_tensor(host.data(), c->ml.pib, A, H, hp->seed, ag);
+                    init_tensor(host.data(), c->ml.vw, H, H, hp->seed, ag);
+                    init_tensor(host.data(), c->ml.vb, 1, H, hp->seed, ag);
+                }
+            }
+            CK(cudaMemcpy(c->x + (long)i * dp, host.data(), dp * sizeof(float), cudaMemcpyHostToDevice));
+        }
+        if (c->conv) {
+            LAUNCH(launch_cast_bf16(c->x, c->shadow, (long)n * dp, c->main_stream));
+            CK(cudaStreamSynchronize(c->main_stream));
+        }
+    }
+    CK(cudaDeviceSynchronize());
+    return GALA_OK;
+}
+
+int gala_destroy(gala_ctx* c) {
+    if (!c) return GALA_EINVAL;
+    cudaDeviceSynchronize();
+    for (Agent& a : c->agents) {
+        if (a.lib_stream) cudaStreamDestroy(a.lib_stream);
+        for (int s = 0; s < 2; s++) if (a.pub_event[s]) cudaEventDestroy(a.pub_event[s]);
+        if (a.sweep_done) cudaEventDestroy(a.sweep_done);
+        if (a.fence) cudaEventDestroy(a.fence);
+    }
+    if (c->main_stream) cudaStreamDestroy(c->main_stream);
+    if (c->main_event) cudaEventDestroy(c->main_event);
+    for (void* p : c->allocs) cudaFree(p);
+    delete c;
+    return GALA_OK;
+}
+
+int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int* actions, float* values) {
+    if (!valid_agent(c, agent) || !obs) return fail(c, GALA_EINVAL, "gala_act: bad agent or null obs");
+    if (actions && !uniforms) return fail(c, GALA_EINVAL, "gala_act: actions requested without uniforms");
+    Agent& ag = c->agents[agent];
+    PtrBatch pb{};
+    pb.p[0] = obs;
+    int r = forward(c, agent, 1, pb, c->E, ag.stream);
+    if (r != GALA_OK) return r;
+    if (actions)
+        LAUNCH(launch_sample(c->logits + (long)agent * c->B * c->A, uniforms, actions, c->E, c->A, ag.stream));
+    if (values)
+        CK(cudaMemcpyAsync(values, c->values + (long)agent * c->B, c->E * sizeof(float), cudaMemcpyDeviceToDevice,
+                           ag.stream));
+    return GALA_OK;
+}
+
+int gala_learn(gala_ctx* c, int agent, const gala_rollout* ro) {
+    if (!valid_agent(c, agent) || !ro || !ro->obs || !ro->actions || !ro->rewards || !ro->dones)
+        return fail(c, GALA_EINVAL, "gala_learn: bad agent or null rollout pointer");
+    Agent& ag = c->agents[agent];
+    if (ag.pending) {  // apply the earlier gradient without mixing, publish
+        int r = sweep_agent(c, agent, false);
+        if (r != GALA_OK) return r;
+        ag.round++;
+    }
+    return learn_range(c, agent, 1, ro, ag.stream);
+}
+
+int gala_gossip(gala_ctx* c, int agent) {
+    if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_gossip: bad agent");
+    int r = sweep_agent(c, agent, true);
+    if (r != GALA_OK) return r;
+    c->agents[agent].round++;
+    return GALA_OK;
+}
+
+int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
+    if (!c) return GALA_EINVAL;
+    const int n = c->n;
+    if (ros)
+        for (int i = 0; i < n; i++)
+            if (!ros[i].obs || !ros[i].actions || !ros[i].rewards || !ros[i].dones)
+                return fail(c, GALA_EINVAL, "gala_step_sync: null rollout pointer for agent %d", i);
+    cudaStream_t st = c->main_stream;
+    for (int i = 0; i < n; i++) {  // everything the agents have enqueued goes first
+        CK(cudaEventRecord(c->agents[i].fence, c->agents[i].stream));
+        CK(cudaStreamWaitEvent(st, c->agents[i].fence, 0));
+    }
+    if (ros) {
+        for (int a0 = 0; a0 < n; a0 += kBatch) {
+            const int cnt = n - a0 < kBatch ? n - a0 : kBatch;
+            int r = learn_range(c, a0, cnt, ros + a0, st);
+            if (r != GALA_OK) return r;
+        }
+    }
+    int off[2] = {0, 0};
+    const int np = topo_offsets(c->topo, n, c->sync_round, off);
+    SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
+    LAUNCH(launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp, st));
+    CK(cudaEventRecord(c->main_event, st));
+    for (int i = 0; i < n; i++) {
+        CK(cudaStreamWaitEvent(c->agents[i].stream, c->main_event, 0));
+        c->agents[i].pending = false;
+        c->agents[i].round++;
+    }
+    c->sync_round++;
+    return GALA_OK;
+}
+
+int gala_sync_agent(gala_ctx* c, int agent, int timeout_ms) {
+    if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_sync_agent: bad agent");
+    int r = host_wait(c, c->agents[agent].stream, timeout_ms);
+    if (r != GALA_OK) return r;
+    return check_error_word(c);
+}
+
+int gala_sync_all(gala_ctx* c, int timeout_ms) {
+    if (!c) return GALA_EINVAL;
+    int r = host_wait(c, c->main_stream, timeout_ms);
+    if (r != GALA_OK) return r;
+    for (int i = 0; i < c->n; i++)
+        if ((r = host_wait(c, c->agents[i].stream, timeout_ms)) != GALA_OK) return r;
+    return check_error_word(c);
+}
+
+int gala_in_peers(const gala_ctx* c, long long round, int agent, int* peers, int* n) {
+    if (!valid_agent(c, agent) || !peers || !n || round < 0) return GALA_EINVAL;
+    int off[2];
+    const int np = topo_offsets(c->topo, c->n, round, off);
+    for (int j = 0; j < np; j++) peers[j] = ((agent - off[j]) % c->n + c->n) % c->n;
+    *n = np;
+    return GALA_OK;
+}
+
+int gala_get_state(gala_ctx* c, int agent, float* params, float* sq_avg, float* grad, long long* round) {
+    if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_get_state: bad agent");
+    CK(cudaStreamSynchronize(c->main_stream));
+    CK(cudaStreamSynchronize(c->agents[agent].stream));
+    const size_t bytes = (size_t)c->d * sizeof(float);
+    if (params) CK(cudaMemcpy(params, c->x + (long)agent * c->d_pad, bytes, cudaMemcpyDefault));
+    if (sq_avg) CK(cudaMemcpy(sq_avg, c->v + (long)agent * c->d_pad, bytes, cudaMemcpyDefault));
+    if (grad) CK(cudaMemcpy(grad, c->g + (long)agent * c->d_pad, bytes, cudaMemcpyDefault));
+    if (round) *round = c->agents[agent].round;
+    return check_error_word(c);
+}
+
+int gala_set_state(gala_ctx* c, int agent, const float* params, const float* sq_avg, long long round) {
+    if (!valid_agent(c, agent) || round < 0) return fail(c, GALA_EINVAL, "gala_set_state: bad agent or round");
+    Agent& ag = c->agents[agent];
+    CK(cudaStreamSynchronize(c->main_stream));
+    CK(cudaStreamSynchronize(ag.stream));
+    const size_t bytes = (size_t)c->d * sizeof(float);
+    if (params) {
+        CK(cudaMemcpy(c->x + (long)agent * c->d_pad, params, bytes, cudaMemcpyDefault));
+        if (c->conv) {
+            LAUNCH(launch_cast_bf16(c->x + (long)agent * c->d_pad, c->shadow + (long)agent * c->d_pad, c->d_pad, ag.stream));
+            CK(cudaStreamSynchronize(ag.stream));
+        }
+    }
+    if (sq_avg) CK(cudaMemcpy(c->v + (long)agent * c->d_pad, sq_avg, bytes, cudaMemcpyDefault));
+    ag.round = round;
+    if (agent == 0) c->sync_round = round;
+    return GALA_OK;
+}
+
+int gala_set_grad(gala_ctx* c, int agent, const float* grad, float clip_coef) {
+    if (!valid_agent(c, agent) || !grad) return fail(c, GALA_EINVAL, "gala_set_grad: bad agent or null gradient");
+    Agent& ag = c->agents[agent];
+    CK(cudaStreamSynchronize(c->main_stream));
+    CK(cudaStreamSynchronize(ag.stream));
+    CK(cudaMemcpy(c->g + (long)agent * c->d_pad, grad, (size_t)c->d * sizeof(float), cudaMemcpyDefault));
+    if (clip_coef >= 0.0f) {
+        CK(cudaMemcpy(c->clip + agent, &clip_coef, sizeof(float), cudaMemcpyHostToDevice));
+    } else {
+        LAUNCH(launch_grad_norm(c->g, c->d, c->d_pad, agent, 1, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
+                                c->norm, c->clip, ag.stream));
+        CK(cudaStreamSynchronize(ag.stream));
+    }
+    ag.pending = true;
+    return GALA_OK;
+}
+
+int gala_param_count(const gala_ctx* c, long long* d, long long* d_padded) {
+    if (!c) return GALA_EINVAL;
+    if (d) *d = c->d;
+    if (d_padded) *d_padded = c->d_pad;
+    return GALA_OK;
+}
+
+int gala_losses(gala_ctx* c, int agent, float out[4]) {
+    if (!valid_agent(c, agent) || !out) return fail(c, GALA_EINVAL, "gala_losses: bad argument");
+    CK(cudaStreamSynchronize(c->main_stream));
+    CK(cudaStreamSynchronize(c->agents[agent].stream));
+    CK(cudaMemcpy(out, c->losses + (long)agent * 4, 3 * sizeof(float), cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(out + 3, c->norm + agent, sizeof(float), cudaMemcpyDeviceToHost));
+    return GALA_OK;
+}
+
+int gala_stats(gala_ctx* c, int agent, long long out[8]) {
+    if (!valid_agent(c, agent) || !out) return GALA_EINVAL;
+    const Agent& a = c->agents[agent];
+    out[0] = a.frames; out[1] = a.round; out[2] = a.mixes; out[3] = a.skipped;
+    out[4] = a.stale_sum; out[5] = a.stale_max; out[6] = a.version; out[7] = 0;
+    return GALA_OK;
+}
+
+int gala_last_mix(gala_ctx* c, int agent, int* peers, long long* versions, int* n, int* mixed) {
+    if (!valid_agent(c, agent)) return GALA_EINVAL;
+    const Agent& a = c->agents[agent];
+    for (int j = 0; j < a.last_n; j++) {
+        if (peers) peers[j] = a.last_peers[j];
+        if (versions) versions[j] = a.last_versions[j];
+    }
+    if (n) *n = a.last_n;
+    if (mixed) *mixed = a.last_mixed;
+    return GALA_OK;
+}
+
+int gala_get_snapshot(gala_ctx* c, int agent, long long version, float* out) {
+    if (!valid_agent(c, agent) || !out) return fail(c, GALA_EINVAL, "gala_get_snapshot: bad argument");
+    Agent& a = c->agents[agent];
+    if (version < 1 || version > a.version || version < a.version - 1)
+        return fail(c, GALA_ESTATE, "snapshot version %lld of agent %d is not held (newest %lld)", version, agent,
+                    a.version);
+    CK(cudaStreamSynchronize(a.stream));
+    CK(cudaMemcpy(out, c->snap + ((long)agent * 2 + (version & 1)) * c->d_pad, (size_t)c->d * sizeof(float),
+                  cudaMemcpyDefault));
+    return GALA_OK;
+}
+
+int gala_set_stream(gala_ctx* c, int agent, void* cuda_stream) {
+    if (!valid_agent(c, agent)) return GALA_EINVAL;
+    Agent& a = c->agents[agent];
+    CK(cudaStreamSynchronize(a.stream));
+    a.stream = cuda_stream ? reinterpret_cast<cudaStream_t>(cuda_stream) : a.lib_stream;
+    return GALA_OK;
+}
+
+int gala_debug_read(gala_ctx* c, int agent, int what, float* out, long long count) {
+    if (!valid_agent(c, agent) || !out || count < 0) return fail(c, GALA_EINVAL, "gala_debug_read: bad argument");
+    CK(cudaStreamSynchronize(c->main_stream));
+    CK(cudaStreamSynchronize(c->agents[agent].stream));
+    const long B = c->B, S = c->S;
+    const int A = c->A;
+    const float* src = nullptr;
+    long avail = 0;
+    switch (what) {
+        case 0: src = c->logits + (long)agent * B * A; avail = B * A; break;
+        case 1: src = c->values + (long)agent * B; avail = B; break;
+        case 2: src = c->returns + (long)agent * S; avail = S; break;
+        case 3: src = c->adv + (long)agent * S; avail = S; break;
+        case 4: src = c->dlogits + (long)agent * S * A; avail = S * A; break;
+        case 5: src = c->dvalues + (long)agent * S; avail = S; break;
+        default: break;
+    }
+    if (src) {
+        if (count > avail) return fail(c, GALA_EINVAL, "gala_debug_read: count %lld > %ld", count, avail);
+        CK(cudaMemcpy(out, src, (size_t)count * sizeof(float), cudaMemcpyDefault));
+        return GALA_OK;
+    }
+    if (what >= 10 && what <= 13) {
+        const int l = what - 10;
+        const void* p = nullptr;
+        bool bf = false;
+        if (c->conv) {
+            const int P[3] = {400, 81, 49};
+            bf = true;
+            if (l < 3) { p = c->act[l] + (long)agent * B * P[l] * kConvCout[l]; avail = B * P[l] * kConvCout[l]; }
+            else { p = c->hid + (long)agent * B * kHidden; avail = B * kHidden; }
+        } else {
+            if (l == 0) p = c->h1 + (long)agent * B * c->H;
+            else if (l == 1) p = c->h2 + (long)agent * B * c->H;
+            avail = B * c->H;
+        }
+        if (!p) return fail(c, GALA_EINVAL, "gala_debug_read: no such layer");
+        if (count > avail) return fail(c, GALA_EINVAL, "gala_debug_read: count %lld > %ld", count, avail);
+        if (!bf) {
+            CK(cudaMemcpy(out, p, (size_t)count * sizeof(float), cudaMemcpyDefault));
+            return GALA_OK;
+        }
+        std::vector<__nv_bfloat16> tmp((size_t)count);
+        CK(cudaMemcpy(tmp.data(), p, (size_t)count * 2, cudaMemcpyDeviceToHost));
+        std::vector<float> f((size_t)count);
+        for (long long i = 0; i < count; i++) f[i] = __bfloat162float(tmp[i]);
+        CK(cudaMemcpy(out, f.data(), (size_t)count * sizeof(float), cudaMemcpyDefault));
+        return GALA_OK;
+    }
+    return fail(c, GALA_EINVAL, "gala_debug_read: unknown selector %d", what);
+}
+
+long long gala_launch_count(const gala_ctx* c) { return c ? c->launches : 0; }
+
+const char* gala_last_error(const gala_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+int gala_gemm_bf16(const void* A, const void* B, float* D, int groups, int M, int N, int K, int a_mn, int b_mn,
+                   int split_k, void* stream) {
+    if (!A || !B || !D || groups < 1 || M < 1 || N < 1 || K < 1 || split_k < 1) return GALA_EINVAL;
+    if ((K % 8) || (a_mn && (M % 8)) || (b_mn && (N % 8))) return GALA_EINVAL;
+    if (gemm_init() != cudaSuccess) return GALA_ECUDA;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int bn = b_mn ? (N > 64 ? 128 : 64) : (N > 64 ? 128 : (N > 32 ? 64 : 32));
+    GemmOperand oa, ob;
+    if (!make_operand(&oa, A, a_mn, M, K, groups, a_mn ? M : K, (uint64_t)M * K, 128)) return GALA_ECUDA;
+    if (!make_operand(&ob, B, b_mn, N, K, groups, b_mn ? N : K, (uint64_t)N * K, bn)) return GALA_ECUDA;
+    int* err = nullptr;
+    if (cudaMalloc(&err, sizeof(int)) != cudaSuccess) return GALA_ENOMEM;
+    cudaMemsetAsync(err, 0, sizeof(int), st);
+    GemmArgs a;
+    memset(&a, 0, sizeof a);
+    a.M = M; a.N = N; a.K = K; a.block_n = bn; a.groups = groups; a.split_k = split_k; a.scale = 1.0f;
+    a.ldc = N; a.error_word = err;
+    int rc = GALA_OK;
+    float* ws = nullptr;
+    const long count = (long)M * N;
+    if (split_k == 1) {
+        a.out = D; a.out_group_stride = count;
+        if (launch_gemm(oa, ob, a, st) != cudaSuccess) rc = GALA_ECUDA;
+    } else {
+        if (cudaMalloc(&ws, (size_t)groups * split_k * count * sizeof(float)) != cudaSuccess) { cudaFree(err); return GALA_ENOMEM; }
+        a.out = ws; a.out_group_stride = (long)split_k * count; a.out_split_stride = count;
+        if (launch_gemm(oa, ob, a, st) != cudaSuccess) rc = GALA_ECUDA;
+        if (rc == GALA_OK &&
+            launch_splitk_reduce(ws, D, count, split_k, count, groups, (long)split_k * count, count, st) != cudaSuccess)
+            rc = GALA_ECUDA;
+    }
+    // scratch (error word, split-K partials) is released here, so this entry point waits for its work
+    if (cudaStreamSynchronize(st) != cudaSuccess) rc = GALA_ECUDA;
+    int w = 0;
+    if (cudaMemcpy(&w, err, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess || w) rc = GALA_ECUDA;
+    cudaFree(err);
+    if (ws) cudaFree(ws);
+    return rc;
+}
+
+int gala_sweep_sync(float* x, const float* g, float* v, const float* clip, int n_agents, long long d_padded,
+                    const gala_topology* topo, long long round, const gala_hparams* hp, void* stream) {
+    if (!x || !g || !v || !topo || !hp || n_agents < 1 || d_padded < 4 || (d_padded % 4) || round < 0) return GALA_EINVAL;
+    if (topo->kind != GALA_TOPO_RING && topo->kind != GALA_TOPO_EXP) return GALA_EINVAL;
+    if (topo->peers < 1 || topo->peers > 2) return GALA_EINVAL;
+    int off[2] = {0, 0};
+    const int np = topo_offsets(*topo, n_agents, round, off);
+    SweepHp s{hp->lr, hp->rms_alpha, hp->rms_eps};
+    cudaError_t e = launch_sweep_sync(x, g, v, clip, nullptr, n_agents, d_padded, np, off, s,
+                                      reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GALA_OK : GALA_ECUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,392 @@
+// Grouped bf16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a.
+//
+//   D[g] (M x N, fp32 accumulate) = A[g] (M x K) * B[g] (N x K)^T       g = group (agent)
+//
+// Either operand may be stored K-contiguous ("K-major": [rows][K]) or M/N-contiguous
+// ("MN-major": [K][rows]); the four combinations cover forward (both K-major), data-gradient
+// (B MN-major) and weight-gradient (both MN-major) products of the conv / dense layers without
+// any transposed copy in global memory.
+//
+// Structure of one CTA (192 threads, one 128 x block_n output tile, one K range):
+//   warp 0   : TMA producer - cp.async.bulk.tensor (3-D maps: inner, rows, group) into a ring of
+//              128-byte-swizzled shared-memory stages, completion on mbarriers
+//   warp 1   : allocates tensor memory, issues tcgen05.mma (one elected thread), releases stages
+//              with tcgen05.commit
+//   warps 2-5: epilogue - tcgen05.ld the fp32 accumulator out of tensor memory (each warp its
+//              own 32-lane quarter), apply scale / bias / ReLU / mask, store
+// Every mbarrier wait is bounded: when a wait runs out the CTA raises an abort flag, sets the
+// caller's error word, drains what it has in flight, frees its tensor memory and returns.
+#include "internal.h"
+
+namespace gala {
+
+constexpr int BM = 128;          // tile rows (UMMA M)
+constexpr int BK = 64;           // K per stage = one 128-byte swizzle atom of bf16
+constexpr int kStages = 4;
+constexpr int kStageA = BM * BK * 2;    // 16 KiB
+constexpr int kStageB = 128 * BK * 2;   // room for block_n = 128
+constexpr int kSmemBytes = kStages * (kStageA + kStageB) + 1024;  // + alignment slack
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises *abort_flag) if the phase did not complete in time
+// or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; i++) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 32) __nanosleep(i < 4096 ? 32 : 256);
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                            int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.
+//   bits [0,14) start address >> 4      bits [16,30) leading byte offset >> 4
+//   bits [32,46) stride byte offset >> 4  bits [46,48) version (1 on sm_100)
+//   bits [61,64) layout type (2 = 128-byte swizzle)
+// K-major tile: rows are 128 B apart, groups of 8 rows 1024 B apart (stride offset); the leading
+//   offset is not used by swizzled K-major layouts.
+// MN-major tile: 64 contiguous M/N elements per 128-B row, 8 K-rows form a 1024-B group (stride
+//   offset), the next 64 M/N elements start one whole 64-row box later (leading offset, 8192 B).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int mn_major) {
+    const uint64_t lbo = mn_major ? (8192u >> 4) : 1u;
+    const uint64_t sbo = 1024u >> 4;
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B.
+__device__ __forceinline__ uint32_t make_instr_desc(int block_n, int a_mn, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ------------------------------------------------------------------ kernel
+__global__ void __launch_bounds__(192, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const GemmArgs p, const int a_mn, const int b_mn) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kStages];
+    __shared__ __align__(8) uint64_t empty_bar[kStages];
+    __shared__ __align__(8) uint64_t accum_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int issued_iters;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smA = smem;
+    uint8_t* smB = smem + kStages * kStageA;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int BN = p.block_n;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const int gz = blockIdx.z / p.split_k, split = blockIdx.z % p.split_k;
+    const int group = p.group0 + gz;
+    const int k_tiles = (p.K + BK - 1) / BK;
+    const int per_split = (k_tiles + p.split_k - 1) / p.split_k;
+    const int kt_begin = split * per_split;
+    const int kt_end = min(k_tiles, kt_begin + per_split);
+    const int num_k = max(0, kt_end - kt_begin);
+    const uint32_t tmem_cols = BN < 32 ? 32u : (uint32_t)BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&accum_bar, 1);
+        abort_flag = 0;
+        issued_iters = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_acc = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t bytes = (uint32_t)kStageA + (uint32_t)BN * BK * 2;
+            for (int it = 0; it < num_k; it++) {
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) break;
+                mbar_expect_tx(&full_bar[s], bytes);
+                const int k0 = (kt_begin + it) * BK;
+                uint8_t* a = smA + s * kStageA;
+                uint8_t* b = smB + s * kStageB;
+                if (!a_mn) {
+                    tma_load_3d(a, &tmA, &full_bar[s], k0, m0, group);
+                } else {
+                    tma_load_3d(a, &tmA, &full_bar[s], m0, k0, group);
+                    tma_load_3d(a + 8192, &tmA, &full_bar[s], m0 + 64, k0, group);
+                }
+                if (!b_mn) {
+                    tma_load_3d(b, &tmB, &full_bar[s], k0, n0, group);
+                } else {
+                    for (int j = 0; j < BN / 64; j++)
+                        tma_load_3d(b + j * 8192, &tmB, &full_bar[s], n0 + 64 * j, k0, group);
+                }
+                issued_iters = it + 1;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_instr_desc(BN, a_mn, b_mn);
+            bool ok = true;
+            for (int it = 0; it < num_k; it++) {
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint32_t a_addr = smem_u32(smA + s * kStageA);
+                const uint32_t b_addr = smem_u32(smB + s * kStageB);
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; kk++) {
+                    // one UMMA consumes K = 16: 32 B along a K-major row, 16 rows (2048 B) of an MN-major tile
+                    const uint64_t ad = make_smem_desc(a_addr + (a_mn ? kk * 2048 : kk * 32), a_mn);
+                    const uint64_t bd = make_smem_desc(b_addr + (b_mn ? kk * 2048 : kk * 32), b_mn);
+                    umma_bf16(tmem_acc, ad, bd, idesc, (it | kk) != 0 ? 1u : 0u);
+                }
+                umma_commit(&empty_bar[s]);
+            }
+            if (ok && num_k > 0) umma_commit(&accum_bar);
+        }
+    } else {
+        // epilogue warps 2..5 -> tensor-memory lane quarters 2,3,0,1
+        const int q = warp & 3;
+        const int m = m0 + q * 32 + lane;
+        bool have = true;
+        if (num_k > 0) {
+            have = mbar_wait(&accum_bar, 0, &abort_flag);
+            tcgen05_fence_after();
+        }
+        if (have) {
+            const bool out_bf16 = p.flags & EPI_OUT_BF16, relu = p.flags & EPI_RELU;
+            const bool transpose = p.flags & EPI_TRANSPOSE, use_mask = p.flags & EPI_MASK;
+            const long obase = (long)gz * p.out_group_stride + (long)split * p.out_split_stride;
+            const float* bias = p.bias ? p.bias + (long)group * p.bias_group_stride : nullptr;
+            const __nv_bfloat16* mask = use_mask ? p.mask + (long)gz * p.mask_group_stride : nullptr;
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                if (num_k > 0) {
+                    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; j++) r[j] = 0u;
+                }
+                const int nb = n0 + c0;
+                if (m >= p.M || nb >= p.N) continue;
+                float vals[32];
+#pragma unroll
+                for (int j = 0; j < 32; j++) {
+                    float v = __uint_as_float(r[j]) * p.scale;
+                    if (bias && nb + j < p.N) v += __ldg(bias + nb + j);
+                    if (relu) v = fmaxf(v, 0.0f);
+                    vals[j] = v;
+                }
+                const bool full = nb + 32 <= p.N;
+                if (!transpose) {
+                    const long row_off = obase + (long)m * p.ldc + nb;
+                    if (use_mask) {
+                        for (int j = 0; j < 32 && nb + j < p.N; j++)
+                            if (!(__bfloat162float(mask[(long)m * p.ldc + nb + j]) > 0.0f)) vals[j] = 0.0f;
+                    }
+                    if (out_bf16) {
+                        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off;
+                        if (full && (reinterpret_cast<uintptr_t>(o) & 15) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                __nv_bfloat162 h0 = __floats2bfloat162_rn(vals[j], vals[j + 1]);
+                                __nv_bfloat162 h1 = __floats2bfloat162_rn(vals[j + 2], vals[j + 3]);
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(vals[j + 4], vals[j + 5]);
+                                __nv_bfloat162 h3 = __floats2bfloat162_rn(vals[j + 6], vals[j + 7]);
+                                uint4 u;
+                                u.x = *reinterpret_cast<uint32_t*>(&h0); u.y = *reinterpret_cast<uint32_t*>(&h1);
+                                u.z = *reinterpret_cast<uint32_t*>(&h2); u.w = *reinterpret_cast<uint32_t*>(&h3);
+                                *reinterpret_cast<uint4*>(o + j) = u;
+                            }
+                        } else {
+                            for (int j = 0; j < 32 && nb + j < p.N; j++) o[j] = __float2bfloat16_rn(vals[j]);
+                        }
+                    } else {
+                        float* o = reinterpret_cast<float*>(p.out) + row_off;
+                        if (full && (reinterpret_cast<uintptr_t>(o) & 15) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(o + j) = make_float4(vals[j], vals[j + 1], vals[j + 2], vals[j + 3]);
+                        } else {
+                            for (int j = 0; j < 32 && nb + j < p.N; j++) o[j] = vals[j];
+                        }
+                    }
+                } else {
+                    // D[m][n] -> out[n * ldc + m]: consecutive lanes write consecutive addresses
+                    if (out_bf16) {
+                        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + obase + m;
+                        for (int j = 0; j < 32 && nb + j < p.N; j++) o[(long)(nb + j) * p.ldc] = __float2bfloat16_rn(vals[j]);
+                    } else {
+                        float* o = reinterpret_cast<float*>(p.out) + obase + m;
+#pragma unroll
+                        for (int j = 0; j < 32; j++)
+                            if (nb + j < p.N) o[(long)(nb + j) * p.ldc] = vals[j];
+                    }
+                }
+            }
+        }
+    }
+
+    // teardown
+    tcgen05_fence_before();
+    __syncthreads();
+    if (abort_flag) {
+        if (threadIdx.x == 0) {
+            if (p.error_word) atomicExch(p.error_word, 1);
+            // let copies that were already issued land before the shared memory goes away
+            const int issued = issued_iters;
+            for (int it = max(0, issued - kStages); it < issued; it++) {
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                for (uint32_t i = 0; i < (1u << 16); i++) {
+                    if (mbar_try_wait(&full_bar[s], ph)) break;
+                    __nanosleep(64);
+                }
+            }
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ split-K reduction
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partials, float* __restrict__ out,
+                                                            long count, int split_k, long split_stride,
+                                                            long partial_group_stride, long out_group_stride) {
+    const int g = blockIdx.y;
+    const float* pg = partials + (long)g * partial_group_stride;
+    float* og = out + (long)g * out_group_stride;
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < count; i += (long)gridDim.x * blockDim.x) {
+        float acc = pg[i];
+        for (int s = 1; s < split_k; s++) acc += pg[(long)s * split_stride + i];  // fixed order
+        og[i] = acc;
+    }
+}
+cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, int split_k, long split_stride,
+                                 int groups, long partial_group_stride, long out_group_stride, cudaStream_t st) {
+    int bx = (int)((count + 255) / 256);
+    if (bx > 148 * 4) bx = 148 * 4;
+    splitk_reduce_kernel<<<dim3(bx, groups), 256, 0, st>>>(partials, out, count, split_k, split_stride,
+                                                           partial_group_stride, out_group_stride);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+cudaError_t gemm_init() {
+    if (g_encode) return cudaSuccess;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t groups,
+                     uint64_t row_stride_bytes, uint64_t group_stride_bytes, uint32_t box_cols, uint32_t box_rows) {
+    if (!g_encode) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15) || (row_stride_bytes & 15) || (group_stride_bytes & 15)) return false;
+    if (groups == 0) groups = 1;
+    if (group_stride_bytes == 0) group_stride_bytes = rows * row_stride_bytes;
+    cuuint64_t dims[3] = {cols, rows, groups};
+    cuuint64_t strides[2] = {row_stride_bytes, group_stride_bytes};
+    cuuint32_t box[3] = {box_cols, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
+                  uint64_t groups, uint64_t ld_elems, uint64_t group_stride_elems, int tile_mn) {
+    op->mn_major = mn_major;
+    if (!mn_major)
+        return make_tensor_map(&op->map, base, k_extent, mn_extent, groups, ld_elems * 2, group_stride_elems * 2, BK,
+                               (uint32_t)tile_mn);
+    return make_tensor_map(&op->map, base, mn_extent, k_extent, groups, ld_elems * 2, group_stride_elems * 2, 64, BK);
+}
+
+cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, cudaStream_t st) {
+    if (args.block_n != 32 && args.block_n != 64 && args.block_n != 128) return cudaErrorInvalidValue;
+    if (B.mn_major && args.block_n < 64) return cudaErrorInvalidValue;
+    if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
+    dim3 grid((args.M + BM - 1) / BM, (args.N + args.block_n - 1) / args.block_n, args.groups * args.split_k);
+    gemm_tcgen05_kernel<<<grid, 192, kSmemBytes, st>>>(A.map, B.map, args, A.mn_major, B.mn_major);
+    return cudaGetLastError();
+}
+
+}  // namespace gala

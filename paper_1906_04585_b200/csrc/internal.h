@@ -1,0 +1,183 @@
+// Internal declarations shared by the CUDA sources of the GALA learner library.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "gala.h"
+
+namespace gala {
+
+// ---------------------------------------------------------------- network layout
+// Offsets (in floats) of every tensor inside one agent's flat vector.
+struct ConvLayout {
+    long w[3], b[3];      // conv1..3
+    long fcw, fcb;        // hidden layer 3136 -> 512
+    long piw, pib, vw, vb;
+};
+struct MlpLayout {
+    long w1, b1, w2, b2;
+    long piw, pib, vw, vb;
+};
+
+// Fixed geometry of the conv trunk (Appendix C.2 network at 84x84x4).
+constexpr int kFrameH = 84, kFrameW = 84, kFrameC = 4;
+constexpr int kConvK[3] = {8, 4, 3};
+constexpr int kConvS[3] = {4, 2, 1};
+constexpr int kConvCin[3] = {4, 32, 64};
+constexpr int kConvCout[3] = {32, 64, 64};
+constexpr int kConvIn[3] = {84, 20, 9};    // input height = width
+constexpr int kConvOut[3] = {20, 9, 7};    // output height = width
+constexpr int kConvKK[3] = {256, 512, 576};  // k*k*cin
+constexpr int kFeat = 3136, kHidden = 512;
+
+// ---------------------------------------------------------------- GEMM
+// One operand of the grouped tensor-core GEMM, as a TMA descriptor plus what
+// the kernel must know about its shared-memory image.
+struct GemmOperand {
+    CUtensorMap map;
+    int mn_major;  // 0: stored [rows = M or N][K]; 1: stored [K][M or N]
+};
+
+enum EpilogueFlags : int {
+    EPI_OUT_BF16 = 1,    // store bf16 (else fp32)
+    EPI_RELU = 2,        // max(.,0) after scale and bias
+    EPI_TRANSPOSE = 4,   // store D[m][n] at out[n*ldc + m]
+    EPI_MASK = 8         // multiply by (mask[m][n] > 0), mask bf16 with the output's layout
+};
+
+struct GemmArgs {
+    int M, N, K;           // valid extents of one group's product
+    int block_n;           // 32, 64 or 128
+    int groups;            // grid.z = groups * split_k
+    int group0;            // first group index (added to the TMA group coordinate)
+    int split_k;
+    int flags;
+    float scale;           // applied to the accumulator before the bias
+    const float* bias;     // per-column (n) bias, may be null; indexed by group with bias_group_stride
+    long bias_group_stride;
+    void* out;             // group g, split s at out + g*out_group_stride + s*out_split_stride (elements)
+    long out_group_stride;
+    long out_split_stride;
+    long ldc;
+    const __nv_bfloat16* mask;  // [m][n] with the output's ldc; group g at mask + g*mask_group_stride
+    long mask_group_stride;
+    int* error_word;       // device int, set non-zero when a bounded wait runs out
+};
+
+cudaError_t gemm_init();   // resolves the driver entry point used to build TMA descriptors
+// rows x cols bf16 matrix per group, cols contiguous.  box_rows x box_cols tile.
+bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t groups,
+                     uint64_t row_stride_bytes, uint64_t group_stride_bytes, uint32_t box_cols,
+                     uint32_t box_rows);
+// Builds the descriptor for an operand of a GEMM with the given tile height
+// (128 for A, block_n for B).
+bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
+                  uint64_t groups, uint64_t ld_elems, uint64_t group_stride_elems, int tile_mn);
+cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, cudaStream_t st);
+cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, int split_k,
+                                 long split_stride, int groups, long partial_group_stride,
+                                 long out_group_stride, cudaStream_t st);
+
+// ---------------------------------------------------------------- sweep
+struct SweepHp {
+    float lr, alpha, eps;
+};
+// Per-agent asynchronous form.  Any of peer0/peer1 may be null (n_peers says how many are used).
+cudaError_t launch_sweep_agent(float* x, const float* g, float* v, float* snap_out, const float* peer0,
+                               const float* peer1, int n_peers, const float* clip, __nv_bfloat16* shadow,
+                               long d_pad, SweepHp hp, cudaStream_t st);
+// Synchronous all-agent form.  peer_off[j]: in-peer j of agent i is (i - peer_off[j]) mod n.
+cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* clip,
+                              __nv_bfloat16* shadow, int n_agents, long d_pad, int n_peers,
+                              const int* peer_off, SweepHp hp, cudaStream_t st);
+// Sum of squares of g[agent][0..d) -> norm[agent], clip[agent] = min(1, max_norm/(norm+1e-6)).
+// partial: [n_agents][kNormChunks] doubles, ticket: [n_agents] uints (zero before first use).
+constexpr int kNormChunks = 32;
+cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
+                             double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st);
+cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st);
+
+// ---------------------------------------------------------------- A2C pieces
+// Caller-owned per-agent pointers travel in kernel parameters, at most kBatch agents a launch.
+constexpr int kBatch = 64;
+struct PtrBatch { const void* p[kBatch]; };
+
+struct LossArgs {
+    int T, E, A;
+    float gamma, ent_coef, vf_coef;
+    const float* logits;   // [agents][B][A]
+    const float* values;   // [agents][B]
+    PtrBatch actions, rewards, dones;  // per agent [T][E]
+    float* returns;        // [agents][S]
+    float* adv;            // [agents][S]
+    float* dlogits;        // [agents][S][A]
+    float* dvalues;        // [agents][S]
+    float* losses;         // [agents][4]
+    long B;                // (T+1)*E
+};
+cudaError_t launch_a2c_loss(const LossArgs& a, int n_agents, cudaStream_t st);
+cudaError_t launch_sample(const float* logits, const float* uniforms, int* actions, int E, int A,
+                          cudaStream_t st);
+
+// Small dense layers on the CUDA cores (fp32 accumulate).  TIn: float or bf16.
+// act: 0 none, 1 relu, 2 tanh.  Group g uses W + g*w_stride etc.
+struct DenseArgs {
+    int rows, in_dim, out_dim, act;
+    PtrBatch in;                           // per group [rows][in_dim]
+    int in_bf16;
+    const float* W; const float* b; long w_stride;  // W[out][in], b[out] inside the flat vector
+    void* out; long out_stride; int out_bf16;       // [g][rows][out_dim]
+};
+cudaError_t launch_dense_fwd(const DenseArgs& a, int groups, cudaStream_t st);
+// heads: logits[g][rows][A], values[g][rows]
+struct HeadsArgs {
+    int rows, H, A;
+    const void* h; long h_stride; int h_bf16;
+    const float* params; long p_stride;   // flat vectors; offsets below
+    long piw, pib, vw, vb;
+    float* logits; long logits_stride;
+    float* values; long values_stride;
+};
+cudaError_t launch_heads_fwd(const HeadsArgs& a, int groups, cudaStream_t st);
+struct HeadsBwdArgs {
+    int rows, H, A, act;   // rows = S; act of the hidden layer (1 relu, 2 tanh)
+    const void* h; long h_stride; int h_bf16;
+    const float* params; long p_stride;
+    long piw, pib, vw, vb;
+    const float* dlogits; long dlogits_stride;   // [g][S][A]
+    const float* dvalues; long dvalues_stride;   // [g][S]
+    float* grad; long g_stride;                  // flat gradient (same offsets)
+    void* dpre; long dpre_stride; int dpre_bf16; // [g][S][H] dL/d(pre-activation of hidden)
+};
+cudaError_t launch_heads_bwd(const HeadsBwdArgs& a, int groups, cudaStream_t st);
+struct DenseBwdArgs {
+    int rows, in_dim, out_dim, act_in;    // act_in: activation that produced `in` (0 none: no dgrad)
+    PtrBatch in;                          // per group [rows][in_dim]  (fp32)
+    const float* dpre; long dpre_stride;  // [g][rows][out_dim]
+    const float* W; long w_stride;        // flat params + offset of W
+    float* gW; float* gb; long g_stride;  // flat grad + offsets
+    float* din; long din_stride;          // [g][rows][in_dim] dL/d(pre-activation of previous layer); null: skip
+};
+cudaError_t launch_dense_bwd(const DenseBwdArgs& a, int groups, cudaStream_t st);
+
+// ---------------------------------------------------------------- conv lowering
+cudaError_t launch_im2col_u8(const PtrBatch& obs, __nv_bfloat16* cols, long cols_group_stride, int samples,
+                             int groups, cudaStream_t st);
+cudaError_t launch_im2col_bf16(const __nv_bfloat16* act, long act_group_stride, __nv_bfloat16* cols,
+                               long cols_group_stride, int layer, int samples, int groups, cudaStream_t st);
+// dX = mask(act_in > 0) * scatter-sum of dcols; layer = 1 or 2 (conv2, conv3)
+cudaError_t launch_col2im(const __nv_bfloat16* dcols, long dcols_group_stride, const __nv_bfloat16* act_in,
+                          long act_group_stride, __nv_bfloat16* dx, long dx_group_stride, int layer,
+                          int samples, int groups, cudaStream_t st);
+// out[g][c] = sum_r dy[g][r][c]   (bf16 in, fp32 out at out + g*out_stride), fixed summation order
+cudaError_t launch_colsum(const __nv_bfloat16* dy, long dy_group_stride, long rows, int C, float* out,
+                          long out_group_stride, double* partial, unsigned* ticket, int groups,
+                          cudaStream_t st);
+constexpr int kColsumChunks = 64;
+
+}  // namespace gala

@@ -1,0 +1,245 @@
+// Fused RMSProp + gossip pass over the flat parameter vectors (Algorithm 1,
+// optimiser step, broadcast and conditional averaging; Eqs. 5-7; Table 2
+// RMSProp rows; mixing weights 1/(1+|N_in|) from the footnote of Algorithm 1).
+//
+// Both forms are pure streaming kernels: every array element is read once and
+// written once with 16-byte accesses.
+#include "internal.h"
+
+namespace gala {
+
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+    // read-once data: bypass L1 allocation
+    return __ldcs(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void st_stream(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+__device__ __forceinline__ void rms1(float& x, float g, float& v, float c, SweepHp hp) {
+    float gi = c * g;
+    v = hp.alpha * v + (1.0f - hp.alpha) * gi * gi;
+    x = x - hp.lr * gi / (sqrtf(v) + hp.eps);
+}
+__device__ __forceinline__ void rms4(float4& x, float4 g, float4& v, float c, SweepHp hp) {
+    rms1(x.x, g.x, v.x, c, hp);
+    rms1(x.y, g.y, v.y, c, hp);
+    rms1(x.z, g.z, v.z, c, hp);
+    rms1(x.w, g.w, v.w, c, hp);
+}
+__device__ __forceinline__ void st_bf16x4(__nv_bfloat16* p, float4 v) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<unsigned*>(&a);
+    u.y = *reinterpret_cast<unsigned*>(&b);
+    *reinterpret_cast<uint2*>(p) = u;
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-agent form: y = RMSProp(x, c*g, v); snapshot <- y; x <- y or (y + sum peers)/(1+p).
+// g == nullptr: no pending gradient (y = x, v untouched).
+template <int P>
+__global__ void __launch_bounds__(256) sweep_agent_kernel(float* __restrict__ x, const float* __restrict__ g,
+                                                          float* __restrict__ v, float* __restrict__ snap,
+                                                          const float* __restrict__ peer0,
+                                                          const float* __restrict__ peer1,
+                                                          const float* __restrict__ clip,
+                                                          __nv_bfloat16* __restrict__ shadow, long n4,
+                                                          SweepHp hp) {
+    const float c = clip ? *clip : 1.0f;
+    const float w = 1.0f / (1.0f + P);
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x) {
+        const long o = i * 4;
+        float4 xi = ld_stream(x + o);
+        if (g) {
+            float4 gi = ld_stream(g + o);
+            float4 vi = ld_stream(v + o);
+            rms4(xi, gi, vi, c, hp);
+            st_stream(v + o, vi);
+        }
+        st_stream(snap + o, xi);
+        if (P >= 1) {
+            float4 m = ld_stream(peer0 + o);
+            xi.x += m.x; xi.y += m.y; xi.z += m.z; xi.w += m.w;
+        }
+        if (P >= 2) {
+            float4 m = ld_stream(peer1 + o);
+            xi.x += m.x; xi.y += m.y; xi.z += m.z; xi.w += m.w;
+        }
+        if (P >= 1) { xi.x *= w; xi.y *= w; xi.z *= w; xi.w *= w; }
+        st_stream(x + o, xi);
+        if (shadow) st_bf16x4(shadow + o, xi);
+    }
+}
+
+cudaError_t launch_sweep_agent(float* x, const float* g, float* v, float* snap_out, const float* peer0,
+                               const float* peer1, int n_peers, const float* clip, __nv_bfloat16* shadow,
+                               long d_pad, SweepHp hp, cudaStream_t st) {
+    long n4 = d_pad / 4;
+    int grid = (int)((n4 + 255) / 256);
+    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid < 1) grid = 1;
+    if (n_peers == 0)
+        sweep_agent_kernel<0><<<grid, 256, 0, st>>>(x, g, v, snap_out, nullptr, nullptr, clip, shadow, n4, hp);
+    else if (n_peers == 1)
+        sweep_agent_kernel<1><<<grid, 256, 0, st>>>(x, g, v, snap_out, peer0, nullptr, clip, shadow, n4, hp);
+    else
+        sweep_agent_kernel<2><<<grid, 256, 0, st>>>(x, g, v, snap_out, peer0, peer1, clip, shadow, n4, hp);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Synchronous all-agent form: each thread owns one 16-byte column across all agents.  It
+// applies RMSProp to every agent's element, parks the results y_i in shared memory (its own
+// private column, so no barrier is needed), then forms x_i = (y_i + sum_j y_{i-off_j}) / (1+p)
+// from those parked values.  x, g, v are read once and x, v written once: 20 B per parameter,
+// independent of the number of in-peers.
+constexpr int kSyncUnroll = 4;
+
+template <int P>
+__global__ void sweep_sync_kernel(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ v,
+                                  const float* __restrict__ clip, __nv_bfloat16* __restrict__ shadow,
+                                  int n_agents, long d_pad, long n4, int off0, int off1, SweepHp hp) {
+    extern __shared__ float4 ysm[];  // [n_agents][blockDim.x]
+    const float w = 1.0f / (1.0f + P);
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x) {
+        const long o = i * 4;
+        int a = 0;
+        for (; a + kSyncUnroll <= n_agents; a += kSyncUnroll) {
+            float4 xi[kSyncUnroll], gi[kSyncUnroll], vi[kSyncUnroll];
+#pragma unroll
+            for (int u = 0; u < kSyncUnroll; u++) {
+                const long off = (long)(a + u) * d_pad + o;
+                xi[u] = ld_stream(x + off);
+                gi[u] = ld_stream(g + off);
+                vi[u] = ld_stream(v + off);
+            }
+#pragma unroll
+            for (int u = 0; u < kSyncUnroll; u++) {
+                const float c = clip ? __ldg(clip + a + u) : 1.0f;
+                rms4(xi[u], gi[u], vi[u], c, hp);
+                st_stream(v + (long)(a + u) * d_pad + o, vi[u]);
+                ysm[(a + u) * blockDim.x + threadIdx.x] = xi[u];
+            }
+        }
+        for (; a < n_agents; a++) {
+            const long off = (long)a * d_pad + o;
+            float4 xi = ld_stream(x + off), gi = ld_stream(g + off), vi = ld_stream(v + off);
+            const float c = clip ? __ldg(clip + a) : 1.0f;
+            rms4(xi, gi, vi, c, hp);
+            st_stream(v + off, vi);
+            ysm[a * blockDim.x + threadIdx.x] = xi;
+        }
+        for (a = 0; a < n_agents; a++) {
+            float4 y = ysm[a * blockDim.x + threadIdx.x];
+            if (P >= 1) {
+                int j = a - off0; if (j < 0) j += n_agents;
+                float4 m = ysm[j * blockDim.x + threadIdx.x];
+                y.x += m.x; y.y += m.y; y.z += m.z; y.w += m.w;
+            }
+            if (P >= 2) {
+                int j = a - off1; if (j < 0) j += n_agents;
+                float4 m = ysm[j * blockDim.x + threadIdx.x];
+                y.x += m.x; y.y += m.y; y.z += m.z; y.w += m.w;
+            }
+            if (P >= 1) { y.x *= w; y.y *= w; y.z *= w; y.w *= w; }
+            const long off = (long)a * d_pad + o;
+            st_stream(x + off, y);
+            if (shadow) st_bf16x4(shadow + off, y);
+        }
+    }
+}
+
+cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* clip,
+                              __nv_bfloat16* shadow, int n_agents, long d_pad, int n_peers,
+                              const int* peer_off, SweepHp hp, cudaStream_t st) {
+    long n4 = d_pad / 4;
+    // shared memory: n_agents * threads * 16 B, kept under 128 KB so that one block always fits
+    int threads = 256;
+    while (threads > 32 && (long)n_agents * threads * 16 > 128 * 1024) threads /= 2;
+    size_t smem = (size_t)n_agents * threads * 16;
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    long blocks = (n4 + threads - 1) / threads;
+    int per_sm = (int)((200 * 1024) / (smem ? smem : 1));
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm > 8) per_sm = 8;
+    long cap = 148L * per_sm;
+    int grid = (int)(blocks < cap ? blocks : cap);
+    if (grid < 1) grid = 1;
+    int o0 = 0, o1 = 0;
+    if (n_peers >= 1) o0 = ((peer_off[0] % n_agents) + n_agents) % n_agents;
+    if (n_peers >= 2) o1 = ((peer_off[1] % n_agents) + n_agents) % n_agents;
+    cudaError_t e;
+#define GALA_SYNC_LAUNCH(P)                                                                          \
+    e = cudaFuncSetAttribute(sweep_sync_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    if (e != cudaSuccess) return e;                                                                  \
+    sweep_sync_kernel<P><<<grid, threads, smem, st>>>(x, g, v, clip, shadow, n_agents, d_pad, n4, o0, o1, hp);
+    if (n_peers == 0) { GALA_SYNC_LAUNCH(0) }
+    else if (n_peers == 1) { GALA_SYNC_LAUNCH(1) }
+    else if (n_peers == 2) { GALA_SYNC_LAUNCH(2) }
+    else return cudaErrorInvalidValue;
+#undef GALA_SYNC_LAUNCH
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Global gradient norm and clip coefficient ("Clip global gradient norm", Table 2):
+// c = min(1, max_norm / (||g||_2 + 1e-6)).  Fixed chunking and a fixed-order final sum in
+// double precision make the result independent of scheduling.
+__global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict__ g, long d, long d_pad,
+                                                        int agent0, float max_norm, double* partial,
+                                                        unsigned* ticket, float* norm, float* clip) {
+    const int agent = agent0 + blockIdx.y;
+    const float* ga = g + (long)agent * d_pad;
+    const long per = ((d + kNormChunks - 1) / kNormChunks + 3) & ~3L;
+    const long lo = (long)blockIdx.x * per;
+    long hi = lo + per; if (hi > d) hi = d;
+    double acc = 0.0;
+    for (long i = lo + threadIdx.x; i < hi; i += blockDim.x) { float t = ga[i]; acc += (double)t * t; }
+    __shared__ double red[256];
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {
+        if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+        __syncthreads();
+    }
+    __shared__ bool last;
+    if (threadIdx.x == 0) {
+        partial[(long)agent * kNormChunks + blockIdx.x] = red[0];
+        __threadfence();
+        unsigned t = atomicAdd(&ticket[agent], 1u);
+        last = (t == kNormChunks - 1);
+    }
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        __threadfence();
+        double s = 0.0;
+        for (int k = 0; k < kNormChunks; k++) s += ((volatile double*)partial)[(long)agent * kNormChunks + k];
+        float nrm = (float)sqrt(s);
+        norm[agent] = nrm;
+        float c = 1.0f;
+        if (max_norm > 0.0f) c = fminf(1.0f, max_norm / (nrm + 1e-6f));
+        clip[agent] = c;
+        ticket[agent] = 0;  // ready for the next launch
+    }
+}
+
+cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
+                             double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st) {
+    dim3 grid(kNormChunks, n_agents);
+    grad_norm_kernel<<<grid, 256, 0, st>>>(g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip);
+    return cudaGetLastError();
+}
+
+__global__ void cast_bf16_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ out, long n4) {
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x)
+        st_bf16x4(out + i * 4, *reinterpret_cast<const float4*>(x + i * 4));
+}
+cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st) {
+    long n4 = count / 4;
+    int grid = (int)((n4 + 255) / 256);
+    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid < 1) grid = 1;
+    cast_bf16_kernel<<<grid, 256, 0, st>>>(x, out, n4);
+    return cudaGetLastError();
+}
+
+}  // namespace gala

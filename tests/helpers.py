@@ -1,0 +1,45 @@
+"""Shared helpers of the GPU parity tests: tolerance rule, oracle <-> library glue."""
+from __future__ import annotations
+
+import numpy as np
+
+import gala_inputs as GI
+from oracle import reference as R
+
+# Tolerances (relative), one per arithmetic path.
+TOL_SWEEP = 1e-5      # fp32 RMSProp + gossip pass fed identical fp32 inputs
+TOL_FP32_NET = 1e-4   # fp32 network (MLP) outputs and gradients
+TOL_BF16 = 2e-2       # bf16-operand GEMM outputs and gradients
+
+
+def assert_close(name, got, want, tol):
+    """Per tensor: ||a-b||_2 <= tol ||b||_2  and  |a_i-b_i| <= tol (|b_i| + rms(b))."""
+    a = np.asarray(got, np.float64).ravel()
+    b = np.asarray(want, np.float64).ravel()
+    assert a.shape == b.shape, (name, a.shape, b.shape)
+    assert np.isfinite(a).all(), name + ": non-finite values"
+    nb = np.linalg.norm(b)
+    rel = np.linalg.norm(a - b) / (nb if nb > 0 else 1.0)
+    rms = nb / np.sqrt(max(1, b.size))
+    worst = np.max(np.abs(a - b) / (np.abs(b) + rms + 1e-30)) if b.size else 0.0
+    assert rel <= tol, "%s: relative l2 error %.3e > %.1e" % (name, rel, tol)
+    assert worst <= tol, "%s: worst element error %.3e > %.1e (rel l2 %.3e)" % (name, worst, tol, rel)
+    return rel
+
+
+def oracle_net(w: GI.Workload) -> R.Net:
+    return R.Net.atari(w.n_actions) if w.net_kind == "conv" else R.Net.mlp(w.obs_dim, w.hidden, w.n_actions)
+
+
+def oracle_hp(hp) -> R.HParams:
+    """Oracle hyper-parameters = the float32 values the library was given, widened."""
+    return R.HParams(lr=float(hp.lr), rms_alpha=float(hp.rms_alpha), rms_eps=float(hp.rms_eps),
+                     gamma=float(hp.gamma), ent_coef=float(hp.ent_coef), vf_coef=float(hp.vf_coef),
+                     max_grad_norm=float(hp.max_grad_norm))
+
+
+def to_bf16_f64(a: np.ndarray) -> np.ndarray:
+    """Round float32 values to bfloat16 (nearest even) and return them as float64."""
+    u = np.ascontiguousarray(a, np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64)

@@ -1,0 +1,296 @@
+"""GPU parity of the learner path against the fp64 oracle, through the C ABI:
+synchronous rounds (Eq. 7 with zero delay), acting, and the per-agent
+asynchronous calls replayed from the library's own schedule log."""
+import numpy as np
+import pytest
+
+import gala_inputs as GI
+from oracle import reference as R
+from tests.helpers import TOL_BF16, TOL_FP32_NET, TOL_SWEEP, assert_close, oracle_hp, oracle_net
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _mods():
+    from paper_1906_04585_b200 import binding, learner
+    return binding, learner
+
+
+def make_learner(w: GI.Workload, **hp):
+    B, LM = _mods()
+    L = LM.Learner(w.n_agents, w.topo_kind, w.topo_peers, w.net_kind, w.n_actions, w.n_envs, w.n_steps,
+                   obs_dim=w.obs_dim, hidden=w.hidden, **hp)
+    return L
+
+
+def seed_identical(L, w, net):
+    """Give GPU and oracle the same float32 starting point (input data, not shared code)."""
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    assert p0.size == L.d == R.param_count(net)
+    for i in range(w.n_agents):
+        L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32), rnd=0)
+    X = np.tile(p0.astype(np.float64), (w.n_agents, 1))
+    return X, np.zeros_like(X)
+
+
+def test_library_init_is_identical_and_scaled():
+    w = GI.WORKLOADS[0]
+    L = make_learner(w, seed=11)
+    p = [L.get_params(i) for i in range(w.n_agents)]
+    for q in p[1:]:
+        np.testing.assert_array_equal(q, p[0])       # identical initialisation (assumed by Prop. 1)
+    w1 = p[0][: 64 * 8]
+    assert np.abs(w1).max() <= 1 / np.sqrt(8) and np.abs(w1).max() > 0.8 / np.sqrt(8)
+    assert abs(w1.mean()) < 0.05
+    L2 = make_learner(w, seed=11, identical_init=0)
+    assert not np.array_equal(L2.get_params(0), L2.get_params(1))
+    np.testing.assert_array_equal(L2.get_params(0), p[0])
+    L.close(); L2.close()
+
+
+def test_topology_schedule_bit_exact():
+    for n, kind, peers in [(4, R.RING, 1), (8, R.EXP, 1), (16, R.EXP, 1), (32, R.EXP, 2), (5, R.EXP, 2), (6, R.RING, 2)]:
+        w = GI.WORKLOADS[0].scaled(n_agents=n, topo_kind=kind, topo_peers=peers, n_envs=2, n_steps=2)
+        L = make_learner(w)
+        for k in list(range(12)) + [1000003]:
+            for i in range(n):
+                assert L.in_peers(k, i) == R.in_peers(kind, peers, n, k, i)
+        L.close()
+
+
+def check_params(name, got, want, before, tol, mode):
+    """mode 'elementwise': the fp32 path, every element within tol.
+    mode 'update': the bf16 path.  RMSProp with a tiny epsilon is close to a sign update, so an
+    element whose gradient is smaller than the bf16 noise may step the other way; the parameters are
+    therefore compared in l2 (relative tol), and the update x_new - x_old in l2 with a loose bound."""
+    if mode == "elementwise":
+        assert_close(name, got, want, tol)
+        return
+    a, b, x0 = (np.asarray(t, np.float64) for t in (got, want, before))
+    assert np.isfinite(a).all()
+    assert np.linalg.norm(a - b) <= tol * np.linalg.norm(b), name
+    du = np.linalg.norm((a - x0) - (b - x0)) / max(np.linalg.norm(b - x0), 1e-30)
+    assert du <= 0.3, "%s: update differs by %.3f in l2" % (name, du)
+
+
+def _sync_rounds(w, rounds, tol_net, tol_params, mode="elementwise", **hp):
+    B_, LM = _mods()
+    net = oracle_net(w)
+    L = make_learner(w, **hp)
+    ohp = oracle_hp(L.hp)
+    X, V = seed_identical(L, w, net)
+    S, B, A = w.n_envs * w.n_steps, w.n_envs * (w.n_steps + 1), w.n_actions
+    for k in range(rounds):
+        ros = [GI.rollout(w, i, k) for i in range(w.n_agents)]
+        dev = [LM.DeviceRollout(r) for r in ros]
+        L.step_sync(dev)
+        L.sync()
+        Xn, Vn, infos = R.sync_round(net, X, V, ros, ohp, w.topo_kind, w.topo_peers, k, workers=4)
+        for i in range(w.n_agents):
+            f = infos[i]
+            assert_close("logits[%d]" % i, L.debug(i, 0, B * A), f["logits"], tol_net)
+            assert_close("values[%d]" % i, L.debug(i, 1, B), f["values"], tol_net)
+            assert_close("returns[%d]" % i, L.debug(i, 2, S), f["G"], tol_net)
+            # advantages are differences of nearly equal numbers: compare on the scale of the returns
+            scale = np.abs(f["G"]).max() + np.abs(f["values"]).max() + 1.0
+            assert np.abs(L.debug(i, 3, S) - f["adv"].ravel()).max() <= tol_net * scale
+            assert_close("grad[%d]" % i, L.get_grad(i), f["grad"], tol_net)
+            ls = B_.gala_losses(L.ctx, i)
+            for q in range(3):
+                assert abs(ls[q] - f["losses"][q]) <= tol_net * (abs(f["losses"][q]) + 1.0)
+            _, nrm = R.clip_coef(f["grad"], ohp.max_grad_norm)
+            assert abs(ls[3] - nrm) <= tol_net * nrm
+            check_params("x[%d]" % i, L.get_params(i), Xn[i], X[i], tol_params, mode)
+            if mode == "elementwise":
+                assert_close("v[%d]" % i, L.get_sq_avg(i), Vn[i], max(tol_params, 2 * tol_net))
+            else:
+                a, b = L.get_sq_avg(i).astype(np.float64), Vn[i]
+                assert np.linalg.norm(a - b) <= 2 * tol_net * np.linalg.norm(b)
+        if mode == "elementwise":
+            X, V = Xn, Vn           # true multi-round trajectory
+        else:
+            # bf16 path: start every round from the oracle's state (rounded to fp32 on both sides), so
+            # that a round's check is not blurred by the previous rounds' bf16 differences
+            X = Xn.astype(np.float32).astype(np.float64)
+            V = Vn.astype(np.float32).astype(np.float64)
+            for i in range(w.n_agents):
+                L.set_state(i, params=X[i], sq_avg=V[i], rnd=k + 1)
+    L.close()
+
+
+def test_config1_mlp_sync_rounds():
+    # the small fp32 workload in full: 4 agents, ring, 16 envs x 5 steps, 3 rounds
+    _sync_rounds(GI.WORKLOADS[0], rounds=3, tol_net=TOL_FP32_NET, tol_params=TOL_SWEEP)
+
+
+@pytest.mark.parametrize("n,kind,peers,E,T,A", [(3, R.RING, 2, 5, 3, 4), (8, R.EXP, 2, 7, 37, 6), (2, R.EXP, 1, 33, 1, 2)])
+def test_mlp_sync_ragged_shapes(n, kind, peers, E, T, A):
+    # ragged env counts, horizons beyond one warp of time steps, horizon 1
+    w = GI.WORKLOADS[0].scaled(n_agents=n, topo_kind=kind, topo_peers=peers, n_envs=E, n_steps=T, n_actions=A,
+                               done_p=0.1)
+    _sync_rounds(w, rounds=2, tol_net=TOL_FP32_NET, tol_params=TOL_SWEEP)
+
+
+def test_mlp_without_clipping():
+    _sync_rounds(GI.WORKLOADS[0].scaled(n_agents=2), rounds=2, tol_net=TOL_FP32_NET, tol_params=TOL_SWEEP,
+                 max_grad_norm=0.0, rms_eps=0.01)
+
+
+def test_act_sampling_matches_oracle():
+    w = GI.WORKLOADS[0].scaled(n_envs=64)
+    net = oracle_net(w)
+    L = make_learner(w)
+    seed_identical(L, w, net)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    obs = GI.rollout(w, 0, 0)["obs"][0]
+    u = GI.uniforms(w, 0, 0, w.n_envs)
+    a, v = L.act(0, torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())
+    L.sync()
+    z, val = R.forward(net, p0, obs)
+    want = R.sample(z, u)
+    got = a.cpu().numpy()
+    assert_close("values", v.cpu().numpy(), val, TOL_FP32_NET)
+    cdf = np.cumsum(R.softmax(z), axis=1)
+    mism = np.nonzero(got != want)[0]
+    for e in mism:   # a different draw is only acceptable on a CDF boundary
+        assert np.min(np.abs(cdf[e] - u[e])) < 1e-5, (e, cdf[e], u[e])
+    assert len(mism) <= 1
+    L.close()
+
+
+def _async_replay(w, order, tol_net, tol_params, mode="elementwise"):
+    """Drive learn/gossip per agent in the given order, waiting after every call so that the
+    schedule is deterministic, and replay the library's own (peer, version) log in the oracle."""
+    B, LM = _mods()
+    net = oracle_net(w)
+    L = make_learner(w)
+    ohp = oracle_hp(L.hp)
+    X, V = seed_identical(L, w, net)
+    n = w.n_agents
+    snaps = {}            # (agent, version) -> oracle snapshot
+    version = [0] * n
+    rnd = [0] * n
+    mixes = 0
+    for step, i in enumerate(order):
+        ro = GI.rollout(w, i, rnd[i])
+        L.learn(i, LM.DeviceRollout(ro))
+        L.gossip(i)
+        L.sync()
+        peers, vers, mixed = B.gala_last_mix(L.ctx, i)
+        assert peers == R.in_peers(w.topo_kind, w.topo_peers, n, rnd[i], i)
+        info = R.learner_grad(net, X[i], ro, ohp)
+        x_before = X[i].copy()
+        msgs = None
+        if mixed:
+            mixes += 1
+            for pj, vj in zip(peers, vers):
+                assert 1 <= vj <= version[pj]          # only complete, published versions
+            msgs = [snaps[(pj, vj)] for pj, vj in zip(peers, vers)]
+        xn, vn, y = R.sweep_replay(X[i], info["grad"], V[i], ohp, msgs)
+        version[i] += 1
+        snaps[(i, version[i])] = y
+        X[i], V[i] = xn, vn
+        rnd[i] += 1
+        assert_close("grad", L.get_grad(i), info["grad"], tol_net)
+        snap = np.empty(L.d, np.float32)
+        B.gala_get_snapshot(L.ctx, i, version[i], snap)
+        check_params("x", L.get_params(i), X[i], x_before, tol_params, mode)
+        check_params("snapshot", snap, y, x_before, tol_params, mode)
+        if mode == "elementwise":
+            assert_close("v", L.get_sq_avg(i), V[i], max(tol_params, 2 * tol_net))
+        else:
+            # keep both sides on the same trajectory (oracle -> library only)
+            X[i] = X[i].astype(np.float32).astype(np.float64)
+            V[i] = V[i].astype(np.float32).astype(np.float64)
+            snaps[(i, version[i])] = y.astype(np.float32).astype(np.float64)
+            L.set_state(i, params=X[i], sq_avg=V[i], rnd=rnd[i])
+        st = B.gala_stats(L.ctx, i)
+        assert st["version"] == version[i] and st["rounds"] == rnd[i]
+    assert mixes > 0
+    total = sum(B.gala_stats(L.ctx, i)["mixes"] + B.gala_stats(L.ctx, i)["skipped"] for i in range(n))
+    assert total == len(order)
+    L.close()
+    return mixes
+
+
+def test_async_replay_mlp():
+    w = GI.WORKLOADS[0]
+    # uneven progress: agent 0 runs ahead, agent 3 lags (stale and missing messages both occur)
+    order = [0, 0, 1, 2, 0, 3, 1, 1, 2, 3, 0, 2, 3, 3, 1, 0]
+    mixes = _async_replay(w, order, TOL_FP32_NET, TOL_SWEEP)
+    assert mixes < len(order)      # some iterations found no fresh message and skipped the average
+
+
+def test_second_learn_applies_pending_gradient_without_mixing():
+    B, LM = _mods()
+    w = GI.WORKLOADS[0].scaled(n_agents=2)
+    net = oracle_net(w)
+    L = make_learner(w)
+    ohp = oracle_hp(L.hp)
+    X, V = seed_identical(L, w, net)
+    r0, r1 = GI.rollout(w, 0, 0), GI.rollout(w, 0, 1)
+    L.learn(0, LM.DeviceRollout(r0))
+    L.learn(0, LM.DeviceRollout(r1))
+    L.sync()
+    i0 = R.learner_grad(net, X[0], r0, ohp)
+    x1, v1, _ = R.sweep_replay(X[0], i0["grad"], V[0], ohp, None)
+    i1 = R.learner_grad(net, x1, r1, ohp)
+    assert_close("x", L.get_params(0), x1, TOL_SWEEP)
+    assert_close("grad", L.get_grad(0), i1["grad"], TOL_FP32_NET)
+    # gossip with nothing pending on the other agent: parameters unchanged, snapshot published
+    p_before = L.get_params(1).astype(np.float64)
+    v_before = L.get_sq_avg(1)
+    L.gossip(1)
+    L.sync()
+    peers, vers, mixed = B.gala_last_mix(L.ctx, 1)
+    assert peers == [0] and vers == [1] and mixed      # agent 0 published version 1 above
+    assert_close("x1", L.get_params(1), 0.5 * (p_before + x1), TOL_SWEEP)
+    np.testing.assert_array_equal(L.get_sq_avg(1), v_before)
+    L.close()
+
+
+# ------------------------------------------------------------------ conv net
+def test_conv_forward_layers():
+    w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=3, n_steps=2)
+    net = oracle_net(w)
+    L = make_learner(w)
+    seed_identical(L, w, net)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    _, LM = _mods()
+    ros = [GI.rollout(w, i, 0) for i in range(2)]
+    L.step_sync([LM.DeviceRollout(r) for r in ros])
+    L.sync()
+    Bn = 3 * 3
+    for i in range(2):
+        obs = ros[i]["obs"].reshape(Bn, -1)
+        for li, shape in enumerate([(20, 20, 32), (9, 9, 64), (7, 7, 64), (512,)]):
+            want = R.forward(net, p0, obs, which_layer=li)[2]
+            got = L.debug(i, 10 + li, want.size)
+            assert_close("layer%d[%d]" % (li, i), got, want, TOL_BF16)
+    L.close()
+
+
+def test_conv_sync_rounds_small():
+    # full-size network, reduced batch: 2 agents x (3 envs x 2 steps)
+    w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=3, n_steps=2)
+    _sync_rounds(w, rounds=2, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
+
+
+def test_conv_sync_rounds_table2_epsilon():
+    # Table 2's RMSProp epsilon (0.01): the update is smooth in the gradient, so the update itself
+    # must agree to the bf16 tolerance scale
+    w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=2, n_steps=2)
+    _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update", rms_eps=0.01)
+
+
+def test_conv_sync_rounds_multi_tile():
+    # 18 actions, batch spanning several 128-row tiles with ragged tails, 2-peer exponential graph
+    w = GI.WORKLOADS[2].scaled(n_agents=4, n_envs=5, n_steps=7, topo_peers=2)
+    _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
+
+
+def test_async_replay_conv():
+    w = GI.WORKLOADS[1].scaled(n_agents=4, n_envs=2, n_steps=3)
+    _async_replay(w, [0, 1, 0, 2, 3, 1, 0, 3], TOL_BF16, TOL_BF16, mode="update")
