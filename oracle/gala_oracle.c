@@ -47,6 +47,11 @@ typedef struct {
     int act;
     int n_actions;
     double in_scale; /* observation multiplier (1/255 for byte frames) */
+    /* Reduced-precision operand emulation ("bf16 GEMMs, fp32 params"): when set, every trunk
+     * layer's output activation and every dL/d(pre-activation) is rounded to bfloat16 (nearest
+     * even), as a kernel that stores them in bf16 would; sums stay exact (double).  The caller
+     * rounds the trunk weights itself.  0 = exact arithmetic throughout. */
+    int round_bf16;
 } orc_net;
 
 typedef struct {
@@ -112,12 +117,24 @@ int orc_param_offsets(const orc_net *net, long *out) {
     return nl;
 }
 
+/* Round to bfloat16 (8 significant bits, nearest, ties to even), via float32. */
+double orc_round_bf16(double v) {
+    float f = (float)v;
+    unsigned int u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) return (double)f; /* inf / nan unchanged */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
 static double act_fn(int act, double z) { return act == 0 ? (z > 0.0 ? z : 0.0) : tanh(z); }
 /* derivative expressed through the layer OUTPUT a = act(z) */
 static double act_grad(int act, double a) { return act == 0 ? (a > 0.0 ? 1.0 : 0.0) : 1.0 - a * a; }
 
 /* One trunk layer, one sample: y = act(W * x + b). */
-static void layer_forward(const orc_layer *l, int act, const double *p, const double *x, double *y) {
+static void layer_forward(const orc_layer *l, int act, int rnd, const double *p, const double *x, double *y) {
     const double *W = p + l->w_off, *b = p + l->b_off;
     if (!l->conv) {
         for (int o = 0; o < l->oc; o++) {
@@ -125,6 +142,7 @@ static void layer_forward(const orc_layer *l, int act, const double *p, const do
             const double *w = W + (long)o * l->in_size;
             for (long i = 0; i < l->in_size; i++) acc += w[i] * x[i];
             y[o] = act_fn(act, acc);
+            if (rnd) y[o] = orc_round_bf16(y[o]);
         }
         return;
     }
@@ -138,18 +156,22 @@ static void layer_forward(const orc_layer *l, int act, const double *p, const do
                         const double *w = W + (((long)o * l->k + ky) * l->k + kx) * l->ic;
                         for (int c = 0; c < l->ic; c++) acc += w[c] * xi[c];
                     }
-                y[((long)oy * l->ow + ox) * l->oc + o] = act_fn(act, acc);
+                double a = act_fn(act, acc);
+                y[((long)oy * l->ow + ox) * l->oc + o] = rnd ? orc_round_bf16(a) : a;
             }
 }
 
 /* One trunk layer, one sample, backward.  dy is dL/d(output); it is turned
  * into dL/d(pre-activation) in place.  Accumulates into g (W and b), writes
  * dx (may be NULL for the first layer). */
-static void layer_backward(const orc_layer *l, int act, const double *p, const double *x,
+static void layer_backward(const orc_layer *l, int act, int rnd, const double *p, const double *x,
                            const double *y, double *dy, double *g, double *dx) {
     const double *W = p + l->w_off;
     double *gW = g + l->w_off, *gb = g + l->b_off;
-    for (long i = 0; i < l->out_size; i++) dy[i] *= act_grad(act, y[i]);
+    for (long i = 0; i < l->out_size; i++) {
+        dy[i] *= act_grad(act, y[i]);
+        if (rnd) dy[i] = orc_round_bf16(dy[i]);
+    }
     if (dx) memset(dx, 0, sizeof(double) * (size_t)l->in_size);
     if (!l->conv) {
         for (int o = 0; o < l->oc; o++) {
@@ -203,7 +225,7 @@ int orc_forward(const orc_net *net, const double *params, const double *obs, int
         for (long i = 0; i < L[0].in_size; i++) a0[i] = o[i] * net->in_scale;
         double *x = a0, *y = a1;
         for (int li = 0; li < nl; li++) {
-            layer_forward(&L[li], net->act, params, x, y);
+            layer_forward(&L[li], net->act, net->round_bf16, params, x, y);
             if (layer_out && li == which_layer)
                 memcpy(layer_out + (long)s * L[li].out_size, y, sizeof(double) * (size_t)L[li].out_size);
             double *t = x; x = y; y = t;
@@ -242,7 +264,7 @@ int orc_backward(const orc_net *net, const double *params, const double *obs, in
     for (int s = 0; s < B; s++) {
         const double *o = obs + (long)s * L[0].in_size;
         for (long i = 0; i < L[0].in_size; i++) acts[0][i] = o[i] * net->in_scale;
-        for (int li = 0; li < nl; li++) layer_forward(&L[li], net->act, params, acts[li], acts[li + 1]);
+        for (int li = 0; li < nl; li++) layer_forward(&L[li], net->act, net->round_bf16, params, acts[li], acts[li + 1]);
         long H = L[nl - 1].out_size;
         const double *h = acts[nl];
         /* heads */
@@ -264,7 +286,7 @@ int orc_backward(const orc_net *net, const double *params, const double *obs, in
         /* trunk */
         double *dy = da, *dx = db;
         for (int li = nl - 1; li >= 0; li--) {
-            layer_backward(&L[li], net->act, params, acts[li], acts[li + 1], dy, grad, li > 0 ? dx : NULL);
+            layer_backward(&L[li], net->act, net->round_bf16, params, acts[li], acts[li + 1], dy, grad, li > 0 ? dx : NULL);
             double *t = dy; dy = dx; dx = t;
         }
     }

@@ -29,7 +29,7 @@ from __future__ import annotations
 import ctypes as C
 import math
 from concurrent.futures import ThreadPoolExecutor
-from dataclasses import dataclass, field
+from dataclasses import dataclass, field, replace
 from typing import Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
@@ -49,6 +49,7 @@ class _CNet(C.Structure):
         ("act", C.c_int),
         ("n_actions", C.c_int),
         ("in_scale", C.c_double),
+        ("round_bf16", C.c_int),
     ]
 
 
@@ -80,6 +81,8 @@ def lib():
                                   C.c_double, dp]
         L.orc_mix.restype = None
         L.orc_mix.argtypes = [C.c_long, dp, C.c_int, C.POINTER(dp), dp]
+        L.orc_round_bf16.restype = C.c_double
+        L.orc_round_bf16.argtypes = [C.c_double]
         L.orc_sample.restype = C.c_int
         L.orc_sample.argtypes = [C.c_int, dp, C.c_double]
         _lib = L
@@ -109,6 +112,14 @@ class Net:
     act: str = "tanh"                                # "relu" | "tanh"
     n_actions: int = 4
     in_scale: float = 1.0
+    # "bf16 GEMMs, fp32 params": operands of every trunk contraction (weights, stored activations,
+    # stored pre-activation gradients) are rounded to bfloat16, sums stay exact.  Chosen so that
+    # the ReLU gate, a yes/no decision taken on a stored activation, is taken on the same number
+    # by the oracle and by a kernel that stores activations in bf16.  False: exact arithmetic.
+    bf16_operands: bool = False
+
+    def with_bf16(self, on: bool = True) -> "Net":
+        return replace(self, bf16_operands=on)
 
     @staticmethod
     def mlp(obs_dim: int = 8, hidden: int = 64, n_actions: int = 4) -> "Net":
@@ -132,6 +143,7 @@ class Net:
         n.act = 0 if self.act == "relu" else 1
         n.n_actions = self.n_actions
         n.in_scale = self.in_scale
+        n.round_bf16 = 1 if self.bf16_operands else 0
         return n
 
     @property
@@ -166,6 +178,34 @@ def param_offsets(net: Net) -> Dict[str, int]:
     return res
 
 
+def round_bf16(a) -> np.ndarray:
+    """Element-wise round to bfloat16 (nearest even), returned as float64."""
+    a = _f64(a)
+    out = np.empty_like(a)
+    L = lib()
+    flat_in, flat_out = a.ravel(), out.ravel()
+    for i in range(flat_in.size):
+        flat_out[i] = L.orc_round_bf16(float(flat_in[i]))
+    return out
+
+
+def effective_params(net: Net, params) -> np.ndarray:
+    """Parameters as the contractions see them: with bf16 operands, the trunk weight tensors are
+    rounded to bfloat16 (biases and the two linear heads stay as given)."""
+    p = _f64(params).copy()
+    if not net.bf16_operands:
+        return p
+    off = param_offsets(net)
+    nl = len(net.convs) + len(net.hidden)
+    for i in range(nl):
+        lo, hi = off["L%d.W" % i], off["L%d.b" % i]
+        f = p[lo:hi].astype(np.float32)
+        u = f.view(np.uint32).astype(np.uint64)
+        u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+        p[lo:hi] = u.astype(np.uint32).view(np.float32).astype(np.float64)
+    return p
+
+
 # --------------------------------------------------------------------------
 # network forward / backward
 # --------------------------------------------------------------------------
@@ -173,7 +213,7 @@ def forward(net: Net, params, obs, which_layer: Optional[int] = None):
     """obs: [B, ...] raw observations (any numeric dtype).  Returns
     (logits [B,A], values [B]) and, if which_layer is given, also that trunk
     layer's post-activation output [B, ...]."""
-    p = _f64(params)
+    p = effective_params(net, params)
     o = _f64(obs).reshape(len(obs), -1)
     assert o.shape[1] == net.in_size and p.size == param_count(net)
     B = o.shape[0]
@@ -191,7 +231,7 @@ def forward(net: Net, params, obs, which_layer: Optional[int] = None):
 
 
 def backward(net: Net, params, obs, dlogits, dvalues) -> np.ndarray:
-    p = _f64(params)
+    p = effective_params(net, params)
     o = _f64(obs).reshape(len(obs), -1)
     dz, dv = _f64(dlogits), _f64(dvalues)
     B = o.shape[0]

@@ -312,3 +312,63 @@ def test_sampling_rule():
     freq = np.bincount(a, minlength=3) / n
     pi = np.array([0.2, 0.5, 0.3])
     assert np.all(np.abs(freq - pi) < 3 * np.sqrt(pi * (1 - pi) / n) + 1e-9)
+
+
+# ------------------------------------------------- bf16-operand reading of "bf16 GEMMs"
+def _bf16_independent(a):
+    """bfloat16 rounding written independently: keep 8 significant bits, nearest, ties to even."""
+    a = np.asarray(a, np.float64)
+    out = np.zeros_like(a)
+    nz = a != 0
+    e = np.floor(np.log2(np.abs(a[nz])))
+    q = 2.0 ** (e - 7)                       # spacing of bf16 numbers in [2^e, 2^(e+1))
+    out[nz] = np.round(a[nz] / q) * q        # np.round: half to even
+    return out
+
+
+def test_bf16_rounding_rule():
+    vals = np.array([1.0, 1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, 1.0 + 2 ** -9, -0.3, 255.0, 1e-3, 3.1415926, 0.0,
+                     1.0 + 2 ** -8 + 2 ** -20, 129.5, 130.5])
+    got = R.round_bf16(vals)
+    np.testing.assert_array_equal(got, _bf16_independent(vals))
+    assert got[1] == 1.0 and got[2] == 1.0 + 2 ** -6 and got[9] == 1.0 + 2 ** -7   # ties to even, above tie
+    rng = np.random.default_rng(9)
+    r = (rng.standard_normal(2000) * 10.0 ** rng.integers(-3, 3, 2000)).astype(np.float32).astype(np.float64)
+    np.testing.assert_array_equal(R.round_bf16(r), _bf16_independent(r))
+
+
+def test_bf16_operand_mode_is_exact_mode_on_rounded_operands():
+    # One dense layer + heads, ReLU.  With bf16 operands the forward pass must equal the exact pass
+    # run on weights rounded beforehand, followed by rounding of the stored activation.
+    net = R.Net(1, 1, 6, (), (5,), "relu", 3, 1.0)
+    rng = np.random.default_rng(10)
+    p = rng.normal(size=R.param_count(net))
+    obs = _bf16_independent(rng.normal(size=(4, 6)))
+    off = R.param_offsets(net)
+    pr = p.copy()
+    pr[off["L0.W"]:off["L0.b"]] = _bf16_independent(p[off["L0.W"]:off["L0.b"]])
+    h_exact = R.forward(net, pr, obs, which_layer=0)[2]
+    z_b, v_b, h_b = R.forward(net.with_bf16(), p, obs, which_layer=0)
+    np.testing.assert_array_equal(h_b, _bf16_independent(h_exact))
+    W = p[off["pi.W"]:off["pi.b"]].reshape(3, 5)
+    np.testing.assert_allclose(z_b, h_b @ W.T + p[off["pi.b"]:off["pi.b"] + 3], rtol=1e-14)
+    # backward: gradient of the heads uses the rounded activation; the hidden layer's weight
+    # gradient uses the rounded pre-activation gradient
+    dz, dv = rng.normal(size=(4, 3)), rng.normal(size=4)
+    g = R.backward(net.with_bf16(), p, obs, dz, dv)
+    np.testing.assert_allclose(g[off["pi.W"]:off["pi.b"]].reshape(3, 5), dz.T @ h_b, rtol=1e-13)
+    dh = (dz @ W + np.outer(dv, p[off["v.W"]:off["v.W"] + 5])) * (h_b > 0)
+    dpre = _bf16_independent(dh)
+    np.testing.assert_allclose(g[off["L0.W"]:off["L0.b"]].reshape(5, 6), dpre.T @ obs, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(g[off["L0.b"]:off["L0.b"] + 5], dpre.sum(axis=0), rtol=1e-13, atol=1e-15)
+
+
+def test_bf16_operand_mode_stays_close_to_exact():
+    rng = np.random.default_rng(11)
+    net255 = R.Net(6, 6, 2, ((3, 1, 3), (2, 2, 4)), (8,), "relu", 3, 1.0 / 255.0)
+    p = rng.normal(size=R.param_count(net255)) * 0.4
+    obs = rng.integers(0, 256, size=(6, net255.in_size)).astype(np.float64)
+    z, v = R.forward(net255, p, obs)
+    zb, vb = R.forward(net255.with_bf16(), p, obs)
+    assert np.linalg.norm(zb - z) <= 2e-2 * np.linalg.norm(z)
+    assert np.linalg.norm(vb - v) <= 2e-2 * np.linalg.norm(v)
