@@ -184,6 +184,19 @@ int gala_set_stream(gala_ctx* ctx, int agent, void* cuda_stream);
 int gala_debug_read(gala_ctx* ctx, int agent, int what, float* out, long long count);
 /* Number of kernel launches issued by this context so far. */
 long long gala_launch_count(const gala_ctx* ctx);
+/* Kernel classes (im2col, each GEMM, sweeps, ...) for per-class accounting. */
+int gala_kernel_classes(void);
+const char* gala_kernel_class_name(int k);
+/* Bracket every launch of the classes in `mask` (bit k = class k) with CUDA timing events on the
+ * launching stream; 0 switches timing off.  Launch counts per class are always kept. */
+int gala_profile_enable(gala_ctx* ctx, unsigned long long mask);
+/* Waits for all work, then fills per class (arrays of gala_kernel_classes() entries, any may be
+ * NULL): summed device time in ms of the timed launches, how many launches were timed, and how
+ * many were issued since the last reset.  reset != 0 clears the counters and recorded events. */
+int gala_profile_read(gala_ctx* ctx, double* ms, long long* timed, long long* launches, int reset);
+/* The CUDA stream (cudaStream_t) an agent's work is enqueued on; agent < 0: the stream of the
+ * synchronous mode.  Owned by the library unless set by gala_set_stream. */
+void* gala_get_stream(gala_ctx* ctx, int agent);
 const char* gala_last_error(const gala_ctx* ctx);
 
 /* Stand-alone grouped GEMM on the tensor cores, exposed for validation:

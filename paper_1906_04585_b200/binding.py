@@ -54,7 +54,8 @@ EXPORTS = (
     "gala_sync_agent", "gala_sync_all", "gala_in_peers", "gala_get_state", "gala_set_state",
     "gala_set_grad", "gala_param_count", "gala_losses", "gala_stats", "gala_last_mix",
     "gala_get_snapshot", "gala_set_stream", "gala_debug_read", "gala_launch_count",
-    "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync",
+    "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync", "gala_kernel_classes",
+    "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
 )
 
 _lib = None
@@ -93,6 +94,11 @@ def lib() -> C.CDLL:
             "gala_debug_read": (i, [vp, i, i, vp, ll]),
             "gala_launch_count": (ll, [vp]),
             "gala_last_error": (C.c_char_p, [vp]),
+            "gala_kernel_classes": (i, []),
+            "gala_kernel_class_name": (C.c_char_p, [i]),
+            "gala_profile_enable": (i, [vp, C.c_ulonglong]),
+            "gala_profile_read": (i, [vp, C.POINTER(C.c_double), C.POINTER(ll), C.POINTER(ll), i]),
+            "gala_get_stream": (vp, [vp, i]),
             "gala_gemm_bf16": (i, [vp, vp, vp, i, i, i, i, i, i, i, vp]),
             "gala_sweep_sync": (i, [vp, vp, vp, vp, i, ll, C.POINTER(gala_topology), ll, C.POINTER(gala_hparams), vp]),
         }
@@ -234,6 +240,30 @@ def gala_debug_read(ctx, agent: int, what: int, count: int) -> np.ndarray:
 
 def gala_launch_count(ctx) -> int:
     return int(lib().gala_launch_count(ctx))
+
+
+def gala_kernel_classes() -> int:
+    return int(lib().gala_kernel_classes())
+
+
+def gala_kernel_class_name(k: int) -> str:
+    return lib().gala_kernel_class_name(k).decode()
+
+
+def gala_profile_enable(ctx, mask: int):
+    _check(ctx, lib().gala_profile_enable(ctx, mask))
+
+
+def gala_profile_read(ctx, reset: bool = True):
+    """{class name: (summed ms of timed launches, timed launches, launches issued)}"""
+    n = gala_kernel_classes()
+    ms, timed, launches = (C.c_double * n)(), (C.c_longlong * n)(), (C.c_longlong * n)()
+    _check(ctx, lib().gala_profile_read(ctx, ms, timed, launches, 1 if reset else 0))
+    return {gala_kernel_class_name(k): (ms[k], timed[k], launches[k]) for k in range(n)}
+
+
+def gala_get_stream(ctx, agent: int = -1) -> int:
+    return int(lib().gala_get_stream(ctx, agent) or 0)
 
 
 def gala_last_error(ctx) -> str:

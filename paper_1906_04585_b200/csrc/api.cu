@@ -33,8 +33,27 @@ struct Agent {
 struct Plan {  // one tensor-core product with its descriptors
     GemmOperand A, B;
     GemmArgs args;
-    long mask_stride = 0;
+    int tag = 0;
 };
+
+// Kernel classes for launch counting and optional per-class device timing.
+enum Tag : int {
+    T_IM2COL_U8 = 0, T_IM2COL_BF16, T_HEADS_FWD, T_LOSS, T_HEADS_BWD, T_COLSUM, T_SPLITK, T_COL2IM, T_GRAD_NORM,
+    T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST,
+    T_GEMM_CONV_FWD,          // +layer (3)
+    T_GEMM_FC_FWD = T_GEMM_CONV_FWD + 3, T_GEMM_FC_WGRAD, T_GEMM_FC_DGRAD,
+    T_GEMM_CONV_WGRAD,        // +layer (3)
+    T_GEMM_CONV_DGRAD = T_GEMM_CONV_WGRAD + 3,  // +layer (3)
+    T_COUNT = T_GEMM_CONV_DGRAD + 3
+};
+const char* const kTagNames[T_COUNT] = {
+    "im2col_u8", "im2col_bf16", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "col2im", "grad_norm",
+    "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16",
+    "gemm_conv1_fwd", "gemm_conv2_fwd", "gemm_conv3_fwd", "gemm_fc_fwd", "gemm_fc_wgrad", "gemm_fc_dgrad",
+    "gemm_conv1_wgrad", "gemm_conv2_wgrad", "gemm_conv3_wgrad", "gemm_conv1_dgrad", "gemm_conv2_dgrad",
+    "gemm_conv3_dgrad"};
+
+struct TimedLaunch { int tag; cudaEvent_t beg, end; };
 
 }  // namespace
 
@@ -54,6 +73,10 @@ struct gala_ctx {
     cudaEvent_t main_event = nullptr;
     long long sync_round = 0;
     long long launches = 0;
+    long long tag_launches[T_COUNT] = {};
+    unsigned long long profile_mask = 0;     // kernel classes bracketed by timing events
+    std::vector<TimedLaunch> timed;          // recorded, not yet read
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
     std::string err;
     std::vector<void*> allocs;
 
@@ -69,8 +92,8 @@ struct gala_ctx {
     float *h1 = nullptr, *h2 = nullptr, *dpre1 = nullptr, *dpre2 = nullptr;
     // conv workspaces (bf16)
     __nv_bfloat16 *cols[3] = {nullptr, nullptr, nullptr}, *act[3] = {nullptr, nullptr, nullptr};
-    __nv_bfloat16 *hid = nullptr, *dh = nullptr, *dy[3] = {nullptr, nullptr, nullptr},
-                  *dcols[3] = {nullptr, nullptr, nullptr};
+    __nv_bfloat16 *hid = nullptr, *dh = nullptr, *dy[3] = {nullptr, nullptr, nullptr};
+    float* dcols[3] = {nullptr, nullptr, nullptr};  // patch gradients stay fp32 until they are summed
     float* splitk_ws = nullptr;
     long splitk_group_stride = 0;
     int max_split = 32;
@@ -97,10 +120,38 @@ int fail(gala_ctx* c, int code, const char* fmt, ...) {
             return fail(c, e__ == cudaErrorMemoryAllocation ? GALA_ENOMEM : GALA_ECUDA, "%s: %s", #call, \
                         cudaGetErrorString(e__));                                                      \
     } while (0)
-#define LAUNCH(call)      \
-    do {                  \
-        CK(call);         \
-        c->launches++;    \
+// Launch bookkeeping: counts every kernel launch per class; classes selected by profile_mask are
+// bracketed by timing events on the launching stream.
+int prof_begin(gala_ctx* c, int tag, cudaStream_t st, TimedLaunch* t) {
+    t->tag = -1;
+    if (!((c->profile_mask >> tag) & 1ull)) return GALA_OK;
+    if (c->event_pool.empty()) {
+        cudaEvent_t a, b;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess)
+            return fail(c, GALA_ECUDA, "cudaEventCreate failed");
+        c->event_pool.push_back({a, b});
+    }
+    t->beg = c->event_pool.back().first; t->end = c->event_pool.back().second;
+    c->event_pool.pop_back();
+    t->tag = tag;
+    if (cudaEventRecord(t->beg, st) != cudaSuccess) return fail(c, GALA_ECUDA, "cudaEventRecord failed");
+    return GALA_OK;
+}
+int prof_end(gala_ctx* c, cudaStream_t st, TimedLaunch* t) {
+    if (t->tag < 0) return GALA_OK;
+    if (cudaEventRecord(t->end, st) != cudaSuccess) return fail(c, GALA_ECUDA, "cudaEventRecord failed");
+    c->timed.push_back(*t);
+    return GALA_OK;
+}
+#define LAUNCH(tag, st, call)                                    \
+    do {                                                         \
+        TimedLaunch tl__;                                        \
+        int pr__ = prof_begin(c, (tag), (st), &tl__);            \
+        if (pr__ != GALA_OK) return pr__;                        \
+        CK(call);                                                \
+        c->launches++;                                           \
+        c->tag_launches[(tag)]++;                                \
+        if ((pr__ = prof_end(c, (st), &tl__)) != GALA_OK) return pr__; \
     } while (0)
 
 template <typename Tp>
@@ -180,6 +231,7 @@ int build_plans(gala_ctx* c) {
         // forward: patches [B*P][KK] x W[CO][KK]^T -> act[l] (bias, ReLU; conv1 also 1/255)
         Plan& f = c->fwd[l];
         zero_args(f);
+        f.tag = T_GEMM_CONV_FWD + l;
         ok &= make_operand(&f.A, c->cols[l], 0, (uint64_t)B * P[l], KK, n, KK, (uint64_t)B * P[l] * KK, 128);
         ok &= make_operand(&f.B, c->shadow + c->cl.w[l], 0, CO, KK, n, KK, dp, bn);
         f.args.M = (int)(B * P[l]); f.args.N = CO; f.args.K = KK; f.args.block_n = bn;
@@ -190,6 +242,7 @@ int build_plans(gala_ctx* c) {
         // weight gradient, transposed product: (patches^T [KK x S*P]) x (dY [S*P x CO]) stored at W[co][kk]
         Plan& w = c->wgrad[l];
         zero_args(w);
+        w.tag = T_GEMM_CONV_WGRAD + l;
         ok &= make_operand(&w.A, c->cols[l], 1, KK, (uint64_t)S * P[l], n, KK, (uint64_t)B * P[l] * KK, 128);
         ok &= make_operand(&w.B, c->dy[l], 1, CO, (uint64_t)S * P[l], n, CO, (uint64_t)S * P[l] * CO, 64);
         w.args.M = KK; w.args.N = CO; w.args.K = (int)(S * P[l]); w.args.block_n = 64;
@@ -200,16 +253,18 @@ int build_plans(gala_ctx* c) {
         if (l > 0) {
             Plan& dg = c->dgrad[l];
             zero_args(dg);
+            dg.tag = T_GEMM_CONV_DGRAD + l;
             ok &= make_operand(&dg.A, c->dy[l], 0, (uint64_t)S * P[l], CO, n, CO, (uint64_t)S * P[l] * CO, 128);
             ok &= make_operand(&dg.B, c->shadow + c->cl.w[l], 1, KK, CO, n, KK, dp, 128);
             dg.args.M = (int)(S * P[l]); dg.args.N = KK; dg.args.K = CO; dg.args.block_n = 128;
-            dg.args.flags = EPI_OUT_BF16;
+            dg.args.flags = 0;
             dg.args.out = c->dcols[l]; dg.args.out_group_stride = S * P[l] * KK; dg.args.ldc = KK;
         }
     }
     {   // hidden layer forward: act3 [B][3136] x Wfc[512][3136]^T -> hid (bias, ReLU)
         Plan& f = c->fc_fwd;
         zero_args(f);
+        f.tag = T_GEMM_FC_FWD;
         ok &= make_operand(&f.A, c->act[2], 0, B, kFeat, n, kFeat, (uint64_t)B * kFeat, 128);
         ok &= make_operand(&f.B, c->shadow + c->cl.fcw, 0, kHidden, kFeat, n, kFeat, dp, 128);
         f.args.M = (int)B; f.args.N = kHidden; f.args.K = kFeat; f.args.block_n = 128;
@@ -219,6 +274,7 @@ int build_plans(gala_ctx* c) {
         // weight gradient: dh^T [512 x S] x act3 [S x 3136] -> gW[512][3136]
         Plan& w = c->fc_wgrad;
         zero_args(w);
+        w.tag = T_GEMM_FC_WGRAD;
         ok &= make_operand(&w.A, c->dh, 1, kHidden, S, n, kHidden, (uint64_t)S * kHidden, 128);
         ok &= make_operand(&w.B, c->act[2], 1, kFeat, S, n, kFeat, (uint64_t)B * kFeat, 128);
         w.args.M = kHidden; w.args.N = kFeat; w.args.K = (int)S; w.args.block_n = 128;
@@ -226,6 +282,7 @@ int build_plans(gala_ctx* c) {
         // data gradient: dh [S][512] x Wfc [512][3136] -> dY3 [S][3136], masked by act3 > 0
         Plan& dg = c->fc_dgrad;
         zero_args(dg);
+        dg.tag = T_GEMM_FC_DGRAD;
         ok &= make_operand(&dg.A, c->dh, 0, S, kHidden, n, kHidden, (uint64_t)S * kHidden, 128);
         ok &= make_operand(&dg.B, c->shadow + c->cl.fcw, 1, kFeat, kHidden, n, kFeat, dp, 128);
         dg.args.M = (int)S; dg.args.N = kFeat; dg.args.K = kHidden; dg.args.block_n = 128;
@@ -243,7 +300,7 @@ int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override,
     const bool bf = a.flags & EPI_OUT_BF16;
     a.out = reinterpret_cast<char*>(a.out) + (long)agent0 * a.out_group_stride * (bf ? 2 : 4);
     if (a.mask) a.mask += (long)agent0 * a.mask_group_stride;
-    LAUNCH(launch_gemm(p.A, p.B, a, st));
+    LAUNCH(p.tag, st, launch_gemm(p.A, p.B, a, st));
     return GALA_OK;
 }
 
@@ -262,8 +319,8 @@ int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t s
     a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
     a.out_group_stride = c->splitk_group_stride;
     a.out_split_stride = count;
-    LAUNCH(launch_gemm(p.A, p.B, a, st));
-    LAUNCH(launch_splitk_reduce(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
+    LAUNCH(p.tag, st, launch_gemm(p.A, p.B, a, st));
+    LAUNCH(T_SPLITK, st, launch_splitk_reduce(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
                                 reinterpret_cast<float*>(p.args.out) + (long)agent0 * p.args.out_group_stride, count,
                                 split, count, groups, c->splitk_group_stride, p.args.out_group_stride, st));
     return GALA_OK;
@@ -275,13 +332,13 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
     const long dp = c->d_pad, B = c->B;
     if (c->conv) {
         const int P[3] = {400, 81, 49};
-        LAUNCH(launch_im2col_u8(obs, c->cols[0] + (long)agent0 * B * 400 * 256, B * 400 * 256, rows, groups, st));
+        LAUNCH(T_IM2COL_U8, st, launch_im2col_u8(obs, c->cols[0] + (long)agent0 * B * 400 * 256, B * 400 * 256, rows, groups, st));
         for (int l = 0; l < 3; l++) {
             int r = run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st);
             if (r != GALA_OK) return r;
             if (l < 2) {
                 const long as = B * P[l] * kConvCout[l], cs = B * P[l + 1] * kConvKK[l + 1];
-                LAUNCH(launch_im2col_bf16(c->act[l] + (long)agent0 * as, as, c->cols[l + 1] + (long)agent0 * cs, cs,
+                LAUNCH(T_IM2COL_BF16, st, launch_im2col_bf16(c->act[l] + (long)agent0 * as, as, c->cols[l + 1] + (long)agent0 * cs, cs,
                                           l + 1, rows, groups, st));
             }
         }
@@ -294,7 +351,7 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         h.piw = c->cl.piw; h.pib = c->cl.pib; h.vw = c->cl.vw; h.vb = c->cl.vb;
         h.logits = c->logits + (long)agent0 * B * c->A; h.logits_stride = B * c->A;
         h.values = c->values + (long)agent0 * B; h.values_stride = B;
-        LAUNCH(launch_heads_fwd(h, groups, st));
+        LAUNCH(T_HEADS_FWD, st, launch_heads_fwd(h, groups, st));
     } else {
         const int H = c->H;
         DenseArgs a{};
@@ -302,13 +359,13 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         a.in = obs; a.in_bf16 = 0;
         a.W = c->x + (long)agent0 * dp + c->ml.w1; a.b = c->x + (long)agent0 * dp + c->ml.b1; a.w_stride = dp;
         a.out = c->h1 + (long)agent0 * B * H; a.out_stride = B * H; a.out_bf16 = 0;
-        LAUNCH(launch_dense_fwd(a, groups, st));
+        LAUNCH(T_DENSE_FWD, st, launch_dense_fwd(a, groups, st));
         DenseArgs b = a;
         b.in_dim = H;
         fill_batch(b.in, c->h1, B * H * 4, agent0, groups);
         b.W = c->x + (long)agent0 * dp + c->ml.w2; b.b = c->x + (long)agent0 * dp + c->ml.b2;
         b.out = c->h2 + (long)agent0 * B * H;
-        LAUNCH(launch_dense_fwd(b, groups, st));
+        LAUNCH(T_DENSE_FWD, st, launch_dense_fwd(b, groups, st));
         HeadsArgs h{};
         h.rows = rows; h.H = H; h.A = c->A;
         h.h = c->h2 + (long)agent0 * B * H; h.h_stride = B * H; h.h_bf16 = 0;
@@ -316,14 +373,14 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         h.piw = c->ml.piw; h.pib = c->ml.pib; h.vw = c->ml.vw; h.vb = c->ml.vb;
         h.logits = c->logits + (long)agent0 * B * c->A; h.logits_stride = B * c->A;
         h.values = c->values + (long)agent0 * B; h.values_stride = B;
-        LAUNCH(launch_heads_fwd(h, groups, st));
+        LAUNCH(T_HEADS_FWD, st, launch_heads_fwd(h, groups, st));
     }
     return GALA_OK;
 }
 
 int colsum(gala_ctx* c, const __nv_bfloat16* dy, long stride, long rows, int C, long grad_off, int agent0, int groups,
            cudaStream_t st) {
-    LAUNCH(launch_colsum(dy + (long)agent0 * stride, stride, rows, C, c->g + (long)agent0 * c->d_pad + grad_off,
+    LAUNCH(T_COLSUM, st, launch_colsum(dy + (long)agent0 * stride, stride, rows, C, c->g + (long)agent0 * c->d_pad + grad_off,
                          c->d_pad, c->colsum_partial + (long)agent0 * kColsumChunks * 512, c->colsum_ticket + agent0,
                          groups, st));
     return GALA_OK;
@@ -348,7 +405,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
     la.returns = c->returns + (long)agent0 * S; la.adv = c->adv + (long)agent0 * S;
     la.dlogits = c->dlogits + (long)agent0 * S * A; la.dvalues = c->dvalues + (long)agent0 * S;
     la.losses = c->losses + (long)agent0 * 4;
-    LAUNCH(launch_a2c_loss(la, groups, st));
+    LAUNCH(T_LOSS, st, launch_a2c_loss(la, groups, st));
 
     HeadsBwdArgs hb{};
     hb.rows = (int)S; hb.A = A;
@@ -362,8 +419,8 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hb.h = c->hid + (long)agent0 * B * kHidden; hb.h_stride = B * kHidden; hb.h_bf16 = 1;
         hb.piw = c->cl.piw; hb.pib = c->cl.pib; hb.vw = c->cl.vw; hb.vb = c->cl.vb;
         hb.dpre = c->dh + (long)agent0 * S * kHidden; hb.dpre_stride = S * kHidden; hb.dpre_bf16 = 1;
-        LAUNCH(launch_heads_bwd(hb, groups, st));
-        c->launches++;  // two kernels
+        LAUNCH(T_HEADS_BWD, st, launch_heads_bwd(hb, groups, st));
+        c->launches++; c->tag_launches[T_HEADS_BWD]++;  // two kernels
         if ((r = colsum(c, c->dh, S * kHidden, S, kHidden, c->cl.fcb, agent0, groups, st)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, st)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
@@ -375,7 +432,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
                 if ((r = run_plan(c, c->dgrad[l], agent0, groups, 0, st)) != GALA_OK) return r;
                 const long ds = S * P[l] * kConvKK[l], as = B * P[l - 1] * kConvCout[l - 1],
                            xs = S * P[l - 1] * kConvCout[l - 1];
-                LAUNCH(launch_col2im(c->dcols[l] + (long)agent0 * ds, ds, c->act[l - 1] + (long)agent0 * as, as,
+                LAUNCH(T_COL2IM, st, launch_col2im(c->dcols[l] + (long)agent0 * ds, ds, c->act[l - 1] + (long)agent0 * as, as,
                                      c->dy[l - 1] + (long)agent0 * xs, xs, l, (int)S, groups, st));
             }
         }
@@ -385,8 +442,8 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hb.h = c->h2 + (long)agent0 * B * H; hb.h_stride = B * H; hb.h_bf16 = 0;
         hb.piw = c->ml.piw; hb.pib = c->ml.pib; hb.vw = c->ml.vw; hb.vb = c->ml.vb;
         hb.dpre = c->dpre2 + (long)agent0 * S * H; hb.dpre_stride = S * H; hb.dpre_bf16 = 0;
-        LAUNCH(launch_heads_bwd(hb, groups, st));
-        c->launches++;
+        LAUNCH(T_HEADS_BWD, st, launch_heads_bwd(hb, groups, st));
+        c->launches++; c->tag_launches[T_HEADS_BWD]++;
         DenseBwdArgs d2{};
         d2.rows = (int)S; d2.in_dim = H; d2.out_dim = H; d2.act_in = 2;
         fill_batch(d2.in, c->h1, B * H * 4, agent0, groups);
@@ -394,8 +451,8 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         d2.W = c->x + (long)agent0 * dp + c->ml.w2; d2.w_stride = dp;
         d2.gW = c->g + (long)agent0 * dp + c->ml.w2; d2.gb = c->g + (long)agent0 * dp + c->ml.b2; d2.g_stride = dp;
         d2.din = c->dpre1 + (long)agent0 * S * H; d2.din_stride = S * H;
-        LAUNCH(launch_dense_bwd(d2, groups, st));
-        c->launches++;
+        LAUNCH(T_DENSE_BWD, st, launch_dense_bwd(d2, groups, st));
+        c->launches++; c->tag_launches[T_DENSE_BWD]++;
         DenseBwdArgs d1{};
         d1.rows = (int)S; d1.in_dim = c->obs_dim; d1.out_dim = H; d1.act_in = 0;
         d1.in = obs;
@@ -403,9 +460,9 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         d1.W = c->x + (long)agent0 * dp + c->ml.w1; d1.w_stride = dp;
         d1.gW = c->g + (long)agent0 * dp + c->ml.w1; d1.gb = c->g + (long)agent0 * dp + c->ml.b1; d1.g_stride = dp;
         d1.din = nullptr;
-        LAUNCH(launch_dense_bwd(d1, groups, st));
+        LAUNCH(T_DENSE_BWD, st, launch_dense_bwd(d1, groups, st));
     }
-    LAUNCH(launch_grad_norm(c->g, c->d, dp, agent0, groups, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
+    LAUNCH(T_GRAD_NORM, st, launch_grad_norm(c->g, c->d, dp, agent0, groups, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
                             c->norm, c->clip, st));
     for (int i = 0; i < groups; i++) {
         c->agents[agent0 + i].pending = true;
@@ -459,7 +516,7 @@ int sweep_agent(gala_ctx* c, int i, bool try_mix) {
         ag.skipped++;
     }
     SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
-    LAUNCH(launch_sweep_agent(c->x + (long)i * dp, ag.pending ? c->g + (long)i * dp : nullptr, c->v + (long)i * dp,
+    LAUNCH(T_SWEEP_AGENT, ag.stream, launch_sweep_agent(c->x + (long)i * dp, ag.pending ? c->g + (long)i * dp : nullptr, c->v + (long)i * dp,
                               c->snap + ((long)i * 2 + slot) * dp, p0, p1, fresh ? np : 0, c->clip + i,
                               c->conv ? c->shadow + (long)i * dp : nullptr, dp, hp, ag.stream));
     CK(cudaEventRecord(ag.pub_event[slot], ag.stream));
@@ -639,7 +696,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
             CK(cudaMemcpy(c->x + (long)i * dp, host.data(), dp * sizeof(float), cudaMemcpyHostToDevice));
         }
         if (c->conv) {
-            LAUNCH(launch_cast_bf16(c->x, c->shadow, (long)n * dp, c->main_stream));
+            LAUNCH(T_CAST, c->main_stream, launch_cast_bf16(c->x, c->shadow, (long)n * dp, c->main_stream));
             CK(cudaStreamSynchronize(c->main_stream));
         }
     }
@@ -658,6 +715,8 @@ int gala_destroy(gala_ctx* c) {
     }
     if (c->main_stream) cudaStreamDestroy(c->main_stream);
     if (c->main_event) cudaEventDestroy(c->main_event);
+    for (auto& t : c->timed) { cudaEventDestroy(t.beg); cudaEventDestroy(t.end); }
+    for (auto& e : c->event_pool) { cudaEventDestroy(e.first); cudaEventDestroy(e.second); }
     for (void* p : c->allocs) cudaFree(p);
     delete c;
     return GALA_OK;
@@ -672,7 +731,7 @@ int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int
     int r = forward(c, agent, 1, pb, c->E, ag.stream);
     if (r != GALA_OK) return r;
     if (actions)
-        LAUNCH(launch_sample(c->logits + (long)agent * c->B * c->A, uniforms, actions, c->E, c->A, ag.stream));
+        LAUNCH(T_SAMPLE, ag.stream, launch_sample(c->logits + (long)agent * c->B * c->A, uniforms, actions, c->E, c->A, ag.stream));
     if (values)
         CK(cudaMemcpyAsync(values, c->values + (long)agent * c->B, c->E * sizeof(float), cudaMemcpyDeviceToDevice,
                            ag.stream));
@@ -721,7 +780,7 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
     int off[2] = {0, 0};
     const int np = topo_offsets(c->topo, n, c->sync_round, off);
     SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
-    LAUNCH(launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp, st));
+    LAUNCH(T_SWEEP_SYNC, st, launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp, st));
     CK(cudaEventRecord(c->main_event, st));
     for (int i = 0; i < n; i++) {
         CK(cudaStreamWaitEvent(c->agents[i].stream, c->main_event, 0));
@@ -778,7 +837,7 @@ int gala_set_state(gala_ctx* c, int agent, const float* params, const float* sq_
     if (params) {
         CK(cudaMemcpy(c->x + (long)agent * c->d_pad, params, bytes, cudaMemcpyDefault));
         if (c->conv) {
-            LAUNCH(launch_cast_bf16(c->x + (long)agent * c->d_pad, c->shadow + (long)agent * c->d_pad, c->d_pad, ag.stream));
+            LAUNCH(T_CAST, ag.stream, launch_cast_bf16(c->x + (long)agent * c->d_pad, c->shadow + (long)agent * c->d_pad, c->d_pad, ag.stream));
             CK(cudaStreamSynchronize(ag.stream));
         }
     }
@@ -797,7 +856,7 @@ int gala_set_grad(gala_ctx* c, int agent, const float* grad, float clip_coef) {
     if (clip_coef >= 0.0f) {
         CK(cudaMemcpy(c->clip + agent, &clip_coef, sizeof(float), cudaMemcpyHostToDevice));
     } else {
-        LAUNCH(launch_grad_norm(c->g, c->d, c->d_pad, agent, 1, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
+        LAUNCH(T_GRAD_NORM, ag.stream, launch_grad_norm(c->g, c->d, c->d_pad, agent, 1, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
                                 c->norm, c->clip, ag.stream));
         CK(cudaStreamSynchronize(ag.stream));
     }
@@ -914,6 +973,45 @@ int gala_debug_read(gala_ctx* c, int agent, int what, float* out, long long coun
 }
 
 long long gala_launch_count(const gala_ctx* c) { return c ? c->launches : 0; }
+
+int gala_kernel_classes(void) { return T_COUNT; }
+
+const char* gala_kernel_class_name(int k) { return (k >= 0 && k < T_COUNT) ? kTagNames[k] : ""; }
+
+int gala_profile_enable(gala_ctx* c, unsigned long long mask) {
+    if (!c) return GALA_EINVAL;
+    c->profile_mask = mask;
+    return GALA_OK;
+}
+
+int gala_profile_read(gala_ctx* c, double* ms, long long* timed, long long* launches, int reset) {
+    if (!c) return GALA_EINVAL;
+    int r = gala_sync_all(c, -1);
+    if (r != GALA_OK) return r;
+    for (int k = 0; k < T_COUNT; k++) {
+        if (ms) ms[k] = 0.0;
+        if (timed) timed[k] = 0;
+        if (launches) launches[k] = c->tag_launches[k];
+    }
+    for (auto& t : c->timed) {
+        float f = 0.0f;
+        CK(cudaEventElapsedTime(&f, t.beg, t.end));
+        if (ms) ms[t.tag] += f;
+        if (timed) timed[t.tag]++;
+    }
+    if (reset) {
+        for (auto& t : c->timed) c->event_pool.push_back({t.beg, t.end});
+        c->timed.clear();
+        for (int k = 0; k < T_COUNT; k++) c->tag_launches[k] = 0;
+    }
+    return GALA_OK;
+}
+
+void* gala_get_stream(gala_ctx* c, int agent) {
+    if (!c) return nullptr;
+    if (agent < 0) return c->main_stream;
+    return agent < c->n ? c->agents[agent].stream : nullptr;
+}
 
 const char* gala_last_error(const gala_ctx* c) { return c ? c->err.c_str() : "null context"; }
 

@@ -171,7 +171,7 @@ cudaError_t launch_im2col_u8(const PtrBatch& obs, __nv_bfloat16* cols, long cols
 cudaError_t launch_im2col_bf16(const __nv_bfloat16* act, long act_group_stride, __nv_bfloat16* cols,
                                long cols_group_stride, int layer, int samples, int groups, cudaStream_t st);
 // dX = mask(act_in > 0) * scatter-sum of dcols; layer = 1 or 2 (conv2, conv3)
-cudaError_t launch_col2im(const __nv_bfloat16* dcols, long dcols_group_stride, const __nv_bfloat16* act_in,
+cudaError_t launch_col2im(const float* dcols, long dcols_group_stride, const __nv_bfloat16* act_in,
                           long act_group_stride, __nv_bfloat16* dx, long dx_group_stride, int layer,
                           int samples, int groups, cudaStream_t st);
 // out[g][c] = sum_r dy[g][r][c]   (bf16 in, fp32 out at out + g*out_stride), fixed summation order

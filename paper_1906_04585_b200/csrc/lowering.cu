@@ -94,16 +94,16 @@ cudaError_t launch_im2col_bf16(const __nv_bfloat16* act, long act_group_stride, 
     return cudaGetLastError();
 }
 
-// Adjoint of the lowering, gather form: every input pixel sums the patch-gradient entries that
-// were copied from it, in a fixed order, then the ReLU derivative of that pixel's forward
-// activation is applied.  One thread per (pixel, 8 channels).
-__global__ void __launch_bounds__(256) col2im_kernel(const __nv_bfloat16* __restrict__ dcols, long dcols_group_stride,
+// Adjoint of the lowering, gather form: every input pixel sums the fp32 patch-gradient entries
+// that were copied from it, in a fixed order, then the ReLU derivative of that pixel's forward
+// activation is applied and the result is stored in bf16.  One thread per (pixel, 8 channels).
+__global__ void __launch_bounds__(256) col2im_kernel(const float* __restrict__ dcols, long dcols_group_stride,
                                                      const __nv_bfloat16* __restrict__ act_in, long act_group_stride,
                                                      __nv_bfloat16* __restrict__ dx, long dx_group_stride, int layer,
                                                      int samples) {
     const ConvGeom cg = conv_geom(layer);
     const int g = blockIdx.y;
-    const uint4* src = reinterpret_cast<const uint4*>(dcols + (long)g * dcols_group_stride);
+    const float4* src = reinterpret_cast<const float4*>(dcols + (long)g * dcols_group_stride);
     const uint4* act = reinterpret_cast<const uint4*>(act_in + (long)g * act_group_stride);
     uint4* dst = reinterpret_cast<uint4*>(dx + (long)g * dx_group_stride);
     const int pix_chunks = cg.cin / 8;
@@ -126,13 +126,10 @@ __global__ void __launch_bounds__(256) col2im_kernel(const __nv_bfloat16* __rest
                 if (x - kx < 0) break;
                 if (ox >= cg.out) continue;
                 const long patch = (long)b * P + oy * cg.out + ox;
-                const uint4 v = __ldg(src + patch * patch_chunks + ky * row_chunks + kx * pix_chunks + cc);
-                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-                for (int q = 0; q < 4; q++) {
-                    float2 f = __bfloat1622float2(h[q]);
-                    acc[2 * q] += f.x; acc[2 * q + 1] += f.y;
-                }
+                const float4* v = src + (patch * patch_chunks + ky * row_chunks + kx * pix_chunks + cc) * 2;
+                const float4 v0 = __ldg(v), v1 = __ldg(v + 1);
+                acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+                acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
             }
         }
         const uint4 a = __ldg(act + idx);
@@ -147,7 +144,7 @@ __global__ void __launch_bounds__(256) col2im_kernel(const __nv_bfloat16* __rest
         dst[idx] = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
-cudaError_t launch_col2im(const __nv_bfloat16* dcols, long dcols_group_stride, const __nv_bfloat16* act_in,
+cudaError_t launch_col2im(const float* dcols, long dcols_group_stride, const __nv_bfloat16* act_in,
                           long act_group_stride, __nv_bfloat16* dx, long dx_group_stride, int layer, int samples,
                           int groups, cudaStream_t st) {
     const ConvGeom cg = conv_geom(layer);

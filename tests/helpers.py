@@ -27,8 +27,13 @@ def assert_close(name, got, want, tol):
     return rel
 
 
-def oracle_net(w: GI.Workload) -> R.Net:
-    return R.Net.atari(w.n_actions) if w.net_kind == "conv" else R.Net.mlp(w.obs_dim, w.hidden, w.n_actions)
+def oracle_net(w: GI.Workload, exact: bool = False) -> R.Net:
+    """The oracle's network for a workload.  The conv workloads are specified with bf16 GEMM
+    operands, so their oracle rounds the contraction operands to bf16 (exact sums); `exact`
+    asks for the unrounded fp64 network instead."""
+    if w.net_kind == "conv":
+        return R.Net.atari(w.n_actions).with_bf16(not exact)
+    return R.Net.mlp(w.obs_dim, w.hidden, w.n_actions)
 
 
 def oracle_hp(hp) -> R.HParams:
@@ -43,3 +48,11 @@ def to_bf16_f64(a: np.ndarray) -> np.ndarray:
     u = np.ascontiguousarray(a, np.float32).view(np.uint32).astype(np.uint64)
     u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
     return u.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def assert_grad_close(name, got, want, net: R.Net, tol):
+    """The tolerance rule applied per parameter tensor (conv1.W, conv1.b, ..., v.b)."""
+    off = R.param_offsets(net)
+    bounds = sorted((v, k) for k, v in off.items())
+    for (lo, key), (hi, _) in zip(bounds[:-1], bounds[1:]):
+        assert_close("%s/%s" % (name, key), np.asarray(got)[lo:hi], np.asarray(want)[lo:hi], tol)
