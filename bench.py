@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Throughput of the GALA-A2C learner step on B200.
+
+One "step" is one synchronous round of the whole learner path for all agents
+of the workload: network forward/backward over each agent's rollout, returns
+/ advantages / A2C objective, global-norm clip, and the fused RMSProp + gossip
+pass.  Default workload: 8 agents, conv net on 84x84x4 frames, 16 envs x 5
+steps per agent, 1-peer exponential graph (synthetic rollouts).
+
+  python bench.py [--gpus N --steps K --warmup W]            the CUDA library
+  python bench.py --impl reference [...]                     the fp64 CPU oracle
+
+Prints one JSON line on rank 0.  With N > 1 (torchrun) every rank runs an
+independent replica of the workload on its own GPU (the path has no
+cross-GPU exchange); the value is the sum over ranks over the slowest rank's
+time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gala_inputs as GI  # noqa: E402
+
+METRIC = "learner frames/s for N agents on 1 B200"
+UNIT = "frames/s"
+L2_BYTES = 126 * 1024 * 1024
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture of the named kernel
+# class on this workload; None until captured, and again None once that kernel changes.
+NCU_TRAFFIC_BYTES = {}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=float(p["hbm_gbs"]), tensor=float(p["bf16_tflops_sustained"]), source="measured")
+    return dict(hbm=6650.0, tensor=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------- work per class
+def class_work(w: GI.Workload, d_pad: int):
+    """Algorithmic work of one step per kernel class: name -> (bound, amount), amount in bytes
+    (hbm) or flops (tensor), summed over the launches of that class in one step."""
+    n, E, T, A = w.n_agents, w.n_envs, w.n_steps, w.n_actions
+    B, S = (T + 1) * E, T * E
+    out = {"sweep_sync": ("hbm", n * d_pad * (22.0 if w.net_kind == "conv" else 20.0)),
+           "grad_norm": ("hbm", n * d_pad * 4.0)}
+    if w.net_kind != "conv":
+        return out
+    P, KK, CO = (400, 81, 49), (256, 512, 576), (32, 64, 64)
+    out["im2col_u8"] = ("hbm", n * B * (84 * 84 * 4 + 400 * 256 * 2.0))
+    out["im2col_bf16"] = ("hbm", n * B * ((400 * 32 + 81 * 512) * 2.0 + (81 * 64 + 49 * 576) * 2.0))
+    for l in range(3):
+        out["gemm_conv%d_fwd" % (l + 1)] = ("tensor", 2.0 * n * B * P[l] * KK[l] * CO[l])
+        out["gemm_conv%d_wgrad" % (l + 1)] = ("tensor", 2.0 * n * S * P[l] * KK[l] * CO[l])
+        if l > 0:
+            out["gemm_conv%d_dgrad" % (l + 1)] = ("tensor", 2.0 * n * S * P[l] * KK[l] * CO[l])
+    out["gemm_fc_fwd"] = ("tensor", 2.0 * n * B * 3136 * 512)
+    out["gemm_fc_wgrad"] = ("tensor", 2.0 * n * S * 3136 * 512)
+    out["gemm_fc_dgrad"] = ("tensor", 2.0 * n * S * 3136 * 512)
+    out["col2im"] = ("hbm", n * S * ((49 * 576 * 4.0 + 81 * 64 * 4.0) + (81 * 512 * 4.0 + 400 * 32 * 4.0)))
+    out["colsum"] = ("hbm", n * S * (512 + 49 * 64 + 81 * 64 + 400 * 32) * 2.0)
+    return out
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu = gpu_index
+        self.path = os.path.join(ROOT, "gpurun_out", "bench_clocks_%d.csv" % os.getpid())
+
+    def start(self):
+        try:
+            os.makedirs(os.path.dirname(self.path), exist_ok=True)
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if sm:
+            out = dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_rate(w: GI.Workload, n_envs: int, workers: int, agents: int = 1):
+    """Frames/s of the oracle on `agents` agents' rollouts cut down to n_envs environments (learner
+    step + optimiser/gossip pass per agent).  Returns (frames_per_s, seconds)."""
+    from oracle import reference as R
+    net = R.Net.atari(w.n_actions).with_bf16() if w.net_kind == "conv" else R.Net.mlp(w.obs_dim, w.hidden, w.n_actions)
+    hp = R.HParams()
+    ws = w.scaled(n_envs=n_envs)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed).astype(np.float64)
+    v0 = np.zeros_like(p0)
+    ros = [GI.rollout(ws, i, 0) for i in range(agents)]
+    t0 = time.perf_counter()
+    for ro in ros:
+        info = R.learner_grad(net, p0, ro, hp, workers=workers)
+        R.sweep_replay(p0, info["grad"], v0, hp, [p0])
+    dt = time.perf_counter() - t0
+    return agents * n_envs * w.n_steps / dt, dt
+
+
+def usable_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = GI.WORKLOADS[args.workload]
+    cores = usable_cores()
+    workers = min(cores, 16)
+    _, t1 = oracle_sample_rate(w, 1, workers)                 # calibration on one environment
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n_envs = int(max(1, min(w.n_envs, budget / max(t1, 1e-3))))
+    for _ in range(args.warmup):
+        oracle_sample_rate(w, n_envs, workers)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_rate(w, n_envs, workers)
+    dt = time.perf_counter() - t0
+    value = args.steps * n_envs * w.n_steps / dt
+    sample = "per step: 1 of %d agents, %d of %d envs x %d steps, learner step + optimiser/gossip pass" % (
+        w.n_agents, n_envs, w.n_envs, w.n_steps)
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * dt / args.steps, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=w.name, sample=sample),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=workers, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- the CUDA library
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1906_04585_b200 import binding as B
+    from paper_1906_04585_b200 import learner as LM
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = GI.WORKLOADS[args.workload]
+    L = LM.Learner(w.n_agents, w.topo_kind, w.topo_peers, w.net_kind, w.n_actions, w.n_envs, w.n_steps,
+                   obs_dim=w.obs_dim, hidden=w.hidden)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    for i in range(w.n_agents):
+        L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32))
+    ext = torch.cuda.ExternalStream(B.gala_get_stream(L.ctx, -1))
+
+    n_sets = 4
+    sets = [[LM.DeviceRollout(GI.rollout(w, i, s + 1000 * rank), pinned=True) for i in range(w.n_agents)]
+            for s in range(n_sets)]
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+    n_classes = B.gala_kernel_classes()
+    work = class_work(w, L.d_pad)
+
+    # warm-up; the first steps time every kernel class to find the dominant one
+    B.gala_profile_enable(L.ctx, (1 << n_classes) - 1)
+    for k in range(max(3, args.warmup)):
+        L.step_sync(sets[k % n_sets])
+    prof_all = B.gala_profile_read(L.ctx, reset=True)
+    per_class_ms = {k: v[0] / max(3, args.warmup) for k, v in prof_all.items() if v[1] > 0}
+    dominant = max(per_class_ms, key=per_class_ms.get)
+    dom_index = [B.gala_kernel_class_name(k) for k in range(n_classes)].index(dominant)
+    B.gala_profile_enable(L.ctx, 1 << dom_index)
+
+    # timed region: K steps, device time per step from events on the launching stream, L2 flushed
+    # between steps (outside the per-step event pairs)
+    clocks = ClockSampler(local)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    clocks.start()
+    launches0 = L.launches()
+    t_wall0 = time.perf_counter()
+    for k in range(args.steps):
+        with torch.cuda.stream(ext):
+            flush.zero_()
+        ev[k][0].record(ext)
+        L.step_sync(sets[k % n_sets])
+        ev[k][1].record(ext)
+    L.sync()
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    launches = L.launches() - launches0
+    clk = clocks.stop()
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(step_ms))
+    prof = B.gala_profile_read(L.ctx, reset=True)
+    B.gala_profile_enable(L.ctx, 0)
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    frames = w.frames_per_round * args.steps * world
+    value = frames / (total_ms * 1e-3)
+
+    # roofline of the dominant kernel class, from its own events inside the timed region
+    pk = peaks()
+    dom_ms, dom_timed, _ = prof[dominant]
+    bound, amount = work.get(dominant, ("hbm", 0.0))
+    per_step_ms = dom_ms / max(1, args.steps)
+    if bound == "hbm":
+        achieved = amount / (per_step_ms * 1e-3) / 1e9 if per_step_ms > 0 else 0.0
+        peak, unit = pk["hbm"], "GB/s"
+    else:
+        achieved = amount / (per_step_ms * 1e-3) / 1e12 if per_step_ms > 0 else 0.0
+        peak, unit = pk["tensor"], "TFLOP/s"
+    roofline = dict(kernel=dominant, bound=bound, achieved=achieved, peak=peak, unit=unit, frac=achieved / peak,
+                    peak_source=pk["source"], traffic=NCU_TRAFFIC_BYTES.get(dominant),
+                    ms_per_step=per_step_ms, launches_timed=int(dom_timed),
+                    share_of_step=per_step_ms / (total_ms / args.steps) if total_ms > 0 else None)
+
+    # end to end through the public API with host buffers: pinned host -> device copy of the step's
+    # rollouts, the step, and a device -> host read of the step's losses, all inside the timed region
+    h2d = sum(r.nbytes for r in sets[0])
+    for k in range(2):
+        for r in sets[k % n_sets]:
+            r.upload(ext)
+        L.step_sync(sets[k % n_sets])
+        B.gala_losses(L.ctx, 0)
+    barrier()
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        cur = sets[k % n_sets]
+        for r in cur:
+            r.upload(ext)
+        L.step_sync(cur)
+        for i in range(w.n_agents):
+            B.gala_losses(L.ctx, i)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = dict(value=frames / e2e_s, unit=UNIT, h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=16 * w.n_agents)
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(3, args.warmup),
+                ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16" if w.net_kind == "conv" else "f32", data="synthetic",
+                config=dict(workload=w.name, n_agents=w.n_agents, envs_per_agent=w.n_envs, n_steps=w.n_steps,
+                            frames_per_step=w.frames_per_round, topology="exp1" if w.topo_kind == GI.EXP else "ring1",
+                            mode="synchronous round (gala_step_sync)", l2="flushed between steps (252 MiB write)",
+                            multi_gpu="replicas only" if world > 1 else "single"),
+                clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roofline,
+                wall_ms_per_step=1e3 * t_wall / args.steps,
+                kernel_ms_per_step={k: round(v, 5) for k, v in sorted(per_class_ms.items(), key=lambda kv: -kv[1])})
+
+    if rank == 0 and world == 1:
+        line["sweep_microbench"] = sweep_microbench(torch, B, pk)
+        if not args.no_cpu_baseline:
+            cores = usable_cores()
+            workers = min(cores, 16)
+            v, dt = oracle_sample_rate(w, w.n_envs, workers, agents=w.n_agents)
+            line["cpu_baseline"] = dict(value=v, unit=UNIT, cores=workers, kind="oracle",
+                                        sample="one full round: %d agents x (%d envs x %d steps), learner step + "
+                                               "optimiser/gossip pass per agent, %.1f s" % (w.n_agents, w.n_envs,
+                                                                                            w.n_steps, dt))
+    L.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def sweep_microbench(torch, B, pk):
+    """Fused RMSProp + gossip pass alone: 32 agents x 1.7M fp32 parameters, 100 rounds, 1- and
+    2-peer exponential graphs; 20 algorithmic bytes per parameter (read x, g, v; write x, v)."""
+    w = GI.WORKLOADS[3]
+    n, d = w.n_agents, w.sweep_only_d
+    x, g, v = GI.sweep_state(n, d, w.seed)
+    tx, tg, tv = (torch.from_numpy(t).cuda() for t in (x, g, v))
+    hp = B.default_hparams(1, 1, max_grad_norm=0.0)
+    st = torch.cuda.current_stream()
+    out = {}
+    for peers in (1, 2):
+        topo = B.gala_topology(B.GALA_TOPO_EXP, peers)
+        for k in range(5):
+            B.gala_sweep_sync(tx, tg, tv, None, n, d, topo, k, hp, st.cuda_stream)
+        torch.cuda.synchronize()
+        rounds = 100
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for k in range(rounds):
+            B.gala_sweep_sync(tx, tg, tv, None, n, d, topo, k, hp, st.cuda_stream)
+        e1.record(st)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / rounds
+        gbs = 20.0 * n * d / (ms * 1e-3) / 1e9
+        out["exp%d" % peers] = dict(ms_per_round=ms, achieved_gbs=gbs, frac_of_measured_peak=gbs / pk["hbm"],
+                                    frac_of_8tbs=gbs / 8000.0)
+    out["config"] = dict(workload=w.name, n_agents=n, d=d, rounds=100, bytes_per_param=20,
+                         working_set_mb=round(3 * n * d * 4 / 1e6, 1), l2="working set 653 MB > L2, no flush")
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=1, help="index into gala_inputs.WORKLOADS (1 = the headline)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
