@@ -91,7 +91,7 @@ class ClockSampler:
             os.makedirs(os.path.dirname(self.path), exist_ok=True)
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -315,6 +315,11 @@ def run_ours(args):
                                         sample="one full round: %d agents x (%d envs x %d steps), learner step + "
                                                "optimiser/gossip pass per agent, %.1f s" % (w.n_agents, w.n_envs,
                                                                                             w.n_steps, dt))
+    # release every tensor that was used on the library's stream while that stream still exists
+    del sets, flush, ev, cur
+    import gc
+    gc.collect()
+    torch.cuda.synchronize()
     L.close()
     if rank == 0:
         print(json.dumps(line))

@@ -12,18 +12,28 @@ TOL_FP32_NET = 1e-4   # fp32 network (MLP) outputs and gradients
 TOL_BF16 = 2e-2       # bf16-operand GEMM outputs and gradients
 
 
-def assert_close(name, got, want, tol):
-    """Per tensor: ||a-b||_2 <= tol ||b||_2  and  |a_i-b_i| <= tol (|b_i| + rms(b))."""
+def assert_close(name, got, want, tol, rule="elementwise"):
+    """Per tensor.  Both rules demand ||a-b||_2 <= tol ||b||_2.
+    rule "elementwise" (fp32 paths) adds |a_i-b_i| <= tol (|b_i| + rms(b)) for every element.
+    rule "norm" (bf16-operand paths) adds max|a_i-b_i| <= tol max|b_i| instead: a stored bf16 operand
+    that lands one unit in the last place apart on the two sides (fp32 vs exact accumulation next to a
+    rounding boundary) moves a single product by 0.4 %, which can exceed tol * rms(b) on an element
+    whose terms are far larger than the tensor's typical entry, but never tol * max|b|."""
     a = np.asarray(got, np.float64).ravel()
     b = np.asarray(want, np.float64).ravel()
     assert a.shape == b.shape, (name, a.shape, b.shape)
     assert np.isfinite(a).all(), name + ": non-finite values"
     nb = np.linalg.norm(b)
     rel = np.linalg.norm(a - b) / (nb if nb > 0 else 1.0)
-    rms = nb / np.sqrt(max(1, b.size))
-    worst = np.max(np.abs(a - b) / (np.abs(b) + rms + 1e-30)) if b.size else 0.0
     assert rel <= tol, "%s: relative l2 error %.3e > %.1e" % (name, rel, tol)
-    assert worst <= tol, "%s: worst element error %.3e > %.1e (rel l2 %.3e)" % (name, worst, tol, rel)
+    if not b.size:
+        return rel
+    if rule == "elementwise":
+        rms = nb / np.sqrt(b.size)
+        worst = np.max(np.abs(a - b) / (np.abs(b) + rms + 1e-30))
+    else:
+        worst = np.max(np.abs(a - b)) / (np.max(np.abs(b)) + 1e-30)
+    assert worst <= tol, "%s: worst element error %.3e > %.1e (rel l2 %.3e, rule %s)" % (name, worst, tol, rel, rule)
     return rel
 
 
@@ -50,9 +60,9 @@ def to_bf16_f64(a: np.ndarray) -> np.ndarray:
     return u.astype(np.uint32).view(np.float32).astype(np.float64)
 
 
-def assert_grad_close(name, got, want, net: R.Net, tol):
+def assert_grad_close(name, got, want, net: R.Net, tol, rule="elementwise"):
     """The tolerance rule applied per parameter tensor (conv1.W, conv1.b, ..., v.b)."""
     off = R.param_offsets(net)
     bounds = sorted((v, k) for k, v in off.items())
     for (lo, key), (hi, _) in zip(bounds[:-1], bounds[1:]):
-        assert_close("%s/%s" % (name, key), np.asarray(got)[lo:hi], np.asarray(want)[lo:hi], tol)
+        assert_close("%s/%s" % (name, key), np.asarray(got)[lo:hi], np.asarray(want)[lo:hi], tol, rule)
