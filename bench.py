@@ -205,6 +205,7 @@ def run_ours(args):
     for i in range(w.n_agents):
         L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32))
     ext = torch.cuda.ExternalStream(B.gala_get_stream(L.ctx, -1))
+    up = torch.cuda.Stream()      # host -> device copies run on a torch stream; the library's stream waits on it
 
     n_sets = 4
     sets = [[LM.DeviceRollout(GI.rollout(w, i, s + 1000 * rank), pinned=True) for i in range(w.n_agents)]
@@ -274,7 +275,8 @@ def run_ours(args):
     h2d = sum(r.nbytes for r in sets[0])
     for k in range(2):
         for r in sets[k % n_sets]:
-            r.upload(ext)
+            r.upload(up)
+        ext.wait_stream(up)
         L.step_sync(sets[k % n_sets])
         B.gala_losses(L.ctx, 0)
     barrier()
@@ -282,7 +284,8 @@ def run_ours(args):
     for k in range(args.steps):
         cur = sets[k % n_sets]
         for r in cur:
-            r.upload(ext)
+            r.upload(up)
+        ext.wait_stream(up)
         L.step_sync(cur)
         for i in range(w.n_agents):
             B.gala_losses(L.ctx, i)
@@ -316,7 +319,7 @@ def run_ours(args):
                                                "optimiser/gossip pass per agent, %.1f s" % (w.n_agents, w.n_envs,
                                                                                             w.n_steps, dt))
     # release every tensor that was used on the library's stream while that stream still exists
-    del sets, flush, ev, cur
+    del sets, flush, ev, cur, r
     import gc
     gc.collect()
     torch.cuda.synchronize()
