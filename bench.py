@@ -77,7 +77,7 @@ def class_work(w: GI.Workload, d_pad: int):
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -96,7 +96,11 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin: float, t_end: float):
+        """Median SM clock and throttle reasons over the samples taken inside [t_begin, t_end]
+        (time.time() values); if the region was shorter than one sampling period, over the
+        samples nearest to it."""
+        import datetime
         out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
         if self.proc is None:
             return out
@@ -106,22 +110,25 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.f.close()
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in open(self.path):
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[1])); mx.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]),
+                             [nm for nm, val in zip(names, parts[5:9]) if val.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, val in zip(names, parts[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        if sm:
-            out = dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
-                       samples=len(sm))
+        inside = [r for r in rows if t_begin - 0.02 <= r[0] <= t_end + 0.02]
+        if not inside and rows:
+            mid = 0.5 * (t_begin + t_end)
+            inside = sorted(rows, key=lambda r: abs(r[0] - mid))[:3]
+        if inside:
+            out = dict(sm_mhz=float(np.median([r[1] for r in inside])), sm_max_mhz=float(max(r[2] for r in inside)),
+                       reasons=sorted({nm for r in inside for nm in r[3]}), samples=len(inside))
         return out
 
 
@@ -228,9 +235,11 @@ def run_ours(args):
     # between steps (outside the per-step event pairs)
     clocks = ClockSampler(local)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
     clocks.start()
+    time.sleep(0.3)               # let the sampler come up; only samples inside the timed region are used
+    barrier()
     launches0 = L.launches()
+    t_clock0 = time.time()
     t_wall0 = time.perf_counter()
     for k in range(args.steps):
         with torch.cuda.stream(ext):
@@ -242,7 +251,7 @@ def run_ours(args):
     barrier()
     t_wall = time.perf_counter() - t_wall0
     launches = L.launches() - launches0
-    clk = clocks.stop()
+    clk = clocks.stop(t_clock0, time.time())
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = float(sum(step_ms))
     prof = B.gala_profile_read(L.ctx, reset=True)
@@ -364,7 +373,7 @@ def sweep_microbench(torch, B, pk):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="index into gala_inputs.WORKLOADS (1 = the headline)")
