@@ -22,6 +22,9 @@ class DeviceRollout:
             self.upload()
         else:
             self.t = {k: torch.from_numpy(np.ascontiguousarray(v)).to(device) for k, v in ro.items()}
+        # The copies above run on torch's stream; the library works on streams of its own that do not
+        # order themselves against it, so the data must have landed before the rollout is handed over.
+        torch.cuda.current_stream().synchronize()
         self.c = B.make_rollout(self.t["obs"], self.t["actions"], self.t["rewards"], self.t["dones"])
 
     def upload(self, stream: Optional[torch.cuda.Stream] = None):
@@ -98,6 +101,7 @@ class Learner:
         B.gala_gossip(self.ctx, agent)
 
     def act(self, agent: int, obs: torch.Tensor, uniforms: torch.Tensor):
+        torch.cuda.current_stream().synchronize()   # obs / uniforms may still be in flight on torch's stream
         actions = torch.empty(self.E, dtype=torch.int32, device=obs.device)
         values = torch.empty(self.E, dtype=torch.float32, device=obs.device)
         B.gala_act(self.ctx, agent, obs, uniforms, actions, values)

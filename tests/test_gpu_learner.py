@@ -148,7 +148,9 @@ def test_act_sampling_matches_oracle():
     p0 = GI.init_params(GI.net_tensors(w), w.seed)
     obs = GI.rollout(w, 0, 0)["obs"][0]
     u = GI.uniforms(w, 0, 0, w.n_envs)
-    a, v = L.act(0, torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())
+    t_obs, t_u = torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda()
+    torch.cuda.synchronize()      # uploads run on torch's stream, the library on its own
+    a, v = L.act(0, t_obs, t_u)
     L.sync()
     z, val = R.forward(net, p0, obs)
     want = R.sample(z, u)
