@@ -210,6 +210,28 @@ const char* gala_last_error(const gala_ctx* ctx);
 int gala_gemm_bf16(const void* A, const void* B, float* D, int groups, int M, int N, int K,
                    int a_mn, int b_mn, int split_k, void* stream);
 
+/* gala_gemm_bf16 without any allocation (this entry point has no counterpart in the paper; it
+ * exists for the way the library gets embedded).  gala_gemm_bf16 obtains its split-K scratch with
+ * cudaMalloc / cudaFree.  Some hosts of this library cannot afford that: a process in which a
+ * framework's caching allocator already holds almost all device memory (the allocation may simply
+ * fail), or a serving / control loop with a fixed memory plan, where the device-wide
+ * synchronisation inside cudaMalloc and cudaFree stalls every other stream.  This variant computes
+ * the same product -- same arguments, same kernels, same summation order -- but keeps its scratch
+ * in an 8 MiB array built into the library image (held by every GPU that loads the library, from
+ * load until exit) and calls no allocating routine.
+ *   Limit: groups * split_k * M * N <= 2 Mi floats when split_k > 1; beyond that the call is
+ *   refused with GALA_EINVAL and a message naming the limit (no limit for split_k == 1).
+ *   First call on each device: looks up the array's device address and resolves the tensor-map
+ *   encoder; make that first call outside any stream capture.
+ *   All calls share the one array, which keeps the previous call's contents (the call clears the
+ *   only word that must start at zero).  Two calls whose GPU work overlaps -- different streams,
+ *   threads or processes' contexts on the same device and library image -- race on it; this entry
+ *   point waits for its own work before returning, so successive calls from one thread are safe.
+ * errbuf (may be NULL) receives a NUL-terminated message of at most errbuf_len bytes on failure.
+ * Returns GALA_OK, GALA_EINVAL or GALA_ECUDA. */
+int gala_gemm_bf16_static(const void* A, const void* B, float* D, int groups, int M, int N, int K,
+                          int a_mn, int b_mn, int split_k, void* stream, char* errbuf, int errbuf_len);
+
 /* Stand-alone fused RMSProp + gossip pass over caller-owned arrays, exposed
  * for the optimiser micro-benchmark and its parity test (Algorithm 1 optimiser
  * and gossip steps; Eq. 7).  x, g, v: DEVICE float32 [n_agents][d_padded],

@@ -56,6 +56,7 @@ EXPORTS = (
     "gala_get_snapshot", "gala_set_stream", "gala_debug_read", "gala_launch_count",
     "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync", "gala_kernel_classes",
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
+    "gala_gemm_bf16_static",
 )
 
 _lib = None
@@ -100,6 +101,7 @@ def lib() -> C.CDLL:
             "gala_profile_read": (i, [vp, C.POINTER(C.c_double), C.POINTER(ll), C.POINTER(ll), i]),
             "gala_get_stream": (vp, [vp, i]),
             "gala_gemm_bf16": (i, [vp, vp, vp, i, i, i, i, i, i, i, vp]),
+            "gala_gemm_bf16_static": (i, [vp, vp, vp, i, i, i, i, i, i, i, vp, C.c_char_p, i]),
             "gala_sweep_sync": (i, [vp, vp, vp, vp, i, ll, C.POINTER(gala_topology), ll, C.POINTER(gala_hparams), vp]),
         }
         for name, (res, args) in sig.items():
@@ -274,6 +276,16 @@ def gala_gemm_bf16(A, B, D, groups, M, N, K, a_mn=0, b_mn=0, split_k=1, stream=N
     rc = lib().gala_gemm_bf16(_ptr(A), _ptr(B), _ptr(D), groups, M, N, K, a_mn, b_mn, split_k, stream)
     if rc < 0:
         raise GalaError(rc, "gala_gemm_bf16")
+
+
+def gala_gemm_bf16_static(A, B, D, groups, M, N, K, a_mn=0, b_mn=0, split_k=1, stream=None):
+    """gala_gemm_bf16 for hosts that cannot allocate device memory: scratch comes from an 8 MiB
+    array inside the library (groups*split_k*M*N <= 2 Mi floats when split_k > 1)."""
+    buf = C.create_string_buffer(512)
+    rc = lib().gala_gemm_bf16_static(_ptr(A), _ptr(B), _ptr(D), groups, M, N, K, a_mn, b_mn, split_k, stream,
+                                     buf, len(buf))
+    if rc < 0:
+        raise GalaError(rc, buf.value.decode())
 
 
 def gala_sweep_sync(x, g, v, clip, n_agents, d_padded, topo: gala_topology, rnd: int, hp: gala_hparams,
