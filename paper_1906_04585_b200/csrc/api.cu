@@ -780,7 +780,8 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
     int off[2] = {0, 0};
     const int np = topo_offsets(c->topo, n, c->sync_round, off);
     SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
-    LAUNCH(T_SWEEP_SYNC, st, launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp, st));
+    LAUNCH(T_SWEEP_SYNC, st, launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp,
+                                            c->error_word, st));
     CK(cudaEventRecord(c->main_event, st));
     for (int i = 0; i < n; i++) {
         CK(cudaStreamWaitEvent(c->agents[i].stream, c->main_event, 0));
@@ -1063,7 +1064,7 @@ int gala_sweep_sync(float* x, const float* g, float* v, const float* clip, int n
     int off[2] = {0, 0};
     const int np = topo_offsets(*topo, n_agents, round, off);
     SweepHp s{hp->lr, hp->rms_alpha, hp->rms_eps};
-    cudaError_t e = launch_sweep_sync(x, g, v, clip, nullptr, n_agents, d_padded, np, off, s,
+    cudaError_t e = launch_sweep_sync(x, g, v, clip, nullptr, n_agents, d_padded, np, off, s, nullptr,
                                       reinterpret_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? GALA_OK : GALA_ECUDA;
 }

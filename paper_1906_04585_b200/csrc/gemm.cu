@@ -127,8 +127,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __shared__ int issued_iters;
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // number of ring stages and the B stage size follow the launch (short reductions and narrow
+    // tiles take less shared memory, so more CTAs fit on an SM and hide each other's prologue/epilogue)
+    const int nst = p.stages;
+    const int stage_b = p.block_n * BK * 2;
     uint8_t* smA = smem;
-    uint8_t* smB = smem + kStages * kStageA;
+    uint8_t* smB = smem + nst * kStageA;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.block_n;
@@ -143,7 +147,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t tmem_cols = BN < 32 ? 32u : (uint32_t)BN;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         mbar_init(&accum_bar, 1);
         abort_flag = 0;
         issued_iters = 0;
@@ -164,13 +168,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (lane == 0) {
             const uint32_t bytes = (uint32_t)kStageA + (uint32_t)BN * BK * 2;
             for (int it = 0; it < num_k; it++) {
-                const int s = it % kStages;
-                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                const int s = it % nst;
+                const uint32_t ph = (uint32_t)(it / nst) & 1u;
                 if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) break;
                 mbar_expect_tx(&full_bar[s], bytes);
                 const int k0 = (kt_begin + it) * BK;
                 uint8_t* a = smA + s * kStageA;
-                uint8_t* b = smB + s * kStageB;
+                uint8_t* b = smB + s * stage_b;
                 if (!a_mn) {
                     tma_load_3d(a, &tmA, &full_bar[s], k0, m0, group);
                 } else {
@@ -191,12 +195,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t idesc = make_instr_desc(BN, a_mn, b_mn);
             bool ok = true;
             for (int it = 0; it < num_k; it++) {
-                const int s = it % kStages;
-                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                const int s = it % nst;
+                const uint32_t ph = (uint32_t)(it / nst) & 1u;
                 if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t a_addr = smem_u32(smA + s * kStageA);
-                const uint32_t b_addr = smem_u32(smB + s * kStageB);
+                const uint32_t b_addr = smem_u32(smB + s * stage_b);
 #pragma unroll
                 for (int kk = 0; kk < BK / 16; kk++) {
                     // one UMMA consumes K = 16: 32 B along a K-major row, 16 rows (2048 B) of an MN-major tile
@@ -299,9 +303,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (p.error_word) atomicExch(p.error_word, 1);
             // let copies that were already issued land before the shared memory goes away
             const int issued = issued_iters;
-            for (int it = max(0, issued - kStages); it < issued; it++) {
-                const int s = it % kStages;
-                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+            for (int it = max(0, issued - nst); it < issued; it++) {
+                const int s = it % nst;
+                const uint32_t ph = (uint32_t)(it / nst) & 1u;
                 for (uint32_t i = 0; i < (1u << 16); i++) {
                     if (mbar_try_wait(&full_bar[s], ph)) break;
                     __nanosleep(64);
@@ -371,6 +375,20 @@ bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t
     return r == CUDA_SUCCESS;
 }
 
+bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
+                         uint32_t box_cols, uint32_t box_rows) {
+    if (!g_encode) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15) || (row_stride_bytes & 15) || box_cols > 256 || box_rows > 256) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {row_stride_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
                   uint64_t groups, uint64_t ld_elems, uint64_t group_stride_elems, int tile_mn) {
     op->mn_major = mn_major;
@@ -385,7 +403,13 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     if (B.mn_major && args.block_n < 64) return cudaErrorInvalidValue;
     if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
     dim3 grid((args.M + BM - 1) / BM, (args.N + args.block_n - 1) / args.block_n, args.groups * args.split_k);
-    gemm_tcgen05_kernel<<<grid, 192, kSmemBytes, st>>>(A.map, B.map, args, A.mn_major, B.mn_major);
+    GemmArgs a = args;
+    const int k_tiles = (a.K + BK - 1) / BK;
+    const int per_split = (k_tiles + a.split_k - 1) / a.split_k;
+    a.stages = per_split < kStages ? per_split : kStages;
+    if (a.stages < 1) a.stages = 1;
+    const size_t smem = (size_t)a.stages * (kStageA + a.block_n * BK * 2) + 1024;
+    gemm_tcgen05_kernel<<<grid, 192, smem, st>>>(A.map, B.map, a, A.mn_major, B.mn_major);
     return cudaGetLastError();
 }
 

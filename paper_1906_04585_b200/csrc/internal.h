@@ -56,6 +56,7 @@ struct GemmArgs {
     int groups;            // grid.z = groups * split_k
     int group0;            // first group index (added to the TMA group coordinate)
     int split_k;
+    int stages;            // shared-memory ring depth; set by launch_gemm
     int flags;
     float scale;           // applied to the accumulator before the bias
     const float* bias;     // per-column (n) bias, may be null; indexed by group with bias_group_stride
@@ -74,6 +75,9 @@ cudaError_t gemm_init();   // resolves the driver entry point used to build TMA 
 bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t groups,
                      uint64_t row_stride_bytes, uint64_t group_stride_bytes, uint32_t box_cols,
                      uint32_t box_rows);
+// rows x cols fp32 matrix, unswizzled box_rows x box_cols tile (gemm_init() first).
+bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
+                         uint32_t box_cols, uint32_t box_rows);
 // Builds the descriptor for an operand of a GEMM with the given tile height
 // (128 for A, block_n for B).
 bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
@@ -94,10 +98,14 @@ cudaError_t launch_sweep_agent(float* x, const float* g, float* v, float* snap_o
 // Synchronous all-agent form.  peer_off[j]: in-peer j of agent i is (i - peer_off[j]) mod n.
 cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* clip,
                               __nv_bfloat16* shadow, int n_agents, long d_pad, int n_peers,
-                              const int* peer_off, SweepHp hp, cudaStream_t st);
+                              const int* peer_off, SweepHp hp, int* error_word, cudaStream_t st);
+// Bulk-copy staged variant; cudaErrorNotSupported when the shape does not suit it.
+cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const float* clip, __nv_bfloat16* shadow,
+                                   int n_agents, long d_pad, int n_peers, int o0, int o1, SweepHp hp,
+                                   int* error_word, cudaStream_t st);
 // Sum of squares of g[agent][0..d) -> norm[agent], clip[agent] = min(1, max_norm/(norm+1e-6)).
 // partial: [n_agents][kNormChunks] doubles, ticket: [n_agents] uints (zero before first use).
-constexpr int kNormChunks = 32;
+constexpr int kNormChunks = 128;
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
                              double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st);
 cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st);

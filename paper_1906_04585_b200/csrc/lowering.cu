@@ -157,34 +157,46 @@ cudaError_t launch_col2im(const float* dcols, long dcols_group_stride, const __n
 }
 
 // Bias gradient: out[c] = sum over rows of dy[row][c].  Rows are cut into kColsumChunks fixed
-// chunks (one block each); the block that finishes last adds the chunk sums in index order, so
-// the result does not depend on scheduling.  C is a power of two <= 512.
+// chunks (one block each).  Inside a block a thread owns 8 adjacent columns (one 16-byte load per
+// row) and every (256*8/C)-th row of the chunk; the row lanes are combined in index order, and the
+// block that finishes last adds the chunk sums in index order, so the result does not depend on
+// scheduling.  C is a power of two, 8 <= C <= 512.
 __global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __restrict__ dy, long dy_group_stride, long rows,
                                                      int C, float* __restrict__ out, long out_group_stride,
                                                      double* partial, unsigned* ticket) {
     const int g = blockIdx.y;
-    const __nv_bfloat16* src = dy + (long)g * dy_group_stride;
+    const uint4* src = reinterpret_cast<const uint4*>(dy + (long)g * dy_group_stride);
     const long per = (rows + kColsumChunks - 1) / kColsumChunks;
     const long lo = (long)blockIdx.x * per;
     long hi = lo + per; if (hi > rows) hi = rows;
-    __shared__ float red[256];
+    __shared__ float red[256 * 8];
     __shared__ bool last;
     double* part = partial + (long)g * kColsumChunks * 512 + (long)blockIdx.x * C;
-    const int lanes = C < 256 ? 256 / C : 1;   // row-lanes per column when C < 256
-    for (int cbase = 0; cbase < C; cbase += 256) {
-        const int c = cbase + (int)(threadIdx.x % (C < 256 ? C : 256));
-        const int rl = C < 256 ? (int)(threadIdx.x / C) : 0;
-        float acc = 0.0f;
-        for (long r = lo + rl; r < hi; r += lanes) acc += __bfloat162float(src[r * C + c]);
-        red[threadIdx.x] = acc;
-        __syncthreads();
-        if (rl == 0) {
-            float s = acc;
-            for (int l = 1; l < lanes; l++) s += red[threadIdx.x + l * C];
-            part[c] = (double)s;
+    const int cchunks = C / 8;                    // 16-byte column groups per row
+    const int lanes = 256 / cchunks > 0 ? 256 / cchunks : 1;   // row lanes (C <= 512 -> cchunks <= 64)
+    const int cc = threadIdx.x % cchunks, rl = threadIdx.x / cchunks;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (rl < lanes) {
+        for (long r = lo + rl; r < hi; r += lanes) {
+            const uint4 v = __ldg(src + r * cchunks + cc);
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                const float2 f = __bfloat1622float2(h[q]);
+                acc[2 * q] += f.x; acc[2 * q + 1] += f.y;
+            }
         }
-        __syncthreads();
     }
+#pragma unroll
+    for (int q = 0; q < 8; q++) red[threadIdx.x * 8 + q] = acc[q];
+    __syncthreads();
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+        const int ccq = c / 8, q = c % 8;
+        float s = 0.0f;
+        for (int l = 0; l < lanes; l++) s += red[(l * cchunks + ccq) * 8 + q];
+        part[c] = (double)s;
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         unsigned t = atomicAdd(&ticket[g], 1u);
@@ -204,7 +216,7 @@ __global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __rest
 }
 cudaError_t launch_colsum(const __nv_bfloat16* dy, long dy_group_stride, long rows, int C, float* out,
                           long out_group_stride, double* partial, unsigned* ticket, int groups, cudaStream_t st) {
-    if (C > 512 || (C & (C - 1))) return cudaErrorInvalidValue;
+    if (C > 512 || C < 8 || (C & (C - 1))) return cudaErrorInvalidValue;
     colsum_kernel<<<dim3(kColsumChunks, groups), 256, 0, st>>>(dy, dy_group_stride, rows, C, out, out_group_stride,
                                                               partial, ticket);
     return cudaGetLastError();

@@ -4,6 +4,8 @@
 //
 // Both forms are pure streaming kernels: every array element is read once and
 // written once with 16-byte accesses.
+#include <cstdlib>
+
 #include "internal.h"
 
 namespace gala {
@@ -150,8 +152,17 @@ __global__ void sweep_sync_kernel(float* __restrict__ x, const float* __restrict
 
 cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* clip,
                               __nv_bfloat16* shadow, int n_agents, long d_pad, int n_peers,
-                              const int* peer_off, SweepHp hp, cudaStream_t st) {
+                              const int* peer_off, SweepHp hp, int* error_word, cudaStream_t st) {
     long n4 = d_pad / 4;
+    {
+        int b0 = 0, b1 = 0;
+        if (n_peers >= 1) b0 = ((peer_off[0] % n_agents) + n_agents) % n_agents;
+        if (n_peers >= 2) b1 = ((peer_off[1] % n_agents) + n_agents) % n_agents;
+        // staged tensor-copy kernel first; the register-staged kernel below serves the shapes it declines
+        cudaError_t eb = launch_sweep_sync_bulk(x, g, v, clip, shadow, n_agents, d_pad, n_peers, b0, b1, hp,
+                                                error_word, st);
+        if (eb != cudaErrorNotSupported) return eb;
+    }
     // shared memory: n_agents * threads * 16 B, kept under 128 KB so that one block always fits
     int threads = 256;
     while (threads > 32 && (long)n_agents * threads * 16 > 128 * 1024) threads /= 2;
@@ -189,11 +200,16 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
                                                         unsigned* ticket, float* norm, float* clip) {
     const int agent = agent0 + blockIdx.y;
     const float* ga = g + (long)agent * d_pad;
-    const long per = ((d + kNormChunks - 1) / kNormChunks + 3) & ~3L;
+    // chunks are multiples of 4 floats and the padding [d, d_pad) is zero: 16-byte loads throughout
+    const long per = ((d_pad / 4 + kNormChunks - 1) / kNormChunks) * 4;
     const long lo = (long)blockIdx.x * per;
-    long hi = lo + per; if (hi > d) hi = d;
-    double acc = 0.0;
-    for (long i = lo + threadIdx.x; i < hi; i += blockDim.x) { float t = ga[i]; acc += (double)t * t; }
+    long hi = lo + per; if (hi > d_pad) hi = d_pad;
+    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+    for (long i = lo + 4L * threadIdx.x; i < hi; i += 4L * blockDim.x) {
+        const float4 t = __ldcs(reinterpret_cast<const float4*>(ga + i));
+        a0 = fmaf(t.x, t.x, a0); a1 = fmaf(t.y, t.y, a1); a2 = fmaf(t.z, t.z, a2); a3 = fmaf(t.w, t.w, a3);
+    }
+    double acc = ((double)a0 + (double)a1) + ((double)a2 + (double)a3);
     __shared__ double red[256];
     red[threadIdx.x] = acc;
     __syncthreads();
