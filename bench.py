@@ -290,12 +290,18 @@ def run_ours(args):
         B.gala_losses(L.ctx, 0)
     barrier()
     t0 = time.perf_counter()
+    # the copy of step k+1's rollouts (other buffer set) is enqueued before step k's losses are read, so
+    # it overlaps step k on the GPU; every step's copy and read still happen inside the timed region
+    cur = sets[0]
+    for r in cur:
+        r.upload(up)
     for k in range(args.steps):
         cur = sets[k % n_sets]
-        for r in cur:
-            r.upload(up)
         ext.wait_stream(up)
         L.step_sync(cur)
+        if k + 1 < args.steps:
+            for r in sets[(k + 1) % n_sets]:
+                r.upload(up)
         for i in range(w.n_agents):
             B.gala_losses(L.ctx, i)
     barrier()
@@ -378,8 +384,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="index into gala_inputs.WORKLOADS (1 = the headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep-only", action="store_true",
+                    help="run only the RMSProp + gossip micro-benchmark (32 agents x 1.7M parameters)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep_only:
+        import torch
+        from paper_1906_04585_b200 import binding as B
+        print(json.dumps(dict(metric="gossip-mix+RMSprop GB/s", sweep_microbench=sweep_microbench(torch, B, peaks()))))
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -378,14 +378,6 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
     return GALA_OK;
 }
 
-int colsum(gala_ctx* c, const __nv_bfloat16* dy, long stride, long rows, int C, long grad_off, int agent0, int groups,
-           cudaStream_t st) {
-    LAUNCH(T_COLSUM, st, launch_colsum(dy + (long)agent0 * stride, stride, rows, C, c->g + (long)agent0 * c->d_pad + grad_off,
-                         c->d_pad, c->colsum_partial + (long)agent0 * kColsumChunks * 512, c->colsum_ticket + agent0,
-                         groups, st));
-    return GALA_OK;
-}
-
 // Learner step for agents [agent0, agent0+groups): forward, returns/advantages/objective,
 // backward into the flat gradient, global norm and clip coefficient.
 int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cudaStream_t st) {
@@ -421,12 +413,10 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hb.dpre = c->dh + (long)agent0 * S * kHidden; hb.dpre_stride = S * kHidden; hb.dpre_bf16 = 1;
         LAUNCH(T_HEADS_BWD, st, launch_heads_bwd(hb, groups, st));
         c->launches++; c->tag_launches[T_HEADS_BWD]++;  // two kernels
-        if ((r = colsum(c, c->dh, S * kHidden, S, kHidden, c->cl.fcb, agent0, groups, st)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, st)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
         for (int l = 2; l >= 0; l--) {
             const int CO = kConvCout[l];
-            if ((r = colsum(c, c->dy[l], S * P[l] * CO, S * P[l], CO, c->cl.b[l], agent0, groups, st)) != GALA_OK) return r;
             if ((r = run_wgrad(c, c->wgrad[l], agent0, groups, st)) != GALA_OK) return r;
             if (l > 0) {
                 if ((r = run_plan(c, c->dgrad[l], agent0, groups, 0, st)) != GALA_OK) return r;
@@ -435,6 +425,16 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
                 LAUNCH(T_COL2IM, st, launch_col2im(c->dcols[l] + (long)agent0 * ds, ds, c->act[l - 1] + (long)agent0 * as, as,
                                      c->dy[l - 1] + (long)agent0 * xs, xs, l, (int)S, groups, st));
             }
+        }
+        {   // all four bias gradients (column sums of dh, dY3, dY2, dY1) in one launch
+            ColsumJobs jobs{};
+            jobs.j[0] = {c->dh + (long)agent0 * S * kHidden, S * kHidden, S, kHidden, c->cl.fcb};
+            for (int l = 0; l < 3; l++)
+                jobs.j[1 + l] = {c->dy[l] + (long)agent0 * S * P[l] * kConvCout[l], S * P[l] * kConvCout[l], S * P[l],
+                                 kConvCout[l], c->cl.b[l]};
+            LAUNCH(T_COLSUM, st, launch_colsum(jobs, 4, c->g + (long)agent0 * dp, dp,
+                                               c->colsum_partial + (long)agent0 * kColsumJobs * kColsumChunks * 512,
+                                               c->colsum_ticket + (long)agent0 * kColsumJobs, groups, st));
         }
     } else {
         const int H = c->H;
@@ -646,7 +646,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         const int P[3] = {400, 81, 49};
         CK(gemm_init());
         ALLOC(c->shadow, (size_t)n * dp);
-        ALLOC(c->colsum_partial, (size_t)n * kColsumChunks * 512); ALLOC(c->colsum_ticket, n);
+        ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {
             ALLOC(c->cols[l], (size_t)n * B * P[l] * kConvKK[l]);
             ALLOC(c->act[l], (size_t)n * B * P[l] * kConvCout[l]);

@@ -182,10 +182,14 @@ cudaError_t launch_im2col_bf16(const __nv_bfloat16* act, long act_group_stride, 
 cudaError_t launch_col2im(const float* dcols, long dcols_group_stride, const __nv_bfloat16* act_in,
                           long act_group_stride, __nv_bfloat16* dx, long dx_group_stride, int layer,
                           int samples, int groups, cudaStream_t st);
-// out[g][c] = sum_r dy[g][r][c]   (bf16 in, fp32 out at out + g*out_stride), fixed summation order
-cudaError_t launch_colsum(const __nv_bfloat16* dy, long dy_group_stride, long rows, int C, float* out,
-                          long out_group_stride, double* partial, unsigned* ticket, int groups,
-                          cudaStream_t st);
+// Column sums (bias gradients) of up to kColsumJobs bf16 tensors in one launch:
+// out_base[g*out_group_stride + out_off + c] = sum_r dy[g][r][c], fixed summation order.
+// partial: [groups][kColsumJobs][kColsumChunks][512] doubles, ticket: [groups][kColsumJobs] (zeroed once).
+constexpr int kColsumJobs = 4;
+struct ColsumJob { const __nv_bfloat16* dy; long group_stride; long rows; int C; long out_off; };
+struct ColsumJobs { ColsumJob j[kColsumJobs]; };
+cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, long out_group_stride, double* partial,
+                          unsigned* ticket, int groups, cudaStream_t st);
 constexpr int kColsumChunks = 64;
 
 }  // namespace gala

@@ -161,17 +161,23 @@ cudaError_t launch_col2im(const float* dcols, long dcols_group_stride, const __n
 // row) and every (256*8/C)-th row of the chunk; the row lanes are combined in index order, and the
 // block that finishes last adds the chunk sums in index order, so the result does not depend on
 // scheduling.  C is a power of two, 8 <= C <= 512.
-__global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __restrict__ dy, long dy_group_stride, long rows,
-                                                     int C, float* __restrict__ out, long out_group_stride,
-                                                     double* partial, unsigned* ticket) {
+// Up to kColsumJobs tensors are reduced by one launch (blockIdx.z picks the tensor).
+__global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, float* __restrict__ out_base, long out_group_stride,
+                                                     double* partial_base, unsigned* ticket_base) {
     const int g = blockIdx.y;
-    const uint4* src = reinterpret_cast<const uint4*>(dy + (long)g * dy_group_stride);
+    const ColsumJob job = jobs.j[blockIdx.z];
+    const long rows = job.rows;
+    const int C = job.C;
+    float* out = out_base + job.out_off;
+    double* partial = partial_base + (long)blockIdx.z * kColsumChunks * 512;
+    unsigned* ticket = ticket_base + blockIdx.z;
+    const uint4* src = reinterpret_cast<const uint4*>(job.dy + (long)g * job.group_stride);
     const long per = (rows + kColsumChunks - 1) / kColsumChunks;
     const long lo = (long)blockIdx.x * per;
     long hi = lo + per; if (hi > rows) hi = rows;
     __shared__ float red[256 * 8];
     __shared__ bool last;
-    double* part = partial + (long)g * kColsumChunks * 512 + (long)blockIdx.x * C;
+    double* part = partial + (long)g * kColsumJobs * kColsumChunks * 512 + (long)blockIdx.x * C;
     const int cchunks = C / 8;                    // 16-byte column groups per row
     const int lanes = 256 / cchunks > 0 ? 256 / cchunks : 1;   // row lanes (C <= 512 -> cchunks <= 64)
     const int cc = threadIdx.x % cchunks, rl = threadIdx.x / cchunks;
@@ -199,26 +205,29 @@ __global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __rest
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        unsigned t = atomicAdd(&ticket[g], 1u);
+        unsigned t = atomicAdd(&ticket[g * kColsumJobs], 1u);
         last = (t == kColsumChunks - 1);
     }
     __syncthreads();
     if (last) {
         __threadfence();
-        const volatile double* pg = partial + (long)g * kColsumChunks * 512;
+        const volatile double* pg = partial + (long)g * kColsumJobs * kColsumChunks * 512;
         for (int c = threadIdx.x; c < C; c += blockDim.x) {
             double s = 0.0;
             for (int k = 0; k < kColsumChunks; k++) s += pg[(long)k * C + c];
             out[(long)g * out_group_stride + c] = (float)s;
         }
-        if (threadIdx.x == 0) ticket[g] = 0;
+        if (threadIdx.x == 0) ticket[g * kColsumJobs] = 0;
     }
 }
-cudaError_t launch_colsum(const __nv_bfloat16* dy, long dy_group_stride, long rows, int C, float* out,
-                          long out_group_stride, double* partial, unsigned* ticket, int groups, cudaStream_t st) {
-    if (C > 512 || C < 8 || (C & (C - 1))) return cudaErrorInvalidValue;
-    colsum_kernel<<<dim3(kColsumChunks, groups), 256, 0, st>>>(dy, dy_group_stride, rows, C, out, out_group_stride,
-                                                              partial, ticket);
+cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, long out_group_stride, double* partial,
+                          unsigned* ticket, int groups, cudaStream_t st) {
+    if (n_jobs < 1 || n_jobs > kColsumJobs) return cudaErrorInvalidValue;
+    for (int i = 0; i < n_jobs; i++) {
+        const int C = jobs.j[i].C;
+        if (C > 512 || C < 8 || (C & (C - 1))) return cudaErrorInvalidValue;
+    }
+    colsum_kernel<<<dim3(kColsumChunks, groups, n_jobs), 256, 0, st>>>(jobs, out_base, out_group_stride, partial, ticket);
     return cudaGetLastError();
 }
 
