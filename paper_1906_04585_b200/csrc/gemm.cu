@@ -7,13 +7,15 @@
 // (B MN-major) and weight-gradient (both MN-major) products of the conv / dense layers without
 // any transposed copy in global memory.
 //
-// Structure of one CTA (192 threads, one 128 x block_n output tile, one K range):
+// Structure of one CTA (192 threads, persistent: it loops over 128 x block_n output tiles):
 //   warp 0   : TMA producer - cp.async.bulk.tensor (3-D maps: inner, rows, group) into a ring of
-//              128-byte-swizzled shared-memory stages, completion on mbarriers
-//   warp 1   : allocates tensor memory, issues tcgen05.mma (one elected thread), releases stages
-//              with tcgen05.commit
-//   warps 2-5: epilogue - tcgen05.ld the fp32 accumulator out of tensor memory (each warp its
-//              own 32-lane quarter), apply scale / bias / ReLU / mask, store
+//              128-byte-swizzled shared-memory stages that runs on across tiles
+//   warp 1   : allocates tensor memory (two accumulator buffers), issues tcgen05.mma (one elected
+//              thread), releases stages and publishes finished accumulators with tcgen05.commit
+//   warps 2-5: epilogue - tcgen05.ld the fp32 accumulator of the previous tile out of tensor memory
+//              (each warp its own 32-lane quarter) while the next tile is being multiplied, re-tile
+//              it through shared memory so that global stores coalesce, apply scale / bias / ReLU /
+//              mask, store
 // Every mbarrier wait is bounded: when a wait runs out the CTA raises an abort flag, sets the
 // caller's error word, drains what it has in flight, frees its tensor memory and returns.
 #include "internal.h"
@@ -25,7 +27,7 @@ constexpr int BK = 64;           // K per stage = one 128-byte swizzle atom of b
 constexpr int kStages = 4;
 constexpr int kStageA = BM * BK * 2;    // 16 KiB
 constexpr int kStageB = 128 * BK * 2;   // room for block_n = 128
-constexpr int kSmemBytes = kStages * (kStageA + kStageB) + 1024;  // + alignment slack
+constexpr int kSmemBytes = kStages * (kStageA + kStageB) + 4 * (32 * (32 * 4 + 16)) + 1024;  // ring + epilogue staging + slack
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -115,40 +117,63 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
 }
 
 // ------------------------------------------------------------------ kernel
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Work decomposition shared by the three roles: tile index -> (group, split, m-tile, n-tile), n fastest
+// so that CTAs running side by side share an A tile in L2.
+struct TileCoord { int gz, split, m0, n0, kt_begin, num_k; };
+__device__ __forceinline__ TileCoord decode_tile(const GemmArgs& p, long tile, int mt, int nt) {
+    TileCoord t;
+    const int n_t = (int)(tile % nt);
+    const long r = tile / nt;
+    const int m_t = (int)(r % mt);
+    const int z = (int)(r / mt);
+    t.gz = z / p.split_k; t.split = z % p.split_k;
+    t.m0 = m_t * BM; t.n0 = n_t * p.block_n;
+    const int k_tiles = (p.K + BK - 1) / BK;
+    const int per_split = (k_tiles + p.split_k - 1) / p.split_k;
+    t.kt_begin = t.split * per_split;
+    const int kt_end = min(k_tiles, t.kt_begin + per_split);
+    t.num_k = max(0, kt_end - t.kt_begin);
+    return t;
+}
+
+constexpr int kEpiRowBytes = 32 * 4 + 16;          // 32 fp32 columns of one row + 16 B against bank conflicts
+constexpr int kEpiWarpBytes = 32 * kEpiRowBytes;   // staging area of one epilogue warp
+
+// Persistent CTA: loops over output tiles.  The shared-memory ring runs on across tiles, and the
+// accumulator is double-buffered in tensor memory, so the loads and MMAs of tile i+1 overlap the
+// epilogue of tile i.
 __global__ void __launch_bounds__(192, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmArgs p, const int a_mn, const int b_mn) {
+                    const GemmArgs p, const int a_mn, const int b_mn, const long total_tiles, const int mt,
+                    const int nt) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kStages];
     __shared__ __align__(8) uint64_t empty_bar[kStages];
-    __shared__ __align__(8) uint64_t accum_bar;
+    __shared__ __align__(8) uint64_t acc_full[2];
+    __shared__ __align__(8) uint64_t acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int issued_iters;
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    // number of ring stages and the B stage size follow the launch (short reductions and narrow
-    // tiles take less shared memory, so more CTAs fit on an SM and hide each other's prologue/epilogue)
     const int nst = p.stages;
-    const int stage_b = p.block_n * BK * 2;
+    const int BN = p.block_n;
+    const int stage_b = BN * BK * 2;
     uint8_t* smA = smem;
     uint8_t* smB = smem + nst * kStageA;
+    uint8_t* smE = smB + nst * stage_b;   // epilogue staging, 4 x kEpiWarpBytes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int BN = p.block_n;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
-    const int gz = blockIdx.z / p.split_k, split = blockIdx.z % p.split_k;
-    const int group = p.group0 + gz;
-    const int k_tiles = (p.K + BK - 1) / BK;
-    const int per_split = (k_tiles + p.split_k - 1) / p.split_k;
-    const int kt_begin = split * per_split;
-    const int kt_end = min(k_tiles, kt_begin + per_split);
-    const int num_k = max(0, kt_end - kt_begin);
-    const uint32_t tmem_cols = BN < 32 ? 32u : (uint32_t)BN;
+    const uint32_t acc_cols = BN < 32 ? 32u : (uint32_t)BN;
+    const uint32_t tmem_cols = 2u * acc_cols;   // 64, 128 or 256: a power of two
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        mbar_init(&accum_bar, 1);
+        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
         abort_flag = 0;
         issued_iters = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -162,136 +187,205 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     tcgen05_fence_before();
     __syncthreads();
     tcgen05_fence_after();
-    const uint32_t tmem_acc = tmem_slot;
+    const uint32_t tmem_base = tmem_slot;
 
     if (warp == 0) {
+        // ------------------------------------------------ TMA producer
         if (lane == 0) {
-            const uint32_t bytes = (uint32_t)kStageA + (uint32_t)BN * BK * 2;
-            for (int it = 0; it < num_k; it++) {
-                const int s = it % nst;
-                const uint32_t ph = (uint32_t)(it / nst) & 1u;
-                if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) break;
-                mbar_expect_tx(&full_bar[s], bytes);
-                const int k0 = (kt_begin + it) * BK;
-                uint8_t* a = smA + s * kStageA;
-                uint8_t* b = smB + s * stage_b;
-                if (!a_mn) {
-                    tma_load_3d(a, &tmA, &full_bar[s], k0, m0, group);
-                } else {
-                    tma_load_3d(a, &tmA, &full_bar[s], m0, k0, group);
-                    tma_load_3d(a + 8192, &tmA, &full_bar[s], m0 + 64, k0, group);
+            const uint32_t bytes = (uint32_t)kStageA + (uint32_t)stage_b;
+            int it = 0;
+            bool ok = true;
+            for (long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                const TileCoord t = decode_tile(p, tile, mt, nt);
+                const int group = p.group0 + t.gz;
+                for (int k = 0; k < t.num_k; k++, it++) {
+                    const int s = it % nst;
+                    const uint32_t ph = (uint32_t)(it / nst) & 1u;
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(&full_bar[s], bytes);
+                    const int k0 = (t.kt_begin + k) * BK;
+                    uint8_t* a = smA + s * kStageA;
+                    uint8_t* b = smB + s * stage_b;
+                    if (!a_mn) {
+                        tma_load_3d(a, &tmA, &full_bar[s], k0, t.m0, group);
+                    } else {
+                        tma_load_3d(a, &tmA, &full_bar[s], t.m0, k0, group);
+                        tma_load_3d(a + 8192, &tmA, &full_bar[s], t.m0 + 64, k0, group);
+                    }
+                    if (!b_mn) {
+                        tma_load_3d(b, &tmB, &full_bar[s], k0, t.n0, group);
+                    } else {
+                        for (int j = 0; j < BN / 64; j++)
+                            tma_load_3d(b + j * 8192, &tmB, &full_bar[s], t.n0 + 64 * j, k0, group);
+                    }
+                    issued_iters = it + 1;
                 }
-                if (!b_mn) {
-                    tma_load_3d(b, &tmB, &full_bar[s], k0, n0, group);
-                } else {
-                    for (int j = 0; j < BN / 64; j++)
-                        tma_load_3d(b + j * 8192, &tmB, &full_bar[s], n0 + 64 * j, k0, group);
-                }
-                issued_iters = it + 1;
             }
         }
     } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = make_instr_desc(BN, a_mn, b_mn);
+            int it = 0, local = 0;
             bool ok = true;
-            for (int it = 0; it < num_k; it++) {
-                const int s = it % nst;
-                const uint32_t ph = (uint32_t)(it / nst) & 1u;
-                if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
+            for (long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, local++) {
+                const TileCoord t = decode_tile(p, tile, mt, nt);
+                const int ab = local & 1;
+                // the epilogue must have drained this accumulator buffer (two tiles ago)
+                if (!mbar_wait(&acc_empty[ab], (((uint32_t)local >> 1) & 1u) ^ 1u, &abort_flag)) break;
                 tcgen05_fence_after();
-                const uint32_t a_addr = smem_u32(smA + s * kStageA);
-                const uint32_t b_addr = smem_u32(smB + s * stage_b);
+                const uint32_t tmem_acc = tmem_base + (uint32_t)ab * acc_cols;
+                for (int k = 0; k < t.num_k; k++, it++) {
+                    const int s = it % nst;
+                    const uint32_t ph = (uint32_t)(it / nst) & 1u;
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t a_addr = smem_u32(smA + s * kStageA);
+                    const uint32_t b_addr = smem_u32(smB + s * stage_b);
 #pragma unroll
-                for (int kk = 0; kk < BK / 16; kk++) {
-                    // one UMMA consumes K = 16: 32 B along a K-major row, 16 rows (2048 B) of an MN-major tile
-                    const uint64_t ad = make_smem_desc(a_addr + (a_mn ? kk * 2048 : kk * 32), a_mn);
-                    const uint64_t bd = make_smem_desc(b_addr + (b_mn ? kk * 2048 : kk * 32), b_mn);
-                    umma_bf16(tmem_acc, ad, bd, idesc, (it | kk) != 0 ? 1u : 0u);
+                    for (int kk = 0; kk < BK / 16; kk++) {
+                        // one UMMA consumes K = 16: 32 B along a K-major row, 16 rows (2048 B) of an MN-major tile
+                        const uint64_t ad = make_smem_desc(a_addr + (a_mn ? kk * 2048 : kk * 32), a_mn);
+                        const uint64_t bd = make_smem_desc(b_addr + (b_mn ? kk * 2048 : kk * 32), b_mn);
+                        umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty_bar[s]);
                 }
-                umma_commit(&empty_bar[s]);
+                if (!ok) break;
+                if (t.num_k > 0) umma_commit(&acc_full[ab]);   // arrives when the MMAs above have completed
+                else mbar_arrive(&acc_full[ab]);               // empty K range: nothing to wait for
             }
-            if (ok && num_k > 0) umma_commit(&accum_bar);
         }
     } else {
-        // epilogue warps 2..5 -> tensor-memory lane quarters 2,3,0,1
+        // ------------------------------------------------ epilogue warps 2..5 -> lane quarters 2,3,0,1
         const int q = warp & 3;
-        const int m = m0 + q * 32 + lane;
-        bool have = true;
-        if (num_k > 0) {
-            have = mbar_wait(&accum_bar, 0, &abort_flag);
+        uint8_t* stage = smE + (warp - 2) * kEpiWarpBytes;
+        const bool out_bf16 = p.flags & EPI_OUT_BF16, relu = p.flags & EPI_RELU;
+        const bool transpose = p.flags & EPI_TRANSPOSE, use_mask = p.flags & EPI_MASK;
+        const bool vec_ok = out_bf16 ? ((p.ldc & 7) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 &&
+                                        (p.out_group_stride & 7) == 0 && (p.out_split_stride & 7) == 0)
+                                     : ((p.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 &&
+                                        (p.out_group_stride & 3) == 0 && (p.out_split_stride & 3) == 0);
+        const bool mask_vec = use_mask && (reinterpret_cast<uintptr_t>(p.mask) & 7) == 0 && (p.mask_group_stride & 3) == 0;
+        int local = 0;
+        for (long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, local++) {
+            const TileCoord t = decode_tile(p, tile, mt, nt);
+            const int ab = local & 1;
+            if (!mbar_wait(&acc_full[ab], ((uint32_t)local >> 1) & 1u, &abort_flag)) break;
             tcgen05_fence_after();
-        }
-        if (have) {
-            const bool out_bf16 = p.flags & EPI_OUT_BF16, relu = p.flags & EPI_RELU;
-            const bool transpose = p.flags & EPI_TRANSPOSE, use_mask = p.flags & EPI_MASK;
-            const long obase = (long)gz * p.out_group_stride + (long)split * p.out_split_stride;
+            const uint32_t tmem_acc = tmem_base + (uint32_t)ab * acc_cols;
+            const int group = p.group0 + t.gz;
+            const long obase = (long)t.gz * p.out_group_stride + (long)t.split * p.out_split_stride;
             const float* bias = p.bias ? p.bias + (long)group * p.bias_group_stride : nullptr;
-            const __nv_bfloat16* mask = use_mask ? p.mask + (long)gz * p.mask_group_stride : nullptr;
+            const __nv_bfloat16* mask = use_mask ? p.mask + (long)t.gz * p.mask_group_stride : nullptr;
+            const int mw = t.m0 + q * 32;   // first row of this warp
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
-                if (num_k > 0) {
+                if (t.num_k > 0) {
                     tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; j++) r[j] = 0u;
                 }
-                const int nb = n0 + c0;
-                if (m >= p.M || nb >= p.N) continue;
-                float vals[32];
-#pragma unroll
-                for (int j = 0; j < 32; j++) {
-                    float v = __uint_as_float(r[j]) * p.scale;
-                    if (bias && nb + j < p.N) v += __ldg(bias + nb + j);
-                    if (relu) v = fmaxf(v, 0.0f);
-                    vals[j] = v;
-                }
-                const bool full = nb + 32 <= p.N;
-                if (!transpose) {
-                    const long row_off = obase + (long)m * p.ldc + nb;
-                    if (use_mask) {
-                        for (int j = 0; j < 32 && nb + j < p.N; j++)
-                            if (!(__bfloat162float(mask[(long)m * p.ldc + nb + j]) > 0.0f)) vals[j] = 0.0f;
-                    }
-                    if (out_bf16) {
-                        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off;
-                        if (full && (reinterpret_cast<uintptr_t>(o) & 15) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                __nv_bfloat162 h0 = __floats2bfloat162_rn(vals[j], vals[j + 1]);
-                                __nv_bfloat162 h1 = __floats2bfloat162_rn(vals[j + 2], vals[j + 3]);
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(vals[j + 4], vals[j + 5]);
-                                __nv_bfloat162 h3 = __floats2bfloat162_rn(vals[j + 6], vals[j + 7]);
-                                uint4 u;
-                                u.x = *reinterpret_cast<uint32_t*>(&h0); u.y = *reinterpret_cast<uint32_t*>(&h1);
-                                u.z = *reinterpret_cast<uint32_t*>(&h2); u.w = *reinterpret_cast<uint32_t*>(&h3);
-                                *reinterpret_cast<uint4*>(o + j) = u;
-                            }
-                        } else {
-                            for (int j = 0; j < 32 && nb + j < p.N; j++) o[j] = __float2bfloat16_rn(vals[j]);
-                        }
-                    } else {
-                        float* o = reinterpret_cast<float*>(p.out) + row_off;
-                        if (full && (reinterpret_cast<uintptr_t>(o) & 15) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4*>(o + j) = make_float4(vals[j], vals[j + 1], vals[j + 2], vals[j + 3]);
-                        } else {
-                            for (int j = 0; j < 32 && nb + j < p.N; j++) o[j] = vals[j];
-                        }
-                    }
-                } else {
+                const int nb = t.n0 + c0;
+                if (mw >= p.M || nb >= p.N) continue;   // warp-uniform
+                if (transpose) {
                     // D[m][n] -> out[n * ldc + m]: consecutive lanes write consecutive addresses
-                    if (out_bf16) {
-                        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + obase + m;
-                        for (int j = 0; j < 32 && nb + j < p.N; j++) o[(long)(nb + j) * p.ldc] = __float2bfloat16_rn(vals[j]);
-                    } else {
-                        float* o = reinterpret_cast<float*>(p.out) + obase + m;
+                    const int m = mw + lane;
+                    if (m < p.M) {
+                        if (out_bf16) {
+                            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + obase + m;
 #pragma unroll
-                        for (int j = 0; j < 32; j++)
-                            if (nb + j < p.N) o[(long)(nb + j) * p.ldc] = vals[j];
+                            for (int j = 0; j < 32; j++)
+                                if (nb + j < p.N) {
+                                    float v = __uint_as_float(r[j]) * p.scale;
+                                    if (bias) v += __ldg(bias + nb + j);
+                                    if (relu) v = fmaxf(v, 0.0f);
+                                    o[(long)(nb + j) * p.ldc] = __float2bfloat16_rn(v);
+                                }
+                        } else {
+                            float* o = reinterpret_cast<float*>(p.out) + obase + m;
+#pragma unroll
+                            for (int j = 0; j < 32; j++)
+                                if (nb + j < p.N) {
+                                    float v = __uint_as_float(r[j]) * p.scale;
+                                    if (bias) v += __ldg(bias + nb + j);
+                                    if (relu) v = fmaxf(v, 0.0f);
+                                    o[(long)(nb + j) * p.ldc] = v;
+                                }
+                        }
+                    }
+                    continue;
+                }
+                // row-major output: park the raw 32 x 32 block in shared memory (lane = row), then let every
+                // 8 lanes handle one row segment of 128 contiguous bytes, so the global accesses coalesce
+                {
+                    uint4* w = reinterpret_cast<uint4*>(stage + lane * kEpiRowBytes);
+#pragma unroll
+                    for (int j = 0; j < 8; j++) w[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                }
+                __syncwarp();
+                const int cl = (lane & 7) * 4;          // first of this lane's 4 columns inside the block
+                const int n = nb + cl;
+#pragma unroll
+                for (int i = 0; i < 8; i++) {
+                    const int rr = i * 4 + (lane >> 3);
+                    const int m = mw + rr;
+                    if (m >= p.M || n >= p.N) continue;
+                    const uint4 raw = *reinterpret_cast<const uint4*>(stage + rr * kEpiRowBytes + cl * 4);
+                    float v[4] = {__uint_as_float(raw.x) * p.scale, __uint_as_float(raw.y) * p.scale,
+                                  __uint_as_float(raw.z) * p.scale, __uint_as_float(raw.w) * p.scale};
+                    const int valid = min(4, p.N - n);
+                    if (bias) {
+#pragma unroll
+                        for (int j = 0; j < 4; j++) if (j < valid) v[j] += __ldg(bias + n + j);
+                    }
+                    if (relu) {
+#pragma unroll
+                        for (int j = 0; j < 4; j++) v[j] = fmaxf(v[j], 0.0f);
+                    }
+                    const long off = (long)m * p.ldc + n;
+                    if (use_mask) {
+                        if (mask_vec && valid == 4 && ((off & 3) == 0)) {
+                            const uint2 mk = __ldg(reinterpret_cast<const uint2*>(mask + off));
+                            const __nv_bfloat162* mh = reinterpret_cast<const __nv_bfloat162*>(&mk);
+                            const float2 m0f = __bfloat1622float2(mh[0]), m1f = __bfloat1622float2(mh[1]);
+                            if (!(m0f.x > 0.0f)) v[0] = 0.0f;
+                            if (!(m0f.y > 0.0f)) v[1] = 0.0f;
+                            if (!(m1f.x > 0.0f)) v[2] = 0.0f;
+                            if (!(m1f.y > 0.0f)) v[3] = 0.0f;
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; j++)
+                                if (j < valid && !(__bfloat162float(mask[off + j]) > 0.0f)) v[j] = 0.0f;
+                        }
+                    }
+                    if (out_bf16) {
+                        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + obase + off;
+                        if (vec_ok && valid == 4 && (((obase + off) & 3) == 0)) {
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
+                            uint2 u;
+                            u.x = *reinterpret_cast<uint32_t*>(&h0); u.y = *reinterpret_cast<uint32_t*>(&h1);
+                            *reinterpret_cast<uint2*>(o) = u;
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; j++) if (j < valid) o[j] = __float2bfloat16_rn(v[j]);
+                        }
+                    } else {
+                        float* o = reinterpret_cast<float*>(p.out) + obase + off;
+                        if (vec_ok && valid == 4 && (((obase + off) & 3) == 0)) {
+                            *reinterpret_cast<float4*>(o) = make_float4(v[0], v[1], v[2], v[3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; j++) if (j < valid) o[j] = v[j];
+                        }
                     }
                 }
+                __syncwarp();   // the staging block is rewritten by the next column block
             }
+            // this warp no longer reads the accumulator buffer
+            tcgen05_fence_before();
+            if (lane == 0) mbar_arrive(&acc_empty[ab]);
         }
     }
 
@@ -316,7 +410,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     if (warp == 1) {
         tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -402,14 +496,21 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     if (args.block_n != 32 && args.block_n != 64 && args.block_n != 128) return cudaErrorInvalidValue;
     if (B.mn_major && args.block_n < 64) return cudaErrorInvalidValue;
     if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
-    dim3 grid((args.M + BM - 1) / BM, (args.N + args.block_n - 1) / args.block_n, args.groups * args.split_k);
     GemmArgs a = args;
+    const int mt = (a.M + BM - 1) / BM, nt = (a.N + a.block_n - 1) / a.block_n;
+    const long total = (long)mt * nt * a.groups * a.split_k;
     const int k_tiles = (a.K + BK - 1) / BK;
     const int per_split = (k_tiles + a.split_k - 1) / a.split_k;
-    a.stages = per_split < kStages ? per_split : kStages;
-    if (a.stages < 1) a.stages = 1;
-    const size_t smem = (size_t)a.stages * (kStageA + a.block_n * BK * 2) + 1024;
-    gemm_tcgen05_kernel<<<grid, 192, smem, st>>>(A.map, B.map, a, A.mn_major, B.mn_major);
+    // ring depth: enough to cover a tile's reduction and keep loads of the next tile in flight
+    a.stages = per_split + 1 < kStages ? per_split + 1 : kStages;
+    if (a.stages < 2) a.stages = 2;
+    const size_t smem = (size_t)a.stages * (kStageA + a.block_n * BK * 2) + 4 * kEpiWarpBytes + 1024;
+    int per_sm = (int)((220u * 1024u) / smem);
+    if (per_sm > 2) per_sm = 2;   // 2 x 256 tensor-memory columns is all an SM has
+    if (per_sm < 1) per_sm = 1;
+    const long cap = 148L * per_sm;
+    const int grid = (int)(total < cap ? total : cap);
+    gemm_tcgen05_kernel<<<grid, 192, smem, st>>>(A.map, B.map, a, A.mn_major, B.mn_major, total, mt, nt);
     return cudaGetLastError();
 }
 
