@@ -138,6 +138,11 @@ int gala_learn(gala_ctx* ctx, int agent, const gala_rollout* rollout);
  * otherwise keep the local result (Eq. 5).  Never waits for a peer. */
 int gala_gossip(gala_ctx* ctx, int agent);
 
+/* Straggler injection for experiments (the slow simulators of Sec. 1 / Sec. 5 "computational
+ * performance"): keeps the agent's stream busy for about `usec` microseconds (0..100000) with one
+ * sleeping thread before whatever is enqueued next on it.  The wait is bounded on the device. */
+int gala_delay(gala_ctx* ctx, int agent, int usec);
+
 /* Deterministic synchronous round for all agents (Eq. 7 with zero delay):
  * learn on rollouts[0..n_agents), then x_i <- (y_i + sum_{j in N_in_i(k)} y_j)/(1+p)
  * with y the post-RMSProp parameters of the SAME round.  Runs on the

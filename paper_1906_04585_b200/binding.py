@@ -56,7 +56,7 @@ EXPORTS = (
     "gala_get_snapshot", "gala_set_stream", "gala_debug_read", "gala_launch_count",
     "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync", "gala_kernel_classes",
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
-    "gala_gemm_bf16_static",
+    "gala_gemm_bf16_static", "gala_delay",
 )
 
 _lib = None
@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
             "gala_act": (i, [vp, i, vp, vp, vp, vp]),
             "gala_learn": (i, [vp, i, C.POINTER(gala_rollout)]),
             "gala_gossip": (i, [vp, i]),
+            "gala_delay": (i, [vp, i, i]),
             "gala_step_sync": (i, [vp, C.POINTER(gala_rollout)]),
             "gala_sync_agent": (i, [vp, i, i]),
             "gala_sync_all": (i, [vp, i]),
@@ -161,6 +162,10 @@ def gala_learn(ctx, agent: int, rollout: gala_rollout):
 
 def gala_gossip(ctx, agent: int):
     _check(ctx, lib().gala_gossip(ctx, agent))
+
+
+def gala_delay(ctx, agent: int, usec: int):
+    _check(ctx, lib().gala_delay(ctx, agent, usec))
 
 
 def gala_step_sync(ctx, rollouts: Optional[Sequence[gala_rollout]]):

@@ -758,6 +758,15 @@ int gala_gossip(gala_ctx* c, int agent) {
     return GALA_OK;
 }
 
+int gala_delay(gala_ctx* c, int agent, int usec) {
+    if (!valid_agent(c, agent) || usec < 0 || usec > 100000)
+        return fail(c, GALA_EINVAL, "gala_delay: bad agent or delay outside 0..100000 us");
+    if (usec == 0) return GALA_OK;
+    Agent& ag = c->agents[agent];
+    CK(launch_delay((unsigned long long)usec, ag.stream));
+    return GALA_OK;
+}
+
 int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
     if (!c) return GALA_EINVAL;
     const int n = c->n;

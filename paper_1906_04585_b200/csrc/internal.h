@@ -108,6 +108,7 @@ cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const flo
 constexpr int kNormChunks = 128;
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
                              double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st);
+cudaError_t launch_delay(unsigned long long usec, cudaStream_t st);
 cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st);
 
 // ---------------------------------------------------------------- A2C pieces

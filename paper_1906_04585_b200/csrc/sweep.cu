@@ -245,6 +245,22 @@ cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int
     return cudaGetLastError();
 }
 
+// Straggler injection: occupies the stream for about `usec` microseconds (one sleeping thread).
+// Bounded twice: by the requested time (capped by the caller) and by an iteration limit.
+__global__ void delay_kernel(unsigned long long usec) {
+    unsigned long long t0, t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (int i = 0; i < 2000000; i++) {
+        __nanosleep(1000);
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        if (t - t0 >= usec * 1000ull) break;
+    }
+}
+cudaError_t launch_delay(unsigned long long usec, cudaStream_t st) {
+    delay_kernel<<<1, 1, 0, st>>>(usec);
+    return cudaGetLastError();
+}
+
 __global__ void cast_bf16_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ out, long n4) {
     for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x)
         st_bf16x4(out + i * 4, *reinterpret_cast<const float4*>(x + i * 4));
