@@ -55,7 +55,10 @@ def class_work(w: GI.Workload, d_pad: int):
     (hbm) or flops (tensor), summed over the launches of that class in one step."""
     n, E, T, A = w.n_agents, w.n_envs, w.n_steps, w.n_actions
     B, S = (T + 1) * E, T * E
-    out = {"sweep_sync": ("hbm", n * d_pad * (22.0 if w.net_kind == "conv" else 20.0)),
+    shadow = 2.0 if w.net_kind == "conv" else 0.0
+    out = {"sweep_sync": ("hbm", n * d_pad * (20.0 + shadow)),
+           # per-agent form: read x, g, v and p snapshots, write x, v and the own snapshot
+           "sweep_agent": ("hbm", n * d_pad * (24.0 + 4.0 * w.topo_peers + shadow)),
            "grad_norm": ("hbm", n * d_pad * 4.0)}
     if w.net_kind != "conv":
         return out
@@ -220,11 +223,38 @@ def run_ours(args):
     flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
     n_classes = B.gala_kernel_classes()
     work = class_work(w, L.d_pad)
+    async_mode = args.mode == "async" or (args.mode == "auto" and w.index == 4)
+    rng = np.random.default_rng(w.seed)
+    mean_delay_us = 0
+
+    def run_step(cur):
+        """One round: the synchronous all-agent call, or (async) every agent once on its own stream in
+        random order, each preceded by an injected straggler delay, nothing synchronised in between."""
+        if not async_mode:
+            L.step_sync(cur)
+            return
+        for i in rng.permutation(w.n_agents):
+            i = int(i)
+            if mean_delay_us > 0:
+                B.gala_delay(L.ctx, i, min(100000, int(rng.exponential(mean_delay_us))))
+            L.learn(i, cur[i])
+            L.gossip(i)
+
+    if async_mode:
+        # one agent's own step time sets the mean of the exponential straggler delay ("mean 1 step")
+        for _ in range(3):
+            L.learn(0, sets[0][0]); L.gossip(0)
+        L.sync()
+        t0 = time.perf_counter()
+        for _ in range(10):
+            L.learn(0, sets[0][0]); L.gossip(0)
+        L.sync()
+        mean_delay_us = 0 if args.no_skew else int(1e6 * (time.perf_counter() - t0) / 10)
 
     # warm-up; the first steps time every kernel class to find the dominant one
     B.gala_profile_enable(L.ctx, (1 << n_classes) - 1)
     for k in range(max(3, args.warmup)):
-        L.step_sync(sets[k % n_sets])
+        run_step(sets[k % n_sets])
     prof_all = B.gala_profile_read(L.ctx, reset=True)
     per_class_ms = {k: v[0] / max(3, args.warmup) for k, v in prof_all.items() if v[1] > 0}
     dominant = max(per_class_ms, key=per_class_ms.get)
@@ -245,7 +275,7 @@ def run_ours(args):
         with torch.cuda.stream(ext):
             flush.zero_()
         ev[k][0].record(ext)
-        L.step_sync(sets[k % n_sets])
+        run_step(sets[k % n_sets])
         ev[k][1].record(ext)
     L.sync()
     barrier()
@@ -254,6 +284,10 @@ def run_ours(args):
     clk = clocks.stop(t_clock0, time.time())
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = float(sum(step_ms))
+    if async_mode:
+        # agents run on their own streams: no single stream brackets a round, so the region is timed
+        # by the host clock between the two synchronisations (the L2 flushes are part of it)
+        total_ms = 1e3 * t_wall
     prof = B.gala_profile_read(L.ctx, reset=True)
     B.gala_profile_enable(L.ctx, 0)
     if world > 1:
@@ -286,7 +320,7 @@ def run_ours(args):
         for r in sets[k % n_sets]:
             r.upload(up)
         ext.wait_stream(up)
-        L.step_sync(sets[k % n_sets])
+        run_step(sets[k % n_sets])
         B.gala_losses(L.ctx, 0)
     barrier()
     t0 = time.perf_counter()
@@ -298,7 +332,9 @@ def run_ours(args):
     for k in range(args.steps):
         cur = sets[k % n_sets]
         ext.wait_stream(up)
-        L.step_sync(cur)
+        if async_mode:
+            up.synchronize()       # per-agent streams: make the copies visible to all of them
+        run_step(cur)
         if k + 1 < args.steps:
             for r in sets[(k + 1) % n_sets]:
                 r.upload(up)
@@ -317,12 +353,19 @@ def run_ours(args):
                 dtype="bf16" if w.net_kind == "conv" else "f32", data="synthetic",
                 config=dict(workload=w.name, n_agents=w.n_agents, envs_per_agent=w.n_envs, n_steps=w.n_steps,
                             frames_per_step=w.frames_per_round, topology="exp1" if w.topo_kind == GI.EXP else "ring1",
-                            mode="synchronous round (gala_step_sync)", l2="flushed between steps (252 MiB write)",
+                            mode=("asynchronous: per-agent streams, learn+gossip per agent in random order, straggler "
+                                  "delay ~Exp(mean %d us) per agent step" % mean_delay_us) if async_mode
+                            else "synchronous round (gala_step_sync)", l2="flushed between steps (252 MiB write)",
                             multi_gpu="replicas only" if world > 1 else "single"),
                 clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roofline,
                 wall_ms_per_step=1e3 * t_wall / args.steps,
                 kernel_ms_per_step={k: round(v, 5) for k, v in sorted(per_class_ms.items(), key=lambda kv: -kv[1])})
 
+    if async_mode:
+        st = [B.gala_stats(L.ctx, i) for i in range(w.n_agents)]
+        line["async"] = dict(mixes=sum(x["mixes"] for x in st), skipped=sum(x["skipped"] for x in st),
+                             staleness_mean=sum(x["staleness_sum"] for x in st) / max(1, sum(x["mixes"] for x in st)),
+                             staleness_max=max(x["staleness_max"] for x in st), timing="host clock between syncs")
     if rank == 0 and world == 1:
         line["sweep_microbench"] = sweep_microbench(torch, B, pk)
         if not args.no_cpu_baseline:
@@ -384,6 +427,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="index into gala_inputs.WORKLOADS (1 = the headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="auto", choices=["auto", "sync", "async"],
+                    help="auto: asynchronous per-agent streams for workload 4, synchronous rounds otherwise")
+    ap.add_argument("--no-skew", action="store_true", help="asynchronous mode without the injected straggler delays")
     ap.add_argument("--sweep-only", action="store_true",
                     help="run only the RMSProp + gossip micro-benchmark (32 agents x 1.7M parameters)")
     args = ap.parse_args()
