@@ -232,7 +232,28 @@ int build_plans(gala_ctx* c) {
         Plan& f = c->fwd[l];
         zero_args(f);
         f.tag = T_GEMM_CONV_FWD + l;
-        ok &= make_operand(&f.A, c->cols[l], 0, (uint64_t)B * P[l], KK, n, KK, (uint64_t)B * P[l] * KK, 128);
+        // conv2 / conv3 read their patches straight from the previous layer's activations: one TMA box
+        // per kernel offset holds the [patch][channel] block of nb samples (see gemm.cu, CONV_FWD)
+        const int nb = l == 1 ? 1 : 2;
+        if (l == 0) {
+            ok &= make_operand(&f.A, c->cols[0], 0, (uint64_t)B * P[l], KK, n, KK, (uint64_t)B * P[l] * KK, 128);
+        } else if (l == 1) {   // act1 [sample][20][20][32] seen as [sample][y/2][y%2][x/2][2 px x 32 ch]
+            const uint64_t dims[5] = {64, 10, 2, 10, (uint64_t)n * B};
+            const uint64_t str[4] = {128, 1280, 2560, 25600};
+            const uint32_t box[5] = {64, 9, 1, 9, 1};
+            ok &= make_tensor_map_nd(&f.A.map, c->act[0], 5, dims, str, box);
+            f.A.mn_major = 0;
+        } else {               // act2 [sample][9][9][64]
+            const uint64_t dims[4] = {64, 9, 9, (uint64_t)n * B};
+            const uint64_t str[3] = {128, 1152, 10368};
+            const uint32_t box[4] = {64, 7, 7, (uint32_t)nb};
+            ok &= make_tensor_map_nd(&f.A.map, c->act[1], 4, dims, str, box);
+            f.A.mn_major = 0;
+        }
+        if (l > 0) {
+            f.args.conv_mode = CONV_FWD; f.args.conv_layer = l; f.args.conv_nb = nb; f.args.a_samples = (int)B;
+            f.args.tile_rows = nb * P[l]; f.args.k_steps = KK / 64;
+        }
         ok &= make_operand(&f.B, c->shadow + c->cl.w[l], 0, CO, KK, n, KK, dp, bn);
         f.args.M = (int)(B * P[l]); f.args.N = CO; f.args.K = KK; f.args.block_n = bn;
         f.args.flags = EPI_OUT_BF16 | EPI_RELU;
@@ -243,8 +264,23 @@ int build_plans(gala_ctx* c) {
         Plan& w = c->wgrad[l];
         zero_args(w);
         w.tag = T_GEMM_CONV_WGRAD + l;
-        ok &= make_operand(&w.A, c->cols[l], 1, KK, (uint64_t)S * P[l], n, KK, (uint64_t)B * P[l] * KK, 128);
-        ok &= make_operand(&w.B, c->dy[l], 1, CO, (uint64_t)S * P[l], n, CO, (uint64_t)S * P[l] * CO, 64);
+        if (l == 0) {
+            ok &= make_operand(&w.A, c->cols[0], 1, KK, (uint64_t)S * P[l], n, KK, (uint64_t)B * P[l] * KK, 128);
+            ok &= make_operand(&w.B, c->dy[l], 1, CO, (uint64_t)S * P[l], n, CO, (uint64_t)S * P[l] * CO, 64);
+        } else {
+            // same activation boxes as the forward pass, now as the transposed patch matrix; dY comes in
+            // boxes of whole samples too, so that one K step is the patches of nb samples
+            w.A = f.A; w.A.mn_major = 1;
+            const uint64_t dims[4] = {64, (uint64_t)P[l], (uint64_t)S, (uint64_t)n};
+            const uint64_t str[3] = {128, (uint64_t)P[l] * 128, (uint64_t)S * P[l] * 128};
+            const uint32_t box[4] = {64, (uint32_t)P[l], (uint32_t)nb, 1};
+            ok &= make_tensor_map_nd(&w.B.map, c->dy[l], 4, dims, str, box);
+            w.B.mn_major = 1;
+            w.args.conv_mode = CONV_WGRAD; w.args.conv_layer = l; w.args.conv_nb = nb;
+            w.args.a_samples = (int)B; w.args.b_samples = (int)S;
+            w.args.kstep_rows = l == 1 ? 96 : 112;
+            w.args.tile_rows = 128; w.args.k_steps = (int)((S + nb - 1) / nb);
+        }
         w.args.M = KK; w.args.N = CO; w.args.K = (int)(S * P[l]); w.args.block_n = 64;
         w.args.flags = EPI_TRANSPOSE;
         w.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
@@ -306,7 +342,7 @@ int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override,
 
 // weight-gradient product with the reduction split over CTAs and a fixed-order second stage
 int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t st) {
-    const int k_tiles = (p.args.K + 63) / 64;
+    const int k_tiles = p.args.conv_mode != CONV_NONE ? p.args.k_steps : (p.args.K + 63) / 64;
     const int tiles = ((p.args.M + 127) / 128) * ((p.args.N + p.args.block_n - 1) / p.args.block_n);
     int split = (2 * 148) / (groups * tiles);
     if (split > k_tiles / 4) split = k_tiles / 4;
@@ -336,11 +372,6 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         for (int l = 0; l < 3; l++) {
             int r = run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st);
             if (r != GALA_OK) return r;
-            if (l < 2) {
-                const long as = B * P[l] * kConvCout[l], cs = B * P[l + 1] * kConvKK[l + 1];
-                LAUNCH(T_IM2COL_BF16, st, launch_im2col_bf16(c->act[l] + (long)agent0 * as, as, c->cols[l + 1] + (long)agent0 * cs, cs,
-                                          l + 1, rows, groups, st));
-            }
         }
         int r = run_plan(c, c->fc_fwd, agent0, groups, rows, st);
         if (r != GALA_OK) return r;
@@ -648,7 +679,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {
-            ALLOC(c->cols[l], (size_t)n * B * P[l] * kConvKK[l]);
+            if (l == 0) ALLOC(c->cols[l], (size_t)n * B * P[l] * kConvKK[l]);
             ALLOC(c->act[l], (size_t)n * B * P[l] * kConvCout[l]);
             ALLOC(c->dy[l], (size_t)n * S * P[l] * kConvCout[l]);
             if (l > 0) ALLOC(c->dcols[l], (size_t)n * S * P[l] * kConvKK[l]);

@@ -27,7 +27,7 @@ constexpr int BK = 64;           // K per stage = one 128-byte swizzle atom of b
 constexpr int kStages = 4;
 constexpr int kStageA = BM * BK * 2;    // 16 KiB
 constexpr int kStageB = 128 * BK * 2;   // room for block_n = 128
-constexpr int kSmemBytes = kStages * (kStageA + kStageB) + 4 * (32 * (32 * 4 + 16)) + 1024;  // ring + epilogue staging + slack
+constexpr int kSmemBytes = 200 * 1024;   // most dynamic shared memory a launch may ask for
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -69,6 +69,21 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                            int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                            int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
+          "r"(c4)
+        : "memory");
+}
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -80,8 +95,8 @@ __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fe
 //   offset is not used by swizzled K-major layouts.
 // MN-major tile: 64 contiguous M/N elements per 128-B row, 8 K-rows form a 1024-B group (stride
 //   offset), the next 64 M/N elements start one whole 64-row box later (leading offset, 8192 B).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int mn_major) {
-    const uint64_t lbo = mn_major ? (8192u >> 4) : 1u;
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int mn_major, uint32_t mn_atom_stride = 8192u) {
+    const uint64_t lbo = mn_major ? (mn_atom_stride >> 4) : 1u;
     const uint64_t sbo = 1024u >> 4;
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
 }
@@ -121,6 +136,11 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
 // Work decomposition shared by the three roles: tile index -> (group, split, m-tile, n-tile), n fastest
 // so that CTAs running side by side share an A tile in L2.
 struct TileCoord { int gz, split, m0, n0, kt_begin, num_k; };
@@ -131,8 +151,8 @@ __device__ __forceinline__ TileCoord decode_tile(const GemmArgs& p, long tile, i
     const int m_t = (int)(r % mt);
     const int z = (int)(r / mt);
     t.gz = z / p.split_k; t.split = z % p.split_k;
-    t.m0 = m_t * BM; t.n0 = n_t * p.block_n;
-    const int k_tiles = (p.K + BK - 1) / BK;
+    t.m0 = m_t * p.tile_rows; t.n0 = n_t * p.block_n;
+    const int k_tiles = p.k_steps;
     const int per_split = (k_tiles + p.split_k - 1) / p.split_k;
     t.kt_begin = t.split * per_split;
     const int kt_end = min(k_tiles, t.kt_begin + per_split);
@@ -162,10 +182,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int nst = p.stages;
     const int BN = p.block_n;
-    const int stage_b = BN * BK * 2;
+    const int stage_a = p.stage_a_bytes, stage_b = p.stage_b_bytes;
     uint8_t* smA = smem;
-    uint8_t* smB = smem + nst * kStageA;
+    uint8_t* smB = smem + nst * stage_a;
     uint8_t* smE = smB + nst * stage_b;   // epilogue staging, 4 x kEpiWarpBytes
+    const int conv = p.conv_mode;
+    // geometry of the implicit convolutions: patches per sample and 64-element blocks per patch
+    const int cP = p.conv_layer == 1 ? 81 : 49;
+    const int cQ = p.conv_layer == 1 ? 8 : 9;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t acc_cols = BN < 32 ? 32u : (uint32_t)BN;
@@ -184,6 +208,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    if (conv) {
+        // The boxes of the convolution modes fill only part of a stage (98 of 128 rows, 81 of 96, ...).
+        // The rest must read as zero wherever it takes part in a reduction, so the ring starts zeroed;
+        // TMA never writes those rows afterwards.
+        uint4* z = reinterpret_cast<uint4*>(smem);
+        const int n16 = nst * (stage_a + stage_b) / 16;
+        for (int i = threadIdx.x; i < n16; i += blockDim.x) z[i] = make_uint4(0, 0, 0, 0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     tcgen05_fence_before();
     __syncthreads();
     tcgen05_fence_after();
@@ -191,35 +224,65 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
-        if (lane == 0) {
-            const uint32_t bytes = (uint32_t)kStageA + (uint32_t)stage_b;
-            int it = 0;
-            bool ok = true;
-            for (long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const TileCoord t = decode_tile(p, tile, mt, nt);
-                const int group = p.group0 + t.gz;
-                for (int k = 0; k < t.num_k; k++, it++) {
-                    const int s = it % nst;
-                    const uint32_t ph = (uint32_t)(it / nst) & 1u;
-                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(&full_bar[s], bytes);
-                    const int k0 = (t.kt_begin + k) * BK;
-                    uint8_t* a = smA + s * kStageA;
-                    uint8_t* b = smB + s * stage_b;
-                    if (!a_mn) {
-                        tma_load_3d(a, &tmA, &full_bar[s], k0, t.m0, group);
+        // The whole warp walks the K steps.  Lane 0 waits for the stage and posts the byte count; the
+        // (up to four) tensor copies of a K step are then issued by lanes 0..3 side by side, because one
+        // thread needs some 200 ns per copy instruction.
+        const uint32_t bytes = (uint32_t)kStageA + (uint32_t)(BN * BK * 2);
+        const uint32_t box_bytes = (uint32_t)(cP * p.conv_nb * 128);   // one [patches of nb samples][64] box
+        int it = 0;
+        bool ok = true;
+        for (long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            const TileCoord t = decode_tile(p, tile, mt, nt);
+            const int group = p.group0 + t.gz;
+            for (int k = 0; k < t.num_k; k++, it++) {
+                const int s = it % nst;
+                const uint32_t ph = (uint32_t)(it / nst) & 1u;
+                int go = 1;
+                if (lane == 0) go = mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag) ? 1 : 0;
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (!go) { ok = false; break; }
+                const int k0 = (t.kt_begin + k) * BK;
+                uint8_t* a = smA + s * stage_a;
+                uint8_t* b = smB + s * stage_b;
+                if (conv) {
+                    // kernel offset of 64-element block q of a patch, and the TMA coordinates of the
+                    // [patch][channel] box that holds it for samples s0, s0+1, ...
+                    auto load_block = [&](uint8_t* dst, int q, int s0) {
+                        if (p.conv_layer == 1) {   // conv2: input seen as [sample][y/2][y%2][x/2][64]
+                            const int ky = q >> 1, h = q & 1;
+                            tma_load_5d(dst, &tmA, &full_bar[s], 0, h, ky & 1, ky >> 1, group * p.a_samples + s0);
+                        } else {                   // conv3: input [sample][y][x][64]
+                            const int ky = q / 3, kx = q - ky * 3;
+                            tma_load_4d(dst, &tmA, &full_bar[s], 0, kx, ky, group * p.a_samples + s0);
+                        }
+                    };
+                    if (conv == CONV_FWD) {
+                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes + (uint32_t)(BN * BK * 2));
+                        __syncwarp();
+                        if (lane == 0) load_block(a, t.kt_begin + k, (t.m0 / p.tile_rows) * p.conv_nb);
+                        else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], k0, t.n0, group);
                     } else {
-                        tma_load_3d(a, &tmA, &full_bar[s], t.m0, k0, group);
-                        tma_load_3d(a + 8192, &tmA, &full_bar[s], t.m0 + 64, k0, group);
+                        const int q0 = t.m0 / 64, s0 = (t.kt_begin + k) * p.conv_nb;
+                        const int nq = (q0 + 1 < cQ) ? 2 : 1;
+                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes * (uint32_t)(nq + 1));
+                        __syncwarp();
+                        if (lane < nq) load_block(a + lane * p.kstep_rows * 128, q0 + lane, s0);
+                        else if (lane == 2) tma_load_4d(b, &tmB, &full_bar[s], t.n0, 0, s0, group);
                     }
-                    if (!b_mn) {
-                        tma_load_3d(b, &tmB, &full_bar[s], k0, t.n0, group);
-                    } else {
-                        for (int j = 0; j < BN / 64; j++)
-                            tma_load_3d(b + j * 8192, &tmB, &full_bar[s], t.n0 + 64 * j, k0, group);
+                } else {
+                    if (lane == 0) mbar_expect_tx(&full_bar[s], bytes);
+                    __syncwarp();
+                    if (lane < 2) {          // A: one box (K-major) or two 64-wide boxes (MN-major)
+                        if (!a_mn) { if (lane == 0) tma_load_3d(a, &tmA, &full_bar[s], k0, t.m0, group); }
+                        else tma_load_3d(a + lane * 8192, &tmA, &full_bar[s], t.m0 + 64 * lane, k0, group);
+                    } else if (lane < 4) {   // B likewise
+                        const int j = lane - 2;
+                        if (!b_mn) { if (j == 0) tma_load_3d(b, &tmB, &full_bar[s], k0, t.n0, group); }
+                        else if (j < BN / 64) tma_load_3d(b + j * 8192, &tmB, &full_bar[s], t.n0 + 64 * j, k0, group);
                     }
-                    issued_iters = it + 1;
                 }
+                __syncwarp();
+                if (lane == 0) issued_iters = it + 1;
             }
         }
     } else if (warp == 1) {
@@ -240,14 +303,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t ph = (uint32_t)(it / nst) & 1u;
                     if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { ok = false; break; }
                     tcgen05_fence_after();
-                    const uint32_t a_addr = smem_u32(smA + s * kStageA);
+                    const uint32_t a_addr = smem_u32(smA + s * stage_a);
                     const uint32_t b_addr = smem_u32(smB + s * stage_b);
+                    if (conv == CONV_WGRAD) {
+                        // a K step is kstep_rows patches (the padding rows are zero on both sides)
+                        const uint32_t atom = (uint32_t)p.kstep_rows * 128u;
+                        for (int kk = 0; kk < p.kstep_rows / 16; kk++) {
+                            const uint64_t ad = make_smem_desc(a_addr + kk * 2048, 1, atom);
+                            const uint64_t bd = make_smem_desc(b_addr + kk * 2048, 1, atom);
+                            umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
+                        }
+                    } else {
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; kk++) {
-                        // one UMMA consumes K = 16: 32 B along a K-major row, 16 rows (2048 B) of an MN-major tile
-                        const uint64_t ad = make_smem_desc(a_addr + (a_mn ? kk * 2048 : kk * 32), a_mn);
-                        const uint64_t bd = make_smem_desc(b_addr + (b_mn ? kk * 2048 : kk * 32), b_mn);
-                        umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < BK / 16; kk++) {
+                            // one UMMA consumes K = 16: 32 B along a K-major row, 16 rows (2048 B) of an MN-major tile
+                            const uint64_t ad = make_smem_desc(a_addr + (a_mn ? kk * 2048 : kk * 32), a_mn);
+                            const uint64_t bd = make_smem_desc(b_addr + (b_mn ? kk * 2048 : kk * 32), b_mn);
+                            umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
+                        }
                     }
                     umma_commit(&empty_bar[s]);
                 }
@@ -288,11 +361,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     for (int j = 0; j < 32; j++) r[j] = 0u;
                 }
                 const int nb = t.n0 + c0;
-                if (mw >= p.M || nb >= p.N) continue;   // warp-uniform
+                if (mw >= p.M || q * 32 >= p.tile_rows || nb >= p.N) continue;   // warp-uniform
                 if (transpose) {
                     // D[m][n] -> out[n * ldc + m]: consecutive lanes write consecutive addresses
                     const int m = mw + lane;
-                    if (m < p.M) {
+                    if (m < p.M && q * 32 + lane < p.tile_rows) {
                         if (out_bf16) {
                             __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + obase + m;
 #pragma unroll
@@ -327,11 +400,54 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 __syncwarp();
                 const int cl = (lane & 7) * 4;          // first of this lane's 4 columns inside the block
                 const int n = nb + cl;
+                // fast path: the whole 32 x 32 block is inside the matrix and 16-byte stores are possible;
+                // straight-line code, the loads it needs (bias, mask) issued up front
+                if (vec_ok && mw + 32 <= p.M && q * 32 + 32 <= p.tile_rows && nb + 32 <= p.N && (!use_mask || mask_vec)) {
+                    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (bias) {
+                        if ((reinterpret_cast<uintptr_t>(bias + n) & 15) == 0) bv = __ldg(reinterpret_cast<const float4*>(bias + n));
+                        else bv = make_float4(__ldg(bias + n), __ldg(bias + n + 1), __ldg(bias + n + 2), __ldg(bias + n + 3));
+                    }
+                    const int r0 = lane >> 3;
+                    const long off0 = (long)(mw + r0) * p.ldc + n;
+                    const long rstep = 4L * p.ldc;
+                    uint2 mk[8];
+                    if (use_mask) {
+#pragma unroll
+                        for (int i = 0; i < 8; i++) mk[i] = __ldg(reinterpret_cast<const uint2*>(mask + off0 + i * rstep));
+                    }
+                    const uint8_t* sp = stage + r0 * kEpiRowBytes + cl * 4;
+#pragma unroll
+                    for (int i = 0; i < 8; i++) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(sp + i * 4 * kEpiRowBytes);
+                        float v0 = fmaf(__uint_as_float(raw.x), p.scale, bv.x), v1 = fmaf(__uint_as_float(raw.y), p.scale, bv.y);
+                        float v2 = fmaf(__uint_as_float(raw.z), p.scale, bv.z), v3 = fmaf(__uint_as_float(raw.w), p.scale, bv.w);
+                        if (relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); v2 = fmaxf(v2, 0.f); v3 = fmaxf(v3, 0.f); }
+                        if (use_mask) {
+                            const __nv_bfloat162* mh = reinterpret_cast<const __nv_bfloat162*>(&mk[i]);
+                            const float2 ma = __bfloat1622float2(mh[0]), mb = __bfloat1622float2(mh[1]);
+                            if (!(ma.x > 0.f)) v0 = 0.f;
+                            if (!(ma.y > 0.f)) v1 = 0.f;
+                            if (!(mb.x > 0.f)) v2 = 0.f;
+                            if (!(mb.y > 0.f)) v3 = 0.f;
+                        }
+                        const long off = obase + off0 + i * rstep;
+                        if (out_bf16) {
+                            uint2 u;
+                            u.x = pack2(v0, v1); u.y = pack2(v2, v3);
+                            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) = u;
+                        } else {
+                            *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) = make_float4(v0, v1, v2, v3);
+                        }
+                    }
+                    __syncwarp();
+                    continue;
+                }
 #pragma unroll
                 for (int i = 0; i < 8; i++) {
                     const int rr = i * 4 + (lane >> 3);
                     const int m = mw + rr;
-                    if (m >= p.M || n >= p.N) continue;
+                    if (m >= p.M || q * 32 + rr >= p.tile_rows || n >= p.N) continue;
                     const uint4 raw = *reinterpret_cast<const uint4*>(stage + rr * kEpiRowBytes + cl * 4);
                     float v[4] = {__uint_as_float(raw.x) * p.scale, __uint_as_float(raw.y) * p.scale,
                                   __uint_as_float(raw.z) * p.scale, __uint_as_float(raw.w) * p.scale};
@@ -483,6 +599,20 @@ bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint
     return r == CUDA_SUCCESS;
 }
 
+bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                        const uint64_t* strides_bytes, const uint32_t* box) {
+    if (!g_encode || rank < 3 || rank > 5) return false;
+    if (reinterpret_cast<uintptr_t>(base) & 15) return false;
+    cuuint64_t d[5], st[4];
+    cuuint32_t b[5], es[5];
+    for (int i = 0; i < rank; i++) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; if (box[i] > 256) return false; }
+    for (int i = 0; i + 1 < rank; i++) { st[i] = strides_bytes[i]; if (st[i] & 15) return false; }
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
                   uint64_t groups, uint64_t ld_elems, uint64_t group_stride_elems, int tile_mn) {
     op->mn_major = mn_major;
@@ -497,14 +627,46 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     if (B.mn_major && args.block_n < 64) return cudaErrorInvalidValue;
     if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
     GemmArgs a = args;
-    const int mt = (a.M + BM - 1) / BM, nt = (a.N + a.block_n - 1) / a.block_n;
+    if (a.conv_mode == CONV_NONE) {
+        a.tile_rows = BM;
+        a.k_steps = (a.K + BK - 1) / BK;
+        a.stage_a_bytes = kStageA;
+        a.stage_b_bytes = a.block_n * BK * 2;
+    } else {
+        if (a.conv_layer != 1 && a.conv_layer != 2) return cudaErrorInvalidValue;
+        const int P = a.conv_layer == 1 ? 81 : 49;
+        if (a.conv_nb < 1 || a.conv_nb * P > 128 || a.tile_rows < 1 || a.tile_rows > BM || a.k_steps < 1)
+            return cudaErrorInvalidValue;
+        if (a.conv_mode == CONV_FWD) {
+            if (A.mn_major || B.mn_major || a.tile_rows != a.conv_nb * P) return cudaErrorInvalidValue;
+            a.stage_a_bytes = kStageA;
+            a.stage_b_bytes = a.block_n * BK * 2;
+        } else {
+            if (!A.mn_major || !B.mn_major || a.block_n != 64 || a.kstep_rows % 16 || a.kstep_rows < a.conv_nb * P ||
+                a.kstep_rows > 128 || a.tile_rows != BM)
+                return cudaErrorInvalidValue;
+            a.stage_a_bytes = 2 * a.kstep_rows * 128;
+            a.stage_b_bytes = a.kstep_rows * 128;
+        }
+    }
+    const int mt = (a.M + a.tile_rows - 1) / a.tile_rows, nt = (a.N + a.block_n - 1) / a.block_n;
     const long total = (long)mt * nt * a.groups * a.split_k;
-    const int k_tiles = (a.K + BK - 1) / BK;
-    const int per_split = (k_tiles + a.split_k - 1) / a.split_k;
+    const int per_split = (a.k_steps + a.split_k - 1) / a.split_k;
     // ring depth: enough to cover a tile's reduction and keep loads of the next tile in flight
     a.stages = per_split + 1 < kStages ? per_split + 1 : kStages;
     if (a.stages < 2) a.stages = 2;
-    const size_t smem = (size_t)a.stages * (kStageA + a.block_n * BK * 2) + 4 * kEpiWarpBytes + 1024;
+    size_t smem = (size_t)a.stages * (a.stage_a_bytes + a.stage_b_bytes) + 4 * kEpiWarpBytes + 1024;
+    // two resident CTAs per SM (two producers, two MMA issuers, eight epilogue warps) beat one CTA
+    // with a deeper ring: shrink the ring until two fit
+    while (smem > (size_t)(110 * 1024) && a.stages > 2) {
+        a.stages--;
+        smem = (size_t)a.stages * (a.stage_a_bytes + a.stage_b_bytes) + 4 * kEpiWarpBytes + 1024;
+    }
+    while (smem > (size_t)kSmemBytes && a.stages > 2) {
+        a.stages--;
+        smem = (size_t)a.stages * (a.stage_a_bytes + a.stage_b_bytes) + 4 * kEpiWarpBytes + 1024;
+    }
+    if (smem > (size_t)kSmemBytes) return cudaErrorInvalidValue;
     int per_sm = (int)((220u * 1024u) / smem);
     if (per_sm > 2) per_sm = 2;   // 2 x 256 tensor-memory columns is all an SM has
     if (per_sm < 1) per_sm = 1;

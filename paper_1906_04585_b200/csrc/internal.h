@@ -68,7 +68,22 @@ struct GemmArgs {
     const __nv_bfloat16* mask;  // [m][n] with the output's ldc; group g at mask + g*mask_group_stride
     long mask_group_stride;
     int* error_word;       // device int, set non-zero when a bounded wait runs out
+    // Tiling (set by the caller for the convolution modes, filled with defaults by launch_gemm)
+    int tile_rows;         // rows of D per M tile (<= 128; default 128)
+    int k_steps;           // number of K steps of the whole reduction (default ceil(K/64))
+    // Implicit convolution operands (conv_mode != CONV_NONE): the patch matrix is never stored; TMA
+    // boxes over the NHWC activations deliver, for one kernel offset, the [patch][channel] block.
+    int conv_mode;
+    int conv_layer;        // 1: conv2 (4x4 stride 2 on 20x20x32), 2: conv3 (3x3 stride 1 on 9x9x64)
+    int conv_nb;           // samples per M tile (forward, data gradient) or per K step (weight gradient)
+    int a_samples;         // samples per group in the activation tensor behind A
+    int b_samples;         // weight gradient: samples per group in the dY tensor behind B
+    int kstep_rows;        // weight gradient: rows of a K step in shared memory (multiple of 16)
+    int stage_a_bytes, stage_b_bytes;   // set by launch_gemm
 };
+//   CONV_FWD  : D[patch][co]  = sum_k patches[patch][k] W[co][k]      A from boxes, B = weights (K-major)
+//   CONV_WGRAD: D[k][co]      = sum_patch patches[patch][k] dY[patch][co]   A (transposed patches) and B from boxes
+enum ConvMode : int { CONV_NONE = 0, CONV_FWD = 1, CONV_WGRAD = 2 };
 
 cudaError_t gemm_init();   // resolves the driver entry point used to build TMA descriptors
 // rows x cols bf16 matrix per group, cols contiguous.  box_rows x box_cols tile.
@@ -78,6 +93,9 @@ bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t
 // rows x cols fp32 matrix, unswizzled box_rows x box_cols tile (gemm_init() first).
 bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
                          uint32_t box_cols, uint32_t box_rows);
+// General bf16 tensor map of rank 3..5, 128-byte swizzle (dims/strides innermost first).
+bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                        const uint64_t* strides_bytes, const uint32_t* box);
 // Builds the descriptor for an operand of a GEMM with the given tile height
 // (128 for A, block_n for B).
 bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
