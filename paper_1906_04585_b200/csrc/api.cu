@@ -93,7 +93,6 @@ struct gala_ctx {
     // conv workspaces (bf16)
     __nv_bfloat16 *cols[3] = {nullptr, nullptr, nullptr}, *act[3] = {nullptr, nullptr, nullptr};
     __nv_bfloat16 *hid = nullptr, *dh = nullptr, *dy[3] = {nullptr, nullptr, nullptr};
-    float* dcols[3] = {nullptr, nullptr, nullptr};  // patch gradients stay fp32 until they are summed
     float* splitk_ws = nullptr;
     long splitk_group_stride = 0;
     int max_split = 32;
@@ -252,7 +251,7 @@ int build_plans(gala_ctx* c) {
         }
         if (l > 0) {
             f.args.conv_mode = CONV_FWD; f.args.conv_layer = l; f.args.conv_nb = nb; f.args.a_samples = (int)B;
-            f.args.tile_rows = nb * P[l]; f.args.k_steps = KK / 64;
+            f.args.tile_rows = nb * P[l]; f.args.box_rows = nb * P[l]; f.args.k_steps = KK / 64;
         }
         ok &= make_operand(&f.B, c->shadow + c->cl.w[l], 0, CO, KK, n, KK, dp, bn);
         f.args.M = (int)(B * P[l]); f.args.N = CO; f.args.K = KK; f.args.block_n = bn;
@@ -279,22 +278,37 @@ int build_plans(gala_ctx* c) {
             w.args.conv_mode = CONV_WGRAD; w.args.conv_layer = l; w.args.conv_nb = nb;
             w.args.a_samples = (int)B; w.args.b_samples = (int)S;
             w.args.kstep_rows = l == 1 ? 96 : 112;
-            w.args.tile_rows = 128; w.args.k_steps = (int)((S + nb - 1) / nb);
+            w.args.tile_rows = 128; w.args.box_rows = nb * P[l]; w.args.k_steps = (int)((S + nb - 1) / nb);
         }
         w.args.M = KK; w.args.N = CO; w.args.K = (int)(S * P[l]); w.args.block_n = 64;
         w.args.flags = EPI_TRANSPOSE;
         w.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
         w.args.out = c->g + c->cl.w[l]; w.args.out_group_stride = dp; w.args.ldc = KK;
-        // data gradient (conv2, conv3): dY [S*P][CO] x W[CO][KK] -> patch gradients [S*P][KK]
+        // data gradient (conv2, conv3), implicit: the gradient of the layer's INPUT pixels is summed over the
+        // kernel offsets inside the accumulator (no patch gradients in memory), gated by the ReLU of the
+        // input activation in the epilogue and stored as the previous layer's dY
         if (l > 0) {
             Plan& dg = c->dgrad[l];
             zero_args(dg);
             dg.tag = T_GEMM_CONV_DGRAD + l;
-            ok &= make_operand(&dg.A, c->dy[l], 0, (uint64_t)S * P[l], CO, n, CO, (uint64_t)S * P[l] * CO, 128);
-            ok &= make_operand(&dg.B, c->shadow + c->cl.w[l], 1, KK, CO, n, KK, dp, 128);
-            dg.args.M = (int)(S * P[l]); dg.args.N = KK; dg.args.K = CO; dg.args.block_n = 128;
-            dg.args.flags = 0;
-            dg.args.out = c->dcols[l]; dg.args.out_group_stride = S * P[l] * KK; dg.args.ldc = KK;
+            const int ow = kConvOut[l], in_pix = kConvIn[l] * kConvIn[l], cin = kConvCin[l];
+            const uint64_t dims[4] = {64, (uint64_t)ow, (uint64_t)ow, (uint64_t)n * S};
+            const uint64_t str[3] = {128, (uint64_t)ow * 128, (uint64_t)ow * ow * 128};
+            const uint32_t box[4] = {64, l == 2 ? 9u : 10u, l == 2 ? 9u : 10u, 1};
+            ok &= make_tensor_map_nd(&dg.A.map, c->dy[l], 4, dims, str, box);
+            dg.A.mn_major = 0;
+            const uint64_t wd[3] = {(uint64_t)KK, (uint64_t)CO, (uint64_t)n};
+            const uint64_t ws[2] = {(uint64_t)KK * 2, (uint64_t)dp * 2};
+            const uint32_t wb[3] = {64, 64, 1};
+            ok &= make_tensor_map_nd(&dg.B.map, c->shadow + c->cl.w[l], 3, wd, ws, wb);
+            dg.B.mn_major = 1;
+            dg.args.M = (int)(S * in_pix); dg.args.N = cin; dg.args.K = KK; dg.args.block_n = 64;
+            dg.args.conv_mode = CONV_DGRAD; dg.args.conv_layer = l; dg.args.conv_nb = 1; dg.args.a_samples = (int)S;
+            dg.args.tile_rows = l == 2 ? 81 : 100; dg.args.box_rows = dg.args.tile_rows;
+            dg.args.k_steps = l == 2 ? 9 : 4;
+            dg.args.flags = EPI_OUT_BF16 | EPI_MASK | (l == 1 ? EPI_ROWMAP_S2 : 0);
+            dg.args.mask = c->act[l - 1]; dg.args.mask_group_stride = B * in_pix * cin;
+            dg.args.out = c->dy[l - 1]; dg.args.out_group_stride = S * in_pix * cin; dg.args.ldc = cin;
         }
     }
     {   // hidden layer forward: act3 [B][3136] x Wfc[512][3136]^T -> hid (bias, ReLU)
@@ -449,13 +463,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         for (int l = 2; l >= 0; l--) {
             const int CO = kConvCout[l];
             if ((r = run_wgrad(c, c->wgrad[l], agent0, groups, st)) != GALA_OK) return r;
-            if (l > 0) {
-                if ((r = run_plan(c, c->dgrad[l], agent0, groups, 0, st)) != GALA_OK) return r;
-                const long ds = S * P[l] * kConvKK[l], as = B * P[l - 1] * kConvCout[l - 1],
-                           xs = S * P[l - 1] * kConvCout[l - 1];
-                LAUNCH(T_COL2IM, st, launch_col2im(c->dcols[l] + (long)agent0 * ds, ds, c->act[l - 1] + (long)agent0 * as, as,
-                                     c->dy[l - 1] + (long)agent0 * xs, xs, l, (int)S, groups, st));
-            }
+            if (l > 0 && (r = run_plan(c, c->dgrad[l], agent0, groups, 0, st)) != GALA_OK) return r;
         }
         {   // all four bias gradients (column sums of dh, dY3, dY2, dY1) in one launch
             ColsumJobs jobs{};
@@ -682,7 +690,6 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
             if (l == 0) ALLOC(c->cols[l], (size_t)n * B * P[l] * kConvKK[l]);
             ALLOC(c->act[l], (size_t)n * B * P[l] * kConvCout[l]);
             ALLOC(c->dy[l], (size_t)n * S * P[l] * kConvCout[l]);
-            if (l > 0) ALLOC(c->dcols[l], (size_t)n * S * P[l] * kConvKK[l]);
         }
         ALLOC(c->hid, (size_t)n * B * kHidden);
         ALLOC(c->dh, (size_t)n * S * kHidden);

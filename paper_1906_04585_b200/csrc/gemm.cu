@@ -166,7 +166,7 @@ constexpr int kEpiWarpBytes = 32 * kEpiRowBytes;   // staging area of one epilog
 // Persistent CTA: loops over output tiles.  The shared-memory ring runs on across tiles, and the
 // accumulator is double-buffered in tensor memory, so the loads and MMAs of tile i+1 overlap the
 // epilogue of tile i.
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmArgs p, const int a_mn, const int b_mn, const long total_tiles, const int mt,
                     const int nt) {
@@ -228,7 +228,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // (up to four) tensor copies of a K step are then issued by lanes 0..3 side by side, because one
         // thread needs some 200 ns per copy instruction.
         const uint32_t bytes = (uint32_t)kStageA + (uint32_t)(BN * BK * 2);
-        const uint32_t box_bytes = (uint32_t)(cP * p.conv_nb * 128);   // one [patches of nb samples][64] box
+        const uint32_t box_bytes = (uint32_t)(p.box_rows * 128);   // one [patches or pixels][64 channels] box
         int it = 0;
         bool ok = true;
         for (long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
@@ -256,7 +256,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                             tma_load_4d(dst, &tmA, &full_bar[s], 0, kx, ky, group * p.a_samples + s0);
                         }
                     };
-                    if (conv == CONV_FWD) {
+                    if (conv == CONV_DGRAD) {
+                        // K step = one kernel offset; the dY box is shifted by it, the weights' [co][ci]
+                        // block of that offset is a 64-wide column block of W[co][(ky, kx, ci)]
+                        int sample, oy_shift, ox_shift, wcol;
+                        const int j = t.kt_begin + k;
+                        if (p.conv_layer == 2) {          // conv3, stride 1: pixel (y, x) <- dY[y - ky][x - kx]
+                            sample = t.m0 / 81;
+                            oy_shift = j / 3; ox_shift = j - oy_shift * 3;
+                            wcol = j * 64;
+                        } else {                          // conv2, stride 2: class (py, px), pixel (2a+py, 2c+px)
+                            sample = t.m0 / 400;          //   <- dY[a - dy][c - dx] with ky = py + 2dy, kx = px + 2dx
+                            const int cls = (t.m0 / 100) & 3;
+                            oy_shift = j >> 1; ox_shift = j & 1;
+                            wcol = (((cls >> 1) + 2 * oy_shift) * 4 + (cls & 1) + 2 * ox_shift) * 32;
+                        }
+                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes + 8192u);
+                        __syncwarp();
+                        if (lane == 0) tma_load_4d(a, &tmA, &full_bar[s], 0, -ox_shift, -oy_shift, group * p.a_samples + sample);
+                        else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], wcol, 0, group);
+                    } else if (conv == CONV_FWD) {
                         if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes + (uint32_t)(BN * BK * 2));
                         __syncwarp();
                         if (lane == 0) load_block(a, t.kt_begin + k, (t.m0 / p.tile_rows) * p.conv_nb);
@@ -352,6 +371,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const float* bias = p.bias ? p.bias + (long)group * p.bias_group_stride : nullptr;
             const __nv_bfloat16* mask = use_mask ? p.mask + (long)t.gz * p.mask_group_stride : nullptr;
             const int mw = t.m0 + q * 32;   // first row of this warp
+            const bool rowmap = p.flags & EPI_ROWMAP_S2;
+            // element offset (inside the group) of output row r of this tile
+            auto row_off = [&](int r) -> long {
+                if (!rowmap) return (long)(t.m0 + r) * p.ldc;
+                const int sample = t.m0 / 400, cls = (t.m0 / 100) & 3;
+                const int ra = r / 10, rc = r - ra * 10;
+                return ((long)(sample * 20 + 2 * ra + (cls >> 1)) * 20 + 2 * rc + (cls & 1)) * p.ldc;
+            };
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 if (t.num_k > 0) {
@@ -409,12 +436,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         else bv = make_float4(__ldg(bias + n), __ldg(bias + n + 1), __ldg(bias + n + 2), __ldg(bias + n + 3));
                     }
                     const int r0 = lane >> 3;
-                    const long off0 = (long)(mw + r0) * p.ldc + n;
-                    const long rstep = 4L * p.ldc;
+                    long roff[8];
+#pragma unroll
+                    for (int i = 0; i < 8; i++) roff[i] = row_off(q * 32 + r0 + 4 * i) + n;
                     uint2 mk[8];
                     if (use_mask) {
 #pragma unroll
-                        for (int i = 0; i < 8; i++) mk[i] = __ldg(reinterpret_cast<const uint2*>(mask + off0 + i * rstep));
+                        for (int i = 0; i < 8; i++) mk[i] = __ldg(reinterpret_cast<const uint2*>(mask + roff[i]));
                     }
                     const uint8_t* sp = stage + r0 * kEpiRowBytes + cl * 4;
 #pragma unroll
@@ -431,7 +459,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                             if (!(mb.x > 0.f)) v2 = 0.f;
                             if (!(mb.y > 0.f)) v3 = 0.f;
                         }
-                        const long off = obase + off0 + i * rstep;
+                        const long off = obase + roff[i];
                         if (out_bf16) {
                             uint2 u;
                             u.x = pack2(v0, v1); u.y = pack2(v2, v3);
@@ -460,7 +488,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                         for (int j = 0; j < 4; j++) v[j] = fmaxf(v[j], 0.0f);
                     }
-                    const long off = (long)m * p.ldc + n;
+                    const long off = row_off(q * 32 + rr) + n;
                     if (use_mask) {
                         if (mask_vec && valid == 4 && ((off & 3) == 0)) {
                             const uint2 mk = __ldg(reinterpret_cast<const uint2*>(mask + off));
@@ -635,12 +663,17 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     } else {
         if (a.conv_layer != 1 && a.conv_layer != 2) return cudaErrorInvalidValue;
         const int P = a.conv_layer == 1 ? 81 : 49;
-        if (a.conv_nb < 1 || a.conv_nb * P > 128 || a.tile_rows < 1 || a.tile_rows > BM || a.k_steps < 1)
-            return cudaErrorInvalidValue;
+        if (a.conv_nb < 1 || a.tile_rows < 1 || a.tile_rows > BM || a.k_steps < 1) return cudaErrorInvalidValue;
+        if (a.conv_mode != CONV_DGRAD && a.conv_nb * P > 128) return cudaErrorInvalidValue;
+        if (a.box_rows < 1 || a.box_rows > 128) return cudaErrorInvalidValue;
         if (a.conv_mode == CONV_FWD) {
-            if (A.mn_major || B.mn_major || a.tile_rows != a.conv_nb * P) return cudaErrorInvalidValue;
+            if (A.mn_major || B.mn_major || a.tile_rows != a.conv_nb * P || a.box_rows != a.tile_rows) return cudaErrorInvalidValue;
             a.stage_a_bytes = kStageA;
             a.stage_b_bytes = a.block_n * BK * 2;
+        } else if (a.conv_mode == CONV_DGRAD) {
+            if (A.mn_major || !B.mn_major || a.block_n != 64 || a.tile_rows != a.box_rows) return cudaErrorInvalidValue;
+            a.stage_a_bytes = kStageA;
+            a.stage_b_bytes = 64 * BK * 2;
         } else {
             if (!A.mn_major || !B.mn_major || a.block_n != 64 || a.kstep_rows % 16 || a.kstep_rows < a.conv_nb * P ||
                 a.kstep_rows > 128 || a.tile_rows != BM)

@@ -47,7 +47,9 @@ enum EpilogueFlags : int {
     EPI_OUT_BF16 = 1,    // store bf16 (else fp32)
     EPI_RELU = 2,        // max(.,0) after scale and bias
     EPI_TRANSPOSE = 4,   // store D[m][n] at out[n*ldc + m]
-    EPI_MASK = 8         // multiply by (mask[m][n] > 0), mask bf16 with the output's layout
+    EPI_MASK = 8,        // multiply by (mask[m][n] > 0), mask bf16 with the output's layout
+    EPI_ROWMAP_S2 = 16   // rows are (sample, parity class, a, c) of a stride-2 data gradient: row r of tile
+                         // (sample, class) goes to pixel (2a + class/2, 2c + class%2) of the 20x20 input grid
 };
 
 struct GemmArgs {
@@ -79,11 +81,14 @@ struct GemmArgs {
     int a_samples;         // samples per group in the activation tensor behind A
     int b_samples;         // weight gradient: samples per group in the dY tensor behind B
     int kstep_rows;        // weight gradient: rows of a K step in shared memory (multiple of 16)
+    int box_rows;          // rows of one A box (patches or pixels it delivers)
     int stage_a_bytes, stage_b_bytes;   // set by launch_gemm
 };
 //   CONV_FWD  : D[patch][co]  = sum_k patches[patch][k] W[co][k]      A from boxes, B = weights (K-major)
 //   CONV_WGRAD: D[k][co]      = sum_patch patches[patch][k] dY[patch][co]   A (transposed patches) and B from boxes
-enum ConvMode : int { CONV_NONE = 0, CONV_FWD = 1, CONV_WGRAD = 2 };
+//   CONV_DGRAD: dX[pixel][ci] = sum_{offset, co} dY[pixel - offset][co] W[co][offset][ci]; A = boxes of dY shifted
+//               by the kernel offset (out-of-range entries read as zero), B = the offset's [co][ci] block of W
+enum ConvMode : int { CONV_NONE = 0, CONV_FWD = 1, CONV_WGRAD = 2, CONV_DGRAD = 3 };
 
 cudaError_t gemm_init();   // resolves the driver entry point used to build TMA descriptors
 // rows x cols bf16 matrix per group, cols contiguous.  box_rows x box_cols tile.
