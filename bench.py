@@ -63,8 +63,7 @@ def class_work(w: GI.Workload, d_pad: int):
     if w.net_kind != "conv":
         return out
     P, KK, CO = (400, 81, 49), (256, 512, 576), (32, 64, 64)
-    out["im2col_u8"] = ("hbm", n * B * (84 * 84 * 4 + 400 * 256 * 2.0))
-    out["im2col_bf16"] = ("hbm", n * B * ((400 * 32 + 81 * 512) * 2.0 + (81 * 64 + 49 * 576) * 2.0))
+    out["cast_frames"] = ("hbm", n * B * (84 * 84 * 4 * 3.0))      # uint8 in, bf16 out
     for l in range(3):
         out["gemm_conv%d_fwd" % (l + 1)] = ("tensor", 2.0 * n * B * P[l] * KK[l] * CO[l])
         out["gemm_conv%d_wgrad" % (l + 1)] = ("tensor", 2.0 * n * S * P[l] * KK[l] * CO[l])
@@ -73,7 +72,6 @@ def class_work(w: GI.Workload, d_pad: int):
     out["gemm_fc_fwd"] = ("tensor", 2.0 * n * B * 3136 * 512)
     out["gemm_fc_wgrad"] = ("tensor", 2.0 * n * S * 3136 * 512)
     out["gemm_fc_dgrad"] = ("tensor", 2.0 * n * S * 3136 * 512)
-    out["col2im"] = ("hbm", n * S * ((49 * 576 * 4.0 + 81 * 64 * 4.0) + (81 * 512 * 4.0 + 400 * 32 * 4.0)))
     out["colsum"] = ("hbm", n * S * (512 + 49 * 64 + 81 * 64 + 400 * 32) * 2.0)
     return out
 

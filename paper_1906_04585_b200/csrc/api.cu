@@ -12,6 +12,8 @@
 
 using namespace gala;
 
+constexpr long kFramePix = 84L * 84 * 4;
+
 namespace {
 
 struct Agent {
@@ -47,7 +49,7 @@ enum Tag : int {
     T_COUNT = T_GEMM_CONV_DGRAD + 3
 };
 const char* const kTagNames[T_COUNT] = {
-    "im2col_u8", "im2col_bf16", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "col2im", "grad_norm",
+    "cast_frames", "im2col_bf16", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "col2im", "grad_norm",
     "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16",
     "gemm_conv1_fwd", "gemm_conv2_fwd", "gemm_conv3_fwd", "gemm_fc_fwd", "gemm_fc_wgrad", "gemm_fc_dgrad",
     "gemm_conv1_wgrad", "gemm_conv2_wgrad", "gemm_conv3_wgrad", "gemm_conv1_dgrad", "gemm_conv2_dgrad",
@@ -91,7 +93,8 @@ struct gala_ctx {
     // MLP workspaces
     float *h1 = nullptr, *h2 = nullptr, *dpre1 = nullptr, *dpre2 = nullptr;
     // conv workspaces (bf16)
-    __nv_bfloat16 *cols[3] = {nullptr, nullptr, nullptr}, *act[3] = {nullptr, nullptr, nullptr};
+    __nv_bfloat16* frames = nullptr;   // bf16 copies of the uint8 frames, [N][B][84][84][4]
+    __nv_bfloat16* act[3] = {nullptr, nullptr, nullptr};
     __nv_bfloat16 *hid = nullptr, *dh = nullptr, *dy[3] = {nullptr, nullptr, nullptr};
     float* splitk_ws = nullptr;
     long splitk_group_stride = 0;
@@ -235,7 +238,14 @@ int build_plans(gala_ctx* c) {
         // per kernel offset holds the [patch][channel] block of nb samples (see gemm.cu, CONV_FWD)
         const int nb = l == 1 ? 1 : 2;
         if (l == 0) {
-            ok &= make_operand(&f.A, c->cols[0], 0, (uint64_t)B * P[l], KK, n, KK, (uint64_t)B * P[l] * KK, 128);
+            // bf16 frames [sample][84][84][4] seen as [sample][y/4][y%4][ox][8 px x 4 ch]: the 20 windows of a
+            // row overlap by half (stride 4 px = 32 B under a 64 B extent); one box = one kernel row of the
+            // 100 patches of a quarter sample
+            const uint64_t dims[5] = {32, 20, 4, 21, (uint64_t)n * B};
+            const uint64_t str[4] = {32, 672, 2688, 56448};
+            const uint32_t box[5] = {32, 20, 1, 5, 1};
+            ok &= make_tensor_map_nd(&f.A.map, c->frames, 5, dims, str, box, 1);
+            f.A.mn_major = 0;
         } else if (l == 1) {   // act1 [sample][20][20][32] seen as [sample][y/2][y%2][x/2][2 px x 32 ch]
             const uint64_t dims[5] = {64, 10, 2, 10, (uint64_t)n * B};
             const uint64_t str[4] = {128, 1280, 2560, 25600};
@@ -249,11 +259,18 @@ int build_plans(gala_ctx* c) {
             ok &= make_tensor_map_nd(&f.A.map, c->act[1], 4, dims, str, box);
             f.A.mn_major = 0;
         }
-        if (l > 0) {
-            f.args.conv_mode = CONV_FWD; f.args.conv_layer = l; f.args.conv_nb = nb; f.args.a_samples = (int)B;
+        f.args.conv_mode = CONV_FWD; f.args.conv_layer = l; f.args.conv_nb = nb; f.args.a_samples = (int)B;
+        if (l == 0) {
+            f.args.conv_nb = 1; f.args.tile_rows = 100; f.args.box_rows = 100; f.args.k_steps = 8;
+            const uint64_t wd[3] = {(uint64_t)KK, (uint64_t)CO, (uint64_t)n};
+            const uint64_t ws[2] = {(uint64_t)KK * 2, (uint64_t)dp * 2};
+            const uint32_t wb[3] = {32, 32, 1};
+            ok &= make_tensor_map_nd(&f.B.map, c->shadow + c->cl.w[0], 3, wd, ws, wb, 1);
+            f.B.mn_major = 0;
+        } else {
             f.args.tile_rows = nb * P[l]; f.args.box_rows = nb * P[l]; f.args.k_steps = KK / 64;
+            ok &= make_operand(&f.B, c->shadow + c->cl.w[l], 0, CO, KK, n, KK, dp, bn);
         }
-        ok &= make_operand(&f.B, c->shadow + c->cl.w[l], 0, CO, KK, n, KK, dp, bn);
         f.args.M = (int)(B * P[l]); f.args.N = CO; f.args.K = KK; f.args.block_n = bn;
         f.args.flags = EPI_OUT_BF16 | EPI_RELU;
         f.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
@@ -264,8 +281,17 @@ int build_plans(gala_ctx* c) {
         zero_args(w);
         w.tag = T_GEMM_CONV_WGRAD + l;
         if (l == 0) {
-            ok &= make_operand(&w.A, c->cols[0], 1, KK, (uint64_t)S * P[l], n, KK, (uint64_t)B * P[l] * KK, 128);
-            ok &= make_operand(&w.B, c->dy[l], 1, CO, (uint64_t)S * P[l], n, CO, (uint64_t)S * P[l] * CO, 64);
+            // transposed patch matrix from the same frame boxes (4 kernel rows = 128 patch elements per M
+            // tile); dY1 [sample][400][32] in boxes of the 100 patches of a quarter sample
+            w.A = f.A; w.A.mn_major = 1;
+            const uint64_t dims[3] = {32, 400, (uint64_t)n * S};
+            const uint64_t str[2] = {64, 25600};
+            const uint32_t box[3] = {32, 100, 1};
+            ok &= make_tensor_map_nd(&w.B.map, c->dy[0], 3, dims, str, box, 1);
+            w.B.mn_major = 1;
+            w.args.conv_mode = CONV_WGRAD; w.args.conv_layer = 0; w.args.conv_nb = 1;
+            w.args.a_samples = (int)B; w.args.b_samples = (int)S;
+            w.args.kstep_rows = 112; w.args.tile_rows = 128; w.args.box_rows = 100; w.args.k_steps = (int)(S * 4);
         } else {
             // same activation boxes as the forward pass, now as the transposed patch matrix; dY comes in
             // boxes of whole samples too, so that one K step is the patches of nb samples
@@ -280,7 +306,7 @@ int build_plans(gala_ctx* c) {
             w.args.kstep_rows = l == 1 ? 96 : 112;
             w.args.tile_rows = 128; w.args.box_rows = nb * P[l]; w.args.k_steps = (int)((S + nb - 1) / nb);
         }
-        w.args.M = KK; w.args.N = CO; w.args.K = (int)(S * P[l]); w.args.block_n = 64;
+        w.args.M = KK; w.args.N = CO; w.args.K = (int)(S * P[l]); w.args.block_n = l == 0 ? 32 : 64;
         w.args.flags = EPI_TRANSPOSE;
         w.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
         w.args.out = c->g + c->cl.w[l]; w.args.out_group_stride = dp; w.args.ldc = KK;
@@ -382,7 +408,7 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
     const long dp = c->d_pad, B = c->B;
     if (c->conv) {
         const int P[3] = {400, 81, 49};
-        LAUNCH(T_IM2COL_U8, st, launch_im2col_u8(obs, c->cols[0] + (long)agent0 * B * 400 * 256, B * 400 * 256, rows, groups, st));
+        LAUNCH(T_IM2COL_U8, st, launch_cast_frames(obs, c->frames + (long)agent0 * B * kFramePix, B * kFramePix, rows, groups, st));
         for (int l = 0; l < 3; l++) {
             int r = run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st);
             if (r != GALA_OK) return r;
@@ -687,10 +713,10 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {
-            if (l == 0) ALLOC(c->cols[l], (size_t)n * B * P[l] * kConvKK[l]);
             ALLOC(c->act[l], (size_t)n * B * P[l] * kConvCout[l]);
             ALLOC(c->dy[l], (size_t)n * S * P[l] * kConvCout[l]);
         }
+        ALLOC(c->frames, (size_t)n * B * kFramePix);
         ALLOC(c->hid, (size_t)n * B * kHidden);
         ALLOC(c->dh, (size_t)n * S * kHidden);
         c->splitk_group_stride = (long)c->max_split * 64 * 576;

@@ -95,10 +95,13 @@ __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fe
 //   offset is not used by swizzled K-major layouts.
 // MN-major tile: 64 contiguous M/N elements per 128-B row, 8 K-rows form a 1024-B group (stride
 //   offset), the next 64 M/N elements start one whole 64-row box later (leading offset, 8192 B).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int mn_major, uint32_t mn_atom_stride = 8192u) {
+// With 64-byte rows (conv1: one kernel row of a patch is 32 bf16) the 64-byte swizzle is used
+// instead: layout type 4, groups of 8 rows 512 B apart, MN-major atoms 32 elements wide.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int mn_major, uint32_t mn_atom_stride = 8192u,
+                                                   int sw64 = 0) {
     const uint64_t lbo = mn_major ? (mn_atom_stride >> 4) : 1u;
-    const uint64_t sbo = 1024u >> 4;
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+    const uint64_t sbo = (sw64 ? 512u : 1024u) >> 4;
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | ((sw64 ? 4ull : 2ull) << 61);
 }
 // Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B.
 __device__ __forceinline__ uint32_t make_instr_desc(int block_n, int a_mn, int b_mn) {
@@ -188,8 +191,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     uint8_t* smE = smB + nst * stage_b;   // epilogue staging, 4 x kEpiWarpBytes
     const int conv = p.conv_mode;
     // geometry of the implicit convolutions: patches per sample and 64-element blocks per patch
-    const int cP = p.conv_layer == 1 ? 81 : 49;
     const int cQ = p.conv_layer == 1 ? 8 : 9;
+    const int sw64 = conv && p.conv_layer == 0;   // conv1: 64-byte rows
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t acc_cols = BN < 32 ? 32u : (uint32_t)BN;
@@ -228,7 +231,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // (up to four) tensor copies of a K step are then issued by lanes 0..3 side by side, because one
         // thread needs some 200 ns per copy instruction.
         const uint32_t bytes = (uint32_t)kStageA + (uint32_t)(BN * BK * 2);
-        const uint32_t box_bytes = (uint32_t)(p.box_rows * 128);   // one [patches or pixels][64 channels] box
+        const uint32_t box_bytes = (uint32_t)(p.box_rows * (sw64 ? 64 : 128));   // one [patches or pixels][channels] box
         int it = 0;
         bool ok = true;
         for (long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
@@ -248,7 +251,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     // kernel offset of 64-element block q of a patch, and the TMA coordinates of the
                     // [patch][channel] box that holds it for samples s0, s0+1, ...
                     auto load_block = [&](uint8_t* dst, int q, int s0) {
-                        if (p.conv_layer == 1) {   // conv2: input seen as [sample][y/2][y%2][x/2][64]
+                        if (p.conv_layer == 0) {
+                            // conv1: frames seen as [sample][y/4][y%4][ox][8 px x 4 ch] with windows that overlap
+                            // by half (ox advances 4 px); q = kernel row ky, s0 = sample*4 + quarter of the sample
+                            // (5 of the 20 output rows, 100 patches)
+                            tma_load_5d(dst, &tmA, &full_bar[s], 0, 0, q & 3, (q >> 2) + 5 * (s0 & 3),
+                                        group * p.a_samples + (s0 >> 2));
+                        } else if (p.conv_layer == 1) {   // conv2: input seen as [sample][y/2][y%2][x/2][64]
                             const int ky = q >> 1, h = q & 1;
                             tma_load_5d(dst, &tmA, &full_bar[s], 0, h, ky & 1, ky >> 1, group * p.a_samples + s0);
                         } else {                   // conv3: input [sample][y][x][64]
@@ -276,10 +285,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         if (lane == 0) tma_load_4d(a, &tmA, &full_bar[s], 0, -ox_shift, -oy_shift, group * p.a_samples + sample);
                         else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], wcol, 0, group);
                     } else if (conv == CONV_FWD) {
-                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes + (uint32_t)(BN * BK * 2));
+                        const int kelems = sw64 ? 32 : BK;   // K elements per step
+                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes + (uint32_t)(BN * kelems * 2));
                         __syncwarp();
                         if (lane == 0) load_block(a, t.kt_begin + k, (t.m0 / p.tile_rows) * p.conv_nb);
-                        else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], k0, t.n0, group);
+                        else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], (t.kt_begin + k) * kelems, t.n0, group);
+                    } else if (sw64) {
+                        // conv1 weight gradient: M tile = 4 kernel rows x 32 elements (4 boxes), K step = the
+                        // 100 patches of one quarter sample; dY1 rows of the same patches from a [sample][400][32] map
+                        const int ks = t.kt_begin + k;
+                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes * 5u);
+                        __syncwarp();
+                        if (lane < 4) load_block(a + lane * p.kstep_rows * 64, (t.m0 / 128) * 4 + lane, ks);
+                        else if (lane == 4) tma_load_3d(b, &tmB, &full_bar[s], t.n0, (ks & 3) * 100, group * p.b_samples + (ks >> 2));
                     } else {
                         const int q0 = t.m0 / 64, s0 = (t.kt_begin + k) * p.conv_nb;
                         const int nq = (q0 + 1 < cQ) ? 2 : 1;
@@ -326,10 +344,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t b_addr = smem_u32(smB + s * stage_b);
                     if (conv == CONV_WGRAD) {
                         // a K step is kstep_rows patches (the padding rows are zero on both sides)
-                        const uint32_t atom = (uint32_t)p.kstep_rows * 128u;
+                        const uint32_t row_bytes = sw64 ? 64u : 128u;
+                        const uint32_t atom = (uint32_t)p.kstep_rows * row_bytes;
                         for (int kk = 0; kk < p.kstep_rows / 16; kk++) {
-                            const uint64_t ad = make_smem_desc(a_addr + kk * 2048, 1, atom);
-                            const uint64_t bd = make_smem_desc(b_addr + kk * 2048, 1, atom);
+                            const uint64_t ad = make_smem_desc(a_addr + kk * 16 * row_bytes, 1, atom, sw64);
+                            const uint64_t bd = make_smem_desc(b_addr + kk * 16 * row_bytes, 1, atom, sw64);
+                            umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
+                        }
+                    } else if (sw64) {
+                        // conv1 forward: 32 K elements per step = two UMMAs along a 64-byte row
+                        for (int kk = 0; kk < 2; kk++) {
+                            const uint64_t ad = make_smem_desc(a_addr + kk * 32, 0, 8192u, 1);
+                            const uint64_t bd = make_smem_desc(b_addr + kk * 32, 0, 8192u, 1);
                             umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
                         }
                     } else {
@@ -628,7 +654,7 @@ bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint
 }
 
 bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                        const uint64_t* strides_bytes, const uint32_t* box) {
+                        const uint64_t* strides_bytes, const uint32_t* box, int sw64) {
     if (!g_encode || rank < 3 || rank > 5) return false;
     if (reinterpret_cast<uintptr_t>(base) & 15) return false;
     cuuint64_t d[5], st[4];
@@ -636,8 +662,8 @@ bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint
     for (int i = 0; i < rank; i++) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; if (box[i] > 256) return false; }
     for (int i = 0; i + 1 < rank; i++) { st[i] = strides_bytes[i]; if (st[i] & 15) return false; }
     CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, sw64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -652,7 +678,7 @@ bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_e
 
 cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, cudaStream_t st) {
     if (args.block_n != 32 && args.block_n != 64 && args.block_n != 128) return cudaErrorInvalidValue;
-    if (B.mn_major && args.block_n < 64) return cudaErrorInvalidValue;
+    if (B.mn_major && args.block_n < 64 && !(args.conv_mode != CONV_NONE && args.conv_layer == 0)) return cudaErrorInvalidValue;
     if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
     GemmArgs a = args;
     if (a.conv_mode == CONV_NONE) {
@@ -661,25 +687,27 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
         a.stage_a_bytes = kStageA;
         a.stage_b_bytes = a.block_n * BK * 2;
     } else {
-        if (a.conv_layer != 1 && a.conv_layer != 2) return cudaErrorInvalidValue;
-        const int P = a.conv_layer == 1 ? 81 : 49;
+        if (a.conv_layer < 0 || a.conv_layer > 2) return cudaErrorInvalidValue;
+        if (a.conv_layer == 0 && (a.conv_mode == CONV_DGRAD || a.block_n != 32)) return cudaErrorInvalidValue;
+        const int P = a.conv_layer == 0 ? 100 : (a.conv_layer == 1 ? 81 : 49);
+        const int row_bytes = a.conv_layer == 0 ? 64 : 128;
         if (a.conv_nb < 1 || a.tile_rows < 1 || a.tile_rows > BM || a.k_steps < 1) return cudaErrorInvalidValue;
         if (a.conv_mode != CONV_DGRAD && a.conv_nb * P > 128) return cudaErrorInvalidValue;
         if (a.box_rows < 1 || a.box_rows > 128) return cudaErrorInvalidValue;
         if (a.conv_mode == CONV_FWD) {
             if (A.mn_major || B.mn_major || a.tile_rows != a.conv_nb * P || a.box_rows != a.tile_rows) return cudaErrorInvalidValue;
-            a.stage_a_bytes = kStageA;
-            a.stage_b_bytes = a.block_n * BK * 2;
+            a.stage_a_bytes = BM * row_bytes;
+            a.stage_b_bytes = a.block_n * row_bytes;
         } else if (a.conv_mode == CONV_DGRAD) {
             if (A.mn_major || !B.mn_major || a.block_n != 64 || a.tile_rows != a.box_rows) return cudaErrorInvalidValue;
             a.stage_a_bytes = kStageA;
             a.stage_b_bytes = 64 * BK * 2;
         } else {
-            if (!A.mn_major || !B.mn_major || a.block_n != 64 || a.kstep_rows % 16 || a.kstep_rows < a.conv_nb * P ||
-                a.kstep_rows > 128 || a.tile_rows != BM)
+            if (!A.mn_major || !B.mn_major || (a.block_n != 64 && a.conv_layer != 0) || a.kstep_rows % 16 ||
+                a.kstep_rows < a.conv_nb * P || a.kstep_rows > 128 || a.tile_rows != BM)
                 return cudaErrorInvalidValue;
-            a.stage_a_bytes = 2 * a.kstep_rows * 128;
-            a.stage_b_bytes = a.kstep_rows * 128;
+            a.stage_a_bytes = (a.conv_layer == 0 ? 4 : 2) * a.kstep_rows * row_bytes;
+            a.stage_b_bytes = a.kstep_rows * row_bytes;
         }
     }
     const int mt = (a.M + a.tile_rows - 1) / a.tile_rows, nt = (a.N + a.block_n - 1) / a.block_n;

@@ -76,7 +76,8 @@ struct GemmArgs {
     // Implicit convolution operands (conv_mode != CONV_NONE): the patch matrix is never stored; TMA
     // boxes over the NHWC activations deliver, for one kernel offset, the [patch][channel] block.
     int conv_mode;
-    int conv_layer;        // 1: conv2 (4x4 stride 2 on 20x20x32), 2: conv3 (3x3 stride 1 on 9x9x64)
+    int conv_layer;        // 0: conv1 (8x8 stride 4 on bf16 copies of the 84x84x4 frames), 1: conv2 (4x4 stride 2
+                           // on 20x20x32), 2: conv3 (3x3 stride 1 on 9x9x64)
     int conv_nb;           // samples per M tile (forward, data gradient) or per K step (weight gradient)
     int a_samples;         // samples per group in the activation tensor behind A
     int b_samples;         // weight gradient: samples per group in the dY tensor behind B
@@ -98,9 +99,10 @@ bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t
 // rows x cols fp32 matrix, unswizzled box_rows x box_cols tile (gemm_init() first).
 bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
                          uint32_t box_cols, uint32_t box_rows);
-// General bf16 tensor map of rank 3..5, 128-byte swizzle (dims/strides innermost first).
+// General bf16 tensor map of rank 3..5, 128-byte swizzle, or 64-byte swizzle for 64-byte rows
+// (dims/strides innermost first).  Dimensions may overlap (a stride smaller than the extent below it).
 bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                        const uint64_t* strides_bytes, const uint32_t* box);
+                        const uint64_t* strides_bytes, const uint32_t* box, int sw64 = 0);
 // Builds the descriptor for an operand of a GEMM with the given tile height
 // (128 for A, block_n for B).
 bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
@@ -198,6 +200,9 @@ struct DenseBwdArgs {
 cudaError_t launch_dense_bwd(const DenseBwdArgs& a, int groups, cudaStream_t st);
 
 // ---------------------------------------------------------------- conv lowering
+// uint8 frames -> bf16 (exact), per group [samples][84*84*4]
+cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out_group_stride, int samples, int groups,
+                               cudaStream_t st);
 cudaError_t launch_im2col_u8(const PtrBatch& obs, __nv_bfloat16* cols, long cols_group_stride, int samples,
                              int groups, cudaStream_t st);
 cudaError_t launch_im2col_bf16(const __nv_bfloat16* act, long act_group_stride, __nv_bfloat16* cols,

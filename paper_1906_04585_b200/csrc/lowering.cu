@@ -61,6 +61,37 @@ cudaError_t launch_im2col_u8(const PtrBatch& obs, __nv_bfloat16* cols, long cols
     return cudaGetLastError();
 }
 
+// uint8 frames -> bf16 frames (0..255 are exact in bf16; the 1/255 scale is applied after the
+// contraction).  16 bytes in, 32 bytes out per thread and step.
+__global__ void __launch_bounds__(256) cast_frames_kernel(PtrBatch obs, __nv_bfloat16* __restrict__ out, long out_group_stride,
+                                                          long n16) {
+    const int g = blockIdx.y;
+    const uint4* src = reinterpret_cast<const uint4*>(obs.p[g]);
+    uint4* dst = reinterpret_cast<uint4*>(out + (long)g * out_group_stride);
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n16; i += (long)gridDim.x * blockDim.x) {
+        const uint4 v = __ldg(src + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+            __nv_bfloat162 p0 = __floats2bfloat162_rn((float)(w[q] & 255u), (float)((w[q] >> 8) & 255u));
+            __nv_bfloat162 p1 = __floats2bfloat162_rn((float)((w[q] >> 16) & 255u), (float)(w[q] >> 24));
+            o[2 * q] = *reinterpret_cast<uint32_t*>(&p0);
+            o[2 * q + 1] = *reinterpret_cast<uint32_t*>(&p1);
+        }
+        dst[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out_group_stride, int samples, int groups,
+                               cudaStream_t st) {
+    const long n16 = (long)samples * (84 * 84 * 4 / 16);
+    int bx = (int)((n16 + 255) / 256);
+    if (bx > 148 * 8) bx = 148 * 8;
+    cast_frames_kernel<<<dim3(bx, groups), 256, 0, st>>>(obs, out, out_group_stride, n16);
+    return cudaGetLastError();
+}
+
 // bf16 NHWC activations -> bf16 patch rows, 16 bytes per thread per step.
 __global__ void __launch_bounds__(256) im2col_bf16_kernel(const __nv_bfloat16* __restrict__ act, long act_group_stride,
                                                           __nv_bfloat16* __restrict__ cols, long cols_group_stride,
