@@ -261,7 +261,8 @@ int build_plans(gala_ctx* c) {
         }
         f.args.conv_mode = CONV_FWD; f.args.conv_layer = l; f.args.conv_nb = nb; f.args.a_samples = (int)B;
         if (l == 0) {
-            f.args.conv_nb = 1; f.args.tile_rows = 100; f.args.box_rows = 100; f.args.k_steps = 8;
+            f.args.conv_nb = 1; f.args.tile_rows = 100; f.args.box_rows = 100;
+            f.args.kpack = 4; f.args.k_steps = 8 / f.args.kpack;   // 4 kernel rows per K step
             const uint64_t wd[3] = {(uint64_t)KK, (uint64_t)CO, (uint64_t)n};
             const uint64_t ws[2] = {(uint64_t)KK * 2, (uint64_t)dp * 2};
             const uint32_t wb[3] = {32, 32, 1};

@@ -285,11 +285,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         if (lane == 0) tma_load_4d(a, &tmA, &full_bar[s], 0, -ox_shift, -oy_shift, group * p.a_samples + sample);
                         else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], wcol, 0, group);
                     } else if (conv == CONV_FWD) {
-                        const int kelems = sw64 ? 32 : BK;   // K elements per step
-                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes + (uint32_t)(BN * kelems * 2));
+                        // kpack kernel-offset blocks per K step: lanes 0..kpack-1 fetch the A boxes, the next
+                        // kpack lanes the matching 64- (or 32-) wide column blocks of the weights
+                        const int kelems = sw64 ? 32 : BK;   // K elements per block
+                        const int kp = p.kpack;
+                        const uint32_t a_sub = (uint32_t)(BM * kelems * 2), b_sub = (uint32_t)(BN * kelems * 2);
+                        if (lane == 0) mbar_expect_tx(&full_bar[s], (uint32_t)kp * (box_bytes + b_sub));
                         __syncwarp();
-                        if (lane == 0) load_block(a, t.kt_begin + k, (t.m0 / p.tile_rows) * p.conv_nb);
-                        else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], (t.kt_begin + k) * kelems, t.n0, group);
+                        const int q = (t.kt_begin + k) * kp + (lane < kp ? lane : lane - kp);
+                        if (lane < kp) load_block(a + lane * a_sub, q, (t.m0 / p.tile_rows) * p.conv_nb);
+                        else if (lane < 2 * kp) tma_load_3d(b + (lane - kp) * b_sub, &tmB, &full_bar[s], q * kelems, t.n0, group);
                     } else if (sw64) {
                         // conv1 weight gradient: M tile = 4 kernel rows x 32 elements (4 boxes), K step = the
                         // 100 patches of one quarter sample; dY1 rows of the same patches from a [sample][400][32] map
@@ -351,13 +356,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                             const uint64_t bd = make_smem_desc(b_addr + kk * 16 * row_bytes, 1, atom, sw64);
                             umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
                         }
-                    } else if (sw64) {
-                        // conv1 forward: 32 K elements per step = two UMMAs along a 64-byte row
-                        for (int kk = 0; kk < 2; kk++) {
-                            const uint64_t ad = make_smem_desc(a_addr + kk * 32, 0, 8192u, 1);
-                            const uint64_t bd = make_smem_desc(b_addr + kk * 32, 0, 8192u, 1);
-                            umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
-                        }
+                    } else if (conv == CONV_FWD) {
+                        // kpack blocks per step, each a [128][32 or 64] A image and a [BN][32 or 64] B image
+                        const int kelems = sw64 ? 32 : BK;
+                        const uint32_t a_sub = (uint32_t)(BM * kelems * 2), b_sub = (uint32_t)(BN * kelems * 2);
+                        for (int j = 0; j < p.kpack; j++)
+                            for (int kk = 0; kk < kelems / 16; kk++) {
+                                const uint64_t ad = make_smem_desc(a_addr + j * a_sub + kk * 32, 0, 8192u, sw64);
+                                const uint64_t bd = make_smem_desc(b_addr + j * b_sub + kk * 32, 0, 8192u, sw64);
+                                umma_bf16(tmem_acc, ad, bd, idesc, (k | j | kk) != 0 ? 1u : 0u);
+                            }
                     } else {
 #pragma unroll
                         for (int kk = 0; kk < BK / 16; kk++) {
@@ -696,8 +704,10 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
         if (a.box_rows < 1 || a.box_rows > 128) return cudaErrorInvalidValue;
         if (a.conv_mode == CONV_FWD) {
             if (A.mn_major || B.mn_major || a.tile_rows != a.conv_nb * P || a.box_rows != a.tile_rows) return cudaErrorInvalidValue;
-            a.stage_a_bytes = BM * row_bytes;
-            a.stage_b_bytes = a.block_n * row_bytes;
+            if (a.kpack < 1) a.kpack = 1;
+            if (a.kpack > 8) return cudaErrorInvalidValue;
+            a.stage_a_bytes = a.kpack * BM * row_bytes;
+            a.stage_b_bytes = a.kpack * a.block_n * row_bytes;
         } else if (a.conv_mode == CONV_DGRAD) {
             if (A.mn_major || !B.mn_major || a.block_n != 64 || a.tile_rows != a.box_rows) return cudaErrorInvalidValue;
             a.stage_a_bytes = kStageA;

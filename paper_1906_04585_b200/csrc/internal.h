@@ -83,6 +83,7 @@ struct GemmArgs {
     int b_samples;         // weight gradient: samples per group in the dY tensor behind B
     int kstep_rows;        // weight gradient: rows of a K step in shared memory (multiple of 16)
     int box_rows;          // rows of one A box (patches or pixels it delivers)
+    int kpack;             // forward: kernel-offset blocks (A box + B box each) per K step (default 1)
     int stage_a_bytes, stage_b_bytes;   // set by launch_gemm
 };
 //   CONV_FWD  : D[patch][co]  = sum_k patches[patch][k] W[co][k]      A from boxes, B = weights (K-major)
