@@ -172,19 +172,25 @@ cudaError_t launch_dense_fwd(const DenseArgs& a, int groups, cudaStream_t st) {
 }
 
 // Heads: logits[r][k] = h[r] . pi.W[k] + pi.b[k], value[r] = h[r] . v.W + v.b.
-// One warp per row; the dot products are split over lanes and combined by a butterfly.
+// The (A+1) x H head weights are staged in shared memory once per block (they would otherwise be
+// re-read from L2 with the full latency for every output); one warp per row, the dot products
+// are split over lanes and combined by a butterfly.
 __global__ void __launch_bounds__(256) heads_fwd_kernel(HeadsArgs a) {
-    extern __shared__ float hs[];  // [warps][H]
+    extern __shared__ float hsm[];  // [A+1][H] weights, then [warps][H] rows
     const int g = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const float* P = a.params + (long)g * a.p_stride;
     const char* hbase = reinterpret_cast<const char*>(a.h) + (long)g * a.h_stride * (a.h_bf16 ? 2 : 4);
-    float* hrow = hs + warp * a.H;
+    float* wsm = hsm;
+    float* hrow = hsm + (a.A + 1) * a.H + warp * a.H;
+    for (int i = threadIdx.x; i < a.A * a.H; i += blockDim.x) wsm[i] = P[a.piw + i];
+    for (int i = threadIdx.x; i < a.H; i += blockDim.x) wsm[a.A * a.H + i] = P[a.vw + i];
+    __syncthreads();
     for (int r = blockIdx.x * nwarps + warp; r < a.rows; r += gridDim.x * nwarps) {
         for (int i = lane; i < a.H; i += 32) hrow[i] = ld_in(hbase, (long)r * a.H + i, a.h_bf16);
         __syncwarp();
         for (int k = 0; k <= a.A; k++) {
-            const float* w = (k < a.A) ? P + a.piw + (long)k * a.H : P + a.vw;
+            const float* w = wsm + k * a.H;
             float acc = 0.0f;
             for (int i = lane; i < a.H; i += 32) acc = fmaf(w[i], hrow[i], acc);
             for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
@@ -197,10 +203,15 @@ __global__ void __launch_bounds__(256) heads_fwd_kernel(HeadsArgs a) {
     }
 }
 cudaError_t launch_heads_fwd(const HeadsArgs& a, int groups, cudaStream_t st) {
-    int bx = (a.rows + 7) / 8;
-    if (bx > 128) bx = 128;
-    dim3 grid(bx, groups);
-    heads_fwd_kernel<<<grid, 256, 8 * a.H * sizeof(float), st>>>(a);
+    int bx = (a.rows + 7) / 8;     // one row per warp while that still gives few enough blocks
+    if (bx * groups > 592) bx = (592 + groups - 1) / groups;
+    if (bx < 1) bx = 1;
+    const size_t smem = (size_t)((a.A + 1) + 8) * a.H * sizeof(float);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(heads_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    heads_fwd_kernel<<<dim3(bx, groups), 256, smem, st>>>(a);
     return cudaGetLastError();
 }
 

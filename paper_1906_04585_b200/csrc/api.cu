@@ -40,7 +40,7 @@ struct Plan {  // one tensor-core product with its descriptors
 
 // Kernel classes for launch counting and optional per-class device timing.
 enum Tag : int {
-    T_IM2COL_U8 = 0, T_IM2COL_BF16, T_HEADS_FWD, T_LOSS, T_HEADS_BWD, T_COLSUM, T_SPLITK, T_COL2IM, T_GRAD_NORM,
+    T_CAST_FRAMES = 0, T_HEADS_FWD, T_LOSS, T_HEADS_BWD, T_COLSUM, T_SPLITK, T_GRAD_NORM,
     T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST,
     T_GEMM_CONV_FWD,          // +layer (3)
     T_GEMM_FC_FWD = T_GEMM_CONV_FWD + 3, T_GEMM_FC_WGRAD, T_GEMM_FC_DGRAD,
@@ -49,7 +49,7 @@ enum Tag : int {
     T_COUNT = T_GEMM_CONV_DGRAD + 3
 };
 const char* const kTagNames[T_COUNT] = {
-    "cast_frames", "im2col_bf16", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "col2im", "grad_norm",
+    "cast_frames", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "grad_norm",
     "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16",
     "gemm_conv1_fwd", "gemm_conv2_fwd", "gemm_conv3_fwd", "gemm_fc_fwd", "gemm_fc_wgrad", "gemm_fc_dgrad",
     "gemm_conv1_wgrad", "gemm_conv2_wgrad", "gemm_conv3_wgrad", "gemm_conv1_dgrad", "gemm_conv2_dgrad",
@@ -409,13 +409,37 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
     const long dp = c->d_pad, B = c->B;
     if (c->conv) {
         const int P[3] = {400, 81, 49};
-        LAUNCH(T_IM2COL_U8, st, launch_cast_frames(obs, c->frames + (long)agent0 * B * kFramePix, B * kFramePix, rows, groups, st));
+        LAUNCH(T_CAST_FRAMES, st, launch_cast_frames(obs, c->frames + (long)agent0 * B * kFramePix, B * kFramePix, rows, groups, st));
         for (int l = 0; l < 3; l++) {
             int r = run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st);
             if (r != GALA_OK) return r;
         }
-        int r = run_plan(c, c->fc_fwd, agent0, groups, rows, st);
-        if (r != GALA_OK) return r;
+        // hidden layer: with few rows there are only a handful of output tiles, each streaming 0.8 MB of
+        // weights through one SM; split the 3136-long reduction over more CTAs then
+        int r;
+        {
+            const Plan& p = c->fc_fwd;
+            const int tiles = ((rows + 127) / 128) * (kHidden / 128);
+            int split = 296 / (groups * tiles);
+            if (split > 7) split = 7;
+            while (split > 1 && (long)split * rows * kHidden > c->splitk_group_stride) split--;
+            if (split <= 1) {
+                r = run_plan(c, p, agent0, groups, rows, st);
+                if (r != GALA_OK) return r;
+            } else {
+                GemmArgs a = p.args;
+                const long count = (long)rows * kHidden;
+                a.group0 = agent0; a.groups = groups; a.M = rows; a.split_k = split;
+                a.flags = 0; a.bias = nullptr;
+                a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+                a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
+                LAUNCH(p.tag, st, launch_gemm(p.A, p.B, a, st));
+                LAUNCH(T_SPLITK, st, launch_splitk_reduce_act(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
+                                                              c->hid + (long)agent0 * B * kHidden, c->x + c->cl.fcb, dp, agent0,
+                                                              count, kHidden, split, count, groups, c->splitk_group_stride,
+                                                              B * kHidden, st));
+            }
+        }
         HeadsArgs h{};
         h.rows = rows; h.H = kHidden; h.A = c->A;
         h.h = c->hid + (long)agent0 * B * kHidden; h.h_stride = B * kHidden; h.h_bf16 = 1;

@@ -605,6 +605,43 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
         og[i] = acc;
     }
 }
+// Same fixed-order reduction followed by the forward epilogue of a dense layer: + bias[n], ReLU, bf16.
+__global__ void __launch_bounds__(256) splitk_reduce_act_kernel(const float* __restrict__ partials,
+                                                                __nv_bfloat16* __restrict__ out, const float* __restrict__ bias,
+                                                                long bias_group_stride, int group0, long count, int N,
+                                                                int split_k, long split_stride, long partial_group_stride,
+                                                                long out_group_stride) {
+    const int g = blockIdx.y;
+    const float4* pg = reinterpret_cast<const float4*>(partials + (long)g * partial_group_stride);
+    const float* bg = bias + (long)(group0 + g) * bias_group_stride;
+    uint2* og = reinterpret_cast<uint2*>(out + (long)g * out_group_stride);
+    const long n4 = count / 4, s4 = split_stride / 4;
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x) {
+        float4 acc = pg[i];
+        for (int s = 1; s < split_k; s++) {   // fixed order
+            const float4 v = pg[(long)s * s4 + i];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        const int n = (int)((i * 4) % N);
+        acc.x = fmaxf(acc.x + __ldg(bg + n), 0.f); acc.y = fmaxf(acc.y + __ldg(bg + n + 1), 0.f);
+        acc.z = fmaxf(acc.z + __ldg(bg + n + 2), 0.f); acc.w = fmaxf(acc.w + __ldg(bg + n + 3), 0.f);
+        uint2 u;
+        u.x = pack2(acc.x, acc.y); u.y = pack2(acc.z, acc.w);
+        og[i] = u;
+    }
+}
+cudaError_t launch_splitk_reduce_act(const float* partials, __nv_bfloat16* out, const float* bias, long bias_group_stride,
+                                     int group0, long count, int N, int split_k, long split_stride, int groups,
+                                     long partial_group_stride, long out_group_stride, cudaStream_t st) {
+    if ((count & 3) || (N & 3) || (split_stride & 3) || (partial_group_stride & 3) || (out_group_stride & 3))
+        return cudaErrorInvalidValue;
+    int bx = (int)((count / 4 + 255) / 256);
+    if (bx > 148 * 4) bx = 148 * 4;
+    splitk_reduce_act_kernel<<<dim3(bx, groups), 256, 0, st>>>(partials, out, bias, bias_group_stride, group0, count, N,
+                                                               split_k, split_stride, partial_group_stride, out_group_stride);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, int split_k, long split_stride,
                                  int groups, long partial_group_stride, long out_group_stride, cudaStream_t st) {
     int bx = (int)((count + 255) / 256);

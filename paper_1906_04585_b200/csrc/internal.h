@@ -109,6 +109,9 @@ bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint
 bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
                   uint64_t groups, uint64_t ld_elems, uint64_t group_stride_elems, int tile_mn);
 cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, cudaStream_t st);
+cudaError_t launch_splitk_reduce_act(const float* partials, __nv_bfloat16* out, const float* bias, long bias_group_stride,
+                                     int group0, long count, int N, int split_k, long split_stride, int groups,
+                                     long partial_group_stride, long out_group_stride, cudaStream_t st);
 cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, int split_k,
                                  long split_stride, int groups, long partial_group_stride,
                                  long out_group_stride, cudaStream_t st);
@@ -204,14 +207,6 @@ cudaError_t launch_dense_bwd(const DenseBwdArgs& a, int groups, cudaStream_t st)
 // uint8 frames -> bf16 (exact), per group [samples][84*84*4]
 cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out_group_stride, int samples, int groups,
                                cudaStream_t st);
-cudaError_t launch_im2col_u8(const PtrBatch& obs, __nv_bfloat16* cols, long cols_group_stride, int samples,
-                             int groups, cudaStream_t st);
-cudaError_t launch_im2col_bf16(const __nv_bfloat16* act, long act_group_stride, __nv_bfloat16* cols,
-                               long cols_group_stride, int layer, int samples, int groups, cudaStream_t st);
-// dX = mask(act_in > 0) * scatter-sum of dcols; layer = 1 or 2 (conv2, conv3)
-cudaError_t launch_col2im(const float* dcols, long dcols_group_stride, const __nv_bfloat16* act_in,
-                          long act_group_stride, __nv_bfloat16* dx, long dx_group_stride, int layer,
-                          int samples, int groups, cudaStream_t st);
 // Column sums (bias gradients) of up to kColsumJobs bf16 tensors in one launch:
 // out_base[g*out_group_stride + out_off + c] = sum_r dy[g][r][c], fixed summation order.
 // partial: [groups][kColsumJobs][kColsumChunks][512] doubles, ticket: [groups][kColsumJobs] (zeroed once).
