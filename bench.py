@@ -307,7 +307,7 @@ def run_ours(args):
         achieved = amount / (per_step_ms * 1e-3) / 1e12 if per_step_ms > 0 else 0.0
         peak, unit = pk["tensor"], "TFLOP/s"
     roofline = dict(kernel=dominant, bound=bound, achieved=achieved, peak=peak, unit=unit, frac=achieved / peak,
-                    peak_source=pk["source"], traffic=NCU_TRAFFIC_BYTES.get(dominant),
+                    peak_source=pk["source"], traffic=NCU_TRAFFIC_BYTES.get(dominant) if w.index == 1 else None,
                     ms_per_step=per_step_ms, launches_timed=int(dom_timed),
                     share_of_step=per_step_ms / (total_ms / args.steps) if total_ms > 0 else None)
 
