@@ -73,6 +73,10 @@ struct gala_ctx {
     std::vector<Agent> agents;
     cudaStream_t main_stream = nullptr;
     cudaEvent_t main_event = nullptr;
+    // second stream of the synchronous mode: weight gradients and bias gradients run beside the chain
+    // of data gradients they do not depend on
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     long long sync_round = 0;
     long long launches = 0;
     long long tag_launches[T_COUNT] = {};
@@ -476,7 +480,8 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
 
 // Learner step for agents [agent0, agent0+groups): forward, returns/advantages/objective,
 // backward into the flat gradient, global norm and clip coefficient.
-int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cudaStream_t st) {
+int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cudaStream_t st,
+                cudaStream_t side = nullptr) {
     const long dp = c->d_pad, B = c->B, S = c->S;
     const int A = c->A;
     PtrBatch obs{}, acts{}, rews{}, dns{};
@@ -509,22 +514,39 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hb.dpre = c->dh + (long)agent0 * S * kHidden; hb.dpre_stride = S * kHidden; hb.dpre_bf16 = 1;
         LAUNCH(T_HEADS_BWD, st, launch_heads_bwd(hb, groups, st));
         c->launches++; c->tag_launches[T_HEADS_BWD]++;  // two kernels
-        if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, st)) != GALA_OK) return r;
+        // The data gradients form a chain (hidden -> conv3 -> conv2); every weight gradient only needs the dY
+        // of its own layer.  With a side stream the weight gradients (and the bias gradients) run beside
+        // the chain; `ws` is where they go, `fork` makes it wait for what `st` has enqueued so far.
+        cudaStream_t ws = side ? side : st;
+        auto fork = [&]() -> int {
+            if (!side) return GALA_OK;
+            CK(cudaEventRecord(c->ev_fork, st));
+            CK(cudaStreamWaitEvent(side, c->ev_fork, 0));
+            return GALA_OK;
+        };
+        if ((r = fork()) != GALA_OK) return r;
+        if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, ws)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
         for (int l = 2; l >= 0; l--) {
-            const int CO = kConvCout[l];
-            if ((r = run_wgrad(c, c->wgrad[l], agent0, groups, st)) != GALA_OK) return r;
+            if ((r = fork()) != GALA_OK) return r;
+            if ((r = run_wgrad(c, c->wgrad[l], agent0, groups, ws)) != GALA_OK) return r;
             if (l > 0 && (r = run_plan(c, c->dgrad[l], agent0, groups, 0, st)) != GALA_OK) return r;
         }
+        // the bias gradients need every dY: they follow conv1's weight gradient on the side stream
         {   // all four bias gradients (column sums of dh, dY3, dY2, dY1) in one launch
             ColsumJobs jobs{};
             jobs.j[0] = {c->dh + (long)agent0 * S * kHidden, S * kHidden, S, kHidden, c->cl.fcb};
             for (int l = 0; l < 3; l++)
                 jobs.j[1 + l] = {c->dy[l] + (long)agent0 * S * P[l] * kConvCout[l], S * P[l] * kConvCout[l], S * P[l],
                                  kConvCout[l], c->cl.b[l]};
-            LAUNCH(T_COLSUM, st, launch_colsum(jobs, 4, c->g + (long)agent0 * dp, dp,
+            if ((r = fork()) != GALA_OK) return r;
+            LAUNCH(T_COLSUM, ws, launch_colsum(jobs, 4, c->g + (long)agent0 * dp, dp,
                                                c->colsum_partial + (long)agent0 * kColsumJobs * kColsumChunks * 512,
-                                               c->colsum_ticket + (long)agent0 * kColsumJobs, groups, st));
+                                               c->colsum_ticket + (long)agent0 * kColsumJobs, groups, ws));
+        }
+        if (side) {   // join: the gradient is complete when both streams are done
+            CK(cudaEventRecord(c->ev_join, side));
+            CK(cudaStreamWaitEvent(st, c->ev_join, 0));
         }
     } else {
         const int H = c->H;
@@ -709,6 +731,9 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
 
     CK(cudaStreamCreateWithFlags(&c->main_stream, cudaStreamNonBlocking));
     CK(cudaEventCreateWithFlags(&c->main_event, cudaEventDisableTiming));
+    CK(cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking));
+    CK(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
     c->agents.resize(n);
     for (int i = 0; i < n; i++) {
         Agent& a = c->agents[i];
@@ -802,6 +827,9 @@ int gala_destroy(gala_ctx* c) {
         if (a.sweep_done) cudaEventDestroy(a.sweep_done);
         if (a.fence) cudaEventDestroy(a.fence);
     }
+    if (c->side_stream) cudaStreamDestroy(c->side_stream);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->main_stream) cudaStreamDestroy(c->main_stream);
     if (c->main_event) cudaEventDestroy(c->main_event);
     for (auto& t : c->timed) { cudaEventDestroy(t.beg); cudaEventDestroy(t.end); }
@@ -871,7 +899,7 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
     if (ros) {
         for (int a0 = 0; a0 < n; a0 += kBatch) {
             const int cnt = n - a0 < kBatch ? n - a0 : kBatch;
-            int r = learn_range(c, a0, cnt, ros + a0, st);
+            int r = learn_range(c, a0, cnt, ros + a0, st, c->side_stream);
             if (r != GALA_OK) return r;
         }
     }
