@@ -274,6 +274,7 @@ int build_plans(gala_ctx* c) {
             f.B.mn_major = 0;
         } else {
             f.args.tile_rows = nb * P[l]; f.args.box_rows = nb * P[l]; f.args.k_steps = KK / 64;
+            f.args.kpack = 2;   // two kernel offsets per K step
             ok &= make_operand(&f.B, c->shadow + c->cl.w[l], 0, CO, KK, n, KK, dp, bn);
         }
         f.args.M = (int)(B * P[l]); f.args.N = CO; f.args.K = KK; f.args.block_n = bn;
@@ -337,6 +338,7 @@ int build_plans(gala_ctx* c) {
             dg.args.conv_mode = CONV_DGRAD; dg.args.conv_layer = l; dg.args.conv_nb = 1; dg.args.a_samples = (int)S;
             dg.args.tile_rows = l == 2 ? 81 : 100; dg.args.box_rows = dg.args.tile_rows;
             dg.args.k_steps = l == 2 ? 9 : 4;
+            dg.args.kpack = 2;  // two kernel offsets per K step
             dg.args.flags = EPI_OUT_BF16 | EPI_MASK | (l == 1 ? EPI_ROWMAP_S2 : 0);
             dg.args.mask = c->act[l - 1]; dg.args.mask_group_stride = B * in_pix * cin;
             dg.args.out = c->dy[l - 1]; dg.args.out_group_stride = S * in_pix * cin; dg.args.ldc = cin;

@@ -265,36 +265,44 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                             tma_load_4d(dst, &tmA, &full_bar[s], 0, kx, ky, group * p.a_samples + s0);
                         }
                     };
-                    if (conv == CONV_DGRAD) {
-                        // K step = one kernel offset; the dY box is shifted by it, the weights' [co][ci]
-                        // block of that offset is a 64-wide column block of W[co][(ky, kx, ci)]
-                        int sample, oy_shift, ox_shift, wcol;
-                        const int j = t.kt_begin + k;
-                        if (p.conv_layer == 2) {          // conv3, stride 1: pixel (y, x) <- dY[y - ky][x - kx]
-                            sample = t.m0 / 81;
-                            oy_shift = j / 3; ox_shift = j - oy_shift * 3;
-                            wcol = j * 64;
-                        } else {                          // conv2, stride 2: class (py, px), pixel (2a+py, 2c+px)
-                            sample = t.m0 / 400;          //   <- dY[a - dy][c - dx] with ky = py + 2dy, kx = px + 2dx
-                            const int cls = (t.m0 / 100) & 3;
-                            oy_shift = j >> 1; ox_shift = j & 1;
-                            wcol = (((cls >> 1) + 2 * oy_shift) * 4 + (cls & 1) + 2 * ox_shift) * 32;
-                        }
-                        if (lane == 0) mbar_expect_tx(&full_bar[s], box_bytes + 8192u);
-                        __syncwarp();
-                        if (lane == 0) tma_load_4d(a, &tmA, &full_bar[s], 0, -ox_shift, -oy_shift, group * p.a_samples + sample);
-                        else if (lane == 1) tma_load_3d(b, &tmB, &full_bar[s], wcol, 0, group);
-                    } else if (conv == CONV_FWD) {
-                        // kpack kernel-offset blocks per K step: lanes 0..kpack-1 fetch the A boxes, the next
-                        // kpack lanes the matching 64- (or 32-) wide column blocks of the weights
+                    if (conv == CONV_DGRAD || conv == CONV_FWD) {
+                        // A K step covers up to kpack kernel offsets ("blocks").  Block j of the step gets an A
+                        // box at a + j * a_sub and a B box at b + j * b_sub; lanes 0..nq-1 fetch the A boxes,
+                        // lanes nq..2nq-1 the B boxes.  a_sub is the box size rounded up to 1 KiB, not a full
+                        // 128-row image: the rows an MMA reads past the box only feed output rows that the
+                        // epilogue drops.
                         const int kelems = sw64 ? 32 : BK;   // K elements per block
                         const int kp = p.kpack;
-                        const uint32_t a_sub = (uint32_t)(BM * kelems * 2), b_sub = (uint32_t)(BN * kelems * 2);
-                        if (lane == 0) mbar_expect_tx(&full_bar[s], (uint32_t)kp * (box_bytes + b_sub));
+                        const uint32_t a_sub = (uint32_t)p.a_sub_bytes, b_sub = (uint32_t)(BN * kelems * 2);
+                        const int q0 = (t.kt_begin + k) * kp;
+                        const int nq = min(kp, p.conv_q - q0);
+                        if (lane == 0) mbar_expect_tx(&full_bar[s], (uint32_t)nq * (box_bytes + b_sub));
                         __syncwarp();
-                        const int q = (t.kt_begin + k) * kp + (lane < kp ? lane : lane - kp);
-                        if (lane < kp) load_block(a + lane * a_sub, q, (t.m0 / p.tile_rows) * p.conv_nb);
-                        else if (lane < 2 * kp) tma_load_3d(b + (lane - kp) * b_sub, &tmB, &full_bar[s], q * kelems, t.n0, group);
+                        const int j = lane < nq ? lane : lane - nq;
+                        const int q = q0 + j;
+                        if (lane < 2 * nq) {
+                            if (conv == CONV_FWD) {
+                                if (lane < nq) load_block(a + j * a_sub, q, (t.m0 / p.tile_rows) * p.conv_nb);
+                                else tma_load_3d(b + j * b_sub, &tmB, &full_bar[s], q * kelems, t.n0, group);
+                            } else {
+                                // data gradient: block = kernel offset; the dY box is shifted by it, the weights'
+                                // [co][ci] block of that offset is a 64-wide column block of W[co][(ky, kx, ci)]
+                                int sample, oy_shift, ox_shift, wcol;
+                                if (p.conv_layer == 2) {      // conv3, stride 1: pixel (y, x) <- dY[y - ky][x - kx]
+                                    sample = t.m0 / 81;
+                                    oy_shift = q / 3; ox_shift = q - oy_shift * 3;
+                                    wcol = q * 64;
+                                } else {                      // conv2, stride 2: class (py, px), pixel (2a+py, 2c+px)
+                                    sample = t.m0 / 400;      //   <- dY[a - dy][c - dx] with ky = py + 2dy, kx = px + 2dx
+                                    const int cls = (t.m0 / 100) & 3;
+                                    oy_shift = q >> 1; ox_shift = q & 1;
+                                    wcol = (((cls >> 1) + 2 * oy_shift) * 4 + (cls & 1) + 2 * ox_shift) * 32;
+                                }
+                                if (lane < nq) tma_load_4d(a + j * a_sub, &tmA, &full_bar[s], 0, -ox_shift, -oy_shift,
+                                                           group * p.a_samples + sample);
+                                else tma_load_3d(b + j * b_sub, &tmB, &full_bar[s], wcol, 0, group);
+                            }
+                        }
                     } else if (sw64) {
                         // conv1 weight gradient: M tile = 4 kernel rows x 32 elements (4 boxes), K step = the
                         // 100 patches of one quarter sample; dY1 rows of the same patches from a [sample][400][32] map
@@ -356,14 +364,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                             const uint64_t bd = make_smem_desc(b_addr + kk * 16 * row_bytes, 1, atom, sw64);
                             umma_bf16(tmem_acc, ad, bd, idesc, (k | kk) != 0 ? 1u : 0u);
                         }
-                    } else if (conv == CONV_FWD) {
-                        // kpack blocks per step, each a [128][32 or 64] A image and a [BN][32 or 64] B image
+                    } else if (conv == CONV_FWD || conv == CONV_DGRAD) {
+                        // up to kpack blocks per step (see the producer); B is K-major (forward: weights as
+                        // stored) or MN-major (data gradient: the offset's [co][ci] block)
                         const int kelems = sw64 ? 32 : BK;
-                        const uint32_t a_sub = (uint32_t)(BM * kelems * 2), b_sub = (uint32_t)(BN * kelems * 2);
-                        for (int j = 0; j < p.kpack; j++)
+                        const uint32_t a_sub = (uint32_t)p.a_sub_bytes, b_sub = (uint32_t)(BN * kelems * 2);
+                        const int nq = min(p.kpack, p.conv_q - (t.kt_begin + k) * p.kpack);
+                        for (int j = 0; j < nq; j++)
                             for (int kk = 0; kk < kelems / 16; kk++) {
                                 const uint64_t ad = make_smem_desc(a_addr + j * a_sub + kk * 32, 0, 8192u, sw64);
-                                const uint64_t bd = make_smem_desc(b_addr + j * b_sub + kk * 32, 0, 8192u, sw64);
+                                const uint64_t bd = make_smem_desc(b_addr + j * b_sub + (b_mn ? kk * 2048 : kk * 32), b_mn, 8192u, sw64);
                                 umma_bf16(tmem_acc, ad, bd, idesc, (k | j | kk) != 0 ? 1u : 0u);
                             }
                     } else {
@@ -739,16 +749,21 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
         if (a.conv_nb < 1 || a.tile_rows < 1 || a.tile_rows > BM || a.k_steps < 1) return cudaErrorInvalidValue;
         if (a.conv_mode != CONV_DGRAD && a.conv_nb * P > 128) return cudaErrorInvalidValue;
         if (a.box_rows < 1 || a.box_rows > 128) return cudaErrorInvalidValue;
-        if (a.conv_mode == CONV_FWD) {
-            if (A.mn_major || B.mn_major || a.tile_rows != a.conv_nb * P || a.box_rows != a.tile_rows) return cudaErrorInvalidValue;
+        if (a.conv_mode == CONV_FWD || a.conv_mode == CONV_DGRAD) {
+            if (a.conv_mode == CONV_FWD) {
+                if (A.mn_major || B.mn_major || a.tile_rows != a.conv_nb * P || a.box_rows != a.tile_rows) return cudaErrorInvalidValue;
+                a.conv_q = a.conv_layer == 2 ? 9 : 8;    // 64-element (conv1: 32-element) blocks of a patch
+            } else {
+                if (A.mn_major || !B.mn_major || a.block_n != 64 || a.tile_rows != a.box_rows) return cudaErrorInvalidValue;
+                a.conv_q = a.conv_layer == 2 ? 9 : 4;    // kernel offsets that reach one pixel (class)
+            }
             if (a.kpack < 1) a.kpack = 1;
             if (a.kpack > 8) return cudaErrorInvalidValue;
-            a.stage_a_bytes = a.kpack * BM * row_bytes;
+            a.k_steps = (a.conv_q + a.kpack - 1) / a.kpack;
+            a.a_sub_bytes = (a.box_rows * row_bytes + 1023) / 1024 * 1024;
+            // the last block's MMA reads 128 rows from its start: keep that inside the stage
+            a.stage_a_bytes = (a.kpack - 1) * a.a_sub_bytes + BM * row_bytes;
             a.stage_b_bytes = a.kpack * a.block_n * row_bytes;
-        } else if (a.conv_mode == CONV_DGRAD) {
-            if (A.mn_major || !B.mn_major || a.block_n != 64 || a.tile_rows != a.box_rows) return cudaErrorInvalidValue;
-            a.stage_a_bytes = kStageA;
-            a.stage_b_bytes = 64 * BK * 2;
         } else {
             if (!A.mn_major || !B.mn_major || (a.block_n != 64 && a.conv_layer != 0) || a.kstep_rows % 16 ||
                 a.kstep_rows < a.conv_nb * P || a.kstep_rows > 128 || a.tile_rows != BM)

@@ -83,7 +83,9 @@ struct GemmArgs {
     int b_samples;         // weight gradient: samples per group in the dY tensor behind B
     int kstep_rows;        // weight gradient: rows of a K step in shared memory (multiple of 16)
     int box_rows;          // rows of one A box (patches or pixels it delivers)
-    int kpack;             // forward: kernel-offset blocks (A box + B box each) per K step (default 1)
+    int kpack;             // forward / data gradient: kernel-offset blocks (A box + B box each) per K step
+    int conv_q;            // number of such blocks in the whole reduction (set by launch_gemm)
+    int a_sub_bytes;       // distance between the A boxes of one K step (set by launch_gemm)
     int stage_a_bytes, stage_b_bytes;   // set by launch_gemm
 };
 //   CONV_FWD  : D[patch][co]  = sum_k patches[patch][k] W[co][k]      A from boxes, B = weights (K-major)
