@@ -364,6 +364,35 @@ def run_ours(args):
         line["async"] = dict(mixes=sum(x["mixes"] for x in st), skipped=sum(x["skipped"] for x in st),
                              staleness_mean=sum(x["staleness_sum"] for x in st) / max(1, sum(x["mixes"] for x in st)),
                              staleness_max=max(x["staleness_max"] for x in st), timing="host clock between syncs")
+    if rank == 0 and world == 1 and not async_mode:
+        # pieces beyond the core step: distance from consensus (one pass over all agents' parameters) and
+        # the synchronous A2C baseline (gradient all-reduce instead of gossip) on the same rollouts
+        t0 = time.perf_counter()
+        reps = 20
+        for _ in range(reps):
+            dist = B.gala_consensus_distance(L.ctx)
+        cons_ms = 1e3 * (time.perf_counter() - t0) / reps
+        L2 = LM.Learner(w.n_agents, GI.COMPLETE, 0, w.net_kind, w.n_actions, w.n_envs, w.n_steps,
+                        obs_dim=w.obs_dim, hidden=w.hidden)
+        ext2 = torch.cuda.ExternalStream(B.gala_get_stream(L2.ctx, -1))
+        for k in range(3):
+            L2.step_sync(sets[k % n_sets])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        L2.sync()
+        e0.record(ext2)
+        for k in range(20):
+            L2.step_sync(sets[k % n_sets])
+        e1.record(ext2)
+        L2.sync()
+        a2c_ms = e0.elapsed_time(e1) / 20
+        L2.close()
+        del ext2
+        line["extras"] = dict(consensus_distance=dist, consensus_call_ms=cons_ms,
+                              consensus_bytes=int(w.n_agents * L.d * 4),
+                              allreduce_a2c_ms_per_round=a2c_ms,
+                              allreduce_a2c_frames_per_s=w.frames_per_round / (a2c_ms * 1e-3),
+                              note="consensus_call_ms is a host-timed call (sync + one kernel + 8-byte read); "
+                                   "all-reduce rounds back to back without L2 flush")
     if rank == 0 and world == 1:
         line["sweep_microbench"] = sweep_microbench(torch, B, pk)
         if not args.no_cpu_baseline:

@@ -76,7 +76,9 @@ typedef enum { GALA_TOPO_RING = 0, GALA_TOPO_EXP = 1, GALA_TOPO_COMPLETE = 2 } g
  *         Fig. 5); in-peers of i are i-1 .. i-peers (mod n).
  *   EXP:  time-varying exponential graph, L = ceil(log2 n): the j-th in-peer
  *         of i at round k is i - 2^((peers*k + j) mod L) (mod n).
- *   COMPLETE: reserved (not implemented; gala_create returns GALA_EINVAL). */
+ *   COMPLETE: the synchronous A2C baseline of Sec. 5 (agents average their GRADIENTS before each
+ *         update, equivalent to one agent with all simulators): only gala_step_sync is defined;
+ *         `peers` is ignored; gala_gossip and gala_in_peers refuse. */
 typedef struct {
     int kind;  /* gala_topo_kind */
     int peers; /* in-peers per round: 1 or 2 */
@@ -94,7 +96,8 @@ typedef struct {
     float max_grad_norm; /* global-norm clip, 0.5; <= 0 switches it off */
     int n_envs;          /* E: simulators per agent */
     int n_steps;         /* T: rollout horizon (N in the paper) */
-    int staleness_tau;   /* reserved; must be < 0 (unbounded staleness) */
+    int staleness_tau;   /* tau of Sec. 3: < 0 unbounded; >= 0: a gossip step that finds no fresh message
+                            after more than tau local iterations without one waits for its in-peers */
     unsigned long long seed; /* initial parameters (library's own generator) */
     int identical_init;  /* 1: all agents start from the same parameters (assumed by Prop. 1) */
 } gala_hparams;
@@ -170,10 +173,18 @@ int gala_set_state(gala_ctx* ctx, int agent, const float* params, const float* s
  * max_grad_norm on the device. */
 int gala_set_grad(gala_ctx* ctx, int agent, const float* grad, float clip_coef);
 
+/* Distance of the agents' parameters from their mean, ||X - mean||_F over all agents and
+ * parameters (left-hand side of Propositions 1 and 2).  Waits for all work first. */
+int gala_consensus_distance(gala_ctx* ctx, double* out);
+/* Longest host wait (ms, default 1000) of a gossip step that is blocked by the staleness bound.
+ * When it runs out, or when an in-peer has published nothing newer, gala_gossip returns
+ * GALA_ETIMEOUT and has enqueued nothing; the pending gradient stays pending. */
+int gala_set_stale_timeout(gala_ctx* ctx, int timeout_ms);
 int gala_param_count(const gala_ctx* ctx, long long* d, long long* d_padded);
 /* out = {policy term, mean squared TD error, mean entropy, gradient norm} of the last learn. */
 int gala_losses(gala_ctx* ctx, int agent, float out[4]);
-/* out = {frames, rounds, mixes, skipped mixes, staleness sum, staleness max, published version, 0} */
+/* out = {frames, rounds, mixes, skipped mixes, staleness sum, staleness max, published version,
+ *        gossip steps that waited because of the staleness bound} */
 int gala_stats(gala_ctx* ctx, int agent, long long out[8]);
 /* Which snapshot versions the agent's last gala_gossip consumed: versions[j]
  * for in-peer peers[j]; *mixed = 1 if the average was taken. */

@@ -56,7 +56,7 @@ EXPORTS = (
     "gala_get_snapshot", "gala_set_stream", "gala_debug_read", "gala_launch_count",
     "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync", "gala_kernel_classes",
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
-    "gala_gemm_bf16_static", "gala_delay",
+    "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_set_stale_timeout",
 )
 
 _lib = None
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
             "gala_learn": (i, [vp, i, C.POINTER(gala_rollout)]),
             "gala_gossip": (i, [vp, i]),
             "gala_delay": (i, [vp, i, i]),
+            "gala_consensus_distance": (i, [vp, C.POINTER(C.c_double)]),
+            "gala_set_stale_timeout": (i, [vp, i]),
             "gala_step_sync": (i, [vp, C.POINTER(gala_rollout)]),
             "gala_sync_agent": (i, [vp, i, i]),
             "gala_sync_all": (i, [vp, i]),
@@ -168,6 +170,16 @@ def gala_delay(ctx, agent: int, usec: int):
     _check(ctx, lib().gala_delay(ctx, agent, usec))
 
 
+def gala_consensus_distance(ctx) -> float:
+    out = C.c_double()
+    _check(ctx, lib().gala_consensus_distance(ctx, C.byref(out)))
+    return out.value
+
+
+def gala_set_stale_timeout(ctx, timeout_ms: int):
+    _check(ctx, lib().gala_set_stale_timeout(ctx, timeout_ms))
+
+
 def gala_step_sync(ctx, rollouts: Optional[Sequence[gala_rollout]]):
     if rollouts is None:
         _check(ctx, lib().gala_step_sync(ctx, None))
@@ -221,7 +233,7 @@ def gala_stats(ctx, agent: int):
     out = (C.c_longlong * 8)()
     _check(ctx, lib().gala_stats(ctx, agent, out))
     return dict(frames=out[0], rounds=out[1], mixes=out[2], skipped=out[3], staleness_sum=out[4],
-                staleness_max=out[5], version=out[6])
+                staleness_max=out[5], version=out[6], stale_waits=out[7])
 
 
 def gala_last_mix(ctx, agent: int):

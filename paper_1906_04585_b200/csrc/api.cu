@@ -24,9 +24,10 @@ struct Agent {
     long long version = 0;                          // newest snapshot version enqueued (0: none)
     long long round = 0;                            // local iteration counter
     bool pending = false;                           // a gradient waits for its optimiser step
+    long long since_mix = 0;                        // local iterations since the last average with the in-peers
     std::vector<long long> consumed;                // newest version consumed from each agent
     std::vector<int> slot_readers[2];               // agents whose sweeps read snapshot slot s
-    long long frames = 0, mixes = 0, skipped = 0, stale_sum = 0, stale_max = 0;
+    long long frames = 0, mixes = 0, skipped = 0, stale_sum = 0, stale_max = 0, stale_waits = 0;
     int last_n = 0, last_mixed = 0;
     int last_peers[2] = {0, 0};
     long long last_versions[2] = {0, 0};
@@ -92,6 +93,9 @@ struct gala_ctx {
     double *norm_partial = nullptr, *colsum_partial = nullptr;
     unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr;
     int* error_word = nullptr;
+    double *cons_partial = nullptr, *cons_out = nullptr;
+    unsigned* cons_ticket = nullptr;
+    int stale_timeout_ms = 1000;   // longest host wait of a staleness-bounded gossip step
     float *logits = nullptr, *values = nullptr, *returns = nullptr, *adv = nullptr, *dlogits = nullptr,
           *dvalues = nullptr;
     // MLP workspaces
@@ -607,6 +611,35 @@ int sweep_agent(gala_ctx* c, int i, bool try_mix) {
         vers[j] = usable_version(c, peers[j]);
         if (vers[j] <= ag.consumed[peers[j]]) fresh = false;
     }
+    // Staleness bound (Sec. 3): if more than tau local iterations have passed since this agent last
+    // averaged, it waits for its in-peers' newest snapshots instead of going on alone.  The wait is a
+    // host wait with a deadline; only snapshots that are already enqueued can complete, so if an
+    // in-peer has nothing newer on its stream the call gives up at once.
+    if (try_mix && np > 0 && !fresh && c->hp.staleness_tau >= 0 && ag.since_mix > c->hp.staleness_tau) {
+        for (int j = 0; j < np; j++) {
+            Agent& pj = c->agents[peers[j]];
+            if (pj.version <= ag.consumed[peers[j]])
+                return fail(c, GALA_ETIMEOUT, "agent %d: %lld iterations without a message and in-peer %d has published "
+                            "nothing newer (tau = %d)", i, ag.since_mix, peers[j], c->hp.staleness_tau);
+        }
+        const auto t0 = std::chrono::steady_clock::now();
+        for (int j = 0; j < np; j++) {
+            Agent& pj = c->agents[peers[j]];
+            for (;;) {
+                cudaError_t e = cudaEventQuery(pj.pub_event[pj.version & 1]);
+                if (e == cudaSuccess) break;
+                if (e != cudaErrorNotReady) return fail(c, GALA_ECUDA, "cudaEventQuery: %s", cudaGetErrorString(e));
+                const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+                if (ms >= c->stale_timeout_ms)
+                    return fail(c, GALA_ETIMEOUT, "agent %d: in-peer %d's snapshot still not complete after %d ms", i,
+                                peers[j], c->stale_timeout_ms);
+                std::this_thread::sleep_for(std::chrono::microseconds(20));
+            }
+            vers[j] = pj.version;
+        }
+        fresh = true;
+        ag.stale_waits++;
+    }
     const long long w = ag.version + 1;
     const int slot = (int)(w & 1);
     // pairwise back-pressure: sweeps that still read the slot we are about to overwrite go first
@@ -626,8 +659,10 @@ int sweep_agent(gala_ctx* c, int i, bool try_mix) {
             ag.consumed[peers[j]] = vers[j];
         }
         ag.mixes++;
+        ag.since_mix = 0;
     } else if (np > 0) {
         ag.skipped++;
+        ag.since_mix++;
     }
     SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
     LAUNCH(T_SWEEP_AGENT, ag.stream, launch_sweep_agent(c->x + (long)i * dp, ag.pending ? c->g + (long)i * dp : nullptr, c->v + (long)i * dp,
@@ -682,11 +717,11 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
     *out = nullptr;
     if (!topo || !net || !hp) return GALA_EINVAL;
     if (n_agents < 1 || n_agents > 256) return GALA_EINVAL;
-    if (topo->kind != GALA_TOPO_RING && topo->kind != GALA_TOPO_EXP) return GALA_EINVAL;
-    if (topo->peers < 1 || topo->peers > 2) return GALA_EINVAL;
+    if (topo->kind != GALA_TOPO_RING && topo->kind != GALA_TOPO_EXP && topo->kind != GALA_TOPO_COMPLETE) return GALA_EINVAL;
+    if (topo->kind != GALA_TOPO_COMPLETE && (topo->peers < 1 || topo->peers > 2)) return GALA_EINVAL;
     if (net->kind != GALA_NET_MLP && net->kind != GALA_NET_CONV) return GALA_EINVAL;
     if (net->n_actions < 2 || net->n_actions > 32) return GALA_EINVAL;
-    if (hp->n_envs < 1 || hp->n_steps < 1 || hp->staleness_tau >= 0) return GALA_EINVAL;
+    if (hp->n_envs < 1 || hp->n_steps < 1) return GALA_EINVAL;
     if (!(hp->rms_eps > 0.0f) || !(hp->lr >= 0.0f) || hp->rms_alpha < 0.0f || hp->rms_alpha > 1.0f) return GALA_EINVAL;
     if (net->kind == GALA_NET_MLP && (net->obs_dim < 1 || net->obs_dim > 4096 || net->hidden < 1 || net->hidden > 1024))
         return GALA_EINVAL;
@@ -752,6 +787,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
     ALLOC(c->clip, n); ALLOC(c->norm, n); ALLOC(c->losses, (size_t)n * 4);
     ALLOC(c->norm_partial, (size_t)n * kNormChunks); ALLOC(c->norm_ticket, n);
     ALLOC(c->error_word, 1);
+    ALLOC(c->cons_partial, 592); ALLOC(c->cons_out, 1); ALLOC(c->cons_ticket, 1);
     ALLOC(c->logits, (size_t)n * B * A); ALLOC(c->values, (size_t)n * B);
     ALLOC(c->returns, (size_t)n * S); ALLOC(c->adv, (size_t)n * S);
     ALLOC(c->dlogits, (size_t)n * S * A); ALLOC(c->dvalues, (size_t)n * S);
@@ -871,6 +907,8 @@ int gala_learn(gala_ctx* c, int agent, const gala_rollout* ro) {
 
 int gala_gossip(gala_ctx* c, int agent) {
     if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_gossip: bad agent");
+    if (c->topo.kind == GALA_TOPO_COMPLETE)
+        return fail(c, GALA_ESTATE, "gala_gossip: the complete graph (gradient all-reduce) exists only as gala_step_sync");
     int r = sweep_agent(c, agent, true);
     if (r != GALA_OK) return r;
     c->agents[agent].round++;
@@ -906,7 +944,15 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
         }
     }
     int off[2] = {0, 0};
-    const int np = topo_offsets(c->topo, n, c->sync_round, off);
+    int np = topo_offsets(c->topo, n, c->sync_round, off);
+    if (c->topo.kind == GALA_TOPO_COMPLETE) {
+        // synchronous A2C baseline: average the gradients over all agents, clip the average, and let every
+        // agent take the same RMSProp step; no parameter mixing
+        np = 0;
+        LAUNCH(T_GRAD_NORM, st, launch_allreduce_grads(c->g, n, c->d_pad, st));
+        LAUNCH(T_GRAD_NORM, st, launch_grad_norm(c->g, c->d, c->d_pad, 0, n, c->hp.max_grad_norm, c->norm_partial,
+                                                 c->norm_ticket, c->norm, c->clip, st));
+    }
     SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
     LAUNCH(T_SWEEP_SYNC, st, launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp,
                                             c->error_word, st));
@@ -937,7 +983,7 @@ int gala_sync_all(gala_ctx* c, int timeout_ms) {
 }
 
 int gala_in_peers(const gala_ctx* c, long long round, int agent, int* peers, int* n) {
-    if (!valid_agent(c, agent) || !peers || !n || round < 0) return GALA_EINVAL;
+    if (!valid_agent(c, agent) || !peers || !n || round < 0 || c->topo.kind == GALA_TOPO_COMPLETE) return GALA_EINVAL;
     int off[2];
     const int np = topo_offsets(c->topo, c->n, round, off);
     for (int j = 0; j < np; j++) peers[j] = ((agent - off[j]) % c->n + c->n) % c->n;
@@ -993,6 +1039,25 @@ int gala_set_grad(gala_ctx* c, int agent, const float* grad, float clip_coef) {
     return GALA_OK;
 }
 
+int gala_consensus_distance(gala_ctx* c, double* out) {
+    if (!c || !out) return GALA_EINVAL;
+    int r = gala_sync_all(c, -1);
+    if (r != GALA_OK) return r;
+    LAUNCH(T_GRAD_NORM, c->main_stream, launch_consensus(c->x, c->n, c->d, c->d_pad, c->cons_partial, c->cons_ticket,
+                                                        c->cons_out, c->main_stream));
+    CK(cudaStreamSynchronize(c->main_stream));
+    double sq = 0.0;
+    CK(cudaMemcpy(&sq, c->cons_out, sizeof sq, cudaMemcpyDeviceToHost));
+    *out = std::sqrt(sq);
+    return GALA_OK;
+}
+
+int gala_set_stale_timeout(gala_ctx* c, int timeout_ms) {
+    if (!c || timeout_ms < 0) return GALA_EINVAL;
+    c->stale_timeout_ms = timeout_ms;
+    return GALA_OK;
+}
+
 int gala_param_count(const gala_ctx* c, long long* d, long long* d_padded) {
     if (!c) return GALA_EINVAL;
     if (d) *d = c->d;
@@ -1013,7 +1078,7 @@ int gala_stats(gala_ctx* c, int agent, long long out[8]) {
     if (!valid_agent(c, agent) || !out) return GALA_EINVAL;
     const Agent& a = c->agents[agent];
     out[0] = a.frames; out[1] = a.round; out[2] = a.mixes; out[3] = a.skipped;
-    out[4] = a.stale_sum; out[5] = a.stale_max; out[6] = a.version; out[7] = 0;
+    out[4] = a.stale_sum; out[5] = a.stale_max; out[6] = a.version; out[7] = a.stale_waits;
     return GALA_OK;
 }
 

@@ -139,6 +139,10 @@ cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const flo
 constexpr int kNormChunks = 128;
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
                              double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st);
+cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStream_t st);
+// partial: 592 doubles, ticket: one zeroed unsigned, out: one double (squared distance)
+cudaError_t launch_consensus(const float* x, int n_agents, long d, long d_pad, double* partial, unsigned* ticket,
+                             double* out, cudaStream_t st);
 cudaError_t launch_delay(unsigned long long usec, cudaStream_t st);
 cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st);
 

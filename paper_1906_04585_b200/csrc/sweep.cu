@@ -245,6 +245,74 @@ cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int
     return cudaGetLastError();
 }
 
+// Gradient all-reduce of the synchronous A2C baseline (Sec. 5: the agents average their gradients
+// before each update): every agent's gradient row is replaced by the mean over agents, summed in
+// agent order.  One thread per 16-byte column; reads N*d, writes N*d.
+__global__ void __launch_bounds__(256) allreduce_grads_kernel(float* __restrict__ g, int n_agents, long d_pad, long n4) {
+    const float inv = 1.0f / (float)n_agents;
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int a = 0; a < n_agents; a++) {
+            const float4 t = *reinterpret_cast<const float4*>(g + (long)a * d_pad + 4 * i);
+            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        }
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        for (int a = 0; a < n_agents; a++) *reinterpret_cast<float4*>(g + (long)a * d_pad + 4 * i) = acc;
+    }
+}
+cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStream_t st) {
+    const long n4 = d_pad / 4;
+    int grid = (int)((n4 + 255) / 256);
+    if (grid > 148 * 8) grid = 148 * 8;
+    allreduce_grads_kernel<<<grid, 256, 0, st>>>(g, n_agents, d_pad, n4);
+    return cudaGetLastError();
+}
+
+// Distance from consensus ||X - mean over agents||_F (left side of Proposition 1) in one pass:
+// per column the sum and the sum of squares over agents in double precision,
+// sum_i (x_i - m)^2 = sum_i x_i^2 - (sum_i x_i)^2 / n.  Block partials, fixed-order final sum by
+// the last block; writes the squared distance.
+constexpr int kConsensusBlocks = 592;
+__global__ void __launch_bounds__(256) consensus_kernel(const float* __restrict__ x, int n_agents, long d, long d_pad,
+                                                        double* partial, unsigned* ticket, double* out) {
+    double acc = 0.0;
+    for (long c = blockIdx.x * (long)blockDim.x + threadIdx.x; c < d; c += (long)gridDim.x * blockDim.x) {
+        double s = 0.0, ss = 0.0;
+        for (int a = 0; a < n_agents; a++) {
+            const double t = (double)__ldcs(x + (long)a * d_pad + c);
+            s += t; ss += t * t;
+        }
+        const double dev = ss - s * s / (double)n_agents;
+        acc += dev > 0.0 ? dev : 0.0;
+    }
+    __shared__ double red[256];
+    __shared__ bool last;
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    for (int st = 128; st > 0; st >>= 1) {
+        if (threadIdx.x < st) red[threadIdx.x] += red[threadIdx.x + st];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        partial[blockIdx.x] = red[0];
+        __threadfence();
+        last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        __threadfence();
+        double s = 0.0;
+        for (unsigned k = 0; k < gridDim.x; k++) s += ((volatile double*)partial)[k];
+        *out = s;
+        *ticket = 0;
+    }
+}
+cudaError_t launch_consensus(const float* x, int n_agents, long d, long d_pad, double* partial, unsigned* ticket,
+                             double* out, cudaStream_t st) {
+    consensus_kernel<<<kConsensusBlocks, 256, 0, st>>>(x, n_agents, d, d_pad, partial, ticket, out);
+    return cudaGetLastError();
+}
+
 // Straggler injection: occupies the stream for about `usec` microseconds (one sleeping thread).
 // Bounded twice: by the requested time (capped by the caller) and by an iteration limit.
 __global__ void delay_kernel(unsigned long long usec) {

@@ -41,7 +41,7 @@ def test_argument_validation_needs_no_gpu():
     net = binding.gala_net_spec(binding.GALA_NET_MLP, 8, 64, 4, 0)
     hp = binding.default_hparams(16, 5)
     assert L.gala_create(0, ctypes.byref(topo), ctypes.byref(net), ctypes.byref(hp), ctypes.byref(h)) == binding.GALA_EINVAL
-    bad = binding.gala_topology(binding.GALA_TOPO_COMPLETE, 1)
+    bad = binding.gala_topology(7, 1)            # no such topology
     assert L.gala_create(4, ctypes.byref(bad), ctypes.byref(net), ctypes.byref(hp), ctypes.byref(h)) == binding.GALA_EINVAL
     hp2 = binding.default_hparams(16, 5, rms_eps=0.0)
     assert L.gala_create(4, ctypes.byref(topo), ctypes.byref(net), ctypes.byref(hp2), ctypes.byref(h)) == binding.GALA_EINVAL

@@ -1,0 +1,119 @@
+"""GPU parity of the pieces beyond the core step: the staleness bound of Sec. 3, the distance
+from consensus of Propositions 1-2, and the gradient all-reduce of the synchronous A2C baseline."""
+import numpy as np
+import pytest
+
+import gala_inputs as GI
+from oracle import reference as R
+from tests.helpers import TOL_FP32_NET, TOL_SWEEP, assert_close, oracle_hp, oracle_net
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _learner(w, **hp):
+    from paper_1906_04585_b200 import learner as LM
+    return LM.Learner(w.n_agents, w.topo_kind, w.topo_peers, w.net_kind, w.n_actions, w.n_envs, w.n_steps,
+                      obs_dim=w.obs_dim, hidden=w.hidden, **hp)
+
+
+def test_consensus_distance_matches_oracle_and_contracts():
+    from paper_1906_04585_b200 import binding as B
+    w = GI.WORKLOADS[0].scaled(n_agents=8, topo_kind=R.EXP)
+    L = _learner(w, max_grad_norm=0.0)
+    rng = np.random.default_rng(5)
+    X = rng.normal(size=(w.n_agents, L.d)).astype(np.float32) * 0.1
+    for i in range(w.n_agents):
+        L.set_state(i, params=X[i], sq_avg=np.zeros(L.d, np.float32))
+    d0 = B.gala_consensus_distance(L.ctx)
+    assert abs(d0 - R.consensus_distance(X)) <= 1e-9 * d0
+    # pure gossip (zero gradients): each round contracts by at most sigma_2 of that round's matrix, and
+    # log2(8) rounds of the 1-peer exponential graph reach the mean exactly (up to fp32 rounding)
+    prev = d0
+    for k in range(3):
+        for i in range(w.n_agents):
+            L.set_grad(i, np.zeros(L.d, np.float32), 1.0)
+        L.step_sync(None)
+        dk = B.gala_consensus_distance(L.ctx)
+        s2 = np.linalg.svd(R.mixing_matrix(R.EXP, 1, w.n_agents, k), compute_uv=False)[1]
+        assert dk <= s2 * prev * (1 + 1e-5) + 1e-6
+        prev = dk
+    assert prev <= 1e-5 * d0
+    Xn = np.stack([L.get_params(i) for i in range(w.n_agents)])
+    assert_close("mean", Xn[3], X.astype(np.float64).mean(axis=0), 1e-5)
+    L.close()
+
+
+def test_allreduce_a2c_mode_matches_oracle():
+    # complete graph: gradients averaged over agents, the average clipped, one common RMSProp step
+    w = GI.WORKLOADS[0].scaled(n_agents=5, topo_kind=R.COMPLETE, topo_peers=0)
+    net = oracle_net(w)
+    L = _learner(w)
+    ohp = oracle_hp(L.hp)
+    from paper_1906_04585_b200 import learner as LM
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    for i in range(w.n_agents):
+        L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32))
+    X = p0.astype(np.float64)
+    V = np.zeros_like(X)
+    for k in range(2):
+        ros = [GI.rollout(w, i, k) for i in range(w.n_agents)]
+        dev = [LM.DeviceRollout(r) for r in ros]
+        L.step_sync(dev)
+        L.sync()
+        gm = np.mean([R.learner_grad(net, X, r, ohp)["grad"] for r in ros], axis=0)
+        # the same as one agent with all simulators (footnote of Sec. 5)
+        big = {key: np.concatenate([r[key] for r in ros], axis=1) for key in ros[0]}
+        np.testing.assert_allclose(gm, R.learner_grad(net, X, big, ohp)["grad"], rtol=1e-9, atol=1e-14)
+        c, _ = R.clip_coef(gm, ohp.max_grad_norm)
+        X, V = R.rmsprop(X, gm, V, c, ohp.lr, ohp.rms_alpha, ohp.rms_eps)
+        for i in range(w.n_agents):
+            assert_close("g[%d]" % i, L.get_grad(i), gm, TOL_FP32_NET)
+            assert_close("x[%d]" % i, L.get_params(i), X, TOL_SWEEP)
+            assert_close("v[%d]" % i, L.get_sq_avg(i), V, 2 * TOL_FP32_NET)
+    from paper_1906_04585_b200 import binding as B
+    assert B.gala_consensus_distance(L.ctx) < 1e-6        # all agents stay identical
+    with pytest.raises(B.GalaError):
+        L.gossip(0)
+    L.close()
+
+
+def test_staleness_bound_waits_for_the_in_peer():
+    from paper_1906_04585_b200 import binding as B
+    from paper_1906_04585_b200 import learner as LM
+    w = GI.WORKLOADS[0].scaled(n_agents=2)
+    L = _learner(w, staleness_tau=1)
+    dev = [LM.DeviceRollout(GI.rollout(w, i, 0)) for i in range(2)]
+    # agent 0 alone: two iterations may pass without a message (tau = 1) ...
+    for _ in range(2):
+        L.learn(0, dev[0]); L.gossip(0)
+        assert not B.gala_last_mix(L.ctx, 0)[2]
+    # ... the third finds the bound exceeded and nothing published by its in-peer: refused, nothing enqueued
+    L.learn(0, dev[0])
+    with pytest.raises(B.GalaError) as ei:
+        L.gossip(0)
+    assert ei.value.status == B.GALA_ETIMEOUT
+    assert B.gala_stats(L.ctx, 0)["version"] == 2
+    # the in-peer publishes behind a 20 ms straggler delay: agent 0 now WAITS for that snapshot and averages
+    B.gala_delay(L.ctx, 1, 20000)
+    L.learn(1, dev[1]); L.gossip(1)
+    L.gossip(0)
+    peers, vers, mixed = B.gala_last_mix(L.ctx, 0)
+    assert mixed and peers == [1] and vers == [1]
+    st = B.gala_stats(L.ctx, 0)
+    assert st["stale_waits"] == 1 and st["mixes"] == 1 and st["version"] == 3
+    # with a deadline shorter than the delay the call gives up instead
+    B.gala_set_stale_timeout(L.ctx, 2)
+    for _ in range(2):
+        L.learn(0, dev[0]); L.gossip(0)
+    B.gala_delay(L.ctx, 1, 50000)
+    L.learn(1, dev[1]); L.gossip(1)
+    L.learn(0, dev[0])
+    with pytest.raises(B.GalaError) as ei:
+        L.gossip(0)
+    assert ei.value.status == B.GALA_ETIMEOUT
+    L.sync()
+    L.gossip(0)                         # the snapshot has landed meanwhile
+    assert B.gala_last_mix(L.ctx, 0)[2]
+    L.close()
