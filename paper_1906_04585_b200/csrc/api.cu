@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <thread>
 
@@ -37,6 +38,12 @@ struct Plan {  // one tensor-core product with its descriptors
     GemmOperand A, B;
     GemmArgs args;
     int tag = 0;
+};
+struct ConvPlan {  // one forward or data-gradient convolution (input resident in shared memory)
+    CUtensorMap x, w;
+    ConvArgs args;
+    int tag = 0;
+    bool built = false;
 };
 
 // Kernel classes for launch counting and optional per-class device timing.
@@ -108,6 +115,9 @@ struct gala_ctx {
     long splitk_group_stride = 0;
     int max_split = 32;
     Plan fwd[3], fc_fwd, fc_wgrad, fc_dgrad, wgrad[3], dgrad[3];
+    ConvPlan cfwd[3], cdgrad[3];
+    uint32_t* gate[2] = {nullptr, nullptr};   // ReLU gate bits of act[0], act[1]
+    bool legacy_conv = false;
 };
 
 namespace {
@@ -377,7 +387,47 @@ int build_plans(gala_ctx* c) {
         dg.args.mask = c->act[2]; dg.args.mask_group_stride = B * kFeat;
         dg.args.out = c->dy[2]; dg.args.out_group_stride = S * kFeat; dg.args.ldc = kFeat;
     }
+    for (int l = 0; l < 3; l++) {
+        const int CO = kConvCout[l];
+        ConvPlan& f = c->cfwd[l];
+        memset(&f.args, 0, sizeof f.args);
+        f.tag = T_GEMM_CONV_FWD + l;
+        f.args.variant = CV_CONV1_FWD + l;
+        f.args.a_samples = (int)B;
+        f.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
+        f.args.bias = c->x + c->cl.b[l]; f.args.bias_group_stride = dp;
+        f.args.out = c->act[l]; f.args.out_group_stride = B * P[l] * CO;
+        if (l < 2) { f.args.gate_out = c->gate[l]; f.args.gate_group_stride = B * P[l] * CO / 32; }
+        f.args.error_word = c->error_word;
+        const void* xin = l == 0 ? (const void*)c->frames : (const void*)c->act[l - 1];
+        ok &= make_conv_maps(f.args.variant, &f.x, &f.w, xin, (uint64_t)n * B, c->shadow + c->cl.w[l], n, dp);
+        f.built = true;
+        if (l > 0) {
+            ConvPlan& d = c->cdgrad[l];
+            memset(&d.args, 0, sizeof d.args);
+            d.tag = T_GEMM_CONV_DGRAD + l;
+            d.args.variant = l == 1 ? CV_CONV2_DGRAD : CV_CONV3_DGRAD;
+            d.args.a_samples = (int)S;
+            d.args.scale = 1.0f;
+            const long in_elems = (long)kConvIn[l] * kConvIn[l] * kConvCin[l];
+            d.args.gate_in = c->gate[l - 1]; d.args.gate_group_stride = B * in_elems / 32;
+            d.args.out = c->dy[l - 1]; d.args.out_group_stride = S * in_elems;
+            d.args.error_word = c->error_word;
+            ok &= make_conv_maps(d.args.variant, &d.x, &d.w, c->dy[l], (uint64_t)n * S, c->shadow + c->cl.w[l], n, dp);
+            d.built = true;
+        }
+    }
     return ok ? GALA_OK : fail(c, GALA_ECUDA, "cuTensorMapEncodeTiled failed while building GEMM descriptors");
+}
+
+int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, cudaStream_t st) {
+    ConvArgs a = p.args;
+    a.group0 = agent0; a.groups = groups; a.rows = rows;
+    a.out += (long)agent0 * a.out_group_stride;
+    if (a.gate_out) a.gate_out += (long)agent0 * a.gate_group_stride;
+    if (a.gate_in) a.gate_in += (long)agent0 * a.gate_group_stride;
+    LAUNCH(p.tag, st, launch_conv(p.x, p.w, a, st));
+    return GALA_OK;
 }
 
 int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override, cudaStream_t st) {
@@ -421,7 +471,8 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         const int P[3] = {400, 81, 49};
         LAUNCH(T_CAST_FRAMES, st, launch_cast_frames(obs, c->frames + (long)agent0 * B * kFramePix, B * kFramePix, rows, groups, st));
         for (int l = 0; l < 3; l++) {
-            int r = run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st);
+            int r = c->legacy_conv ? run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st)
+                                   : run_conv(c, c->cfwd[l], agent0, groups, rows, st);
             if (r != GALA_OK) return r;
         }
         // hidden layer: with few rows there are only a handful of output tiles, each streaming 0.8 MB of
@@ -536,7 +587,11 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         for (int l = 2; l >= 0; l--) {
             if ((r = fork()) != GALA_OK) return r;
             if ((r = run_wgrad(c, c->wgrad[l], agent0, groups, ws)) != GALA_OK) return r;
-            if (l > 0 && (r = run_plan(c, c->dgrad[l], agent0, groups, 0, st)) != GALA_OK) return r;
+            if (l > 0) {
+                r = c->legacy_conv ? run_plan(c, c->dgrad[l], agent0, groups, 0, st)
+                                   : run_conv(c, c->cdgrad[l], agent0, groups, (int)S, st);
+                if (r != GALA_OK) return r;
+            }
         }
         // the bias gradients need every dY: they follow conv1's weight gradient on the side stream
         {   // all four bias gradients (column sums of dh, dY3, dY2, dY1) in one launch
@@ -798,10 +853,13 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
     if (c->conv) {
         const int P[3] = {400, 81, 49};
         CK(gemm_init());
+        CK(conv_init());
+        c->legacy_conv = getenv("GALA_CONV_LEGACY") != nullptr;
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {
             ALLOC(c->act[l], (size_t)n * B * P[l] * kConvCout[l]);
+            if (l < 2) ALLOC(c->gate[l], (size_t)n * B * P[l] * kConvCout[l] / 32);
             ALLOC(c->dy[l], (size_t)n * S * P[l] * kConvCout[l]);
         }
         ALLOC(c->frames, (size_t)n * B * kFramePix);

@@ -1,0 +1,479 @@
+// Convolutions of the 84x84x4 -> 20x20x32 -> 9x9x64 -> 7x7x64 trunk (Appendix C.2 network), forward
+// and data gradient, on the tcgen05 tensor cores with the layer input resident in shared memory.
+//
+// A convolution is a sum over kernel offsets ("taps") of small products
+//     D[pixel][n] += X[pixel + offset(tap)][k] * Wtap[k][n] .
+// When the pixels of an image are laid out row after row with a fixed pitch, "pixel + offset" is a
+// constant row shift, so every tap reads the SAME shared-memory image of the input, only from a
+// start address moved by shift * row_bytes.  The input of one work unit (a sample, or five output
+// lines of conv1) is therefore fetched once by TMA - not once per tap - and all weights of the layer
+// stay in shared memory while a CTA works on one agent.  Rows whose pixel falls outside the valid
+// output range (the pitch minus the output width, the tail of the 128-row MMA tile) are computed
+// and dropped by the epilogue.
+//
+// Strided layers are turned into shifts by splitting the input into phase planes:
+//   conv1 (8x8, stride 4): plane py = input lines y = 4u + py, each line seen as 21 groups of
+//          4 pixels x 4 channels (16 elements = one K=16 MMA); tap (ky, b): plane ky % 4,
+//          shift (ky / 4) * 21 + b
+//   conv2 (4x4, stride 2): plane (py, px) = pixels (2u + py, 2v + px), 32 channels a row; tap (ky, kx):
+//          plane (ky % 2, kx % 2), shift (ky / 2) * 10 + kx / 2
+//   conv3 (3x3, stride 1): one plane, shift ky * 9 + kx
+// Data gradients use the zero-padded gradient image of the layer output (TMA fills out-of-range
+// coordinates with zeros), pitch 11:
+//   conv3: dX[y][x] = sum_taps dY[y - ky][x - kx] W[.][ky][kx][.], shift (2 - ky) * 11 + (2 - kx)
+//   conv2: the four parity classes (py, px) of input pixels (2u + py, 2v + px) share the shifted dY
+//          view of tap (a, b) = (ky / 2, kx / 2) and differ only in the weight block, so they become
+//          the N = 4 x 32 columns of one product: shift (1 - a) * 11 + (1 - b)
+//
+// One CTA (320 threads, persistent over a contiguous range of work units):
+//   warp 0    TMA producer: input planes of the next units into a ring of stages; the agent's weights
+//             whenever the agent changes
+//   warp 1    MMA issuer (one thread): taps x K-chunks tcgen05.mma per unit into one of two
+//             tensor-memory accumulators
+//   warps 2-9 two epilogue groups of four warps, one per accumulator buffer: tcgen05.ld (a thread owns a
+//             pixel), scale / bias / ReLU (+ gate bits) or the ReLU gate, 64 contiguous bytes of bf16 per 32 columns
+// Every wait is bounded; when one runs out the CTA raises the caller's error word, lets the copies it
+// issued land, frees its tensor memory and returns.
+#include "internal.h"
+#include "tcgen05.cuh"
+
+namespace gala {
+
+template <int V> struct ConvTraits;
+template <> struct ConvTraits<CV_CONV1_FWD> {
+    static constexpr int ROWB = 32, LAYOUT = 6, PLANES = 4, PLANE_ROWS = 126, PLANE_STRIDE = 4096, UPS = 4;
+    static constexpr int TAPS = 16, KKN = 1, BN = 32, PITCH = 21, OH = 5, OW = 20;
+    static constexpr int W_BOXES = 16, W_BOX_BYTES = 1024, B_MN = 0, B_LAYOUT = 6, B_SBO = 256, B_LBO = 16;
+};
+template <> struct ConvTraits<CV_CONV2_FWD> {
+    static constexpr int ROWB = 64, LAYOUT = 4, PLANES = 4, PLANE_ROWS = 100, PLANE_STRIDE = 6656, UPS = 1;
+    static constexpr int TAPS = 16, KKN = 2, BN = 64, PITCH = 10, OH = 9, OW = 9;
+    static constexpr int W_BOXES = 16, W_BOX_BYTES = 4096, B_MN = 0, B_LAYOUT = 4, B_SBO = 512, B_LBO = 16;
+};
+template <> struct ConvTraits<CV_CONV3_FWD> {
+    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 81, PLANE_STRIDE = 11264, UPS = 1;
+    static constexpr int TAPS = 9, KKN = 4, BN = 64, PITCH = 9, OH = 7, OW = 7;
+    static constexpr int W_BOXES = 9, W_BOX_BYTES = 8192, B_MN = 0, B_LAYOUT = 2, B_SBO = 1024, B_LBO = 16;
+};
+template <> struct ConvTraits<CV_CONV2_DGRAD> {
+    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 121, PLANE_STRIDE = 16384, UPS = 1;
+    static constexpr int TAPS = 4, KKN = 4, BN = 128, PITCH = 11, OH = 10, OW = 10;
+    static constexpr int W_BOXES = 16, W_BOX_BYTES = 4096, B_MN = 1, B_LAYOUT = 4, B_SBO = 512, B_LBO = 4096;
+};
+template <> struct ConvTraits<CV_CONV3_DGRAD> {
+    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 121, PLANE_STRIDE = 16384, UPS = 1;
+    static constexpr int TAPS = 9, KKN = 4, BN = 64, PITCH = 11, OH = 9, OW = 9;
+    static constexpr int W_BOXES = 9, W_BOX_BYTES = 8192, B_MN = 1, B_LAYOUT = 2, B_SBO = 1024, B_LBO = 8192;
+};
+
+constexpr int kConvMaxStages = 8;
+constexpr int kConvSlack = 8 * 1024;             // rows an MMA reads past the last plane of the ring
+constexpr int kConvEpiWarpBytes = 512;           // an epilogue warp's copy of the layer's bias
+constexpr int kConvSmemMax = 224 * 1024;
+
+// plane and row shift of a tap
+template <int V> __host__ __device__ constexpr void tap_view(int t, int& plane, int& shift) {
+    if constexpr (V == CV_CONV1_FWD) { const int ky = t >> 1; plane = ky & 3; shift = (ky >> 2) * 21 + (t & 1); }
+    else if constexpr (V == CV_CONV2_FWD) { const int ky = t >> 2, kx = t & 3; plane = (ky & 1) * 2 + (kx & 1); shift = (ky >> 1) * 10 + (kx >> 1); }
+    else if constexpr (V == CV_CONV3_FWD) { const int ky = t / 3; plane = 0; shift = ky * 9 + (t - ky * 3); }
+    else if constexpr (V == CV_CONV2_DGRAD) { plane = 0; shift = (1 - (t >> 1)) * 11 + (1 - (t & 1)); }
+    else { const int ky = t / 3; plane = 0; shift = (2 - ky) * 11 + (2 - (t - ky * 3)); }
+}
+// first column (inside W[co][(ky, kx, ci)]) of the weight box that goes to shared-memory slot j
+template <int V> __device__ __forceinline__ int weight_col(int j) {
+    if constexpr (V == CV_CONV1_FWD) return j * 16;
+    else if constexpr (V == CV_CONV2_FWD) return j * 32;
+    else if constexpr (V == CV_CONV2_DGRAD) {
+        // slot = tap * 4 + class: the four classes of a tap side by side form its N = 128 operand
+        const int t = j >> 2, cls = j & 3;
+        return (((cls >> 1) + 2 * (t >> 1)) * 4 + (cls & 1) + 2 * (t & 1)) * 32;
+    } else return j * 64;
+}
+
+struct UnitCoord { int gz, s, q; };
+template <int V> __device__ __forceinline__ UnitCoord decode_unit(int u, int rows) {
+    constexpr int UPS = ConvTraits<V>::UPS;
+    UnitCoord c;
+    c.q = u % UPS;
+    const int r = u / UPS;
+    c.gz = r / rows;
+    c.s = r - c.gz * rows;
+    return c;
+}
+
+template <int V>
+__global__ void __launch_bounds__(320, 1)
+conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const ConvArgs p,
+                     const int nst, const long total_units) {
+    using T = ConvTraits<V>;
+    constexpr int STAGE = T::PLANES * T::PLANE_STRIDE;
+    constexpr int W_BYTES = T::W_BOXES * T::W_BOX_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kConvMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kConvMaxStages];
+    __shared__ __align__(8) uint64_t acc_full[2];
+    __shared__ __align__(8) uint64_t acc_empty[2];
+    __shared__ __align__(8) uint64_t w_full;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int issued_iters, issued_w;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smW = smem;
+    uint8_t* smX = smem + W_BYTES;
+    uint8_t* smE = smX + nst * STAGE + kConvSlack;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr uint32_t tmem_cols = 2u * T::BN;   // 64, 128 or 256
+
+    // contiguous range of units of this CTA: at most a few agents, so few weight reloads
+    const int u_begin = (int)(total_units * blockIdx.x / gridDim.x);
+    const int u_end = (int)(total_units * (blockIdx.x + 1) / gridDim.x);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        mbar_init(&w_full, 1);
+        abort_flag = 0;
+        issued_iters = 0;
+        issued_w = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        int it = 0, cur_g = -1, wl = 0;
+        for (int u = u_begin; u < u_end; u++, it++) {
+            const UnitCoord c = decode_unit<V>(u, p.rows);
+            const int group = p.group0 + c.gz;
+            if (c.gz != cur_g) {
+                // new agent: its weights replace the previous agent's once every MMA that read those is done
+                int go = 1;
+                if (lane == 0 && it > 0)
+                    go = mbar_wait(&empty_bar[(it - 1) % nst], (uint32_t)((it - 1) / nst) & 1u, &abort_flag) ? 1 : 0;
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (!go) break;
+                if (lane == 0) mbar_expect_tx(&w_full, (uint32_t)W_BYTES);
+                __syncwarp();
+                if (lane < T::W_BOXES) tma_load_3d(smW + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
+                __syncwarp();
+                cur_g = c.gz;
+                wl++;
+                if (lane == 0) issued_w = wl;
+            }
+            const int s = it % nst;
+            int go = 1;
+            if (lane == 0) go = mbar_wait(&empty_bar[s], ((uint32_t)(it / nst) & 1u) ^ 1u, &abort_flag) ? 1 : 0;
+            go = __shfl_sync(0xffffffffu, go, 0);
+            if (!go) break;
+            if (lane == 0) mbar_expect_tx(&full_bar[s], (uint32_t)(T::PLANES * T::PLANE_ROWS * T::ROWB));
+            __syncwarp();
+            const int sample = group * p.a_samples + c.s;
+            if (lane < T::PLANES) {
+                uint8_t* dst = smX + s * STAGE + lane * T::PLANE_STRIDE;
+                if constexpr (V == CV_CONV1_FWD) tma_load_5d(dst, &tmX, &full_bar[s], 0, 0, lane, 5 * c.q, sample);
+                else if constexpr (V == CV_CONV2_FWD) tma_load_5d(dst, &tmX, &full_bar[s], 32 * (lane & 1), 0, lane >> 1, 0, sample);
+                else if constexpr (V == CV_CONV3_FWD) tma_load_3d(dst, &tmX, &full_bar[s], 0, 0, sample);
+                else if constexpr (V == CV_CONV2_DGRAD) tma_load_4d(dst, &tmX, &full_bar[s], 0, -1, -1, sample);
+                else tma_load_4d(dst, &tmX, &full_bar[s], 0, -2, -2, sample);
+            }
+            __syncwarp();
+            if (lane == 0) issued_iters = it + 1;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_instr_desc(T::BN, 0, T::B_MN);
+            const uint64_t bd_base = make_smem_desc_raw(smem_u32(smW), T::B_LAYOUT, T::B_SBO, T::B_LBO);
+            int it = 0, cur_g = -1, wl = 0;
+            for (int u = u_begin; u < u_end; u++, it++) {
+                const UnitCoord c = decode_unit<V>(u, p.rows);
+                if (c.gz != cur_g) {
+                    if (!mbar_wait(&w_full, (uint32_t)wl & 1u, &abort_flag)) break;
+                    wl++;
+                    cur_g = c.gz;
+                }
+                const int ab = it & 1;
+                if (!mbar_wait(&acc_empty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, &abort_flag)) break;
+                const int s = it % nst;
+                if (!mbar_wait(&full_bar[s], (uint32_t)(it / nst) & 1u, &abort_flag)) break;
+                tcgen05_fence_after();
+                const uint32_t tmem_acc = tmem_base + (uint32_t)ab * T::BN;
+                const uint32_t x_addr = smem_u32(smX + s * STAGE);
+                // One thread issues every MMA, so the loop is unrolled completely: the tap's plane, row shift
+                // and weight slot fold into constants that are added to the address field of two base
+                // descriptors (16-byte units; the ring and the weights lie below 256 KiB, so no carry leaves it).
+                const uint64_t ad_base = make_smem_desc_raw(x_addr, T::LAYOUT, 8 * T::ROWB, 16);
+#pragma unroll
+                for (int t = 0; t < T::TAPS; t++) {
+                    int plane, shift;
+                    tap_view<V>(t, plane, shift);
+                    const uint32_t a_off = plane * T::PLANE_STRIDE + shift * T::ROWB;
+                    const uint32_t b_off = (V == CV_CONV2_DGRAD ? t * 4 * T::W_BOX_BYTES : t * T::W_BOX_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < T::KKN; kk++) {
+                        // K = 16 further on: 32 B along a K-major row, 16 rows of an MN-major tile
+                        const uint32_t bk = T::B_MN ? kk * 16 * (T::B_LAYOUT == 4 ? 64 : 128) : kk * 32;
+                        umma_bf16(tmem_acc, ad_base + (uint64_t)((a_off + kk * 32) >> 4), bd_base + (uint64_t)((b_off + bk) >> 4),
+                                  idesc, (t | kk) != 0 ? 1u : 0u);
+                    }
+                }
+                umma_commit(&empty_bar[s]);     // the stage may be refilled ...
+                umma_commit(&acc_full[ab]);     // ... and the accumulator read, once the MMAs above are done
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue: group eg owns accumulator buffer eg
+        // A thread owns one row of the tile (one pixel): per 32-column block it reads its 32 accumulators
+        // from tensor memory, applies scale / bias / ReLU or the ReLU gate, and stores 64 contiguous bytes.
+        // The gate values depend only on the unit, so they are fetched before the wait for the MMAs.
+        const int eg = (warp - 2) >> 2;
+        const int q = warp & 3;                    // lane quarter of tensor memory this warp may read
+        constexpr int kLastRow = (T::OH - 1) * T::PITCH + T::OW - 1;   // last row of a tile that is a real pixel
+        constexpr bool kFwd = V == CV_CONV1_FWD || V == CV_CONV2_FWD || V == CV_CONV3_FWD;
+        constexpr int NCH = T::BN / 32;
+        float* sbias = reinterpret_cast<float*>(smE + (warp - 2) * kConvEpiWarpBytes);   // this warp's copy of the bias
+        const int m = q * 32 + lane;
+        const int pa = m / T::PITCH, pb = m - pa * T::PITCH;
+        const bool valid = pa < T::OH && pb < T::OW;
+        // element offset of this thread's pixel inside the agent's tensor (pixel (2a, 2b) for the conv2 gradient)
+        auto pixel_off = [&](const UnitCoord& c) -> long {
+            if constexpr (V == CV_CONV1_FWD) return ((long)c.s * 400 + (5 * c.q + pa) * 20 + pb) * 32;
+            else if constexpr (V == CV_CONV2_FWD) return ((long)c.s * 81 + pa * 9 + pb) * 64;
+            else if constexpr (V == CV_CONV3_FWD) return ((long)c.s * 49 + pa * 7 + pb) * 64;
+            else if constexpr (V == CV_CONV2_DGRAD) return ((long)c.s * 400 + (2 * pa) * 20 + 2 * pb) * 32;
+            else return ((long)c.s * 81 + pa * 9 + pb) * 64;
+        };
+        // ReLU gates of the layer input, one bit per channel (bit set: the activation was positive), written
+        // by the forward pass of the layer below.  They depend only on the unit, so the words of the NEXT
+        // tile of this group are fetched before the current one is processed.
+        uint32_t gate[kFwd ? 1 : NCH];
+        auto load_gates = [&](int u, uint32_t* g) {
+            if constexpr (!kFwd) {
+#pragma unroll
+                for (int ch = 0; ch < NCH; ch++) g[ch] = 0u;
+                if (u < u_end && valid) {
+                    const UnitCoord c = decode_unit<V>(u, p.rows);
+                    const uint32_t* gp = p.gate_in + (long)c.gz * p.gate_group_stride + pixel_off(c) / 32;
+                    if constexpr (V == CV_CONV2_DGRAD) {   // words of pixels (2a, 2b), (2a, 2b+1), (2a+1, 2b), (2a+1, 2b+1)
+                        const uint2 g0 = __ldg(reinterpret_cast<const uint2*>(gp));
+                        const uint2 g1 = __ldg(reinterpret_cast<const uint2*>(gp + 20));
+                        g[0] = g0.x; g[1] = g0.y; g[2] = g1.x; g[3] = g1.y;
+                    } else {                               // the two words (64 channels) of pixel (a, b)
+                        const uint2 g0 = __ldg(reinterpret_cast<const uint2*>(gp));
+                        g[0] = g0.x; g[1] = g0.y;
+                    }
+                }
+            }
+        };
+        load_gates(u_begin + eg, gate);
+        int cur_g = -1;
+        int it = eg;
+        for (int u = u_begin + eg; u < u_end; u += 2, it += 2) {
+            const UnitCoord c = decode_unit<V>(u, p.rows);
+            const long off = pixel_off(c);
+            __nv_bfloat16* out = p.out + (long)c.gz * p.out_group_stride + off;
+            // column block c0 -> where it goes: forward, conv3 gradient: channels c0.. of the pixel; conv2
+            // gradient: block = parity class (py, px) -> pixel (2a + py, 2b + px), all 32 channels
+            auto block_add = [](int c0) -> int {
+                if constexpr (V == CV_CONV2_DGRAD) return ((c0 >> 6) * 20 + ((c0 >> 5) & 1)) * 32;
+                else return c0;
+            };
+            uint32_t gate_next[kFwd ? 1 : NCH];
+            if constexpr (kFwd) {
+                if (c.gz != cur_g) {
+                    const float* bias = p.bias + (long)(p.group0 + c.gz) * p.bias_group_stride;
+                    __syncwarp();
+                    for (int j = lane; j < T::BN; j += 32) sbias[j] = __ldg(bias + j);
+                    __syncwarp();
+                    cur_g = c.gz;
+                }
+            } else {
+                load_gates(u + 2, gate_next);
+            }
+            if (!mbar_wait(&acc_full[eg], ((uint32_t)it >> 1) & 1u, &abort_flag)) break;
+            tcgen05_fence_after();
+            if (q * 32 <= kLastRow) {
+                const uint32_t tmem_acc = tmem_base + (uint32_t)eg * T::BN + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+                for (int ch = 0; ch < NCH; ch++) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_acc + (uint32_t)(ch * 32), r);
+                    uint32_t o[16];
+                    uint32_t bits = 0u;
+#pragma unroll
+                    for (int j = 0; j < 16; j++) {
+                        float v0 = __uint_as_float(r[2 * j]), v1 = __uint_as_float(r[2 * j + 1]);
+                        if constexpr (kFwd) {
+                            const float2 bv = *reinterpret_cast<const float2*>(sbias + ch * 32 + 2 * j);
+                            v0 = fmaxf(fmaf(v0, p.scale, bv.x), 0.0f);
+                            v1 = fmaxf(fmaf(v1, p.scale, bv.y), 0.0f);
+                        } else {
+                            if (!((gate[ch] >> (2 * j)) & 1u)) v0 = 0.0f;
+                            if (!((gate[ch] >> (2 * j + 1)) & 1u)) v1 = 0.0f;
+                        }
+                        o[j] = pack2(v0, v1);
+                        if constexpr (kFwd) {   // gate of the stored (rounded) activation
+                            if (o[j] & 0x00007fffu) bits |= 1u << (2 * j);
+                            if (o[j] & 0x7fff0000u) bits |= 1u << (2 * j + 1);
+                        }
+                    }
+                    if (valid) {   // two 32-byte stores: every store fills whole sectors
+                        st_global_v8(out + block_add(ch * 32), &o[0]);
+                        st_global_v8(out + block_add(ch * 32) + 16, &o[8]);
+                        if constexpr (kFwd) {
+                            if (p.gate_out) p.gate_out[(long)c.gz * p.gate_group_stride + off / 32 + ch] = bits;
+                        }
+                    }
+                }
+            }
+            if constexpr (!kFwd) {
+#pragma unroll
+                for (int ch = 0; ch < NCH; ch++) gate[ch] = gate_next[ch];
+            }
+            // this warp no longer reads the accumulator buffer
+            tcgen05_fence_before();
+            if (lane == 0) mbar_arrive(&acc_empty[eg]);
+        }
+    }
+
+    // teardown
+    tcgen05_fence_before();
+    __syncthreads();
+    if (abort_flag) {
+        if (threadIdx.x == 0) {
+            if (p.error_word) atomicExch(p.error_word, 1);
+            // let copies that were already issued land before the shared memory goes away
+            const int issued = issued_iters;
+            for (int it = max(0, issued - nst); it < issued; it++) {
+                const int s = it % nst;
+                const uint32_t ph = (uint32_t)(it / nst) & 1u;
+                for (uint32_t i = 0; i < (1u << 16); i++) {
+                    if (mbar_try_wait(&full_bar[s], ph)) break;
+                    __nanosleep(64);
+                }
+            }
+            if (issued_w > 0)
+                for (uint32_t i = 0; i < (1u << 16); i++) {
+                    if (mbar_try_wait(&w_full, (uint32_t)(issued_w - 1) & 1u)) break;
+                    __nanosleep(64);
+                }
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+template <int V> static cudaError_t conv_attr() {
+    return cudaFuncSetAttribute(conv_resident_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, kConvSmemMax);
+}
+cudaError_t conv_init() {
+    static bool done = false;
+    if (done) return cudaSuccess;
+    cudaError_t e;
+    if ((e = conv_attr<CV_CONV1_FWD>()) != cudaSuccess) return e;
+    if ((e = conv_attr<CV_CONV2_FWD>()) != cudaSuccess) return e;
+    if ((e = conv_attr<CV_CONV3_FWD>()) != cudaSuccess) return e;
+    if ((e = conv_attr<CV_CONV2_DGRAD>()) != cudaSuccess) return e;
+    if ((e = conv_attr<CV_CONV3_DGRAD>()) != cudaSuccess) return e;
+    done = true;
+    return cudaSuccess;
+}
+
+bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const void* x_base, uint64_t samples,
+                    const void* w_base, uint64_t groups, uint64_t w_group_stride_elems) {
+    bool ok = true;
+    switch (variant) {
+    case CV_CONV1_FWD: {   // bf16 frames [sample][84][84][4] as [sample][y/4][y%4][x/4][4 px x 4 ch]
+        const uint64_t dims[5] = {16, 21, 4, 21, samples}, str[4] = {32, 672, 2688, 56448};
+        const uint32_t box[5] = {16, 21, 1, 6, 1};
+        ok &= make_tensor_map_nd(x_map, x_base, 5, dims, str, box, 2);
+        const uint64_t wd[3] = {256, 32, groups}, ws[2] = {512, w_group_stride_elems * 2};
+        const uint32_t wb[3] = {16, 32, 1};
+        ok &= make_tensor_map_nd(w_map, w_base, 3, wd, ws, wb, 2);
+        break;
+    }
+    case CV_CONV2_FWD: {   // act1 [sample][20][20][32] as [sample][y/2][y%2][x/2][2 px x 32 ch]
+        const uint64_t dims[5] = {64, 10, 2, 10, samples}, str[4] = {128, 1280, 2560, 25600};
+        const uint32_t box[5] = {32, 10, 1, 10, 1};
+        ok &= make_tensor_map_nd(x_map, x_base, 5, dims, str, box, 1);
+        break;
+    }
+    case CV_CONV3_FWD: {   // act2 [sample][81 pixels][64]
+        const uint64_t dims[3] = {64, 81, samples}, str[2] = {128, 10368};
+        const uint32_t box[3] = {64, 81, 1};
+        ok &= make_tensor_map_nd(x_map, x_base, 3, dims, str, box, 0);
+        break;
+    }
+    case CV_CONV2_DGRAD: { // dY2 [sample][9][9][64], boxes reach one pixel past every edge
+        const uint64_t dims[4] = {64, 9, 9, samples}, str[3] = {128, 1152, 10368};
+        const uint32_t box[4] = {64, 11, 11, 1};
+        ok &= make_tensor_map_nd(x_map, x_base, 4, dims, str, box, 0);
+        break;
+    }
+    case CV_CONV3_DGRAD: { // dY3 [sample][7][7][64], boxes reach two pixels past every edge
+        const uint64_t dims[4] = {64, 7, 7, samples}, str[3] = {128, 896, 6272};
+        const uint32_t box[4] = {64, 11, 11, 1};
+        ok &= make_tensor_map_nd(x_map, x_base, 4, dims, str, box, 0);
+        break;
+    }
+    default: return false;
+    }
+    if (variant == CV_CONV2_FWD || variant == CV_CONV2_DGRAD) {   // W2[64][512]: 32-column blocks
+        const uint64_t wd[3] = {512, 64, groups}, ws[2] = {1024, w_group_stride_elems * 2};
+        const uint32_t wb[3] = {32, 64, 1};
+        ok &= make_tensor_map_nd(w_map, w_base, 3, wd, ws, wb, 1);
+    } else if (variant == CV_CONV3_FWD || variant == CV_CONV3_DGRAD) {   // W3[64][576]: 64-column blocks
+        const uint64_t wd[3] = {576, 64, groups}, ws[2] = {1152, w_group_stride_elems * 2};
+        const uint32_t wb[3] = {64, 64, 1};
+        ok &= make_tensor_map_nd(w_map, w_base, 3, wd, ws, wb, 0);
+    }
+    return ok;
+}
+
+template <int V>
+static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, const ConvArgs& a, cudaStream_t st) {
+    using T = ConvTraits<V>;
+    constexpr int STAGE = T::PLANES * T::PLANE_STRIDE;
+    constexpr int fixed = T::W_BOXES * T::W_BOX_BYTES + kConvSlack + 8 * kConvEpiWarpBytes + 1024;
+    int nst = (kConvSmemMax - fixed) / STAGE;
+    if (nst > kConvMaxStages) nst = kConvMaxStages;
+    if (nst < 2) return cudaErrorInvalidValue;
+    const long units = (long)a.groups * a.rows * T::UPS;
+    if (units <= 0) return cudaSuccess;
+    if (units > 0x7fffffffL) return cudaErrorInvalidValue;
+    const size_t smem = (size_t)fixed + (size_t)nst * STAGE;
+    const int grid = (int)(units < 148 ? units : 148);
+    conv_resident_kernel<V><<<grid, 320, smem, st>>>(x, w, a, nst, units);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_conv(const CUtensorMap& x, const CUtensorMap& w, const ConvArgs& a, cudaStream_t st) {
+    if (a.groups < 1 || a.rows < 0 || !a.out) return cudaErrorInvalidValue;
+    const bool fwd = a.variant == CV_CONV1_FWD || a.variant == CV_CONV2_FWD || a.variant == CV_CONV3_FWD;
+    if (fwd ? !a.bias : !a.gate_in) return cudaErrorInvalidValue;
+    switch (a.variant) {
+    case CV_CONV1_FWD: return launch_conv_v<CV_CONV1_FWD>(x, w, a, st);
+    case CV_CONV2_FWD: return launch_conv_v<CV_CONV2_FWD>(x, w, a, st);
+    case CV_CONV3_FWD: return launch_conv_v<CV_CONV3_FWD>(x, w, a, st);
+    case CV_CONV2_DGRAD: return launch_conv_v<CV_CONV2_DGRAD>(x, w, a, st);
+    case CV_CONV3_DGRAD: return launch_conv_v<CV_CONV3_DGRAD>(x, w, a, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace gala

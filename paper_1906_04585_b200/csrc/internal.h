@@ -102,10 +102,11 @@ bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t
 // rows x cols fp32 matrix, unswizzled box_rows x box_cols tile (gemm_init() first).
 bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
                          uint32_t box_cols, uint32_t box_rows);
-// General bf16 tensor map of rank 3..5, 128-byte swizzle, or 64-byte swizzle for 64-byte rows
-// (dims/strides innermost first).  Dimensions may overlap (a stride smaller than the extent below it).
+// General bf16 tensor map of rank 3..5 (dims/strides innermost first).  swizzle: 0 = 128-byte, 1 = 64-byte
+// (64-byte rows), 2 = 32-byte (32-byte rows).  Dimensions may overlap (a stride smaller than the extent
+// below it); a box may be larger than a dimension (the rest reads as zero).
 bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                        const uint64_t* strides_bytes, const uint32_t* box, int sw64 = 0);
+                        const uint64_t* strides_bytes, const uint32_t* box, int swizzle = 0);
 // Builds the descriptor for an operand of a GEMM with the given tile height
 // (128 for A, block_n for B).
 bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_extent, uint64_t k_extent,
@@ -117,6 +118,33 @@ cudaError_t launch_splitk_reduce_act(const float* partials, __nv_bfloat16* out, 
 cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, int split_k,
                                  long split_stride, int groups, long partial_group_stride,
                                  long out_group_stride, cudaStream_t st);
+
+// ---------------------------------------------------------------- convolutions with a resident input
+// Forward and data-gradient convolutions of the trunk (conv.cu).  Tensors are NHWC bf16; weights
+// W[co][(ky, kx, ci)] bf16; group g (agent) uses sample block g * a_samples.. of the input tensor.
+enum ConvVariant : int { CV_CONV1_FWD = 0, CV_CONV2_FWD, CV_CONV3_FWD, CV_CONV2_DGRAD, CV_CONV3_DGRAD };
+struct ConvArgs {
+    int variant;
+    int groups, group0;    // agents of this launch: group0 .. group0 + groups - 1
+    int rows;              // samples per agent to process
+    int a_samples;         // samples per agent in the input tensor
+    float scale;           // forward: applied to the accumulator before the bias
+    const float* bias;     // forward: per output channel, agent g at bias + g * bias_group_stride
+    long bias_group_stride;
+    __nv_bfloat16* out;    // first agent of the launch; agent i of the launch at out + i * out_group_stride
+    long out_group_stride;
+    // ReLU gates, one bit per channel and pixel: word [sample][pixel][channel / 32], bit channel % 32 set
+    // when the stored activation is positive.  Forward (conv1, conv2): written next to the activation
+    // (may be null); data gradient: the gates of the layer input, which multiply the result.
+    uint32_t* gate_out;
+    const uint32_t* gate_in;
+    long gate_group_stride;      // words per agent
+    int* error_word;
+};
+cudaError_t conv_init();
+bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const void* x_base, uint64_t samples,
+                    const void* w_base, uint64_t groups, uint64_t w_group_stride_elems);
+cudaError_t launch_conv(const CUtensorMap& x, const CUtensorMap& w, const ConvArgs& a, cudaStream_t st);
 
 // ---------------------------------------------------------------- sweep
 struct SweepHp {
