@@ -32,6 +32,8 @@ __device__ __forceinline__ float act_deriv(int act, float a) {
 //   L = mean[-log pi(a) Adv - eta H] + c_v mean[(G - V)^2] w.r.t. logits and value,
 //   Adv and G held constant.
 __global__ void __launch_bounds__(256) a2c_loss_kernel(LossArgs p) {
+    pdl_wait();
+    pdl_launch();
     const int agent = blockIdx.x;
     const int T = p.T, E = p.E, A = p.A, S = T * E;
     const float* logits = p.logits + (long)agent * p.B * A;
@@ -111,13 +113,15 @@ __global__ void __launch_bounds__(256) a2c_loss_kernel(LossArgs p) {
 }
 
 cudaError_t launch_a2c_loss(const LossArgs& a, int n_agents, cudaStream_t st) {
-    a2c_loss_kernel<<<n_agents, 256, 0, st>>>(a);
+    (void)launch_pdl(a2c_loss_kernel, dim3(n_agents), dim3(256), 0, st, a);
     return cudaGetLastError();
 }
 
 // Inverse-CDF draw: smallest k with sum_{j<=k} pi_j > u, clamped to A-1.
 __global__ void sample_kernel(const float* __restrict__ logits, const float* __restrict__ u,
                               int* __restrict__ actions, int E, int A) {
+    pdl_wait();
+    pdl_launch();
     int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= E) return;
     const float* z = logits + (long)e * A;
@@ -136,7 +140,7 @@ __global__ void sample_kernel(const float* __restrict__ logits, const float* __r
 }
 cudaError_t launch_sample(const float* logits, const float* uniforms, int* actions, int E, int A,
                           cudaStream_t st) {
-    sample_kernel<<<(E + 127) / 128, 128, 0, st>>>(logits, uniforms, actions, E, A);
+    (void)launch_pdl(sample_kernel, dim3((E + 127) / 128), dim3(128), 0, st, logits, uniforms, actions, E, A);
     return cudaGetLastError();
 }
 
@@ -144,6 +148,8 @@ cudaError_t launch_sample(const float* logits, const float* uniforms, int* actio
 // out[r][o] = act(sum_i in[r][i] W[o][i] + b[o]); one warp per output row r, lanes over o with
 // the input row staged in shared memory.
 __global__ void __launch_bounds__(256) dense_fwd_kernel(DenseArgs a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ float xin[];  // [warps][in_dim]
     const int g = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -167,7 +173,7 @@ cudaError_t launch_dense_fwd(const DenseArgs& a, int groups, cudaStream_t st) {
     int bx = (a.rows + 7) / 8;
     if (bx > 64) bx = 64;
     dim3 grid(bx, groups);
-    dense_fwd_kernel<<<grid, 256, 8 * a.in_dim * sizeof(float), st>>>(a);
+    (void)launch_pdl(dense_fwd_kernel, dim3(grid), dim3(256), 8 * a.in_dim * sizeof(float), st, a);
     return cudaGetLastError();
 }
 
@@ -176,6 +182,8 @@ cudaError_t launch_dense_fwd(const DenseArgs& a, int groups, cudaStream_t st) {
 // re-read from L2 with the full latency for every output); one warp per row, the dot products
 // are split over lanes and combined by a butterfly.
 __global__ void __launch_bounds__(256) heads_fwd_kernel(HeadsArgs a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ float hsm[];  // [A+1][H] weights, then [warps][H] rows
     const int g = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -211,12 +219,14 @@ cudaError_t launch_heads_fwd(const HeadsArgs& a, int groups, cudaStream_t st) {
         cudaError_t e = cudaFuncSetAttribute(heads_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    heads_fwd_kernel<<<dim3(bx, groups), 256, smem, st>>>(a);
+    (void)launch_pdl(heads_fwd_kernel, dim3(dim3(bx, groups)), dim3(256), smem, st, a);
     return cudaGetLastError();
 }
 
 // Heads backward, data part: dpre[s][j] = (sum_k dz[s][k] pi.W[k][j] + dv[s] v.W[j]) * act'(h[s][j]).
 __global__ void __launch_bounds__(256) heads_dgrad_kernel(HeadsBwdArgs a) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const float* P = a.params + (long)g * a.p_stride;
     const char* hbase = reinterpret_cast<const char*>(a.h) + (long)g * a.h_stride * (a.h_bf16 ? 2 : 4);
@@ -234,6 +244,8 @@ __global__ void __launch_bounds__(256) heads_dgrad_kernel(HeadsBwdArgs a) {
 // Heads backward, parameter part: d pi.W[k][j] = sum_s dz[s][k] h[s][j] (k = A: value head),
 // biases are the plain sums over s.  Serial over s: fixed summation order.
 __global__ void __launch_bounds__(256) heads_wgrad_kernel(HeadsBwdArgs a) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const char* hbase = reinterpret_cast<const char*>(a.h) + (long)g * a.h_stride * (a.h_bf16 ? 2 : 4);
     const float* dz = a.dlogits + (long)g * a.dlogits_stride;
@@ -262,16 +274,18 @@ cudaError_t launch_heads_bwd(const HeadsBwdArgs& a, int groups, cudaStream_t st)
     long total = (long)a.rows * a.H;
     int bx = (int)((total + 255) / 256);
     if (bx > 256) bx = 256;
-    heads_dgrad_kernel<<<dim3(bx, groups), 256, 0, st>>>(a);
+    (void)launch_pdl(heads_dgrad_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, a);
     long tw = (long)(a.A + 1) * (a.H + 1);
     int bw = (int)((tw + 255) / 256);
-    heads_wgrad_kernel<<<dim3(bw, groups), 256, 0, st>>>(a);
+    (void)launch_pdl(heads_wgrad_kernel, dim3(dim3(bw, groups)), dim3(256), 0, st, a);
     return cudaGetLastError();
 }
 
 // Dense layer backward (MLP trunk): gW[o][i] = sum_r dpre[r][o] in[r][i], gb[o] = sum_r dpre[r][o],
 // and (if din) din[r][i] = (sum_o dpre[r][o] W[o][i]) * act'(in[r][i]).
 __global__ void __launch_bounds__(256) dense_wgrad_kernel(DenseBwdArgs a) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const float* in = reinterpret_cast<const float*>(a.in.p[g]);
     const float* dp = a.dpre + (long)g * a.dpre_stride;
@@ -292,6 +306,8 @@ __global__ void __launch_bounds__(256) dense_wgrad_kernel(DenseBwdArgs a) {
     }
 }
 __global__ void __launch_bounds__(256) dense_dgrad_kernel(DenseBwdArgs a) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const float* in = reinterpret_cast<const float*>(a.in.p[g]);
     const float* dp = a.dpre + (long)g * a.dpre_stride;
@@ -309,12 +325,12 @@ cudaError_t launch_dense_bwd(const DenseBwdArgs& a, int groups, cudaStream_t st)
     long tw = (long)a.out_dim * (a.in_dim + 1);
     int bw = (int)((tw + 255) / 256);
     if (bw > 1024) bw = 1024;
-    dense_wgrad_kernel<<<dim3(bw, groups), 256, 0, st>>>(a);
+    (void)launch_pdl(dense_wgrad_kernel, dim3(dim3(bw, groups)), dim3(256), 0, st, a);
     if (a.din) {
         long td = (long)a.rows * a.in_dim;
         int bd = (int)((td + 255) / 256);
         if (bd > 1024) bd = 1024;
-        dense_dgrad_kernel<<<dim3(bd, groups), 256, 0, st>>>(a);
+        (void)launch_pdl(dense_dgrad_kernel, dim3(dim3(bd, groups)), dim3(256), 0, st, a);
     }
     return cudaGetLastError();
 }

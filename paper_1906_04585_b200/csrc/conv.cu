@@ -139,6 +139,15 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         issued_w = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (warp == 0 && u_begin < u_end) {
+        // The weights of the first agent are fetched before the wait for the previous kernel: they were
+        // written by the optimiser pass (or a state upload), which lies at least two kernels back.
+        __syncwarp();
+        if (lane == 0) { mbar_expect_tx(&w_full, (uint32_t)W_BYTES); issued_w = 1; }
+        __syncwarp();
+        const int group = p.group0 + decode_unit<V>(u_begin, p.rows).gz;
+        if (lane < T::W_BOXES) tma_load_3d(smW + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                      "r"(tmem_cols)
@@ -149,10 +158,13 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    pdl_wait();     // set-up above overlaps the previous kernel; its results are read from here on
+    pdl_launch();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
-        int it = 0, cur_g = -1, wl = 0;
+        int it = 0, wl = 1;
+        int cur_g = u_begin < u_end ? decode_unit<V>(u_begin, p.rows).gz : -1;   // already on its way
         for (int u = u_begin; u < u_end; u++, it++) {
             const UnitCoord c = decode_unit<V>(u, p.rows);
             const int group = p.group0 + c.gz;
@@ -458,7 +470,7 @@ static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, con
     if (units > 0x7fffffffL) return cudaErrorInvalidValue;
     const size_t smem = (size_t)fixed + (size_t)nst * STAGE;
     const int grid = (int)(units < 148 ? units : 148);
-    conv_resident_kernel<V><<<grid, 320, smem, st>>>(x, w, a, nst, units);
+    (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), dim3(320), smem, st, x, w, a, nst, units);
     return cudaGetLastError();
 }
 

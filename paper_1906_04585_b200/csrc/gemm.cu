@@ -111,6 +111,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    pdl_wait();     // set-up above overlaps the previous kernel; its results are read from here on
+    pdl_launch();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -493,6 +495,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partials, float* __restrict__ out,
                                                             long count, int split_k, long split_stride,
                                                             long partial_group_stride, long out_group_stride) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const float* pg = partials + (long)g * partial_group_stride;
     float* og = out + (long)g * out_group_stride;
@@ -508,6 +512,8 @@ __global__ void __launch_bounds__(256) splitk_reduce_act_kernel(const float* __r
                                                                 long bias_group_stride, int group0, long count, int N,
                                                                 int split_k, long split_stride, long partial_group_stride,
                                                                 long out_group_stride) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const float4* pg = reinterpret_cast<const float4*>(partials + (long)g * partial_group_stride);
     const float* bg = bias + (long)(group0 + g) * bias_group_stride;
@@ -534,7 +540,7 @@ cudaError_t launch_splitk_reduce_act(const float* partials, __nv_bfloat16* out, 
         return cudaErrorInvalidValue;
     int bx = (int)((count / 4 + 255) / 256);
     if (bx > 148 * 4) bx = 148 * 4;
-    splitk_reduce_act_kernel<<<dim3(bx, groups), 256, 0, st>>>(partials, out, bias, bias_group_stride, group0, count, N,
+    (void)launch_pdl(splitk_reduce_act_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, partials, out, bias, bias_group_stride, group0, count, N,
                                                                split_k, split_stride, partial_group_stride, out_group_stride);
     return cudaGetLastError();
 }
@@ -543,7 +549,7 @@ cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, 
                                  int groups, long partial_group_stride, long out_group_stride, cudaStream_t st) {
     int bx = (int)((count + 255) / 256);
     if (bx > 148 * 4) bx = 148 * 4;
-    splitk_reduce_kernel<<<dim3(bx, groups), 256, 0, st>>>(partials, out, count, split_k, split_stride,
+    (void)launch_pdl(splitk_reduce_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, partials, out, count, split_k, split_stride,
                                                            partial_group_stride, out_group_stride);
     return cudaGetLastError();
 }
@@ -683,7 +689,7 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     if (per_sm < 1) per_sm = 1;
     const long cap = 148L * per_sm;
     const int grid = (int)(total < cap ? total : cap);
-    gemm_tcgen05_kernel<<<grid, 192, smem, st>>>(A.map, B.map, a, A.mn_major, B.mn_major, total, mt, nt);
+    (void)launch_pdl(gemm_tcgen05_kernel, dim3(grid), dim3(192), smem, st, A.map, B.map, a, A.mn_major, B.mn_major, total, mt, nt);
     return cudaGetLastError();
 }
 

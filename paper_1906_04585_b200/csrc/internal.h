@@ -12,6 +12,28 @@
 
 namespace gala {
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Kernels of the learner step are launched so that a kernel may become resident while its predecessor
+// in the stream is still running.  A kernel first does the set-up that touches no data of the step
+// (barriers, tensor memory, descriptor prefetch), then waits for the predecessor to complete and its
+// writes to be visible (pdl_wait), then lets its own successor start (pdl_launch).  Because the trigger
+// comes after the wait, at most two consecutive kernels overlap: what a kernel reads before pdl_wait
+// must have been written at least two kernels earlier.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---------------------------------------------------------------- network layout
 // Offsets (in floats) of every tensor inside one agent's flat vector.
 struct ConvLayout {

@@ -10,6 +10,8 @@ namespace gala {
 // contraction).  16 bytes in, 32 bytes out per thread and step.
 __global__ void __launch_bounds__(256) cast_frames_kernel(PtrBatch obs, __nv_bfloat16* __restrict__ out, long out_group_stride,
                                                           long n16) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const uint4* src = reinterpret_cast<const uint4*>(obs.p[g]);
     uint4* dst = reinterpret_cast<uint4*>(out + (long)g * out_group_stride);
@@ -33,7 +35,7 @@ cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out
     const long n16 = (long)samples * (84 * 84 * 4 / 16);
     int bx = (int)((n16 + 255) / 256);
     if (bx > 148 * 8) bx = 148 * 8;
-    cast_frames_kernel<<<dim3(bx, groups), 256, 0, st>>>(obs, out, out_group_stride, n16);
+    (void)launch_pdl(cast_frames_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, obs, out, out_group_stride, n16);
     return cudaGetLastError();
 }
 
@@ -45,6 +47,8 @@ cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out
 // Up to kColsumJobs tensors are reduced by one launch (blockIdx.z picks the tensor).
 __global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, float* __restrict__ out_base, long out_group_stride,
                                                      double* partial_base, unsigned* ticket_base) {
+    pdl_wait();
+    pdl_launch();
     const int g = blockIdx.y;
     const ColsumJob job = jobs.j[blockIdx.z];
     const long rows = job.rows;
@@ -108,7 +112,7 @@ cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, l
         const int C = jobs.j[i].C;
         if (C > 512 || C < 8 || (C & (C - 1))) return cudaErrorInvalidValue;
     }
-    colsum_kernel<<<dim3(kColsumChunks, groups, n_jobs), 256, 0, st>>>(jobs, out_base, out_group_stride, partial, ticket);
+    (void)launch_pdl(colsum_kernel, dim3(dim3(kColsumChunks, groups, n_jobs)), dim3(256), 0, st, jobs, out_base, out_group_stride, partial, ticket);
     return cudaGetLastError();
 }
 

@@ -46,6 +46,8 @@ __global__ void __launch_bounds__(256) sweep_agent_kernel(float* __restrict__ x,
                                                           const float* __restrict__ clip,
                                                           __nv_bfloat16* __restrict__ shadow, long n4,
                                                           SweepHp hp) {
+    pdl_wait();
+    pdl_launch();
     const float c = clip ? *clip : 1.0f;
     const float w = 1.0f / (1.0f + P);
     for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x) {
@@ -80,11 +82,11 @@ cudaError_t launch_sweep_agent(float* x, const float* g, float* v, float* snap_o
     if (grid > 148 * 8) grid = 148 * 8;
     if (grid < 1) grid = 1;
     if (n_peers == 0)
-        sweep_agent_kernel<0><<<grid, 256, 0, st>>>(x, g, v, snap_out, nullptr, nullptr, clip, shadow, n4, hp);
+        (void)launch_pdl(sweep_agent_kernel<0>, dim3(grid), dim3(256), 0, st, x, g, v, snap_out, nullptr, nullptr, clip, shadow, n4, hp);
     else if (n_peers == 1)
-        sweep_agent_kernel<1><<<grid, 256, 0, st>>>(x, g, v, snap_out, peer0, nullptr, clip, shadow, n4, hp);
+        (void)launch_pdl(sweep_agent_kernel<1>, dim3(grid), dim3(256), 0, st, x, g, v, snap_out, peer0, nullptr, clip, shadow, n4, hp);
     else
-        sweep_agent_kernel<2><<<grid, 256, 0, st>>>(x, g, v, snap_out, peer0, peer1, clip, shadow, n4, hp);
+        (void)launch_pdl(sweep_agent_kernel<2>, dim3(grid), dim3(256), 0, st, x, g, v, snap_out, peer0, peer1, clip, shadow, n4, hp);
     return cudaGetLastError();
 }
 
@@ -100,6 +102,8 @@ template <int P>
 __global__ void sweep_sync_kernel(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ v,
                                   const float* __restrict__ clip, __nv_bfloat16* __restrict__ shadow,
                                   int n_agents, long d_pad, long n4, int off0, int off1, SweepHp hp) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ float4 ysm[];  // [n_agents][blockDim.x]
     const float w = 1.0f / (1.0f + P);
     for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x) {
@@ -182,7 +186,7 @@ cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* c
 #define GALA_SYNC_LAUNCH(P)                                                                          \
     e = cudaFuncSetAttribute(sweep_sync_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
     if (e != cudaSuccess) return e;                                                                  \
-    sweep_sync_kernel<P><<<grid, threads, smem, st>>>(x, g, v, clip, shadow, n_agents, d_pad, n4, o0, o1, hp);
+    (void)launch_pdl(sweep_sync_kernel<P>, dim3(grid), dim3(threads), smem, st, x, g, v, clip, shadow, n_agents, d_pad, n4, o0, o1, hp);
     if (n_peers == 0) { GALA_SYNC_LAUNCH(0) }
     else if (n_peers == 1) { GALA_SYNC_LAUNCH(1) }
     else if (n_peers == 2) { GALA_SYNC_LAUNCH(2) }
@@ -198,6 +202,8 @@ cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* c
 __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict__ g, long d, long d_pad,
                                                         int agent0, float max_norm, double* partial,
                                                         unsigned* ticket, float* norm, float* clip) {
+    pdl_wait();
+    pdl_launch();
     const int agent = agent0 + blockIdx.y;
     const float* ga = g + (long)agent * d_pad;
     // chunks are multiples of 4 floats and the padding [d, d_pad) is zero: 16-byte loads throughout
@@ -241,7 +247,7 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
                              double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st) {
     dim3 grid(kNormChunks, n_agents);
-    grad_norm_kernel<<<grid, 256, 0, st>>>(g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip);
+    (void)launch_pdl(grad_norm_kernel, dim3(grid), dim3(256), 0, st, g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip);
     return cudaGetLastError();
 }
 
@@ -249,6 +255,8 @@ cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int
 // before each update): every agent's gradient row is replaced by the mean over agents, summed in
 // agent order.  One thread per 16-byte column; reads N*d, writes N*d.
 __global__ void __launch_bounds__(256) allreduce_grads_kernel(float* __restrict__ g, int n_agents, long d_pad, long n4) {
+    pdl_wait();
+    pdl_launch();
     const float inv = 1.0f / (float)n_agents;
     for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -264,7 +272,7 @@ cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStrea
     const long n4 = d_pad / 4;
     int grid = (int)((n4 + 255) / 256);
     if (grid > 148 * 8) grid = 148 * 8;
-    allreduce_grads_kernel<<<grid, 256, 0, st>>>(g, n_agents, d_pad, n4);
+    (void)launch_pdl(allreduce_grads_kernel, dim3(grid), dim3(256), 0, st, g, n_agents, d_pad, n4);
     return cudaGetLastError();
 }
 
@@ -275,6 +283,8 @@ cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStrea
 constexpr int kConsensusBlocks = 592;
 __global__ void __launch_bounds__(256) consensus_kernel(const float* __restrict__ x, int n_agents, long d, long d_pad,
                                                         double* partial, unsigned* ticket, double* out) {
+    pdl_wait();
+    pdl_launch();
     double acc = 0.0;
     for (long c = blockIdx.x * (long)blockDim.x + threadIdx.x; c < d; c += (long)gridDim.x * blockDim.x) {
         double s = 0.0, ss = 0.0;
@@ -309,13 +319,15 @@ __global__ void __launch_bounds__(256) consensus_kernel(const float* __restrict_
 }
 cudaError_t launch_consensus(const float* x, int n_agents, long d, long d_pad, double* partial, unsigned* ticket,
                              double* out, cudaStream_t st) {
-    consensus_kernel<<<kConsensusBlocks, 256, 0, st>>>(x, n_agents, d, d_pad, partial, ticket, out);
+    (void)launch_pdl(consensus_kernel, dim3(kConsensusBlocks), dim3(256), 0, st, x, n_agents, d, d_pad, partial, ticket, out);
     return cudaGetLastError();
 }
 
 // Straggler injection: occupies the stream for about `usec` microseconds (one sleeping thread).
 // Bounded twice: by the requested time (capped by the caller) and by an iteration limit.
 __global__ void delay_kernel(unsigned long long usec) {
+    pdl_wait();
+    pdl_launch();
     unsigned long long t0, t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
     for (int i = 0; i < 2000000; i++) {
@@ -325,11 +337,13 @@ __global__ void delay_kernel(unsigned long long usec) {
     }
 }
 cudaError_t launch_delay(unsigned long long usec, cudaStream_t st) {
-    delay_kernel<<<1, 1, 0, st>>>(usec);
+    (void)launch_pdl(delay_kernel, dim3(1), dim3(1), 0, st, usec);
     return cudaGetLastError();
 }
 
 __global__ void cast_bf16_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ out, long n4) {
+    pdl_wait();
+    pdl_launch();
     for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n4; i += (long)gridDim.x * blockDim.x)
         st_bf16x4(out + i * 4, *reinterpret_cast<const float4*>(x + i * 4));
 }
@@ -338,7 +352,7 @@ cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cud
     int grid = (int)((n4 + 255) / 256);
     if (grid > 148 * 8) grid = 148 * 8;
     if (grid < 1) grid = 1;
-    cast_bf16_kernel<<<grid, 256, 0, st>>>(x, out, n4);
+    (void)launch_pdl(cast_bf16_kernel, dim3(grid), dim3(256), 0, st, x, out, n4);
     return cudaGetLastError();
 }
 

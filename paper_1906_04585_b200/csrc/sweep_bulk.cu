@@ -100,6 +100,8 @@ sweep_sync_bulk_kernel(const __grid_constant__ CUtensorMap mx, const __grid_cons
         for (int s = 0; s < kBulkStages; s++) { bar_init(&full[s], 1); bar_init(&done[s], kConsumers); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    pdl_wait();     // the gradients and clip factors come from the kernels before
+    pdl_launch();
     for (int a = threadIdx.x; a < n_agents; a += blockDim.x) clip_s[a] = clip ? clip[a] : 1.0f;
     __syncthreads();
 
@@ -222,7 +224,7 @@ cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const flo
 #define GALA_BULK_LAUNCH(P)                                                                                  \
     e = cudaFuncSetAttribute(sweep_sync_bulk_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
     if (e != cudaSuccess) return e;                                                                          \
-    sweep_sync_bulk_kernel<P><<<grid, kConsumers + 32, smem, st>>>(mx, mg, mv, clip, shadow, n_agents, d_pad, cols, \
+    (void)launch_pdl(sweep_sync_bulk_kernel<P>, dim3(grid), dim3(kConsumers + 32), smem, st, mx, mg, mv, clip, shadow, n_agents, d_pad, cols, \
                                                                    stages, n_tiles, o0, o1, hp, error_word);
     if (n_peers == 0) { GALA_BULK_LAUNCH(0) }
     else if (n_peers == 1) { GALA_BULK_LAUNCH(1) }
