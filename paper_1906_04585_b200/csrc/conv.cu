@@ -25,12 +25,13 @@
 //          view of tap (a, b) = (ky / 2, kx / 2) and differ only in the weight block, so they become
 //          the N = 4 x 32 columns of one product: shift (1 - a) * 11 + (1 - b)
 //
-// One CTA (320 threads, persistent over a contiguous range of work units):
+// One CTA (352 threads, persistent over a contiguous range of work units):
 //   warp 0    TMA producer: input planes of the next units into a ring of stages; the agent's weights
 //             whenever the agent changes
-//   warp 1    MMA issuer (one thread): taps x K-chunks tcgen05.mma per unit into one of two
-//             tensor-memory accumulators
-//   warps 2-9 two epilogue groups of four warps, one per accumulator buffer: tcgen05.ld (a thread owns a
+//   warps 1, 10  two MMA issuers (one thread each) that take the units alternately, each with its own
+//             tensor-memory accumulator: taps x K-chunks tcgen05.mma per unit.  While one waits for the
+//             barriers of its next unit, the tensor pipe works on the other's MMAs.
+//   warps 2-9 two epilogue groups of four warps, one per issuer (two accumulator buffers each): tcgen05.ld (a thread owns a
 //             pixel), scale / bias / ReLU (+ gate bits) or the ReLU gate, 64 contiguous bytes of bf16 per 32 columns
 // Every wait is bounded; when one runs out the CTA raises the caller's error word, lets the copies it
 // issued land, frees its tensor memory and returns.
@@ -102,7 +103,7 @@ template <int V> __device__ __forceinline__ UnitCoord decode_unit(int u, int row
 }
 
 template <int V>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(352, 1)
 conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const ConvArgs p,
                      const int nst, const long total_units) {
     using T = ConvTraits<V>;
@@ -111,9 +112,9 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kConvMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kConvMaxStages];
-    __shared__ __align__(8) uint64_t acc_full[2];
-    __shared__ __align__(8) uint64_t acc_empty[2];
-    __shared__ __align__(8) uint64_t w_full;
+    __shared__ __align__(8) uint64_t acc_full[4];
+    __shared__ __align__(8) uint64_t acc_empty[4];
+    __shared__ __align__(8) uint64_t w_full, w_empty;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int issued_iters, issued_w;
@@ -124,7 +125,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     uint8_t* smE = smX + nst * STAGE + kConvSlack;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr uint32_t tmem_cols = 2u * T::BN;   // 64, 128 or 256
+    constexpr uint32_t tmem_cols = 4u * T::BN;   // 128, 256 or 512: two accumulators per issuer
 
     // contiguous range of units of this CTA: at most a few agents, so few weight reloads
     const int u_begin = (int)(total_units * blockIdx.x / gridDim.x);
@@ -132,8 +133,9 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        for (int b = 0; b < 4; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
         mbar_init(&w_full, 1);
+        mbar_init(&w_empty, 2);
         abort_flag = 0;
         issued_iters = 0;
         issued_w = 0;
@@ -169,10 +171,10 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const UnitCoord c = decode_unit<V>(u, p.rows);
             const int group = p.group0 + c.gz;
             if (c.gz != cur_g) {
-                // new agent: its weights replace the previous agent's once every MMA that read those is done
+                // new agent: its weights replace the previous agent's once both issuers have signalled that
+                // every MMA that read those is done
                 int go = 1;
-                if (lane == 0 && it > 0)
-                    go = mbar_wait(&empty_bar[(it - 1) % nst], (uint32_t)((it - 1) / nst) & 1u, &abort_flag) ? 1 : 0;
+                if (lane == 0) go = mbar_wait(&w_empty, (uint32_t)(wl - 1) & 1u, &abort_flag) ? 1 : 0;
                 go = __shfl_sync(0xffffffffu, go, 0);
                 if (!go) break;
                 if (lane == 0) mbar_expect_tx(&w_full, (uint32_t)W_BYTES);
@@ -202,21 +204,27 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             __syncwarp();
             if (lane == 0) issued_iters = it + 1;
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == 10) {
+        // ------------------------------------------------ MMA issuers: warp 1 takes the even units, warp 10 the odd
         if (lane == 0) {
+            const int ii = warp == 1 ? 0 : 1;
             const uint32_t idesc = make_instr_desc(T::BN, 0, T::B_MN);
             const uint64_t bd_base = make_smem_desc_raw(smem_u32(smW), T::B_LAYOUT, T::B_SBO, T::B_LBO);
             int it = 0, cur_g = -1, wl = 0;
             for (int u = u_begin; u < u_end; u++, it++) {
-                const UnitCoord c = decode_unit<V>(u, p.rows);
-                if (c.gz != cur_g) {
+                // Both issuers follow every change of agent: each reports (through a commit, so only once its
+                // MMAs are complete) that it is done with the old weights, then waits for the new ones.
+                const int gz = (u / T::UPS) / p.rows;
+                if (gz != cur_g) {
+                    if (cur_g >= 0) umma_commit(&w_empty);
                     if (!mbar_wait(&w_full, (uint32_t)wl & 1u, &abort_flag)) break;
                     wl++;
-                    cur_g = c.gz;
+                    cur_g = gz;
                 }
-                const int ab = it & 1;
-                if (!mbar_wait(&acc_empty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, &abort_flag)) break;
+                if ((it & 1) != ii) continue;
+                const int k = it >> 1;                  // this issuer's k-th unit goes to its buffer k % 2
+                const int ab = ii * 2 + (k & 1);
+                if (!mbar_wait(&acc_empty[ab], (((uint32_t)k >> 1) & 1u) ^ 1u, &abort_flag)) break;
                 const int s = it % nst;
                 if (!mbar_wait(&full_bar[s], (uint32_t)(it / nst) & 1u, &abort_flag)) break;
                 tcgen05_fence_after();
@@ -245,7 +253,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             }
         }
     } else {
-        // ------------------------------------------------ epilogue: group eg owns accumulator buffer eg
+        // ------------------------------------------------ epilogue: group eg drains the accumulators of issuer eg
         // A thread owns one row of the tile (one pixel): per 32-column block it reads its 32 accumulators
         // from tensor memory, applies scale / bias / ReLU or the ReLU gate, and stores 64 contiguous bytes.
         // The gate values depend only on the unit, so they are fetched before the wait for the MMAs.
@@ -313,10 +321,11 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             } else {
                 load_gates(u + 2, gate_next);
             }
-            if (!mbar_wait(&acc_full[eg], ((uint32_t)it >> 1) & 1u, &abort_flag)) break;
+            const int ab = eg * 2 + ((it >> 1) & 1);
+            if (!mbar_wait(&acc_full[ab], ((uint32_t)it >> 2) & 1u, &abort_flag)) break;
             tcgen05_fence_after();
             if (q * 32 <= kLastRow) {
-                const uint32_t tmem_acc = tmem_base + (uint32_t)eg * T::BN + ((uint32_t)(q * 32) << 16);
+                const uint32_t tmem_acc = tmem_base + (uint32_t)ab * T::BN + ((uint32_t)(q * 32) << 16);
 #pragma unroll
                 for (int ch = 0; ch < NCH; ch++) {
                     uint32_t r[32];
@@ -355,7 +364,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             }
             // this warp no longer reads the accumulator buffer
             tcgen05_fence_before();
-            if (lane == 0) mbar_arrive(&acc_empty[eg]);
+            if (lane == 0) mbar_arrive(&acc_empty[ab]);
         }
     }
 
@@ -470,7 +479,7 @@ static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, con
     if (units > 0x7fffffffL) return cudaErrorInvalidValue;
     const size_t smem = (size_t)fixed + (size_t)nst * STAGE;
     const int grid = (int)(units < 148 ? units : 148);
-    (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), dim3(320), smem, st, x, w, a, nst, units);
+    (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), dim3(352), smem, st, x, w, a, nst, units);
     return cudaGetLastError();
 }
 
