@@ -39,6 +39,11 @@ struct Plan {  // one tensor-core product with its descriptors
     GemmArgs args;
     int tag = 0;
 };
+struct WgradPlan {  // conv2 / conv3 weight gradient with resident operands
+    CUtensorMap x, y;
+    WgradArgs args;
+    int tag = 0;
+};
 struct ConvPlan {  // one forward or data-gradient convolution (input resident in shared memory)
     CUtensorMap x, w;
     ConvArgs args;
@@ -116,6 +121,7 @@ struct gala_ctx {
     int max_split = 32;
     Plan fwd[3], fc_fwd, fc_wgrad, fc_dgrad, wgrad[3], dgrad[3];
     ConvPlan cfwd[3], cdgrad[3];
+    WgradPlan cwgrad[3];
     uint32_t* gate[2] = {nullptr, nullptr};   // ReLU gate bits of act[0], act[1]
     bool legacy_conv = false;
 };
@@ -403,6 +409,14 @@ int build_plans(gala_ctx* c) {
         ok &= make_conv_maps(f.args.variant, &f.x, &f.w, xin, (uint64_t)n * B, c->shadow + c->cl.w[l], n, dp);
         f.built = true;
         if (l > 0) {
+            WgradPlan& wg = c->cwgrad[l];
+            memset(&wg.args, 0, sizeof wg.args);
+            wg.tag = T_GEMM_CONV_WGRAD + l;
+            wg.args.variant = l == 1 ? WG_CONV2 : WG_CONV3;
+            wg.args.x_samples = (int)B; wg.args.y_samples = (int)S; wg.args.samples = (int)S;
+            wg.args.out = c->g + c->cl.w[l]; wg.args.out_group_stride = dp;
+            wg.args.error_word = c->error_word;
+            ok &= make_wgrad_maps(wg.args.variant, &wg.x, &wg.y, c->act[l - 1], (uint64_t)n * B, c->dy[l], (uint64_t)n * S);
             ConvPlan& d = c->cdgrad[l];
             memset(&d.args, 0, sizeof d.args);
             d.tag = T_GEMM_CONV_DGRAD + l;
@@ -418,6 +432,36 @@ int build_plans(gala_ctx* c) {
         }
     }
     return ok ? GALA_OK : fail(c, GALA_ECUDA, "cuTensorMapEncodeTiled failed while building GEMM descriptors");
+}
+
+// conv2 / conv3 weight gradient: slices of the samples per agent chosen so that the CTAs fill the SMs in
+// whole waves; with more than one slice the partial sums go through the fixed-order reduction
+int run_conv_wgrad(gala_ctx* c, const WgradPlan& p, int agent0, int groups, cudaStream_t st) {
+    WgradArgs a = p.args;
+    const int S = a.samples;
+    const long count = (long)(a.variant == WG_CONV2 ? 64 * 512 : 64 * 576);
+    int best = 1;
+    long best_cost = -1;
+    for (int sp = 1; sp <= c->max_split && sp <= S; sp++) {
+        if (sp > 1 && (S / sp < 4 || sp * count > c->splitk_group_stride)) break;
+        const long waves = ((long)groups * sp + 147) / 148, per = (S + sp - 1) / sp;
+        const long cost = waves * (per + 6) + (sp > 1 ? 8 : 0);   // samples per CTA plus fixed costs, in sample units
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = sp; }
+    }
+    a.group0 = agent0; a.groups = groups; a.splits = best;
+    if (best == 1) {
+        a.out += (long)agent0 * a.out_group_stride;
+        a.out_split_stride = 0;
+        LAUNCH(p.tag, st, launch_wgrad(p.x, p.y, a, st));
+        return GALA_OK;
+    }
+    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+    a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
+    LAUNCH(p.tag, st, launch_wgrad(p.x, p.y, a, st));
+    LAUNCH(T_SPLITK, st, launch_splitk_reduce(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
+                                p.args.out + (long)agent0 * p.args.out_group_stride, count, best, count, groups,
+                                c->splitk_group_stride, p.args.out_group_stride, st));
+    return GALA_OK;
 }
 
 int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, cudaStream_t st) {
@@ -586,7 +630,9 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
         for (int l = 2; l >= 0; l--) {
             if ((r = fork()) != GALA_OK) return r;
-            if ((r = run_wgrad(c, c->wgrad[l], agent0, groups, ws)) != GALA_OK) return r;
+            r = (l > 0 && !c->legacy_conv) ? run_conv_wgrad(c, c->cwgrad[l], agent0, groups, ws)
+                                           : run_wgrad(c, c->wgrad[l], agent0, groups, ws);
+            if (r != GALA_OK) return r;
             if (l > 0) {
                 r = c->legacy_conv ? run_plan(c, c->dgrad[l], agent0, groups, 0, st)
                                    : run_conv(c, c->cdgrad[l], agent0, groups, (int)S, st);
@@ -854,6 +900,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         const int P[3] = {400, 81, 49};
         CK(gemm_init());
         CK(conv_init());
+        CK(wgrad_init());
         c->legacy_conv = getenv("GALA_CONV_LEGACY") != nullptr;
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);

@@ -168,6 +168,24 @@ bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const v
                     const void* w_base, uint64_t groups, uint64_t w_group_stride_elems);
 cudaError_t launch_conv(const CUtensorMap& x, const CUtensorMap& w, const ConvArgs& a, cudaStream_t st);
 
+// ---------------------------------------------------------------- conv weight gradients, resident operands
+// conv2 / conv3 weight gradients (wgrad.cu): x = the layer's input activation, y = dY of the layer.
+enum WgradVariant : int { WG_CONV2 = 1, WG_CONV3 = 2 };
+struct WgradArgs {
+    int variant;
+    int groups, group0;    // agents of this launch
+    int splits;            // CTAs per agent, each takes a slice of the samples
+    int samples;           // samples per agent to reduce over
+    int x_samples, y_samples;   // samples per agent in the two tensors
+    float* out;            // agent i, slice s at out + i * out_group_stride + s * out_split_stride, as W[co][KK]
+    long out_group_stride, out_split_stride;
+    int* error_word;
+};
+cudaError_t wgrad_init();
+bool make_wgrad_maps(int variant, CUtensorMap* x_map, CUtensorMap* y_map, const void* x_base, uint64_t x_samples,
+                     const void* y_base, uint64_t y_samples);
+cudaError_t launch_wgrad(const CUtensorMap& x, const CUtensorMap& y, const WgradArgs& a, cudaStream_t st);
+
 // ---------------------------------------------------------------- sweep
 struct SweepHp {
     float lr, alpha, eps;
