@@ -104,7 +104,7 @@ typedef struct {
 
 /* One agent's rollout {(s_t, a_t, r_t, s_{t+1})} (Algorithm 1, acting step). DEVICE pointers. */
 typedef struct {
-    const void* obs;            /* [T+1][E][84][84][4] uint8  or  [T+1][E][obs_dim] float32 */
+    const void* obs;            /* [T+1][E][84][84][4] uint8 (16-byte aligned)  or  [T+1][E][obs_dim] float32 */
     const int* actions;         /* [T][E], each in [0, n_actions) */
     const float* rewards;       /* [T][E] */
     const unsigned char* dones; /* [T][E]; 1 = the episode ended at this step */

@@ -464,8 +464,10 @@ int run_conv_wgrad(gala_ctx* c, const WgradPlan& p, int agent0, int groups, cuda
     return GALA_OK;
 }
 
-int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, cudaStream_t st) {
+int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, cudaStream_t st,
+             const PtrBatch* obs = nullptr) {
     ConvArgs a = p.args;
+    if (obs) a.obs = *obs;
     a.group0 = agent0; a.groups = groups; a.rows = rows;
     a.out += (long)agent0 * a.out_group_stride;
     if (a.gate_out) a.gate_out += (long)agent0 * a.gate_group_stride;
@@ -513,10 +515,13 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
     const long dp = c->d_pad, B = c->B;
     if (c->conv) {
         const int P[3] = {400, 81, 49};
+        for (int i = 0; i < groups; i++)
+            if (reinterpret_cast<uintptr_t>(obs.p[i]) & 15)
+                return fail(c, GALA_EINVAL, "uint8 observations must be 16-byte aligned");
         LAUNCH(T_CAST_FRAMES, st, launch_cast_frames(obs, c->frames + (long)agent0 * B * kFramePix, B * kFramePix, rows, groups, st));
         for (int l = 0; l < 3; l++) {
             int r = c->legacy_conv ? run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st)
-                                   : run_conv(c, c->cfwd[l], agent0, groups, rows, st);
+                                   : run_conv(c, c->cfwd[l], agent0, groups, rows, st, l == 0 ? &obs : nullptr);
             if (r != GALA_OK) return r;
         }
         // hidden layer: with few rows there are only a handful of output tiles, each streaming 0.8 MB of

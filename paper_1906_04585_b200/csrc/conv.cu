@@ -71,6 +71,12 @@ constexpr int kConvMaxStages = 8;
 constexpr int kConvSlack = 8 * 1024;             // rows an MMA reads past the last plane of the ring
 constexpr int kConvEpiWarpBytes = 512;           // an epilogue warp's copy of the layer's bias
 constexpr int kConvSmemMax = 224 * 1024;
+// conv1 reads the uint8 frames themselves: the 24 input lines behind five output lines are one
+// contiguous piece of 24 * 84 * 4 bytes, staged as it is and widened to bf16 planes by four more warps
+constexpr int kU8Stages = 4;
+constexpr int kU8Bytes = 24 * 336;       // 8064
+constexpr int kU8Stride = 8192;
+constexpr int kConvThreads = 352, kConv1Threads = 352 + 128;
 
 // plane and row shift of a tap
 template <int V> __host__ __device__ constexpr void tap_view(int t, int& plane, int& shift) {
@@ -103,7 +109,7 @@ template <int V> __device__ __forceinline__ UnitCoord decode_unit(int u, int row
 }
 
 template <int V>
-__global__ void __launch_bounds__(352, 1)
+__global__ void __launch_bounds__(V == CV_CONV1_FWD ? kConv1Threads : kConvThreads, 1)
 conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const ConvArgs p,
                      const int nst, const long total_units) {
     using T = ConvTraits<V>;
@@ -115,6 +121,8 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     __shared__ __align__(8) uint64_t acc_full[4];
     __shared__ __align__(8) uint64_t acc_empty[4];
     __shared__ __align__(8) uint64_t w_full, w_empty;
+    __shared__ __align__(8) uint64_t u8_full[kU8Stages];
+    __shared__ __align__(8) uint64_t u8_empty[kU8Stages];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int issued_iters, issued_w;
@@ -123,6 +131,8 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     uint8_t* smW = smem;
     uint8_t* smX = smem + W_BYTES;
     uint8_t* smE = smX + nst * STAGE + kConvSlack;
+    uint8_t* smU = smE + 8 * kConvEpiWarpBytes;   // conv1 only: ring of uint8 line blocks
+    constexpr bool kU8 = V == CV_CONV1_FWD;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr uint32_t tmem_cols = 4u * T::BN;   // 128, 256 or 512: two accumulators per issuer
@@ -132,7 +142,9 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const int u_end = (int)(total_units * (blockIdx.x + 1) / gridDim.x);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        // conv1: a stage is filled by the four converting warps, otherwise by TMA (one arrival with a byte count)
+        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], kU8 ? 4 : 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kU8Stages; s++) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], 4); }
         for (int b = 0; b < 4; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
         mbar_init(&w_full, 1);
         mbar_init(&w_empty, 2);
@@ -185,6 +197,21 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 wl++;
                 if (lane == 0) issued_w = wl;
             }
+            if constexpr (kU8) {
+                // lines 20q .. 20q+23 of the frame, as stored: one bulk copy of 8064 bytes
+                const int su = it % kU8Stages;
+                int go = 1;
+                if (lane == 0) go = mbar_wait(&u8_empty[su], ((uint32_t)(it / kU8Stages) & 1u) ^ 1u, &abort_flag) ? 1 : 0;
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (!go) break;
+                if (lane == 0) {
+                    mbar_expect_tx(&u8_full[su], (uint32_t)kU8Bytes);
+                    const uint8_t* src = reinterpret_cast<const uint8_t*>(p.obs.p[c.gz]) + (long)c.s * (84 * 336) + c.q * (20 * 336);
+                    bulk_load_1d(smU + su * kU8Stride, src, (uint32_t)kU8Bytes, &u8_full[su]);
+                    issued_iters = it + 1;
+                }
+                continue;
+            }
             const int s = it % nst;
             int go = 1;
             if (lane == 0) go = mbar_wait(&empty_bar[s], ((uint32_t)(it / nst) & 1u) ^ 1u, &abort_flag) ? 1 : 0;
@@ -195,8 +222,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const int sample = group * p.a_samples + c.s;
             if (lane < T::PLANES) {
                 uint8_t* dst = smX + s * STAGE + lane * T::PLANE_STRIDE;
-                if constexpr (V == CV_CONV1_FWD) tma_load_5d(dst, &tmX, &full_bar[s], 0, 0, lane, 5 * c.q, sample);
-                else if constexpr (V == CV_CONV2_FWD) tma_load_5d(dst, &tmX, &full_bar[s], 32 * (lane & 1), 0, lane >> 1, 0, sample);
+                if constexpr (V == CV_CONV2_FWD) tma_load_5d(dst, &tmX, &full_bar[s], 32 * (lane & 1), 0, lane >> 1, 0, sample);
                 else if constexpr (V == CV_CONV3_FWD) tma_load_3d(dst, &tmX, &full_bar[s], 0, 0, sample);
                 else if constexpr (V == CV_CONV2_DGRAD) tma_load_4d(dst, &tmX, &full_bar[s], 0, -1, -1, sample);
                 else tma_load_4d(dst, &tmX, &full_bar[s], 0, -2, -2, sample);
@@ -250,6 +276,46 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 }
                 umma_commit(&empty_bar[s]);     // the stage may be refilled ...
                 umma_commit(&acc_full[ab]);     // ... and the accumulator read, once the MMAs above are done
+            }
+        }
+    } else if (warp >= 11) {
+        // ------------------------------------------------ conv1: uint8 lines -> bf16 phase planes
+        // Line yl of the block (y = 20q + yl) belongs to plane yl % 4, row (yl / 4) * 21 + xq for its 16-byte
+        // group xq (4 pixels x 4 channels); a row is 32 bytes of bf16 whose two halves swap when bit 7 of
+        // its address is set (32-byte swizzle).  0..255 are exact in bf16; 1/255 is applied after the MMAs.
+        if constexpr (kU8) {
+            const int ct = threadIdx.x - 11 * 32;   // 0..127
+            int it = 0;
+            for (int u = u_begin; u < u_end; u++, it++) {
+                const int su = it % kU8Stages, s = it % nst;
+                if (!mbar_wait(&u8_full[su], (uint32_t)(it / kU8Stages) & 1u, &abort_flag)) break;
+                if (!mbar_wait(&empty_bar[s], ((uint32_t)(it / nst) & 1u) ^ 1u, &abort_flag)) break;
+                const uint8_t* src = smU + su * kU8Stride;
+                uint8_t* dstage = smX + s * STAGE;
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const int ch = ct + k * 128;          // 16-byte group of the block, 504 in all
+                    if (ch < 24 * 21) {
+                        const int yl = ch / 21, xq = ch - yl * 21;
+                        const uint4 v = *reinterpret_cast<const uint4*>(src + ch * 16);
+                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                        uint32_t o[8];
+#pragma unroll
+                        for (int e = 0; e < 4; e++) {
+                            o[2 * e] = pack2((float)(w[e] & 255u), (float)((w[e] >> 8) & 255u));
+                            o[2 * e + 1] = pack2((float)((w[e] >> 16) & 255u), (float)(w[e] >> 24));
+                        }
+                        const int r = (yl >> 2) * 21 + xq;
+                        uint8_t* row = dstage + (yl & 3) * T::PLANE_STRIDE + r * 32;
+                        const int sw = ((r >> 2) & 1) * 16;
+                        *reinterpret_cast<uint4*>(row + sw) = make_uint4(o[0], o[1], o[2], o[3]);
+                        *reinterpret_cast<uint4*>(row + (sw ^ 16)) = make_uint4(o[4], o[5], o[6], o[7]);
+                    }
+                }
+                // make the generic-proxy writes visible to the tensor core's reads, then hand the stage over
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(&full_bar[s]); mbar_arrive(&u8_empty[su]); }
             }
         }
     } else {
@@ -376,11 +442,12 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if (p.error_word) atomicExch(p.error_word, 1);
             // let copies that were already issued land before the shared memory goes away
             const int issued = issued_iters;
-            for (int it = max(0, issued - nst); it < issued; it++) {
-                const int s = it % nst;
-                const uint32_t ph = (uint32_t)(it / nst) & 1u;
+            const int ring = kU8 ? kU8Stages : nst;
+            for (int it = max(0, issued - ring); it < issued; it++) {
+                const int s = it % ring;
+                const uint32_t ph = (uint32_t)(it / ring) & 1u;
                 for (uint32_t i = 0; i < (1u << 16); i++) {
-                    if (mbar_try_wait(&full_bar[s], ph)) break;
+                    if (mbar_try_wait(kU8 ? &u8_full[s] : &full_bar[s], ph)) break;
                     __nanosleep(64);
                 }
             }
@@ -470,7 +537,8 @@ template <int V>
 static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, const ConvArgs& a, cudaStream_t st) {
     using T = ConvTraits<V>;
     constexpr int STAGE = T::PLANES * T::PLANE_STRIDE;
-    constexpr int fixed = T::W_BOXES * T::W_BOX_BYTES + kConvSlack + 8 * kConvEpiWarpBytes + 1024;
+    constexpr int fixed = T::W_BOXES * T::W_BOX_BYTES + kConvSlack + 8 * kConvEpiWarpBytes + 1024 +
+                          (V == CV_CONV1_FWD ? kU8Stages * kU8Stride : 0);
     int nst = (kConvSmemMax - fixed) / STAGE;
     if (nst > kConvMaxStages) nst = kConvMaxStages;
     if (nst < 2) return cudaErrorInvalidValue;
@@ -479,7 +547,7 @@ static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, con
     if (units > 0x7fffffffL) return cudaErrorInvalidValue;
     const size_t smem = (size_t)fixed + (size_t)nst * STAGE;
     const int grid = (int)(units < 148 ? units : 148);
-    (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), dim3(352), smem, st, x, w, a, nst, units);
+    (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), dim3(V == CV_CONV1_FWD ? kConv1Threads : kConvThreads), smem, st, x, w, a, nst, units);
     return cudaGetLastError();
 }
 

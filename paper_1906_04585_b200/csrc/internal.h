@@ -141,6 +141,10 @@ cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, 
                                  long split_stride, int groups, long partial_group_stride,
                                  long out_group_stride, cudaStream_t st);
 
+// Caller-owned per-agent pointers travel in kernel parameters, at most kBatch agents a launch.
+constexpr int kBatch = 64;
+struct PtrBatch { const void* p[kBatch]; };
+
 // ---------------------------------------------------------------- convolutions with a resident input
 // Forward and data-gradient convolutions of the trunk (conv.cu).  Tensors are NHWC bf16; weights
 // W[co][(ky, kx, ci)] bf16; group g (agent) uses sample block g * a_samples.. of the input tensor.
@@ -162,6 +166,7 @@ struct ConvArgs {
     const uint32_t* gate_in;
     long gate_group_stride;      // words per agent
     int* error_word;
+    PtrBatch obs;          // conv1 forward: the agents' uint8 frames [rows][84][84][4], 16-byte aligned
 };
 cudaError_t conv_init();
 bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const void* x_base, uint64_t samples,
@@ -215,9 +220,6 @@ cudaError_t launch_delay(unsigned long long usec, cudaStream_t st);
 cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st);
 
 // ---------------------------------------------------------------- A2C pieces
-// Caller-owned per-agent pointers travel in kernel parameters, at most kBatch agents a launch.
-constexpr int kBatch = 64;
-struct PtrBatch { const void* p[kBatch]; };
 
 struct LossArgs {
     int T, E, A;
