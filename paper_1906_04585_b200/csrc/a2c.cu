@@ -270,11 +270,14 @@ __global__ void __launch_bounds__(256) heads_wgrad_kernel(HeadsBwdArgs a) {
         }
     }
 }
-cudaError_t launch_heads_bwd(const HeadsBwdArgs& a, int groups, cudaStream_t st) {
+cudaError_t launch_heads_dgrad(const HeadsBwdArgs& a, int groups, cudaStream_t st) {
     long total = (long)a.rows * a.H;
     int bx = (int)((total + 255) / 256);
     if (bx > 256) bx = 256;
     (void)launch_pdl(heads_dgrad_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, a);
+    return cudaGetLastError();
+}
+cudaError_t launch_heads_wgrad(const HeadsBwdArgs& a, int groups, cudaStream_t st) {
     long tw = (long)(a.A + 1) * (a.H + 1);
     int bw = (int)((tw + 255) / 256);
     (void)launch_pdl(heads_wgrad_kernel, dim3(dim3(bw, groups)), dim3(256), 0, st, a);

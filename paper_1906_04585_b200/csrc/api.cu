@@ -511,14 +511,18 @@ int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t s
 
 // ------------------------------------------------------------------ forward / backward
 // Forward on `rows` observations per agent for agents [agent0, agent0+groups).
-int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, cudaStream_t st) {
+// frames_st: stream on which the bf16 copies of the frames are made (they feed conv1's weight gradient and
+// the legacy conv1 forward); null: no copy (forward only).
+int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, cudaStream_t st,
+            cudaStream_t frames_st) {
     const long dp = c->d_pad, B = c->B;
     if (c->conv) {
         const int P[3] = {400, 81, 49};
         for (int i = 0; i < groups; i++)
             if (reinterpret_cast<uintptr_t>(obs.p[i]) & 15)
                 return fail(c, GALA_EINVAL, "uint8 observations must be 16-byte aligned");
-        LAUNCH(T_CAST_FRAMES, st, launch_cast_frames(obs, c->frames + (long)agent0 * B * kFramePix, B * kFramePix, rows, groups, st));
+        if (frames_st)
+            LAUNCH(T_CAST_FRAMES, frames_st, launch_cast_frames(obs, c->frames + (long)agent0 * B * kFramePix, B * kFramePix, rows, groups, frames_st));
         for (int l = 0; l < 3; l++) {
             int r = c->legacy_conv ? run_plan(c, c->fwd[l], agent0, groups, rows * P[l], st)
                                    : run_conv(c, c->cfwd[l], agent0, groups, rows, st, l == 0 ? &obs : nullptr);
@@ -594,7 +598,20 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
     for (int i = 0; i < groups; i++) {
         obs.p[i] = ro[i].obs; acts.p[i] = ro[i].actions; rews.p[i] = ro[i].rewards; dns.p[i] = ro[i].dones;
     }
-    int r = forward(c, agent0, groups, obs, (int)B, st);
+    // Second stream of the synchronous mode: work that the chain forward -> loss -> data gradients does not
+    // wait for.  `fork` makes it wait for what `st` has enqueued so far.
+    cudaStream_t ws = side ? side : st;
+    auto fork = [&]() -> int {
+        if (!side) return GALA_OK;
+        CK(cudaEventRecord(c->ev_fork, st));
+        CK(cudaStreamWaitEvent(side, c->ev_fork, 0));
+        return GALA_OK;
+    };
+    int r;
+    // the forward pass reads the uint8 frames itself; their bf16 copies are first needed by conv1's weight gradient
+    const bool frames_aside = c->conv && side && !c->legacy_conv;
+    if (frames_aside && (r = fork()) != GALA_OK) return r;
+    r = forward(c, agent0, groups, obs, (int)B, st, frames_aside ? side : st);
     if (r != GALA_OK) return r;
     LossArgs la{};
     la.T = c->T; la.E = c->E; la.A = A; la.B = B;
@@ -618,18 +635,12 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hb.h = c->hid + (long)agent0 * B * kHidden; hb.h_stride = B * kHidden; hb.h_bf16 = 1;
         hb.piw = c->cl.piw; hb.pib = c->cl.pib; hb.vw = c->cl.vw; hb.vb = c->cl.vb;
         hb.dpre = c->dh + (long)agent0 * S * kHidden; hb.dpre_stride = S * kHidden; hb.dpre_bf16 = 1;
-        LAUNCH(T_HEADS_BWD, st, launch_heads_bwd(hb, groups, st));
-        c->launches++; c->tag_launches[T_HEADS_BWD]++;  // two kernels
-        // The data gradients form a chain (hidden -> conv3 -> conv2); every weight gradient only needs the dY
-        // of its own layer.  With a side stream the weight gradients (and the bias gradients) run beside
-        // the chain; `ws` is where they go, `fork` makes it wait for what `st` has enqueued so far.
-        cudaStream_t ws = side ? side : st;
-        auto fork = [&]() -> int {
-            if (!side) return GALA_OK;
-            CK(cudaEventRecord(c->ev_fork, st));
-            CK(cudaStreamWaitEvent(side, c->ev_fork, 0));
-            return GALA_OK;
-        };
+        // The data gradients form a chain (heads -> hidden -> conv3 -> conv2); every weight gradient only needs
+        // the dY of its own layer.  With a side stream the weight gradients (and the bias gradients) run beside
+        // the chain.
+        if ((r = fork()) != GALA_OK) return r;
+        LAUNCH(T_HEADS_BWD, ws, launch_heads_wgrad(hb, groups, ws));
+        LAUNCH(T_HEADS_BWD, st, launch_heads_dgrad(hb, groups, st));
         if ((r = fork()) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, ws)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
@@ -666,8 +677,8 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hb.h = c->h2 + (long)agent0 * B * H; hb.h_stride = B * H; hb.h_bf16 = 0;
         hb.piw = c->ml.piw; hb.pib = c->ml.pib; hb.vw = c->ml.vw; hb.vb = c->ml.vb;
         hb.dpre = c->dpre2 + (long)agent0 * S * H; hb.dpre_stride = S * H; hb.dpre_bf16 = 0;
-        LAUNCH(T_HEADS_BWD, st, launch_heads_bwd(hb, groups, st));
-        c->launches++; c->tag_launches[T_HEADS_BWD]++;
+        LAUNCH(T_HEADS_BWD, st, launch_heads_dgrad(hb, groups, st));
+        LAUNCH(T_HEADS_BWD, st, launch_heads_wgrad(hb, groups, st));
         DenseBwdArgs d2{};
         d2.rows = (int)S; d2.in_dim = H; d2.out_dim = H; d2.act_in = 2;
         fill_batch(d2.in, c->h1, B * H * 4, agent0, groups);
@@ -993,7 +1004,7 @@ int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int
     Agent& ag = c->agents[agent];
     PtrBatch pb{};
     pb.p[0] = obs;
-    int r = forward(c, agent, 1, pb, c->E, ag.stream);
+    int r = forward(c, agent, 1, pb, c->E, ag.stream, c->legacy_conv ? ag.stream : nullptr);
     if (r != GALA_OK) return r;
     if (actions)
         LAUNCH(T_SAMPLE, ag.stream, launch_sample(c->logits + (long)agent * c->B * c->A, uniforms, actions, c->E, c->A, ag.stream));

@@ -268,7 +268,9 @@ struct HeadsBwdArgs {
     float* grad; long g_stride;                  // flat gradient (same offsets)
     void* dpre; long dpre_stride; int dpre_bf16; // [g][S][H] dL/d(pre-activation of hidden)
 };
-cudaError_t launch_heads_bwd(const HeadsBwdArgs& a, int groups, cudaStream_t st);
+// data part (dpre) and parameter part (gradients of the head weights and biases): independent of each other
+cudaError_t launch_heads_dgrad(const HeadsBwdArgs& a, int groups, cudaStream_t st);
+cudaError_t launch_heads_wgrad(const HeadsBwdArgs& a, int groups, cudaStream_t st);
 struct DenseBwdArgs {
     int rows, in_dim, out_dim, act_in;    // act_in: activation that produced `in` (0 none: no dgrad)
     PtrBatch in;                          // per group [rows][in_dim]  (fp32)
