@@ -284,6 +284,334 @@ cudaError_t launch_heads_wgrad(const HeadsBwdArgs& a, int groups, cudaStream_t s
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------
+// Heads of the conv net in one kernel (hidden width 512, bf16-stored ReLU activations): policy and
+// value outputs, the returns / advantages / objective of a2c_loss_kernel, and the gradient with
+// respect to the hidden layer's pre-activation.  The only coupling between samples is the return
+// recursion along the time axis of ONE environment, so a block takes a few environments of one
+// agent with all their T+1 time steps (rows t*E + e of the agent's batch) and needs no other
+// block; the three objective sums go through per-block partials and a fixed-order final sum by the
+// agent's last block.  When the hidden layer's product arrives as split-K partial sums, the block
+// also finishes that product for its rows (sum in split order, bias, ReLU, rounding to bf16) and
+// stores the activations.
+constexpr int kHeadsH = 512;
+constexpr int kHeadsMaxA1 = 19;   // 18 actions + value
+
+__global__ void __launch_bounds__(256) heads_fused_kernel(HeadsFusedArgs p) {
+    extern __shared__ __align__(16) unsigned char hf_smem[];
+    const int g = blockIdx.y, bi = blockIdx.x;
+    const int T = p.T, E = p.E, A = p.A, A1 = A + 1, T1 = T + 1;
+    const int e0 = bi * p.ne;
+    const int ne = min(p.ne, E - e0);
+    const int R = ne * T1;              // local row el * (T+1) + t  <->  row t * E + e0 + el of the agent's batch
+    const int rcap = p.ne * T1;
+    float* Wsm = reinterpret_cast<float*>(hf_smem);                                  // [A1][512]: pi.W rows, then v.W
+    __nv_bfloat162* hsm = reinterpret_cast<__nv_bfloat162*>(Wsm + A1 * kHeadsH);     // [rcap][256]
+    float* zsm = reinterpret_cast<float*>(hsm + rcap * (kHeadsH / 2));               // [rcap][A1] logits, value
+    float* dsm = zsm + rcap * A1;                                                    // [rcap][A1] dL/dlogits, dL/dvalue
+    float* gsm = dsm + rcap * A1;                                                    // [rcap] returns
+    float* asm_ = gsm + rcap;                                                        // [rcap] advantages
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* P = p.params + (long)g * p.p_stride;
+    const long B = p.B;
+
+    // The head weights were last written by the optimiser pass, which lies at least two kernels back, so
+    // they are fetched before the wait for the previous kernel.
+    for (int i = tid; i < A * kHeadsH; i += 256) Wsm[i] = P[p.piw + i];
+    for (int i = tid; i < kHeadsH; i += 256) Wsm[A * kHeadsH + i] = P[p.vw + i];
+    pdl_wait();
+    pdl_launch();
+    if (p.partials) {
+        const float* pg = p.partials + (long)g * p.partial_group_stride;
+        __nv_bfloat16* hout = p.hid_out + (long)g * p.h_stride;
+        for (int i = tid; i < R * (kHeadsH / 4); i += 256) {
+            const int r = i / (kHeadsH / 4), c4 = i - r * (kHeadsH / 4);
+            const int el = r / T1, t = r - el * T1;
+            const long row = (long)t * E + e0 + el;
+            const float4* src = reinterpret_cast<const float4*>(pg + row * kHeadsH) + c4;
+            float4 acc = *src;
+            for (int s0 = 1; s0 < p.split; s0 += 4) {   // fixed order; four loads in flight
+                float4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; u++)
+                    v[u] = s0 + u < p.split
+                               ? *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + (long)(s0 + u) * p.split_stride)
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < 4; u++)
+                    if (s0 + u < p.split) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+            }
+            const float* bg = P + p.fcb + c4 * 4;
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(acc.x + bg[0], 0.f), fmaxf(acc.y + bg[1], 0.f));
+            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(acc.z + bg[2], 0.f), fmaxf(acc.w + bg[3], 0.f));
+            hsm[r * (kHeadsH / 2) + c4 * 2] = h0;
+            hsm[r * (kHeadsH / 2) + c4 * 2 + 1] = h1;
+            uint2 u;
+            u.x = *reinterpret_cast<const unsigned*>(&h0); u.y = *reinterpret_cast<const unsigned*>(&h1);
+            *reinterpret_cast<uint2*>(hout + row * kHeadsH + c4 * 4) = u;
+        }
+    } else {
+        const __nv_bfloat16* hin = p.hid + (long)g * p.h_stride;
+        for (int i = tid; i < R * (kHeadsH / 8); i += 256) {
+            const int r = i / (kHeadsH / 8), c8 = i - r * (kHeadsH / 8);
+            const int el = r / T1, t = r - el * T1;
+            const long row = (long)t * E + e0 + el;
+            reinterpret_cast<uint4*>(hsm + r * (kHeadsH / 2))[c8] = *(reinterpret_cast<const uint4*>(hin + row * kHeadsH) + c8);
+        }
+    }
+    __syncthreads();
+
+    // outputs: a warp per row, the row's 512 activations spread over the lanes (16 each) and kept in registers
+    for (int r = warp; r < R; r += 8) {
+        float hx[16];
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            const float2 f = __bfloat1622float2(hsm[r * (kHeadsH / 2) + lane + 32 * i]);
+            hx[2 * i] = f.x; hx[2 * i + 1] = f.y;
+        }
+        for (int k = 0; k < A1; k++) {
+            const float2* w2 = reinterpret_cast<const float2*>(Wsm + k * kHeadsH);
+            float acc = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const float2 w = w2[lane + 32 * i];
+                acc = fmaf(w.x, hx[2 * i], acc);
+                acc = fmaf(w.y, hx[2 * i + 1], acc);
+            }
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (lane == 0) zsm[r * A1 + k] = acc + (k < A ? P[p.pib + k] : P[p.vb]);
+        }
+    }
+    __syncthreads();
+    {
+        float* logits = p.logits + (long)g * B * A;
+        float* values = p.values + (long)g * B;
+        for (int i = tid; i < R * A1; i += 256) {
+            const int r = i / A1, k = i - r * A1;
+            const int el = r / T1, t = r - el * T1;
+            const long row = (long)t * E + e0 + el;
+            if (k < A) logits[row * A + k] = zsm[i]; else values[row] = zsm[i];
+        }
+    }
+    const int* actions = reinterpret_cast<const int*>(p.actions.p[g]);
+    const float* rewards = reinterpret_cast<const float*>(p.rewards.p[g]);
+    const unsigned char* dones = reinterpret_cast<const unsigned char*>(p.dones.p[g]);
+    const long S = (long)T * E;
+    // returns: a warp per environment, time steps in the lanes, reverse scan of the maps G -> r + gamma (1 - done) G
+    for (int el = warp; el < ne; el += 8) {
+        const int e = e0 + el;
+        float carry = zsm[(el * T1 + T) * A1 + A];   // bootstrap V(s_T)
+        for (int t_hi = T; t_hi > 0; t_hi -= 32) {
+            const int t_lo = t_hi > 32 ? t_hi - 32 : 0;
+            const int n = t_hi - t_lo;
+            const int t = t_lo + lane;
+            float a = 1.0f, b = 0.0f;
+            if (lane < n) {
+                a = p.gamma * (dones[(long)t * E + e] ? 0.0f : 1.0f);
+                b = rewards[(long)t * E + e];
+            }
+            for (int off = 1; off < 32; off <<= 1) {
+                const float a2 = __shfl_down_sync(0xffffffffu, a, off);
+                const float b2 = __shfl_down_sync(0xffffffffu, b, off);
+                if (lane + off < 32) { b = a * b2 + b; a = a * a2; }
+            }
+            const float gt = a * carry + b;
+            if (lane < n) {
+                gsm[el * T1 + t] = gt;
+                asm_[el * T1 + t] = gt - zsm[(el * T1 + t) * A1 + A];
+            }
+            carry = __shfl_sync(0xffffffffu, gt, 0);
+        }
+    }
+    __syncthreads();
+
+    float lp = 0.0f, lv = 0.0f, le = 0.0f;
+    const float invS = 1.0f / (float)S;
+    for (int i = tid; i < ne * T; i += 256) {
+        const int el = i / T, t = i - el * T;
+        const int r = el * T1 + t;
+        const long srow = (long)t * E + e0 + el;
+        const float* z = zsm + r * A1;
+        float mx = z[0];
+        for (int k = 1; k < A; k++) mx = fmaxf(mx, z[k]);
+        float sum = 0.0f;
+        for (int k = 0; k < A; k++) sum += expf(z[k] - mx);
+        const float lse = mx + logf(sum);
+        float H = 0.0f;
+        for (int k = 0; k < A; k++) { const float lg = z[k] - lse; H -= expf(lg) * lg; }
+        const int act = actions[srow];
+        const float adv = asm_[r], gt = gsm[r], v = z[A];
+        float* dz = p.dlogits + ((long)g * S + srow) * A;
+        for (int k = 0; k < A; k++) {
+            const float lg = z[k] - lse, pi = expf(lg);
+            const float d = (adv * (pi - (k == act ? 1.0f : 0.0f)) + p.ent_coef * pi * (lg + H)) * invS;
+            dsm[r * A1 + k] = d;
+            dz[k] = d;
+        }
+        const float dvv = 2.0f * p.vf_coef * (v - gt) * invS;
+        dsm[r * A1 + A] = dvv;
+        p.dvalues[(long)g * S + srow] = dvv;
+        p.returns[(long)g * S + srow] = gt;
+        p.adv[(long)g * S + srow] = adv;
+        lp += -(z[act] - lse) * adv;
+        lv += (gt - v) * (gt - v);
+        le += H;
+    }
+    __shared__ float red[3][256];
+    __shared__ bool last;
+    red[0][tid] = lp; red[1][tid] = lv; red[2][tid] = le;
+    __syncthreads();   // also publishes dsm
+    for (int st = 128; st > 0; st >>= 1) {
+        if (tid < st)
+            for (int q = 0; q < 3; q++) red[q][tid] += red[q][tid + st];
+        __syncthreads();
+    }
+    if (tid == 0) {
+        float* lpart = p.loss_partial + ((long)g * E + bi) * 4;
+        lpart[0] = red[0][0]; lpart[1] = red[1][0]; lpart[2] = red[2][0];
+        __threadfence();
+        last = atomicAdd(p.ticket + g, 1u) == gridDim.x - 1;
+    }
+
+    // gradient of the hidden pre-activation: thread owns columns 2 tid, 2 tid + 1; its slice of the head
+    // weights sits in registers, the samples' dL/dlogits, dL/dvalue are broadcast from shared memory
+    float2 wr[kHeadsMaxA1];
+#pragma unroll
+    for (int k = 0; k < kHeadsMaxA1; k++)
+        wr[k] = k < A1 ? reinterpret_cast<const float2*>(Wsm + k * kHeadsH)[tid] : make_float2(0.f, 0.f);
+    __nv_bfloat16* dh = p.dh + (long)g * p.dh_stride;
+    for (int i = 0; i < ne * T; i++) {
+        const int el = i / T, t = i - el * T;
+        const int r = el * T1 + t;
+        const long srow = (long)t * E + e0 + el;
+        float a0 = 0.0f, a1 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kHeadsMaxA1; k++)
+            if (k < A1) {
+                const float d = dsm[r * A1 + k];
+                a0 = fmaf(d, wr[k].x, a0);
+                a1 = fmaf(d, wr[k].y, a1);
+            }
+        const float2 h = __bfloat1622float2(hsm[r * (kHeadsH / 2) + tid]);
+        const __nv_bfloat162 o = __floats2bfloat162_rn(h.x > 0.0f ? a0 : 0.0f, h.y > 0.0f ? a1 : 0.0f);
+        reinterpret_cast<__nv_bfloat162*>(dh + srow * kHeadsH)[tid] = o;
+    }
+    __syncthreads();
+    if (last) {   // the agent's last block adds the blocks' sums in block order
+        __threadfence();
+        const volatile float* lp0 = p.loss_partial + (long)g * E * 4;
+        float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f;
+        for (unsigned k0 = 0; k0 < gridDim.x; k0 += 256) {
+            const unsigned k = k0 + tid;
+            __syncthreads();
+            if (k < gridDim.x) { red[0][tid] = lp0[k * 4]; red[1][tid] = lp0[k * 4 + 1]; red[2][tid] = lp0[k * 4 + 2]; }
+            __syncthreads();
+            if (tid == 0)
+                for (unsigned q = 0; q < min(256u, gridDim.x - k0); q++) { s0 += red[0][q]; s1 += red[1][q]; s2 += red[2][q]; }
+        }
+        if (tid == 0) {
+            p.losses[g * 4 + 0] = s0 * invS;
+            p.losses[g * 4 + 1] = s1 * invS;
+            p.losses[g * 4 + 2] = s2 * invS;
+            p.ticket[g] = 0;   // ready for the next launch
+        }
+    }
+}
+
+int heads_fused_envs_per_block(int T, int E, int groups) {
+    int ne = 32 / (T + 1);
+    if (ne > E) ne = E;
+    if (ne < 1) ne = 1;
+    while (ne > 1 && (long)groups * ((E + ne - 1) / ne) < 296) ne--;
+    return ne;
+}
+static size_t heads_fused_smem(int A, int rcap) {
+    const int A1 = A + 1;
+    return (size_t)A1 * kHeadsH * 4 + (size_t)rcap * kHeadsH * 2 + (size_t)rcap * A1 * 8 + (size_t)rcap * 8;
+}
+bool heads_fused_supported(int T, int E, int A, int H) {
+    return H == kHeadsH && A + 1 <= kHeadsMaxA1 && A >= 1 && T >= 1 && E >= 1 &&
+           heads_fused_smem(A, T + 1) <= 160 * 1024;
+}
+int heads_fused_blocks(int T, int E, int groups) {
+    const int ne = heads_fused_envs_per_block(T, E, groups);
+    return (E + ne - 1) / ne;
+}
+cudaError_t launch_heads_fused(const HeadsFusedArgs& a0, int groups, cudaStream_t st) {
+    HeadsFusedArgs a = a0;
+    if (!heads_fused_supported(a.T, a.E, a.A, kHeadsH)) return cudaErrorNotSupported;
+    a.ne = heads_fused_envs_per_block(a.T, a.E, groups);
+    const size_t smem = heads_fused_smem(a.A, a.ne * (a.T + 1));
+    static size_t attr_set = 0;
+    if (smem > 48 * 1024 && smem > attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(heads_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(160 * 1024));
+        if (e != cudaSuccess) return e;
+        attr_set = 160 * 1024;
+    }
+    (void)launch_pdl(heads_fused_kernel, dim3((a.E + a.ne - 1) / a.ne, groups), dim3(256), smem, st, a);
+    return cudaGetLastError();
+}
+
+// Parameter gradients of the heads, d pi.W[k][j] = sum_s dz[s][k] h[s][j] (k = A: value head) and the
+// biases as one more column tile whose "activation" is 1.  A block owns 32 columns of one agent; its
+// eight warps take contiguous slices of the samples (lane = column, one accumulator per output row),
+// and the slices are added in warp order, so the sum has a fixed order.
+__global__ void __launch_bounds__(256) heads_wgrad_tiled_kernel(HeadsBwdArgs a) {
+    pdl_wait();
+    pdl_launch();
+    constexpr int kChunk = 256;
+    __shared__ float dzs[kChunk][kHeadsMaxA1 + 1];
+    __shared__ float part[8][kHeadsMaxA1][32];
+    const int g = blockIdx.y, tile = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int A = a.A, A1 = A + 1, H = a.H;
+    const bool bias_tile = tile * 32 >= H;
+    const char* hbase = reinterpret_cast<const char*>(a.h) + (long)g * a.h_stride * (a.h_bf16 ? 2 : 4);
+    const float* dz = a.dlogits + (long)g * a.dlogits_stride;
+    const float* dv = a.dvalues + (long)g * a.dvalues_stride;
+    const int j = tile * 32 + lane;
+    float acc[kHeadsMaxA1];
+#pragma unroll
+    for (int k = 0; k < kHeadsMaxA1; k++) acc[k] = 0.0f;
+    for (int s0 = 0; s0 < a.rows; s0 += kChunk) {
+        const int n = min(kChunk, a.rows - s0);
+        __syncthreads();
+        for (int i = tid; i < n * A1; i += 256) {
+            const int s = i / A1, k = i - s * A1;
+            dzs[s][k] = k < A ? dz[(long)(s0 + s) * A + k] : dv[s0 + s];
+        }
+        __syncthreads();
+        const int per = (n + 7) / 8;
+        const int lo = warp * per, hi = min(n, lo + per);
+        for (int s = lo; s < hi; s++) {
+            const float h = bias_tile ? 1.0f : ld_in(hbase, (long)(s0 + s) * H + j, a.h_bf16);
+#pragma unroll
+            for (int k = 0; k < kHeadsMaxA1; k++)
+                if (k < A1) acc[k] = fmaf(dzs[s][k], h, acc[k]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kHeadsMaxA1; k++)
+        if (k < A1) part[warp][k][lane] = acc[k];
+    __syncthreads();
+    float* G = a.grad + (long)g * a.g_stride;
+    for (int i = tid; i < A1 * 32; i += 256) {
+        const int k = i >> 5, l = i & 31;
+        float s = part[0][k][l];
+        for (int w = 1; w < 8; w++) s += part[w][k][l];
+        if (!bias_tile) {
+            if (k < A) G[a.piw + (long)k * H + tile * 32 + l] = s; else G[a.vw + tile * 32 + l] = s;
+        } else if (l == 0) {
+            if (k < A) G[a.pib + k] = s; else G[a.vb] = s;
+        }
+    }
+}
+cudaError_t launch_heads_wgrad_tiled(const HeadsBwdArgs& a, int groups, cudaStream_t st) {
+    if (a.A + 1 > kHeadsMaxA1 || (a.H & 31)) return cudaErrorNotSupported;
+    (void)launch_pdl(heads_wgrad_tiled_kernel, dim3(a.H / 32 + 1, groups), dim3(256), 0, st, a);
+    return cudaGetLastError();
+}
+
 // Dense layer backward (MLP trunk): gW[o][i] = sum_r dpre[r][o] in[r][i], gb[o] = sum_r dpre[r][o],
 // and (if din) din[r][i] = (sum_o dpre[r][o] W[o][i]) * act'(in[r][i]).
 __global__ void __launch_bounds__(256) dense_wgrad_kernel(DenseBwdArgs a) {

@@ -44,6 +44,10 @@ struct WgradPlan {  // conv2 / conv3 weight gradient with resident operands
     WgradArgs args;
     int tag = 0;
 };
+struct Wgrad1Plan {  // conv1 weight gradient from the uint8 frames
+    CUtensorMap y;
+    Wgrad1Args args;
+};
 struct ConvPlan {  // one forward or data-gradient convolution (input resident in shared memory)
     CUtensorMap x, w;
     ConvArgs args;
@@ -54,7 +58,7 @@ struct ConvPlan {  // one forward or data-gradient convolution (input resident i
 // Kernel classes for launch counting and optional per-class device timing.
 enum Tag : int {
     T_CAST_FRAMES = 0, T_HEADS_FWD, T_LOSS, T_HEADS_BWD, T_COLSUM, T_SPLITK, T_GRAD_NORM,
-    T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST,
+    T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST, T_HEADS_FUSED,
     T_GEMM_CONV_FWD,          // +layer (3)
     T_GEMM_FC_FWD = T_GEMM_CONV_FWD + 3, T_GEMM_FC_WGRAD, T_GEMM_FC_DGRAD,
     T_GEMM_CONV_WGRAD,        // +layer (3)
@@ -63,7 +67,7 @@ enum Tag : int {
 };
 const char* const kTagNames[T_COUNT] = {
     "cast_frames", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "grad_norm",
-    "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16",
+    "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16", "heads_fused",
     "gemm_conv1_fwd", "gemm_conv2_fwd", "gemm_conv3_fwd", "gemm_fc_fwd", "gemm_fc_wgrad", "gemm_fc_dgrad",
     "gemm_conv1_wgrad", "gemm_conv2_wgrad", "gemm_conv3_wgrad", "gemm_conv1_dgrad", "gemm_conv2_dgrad",
     "gemm_conv3_dgrad"};
@@ -103,7 +107,9 @@ struct gala_ctx {
     __nv_bfloat16* shadow = nullptr;
     float *clip = nullptr, *norm = nullptr, *losses = nullptr;
     double *norm_partial = nullptr, *colsum_partial = nullptr;
-    unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr;
+    unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr, *heads_ticket = nullptr;
+    float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
+    bool fused_heads = false;
     int* error_word = nullptr;
     double *cons_partial = nullptr, *cons_out = nullptr;
     unsigned* cons_ticket = nullptr;
@@ -122,6 +128,7 @@ struct gala_ctx {
     Plan fwd[3], fc_fwd, fc_wgrad, fc_dgrad, wgrad[3], dgrad[3];
     ConvPlan cfwd[3], cdgrad[3];
     WgradPlan cwgrad[3];
+    Wgrad1Plan cwgrad1;
     uint32_t* gate[2] = {nullptr, nullptr};   // ReLU gate bits of act[0], act[1]
     bool legacy_conv = false;
 };
@@ -431,7 +438,51 @@ int build_plans(gala_ctx* c) {
             d.built = true;
         }
     }
+    {
+        Wgrad1Plan& w1 = c->cwgrad1;
+        memset(&w1.args, 0, sizeof w1.args);
+        w1.args.samples = (int)S; w1.args.y_samples = (int)S;
+        w1.args.scale = 1.0f / 255.0f;
+        w1.args.out = c->g + c->cl.w[0]; w1.args.out_group_stride = dp;
+        w1.args.error_word = c->error_word;
+        ok &= make_wgrad1_map(&w1.y, c->dy[0], (uint64_t)n * S);
+    }
     return ok ? GALA_OK : fail(c, GALA_ECUDA, "cuTensorMapEncodeTiled failed while building GEMM descriptors");
+}
+
+// Slices of the samples per agent for a weight gradient whose CTAs each own one agent and a slice: chosen so
+// that the CTAs fill the SMs in whole waves.  `fixed` = set-up and epilogue of a CTA in units of one sample.
+int pick_splits(gala_ctx* c, int groups, int S, long count, int fixed) {
+    int best = 1;
+    long best_cost = -1;
+    for (int sp = 1; sp <= c->max_split && sp <= S; sp++) {
+        if (sp > 1 && (S / sp < 4 || sp * count > c->splitk_group_stride)) break;
+        const long waves = ((long)groups * sp + 147) / 148, per = (S + sp - 1) / sp;
+        const long cost = waves * (per + fixed) + (sp > 1 ? 8 : 0);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = sp; }
+    }
+    return best;
+}
+
+// conv1 weight gradient from the uint8 frames; with more than one slice the partial sums go through the
+// fixed-order reduction
+int run_conv1_wgrad(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, cudaStream_t st) {
+    Wgrad1Args a = c->cwgrad1.args;
+    const long count = 32 * 256;
+    a.group0 = agent0; a.groups = groups; a.obs = obs;
+    a.splits = pick_splits(c, groups, a.samples, count, 3);
+    float* final_out = a.out + (long)agent0 * a.out_group_stride;
+    if (a.splits == 1) {
+        a.out = final_out; a.out_split_stride = 0;
+        LAUNCH(T_GEMM_CONV_WGRAD, st, launch_wgrad1(c->cwgrad1.y, a, st));
+        return GALA_OK;
+    }
+    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+    a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
+    LAUNCH(T_GEMM_CONV_WGRAD, st, launch_wgrad1(c->cwgrad1.y, a, st));
+    LAUNCH(T_SPLITK, st, launch_splitk_reduce(c->splitk_ws + (long)agent0 * c->splitk_group_stride, final_out, count, a.splits,
+                                count, groups, c->splitk_group_stride, c->cwgrad1.args.out_group_stride, st));
+    return GALA_OK;
 }
 
 // conv2 / conv3 weight gradient: slices of the samples per agent chosen so that the CTAs fill the SMs in
@@ -511,10 +562,15 @@ int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t s
 
 // ------------------------------------------------------------------ forward / backward
 // Forward on `rows` observations per agent for agents [agent0, agent0+groups).
-// frames_st: stream on which the bf16 copies of the frames are made (they feed conv1's weight gradient and
-// the legacy conv1 forward); null: no copy (forward only).
+// What forward() leaves undone when the caller fuses the heads with the objective: the hidden layer's
+// split-K partial sums (split > 1) still wait for their reduction, bias and ReLU.
+struct HiddenPending { int split = 0; long count = 0; };
+
+// frames_st: stream on which the bf16 copies of the frames are made (they feed the legacy conv1 products);
+// null: no copy.
+// pend != null: stop before the heads (and before the reduction of a split hidden-layer product).
 int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, cudaStream_t st,
-            cudaStream_t frames_st) {
+            cudaStream_t frames_st, HiddenPending* pend = nullptr) {
     const long dp = c->d_pad, B = c->B;
     if (c->conv) {
         const int P[3] = {400, 81, 49};
@@ -548,12 +604,14 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
                 a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
                 a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
                 LAUNCH(p.tag, st, launch_gemm(p.A, p.B, a, st));
+                if (pend) { pend->split = split; pend->count = count; return GALA_OK; }
                 LAUNCH(T_SPLITK, st, launch_splitk_reduce_act(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
                                                               c->hid + (long)agent0 * B * kHidden, c->x + c->cl.fcb, dp, agent0,
                                                               count, kHidden, split, count, groups, c->splitk_group_stride,
                                                               B * kHidden, st));
             }
         }
+        if (pend) return GALA_OK;
         HeadsArgs h{};
         h.rows = rows; h.H = kHidden; h.A = c->A;
         h.h = c->hid + (long)agent0 * B * kHidden; h.h_stride = B * kHidden; h.h_bf16 = 1;
@@ -607,11 +665,11 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         CK(cudaStreamWaitEvent(side, c->ev_fork, 0));
         return GALA_OK;
     };
-    int r;
-    // the forward pass reads the uint8 frames itself; their bf16 copies are first needed by conv1's weight gradient
-    const bool frames_aside = c->conv && side && !c->legacy_conv;
-    if (frames_aside && (r = fork()) != GALA_OK) return r;
-    r = forward(c, agent0, groups, obs, (int)B, st, frames_aside ? side : st);
+    // forward pass and weight gradient of conv1 read the uint8 frames themselves; only the legacy products
+    // need bf16 copies
+    HiddenPending pend;
+    const bool fused = c->conv && c->fused_heads;
+    int r = forward(c, agent0, groups, obs, (int)B, st, c->legacy_conv ? st : nullptr, fused ? &pend : nullptr);
     if (r != GALA_OK) return r;
     LossArgs la{};
     la.T = c->T; la.E = c->E; la.A = A; la.B = B;
@@ -621,7 +679,29 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
     la.returns = c->returns + (long)agent0 * S; la.adv = c->adv + (long)agent0 * S;
     la.dlogits = c->dlogits + (long)agent0 * S * A; la.dvalues = c->dvalues + (long)agent0 * S;
     la.losses = c->losses + (long)agent0 * 4;
-    LAUNCH(T_LOSS, st, launch_a2c_loss(la, groups, st));
+    if (fused) {
+        HeadsFusedArgs hf{};
+        hf.T = c->T; hf.E = c->E; hf.A = A; hf.B = B;
+        hf.gamma = c->hp.gamma; hf.ent_coef = c->hp.ent_coef; hf.vf_coef = c->hp.vf_coef;
+        hf.hid = c->hid + (long)agent0 * B * kHidden; hf.hid_out = c->hid + (long)agent0 * B * kHidden;
+        hf.h_stride = B * kHidden;
+        if (pend.split > 1) {
+            hf.partials = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+            hf.split = pend.split; hf.split_stride = pend.count; hf.partial_group_stride = c->splitk_group_stride;
+        }
+        hf.params = c->x + (long)agent0 * dp; hf.p_stride = dp;
+        hf.piw = c->cl.piw; hf.pib = c->cl.pib; hf.vw = c->cl.vw; hf.vb = c->cl.vb; hf.fcb = c->cl.fcb;
+        hf.actions = acts; hf.rewards = rews; hf.dones = dns;
+        hf.logits = c->logits + (long)agent0 * B * A; hf.values = c->values + (long)agent0 * B;
+        hf.returns = la.returns; hf.adv = la.adv; hf.dlogits = la.dlogits; hf.dvalues = la.dvalues;
+        hf.losses = la.losses;
+        hf.dh = c->dh + (long)agent0 * S * kHidden; hf.dh_stride = S * kHidden;
+        hf.loss_partial = c->heads_partial + (long)agent0 * c->E * 4;
+        hf.ticket = c->heads_ticket + agent0;
+        LAUNCH(T_HEADS_FUSED, st, launch_heads_fused(hf, groups, st));
+    } else {
+        LAUNCH(T_LOSS, st, launch_a2c_loss(la, groups, st));
+    }
 
     HeadsBwdArgs hb{};
     hb.rows = (int)S; hb.A = A;
@@ -639,15 +719,20 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         // the dY of its own layer.  With a side stream the weight gradients (and the bias gradients) run beside
         // the chain.
         if ((r = fork()) != GALA_OK) return r;
-        LAUNCH(T_HEADS_BWD, ws, launch_heads_wgrad(hb, groups, ws));
-        LAUNCH(T_HEADS_BWD, st, launch_heads_dgrad(hb, groups, st));
+        if (fused) {
+            LAUNCH(T_HEADS_BWD, ws, launch_heads_wgrad_tiled(hb, groups, ws));
+        } else {
+            LAUNCH(T_HEADS_BWD, ws, launch_heads_wgrad(hb, groups, ws));
+            LAUNCH(T_HEADS_BWD, st, launch_heads_dgrad(hb, groups, st));
+        }
         if ((r = fork()) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, ws)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
         for (int l = 2; l >= 0; l--) {
             if ((r = fork()) != GALA_OK) return r;
-            r = (l > 0 && !c->legacy_conv) ? run_conv_wgrad(c, c->cwgrad[l], agent0, groups, ws)
-                                           : run_wgrad(c, c->wgrad[l], agent0, groups, ws);
+            r = c->legacy_conv ? run_wgrad(c, c->wgrad[l], agent0, groups, ws)
+                : l > 0        ? run_conv_wgrad(c, c->cwgrad[l], agent0, groups, ws)
+                               : run_conv1_wgrad(c, agent0, groups, obs, ws);
             if (r != GALA_OK) return r;
             if (l > 0) {
                 r = c->legacy_conv ? run_plan(c, c->dgrad[l], agent0, groups, 0, st)
@@ -917,7 +1002,10 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         CK(gemm_init());
         CK(conv_init());
         CK(wgrad_init());
+        CK(wgrad1_init());
         c->legacy_conv = getenv("GALA_CONV_LEGACY") != nullptr;
+        c->fused_heads = heads_fused_supported(c->T, c->E, c->A, kHidden) && getenv("GALA_HEADS_UNFUSED") == nullptr;
+        ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {

@@ -78,15 +78,6 @@ constexpr int kU8Bytes = 24 * 336;       // 8064
 constexpr int kU8Stride = 8192;
 constexpr int kConvThreads = 352, kConv1Threads = 352 + 128;
 
-// Bytes k and k+1 of w as two bf16 numbers, without the (slow) integer -> float conversion unit: a byte
-// dropped into the low mantissa bits of 2^23 is the float 2^23 + b, so subtracting 2^23 leaves b exactly;
-// an integer below 256 has no bits in the lower half of its float, so the upper halves are its bf16.
-__device__ __forceinline__ uint32_t u8x2_to_bf16x2(uint32_t w, int k) {
-    const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7650u + k)) - 8388608.0f;
-    const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7651u + k)) - 8388608.0f;
-    return __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632u);
-}
-
 // plane and row shift of a tap
 template <int V> __host__ __device__ constexpr void tap_view(int t, int& plane, int& shift) {
     if constexpr (V == CV_CONV1_FWD) { const int ky = t >> 1; plane = ky & 3; shift = (ky >> 2) * 21 + (t & 1); }

@@ -191,6 +191,22 @@ bool make_wgrad_maps(int variant, CUtensorMap* x_map, CUtensorMap* y_map, const 
                      const void* y_base, uint64_t y_samples);
 cudaError_t launch_wgrad(const CUtensorMap& x, const CUtensorMap& y, const WgradArgs& a, cudaStream_t st);
 
+// conv1 weight gradient from the uint8 frames (wgrad1.cu); y = dY of conv1 [sample][20][20][32] bf16
+struct Wgrad1Args {
+    int groups, group0;    // agents of this launch
+    int splits;            // CTAs per agent, each takes a slice of the samples
+    int samples;           // samples per agent to reduce over (the first `samples` frames of each agent)
+    int y_samples;         // samples per agent in the dY tensor
+    float scale;           // applied to the sums (1/255: the frames enter the network divided by 255)
+    float* out;            // agent i, slice s at out + i * out_group_stride + s * out_split_stride, as W[32][256]
+    long out_group_stride, out_split_stride;
+    int* error_word;
+    PtrBatch obs;          // the agents' uint8 frames [..][84][84][4], 16-byte aligned
+};
+cudaError_t wgrad1_init();
+bool make_wgrad1_map(CUtensorMap* y_map, const void* y_base, uint64_t y_samples);
+cudaError_t launch_wgrad1(const CUtensorMap& y, const Wgrad1Args& a, cudaStream_t st);
+
 // ---------------------------------------------------------------- sweep
 struct SweepHp {
     float lr, alpha, eps;
@@ -271,6 +287,34 @@ struct HeadsBwdArgs {
 // data part (dpre) and parameter part (gradients of the head weights and biases): independent of each other
 cudaError_t launch_heads_dgrad(const HeadsBwdArgs& a, int groups, cudaStream_t st);
 cudaError_t launch_heads_wgrad(const HeadsBwdArgs& a, int groups, cudaStream_t st);
+// same sums with the samples split over the warps of a block per 32 columns (fixed order); not supported
+// (cudaErrorNotSupported) for more than 18 actions or a width that is not a multiple of 32
+cudaError_t launch_heads_wgrad_tiled(const HeadsBwdArgs& a, int groups, cudaStream_t st);
+// Heads of the conv net (width 512, bf16 ReLU activations) fused with returns, advantages, objective and
+// the gradient of the hidden pre-activation; see a2c.cu.
+struct HeadsFusedArgs {
+    int T, E, A;
+    int ne;                 // environments per block (set by the launcher)
+    float gamma, ent_coef, vf_coef;
+    const __nv_bfloat16* hid;   // [g][B][512] stored activations (used when partials == null)
+    __nv_bfloat16* hid_out;     // where the activations are stored when they are formed here
+    long h_stride;
+    const float* partials;      // optional split-K partial sums of the hidden layer [g][split][B][512]
+    int split; long split_stride, partial_group_stride;
+    const float* params; long p_stride;   // flat vectors of the first agent of the launch
+    long piw, pib, vw, vb, fcb;
+    PtrBatch actions, rewards, dones;     // per agent [T][E]
+    float *logits, *values;               // [g][B][A], [g][B]
+    float *returns, *adv, *dlogits, *dvalues;   // [g][S], [g][S], [g][S][A], [g][S]
+    float* losses;                        // [g][4]
+    long B;                               // (T+1)*E
+    __nv_bfloat16* dh; long dh_stride;    // [g][S][512]
+    float* loss_partial;                  // [g][E][4] scratch
+    unsigned* ticket;                     // [g], zero before the first launch
+};
+bool heads_fused_supported(int T, int E, int A, int H);
+int heads_fused_blocks(int T, int E, int groups);   // blocks per agent of a launch with `groups` agents
+cudaError_t launch_heads_fused(const HeadsFusedArgs& a, int groups, cudaStream_t st);
 struct DenseBwdArgs {
     int rows, in_dim, out_dim, act_in;    // act_in: activation that produced `in` (0 none: no dgrad)
     PtrBatch in;                          // per group [rows][in_dim]  (fp32)

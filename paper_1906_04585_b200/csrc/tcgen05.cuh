@@ -147,4 +147,13 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// Bytes k and k+1 of w as two bf16 numbers, without the (slow) integer -> float conversion unit: a byte
+// dropped into the low mantissa bits of 2^23 is the float 2^23 + b, so subtracting 2^23 leaves b exactly;
+// an integer below 256 has no bits in the lower half of its float, so the upper halves are its bf16.
+__device__ __forceinline__ uint32_t u8x2_to_bf16x2(uint32_t w, int k) {
+    const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7650u + k)) - 8388608.0f;
+    const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7651u + k)) - 8388608.0f;
+    return __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632u);
+}
+
 }  // namespace gala
