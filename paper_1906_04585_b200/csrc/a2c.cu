@@ -361,25 +361,36 @@ __global__ void __launch_bounds__(256) heads_fused_kernel(HeadsFusedArgs p) {
     }
     __syncthreads();
 
-    // outputs: a warp per row, the row's 512 activations spread over the lanes (16 each) and kept in registers
-    for (int r = warp; r < R; r += 8) {
-        float hx[16];
+    // outputs: a warp takes three rows at a time, their 512 activations spread over the lanes (16 each) and
+    // kept in registers, so that every weight fetched from shared memory serves three rows
+    for (int r0 = warp * 3; r0 < R; r0 += 24) {
+        float hx[3][16];
 #pragma unroll
-        for (int i = 0; i < 8; i++) {
-            const float2 f = __bfloat1622float2(hsm[r * (kHeadsH / 2) + lane + 32 * i]);
-            hx[2 * i] = f.x; hx[2 * i + 1] = f.y;
+        for (int u = 0; u < 3; u++) {
+            const int r = min(r0 + u, R - 1);
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const float2 f = __bfloat1622float2(hsm[r * (kHeadsH / 2) + lane + 32 * i]);
+                hx[u][2 * i] = f.x; hx[u][2 * i + 1] = f.y;
+            }
         }
         for (int k = 0; k < A1; k++) {
             const float2* w2 = reinterpret_cast<const float2*>(Wsm + k * kHeadsH);
-            float acc = 0.0f;
+            float acc[3] = {0.0f, 0.0f, 0.0f};
 #pragma unroll
             for (int i = 0; i < 8; i++) {
                 const float2 w = w2[lane + 32 * i];
-                acc = fmaf(w.x, hx[2 * i], acc);
-                acc = fmaf(w.y, hx[2 * i + 1], acc);
+#pragma unroll
+                for (int u = 0; u < 3; u++) {
+                    acc[u] = fmaf(w.x, hx[u][2 * i], acc[u]);
+                    acc[u] = fmaf(w.y, hx[u][2 * i + 1], acc[u]);
+                }
             }
-            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            if (lane == 0) zsm[r * A1 + k] = acc + (k < A ? P[p.pib + k] : P[p.vb]);
+#pragma unroll
+            for (int u = 0; u < 3; u++)
+                for (int off = 16; off > 0; off >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
+            const float bk = k < A ? P[p.pib + k] : P[p.vb];
+            if (lane < 3 && r0 + lane < R) zsm[(r0 + lane) * A1 + k] = (lane == 0 ? acc[0] : lane == 1 ? acc[1] : acc[2]) + bk;
         }
     }
     __syncthreads();
@@ -560,7 +571,7 @@ __global__ void __launch_bounds__(256) heads_wgrad_tiled_kernel(HeadsBwdArgs a) 
     pdl_wait();
     pdl_launch();
     constexpr int kChunk = 256;
-    __shared__ float dzs[kChunk][kHeadsMaxA1 + 1];
+    __shared__ __align__(16) float dzs[kChunk][kHeadsMaxA1 + 1];   // rows of 20 floats; entries from A + 1 on are zero
     __shared__ float part[8][kHeadsMaxA1][32];
     const int g = blockIdx.y, tile = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -576,18 +587,34 @@ __global__ void __launch_bounds__(256) heads_wgrad_tiled_kernel(HeadsBwdArgs a) 
     for (int s0 = 0; s0 < a.rows; s0 += kChunk) {
         const int n = min(kChunk, a.rows - s0);
         __syncthreads();
-        for (int i = tid; i < n * A1; i += 256) {
-            const int s = i / A1, k = i - s * A1;
-            dzs[s][k] = k < A ? dz[(long)(s0 + s) * A + k] : dv[s0 + s];
+        for (int i = tid; i < n * (kHeadsMaxA1 + 1); i += 256) {
+            const int s = i / (kHeadsMaxA1 + 1), k = i - s * (kHeadsMaxA1 + 1);
+            dzs[s][k] = k < A ? dz[(long)(s0 + s) * A + k] : (k == A ? dv[s0 + s] : 0.0f);
         }
         __syncthreads();
         const int per = (n + 7) / 8;
         const int lo = warp * per, hi = min(n, lo + per);
-        for (int s = lo; s < hi; s++) {
-            const float h = bias_tile ? 1.0f : ld_in(hbase, (long)(s0 + s) * H + j, a.h_bf16);
+        for (int sb = lo; sb < hi; sb += 8) {   // eight activations in flight, then their products
+            float hv[8];
 #pragma unroll
-            for (int k = 0; k < kHeadsMaxA1; k++)
-                if (k < A1) acc[k] = fmaf(dzs[s][k], h, acc[k]);
+            for (int u = 0; u < 8; u++)
+                hv[u] = sb + u < hi ? (bias_tile ? 1.0f : ld_in(hbase, (long)(s0 + sb + u) * H + j, a.h_bf16)) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < 8; u++) {
+                if (sb + u < hi) {
+                    const float4* d4 = reinterpret_cast<const float4*>(&dzs[sb + u][0]);
+#pragma unroll
+                    for (int k4 = 0; k4 < (kHeadsMaxA1 + 1) / 4; k4++) {
+                        if (k4 * 4 < A1) {
+                            const float4 d = d4[k4];
+                            acc[k4 * 4] = fmaf(d.x, hv[u], acc[k4 * 4]);
+                            if (k4 * 4 + 1 < kHeadsMaxA1) acc[k4 * 4 + 1] = fmaf(d.y, hv[u], acc[k4 * 4 + 1]);
+                            if (k4 * 4 + 2 < kHeadsMaxA1) acc[k4 * 4 + 2] = fmaf(d.z, hv[u], acc[k4 * 4 + 2]);
+                            if (k4 * 4 + 3 < kHeadsMaxA1) acc[k4 * 4 + 3] = fmaf(d.w, hv[u], acc[k4 * 4 + 3]);
+                        }
+                    }
+                }
+            }
         }
     }
 #pragma unroll
