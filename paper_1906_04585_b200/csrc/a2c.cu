@@ -317,7 +317,12 @@ __global__ void __launch_bounds__(256) heads_fused_kernel(HeadsFusedArgs p) {
 
     // The head weights were last written by the optimiser pass, which lies at least two kernels back, so
     // they are fetched before the wait for the previous kernel.
-    for (int i = tid; i < A * kHeadsH; i += 256) Wsm[i] = P[p.piw + i];
+    if (((p.piw | p.p_stride) & 3) == 0) {   // 16-byte loads when the policy weights are aligned
+        const float4* src = reinterpret_cast<const float4*>(P + p.piw);
+        for (int i = tid; i < A * (kHeadsH / 4); i += 256) reinterpret_cast<float4*>(Wsm)[i] = src[i];
+    } else {
+        for (int i = tid; i < A * kHeadsH; i += 256) Wsm[i] = P[p.piw + i];
+    }
     for (int i = tid; i < kHeadsH; i += 256) Wsm[A * kHeadsH + i] = P[p.vw + i];
     pdl_wait();
     pdl_launch();
@@ -461,6 +466,11 @@ __global__ void __launch_bounds__(256) heads_fused_kernel(HeadsFusedArgs p) {
         }
         const float dvv = 2.0f * p.vf_coef * (v - gt) * invS;
         dsm[r * A1 + A] = dvv;
+        {   // the same numbers as one padded row (dlogits, dvalue, zeros) for the weight-gradient kernel
+            float* row = p.dzv + ((long)g * S + srow) * (kHeadsMaxA1 + 1);
+            for (int k = 0; k < A1; k++) row[k] = dsm[r * A1 + k];
+            for (int k = A1; k < kHeadsMaxA1 + 1; k++) row[k] = 0.0f;
+        }
         p.dvalues[(long)g * S + srow] = dvv;
         p.returns[(long)g * S + srow] = gt;
         p.adv[(long)g * S + srow] = adv;
@@ -587,9 +597,14 @@ __global__ void __launch_bounds__(256) heads_wgrad_tiled_kernel(HeadsBwdArgs a) 
     for (int s0 = 0; s0 < a.rows; s0 += kChunk) {
         const int n = min(kChunk, a.rows - s0);
         __syncthreads();
-        for (int i = tid; i < n * (kHeadsMaxA1 + 1); i += 256) {
-            const int s = i / (kHeadsMaxA1 + 1), k = i - s * (kHeadsMaxA1 + 1);
-            dzs[s][k] = k < A ? dz[(long)(s0 + s) * A + k] : (k == A ? dv[s0 + s] : 0.0f);
+        if (a.dzv) {   // padded rows written by the fused heads kernel: a straight copy
+            const float4* src = reinterpret_cast<const float4*>(a.dzv + ((long)g * a.rows + s0) * (kHeadsMaxA1 + 1));
+            for (int i = tid; i < n * ((kHeadsMaxA1 + 1) / 4); i += 256) reinterpret_cast<float4*>(&dzs[0][0])[i] = src[i];
+        } else {
+            for (int i = tid; i < n * (kHeadsMaxA1 + 1); i += 256) {
+                const int s = i / (kHeadsMaxA1 + 1), k = i - s * (kHeadsMaxA1 + 1);
+                dzs[s][k] = k < A ? dz[(long)(s0 + s) * A + k] : (k == A ? dv[s0 + s] : 0.0f);
+            }
         }
         __syncthreads();
         const int per = (n + 7) / 8;

@@ -108,6 +108,7 @@ struct gala_ctx {
     float *clip = nullptr, *norm = nullptr, *losses = nullptr;
     double *norm_partial = nullptr, *colsum_partial = nullptr;
     unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr, *heads_ticket = nullptr;
+    float* dzv = nullptr;                    // [N][S][20] rows (dlogits, dvalue, zeros) of the fused heads kernel
     float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
     bool fused_heads = false;
     int* error_word = nullptr;
@@ -695,6 +696,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hf.logits = c->logits + (long)agent0 * B * A; hf.values = c->values + (long)agent0 * B;
         hf.returns = la.returns; hf.adv = la.adv; hf.dlogits = la.dlogits; hf.dvalues = la.dvalues;
         hf.losses = la.losses;
+        hf.dzv = c->dzv + (long)agent0 * S * 20;
         hf.dh = c->dh + (long)agent0 * S * kHidden; hf.dh_stride = S * kHidden;
         hf.loss_partial = c->heads_partial + (long)agent0 * c->E * 4;
         hf.ticket = c->heads_ticket + agent0;
@@ -720,6 +722,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         // the chain.
         if ((r = fork()) != GALA_OK) return r;
         if (fused) {
+            hb.dzv = c->dzv + (long)agent0 * S * 20;
             LAUNCH(T_HEADS_BWD, ws, launch_heads_wgrad_tiled(hb, groups, ws));
         } else {
             LAUNCH(T_HEADS_BWD, ws, launch_heads_wgrad(hb, groups, ws));
@@ -1006,6 +1009,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         c->legacy_conv = getenv("GALA_CONV_LEGACY") != nullptr;
         c->fused_heads = heads_fused_supported(c->T, c->E, c->A, kHidden) && getenv("GALA_HEADS_UNFUSED") == nullptr;
         ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
+        ALLOC(c->dzv, (size_t)n * S * 20);
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {

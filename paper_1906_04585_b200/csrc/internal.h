@@ -281,6 +281,7 @@ struct HeadsBwdArgs {
     long piw, pib, vw, vb;
     const float* dlogits; long dlogits_stride;   // [g][S][A]
     const float* dvalues; long dvalues_stride;   // [g][S]
+    const float* dzv;                            // optional [g][S][20]: rows (dlogits, dvalue, zeros), 16-byte aligned
     float* grad; long g_stride;                  // flat gradient (same offsets)
     void* dpre; long dpre_stride; int dpre_bf16; // [g][S][H] dL/d(pre-activation of hidden)
 };
@@ -306,6 +307,7 @@ struct HeadsFusedArgs {
     PtrBatch actions, rewards, dones;     // per agent [T][E]
     float *logits, *values;               // [g][B][A], [g][B]
     float *returns, *adv, *dlogits, *dvalues;   // [g][S], [g][S], [g][S][A], [g][S]
+    float* dzv;                           // [g][S][20]: rows (dlogits, dvalue, zeros) for the weight-gradient kernel
     float* losses;                        // [g][4]
     long B;                               // (T+1)*E
     __nv_bfloat16* dh; long dh_stride;    // [g][S][512]
