@@ -180,6 +180,13 @@ int gala_consensus_distance(gala_ctx* ctx, double* out);
  * When it runs out, or when an in-peer has published nothing newer, gala_gossip returns
  * GALA_ETIMEOUT and has enqueued nothing; the pending gradient stays pending. */
 int gala_set_stale_timeout(gala_ctx* ctx, int timeout_ms);
+/* SM budget of one agent's tensor-core kernels in the per-agent calls (gala_learn, gala_act): at most `ctas`
+ * thread blocks per kernel, so that kernels of several agents' streams run side by side instead of each
+ * taking every SM in turn (Sec. 3: the agents progress independently).  0 or >= 148: no limit (default at
+ * creation: 148 * 8 / n_agents, at least 32, no limit for fewer than 5 agents).  gala_step_sync is not
+ * affected.  Results do not depend on the budget except through the summation order of sliced weight
+ * gradients. */
+int gala_set_agent_ctas(gala_ctx* ctx, int ctas);
 int gala_param_count(const gala_ctx* ctx, long long* d, long long* d_padded);
 /* out = {policy term, mean squared TD error, mean entropy, gradient norm} of the last learn. */
 int gala_losses(gala_ctx* ctx, int agent, float out[4]);

@@ -111,6 +111,8 @@ struct gala_ctx {
     float* dzv = nullptr;                    // [N][S][20] rows (dlogits, dvalue, zeros) of the fused heads kernel
     float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
     bool fused_heads = false;
+    int agent_ctas = 0;                      // SM budget of one agent's kernels in the per-agent calls (0: all)
+    int cur_ctas = 0;                        // budget of the launches being enqueued (0 in the synchronous round)
     int* error_word = nullptr;
     double *cons_partial = nullptr, *cons_out = nullptr;
     unsigned* cons_ticket = nullptr;
@@ -451,14 +453,17 @@ int build_plans(gala_ctx* c) {
     return ok ? GALA_OK : fail(c, GALA_ECUDA, "cuTensorMapEncodeTiled failed while building GEMM descriptors");
 }
 
+
 // Slices of the samples per agent for a weight gradient whose CTAs each own one agent and a slice: chosen so
 // that the CTAs fill the SMs in whole waves.  `fixed` = set-up and epilogue of a CTA in units of one sample.
 int pick_splits(gala_ctx* c, int groups, int S, long count, int fixed) {
     int best = 1;
     long best_cost = -1;
+    const long sms = c->cur_ctas > 0 ? c->cur_ctas : 148;
     for (int sp = 1; sp <= c->max_split && sp <= S; sp++) {
         if (sp > 1 && (S / sp < 4 || sp * count > c->splitk_group_stride)) break;
-        const long waves = ((long)groups * sp + 147) / 148, per = (S + sp - 1) / sp;
+        if (sp > 1 && c->cur_ctas > 0 && (long)groups * sp > sms) break;
+        const long waves = ((long)groups * sp + sms - 1) / sms, per = (S + sp - 1) / sp;
         const long cost = waves * (per + fixed) + (sp > 1 ? 8 : 0);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = sp; }
     }
@@ -486,20 +491,14 @@ int run_conv1_wgrad(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, cu
     return GALA_OK;
 }
 
+
 // conv2 / conv3 weight gradient: slices of the samples per agent chosen so that the CTAs fill the SMs in
 // whole waves; with more than one slice the partial sums go through the fixed-order reduction
 int run_conv_wgrad(gala_ctx* c, const WgradPlan& p, int agent0, int groups, cudaStream_t st) {
     WgradArgs a = p.args;
     const int S = a.samples;
     const long count = (long)(a.variant == WG_CONV2 ? 64 * 512 : 64 * 576);
-    int best = 1;
-    long best_cost = -1;
-    for (int sp = 1; sp <= c->max_split && sp <= S; sp++) {
-        if (sp > 1 && (S / sp < 4 || sp * count > c->splitk_group_stride)) break;
-        const long waves = ((long)groups * sp + 147) / 148, per = (S + sp - 1) / sp;
-        const long cost = waves * (per + 6) + (sp > 1 ? 8 : 0);   // samples per CTA plus fixed costs, in sample units
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = sp; }
-    }
+    const int best = pick_splits(c, groups, S, count, 6);
     a.group0 = agent0; a.groups = groups; a.splits = best;
     if (best == 1) {
         a.out += (long)agent0 * a.out_group_stride;
@@ -520,7 +519,7 @@ int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, c
              const PtrBatch* obs = nullptr) {
     ConvArgs a = p.args;
     if (obs) a.obs = *obs;
-    a.group0 = agent0; a.groups = groups; a.rows = rows;
+    a.group0 = agent0; a.groups = groups; a.rows = rows; a.max_ctas = c->cur_ctas;
     a.out += (long)agent0 * a.out_group_stride;
     if (a.gate_out) a.gate_out += (long)agent0 * a.gate_group_stride;
     if (a.gate_in) a.gate_in += (long)agent0 * a.gate_group_stride;
@@ -530,7 +529,7 @@ int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, c
 
 int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override, cudaStream_t st) {
     GemmArgs a = p.args;
-    a.group0 = agent0; a.groups = groups;
+    a.group0 = agent0; a.groups = groups; a.max_ctas = c->cur_ctas;
     if (m_override > 0) a.M = m_override;
     const bool bf = a.flags & EPI_OUT_BF16;
     a.out = reinterpret_cast<char*>(a.out) + (long)agent0 * a.out_group_stride * (bf ? 2 : 4);
@@ -550,7 +549,7 @@ int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t s
     if (split == 1) return run_plan(c, p, agent0, groups, 0, st);
     GemmArgs a = p.args;
     const long count = (long)p.args.M * p.args.N;
-    a.group0 = agent0; a.groups = groups; a.split_k = split;
+    a.group0 = agent0; a.groups = groups; a.split_k = split; a.max_ctas = c->cur_ctas;
     a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
     a.out_group_stride = c->splitk_group_stride;
     a.out_split_stride = count;
@@ -591,7 +590,7 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         {
             const Plan& p = c->fc_fwd;
             const int tiles = ((rows + 127) / 128) * (kHidden / 128);
-            int split = 296 / (groups * tiles);
+            int split = (c->cur_ctas > 0 ? 2 * c->cur_ctas : 296) / (groups * tiles);
             if (split > 7) split = 7;
             while (split > 1 && (long)split * rows * kHidden > c->splitk_group_stride) split--;
             if (split <= 1) {
@@ -600,7 +599,7 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
             } else {
                 GemmArgs a = p.args;
                 const long count = (long)rows * kHidden;
-                a.group0 = agent0; a.groups = groups; a.M = rows; a.split_k = split;
+                a.group0 = agent0; a.groups = groups; a.M = rows; a.split_k = split; a.max_ctas = c->cur_ctas;
                 a.flags = 0; a.bias = nullptr;
                 a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
                 a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
@@ -1007,6 +1006,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         CK(wgrad_init());
         CK(wgrad1_init());
         c->legacy_conv = getenv("GALA_CONV_LEGACY") != nullptr;
+        if (n >= 5) c->agent_ctas = 148 * 8 / n < 32 ? 32 : 148 * 8 / n;   // measured on 64 agents: 32 beats 16 and 64
         c->fused_heads = heads_fused_supported(c->T, c->E, c->A, kHidden) && getenv("GALA_HEADS_UNFUSED") == nullptr;
         ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
         ALLOC(c->dzv, (size_t)n * S * 20);
@@ -1096,7 +1096,9 @@ int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int
     Agent& ag = c->agents[agent];
     PtrBatch pb{};
     pb.p[0] = obs;
+    c->cur_ctas = c->agent_ctas;
     int r = forward(c, agent, 1, pb, c->E, ag.stream, c->legacy_conv ? ag.stream : nullptr);
+    c->cur_ctas = 0;
     if (r != GALA_OK) return r;
     if (actions)
         LAUNCH(T_SAMPLE, ag.stream, launch_sample(c->logits + (long)agent * c->B * c->A, uniforms, actions, c->E, c->A, ag.stream));
@@ -1115,7 +1117,10 @@ int gala_learn(gala_ctx* c, int agent, const gala_rollout* ro) {
         if (r != GALA_OK) return r;
         ag.round++;
     }
-    return learn_range(c, agent, 1, ro, ag.stream);
+    c->cur_ctas = c->agent_ctas;
+    int r = learn_range(c, agent, 1, ro, ag.stream);
+    c->cur_ctas = 0;
+    return r;
 }
 
 int gala_gossip(gala_ctx* c, int agent) {
@@ -1262,6 +1267,12 @@ int gala_consensus_distance(gala_ctx* c, double* out) {
     double sq = 0.0;
     CK(cudaMemcpy(&sq, c->cons_out, sizeof sq, cudaMemcpyDeviceToHost));
     *out = std::sqrt(sq);
+    return GALA_OK;
+}
+
+int gala_set_agent_ctas(gala_ctx* c, int ctas) {
+    if (!c || ctas < 0) return fail(c, GALA_EINVAL, "gala_set_agent_ctas: negative budget");
+    c->agent_ctas = ctas >= 148 ? 0 : ctas;
     return GALA_OK;
 }
 

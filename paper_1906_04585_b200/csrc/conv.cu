@@ -546,7 +546,8 @@ static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, con
     if (units <= 0) return cudaSuccess;
     if (units > 0x7fffffffL) return cudaErrorInvalidValue;
     const size_t smem = (size_t)fixed + (size_t)nst * STAGE;
-    const int grid = (int)(units < 148 ? units : 148);
+    int grid = (int)(units < 148 ? units : 148);
+    if (a.max_ctas > 0 && grid > a.max_ctas) grid = a.max_ctas;
     (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), dim3(V == CV_CONV1_FWD ? kConv1Threads : kConvThreads), smem, st, x, w, a, nst, units);
     return cudaGetLastError();
 }

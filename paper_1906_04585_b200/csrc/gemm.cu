@@ -687,7 +687,8 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     int per_sm = (int)((220u * 1024u) / smem);
     if (per_sm > 2) per_sm = 2;   // 2 x 256 tensor-memory columns is all an SM has
     if (per_sm < 1) per_sm = 1;
-    const long cap = 148L * per_sm;
+    long cap = 148L * per_sm;
+    if (a.max_ctas > 0 && cap > (long)a.max_ctas * per_sm) cap = (long)a.max_ctas * per_sm;
     const int grid = (int)(total < cap ? total : cap);
     (void)launch_pdl(gemm_tcgen05_kernel, dim3(grid), dim3(192), smem, st, A.map, B.map, a, A.mn_major, B.mn_major, total, mt, nt);
     return cudaGetLastError();

@@ -92,6 +92,7 @@ struct GemmArgs {
     const __nv_bfloat16* mask;  // [m][n] with the output's ldc; group g at mask + g*mask_group_stride
     long mask_group_stride;
     int* error_word;       // device int, set non-zero when a bounded wait runs out
+    int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
     // Tiling (set by the caller for the convolution modes, filled with defaults by launch_gemm)
     int tile_rows;         // rows of D per M tile (<= 128; default 128)
     int k_steps;           // number of K steps of the whole reduction (default ceil(K/64))
@@ -166,6 +167,7 @@ struct ConvArgs {
     const uint32_t* gate_in;
     long gate_group_stride;      // words per agent
     int* error_word;
+    int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
     PtrBatch obs;          // conv1 forward: the agents' uint8 frames [rows][84][84][4], 16-byte aligned
 };
 cudaError_t conv_init();
