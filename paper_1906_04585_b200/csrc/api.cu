@@ -132,7 +132,7 @@ struct gala_ctx {
     ConvPlan cfwd[3], cdgrad[3];
     WgradPlan cwgrad[3];
     Wgrad1Plan cwgrad1;
-    uint32_t* gate[2] = {nullptr, nullptr};   // ReLU gate bits of act[0], act[1]
+    uint32_t* gate[3] = {nullptr, nullptr, nullptr};   // ReLU gate bits of act[0..2]
     bool legacy_conv = false;
 };
 
@@ -399,8 +399,13 @@ int build_plans(gala_ctx* c) {
         ok &= make_operand(&dg.A, c->dh, 0, S, kHidden, n, kHidden, (uint64_t)S * kHidden, 128);
         ok &= make_operand(&dg.B, c->shadow + c->cl.fcw, 1, kFeat, kHidden, n, kFeat, dp, 128);
         dg.args.M = (int)S; dg.args.N = kFeat; dg.args.K = kHidden; dg.args.block_n = 128;
-        dg.args.flags = EPI_OUT_BF16 | EPI_MASK;
-        dg.args.mask = c->act[2]; dg.args.mask_group_stride = B * kFeat;
+        if (c->legacy_conv) {   // the legacy conv3 forward writes no gate bits: gate on the stored activation itself
+            dg.args.flags = EPI_OUT_BF16 | EPI_MASK;
+            dg.args.mask = c->act[2]; dg.args.mask_group_stride = B * kFeat;
+        } else {                // one gate word per row and 32 columns instead of 64 bytes of activations
+            dg.args.flags = EPI_OUT_BF16 | EPI_GATE;
+            dg.args.gate = c->gate[2]; dg.args.gate_group_stride = B * kFeat / 32;
+        }
         dg.args.out = c->dy[2]; dg.args.out_group_stride = S * kFeat; dg.args.ldc = kFeat;
     }
     for (int l = 0; l < 3; l++) {
@@ -413,7 +418,7 @@ int build_plans(gala_ctx* c) {
         f.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
         f.args.bias = c->x + c->cl.b[l]; f.args.bias_group_stride = dp;
         f.args.out = c->act[l]; f.args.out_group_stride = B * P[l] * CO;
-        if (l < 2) { f.args.gate_out = c->gate[l]; f.args.gate_group_stride = B * P[l] * CO / 32; }
+        f.args.gate_out = c->gate[l]; f.args.gate_group_stride = B * P[l] * CO / 32;
         f.args.error_word = c->error_word;
         const void* xin = l == 0 ? (const void*)c->frames : (const void*)c->act[l - 1];
         ok &= make_conv_maps(f.args.variant, &f.x, &f.w, xin, (uint64_t)n * B, c->shadow + c->cl.w[l], n, dp);
@@ -534,6 +539,7 @@ int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override,
     const bool bf = a.flags & EPI_OUT_BF16;
     a.out = reinterpret_cast<char*>(a.out) + (long)agent0 * a.out_group_stride * (bf ? 2 : 4);
     if (a.mask) a.mask += (long)agent0 * a.mask_group_stride;
+    if (a.gate) a.gate += (long)agent0 * a.gate_group_stride;
     LAUNCH(p.tag, st, launch_gemm(p.A, p.B, a, st));
     return GALA_OK;
 }
@@ -1014,7 +1020,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {
             ALLOC(c->act[l], (size_t)n * B * P[l] * kConvCout[l]);
-            if (l < 2) ALLOC(c->gate[l], (size_t)n * B * P[l] * kConvCout[l] / 32);
+            ALLOC(c->gate[l], (size_t)n * B * P[l] * kConvCout[l] / 32);
             ALLOC(c->dy[l], (size_t)n * S * P[l] * kConvCout[l]);
         }
         ALLOC(c->frames, (size_t)n * B * kFramePix);

@@ -296,6 +296,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, local++) {
             const TileCoord t = decode_tile(p, tile, mt, nt);
             const int ab = local & 1;
+            // gate words of this thread's row (one per 32 columns): they depend only on the tile, so they are
+            // fetched before the wait for the MMAs
+            uint32_t gw0 = 0xffffffffu, gw1 = 0xffffffffu, gw2 = 0xffffffffu, gw3 = 0xffffffffu;
+            if (p.flags & EPI_GATE) {
+                const int m = t.m0 + q * 32 + lane;
+                if (m < p.M) {
+                    const uint32_t* gp = p.gate + (long)t.gz * p.gate_group_stride + (long)m * (p.N >> 5) + (t.n0 >> 5);
+                    const int nw = (p.N - t.n0) >> 5;
+                    if (nw > 0) gw0 = __ldg(gp);
+                    if (nw > 1 && BN > 32) gw1 = __ldg(gp + 1);
+                    if (nw > 2 && BN > 64) gw2 = __ldg(gp + 2);
+                    if (nw > 3 && BN > 96) gw3 = __ldg(gp + 3);
+                }
+            }
             if (!mbar_wait(&acc_full[ab], ((uint32_t)local >> 1) & 1u, &abort_flag)) break;
             tcgen05_fence_after();
             const uint32_t tmem_acc = tmem_base + (uint32_t)ab * acc_cols;
@@ -319,6 +333,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; j++) r[j] = 0u;
+                }
+                if (p.flags & EPI_GATE) {
+                    const uint32_t gw = c0 == 0 ? gw0 : c0 == 32 ? gw1 : c0 == 64 ? gw2 : gw3;
+#pragma unroll
+                    for (int j = 0; j < 32; j++)
+                        if (!((gw >> j) & 1u)) r[j] = 0u;
                 }
                 const int nb = t.n0 + c0;
                 if (mw >= p.M || q * 32 >= p.tile_rows || nb >= p.N) continue;   // warp-uniform
@@ -629,6 +649,8 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     if (args.block_n != 32 && args.block_n != 64 && args.block_n != 128) return cudaErrorInvalidValue;
     if (B.mn_major && args.block_n < 64 && !(args.conv_mode != CONV_NONE && args.conv_layer == 0)) return cudaErrorInvalidValue;
     if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
+    if ((args.flags & EPI_GATE) && (!args.gate || (args.N & 31) || (args.flags & (EPI_TRANSPOSE | EPI_ROWMAP_S2))))
+        return cudaErrorInvalidValue;
     GemmArgs a = args;
     if (a.conv_mode == CONV_NONE) {
         a.tile_rows = BM;

@@ -70,6 +70,7 @@ enum EpilogueFlags : int {
     EPI_RELU = 2,        // max(.,0) after scale and bias
     EPI_TRANSPOSE = 4,   // store D[m][n] at out[n*ldc + m]
     EPI_MASK = 8,        // multiply by (mask[m][n] > 0), mask bf16 with the output's layout
+    EPI_GATE = 32,       // zero where bit n % 32 of gate[m][n / 32] is clear (ReLU gate bits; N a multiple of 32)
     EPI_ROWMAP_S2 = 16   // rows are (sample, parity class, a, c) of a stride-2 data gradient: row r of tile
                          // (sample, class) goes to pixel (2a + class/2, 2c + class%2) of the 20x20 input grid
 };
@@ -91,6 +92,8 @@ struct GemmArgs {
     long ldc;
     const __nv_bfloat16* mask;  // [m][n] with the output's ldc; group g at mask + g*mask_group_stride
     long mask_group_stride;
+    const uint32_t* gate;       // [m][N / 32] words; group g at gate + g*gate_group_stride
+    long gate_group_stride;
     int* error_word;       // device int, set non-zero when a bounded wait runs out
     int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
     // Tiling (set by the caller for the convolution modes, filled with defaults by launch_gemm)
