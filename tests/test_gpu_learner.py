@@ -164,12 +164,14 @@ def test_act_sampling_matches_oracle():
     L.close()
 
 
-def _async_replay(w, order, tol_net, tol_params, mode="elementwise"):
+def _async_replay(w, order, tol_net, tol_params, mode="elementwise", agent_ctas=None):
     """Drive learn/gossip per agent in the given order, waiting after every call so that the
     schedule is deterministic, and replay the library's own (peer, version) log in the oracle."""
     B, LM = _mods()
     net = oracle_net(w)
     L = make_learner(w)
+    if agent_ctas is not None:
+        B.gala_set_agent_ctas(L.ctx, agent_ctas)
     ohp = oracle_hp(L.hp)
     X, V = seed_identical(L, w, net)
     n = w.n_agents
@@ -321,3 +323,26 @@ def test_conv_gradient_close_to_exact_arithmetic():
 def test_async_replay_conv():
     w = GI.WORKLOADS[1].scaled(n_agents=4, n_envs=2, n_steps=3)
     _async_replay(w, [0, 1, 0, 2, 3, 1, 0, 3], TOL_BF16, TOL_BF16, mode="update")
+
+
+def test_async_replay_conv_with_sm_budget():
+    # per-agent kernels limited to a few thread blocks (so that several agents' streams share the SMs):
+    # same results, the work units are only spread over fewer blocks
+    w = GI.WORKLOADS[1].scaled(n_agents=4, n_envs=2, n_steps=3)
+    _async_replay(w, [0, 1, 0, 2, 3, 1, 0, 3], TOL_BF16, TOL_BF16, mode="update", agent_ctas=5)
+
+
+def test_conv_sync_round_unfused_heads(monkeypatch):
+    # the separate heads / objective / head-gradient kernels (used when a rollout is too long for the fused
+    # kernel's shared memory) against the same oracle
+    monkeypatch.setenv("GALA_HEADS_UNFUSED", "1")
+    w = GI.WORKLOADS[2].scaled(n_agents=2, n_envs=3, n_steps=4)
+    _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
+
+
+def test_conv_sync_round_legacy_products(monkeypatch):
+    # the previous generation of the convolution products (one TMA box per kernel offset, bf16 frame copies)
+    # is kept as an independent cross-check of the resident-input kernels
+    monkeypatch.setenv("GALA_CONV_LEGACY", "1")
+    w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=3, n_steps=2)
+    _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
