@@ -187,6 +187,14 @@ int gala_set_stale_timeout(gala_ctx* ctx, int timeout_ms);
  * affected.  Results do not depend on the budget except through the summation order of sliced weight
  * gradients. */
 int gala_set_agent_ctas(gala_ctx* ctx, int ctas);
+/* CUDA-graph replay of the learner step (default on).  The first gala_learn / gala_step_sync with a given set
+ * of rollout buffers launches its kernels one by one; the second captures the same launches into a graph; from
+ * then on the step is one graph launch (the kernels and their results are the same).  A caller that reuses its
+ * rollout buffers, as an actor that writes each rollout into the same device memory does, gets this for every
+ * step; one that passes new buffers every time never pays for a capture.  Up to 512 distinct buffer sets are
+ * remembered.  Off while per-class timing (gala_profile_enable) of a kernel inside the step is on.  If the
+ * application itself captures the library's streams into a graph, switch this off first. */
+int gala_set_graphs(gala_ctx* ctx, int on);
 int gala_param_count(const gala_ctx* ctx, long long* d, long long* d_padded);
 /* out = {policy term, mean squared TD error, mean entropy, gradient norm} of the last learn. */
 int gala_losses(gala_ctx* ctx, int agent, float out[4]);

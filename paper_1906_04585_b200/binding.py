@@ -57,7 +57,7 @@ EXPORTS = (
     "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync", "gala_kernel_classes",
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
     "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_set_stale_timeout",
-    "gala_set_agent_ctas",
+    "gala_set_agent_ctas", "gala_set_graphs",
 )
 
 _lib = None
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
             "gala_consensus_distance": (i, [vp, C.POINTER(C.c_double)]),
             "gala_set_stale_timeout": (i, [vp, i]),
             "gala_set_agent_ctas": (i, [vp, i]),
+            "gala_set_graphs": (i, [vp, i]),
             "gala_step_sync": (i, [vp, C.POINTER(gala_rollout)]),
             "gala_sync_agent": (i, [vp, i, i]),
             "gala_sync_all": (i, [vp, i]),
@@ -176,6 +177,10 @@ def gala_consensus_distance(ctx) -> float:
     out = C.c_double()
     _check(ctx, lib().gala_consensus_distance(ctx, C.byref(out)))
     return out.value
+
+
+def gala_set_graphs(ctx, on: bool):
+    _check(ctx, lib().gala_set_graphs(ctx, 1 if on else 0))
 
 
 def gala_set_agent_ctas(ctx, ctas: int):

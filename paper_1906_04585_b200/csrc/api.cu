@@ -74,6 +74,16 @@ const char* const kTagNames[T_COUNT] = {
 
 struct TimedLaunch { int tag; cudaEvent_t beg, end; };
 
+// The kernels of one learner step (forward, objective, backward, norm) for a given set of rollout buffers,
+// captured once as a CUDA graph: replaying it costs one launch on the host instead of ~17.
+struct StepGraph {
+    std::vector<const void*> key;   // streams, first agent, count, SM budget, the rollouts' pointers
+    cudaGraphExec_t exec = nullptr;
+    bool failed = false;            // capture or instantiation did not work: launch directly
+    long long launches = 0;         // kernels inside
+    long long tag_launches[T_COUNT] = {};
+};
+
 }  // namespace
 
 struct gala_ctx {
@@ -111,6 +121,8 @@ struct gala_ctx {
     float* dzv = nullptr;                    // [N][S][20] rows (dlogits, dvalue, zeros) of the fused heads kernel
     float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
     bool fused_heads = false;
+    bool use_graphs = true;                  // replay a learner step whose rollout buffers were seen before as a graph
+    std::vector<StepGraph> graphs;
     int agent_ctas = 0;                      // SM budget of one agent's kernels in the per-agent calls (0: all)
     int cur_ctas = 0;                        // budget of the launches being enqueued (0 in the synchronous round)
     int* error_word = nullptr;
@@ -799,6 +811,72 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
     return GALA_OK;
 }
 
+// learn_range through the graph cache.  First time a set of rollout buffers is seen: direct launches.  Second
+// time: the same launches are captured into a graph, which is instantiated and launched.  From then on: one
+// graph launch.  Per-class timing of a kernel inside the step and the legacy products go the direct way.
+constexpr size_t kMaxStepGraphs = 512;
+int learn_range_cached(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cudaStream_t st,
+                       cudaStream_t side = nullptr) {
+    // per-class timing brackets launches with events: not inside a graph (the optimiser / gossip pass and the
+    // sampling kernel lie outside this step, so timing only those does not matter)
+    const unsigned long long outside = (1ull << T_SWEEP_SYNC) | (1ull << T_SWEEP_AGENT) | (1ull << T_SAMPLE);
+    if (!c->use_graphs || (c->profile_mask & ~outside) != 0 || c->legacy_conv)
+        return learn_range(c, agent0, groups, ro, st, side);
+    std::vector<const void*> key;
+    key.reserve(6 + 4 * (size_t)groups);
+    key.push_back(st); key.push_back(side);
+    key.push_back(reinterpret_cast<const void*>((uintptr_t)agent0));
+    key.push_back(reinterpret_cast<const void*>((uintptr_t)groups));
+    key.push_back(reinterpret_cast<const void*>((uintptr_t)c->cur_ctas));
+    for (int i = 0; i < groups; i++) {
+        key.push_back(ro[i].obs); key.push_back(ro[i].actions); key.push_back(ro[i].rewards); key.push_back(ro[i].dones);
+    }
+    StepGraph* g = nullptr;
+    for (StepGraph& e : c->graphs)
+        if (e.key == key) { g = &e; break; }
+    if (!g) {
+        if (c->graphs.size() < kMaxStepGraphs) { c->graphs.emplace_back(); c->graphs.back().key = std::move(key); }
+        return learn_range(c, agent0, groups, ro, st, side);
+    }
+    if (g->failed) return learn_range(c, agent0, groups, ro, st, side);
+    if (!g->exec) {
+        if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+            (void)cudaGetLastError();
+            g->failed = true;
+            return learn_range(c, agent0, groups, ro, st, side);
+        }
+        const long long l0 = c->launches;
+        long long t0[T_COUNT];
+        for (int k = 0; k < T_COUNT; k++) t0[k] = c->tag_launches[k];
+        const int r = learn_range(c, agent0, groups, ro, st, side);   // enqueues nothing: the launches are recorded
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(st, &graph);
+        if (r == GALA_OK && e == cudaSuccess && graph) e = cudaGraphInstantiate(&g->exec, graph, 0);
+        if (graph) cudaGraphDestroy(graph);
+        if (r != GALA_OK || e != cudaSuccess || !g->exec) {
+            (void)cudaGetLastError();
+            g->failed = true; g->exec = nullptr;
+            c->launches = l0;
+            for (int k = 0; k < T_COUNT; k++) c->tag_launches[k] = t0[k];
+            if (r != GALA_OK) return r;
+            for (int i = 0; i < groups; i++) c->agents[agent0 + i].frames -= c->S;   // counted again below
+            return learn_range(c, agent0, groups, ro, st, side);
+        }
+        g->launches = c->launches - l0;
+        for (int k = 0; k < T_COUNT; k++) g->tag_launches[k] = c->tag_launches[k] - t0[k];
+        CK(cudaGraphLaunch(g->exec, st));
+        return GALA_OK;   // learn_range has already updated the host-side state for this step
+    }
+    CK(cudaGraphLaunch(g->exec, st));
+    c->launches += g->launches;
+    for (int k = 0; k < T_COUNT; k++) c->tag_launches[k] += g->tag_launches[k];
+    for (int i = 0; i < groups; i++) {
+        c->agents[agent0 + i].pending = true;
+        c->agents[agent0 + i].frames += c->S;
+    }
+    return GALA_OK;
+}
+
 // Newest snapshot version of agent j whose writing sweep has completed (0: none usable).
 long long usable_version(gala_ctx* c, int j) {
     Agent& a = c->agents[j];
@@ -1084,6 +1162,7 @@ int gala_destroy(gala_ctx* c) {
         if (a.sweep_done) cudaEventDestroy(a.sweep_done);
         if (a.fence) cudaEventDestroy(a.fence);
     }
+    for (StepGraph& g : c->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
     if (c->side_stream) cudaStreamDestroy(c->side_stream);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
@@ -1124,7 +1203,7 @@ int gala_learn(gala_ctx* c, int agent, const gala_rollout* ro) {
         ag.round++;
     }
     c->cur_ctas = c->agent_ctas;
-    int r = learn_range(c, agent, 1, ro, ag.stream);
+    int r = learn_range_cached(c, agent, 1, ro, ag.stream);
     c->cur_ctas = 0;
     return r;
 }
@@ -1163,7 +1242,7 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
     if (ros) {
         for (int a0 = 0; a0 < n; a0 += kBatch) {
             const int cnt = n - a0 < kBatch ? n - a0 : kBatch;
-            int r = learn_range(c, a0, cnt, ros + a0, st, c->side_stream);
+            int r = learn_range_cached(c, a0, cnt, ros + a0, st, c->side_stream);
             if (r != GALA_OK) return r;
         }
     }
@@ -1273,6 +1352,12 @@ int gala_consensus_distance(gala_ctx* c, double* out) {
     double sq = 0.0;
     CK(cudaMemcpy(&sq, c->cons_out, sizeof sq, cudaMemcpyDeviceToHost));
     *out = std::sqrt(sq);
+    return GALA_OK;
+}
+
+int gala_set_graphs(gala_ctx* c, int on) {
+    if (!c) return GALA_EINVAL;
+    c->use_graphs = on != 0;
     return GALA_OK;
 }
 
