@@ -198,6 +198,9 @@ int gala_set_graphs(gala_ctx* ctx, int on);
 int gala_param_count(const gala_ctx* ctx, long long* d, long long* d_padded);
 /* out = {policy term, mean squared TD error, mean entropy, gradient norm} of the last learn. */
 int gala_losses(gala_ctx* ctx, int agent, float out[4]);
+/* The same four numbers for every agent, out[agent][4] (host memory, 4 * n_agents floats): one wait and two
+ * copies instead of two per agent. */
+int gala_losses_all(gala_ctx* ctx, float* out);
 /* out = {frames, rounds, mixes, skipped mixes, staleness sum, staleness max, published version,
  *        gossip steps that waited because of the staleness bound} */
 int gala_stats(gala_ctx* ctx, int agent, long long out[8]);

@@ -57,7 +57,7 @@ EXPORTS = (
     "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync", "gala_kernel_classes",
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
     "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_set_stale_timeout",
-    "gala_set_agent_ctas", "gala_set_graphs",
+    "gala_set_agent_ctas", "gala_set_graphs", "gala_losses_all",
 )
 
 _lib = None
@@ -94,6 +94,7 @@ def lib() -> C.CDLL:
             "gala_set_grad": (i, [vp, i, vp, f]),
             "gala_param_count": (i, [vp, C.POINTER(ll), C.POINTER(ll)]),
             "gala_losses": (i, [vp, i, C.POINTER(f)]),
+            "gala_losses_all": (i, [vp, C.POINTER(f)]),
             "gala_stats": (i, [vp, i, C.POINTER(ll)]),
             "gala_last_mix": (i, [vp, i, C.POINTER(i), C.POINTER(ll), C.POINTER(i), C.POINTER(i)]),
             "gala_get_snapshot": (i, [vp, i, ll, vp]),
@@ -238,6 +239,12 @@ def gala_losses(ctx, agent: int):
     out = (C.c_float * 4)()
     _check(ctx, lib().gala_losses(ctx, agent, out))
     return [out[j] for j in range(4)]
+
+
+def gala_losses_all(ctx, n_agents: int) -> np.ndarray:
+    out = np.empty((n_agents, 4), dtype=np.float32)
+    _check(ctx, lib().gala_losses_all(ctx, out.ctypes.data_as(C.POINTER(C.c_float))))
+    return out
 
 
 def gala_stats(ctx, agent: int):

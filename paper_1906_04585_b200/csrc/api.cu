@@ -1389,6 +1389,17 @@ int gala_losses(gala_ctx* c, int agent, float out[4]) {
     return GALA_OK;
 }
 
+int gala_losses_all(gala_ctx* c, float* out) {
+    if (!c || !out) return fail(c, GALA_EINVAL, "gala_losses_all: bad argument");
+    CK(cudaStreamSynchronize(c->main_stream));
+    for (Agent& a : c->agents) CK(cudaStreamSynchronize(a.stream));
+    std::vector<float> nrm(c->n);
+    CK(cudaMemcpy(out, c->losses, (size_t)c->n * 4 * sizeof(float), cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(nrm.data(), c->norm, (size_t)c->n * sizeof(float), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < c->n; i++) out[4 * i + 3] = nrm[i];
+    return GALA_OK;
+}
+
 int gala_stats(gala_ctx* c, int agent, long long out[8]) {
     if (!valid_agent(c, agent) || !out) return GALA_EINVAL;
     const Agent& a = c->agents[agent];

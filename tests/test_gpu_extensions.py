@@ -117,3 +117,41 @@ def test_staleness_bound_waits_for_the_in_peer():
     L.gossip(0)                         # the snapshot has landed meanwhile
     assert B.gala_last_mix(L.ctx, 0)[2]
     L.close()
+
+
+def test_losses_all_agrees_with_per_agent_reads_and_graph_replay_repeats_the_step():
+    """Three rounds on the SAME rollout buffers from the same state: the first is launched kernel by kernel, the
+    second is captured into a graph, the third replays it.  All three must give the same gradient bit for
+    bit, and the batched read of the losses must equal the per-agent reads."""
+    from paper_1906_04585_b200 import binding as B, learner as LM
+    w = GI.WORKLOADS[1].scaled(n_agents=3, n_envs=2, n_steps=3)
+    L = _learner(w)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    dev = [LM.DeviceRollout(GI.rollout(w, i, 0)) for i in range(w.n_agents)]
+    grads, losses, counted = [], [], []
+    for k in range(3):
+        for i in range(w.n_agents):
+            L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32), rnd=0)
+        n0 = B.gala_launch_count(L.ctx)
+        L.step_sync(dev)
+        L.sync()
+        counted.append(B.gala_launch_count(L.ctx) - n0)
+        grads.append([L.get_grad(i) for i in range(w.n_agents)])
+        la = B.gala_losses_all(L.ctx, w.n_agents)
+        for i in range(w.n_agents):
+            np.testing.assert_array_equal(la[i], np.array(B.gala_losses(L.ctx, i), np.float32))
+        losses.append(la.copy())
+    assert counted[0] > 10 and counted[1] == counted[0] and counted[2] == counted[0]   # replayed kernels are counted too
+    for k in (1, 2):
+        np.testing.assert_array_equal(losses[k], losses[0])
+        for i in range(w.n_agents):
+            np.testing.assert_array_equal(grads[k][i], grads[0][i])
+    # and with the replay switched off
+    B.gala_set_graphs(L.ctx, False)
+    for i in range(w.n_agents):
+        L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32), rnd=0)
+    L.step_sync(dev)
+    L.sync()
+    for i in range(w.n_agents):
+        np.testing.assert_array_equal(L.get_grad(i), grads[0][i])
+    L.close()
