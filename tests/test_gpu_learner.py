@@ -346,3 +346,11 @@ def test_conv_sync_round_legacy_products(monkeypatch):
     monkeypatch.setenv("GALA_CONV_LEGACY", "1")
     w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=3, n_steps=2)
     _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
+
+
+@pytest.mark.parametrize("n_agents,n_envs,n_steps,peers", [(1, 1, 1, 1), (3, 1, 34, 2), (2, 5, 1, 1)])
+def test_conv_degenerate_shapes(n_agents, n_envs, n_steps, peers):
+    # one agent (no in-peer differs from itself), one environment, one step; a rollout longer than a warp
+    # (the return scan runs in chunks of 32 steps); a single step with several environments
+    w = GI.WORKLOADS[1].scaled(n_agents=n_agents, n_envs=n_envs, n_steps=n_steps, topo_peers=peers)
+    _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
