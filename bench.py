@@ -436,6 +436,22 @@ def run_ours(args):
         a2c_ms = e0.elapsed_time(e1) / 20
         L2.close()
         del ext2
+        # closed actor loop: every agent acts T times on the synthetic environment, learns and gossips, nothing
+        # crosses the host; timed by the host clock between two synchronisations
+        loop_iters = 10
+        for i in range(w.n_agents):
+            B.gala_actor_loop(L.ctx, i, 2, 12345)
+        L.sync()
+        t0 = time.perf_counter()
+        for _ in range(loop_iters):
+            for i in range(w.n_agents):
+                B.gala_actor_loop(L.ctx, i, 1, 12345)
+        L.sync()
+        loop_s = time.perf_counter() - t0
+        line["closed_loop"] = dict(frames_per_s=w.frames_per_round * loop_iters / loop_s,
+                                   ms_per_round=1e3 * loop_s / loop_iters,
+                                   note="act x T + environment step x T + learn + gossip per agent on its own stream, "
+                                        "synthetic on-GPU environment, host clock")
         line["extras"] = dict(consensus_distance=dist, consensus_call_ms=cons_ms,
                               consensus_bytes=int(w.n_agents * L.d * 4),
                               allreduce_a2c_ms_per_round=a2c_ms,

@@ -151,3 +151,44 @@ def sweep_state(n_agents: int, d: int, seed: int, rnd: int = 0):
          * np.float32(1e-3))
     v = _rng(seed, (_S_SQ << 40) + 1).random(size=(n_agents, d), dtype=np.float32) * np.float32(1e-4)
     return x, g, v
+
+
+# ----------------------------------------------------------------------------- synthetic environment
+# Counter-based stand-in for the simulators in the closed actor loop: a pure function of
+# (seed, agent, environment, step) on the SplitMix64 output function.  No arithmetic of the method
+# lives here; the CUDA library has its own statement of the same definition.
+_M64 = np.uint64(0xFFFFFFFFFFFFFFFF)
+
+
+def _sm64(z: np.ndarray) -> np.ndarray:
+    z = np.asarray(z, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        z = z + np.uint64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+    return z ^ (z >> np.uint64(31))
+
+
+def synthetic_env(seed: int, agent: int, n_envs: int, step: int, n_actions: int, frames: bool, obs_dim: int = 8,
+                  actions: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """Observation [E,...] and action-draw uniform [E] of `step`; with `actions` [E] also the reward and the
+    done flag of the transition taken at `step`."""
+    with np.errstate(over="ignore"):
+        env = np.arange(n_envs, dtype=np.uint64)
+        base = _sm64(_sm64(_sm64(np.uint64(seed & 0xFFFFFFFFFFFFFFFF) + np.uint64(agent)) + env) + np.uint64(step))
+        out = {}
+        out["uniforms"] = ((_sm64(base + (np.uint64(3) << np.uint64(56))) >> np.uint64(40)).astype(np.float32)
+                           * np.float32(2.0 ** -24))
+        if frames:
+            n8 = 84 * 84 * 4 // 8
+            words = _sm64(base[:, None] + np.arange(n8, dtype=np.uint64)[None, :])
+            out["obs"] = words.view(np.uint8).reshape(n_envs, 84, 84, 4)      # little-endian: byte j%8 of word j/8
+        else:
+            h = _sm64(base[:, None] + np.arange(obs_dim, dtype=np.uint64)[None, :]) >> np.uint64(40)
+            out["obs"] = ((h.astype(np.float32) * np.float32(2.0 ** -23) - np.float32(1.0)) * np.float32(1.7320508))
+        if actions is not None:
+            hr = _sm64(base + (np.uint64(1) << np.uint64(56)))
+            hd = _sm64(base + (np.uint64(2) << np.uint64(56))) >> np.uint64(40)
+            out["rewards"] = ((hr % np.uint64(n_actions)).astype(np.int64) == np.asarray(actions, np.int64)).astype(np.float32)
+            out["dones"] = (hd < np.uint64(167772)).astype(np.uint8)
+    return out

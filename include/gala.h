@@ -187,6 +187,22 @@ int gala_set_stale_timeout(gala_ctx* ctx, int timeout_ms);
  * affected.  Results do not depend on the budget except through the summation order of sliced weight
  * gradients. */
 int gala_set_agent_ctas(gala_ctx* ctx, int ctas);
+/* Closed actor loop for one agent, enqueued on its stream without a host wait (Algorithm 1, whole loop body):
+ * `iterations` times { T times: act on the current observations of the agent's E environments, step the
+ * environments with the sampled actions and store the transition; then gala_learn on the stored rollout and
+ * gala_gossip }.  The environments are a synthetic stand-in for the paper's simulators (which run on CPUs and
+ * are no part of this library): a counter-based function of (env_seed, agent, environment, step), defined next
+ * to its kernel in csrc/env.cu and restated in gala_inputs.synthetic_env: observations (uint8 frames or float
+ * vectors) and the uniform for the action draw depend on the step only, reward = 1 when the action equals a
+ * hidden per-step target, done with probability 0.01.  Steps are numbered per agent from 0 and continue over
+ * calls.  The rollout buffers belong to the library (allocated by the first call for an agent).  Returns as
+ * gala_learn / gala_gossip do (GALA_ETIMEOUT from a staleness-bounded gossip step ends the loop early). */
+int gala_actor_loop(gala_ctx* ctx, int agent, int iterations, unsigned long long env_seed);
+/* Waits for the agent's stream and copies the rollout of its last loop iteration to HOST memory (any pointer
+ * may be NULL): obs [T+1][E][...], actions [T][E], rewards [T][E], dones [T][E]; *next_step = number of
+ * environment steps taken so far. */
+int gala_actor_read(gala_ctx* ctx, int agent, void* obs, int* actions, float* rewards, unsigned char* dones,
+                    long long* next_step);
 /* CUDA-graph replay of the learner step (default on).  The first gala_learn / gala_step_sync with a given set
  * of rollout buffers launches its kernels one by one; the second captures the same launches into a graph; from
  * then on the step is one graph launch (the kernels and their results are the same).  A caller that reuses its

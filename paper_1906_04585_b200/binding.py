@@ -58,6 +58,7 @@ EXPORTS = (
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
     "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_set_stale_timeout",
     "gala_set_agent_ctas", "gala_set_graphs", "gala_losses_all",
+    "gala_actor_loop", "gala_actor_read",
 )
 
 _lib = None
@@ -85,6 +86,8 @@ def lib() -> C.CDLL:
             "gala_set_stale_timeout": (i, [vp, i]),
             "gala_set_agent_ctas": (i, [vp, i]),
             "gala_set_graphs": (i, [vp, i]),
+            "gala_actor_loop": (i, [vp, i, i, C.c_ulonglong]),
+            "gala_actor_read": (i, [vp, i, vp, vp, vp, vp, C.POINTER(C.c_longlong)]),
             "gala_step_sync": (i, [vp, C.POINTER(gala_rollout)]),
             "gala_sync_agent": (i, [vp, i, i]),
             "gala_sync_all": (i, [vp, i]),
@@ -178,6 +181,22 @@ def gala_consensus_distance(ctx) -> float:
     out = C.c_double()
     _check(ctx, lib().gala_consensus_distance(ctx, C.byref(out)))
     return out.value
+
+
+def gala_actor_loop(ctx, agent: int, iterations: int, env_seed: int):
+    _check(ctx, lib().gala_actor_loop(ctx, agent, iterations, env_seed))
+
+
+def gala_actor_read(ctx, agent: int, n_envs: int, n_steps: int, obs_shape, obs_dtype):
+    """Host copies of the agent's last closed-loop rollout: dict(obs, actions, rewards, dones), next step."""
+    obs = np.empty((n_steps + 1, n_envs) + tuple(obs_shape), dtype=obs_dtype)
+    actions = np.empty((n_steps, n_envs), dtype=np.int32)
+    rewards = np.empty((n_steps, n_envs), dtype=np.float32)
+    dones = np.empty((n_steps, n_envs), dtype=np.uint8)
+    nxt = C.c_longlong()
+    _check(ctx, lib().gala_actor_read(ctx, agent, obs.ctypes.data, actions.ctypes.data, rewards.ctypes.data,
+                                      dones.ctypes.data, C.byref(nxt)))
+    return dict(obs=obs, actions=actions, rewards=rewards, dones=dones), int(nxt.value)
 
 
 def gala_set_graphs(ctx, on: bool):

@@ -29,6 +29,10 @@ struct Agent {
     std::vector<long long> consumed;                // newest version consumed from each agent
     std::vector<int> slot_readers[2];               // agents whose sweeps read snapshot slot s
     long long frames = 0, mixes = 0, skipped = 0, stale_sum = 0, stale_max = 0, stale_waits = 0;
+    // closed actor loop: rollout buffers owned by the library and the environment's step counter
+    void* loop_obs = nullptr; int* loop_actions = nullptr; float* loop_rewards = nullptr;
+    unsigned char* loop_dones = nullptr; float* loop_uniforms = nullptr;
+    long long env_step = 0;
     int last_n = 0, last_mixed = 0;
     int last_peers[2] = {0, 0};
     long long last_versions[2] = {0, 0};
@@ -58,7 +62,7 @@ struct ConvPlan {  // one forward or data-gradient convolution (input resident i
 // Kernel classes for launch counting and optional per-class device timing.
 enum Tag : int {
     T_CAST_FRAMES = 0, T_HEADS_FWD, T_LOSS, T_HEADS_BWD, T_COLSUM, T_SPLITK, T_GRAD_NORM,
-    T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST, T_HEADS_FUSED,
+    T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST, T_HEADS_FUSED, T_ENV,
     T_GEMM_CONV_FWD,          // +layer (3)
     T_GEMM_FC_FWD = T_GEMM_CONV_FWD + 3, T_GEMM_FC_WGRAD, T_GEMM_FC_DGRAD,
     T_GEMM_CONV_WGRAD,        // +layer (3)
@@ -67,7 +71,7 @@ enum Tag : int {
 };
 const char* const kTagNames[T_COUNT] = {
     "cast_frames", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "grad_norm",
-    "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16", "heads_fused",
+    "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16", "heads_fused", "env",
     "gemm_conv1_fwd", "gemm_conv2_fwd", "gemm_conv3_fwd", "gemm_fc_fwd", "gemm_fc_wgrad", "gemm_fc_dgrad",
     "gemm_conv1_wgrad", "gemm_conv2_wgrad", "gemm_conv3_wgrad", "gemm_conv1_dgrad", "gemm_conv2_dgrad",
     "gemm_conv3_dgrad"};
@@ -1190,6 +1194,64 @@ int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int
     if (values)
         CK(cudaMemcpyAsync(values, c->values + (long)agent * c->B, c->E * sizeof(float), cudaMemcpyDeviceToDevice,
                            ag.stream));
+    return GALA_OK;
+}
+
+int gala_actor_loop(gala_ctx* c, int agent, int iterations, unsigned long long env_seed) {
+    if (!valid_agent(c, agent) || iterations < 0) return fail(c, GALA_EINVAL, "gala_actor_loop: bad agent or iteration count");
+    if (c->topo.kind == GALA_TOPO_COMPLETE)
+        return fail(c, GALA_ESTATE, "gala_actor_loop: the complete graph (gradient all-reduce) exists only as gala_step_sync");
+    Agent& ag = c->agents[agent];
+    const int T = c->T, E = c->E;
+    const long obs_elems = c->conv ? kFramePix : c->obs_dim;
+    const long obs_bytes = obs_elems * (c->conv ? 1 : 4);
+    if (!ag.loop_obs) {
+        uint8_t* ob = nullptr;
+        ALLOC(ob, (size_t)(T + 1) * E * obs_bytes);
+        ALLOC(ag.loop_actions, (size_t)T * E); ALLOC(ag.loop_rewards, (size_t)T * E);
+        ALLOC(ag.loop_dones, (size_t)T * E); ALLOC(ag.loop_uniforms, (size_t)E);
+        ag.loop_obs = ob;
+    }
+    uint8_t* obs = reinterpret_cast<uint8_t*>(ag.loop_obs);
+    EnvArgs ea{};
+    ea.seed = env_seed; ea.agent = agent; ea.n_actions = c->A;
+    ea.uniforms = ag.loop_uniforms; ea.obs_elems = obs_elems; ea.frames = c->conv ? 1 : 0;
+    for (int it = 0; it < iterations; it++) {
+        const long long s0 = ag.env_step;
+        EnvArgs first = ea;   // the observation the rollout starts from (the environment is a function of the step)
+        first.obs_step = s0; first.obs_out = obs;
+        LAUNCH(T_ENV, ag.stream, launch_env(first, E, ag.stream));
+        for (int t = 0; t < T; t++) {
+            int r = gala_act(c, agent, obs + (long)t * E * obs_bytes, ag.loop_uniforms, ag.loop_actions + (long)t * E, nullptr);
+            if (r != GALA_OK) return r;
+            EnvArgs st = ea;
+            st.step = s0 + t; st.actions = ag.loop_actions + (long)t * E;
+            st.rewards = ag.loop_rewards + (long)t * E; st.dones = ag.loop_dones + (long)t * E;
+            st.obs_step = s0 + t + 1; st.obs_out = obs + (long)(t + 1) * E * obs_bytes;
+            LAUNCH(T_ENV, ag.stream, launch_env(st, E, ag.stream));
+        }
+        gala_rollout ro{obs, ag.loop_actions, ag.loop_rewards, ag.loop_dones};
+        int r = gala_learn(c, agent, &ro);
+        if (r != GALA_OK) return r;
+        if ((r = gala_gossip(c, agent)) != GALA_OK) return r;
+        ag.env_step += T;
+    }
+    return GALA_OK;
+}
+
+int gala_actor_read(gala_ctx* c, int agent, void* obs, int* actions, float* rewards, unsigned char* dones,
+                    long long* next_step) {
+    if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_actor_read: bad agent");
+    Agent& ag = c->agents[agent];
+    if (!ag.loop_obs) return fail(c, GALA_ESTATE, "gala_actor_read: gala_actor_loop has not run for this agent");
+    CK(cudaStreamSynchronize(ag.stream));
+    const long obs_bytes = (c->conv ? kFramePix : (long)c->obs_dim * 4);
+    const size_t TE = (size_t)c->T * c->E;
+    if (obs) CK(cudaMemcpy(obs, ag.loop_obs, (size_t)(c->T + 1) * c->E * obs_bytes, cudaMemcpyDeviceToHost));
+    if (actions) CK(cudaMemcpy(actions, ag.loop_actions, TE * sizeof(int), cudaMemcpyDeviceToHost));
+    if (rewards) CK(cudaMemcpy(rewards, ag.loop_rewards, TE * sizeof(float), cudaMemcpyDeviceToHost));
+    if (dones) CK(cudaMemcpy(dones, ag.loop_dones, TE, cudaMemcpyDeviceToHost));
+    if (next_step) *next_step = ag.env_step;
     return GALA_OK;
 }
 

@@ -332,6 +332,22 @@ struct DenseBwdArgs {
 };
 cudaError_t launch_dense_bwd(const DenseBwdArgs& a, int groups, cudaStream_t st);
 
+// ---------------------------------------------------------------- synthetic environment (env.cu)
+struct EnvArgs {
+    unsigned long long seed;
+    int agent, n_actions;
+    long long step;              // transition whose reward / done flag is produced (if actions != null)
+    const int* actions;          // [E] actions taken at `step`, or null
+    float* rewards;              // [E]
+    unsigned char* dones;        // [E]
+    long long obs_step;          // step whose observation and action-draw uniform are produced (if obs_out != null)
+    void* obs_out;               // [E][obs_elems] uint8 frames or float vectors, or null
+    float* uniforms;             // [E]
+    long obs_elems;              // bytes (frames) or floats (vectors) per environment
+    int frames;                  // 1: uint8 frames, 0: float vectors
+};
+cudaError_t launch_env(const EnvArgs& a, int n_envs, cudaStream_t st);
+
 // ---------------------------------------------------------------- conv lowering
 // uint8 frames -> bf16 (exact), per group [samples][84*84*4]
 cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out_group_stride, int samples, int groups,

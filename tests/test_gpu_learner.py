@@ -354,3 +354,61 @@ def test_conv_degenerate_shapes(n_agents, n_envs, n_steps, peers):
     # (the return scan runs in chunks of 32 steps); a single step with several environments
     w = GI.WORKLOADS[1].scaled(n_agents=n_agents, n_envs=n_envs, n_steps=n_steps, topo_peers=peers)
     _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
+
+
+def _closed_loop(w, iters, tol_net, tol_params, cdf_tol, mode):
+    """Closed actor loop of one agent (no in-peers, so no averaging) against the oracle, one iteration at a time:
+    the environment's observations, rewards and done flags bit for bit; every sampled action equal to the
+    oracle's draw from the same uniform unless that uniform lies within cdf_tol of a boundary of the oracle's
+    CDF; then gradient and parameters as in the synchronous tests, with the library's actions."""
+    B, LM = _mods()
+    assert w.n_agents == 1
+    seed = 20190611
+    net = oracle_net(w)
+    L = make_learner(w)
+    ohp = oracle_hp(L.hp)
+    X, V = seed_identical(L, w, net)
+    T, E, A = w.n_steps, w.n_envs, w.n_actions
+    frames = w.net_kind == "conv"
+    mismatches = 0
+    for it in range(iters):
+        B.gala_actor_loop(L.ctx, 0, 1, seed)
+        L.sync()
+        ro, nxt = B.gala_actor_read(L.ctx, 0, E, T, GI.obs_shape(w), np.uint8 if frames else np.float32)
+        assert nxt == (it + 1) * T
+        for t in range(T + 1):
+            env = GI.synthetic_env(seed, 0, E, it * T + t, A, frames, w.obs_dim, actions=ro["actions"][t] if t < T else None)
+            np.testing.assert_array_equal(ro["obs"][t], env["obs"])
+            if t == T:
+                break
+            np.testing.assert_array_equal(ro["rewards"][t], env["rewards"])
+            np.testing.assert_array_equal(ro["dones"][t], env["dones"])
+            z, _ = R.forward(net, X[0], env["obs"])
+            want = R.sample(z, env["uniforms"])
+            cdf = np.cumsum(R.softmax(z), axis=1)
+            assert ro["actions"][t].min() >= 0 and ro["actions"][t].max() < A
+            for e in np.nonzero(ro["actions"][t] != want)[0]:
+                assert np.min(np.abs(cdf[e] - env["uniforms"][e])) < cdf_tol, (it, t, e, cdf[e], env["uniforms"][e])
+                mismatches += 1
+        info = R.learner_grad(net, X[0], ro, ohp)
+        x_before = X[0].copy()
+        xn, vn, _ = R.sweep_replay(X[0], info["grad"], V[0], ohp, None)
+        assert_grad_close("grad", L.get_grad(0), info["grad"], net, tol_net, "elementwise" if mode == "elementwise" else "norm")
+        check_params("x", L.get_params(0), xn, x_before, tol_params, mode)
+        X[0], V[0] = xn, vn
+        if mode != "elementwise":   # keep both sides on the same trajectory (oracle -> library only)
+            X[0] = X[0].astype(np.float32).astype(np.float64)
+            V[0] = V[0].astype(np.float32).astype(np.float64)
+            L.set_state(0, params=X[0], sq_avg=V[0], rnd=it + 1)
+    assert mismatches <= max(1, iters * T * E // 50)
+    L.close()
+
+
+def test_closed_actor_loop_mlp():
+    w = GI.WORKLOADS[0].scaled(n_agents=1, n_envs=8, n_steps=5)
+    _closed_loop(w, 3, TOL_FP32_NET, TOL_SWEEP, 1e-5, "elementwise")
+
+
+def test_closed_actor_loop_conv():
+    w = GI.WORKLOADS[1].scaled(n_agents=1, n_envs=3, n_steps=2)
+    _closed_loop(w, 3, TOL_BF16, TOL_BF16, 1e-2, "update")
