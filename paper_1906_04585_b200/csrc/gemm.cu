@@ -291,6 +291,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                         (p.out_group_stride & 7) == 0 && (p.out_split_stride & 7) == 0)
                                      : ((p.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 &&
                                         (p.out_group_stride & 3) == 0 && (p.out_split_stride & 3) == 0);
+        // 32-byte stores need every row start on a 32-byte boundary
+        const bool direct_ok = !transpose &&
+                               (out_bf16 ? ((p.ldc & 15) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 31) == 0 &&
+                                            (p.out_group_stride & 15) == 0 && (p.out_split_stride & 15) == 0)
+                                         : ((p.ldc & 7) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 31) == 0 &&
+                                            (p.out_group_stride & 7) == 0 && (p.out_split_stride & 7) == 0));
+        const bool direct_bias_vec = p.bias && (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0 && (p.bias_group_stride & 3) == 0;
         const bool mask_vec = use_mask && (reinterpret_cast<uintptr_t>(p.mask) & 7) == 0 && (p.mask_group_stride & 3) == 0;
         int local = 0;
         for (long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, local++) {
@@ -366,6 +373,43 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                     if (relu) v = fmaxf(v, 0.0f);
                                     o[(long)(nb + j) * p.ldc] = v;
                                 }
+                        }
+                    }
+                    continue;
+                }
+                // Direct path: the thread owns row mw + lane and holds its 32 columns, 64 contiguous bytes of bf16
+                // or 128 of fp32 in the output: whole 32-byte sectors, written with 32-byte stores from registers.
+                if (direct_ok && !use_mask && !rowmap && nb + 32 <= p.N) {
+                    const int m = mw + lane;
+                    if (m < p.M && q * 32 + lane < p.tile_rows) {
+                        float vals[32];
+#pragma unroll
+                        for (int j = 0; j < 32; j++) vals[j] = __uint_as_float(r[j]) * p.scale;
+                        if (bias) {
+#pragma unroll
+                            for (int j4 = 0; j4 < 8; j4++) {   // all lanes read the same addresses: one broadcast each
+                                const float4 bv = direct_bias_vec ? __ldg(reinterpret_cast<const float4*>(bias + nb) + j4)
+                                                                  : make_float4(__ldg(bias + nb + 4 * j4), __ldg(bias + nb + 4 * j4 + 1),
+                                                                                __ldg(bias + nb + 4 * j4 + 2), __ldg(bias + nb + 4 * j4 + 3));
+                                vals[4 * j4] += bv.x; vals[4 * j4 + 1] += bv.y; vals[4 * j4 + 2] += bv.z; vals[4 * j4 + 3] += bv.w;
+                            }
+                        }
+                        if (relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; j++) vals[j] = fmaxf(vals[j], 0.0f);
+                        }
+                        const long off = obase + (long)m * p.ldc + nb;
+                        if (out_bf16) {
+                            uint32_t o[16];
+#pragma unroll
+                            for (int j = 0; j < 16; j++) o[j] = pack2(vals[2 * j], vals[2 * j + 1]);
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + off;
+                            st_global_v8(dst, &o[0]);
+                            st_global_v8(dst + 16, &o[8]);
+                        } else {
+                            float* dst = reinterpret_cast<float*>(p.out) + off;
+#pragma unroll
+                            for (int j8 = 0; j8 < 4; j8++) st_global_v8(dst + 8 * j8, reinterpret_cast<const uint32_t*>(&vals[8 * j8]));
                         }
                     }
                     continue;
