@@ -413,7 +413,7 @@ def run_ours(args):
         line["async"] = dict(mixes=sum(x["mixes"] for x in st), skipped=sum(x["skipped"] for x in st),
                              staleness_mean=sum(x["staleness_sum"] for x in st) / max(1, sum(x["mixes"] for x in st)),
                              staleness_max=max(x["staleness_max"] for x in st), timing="host clock between syncs")
-    if rank == 0 and world == 1 and not async_mode:
+    if rank == 0 and world == 1 and not async_mode and not args.no_extras:
         # pieces beyond the core step: distance from consensus (one pass over all agents' parameters) and
         # the synchronous A2C baseline (gradient all-reduce instead of gossip) on the same rollouts
         t0 = time.perf_counter()
@@ -458,7 +458,7 @@ def run_ours(args):
                               allreduce_a2c_frames_per_s=w.frames_per_round / (a2c_ms * 1e-3),
                               note="consensus_call_ms is a host-timed call (sync + one kernel + 8-byte read); "
                                    "all-reduce rounds back to back without L2 flush")
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.no_extras:
         line["sweep_microbench"] = sweep_microbench(torch, B, pk)
         if not args.no_cpu_baseline:
             cores = usable_cores()
@@ -519,6 +519,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="index into gala_inputs.WORKLOADS (1 = the headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the legs beyond the timed rounds and the end-to-end leg (consensus distance, all-reduce "
+                         "baseline, closed actor loop, optimiser micro-benchmark, CPU oracle): for profiler runs")
     ap.add_argument("--mode", default="auto", choices=["auto", "sync", "async"],
                     help="auto: asynchronous per-agent streams for workload 4, synchronous rounds otherwise")
     ap.add_argument("--agent-ctas", type=int, default=-1,
