@@ -101,6 +101,24 @@ def round_work(w: GI.Workload, d_pad: int):
     return n * by, n * fl
 
 
+# ----------------------------------------------------------------------------- ranks
+def max_over_ranks(x: float, device: str = "cuda") -> float:
+    """The slowest rank's value (every rank gets it); the local value when there is one process.  The agents of
+    one rank never talk to those of another (replicas only), so this is the only collective of a multi-rank run."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(frames_per_rank: float, local_seconds: float, world: int, device: str = "cuda") -> float:
+    """Frames/s of the whole job: all ranks' frames over the slowest rank's time."""
+    return frames_per_rank * world / max_over_ranks(local_seconds, device)
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -322,12 +340,9 @@ def run_ours(args):
         total_ms = 1e3 * t_wall
     prof = B.gala_profile_read(L.ctx, reset=True)
     B.gala_profile_enable(L.ctx, 0)
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms)
     frames = w.frames_per_round * args.steps * world
-    value = frames / (total_ms * 1e-3)
+    value = whole_job_rate(w.frames_per_round * args.steps, total_ms * 1e-3, world)
 
     # roofline of the dominant kernel class, from its own events inside the timed region
     pk = peaks()
@@ -383,10 +398,7 @@ def run_ours(args):
         B.gala_losses_all(L.ctx, w.n_agents)
     barrier()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s)
     e2e = dict(value=frames / e2e_s, unit=UNIT, h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=20 * w.n_agents)
 
     rb, rf = round_work(w, L.d_pad)
