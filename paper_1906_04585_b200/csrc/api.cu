@@ -128,6 +128,8 @@ struct gala_ctx {
     bool use_graphs = true;                  // replay a learner step whose rollout buffers were seen before as a graph
     std::vector<StepGraph> graphs;
     int agent_ctas = 0;                      // SM budget of one agent's kernels in the per-agent calls (0: all)
+    ReduceSegs pending{};                    // sliced conv weight gradients of the step that still wait for their sum
+    long splitk_region[3] = {0, 0, 0};       // offset of conv layer l's slices inside an agent's split-K workspace
     int cur_ctas = 0;                        // budget of the launches being enqueued (0 in the synchronous round)
     int* error_word = nullptr;
     double *cons_partial = nullptr, *cons_out = nullptr;
@@ -482,7 +484,7 @@ int pick_splits(gala_ctx* c, int groups, int S, long count, int fixed) {
     long best_cost = -1;
     const long sms = c->cur_ctas > 0 ? c->cur_ctas : 148;
     for (int sp = 1; sp <= c->max_split && sp <= S; sp++) {
-        if (sp > 1 && (S / sp < 4 || sp * count > c->splitk_group_stride)) break;
+        if (sp > 1 && S / sp < 4) break;   // max_split slices of every layer fit its region of the workspace
         if (sp > 1 && c->cur_ctas > 0 && (long)groups * sp > sms) break;
         const long waves = ((long)groups * sp + sms - 1) / sms, per = (S + sp - 1) / sp;
         const long cost = waves * (per + fixed) + (sp > 1 ? 8 : 0);
@@ -504,14 +506,12 @@ int run_conv1_wgrad(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, cu
         LAUNCH(T_GEMM_CONV_WGRAD, st, launch_wgrad1(c->cwgrad1.y, a, st));
         return GALA_OK;
     }
-    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride + c->splitk_region[0];
     a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
     LAUNCH(T_GEMM_CONV_WGRAD, st, launch_wgrad1(c->cwgrad1.y, a, st));
-    LAUNCH(T_SPLITK, st, launch_splitk_reduce(c->splitk_ws + (long)agent0 * c->splitk_group_stride, final_out, count, a.splits,
-                                count, groups, c->splitk_group_stride, c->cwgrad1.args.out_group_stride, st));
+    c->pending.s[c->pending.n++] = ReduceSeg{c->cl.w[0], count, c->splitk_region[0], a.splits};
     return GALA_OK;
 }
-
 
 // conv2 / conv3 weight gradient: slices of the samples per agent chosen so that the CTAs fill the SMs in
 // whole waves; with more than one slice the partial sums go through the fixed-order reduction
@@ -527,12 +527,22 @@ int run_conv_wgrad(gala_ctx* c, const WgradPlan& p, int agent0, int groups, cuda
         LAUNCH(p.tag, st, launch_wgrad(p.x, p.y, a, st));
         return GALA_OK;
     }
-    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+    const int l = a.variant == WG_CONV2 ? 1 : 2;
+    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride + c->splitk_region[l];
     a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
     LAUNCH(p.tag, st, launch_wgrad(p.x, p.y, a, st));
-    LAUNCH(T_SPLITK, st, launch_splitk_reduce(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
-                                p.args.out + (long)agent0 * p.args.out_group_stride, count, best, count, groups,
-                                c->splitk_group_stride, p.args.out_group_stride, st));
+    c->pending.s[c->pending.n++] = ReduceSeg{c->cl.w[l], count, c->splitk_region[l], best};
+    return GALA_OK;
+}
+
+// One launch adds up the slices of every conv weight gradient that was sliced in this step.
+int flush_pending_reduces(gala_ctx* c, int agent0, int groups, cudaStream_t st) {
+    if (c->pending.n == 0) return GALA_OK;
+    const ReduceSegs segs = c->pending;
+    c->pending.n = 0;
+    LAUNCH(T_SPLITK, st, launch_splitk_reduce_multi(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
+                                                   c->g + (long)agent0 * c->d_pad, segs, groups, c->splitk_group_stride,
+                                                   c->d_pad, st));
     return GALA_OK;
 }
 
@@ -687,6 +697,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         CK(cudaStreamWaitEvent(side, c->ev_fork, 0));
         return GALA_OK;
     };
+    c->pending.n = 0;
     // forward pass and weight gradient of conv1 read the uint8 frames themselves; only the legacy products
     // need bf16 copies
     HiddenPending pend;
@@ -764,6 +775,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
                 if (r != GALA_OK) return r;
             }
         }
+        if ((r = flush_pending_reduces(c, agent0, groups, ws)) != GALA_OK) return r;
         // the bias gradients need every dY: they follow conv1's weight gradient on the side stream
         {   // all four bias gradients (column sums of dh, dY3, dY2, dY1) in one launch
             ColsumJobs jobs{};
@@ -1108,7 +1120,11 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         ALLOC(c->frames, (size_t)n * B * kFramePix);
         ALLOC(c->hid, (size_t)n * B * kHidden);
         ALLOC(c->dh, (size_t)n * S * kHidden);
-        c->splitk_group_stride = (long)c->max_split * 64 * 576;
+        // slices of conv3 (also the hidden layer's split-K partial sums), conv2, conv1 weight gradients
+        c->splitk_region[2] = 0;
+        c->splitk_region[1] = (long)c->max_split * 64 * 576;
+        c->splitk_region[0] = c->splitk_region[1] + (long)c->max_split * 64 * 512;
+        c->splitk_group_stride = c->splitk_region[0] + (long)c->max_split * 32 * 256;
         ALLOC(c->splitk_ws, (size_t)n * c->splitk_group_stride);
         int r = build_plans(c);
         if (r != GALA_OK) return r;

@@ -570,6 +570,51 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
         og[i] = acc;
     }
 }
+// Up to three such reductions in one launch (the conv weight gradients of a step), 16 bytes per thread.
+__global__ void __launch_bounds__(256) splitk_reduce_multi_kernel(const float* __restrict__ ws, float* __restrict__ out,
+                                                                  ReduceSegs sg, long total4, long ws_group_stride,
+                                                                  long out_group_stride) {
+    pdl_wait();
+    pdl_launch();
+    const int g = blockIdx.y;
+    const float* wg = ws + (long)g * ws_group_stride;
+    float* og = out + (long)g * out_group_stride;
+    for (long j = blockIdx.x * (long)blockDim.x + threadIdx.x; j < total4; j += (long)gridDim.x * blockDim.x) {
+        int k = 0;
+        long jj = j;
+        while (k + 1 < sg.n && jj >= sg.s[k].count / 4) { jj -= sg.s[k].count / 4; k++; }
+        const float* src = wg + sg.s[k].ws_off + jj * 4;
+        const long cnt = sg.s[k].count;
+        const int split = sg.s[k].split;
+        float4 t = *reinterpret_cast<const float4*>(src);
+        for (int s0 = 1; s0 < split; s0 += 4) {   // fixed order; four loads in flight
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; u++)
+                v[u] = s0 + u < split ? *reinterpret_cast<const float4*>(src + (long)(s0 + u) * cnt) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 4; u++)
+                if (s0 + u < split) { t.x += v[u].x; t.y += v[u].y; t.z += v[u].z; t.w += v[u].w; }
+        }
+        *reinterpret_cast<float4*>(og + sg.s[k].out_off + jj * 4) = t;
+    }
+}
+cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const ReduceSegs& segs, int groups,
+                                       long ws_group_stride, long out_group_stride, cudaStream_t st) {
+    if (segs.n < 1 || segs.n > 3 || ((ws_group_stride | out_group_stride) & 3)) return cudaErrorInvalidValue;
+    long total4 = 0;
+    for (int k = 0; k < segs.n; k++) {
+        if ((segs.s[k].out_off | segs.s[k].count | segs.s[k].ws_off) & 3 || segs.s[k].split < 1) return cudaErrorInvalidValue;
+        total4 += segs.s[k].count / 4;
+    }
+    if ((reinterpret_cast<uintptr_t>(ws) | reinterpret_cast<uintptr_t>(out)) & 15) return cudaErrorInvalidValue;
+    int bx = (int)((total4 + 255) / 256);
+    if (bx > 148 * 4) bx = 148 * 4;
+    (void)launch_pdl(splitk_reduce_multi_kernel, dim3(bx, groups), dim3(256), 0, st, ws, out, segs, total4, ws_group_stride,
+                     out_group_stride);
+    return cudaGetLastError();
+}
+
 // Same fixed-order reduction followed by the forward epilogue of a dense layer: + bias[n], ReLU, bf16.
 __global__ void __launch_bounds__(256) splitk_reduce_act_kernel(const float* __restrict__ partials,
                                                                 __nv_bfloat16* __restrict__ out, const float* __restrict__ bias,

@@ -145,6 +145,14 @@ cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, 
                                  long split_stride, int groups, long partial_group_stride,
                                  long out_group_stride, cudaStream_t st);
 
+// Several sliced weight gradients finished in one launch: range k of the output (out_off, count floats) is the sum,
+// in slice order, of `split` slices that lie `count` floats apart from ws_off on in the group's workspace.  Offsets
+// and counts are multiples of 4 floats.
+struct ReduceSeg { long out_off, count, ws_off; int split; };
+struct ReduceSegs { ReduceSeg s[3]; int n; };
+cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const ReduceSegs& segs, int groups,
+                                       long ws_group_stride, long out_group_stride, cudaStream_t st);
+
 // Caller-owned per-agent pointers travel in kernel parameters, at most kBatch agents a launch.
 constexpr int kBatch = 64;
 struct PtrBatch { const void* p[kBatch]; };
