@@ -128,7 +128,11 @@ class ClockSampler:
     def __init__(self, gpu_index: int):
         self.proc = None
         self.gpu = gpu_index
-        self.path = os.path.join(ROOT, "gpurun_out", "bench_clocks_%d.csv" % os.getpid())
+        # samples go to a scratch file (BENCH_CLOCKS_DIR, else the system's temporary directory); the line that is
+        # printed carries their summary
+        import tempfile
+        self.path = os.path.join(os.environ.get("BENCH_CLOCKS_DIR", tempfile.gettempdir()),
+                                 "bench_clocks_%d.csv" % os.getpid())
 
     def start(self):
         try:
