@@ -62,7 +62,7 @@ struct ConvPlan {  // one forward or data-gradient convolution (input resident i
 // Kernel classes for launch counting and optional per-class device timing.
 enum Tag : int {
     T_CAST_FRAMES = 0, T_HEADS_FWD, T_LOSS, T_HEADS_BWD, T_COLSUM, T_SPLITK, T_GRAD_NORM,
-    T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST, T_HEADS_FUSED, T_ENV,
+    T_SWEEP_SYNC, T_SWEEP_AGENT, T_DENSE_FWD, T_DENSE_BWD, T_SAMPLE, T_CAST, T_HEADS_FUSED, T_ENV, T_MLP_FUSED,
     T_GEMM_CONV_FWD,          // +layer (3)
     T_GEMM_FC_FWD = T_GEMM_CONV_FWD + 3, T_GEMM_FC_WGRAD, T_GEMM_FC_DGRAD,
     T_GEMM_CONV_WGRAD,        // +layer (3)
@@ -71,7 +71,7 @@ enum Tag : int {
 };
 const char* const kTagNames[T_COUNT] = {
     "cast_frames", "heads_fwd", "a2c_loss", "heads_bwd", "colsum", "splitk_reduce", "grad_norm",
-    "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16", "heads_fused", "env",
+    "sweep_sync", "sweep_agent", "dense_fwd", "dense_bwd", "sample", "cast_bf16", "heads_fused", "env", "mlp_fused",
     "gemm_conv1_fwd", "gemm_conv2_fwd", "gemm_conv3_fwd", "gemm_fc_fwd", "gemm_fc_wgrad", "gemm_fc_dgrad",
     "gemm_conv1_wgrad", "gemm_conv2_wgrad", "gemm_conv3_wgrad", "gemm_conv1_dgrad", "gemm_conv2_dgrad",
     "gemm_conv3_dgrad"};
@@ -125,6 +125,8 @@ struct gala_ctx {
     float* dzv = nullptr;                    // [N][S][20] rows (dlogits, dvalue, zeros) of the fused heads kernel
     float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
     bool fused_heads = false;
+    bool fused_mlp = false;                  // the MLP learner step as one kernel
+    float* mlp_partial = nullptr;            // [N][kMlpMaxBlocks][d + 4] partial gradients of its blocks
     bool use_graphs = true;                  // replay a learner step whose rollout buffers were seen before as a graph
     std::vector<StepGraph> graphs;
     int agent_ctas = 0;                      // SM budget of one agent's kernels in the per-agent calls (0: all)
@@ -700,6 +702,28 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
     c->pending.n = 0;
     // forward pass and weight gradient of conv1 read the uint8 frames themselves; only the legacy products
     // need bf16 copies
+    if (!c->conv && c->fused_mlp) {
+        MlpFusedArgs m{};
+        m.D = c->obs_dim; m.H = c->H; m.A = A; m.T = c->T; m.E = c->E; m.d = c->d; m.l = c->ml;
+        m.gamma = c->hp.gamma; m.ent_coef = c->hp.ent_coef; m.vf_coef = c->hp.vf_coef; m.max_norm = c->hp.max_grad_norm;
+        m.params = c->x + (long)agent0 * dp; m.p_stride = dp;
+        m.obs = obs; m.actions = acts; m.rewards = rews; m.dones = dns;
+        m.logits = c->logits + (long)agent0 * B * A; m.values = c->values + (long)agent0 * B;
+        m.returns = c->returns + (long)agent0 * S; m.adv = c->adv + (long)agent0 * S;
+        m.dlogits = c->dlogits + (long)agent0 * S * A; m.dvalues = c->dvalues + (long)agent0 * S;
+        m.losses = c->losses + (long)agent0 * 4;
+        m.h1_out = c->h1 + (long)agent0 * B * c->H; m.h2_out = c->h2 + (long)agent0 * B * c->H;
+        m.grad = c->g + (long)agent0 * dp; m.g_stride = dp;
+        m.norm = c->norm + agent0; m.clip = c->clip + agent0;
+        m.partial = c->mlp_partial + (long)agent0 * kMlpMaxBlocks * mlp_fused_partial_stride(c->d);
+        m.ticket = c->heads_ticket + agent0;
+        LAUNCH(T_MLP_FUSED, st, launch_mlp_fused(m, groups, st));
+        for (int i = 0; i < groups; i++) {
+            c->agents[agent0 + i].pending = true;
+            c->agents[agent0 + i].frames += S;
+        }
+        return GALA_OK;
+    }
     HiddenPending pend;
     const bool fused = c->conv && c->fused_heads;
     int r = forward(c, agent0, groups, obs, (int)B, st, c->legacy_conv ? st : nullptr, fused ? &pend : nullptr);
@@ -1132,6 +1156,8 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         const int H = c->H;
         ALLOC(c->h1, (size_t)n * B * H); ALLOC(c->h2, (size_t)n * B * H);
         ALLOC(c->dpre1, (size_t)n * S * H); ALLOC(c->dpre2, (size_t)n * S * H);
+        c->fused_mlp = mlp_fused_supported(c->obs_dim, H, A, c->T, c->E, c->d) && getenv("GALA_MLP_UNFUSED") == nullptr;
+        ALLOC(c->mlp_partial, (size_t)n * kMlpMaxBlocks * mlp_fused_partial_stride(c->d)); ALLOC(c->heads_ticket, n);
     }
     // initial parameters: uniform(-1,1)/sqrt(fan_in), biases included
     {

@@ -340,6 +340,27 @@ struct DenseBwdArgs {
 };
 cudaError_t launch_dense_bwd(const DenseBwdArgs& a, int groups, cudaStream_t st);
 
+// ---------------------------------------------------------------- MLP learner step in one kernel (mlp_fused.cu)
+struct MlpFusedArgs {
+    int D, H, A, T, E;
+    long d;                               // parameters per agent
+    MlpLayout l;
+    float gamma, ent_coef, vf_coef, max_norm;
+    const float* params; long p_stride;   // first agent of the launch
+    PtrBatch obs, actions, rewards, dones;
+    float *logits, *values, *returns, *adv, *dlogits, *dvalues, *losses;   // first agent of the launch
+    float *h1_out, *h2_out;               // [g][B][H] hidden activations
+    float* grad; long g_stride;
+    float *norm, *clip;                   // [g]
+    float* partial;                       // [g][kMlpMaxBlocks][mlp_fused_partial_stride(d)] scratch
+    unsigned* ticket;                     // [g], zero before the first launch
+    int ne, nb_max; long partial_stride;  // set by the launcher
+};
+constexpr int kMlpMaxBlocks = 16;         // blocks per agent
+long mlp_fused_partial_stride(long d);
+bool mlp_fused_supported(int D, int H, int A, int T, int E, long d);
+cudaError_t launch_mlp_fused(const MlpFusedArgs& a, int groups, cudaStream_t st);
+
 // ---------------------------------------------------------------- synthetic environment (env.cu)
 struct EnvArgs {
     unsigned long long seed;

@@ -412,3 +412,10 @@ def test_closed_actor_loop_mlp():
 def test_closed_actor_loop_conv():
     w = GI.WORKLOADS[1].scaled(n_agents=1, n_envs=3, n_steps=2)
     _closed_loop(w, 3, TOL_BF16, TOL_BF16, 1e-2, "update")
+
+
+def test_mlp_sync_round_unfused_kernels(monkeypatch):
+    # the layer-by-layer MLP kernels (used when a rollout is too large for the one-kernel step's shared memory)
+    monkeypatch.setenv("GALA_MLP_UNFUSED", "1")
+    w = GI.WORKLOADS[0].scaled(n_agents=3, n_envs=5, n_steps=4, topo_peers=2)
+    _sync_rounds(w, rounds=2, tol_net=TOL_FP32_NET, tol_params=TOL_SWEEP)
