@@ -12,11 +12,14 @@
 // zeros by TMA) the 16 elements (kx % 4, ci) of tap (ky, kx / 4) are row r + (ky / 4) * 21 + kx / 4 of
 // plane ky % 4.  Each plane is stored twice, the second copy one row up, so that the eight taps
 // (ky % 4, kx / 4) of one ky / 4 start at the same row of eight planes a constant distance apart: they
-// are the eight 16-element atoms of one MN-major A operand, and one MMA is
-//     D[(ky % 4, kx / 4, kx % 4, ci)][co] += A[128 x 16 pixels] * dY[16 pixels x 32]
-// with the pixel index as K.  Two accumulators (ky / 4 = 0, 1) of 32 columns stay in tensor memory over
-// the CTA's whole slice of samples; there is one epilogue per CTA, and with more than one slice per agent
-// the partial sums go through the fixed-order reduction.
+// are the eight 16-element atoms of one MN-major A operand.  The remaining shift, 21 rows for ky / 4 = 1, is
+// moved to the other operand: sum_r X[r + 21][m] dY[r][co] = sum_r' X[r'][m] dY[r' - 21][co], so the B operand
+// is two views of the same dY tile, 21 rows apart (rows before and after the tile are zero), as the two
+// 32-channel atoms of one MN-major N = 64 operand.  One MMA is
+//     D[(ky % 4, kx / 4, kx % 4, ci)][(ky / 4, co)] += A[128 x 16 pixels] * B[16 pixels x 64]
+// with the pixel index as K: 8 MMAs per unit instead of 14 with N = 32.  The accumulator (64 columns) stays in
+// tensor memory over the CTA's whole slice of samples; there is one epilogue per CTA, and with more than one
+// slice per agent the partial sums go through the fixed-order reduction.
 //
 //   warp 0     producer: bulk copy of the frame lines, TMA copy of the dY tile
 //   warp 1     MMA issuer (one thread)
@@ -28,13 +31,14 @@
 namespace gala {
 
 constexpr int kW1Planes = 8, kW1PlaneStride = 4096, kW1XBytes = kW1Planes * kW1PlaneStride;
-constexpr int kW1DyRows = 105, kW1DyBytes = 112 * 64;
-constexpr int kW1Stage = kW1XBytes + kW1DyBytes;            // 39936
+// dY region of a stage: 24 zero rows, the 105 rows of the tile (five lines in pitch 21), zero rows up to 160
+constexpr int kW1DyRows = 105, kW1DyPad = 24, kW1DyBytes = 160 * 64;
+constexpr int kW1Stage = kW1XBytes + kW1DyBytes;            // 43008
 constexpr int kW1Stages = 4;
 constexpr int kW1U8Stages = 4, kW1U8Bytes = 24 * 336, kW1U8Stride = 8192;
 constexpr int kW1Smem = kW1Stages * kW1Stage + kW1U8Stages * kW1U8Stride + 1024;
 constexpr int kW1Threads = 320, kW1ConvWarps = 8;
-constexpr int kW1KSteps = 7;                                // 112 pixel rows of 16
+constexpr int kW1KSteps = 8;                                // 128 pixel rows of 16 (105 of the tile + the 21-row shift)
 
 __global__ void __launch_bounds__(kW1Threads, 1)
 wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) {
@@ -73,8 +77,8 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    {   // Rows that nothing ever writes (the tail of a plane, dY rows 105..111) are read by MMAs; the dY rows
-        // must be zero and the others finite, so the ring starts zeroed.
+    {   // Rows that nothing ever writes (the tail of a plane, the rows around the dY tile) are read by MMAs; the
+        // dY rows must be zero and the others finite, so the ring starts zeroed.
         uint4* z = reinterpret_cast<uint4*>(smem);
         const int n16 = kW1Stages * kW1Stage / 16;
         for (int i = threadIdx.x; i < n16; i += blockDim.x) z[i] = make_uint4(0, 0, 0, 0);
@@ -108,7 +112,7 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
             if (!go) break;
             if (lane == 0) {
                 mbar_expect_tx(&full_bar[s], (uint32_t)(kW1DyRows * 64));
-                tma_load_4d(smem + s * kW1Stage + kW1XBytes, &tmY, &full_bar[s], 0, 0, 5 * q,
+                tma_load_4d(smem + s * kW1Stage + kW1XBytes + kW1DyPad * 64, &tmY, &full_bar[s], 0, 0, 5 * q,
                             (p.group0 + gz) * p.y_samples + sample);
                 issued_dy = it + 1;
             }
@@ -116,23 +120,21 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = make_instr_desc(32, 1, 1);   // A and B MN-major, N = 32, M = 128
+            const uint32_t idesc = make_instr_desc(64, 1, 1);   // A and B MN-major, N = 64, M = 128
             bool ok = true;
             for (int it = 0; ok && it < n_it; it++) {
                 const int s = it % kW1Stages;
                 if (!mbar_wait(&full_bar[s], (uint32_t)(it / kW1Stages) & 1u, &abort_flag)) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t x_addr = smem_u32(smem + s * kW1Stage);
-                const uint64_t bd_base = make_smem_desc_raw(x_addr + kW1XBytes, 4, 512, 512);
+                // B: atom 0 = the tile moved down by 21 rows (ky / 4 = 1), atom 1 = the tile itself (ky / 4 = 0)
+                const uint64_t bd_base = make_smem_desc_raw(x_addr + kW1XBytes + (kW1DyPad - 21) * 64, 4, 512, 21 * 64);
+                // A: 32-byte rows, groups of 8 rows 256 bytes apart, the eight atoms one plane apart
+                const uint64_t ad_base = make_smem_desc_raw(x_addr, 6, 256, kW1PlaneStride);
 #pragma unroll
-                for (int h = 0; h < 2; h++) {
-                    // 32-byte rows, groups of 8 rows 256 bytes apart, the eight atoms one plane apart
-                    const uint64_t ad_base = make_smem_desc_raw(x_addr + h * 21 * 32, 6, 256, kW1PlaneStride);
-#pragma unroll
-                    for (int kk = 0; kk < kW1KSteps; kk++)   // 16 pixels further: 16 rows of either image
-                        umma_bf16(tmem_base + (uint32_t)(h * 32), ad_base + (uint64_t)((kk * 16 * 32) >> 4),
-                                  bd_base + (uint64_t)((kk * 16 * 64) >> 4), idesc, (it | kk) != 0 ? 1u : 0u);
-                }
+                for (int kk = 0; kk < kW1KSteps; kk++)   // 16 pixels further: 16 rows of either image
+                    umma_bf16(tmem_base, ad_base + (uint64_t)((kk * 16 * 32) >> 4), bd_base + (uint64_t)((kk * 16 * 64) >> 4),
+                              idesc, (it | kk) != 0 ? 1u : 0u);
                 umma_commit(&empty_bar[s]);
             }
             if (ok) {
@@ -198,7 +200,7 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
             for (int h = 0; h < 2; h++) {
                 const int col = ((4 * h + py) * 8 + 4 * b) * 4 + el;   // (ky, kx, ci) inside W[co][256]
                 uint32_t r[32];
-                if (n_it > 0) tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 32), r);
+                if (n_it > 0) tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((1 - h) * 32), r);
                 else {
 #pragma unroll
                     for (int j = 0; j < 32; j++) r[j] = 0u;
