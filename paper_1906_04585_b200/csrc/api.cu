@@ -132,6 +132,7 @@ struct gala_ctx {
     int agent_ctas = 0;                      // SM budget of one agent's kernels in the per-agent calls (0: all)
     ReduceSegs pending{};                    // sliced conv weight gradients of the step that still wait for their sum
     long splitk_region[3] = {0, 0, 0};       // offset of conv layer l's slices inside an agent's split-K workspace
+    long bias_region[3] = {0, 0, 0};         // ... and of the slices of its bias gradient (64 floats each; conv2, conv3)
     int cur_ctas = 0;                        // budget of the launches being enqueued (0 in the synchronous round)
     int* error_word = nullptr;
     double *cons_partial = nullptr, *cons_out = nullptr;
@@ -508,8 +509,11 @@ int run_conv1_wgrad(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, cu
         LAUNCH(T_GEMM_CONV_WGRAD, st, launch_wgrad1(c->cwgrad1.y, a, st));
         return GALA_OK;
     }
-    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride + c->splitk_region[0];
+    float* ws = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+    a.out = ws + c->splitk_region[0];
     a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
+    // (conv1's bias gradient stays with the column-sum kernel: all warps of this kernel are busy converting, and one
+    // more warp that summed the dY tiles became its bottleneck, 0.19 -> 0.37 ms at 16 agents x 640 samples)
     LAUNCH(T_GEMM_CONV_WGRAD, st, launch_wgrad1(c->cwgrad1.y, a, st));
     c->pending.s[c->pending.n++] = ReduceSeg{c->cl.w[0], count, c->splitk_region[0], a.splits};
     return GALA_OK;
@@ -523,17 +527,21 @@ int run_conv_wgrad(gala_ctx* c, const WgradPlan& p, int agent0, int groups, cuda
     const long count = (long)(a.variant == WG_CONV2 ? 64 * 512 : 64 * 576);
     const int best = pick_splits(c, groups, S, count, 6);
     a.group0 = agent0; a.groups = groups; a.splits = best;
+    const int l = a.variant == WG_CONV2 ? 1 : 2;
     if (best == 1) {
         a.out += (long)agent0 * a.out_group_stride;
         a.out_split_stride = 0;
+        a.bias_out = c->g + (long)agent0 * c->d_pad + c->cl.b[l]; a.bias_group_stride = c->d_pad; a.bias_split_stride = 0;
         LAUNCH(p.tag, st, launch_wgrad(p.x, p.y, a, st));
         return GALA_OK;
     }
-    const int l = a.variant == WG_CONV2 ? 1 : 2;
-    a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride + c->splitk_region[l];
+    float* ws = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
+    a.out = ws + c->splitk_region[l];
     a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
+    a.bias_out = ws + c->bias_region[l]; a.bias_group_stride = c->splitk_group_stride; a.bias_split_stride = 64;
     LAUNCH(p.tag, st, launch_wgrad(p.x, p.y, a, st));
     c->pending.s[c->pending.n++] = ReduceSeg{c->cl.w[l], count, c->splitk_region[l], best};
+    c->pending.s[c->pending.n++] = ReduceSeg{c->cl.b[l], 64, c->bias_region[l], best};
     return GALA_OK;
 }
 
@@ -800,15 +808,20 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
             }
         }
         if ((r = flush_pending_reduces(c, agent0, groups, ws)) != GALA_OK) return r;
-        // the bias gradients need every dY: they follow conv1's weight gradient on the side stream
-        {   // all four bias gradients (column sums of dh, dY3, dY2, dY1) in one launch
+        // Bias gradients = column sums.  conv2's and conv3's come out of their weight-gradient kernels (summed from
+        // the dY tiles while those are in shared memory); the hidden layer's and conv1's, and in the legacy mode all
+        // four, here.
+        {
             ColsumJobs jobs{};
             jobs.j[0] = {c->dh + (long)agent0 * S * kHidden, S * kHidden, S, kHidden, c->cl.fcb};
-            for (int l = 0; l < 3; l++)
-                jobs.j[1 + l] = {c->dy[l] + (long)agent0 * S * P[l] * kConvCout[l], S * P[l] * kConvCout[l], S * P[l],
+            const int order[3] = {0, 1, 2};
+            for (int k = 0; k < 3; k++) {
+                const int l = order[k];
+                jobs.j[1 + k] = {c->dy[l] + (long)agent0 * S * P[l] * kConvCout[l], S * P[l] * kConvCout[l], S * P[l],
                                  kConvCout[l], c->cl.b[l]};
+            }
             if ((r = fork()) != GALA_OK) return r;
-            LAUNCH(T_COLSUM, ws, launch_colsum(jobs, 4, c->g + (long)agent0 * dp, dp,
+            LAUNCH(T_COLSUM, ws, launch_colsum(jobs, c->legacy_conv ? 4 : 2, c->g + (long)agent0 * dp, dp,
                                                c->colsum_partial + (long)agent0 * kColsumJobs * kColsumChunks * 512,
                                                c->colsum_ticket + (long)agent0 * kColsumJobs, groups, ws));
         }
@@ -1148,7 +1161,10 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         c->splitk_region[2] = 0;
         c->splitk_region[1] = (long)c->max_split * 64 * 576;
         c->splitk_region[0] = c->splitk_region[1] + (long)c->max_split * 64 * 512;
-        c->splitk_group_stride = c->splitk_region[0] + (long)c->max_split * 32 * 256;
+        c->bias_region[0] = c->splitk_region[0] + (long)c->max_split * 32 * 256;
+        c->bias_region[1] = c->bias_region[0] + (long)c->max_split * 64;
+        c->bias_region[2] = c->bias_region[1] + (long)c->max_split * 64;
+        c->splitk_group_stride = c->bias_region[2] + (long)c->max_split * 64;
         ALLOC(c->splitk_ws, (size_t)n * c->splitk_group_stride);
         int r = build_plans(c);
         if (r != GALA_OK) return r;

@@ -570,7 +570,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
         og[i] = acc;
     }
 }
-// Up to three such reductions in one launch (the conv weight gradients of a step), 16 bytes per thread.
+// Up to six such reductions in one launch (the conv weight and bias gradients of a step), 16 bytes per thread.
 __global__ void __launch_bounds__(256) splitk_reduce_multi_kernel(const float* __restrict__ ws, float* __restrict__ out,
                                                                   ReduceSegs sg, long total4, long ws_group_stride,
                                                                   long out_group_stride) {
@@ -601,7 +601,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_multi_kernel(const float* _
 }
 cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const ReduceSegs& segs, int groups,
                                        long ws_group_stride, long out_group_stride, cudaStream_t st) {
-    if (segs.n < 1 || segs.n > 3 || ((ws_group_stride | out_group_stride) & 3)) return cudaErrorInvalidValue;
+    if (segs.n < 1 || segs.n > 6 || ((ws_group_stride | out_group_stride) & 3)) return cudaErrorInvalidValue;
     long total4 = 0;
     for (int k = 0; k < segs.n; k++) {
         if ((segs.s[k].out_off | segs.s[k].count | segs.s[k].ws_off) & 3 || segs.s[k].split < 1) return cudaErrorInvalidValue;

@@ -145,11 +145,11 @@ cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, 
                                  long split_stride, int groups, long partial_group_stride,
                                  long out_group_stride, cudaStream_t st);
 
-// Several sliced weight gradients finished in one launch: range k of the output (out_off, count floats) is the sum,
+// Several sliced weight (and bias) gradients finished in one launch: range k of the output (out_off, count floats) is the sum,
 // in slice order, of `split` slices that lie `count` floats apart from ws_off on in the group's workspace.  Offsets
 // and counts are multiples of 4 floats.
 struct ReduceSeg { long out_off, count, ws_off; int split; };
-struct ReduceSegs { ReduceSeg s[3]; int n; };
+struct ReduceSegs { ReduceSeg s[6]; int n; };
 cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const ReduceSegs& segs, int groups,
                                        long ws_group_stride, long out_group_stride, cudaStream_t st);
 
@@ -197,6 +197,10 @@ struct WgradArgs {
     int x_samples, y_samples;   // samples per agent in the two tensors
     float* out;            // agent i, slice s at out + i * out_group_stride + s * out_split_stride, as W[co][KK]
     long out_group_stride, out_split_stride;
+    // bias gradient (column sums of dY over the same samples), summed from the dY tiles while they are in shared
+    // memory: agent i, slice s at bias_out + i * bias_group_stride + s * bias_split_stride, 64 floats; null: not wanted
+    float* bias_out;
+    long bias_group_stride, bias_split_stride;
     int* error_word;
 };
 cudaError_t wgrad_init();

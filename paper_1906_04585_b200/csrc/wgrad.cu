@@ -63,6 +63,7 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int issued_iters;
+    __shared__ float bias_part[4][64];
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -73,7 +74,8 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int n_it = s_end - s_begin;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        // a stage is released by the MMA issuer's commit and, when bias sums are wanted, by the four summing warps
+        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], p.bias_out ? 5 : 1); }
         mbar_init(&acc_full, 1);
         abort_flag = 0;
         issued_iters = 0;
@@ -151,6 +153,40 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             }
         }
     } else {
+        if (p.bias_out) {
+            // ------------------------------------------------ bias gradient: column sums of the dY tiles while they
+            // are in shared memory (rows of 64 channels, 128-byte swizzle; rows beyond the output width are zero).
+            // The four warps take every fourth row, lane l owns channels 2l, 2l + 1, four independent partial
+            // sums per lane keep loads in flight; fixed order: rows, samples, partial sums, warps.
+            const int wq = warp - 2;
+            float b0[4] = {0.f, 0.f, 0.f, 0.f}, b1[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t lane_off = (uint32_t)((lane & 3) << 2);
+            for (int it = 0; it < n_it; it++) {
+                const int s = it % nst;
+                if (!mbar_wait(&full_bar[s], (uint32_t)(it / nst) & 1u, &abort_flag)) break;
+                const uint8_t* dy = smem + s * STAGE + T::X_BYTES;
+                for (int r0 = wq; r0 < T::DY_ROWS; r0 += 16) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int u = 0; u < 4; u++) {
+                        const int r = r0 + 4 * u;
+                        w[u] = r < T::DY_ROWS ? *reinterpret_cast<const uint32_t*>(dy + r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + lane_off) : 0u;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; u++) { b0[u] += __uint_as_float(w[u] << 16); b1[u] += __uint_as_float(w[u] & 0xffff0000u); }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[s]);
+            }
+            bias_part[wq][2 * lane] = (b0[0] + b0[1]) + (b0[2] + b0[3]);
+            bias_part[wq][2 * lane + 1] = (b1[0] + b1[1]) + (b1[2] + b1[3]);
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
+            if (wq == 0) {
+                float* bo = p.bias_out + (long)gz * p.bias_group_stride + (long)ss * p.bias_split_stride;
+                for (int c0 = lane; c0 < 64; c0 += 32)
+                    bo[c0] = ((bias_part[0][c0] + bias_part[1][c0]) + bias_part[2][c0]) + bias_part[3][c0];
+            }
+        }
         // ------------------------------------------------ epilogue (once): thread = row (tap, ci) of D
         const int q = warp & 3;
         if (mbar_wait(&acc_full, 0u, &abort_flag)) {
