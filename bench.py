@@ -261,6 +261,8 @@ def run_ours(args):
         L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32))
     if args.agent_ctas >= 0:
         B.gala_set_agent_ctas(L.ctx, args.agent_ctas)
+    if args.no_graphs:
+        B.gala_set_graphs(L.ctx, False)
     ext = torch.cuda.ExternalStream(B.gala_get_stream(L.ctx, -1))
     up = torch.cuda.Stream()      # host -> device copies run on a torch stream; the library's stream waits on it
 
@@ -546,6 +548,7 @@ def main():
                     help="auto: asynchronous per-agent streams for workload 4, synchronous rounds otherwise")
     ap.add_argument("--agent-ctas", type=int, default=-1,
                     help="asynchronous mode: thread blocks per kernel of one agent (-1: the library's default)")
+    ap.add_argument("--no-graphs", action="store_true", help="launch every kernel of a learner step directly (no graph replay)")
     ap.add_argument("--no-skew", action="store_true", help="asynchronous mode without the injected straggler delays")
     ap.add_argument("--sweep-only", action="store_true",
                     help="run only the RMSProp + gossip micro-benchmark (32 agents x 1.7M parameters)")

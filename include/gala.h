@@ -203,14 +203,17 @@ int gala_actor_loop(gala_ctx* ctx, int agent, int iterations, unsigned long long
  * environment steps taken so far. */
 int gala_actor_read(gala_ctx* ctx, int agent, void* obs, int* actions, float* rewards, unsigned char* dones,
                     long long* next_step);
-/* CUDA-graph replay of the learner step (default on).  The first gala_learn / gala_step_sync with a given set
- * of rollout buffers launches its kernels one by one; the second captures the same launches into a graph; from
- * then on the step is one graph launch (the kernels and their results are the same).  A caller that reuses its
- * rollout buffers, as an actor that writes each rollout into the same device memory does, gets this for every
- * step; one that passes new buffers every time never pays for a capture.  Up to 512 distinct buffer sets are
- * remembered.  Off while per-class timing (gala_profile_enable) of a kernel inside the step is on.  If the
- * application itself captures the library's streams into a graph, switch this off first. */
-int gala_set_graphs(gala_ctx* ctx, int on);
+/* CUDA-graph replay of the learner step.  mode 1 (default): in gala_step_sync; 2: also in gala_learn; 0: never.
+ * The first call with a given set of rollout buffers launches its kernels one by one; the second captures the
+ * same launches into a graph; from then on the step is one graph launch (the kernels and their results are the
+ * same).  A caller that reuses its rollout buffers, as an actor that writes each rollout into the same device
+ * memory does, gets this for every step; one that passes new buffers every time never pays for a capture.  Up to
+ * 512 distinct buffer sets are remembered.  Instantiating a graph costs about a millisecond of host time, which
+ * pays off in the synchronous round (host-bound at small batches) and not in the per-agent calls of many agents
+ * (bound by the device; 64 agents x 4 buffer sets are 256 graphs), hence the default.  Off while per-class timing
+ * (gala_profile_enable) of a kernel inside the step is on.  If the application itself captures the library's
+ * streams into a graph, switch this off first. */
+int gala_set_graphs(gala_ctx* ctx, int mode);
 int gala_param_count(const gala_ctx* ctx, long long* d, long long* d_padded);
 /* out = {policy term, mean squared TD error, mean entropy, gradient norm} of the last learn. */
 int gala_losses(gala_ctx* ctx, int agent, float out[4]);

@@ -199,8 +199,9 @@ def gala_actor_read(ctx, agent: int, n_envs: int, n_steps: int, obs_shape, obs_d
     return dict(obs=obs, actions=actions, rewards=rewards, dones=dones), int(nxt.value)
 
 
-def gala_set_graphs(ctx, on: bool):
-    _check(ctx, lib().gala_set_graphs(ctx, 1 if on else 0))
+def gala_set_graphs(ctx, mode):
+    """0 / False: never; 1 / True: graph replay in the synchronous round; 2: also in the per-agent calls."""
+    _check(ctx, lib().gala_set_graphs(ctx, int(mode)))
 
 
 def gala_set_agent_ctas(ctx, ctas: int):

@@ -127,7 +127,8 @@ struct gala_ctx {
     bool fused_heads = false;
     bool fused_mlp = false;                  // the MLP learner step as one kernel
     float* mlp_partial = nullptr;            // [N][kMlpMaxBlocks][d + 4] partial gradients of its blocks
-    bool use_graphs = true;                  // replay a learner step whose rollout buffers were seen before as a graph
+    int use_graphs = 1;                      // replay a learner step whose rollout buffers were seen before as a graph:
+                                             // 0 never, 1 in the synchronous round, 2 also in the per-agent calls
     std::vector<StepGraph> graphs;
     int agent_ctas = 0;                      // SM budget of one agent's kernels in the per-agent calls (0: all)
     ReduceSegs pending{};                    // sliced conv weight gradients of the step that still wait for their sum
@@ -873,7 +874,7 @@ int learn_range_cached(gala_ctx* c, int agent0, int groups, const gala_rollout* 
     // per-class timing brackets launches with events: not inside a graph (the optimiser / gossip pass and the
     // sampling kernel lie outside this step, so timing only those does not matter)
     const unsigned long long outside = (1ull << T_SWEEP_SYNC) | (1ull << T_SWEEP_AGENT) | (1ull << T_SAMPLE);
-    if (!c->use_graphs || (c->profile_mask & ~outside) != 0 || c->legacy_conv)
+    if (c->use_graphs < (side ? 1 : 2) || (c->profile_mask & ~outside) != 0 || c->legacy_conv)
         return learn_range(c, agent0, groups, ro, st, side);
     std::vector<const void*> key;
     key.reserve(6 + 4 * (size_t)groups);
@@ -1477,7 +1478,8 @@ int gala_consensus_distance(gala_ctx* c, double* out) {
 
 int gala_set_graphs(gala_ctx* c, int on) {
     if (!c) return GALA_EINVAL;
-    c->use_graphs = on != 0;
+    if (on < 0 || on > 2) return fail(c, GALA_EINVAL, "gala_set_graphs: mode must be 0, 1 or 2");
+    c->use_graphs = on;
     return GALA_OK;
 }
 

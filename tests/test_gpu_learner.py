@@ -356,7 +356,7 @@ def test_conv_degenerate_shapes(n_agents, n_envs, n_steps, peers):
     _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
 
 
-def _closed_loop(w, iters, tol_net, tol_params, cdf_tol, mode):
+def _closed_loop(w, iters, tol_net, tol_params, cdf_tol, mode, graphs=1):
     """Closed actor loop of one agent (no in-peers, so no averaging) against the oracle, one iteration at a time:
     the environment's observations, rewards and done flags bit for bit; every sampled action equal to the
     oracle's draw from the same uniform unless that uniform lies within cdf_tol of a boundary of the oracle's
@@ -366,6 +366,7 @@ def _closed_loop(w, iters, tol_net, tol_params, cdf_tol, mode):
     seed = 20190611
     net = oracle_net(w)
     L = make_learner(w)
+    B.gala_set_graphs(L.ctx, graphs)     # 2: the per-agent learner step is captured (2nd iteration) and replayed (3rd)
     ohp = oracle_hp(L.hp)
     X, V = seed_identical(L, w, net)
     T, E, A = w.n_steps, w.n_envs, w.n_actions
@@ -411,7 +412,7 @@ def test_closed_actor_loop_mlp():
 
 def test_closed_actor_loop_conv():
     w = GI.WORKLOADS[1].scaled(n_agents=1, n_envs=3, n_steps=2)
-    _closed_loop(w, 3, TOL_BF16, TOL_BF16, 1e-2, "update")
+    _closed_loop(w, 3, TOL_BF16, TOL_BF16, 1e-2, "update", graphs=2)
 
 
 def test_mlp_sync_round_unfused_kernels(monkeypatch):
