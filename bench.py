@@ -267,8 +267,8 @@ def run_ours(args):
     up = torch.cuda.Stream()      # host -> device copies run on a torch stream; the library's stream waits on it
 
     n_sets = 4
-    sets = [[LM.DeviceRollout(GI.rollout(w, i, s + 1000 * rank), pinned=True) for i in range(w.n_agents)]
-            for s in range(n_sets)]
+    # a round's rollouts of all agents share one pinned host buffer and one device buffer per field
+    sets = [LM.RolloutBatch([GI.rollout(w, i, s + 1000 * rank) for i in range(w.n_agents)]) for s in range(n_sets)]
     flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
     n_classes = B.gala_kernel_classes()
     work = class_work(w, L.d_pad)
@@ -372,13 +372,12 @@ def run_ours(args):
 
     # end to end through the public API with host buffers: pinned host -> device copy of the step's
     # rollouts, the step, and a device -> host read of the step's losses, all inside the timed region
-    h2d = sum(r.nbytes for r in sets[0])
+    h2d = sets[0].nbytes
     up_done = [torch.cuda.Event() for _ in range(n_sets)]
 
     def upload(j):
         """Enqueue the pinned-host -> device copy of buffer set j on the copy stream."""
-        for r in sets[j]:
-            r.upload(up)
+        sets[j].upload(up)
         up_done[j].record(up)
 
     def step_from_host(k):

@@ -38,6 +38,46 @@ class DeviceRollout:
         return sum(v.numel() * v.element_size() for v in self.t.values())
 
 
+class _RolloutView:
+    """One agent's part of a RolloutBatch: the same attribute the library calls need (`c`)."""
+
+    def __init__(self, c):
+        self.c = c
+
+
+class RolloutBatch:
+    """The rollouts of all agents of one round in ONE pinned host buffer and ONE device buffer per field, so that
+    a round's inputs travel host -> device as four copies (one of them carries all the frames) instead of four per
+    agent; each agent still gets its own pointers.  Indexing and iteration give per-agent views."""
+
+    def __init__(self, ros: Sequence[Dict[str, np.ndarray]], device="cuda"):
+        keys = ("obs", "actions", "rewards", "dones")
+        self.host = {k: torch.from_numpy(np.ascontiguousarray(np.stack([r[k] for r in ros]))).pin_memory() for k in keys}
+        self.t = {k: torch.empty_like(v, device=device) for k, v in self.host.items()}
+        self.upload()
+        torch.cuda.current_stream().synchronize()     # the library's streams do not order themselves against torch's
+        self.views = [_RolloutView(B.make_rollout(self.t["obs"][i], self.t["actions"][i], self.t["rewards"][i],
+                                                  self.t["dones"][i])) for i in range(len(ros))]
+
+    def upload(self, stream: Optional[torch.cuda.Stream] = None):
+        with torch.cuda.stream(stream) if stream is not None else torch.cuda.stream(torch.cuda.current_stream()):
+            for k, v in self.host.items():
+                self.t[k].copy_(v, non_blocking=True)
+
+    def __len__(self):
+        return len(self.views)
+
+    def __getitem__(self, i):
+        return self.views[i]
+
+    def __iter__(self):
+        return iter(self.views)
+
+    @property
+    def nbytes(self) -> int:
+        return sum(v.numel() * v.element_size() for v in self.t.values())
+
+
 class Learner:
     def __init__(self, n_agents: int, topo_kind: int, topo_peers: int, net_kind: str, n_actions: int,
                  n_envs: int, n_steps: int, obs_dim: int = 8, hidden: int = 64, **hp_overrides):

@@ -155,3 +155,24 @@ def test_losses_all_agrees_with_per_agent_reads_and_graph_replay_repeats_the_ste
     for i in range(w.n_agents):
         np.testing.assert_array_equal(L.get_grad(i), grads[0][i])
     L.close()
+
+
+def test_rollout_batch_gives_the_same_round_as_separate_rollouts():
+    """All agents' rollouts in one buffer per field (per-agent pointers into it) against one buffer set per agent."""
+    from paper_1906_04585_b200 import learner as LM
+    w = GI.WORKLOADS[1].scaled(n_agents=3, n_envs=2, n_steps=2)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    ros = [GI.rollout(w, i, 0) for i in range(w.n_agents)]
+    grads = []
+    for batch in (False, True):
+        L = _learner(w)
+        for i in range(w.n_agents):
+            L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32), rnd=0)
+        dev = LM.RolloutBatch(ros) if batch else [LM.DeviceRollout(r) for r in ros]
+        assert len(dev) == w.n_agents
+        L.step_sync(dev)
+        L.sync()
+        grads.append([L.get_grad(i) for i in range(w.n_agents)])
+        L.close()
+    for i in range(w.n_agents):
+        np.testing.assert_array_equal(grads[0][i], grads[1][i])
