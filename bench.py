@@ -59,7 +59,8 @@ def class_work(w: GI.Workload, d_pad: int):
     out = {"sweep_sync": ("hbm", n * d_pad * (20.0 + shadow)),
            # per-agent form: read x, g, v and p snapshots, write x, v and the own snapshot
            "sweep_agent": ("hbm", n * d_pad * (24.0 + 4.0 * w.topo_peers + shadow)),
-           "grad_norm": ("hbm", n * d_pad * 4.0)}
+           # the conv net's norm pass skips the hidden layer's weight gradient (its sums of squares come with it)
+           "grad_norm": ("hbm", n * (d_pad - (512 * 3136 if w.net_kind == "conv" else 0)) * 4.0)}
     if w.net_kind != "conv":
         return out
     P, KK, CO = (400, 81, 49), (256, 512, 576), (32, 64, 64)

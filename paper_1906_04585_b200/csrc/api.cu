@@ -122,6 +122,7 @@ struct gala_ctx {
     float *clip = nullptr, *norm = nullptr, *losses = nullptr;
     double *norm_partial = nullptr, *colsum_partial = nullptr;
     unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr, *heads_ticket = nullptr;
+    float* fc_sq = nullptr;                  // [N][1600] sums of squares of the hidden layer's weight gradient, by 32 x 32 block
     float* dzv = nullptr;                    // [N][S][20] rows (dlogits, dvalue, zeros) of the fused heads kernel
     float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
     bool fused_heads = false;
@@ -414,6 +415,7 @@ int build_plans(gala_ctx* c) {
         ok &= make_operand(&w.B, c->act[2], 1, kFeat, S, n, kFeat, (uint64_t)B * kFeat, 128);
         w.args.M = kHidden; w.args.N = kFeat; w.args.K = (int)S; w.args.block_n = 128;
         w.args.out = c->g + c->cl.fcw; w.args.out_group_stride = dp; w.args.ldc = kFeat;
+        w.args.sq_partial = c->fc_sq;   // so that the norm pass need not read these 95 % of the gradient again
         // data gradient: dh [S][512] x Wfc [512][3136] -> dY3 [S][3136], masked by act3 > 0
         Plan& dg = c->fc_dgrad;
         zero_args(dg);
@@ -577,6 +579,7 @@ int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override,
     a.out = reinterpret_cast<char*>(a.out) + (long)agent0 * a.out_group_stride * (bf ? 2 : 4);
     if (a.mask) a.mask += (long)agent0 * a.mask_group_stride;
     if (a.gate) a.gate += (long)agent0 * a.gate_group_stride;
+    if (a.sq_partial) a.sq_partial += (long)agent0 * ((a.M + 127) / 128) * ((a.N + a.block_n - 1) / a.block_n) * 16;
     LAUNCH(p.tag, st, launch_gemm(p.A, p.B, a, st));
     return GALA_OK;
 }
@@ -856,8 +859,14 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         d1.din = nullptr;
         LAUNCH(T_DENSE_BWD, st, launch_dense_bwd(d1, groups, st));
     }
+    NormKnown kn{};
+    if (c->conv) {   // the hidden layer's weight gradient left the sums of squares of its 32 x 32 blocks behind
+        kn.n_partials = (long)(kHidden / 128) * ((kFeat + 127) / 128) * 16;
+        kn.off = c->cl.fcw; kn.count = (long)kHidden * kFeat;
+        kn.partial = c->fc_sq + (long)agent0 * kn.n_partials; kn.partial_group_stride = kn.n_partials;
+    }
     LAUNCH(T_GRAD_NORM, st, launch_grad_norm(c->g, c->d, dp, agent0, groups, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
-                            c->norm, c->clip, st));
+                            c->norm, c->clip, st, c->conv ? &kn : nullptr));
     for (int i = 0; i < groups; i++) {
         c->agents[agent0 + i].pending = true;
         c->agents[agent0 + i].frames += S;
@@ -1148,6 +1157,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         c->fused_heads = heads_fused_supported(c->T, c->E, c->A, kHidden) && getenv("GALA_HEADS_UNFUSED") == nullptr;
         ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
         ALLOC(c->dzv, (size_t)n * S * 20);
+        ALLOC(c->fc_sq, (size_t)n * (kHidden / 128) * ((kFeat + 127) / 128) * 16);
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {

@@ -348,7 +348,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         if (!((gw >> j) & 1u)) r[j] = 0u;
                 }
                 const int nb = t.n0 + c0;
-                if (mw >= p.M || q * 32 >= p.tile_rows || nb >= p.N) continue;   // warp-uniform
+                if (mw >= p.M || q * 32 >= p.tile_rows || nb >= p.N) {   // warp-uniform
+                    if (p.sq_partial && lane == 0) p.sq_partial[tile * 16 + q * 4 + (c0 >> 5)] = 0.0f;
+                    continue;
+                }
                 if (transpose) {
                     // D[m][n] -> out[n * ldc + m]: consecutive lanes write consecutive addresses
                     const int m = mw + lane;
@@ -381,6 +384,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 // or 128 of fp32 in the output: whole 32-byte sectors, written with 32-byte stores from registers.
                 if (direct_ok && !use_mask && !rowmap && nb + 32 <= p.N) {
                     const int m = mw + lane;
+                    float row_sq = 0.0f;
                     if (m < p.M && q * 32 + lane < p.tile_rows) {
                         float vals[32];
 #pragma unroll
@@ -398,6 +402,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                             for (int j = 0; j < 32; j++) vals[j] = fmaxf(vals[j], 0.0f);
                         }
+                        if (p.sq_partial) {   // this row's share of the block's sum of squares (fixed order)
+                            float sq = 0.0f;
+#pragma unroll
+                            for (int j = 0; j < 32; j++) sq = fmaf(vals[j], vals[j], sq);
+                            row_sq = sq;
+                        }
                         const long off = obase + (long)m * p.ldc + nb;
                         if (out_bf16) {
                             uint32_t o[16];
@@ -411,6 +421,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                             for (int j8 = 0; j8 < 4; j8++) st_global_v8(dst + 8 * j8, reinterpret_cast<const uint32_t*>(&vals[8 * j8]));
                         }
+                    }
+                    if (p.sq_partial) {   // rows of the block added by a butterfly: the same tree every time
+                        for (int o = 16; o > 0; o >>= 1) row_sq += __shfl_xor_sync(0xffffffffu, row_sq, o);
+                        if (lane == 0) p.sq_partial[tile * 16 + q * 4 + (c0 >> 5)] = row_sq;
                     }
                     continue;
                 }
@@ -738,6 +752,11 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     if (args.block_n != 32 && args.block_n != 64 && args.block_n != 128) return cudaErrorInvalidValue;
     if (B.mn_major && args.block_n < 64 && !(args.conv_mode != CONV_NONE && args.conv_layer == 0)) return cudaErrorInvalidValue;
     if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
+    if (args.sq_partial && (args.block_n != 128 || args.split_k != 1 || (args.N & 31) || (args.ldc & 7) ||
+                            (args.flags & (EPI_OUT_BF16 | EPI_TRANSPOSE | EPI_MASK | EPI_ROWMAP_S2)) ||
+                            (reinterpret_cast<uintptr_t>(args.out) & 31) || (args.out_group_stride & 7) ||
+                            args.conv_mode != CONV_NONE))
+        return cudaErrorInvalidValue;
     if ((args.flags & EPI_GATE) && (!args.gate || (args.N & 31) || (args.flags & (EPI_TRANSPOSE | EPI_ROWMAP_S2))))
         return cudaErrorInvalidValue;
     GemmArgs a = args;

@@ -96,6 +96,11 @@ struct GemmArgs {
     long gate_group_stride;
     int* error_word;       // device int, set non-zero when a bounded wait runs out
     int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
+    // Optional sums of squares of the stored outputs (for a gradient norm without a second pass over this
+    // product): slot [tile * 16 + warp quarter * 4 + 32-column block] of sq_partial gets the sum over that
+    // 32 x 32 block (0 where the block lies outside the matrix).  Needs block_n = 128, split_k = 1, fp32 row-major
+    // output with 32-byte aligned rows and N a multiple of 32; tile = (group * m_tiles + m_tile) * n_tiles + n_tile.
+    float* sq_partial;
     // Tiling (set by the caller for the convolution modes, filled with defaults by launch_gemm)
     int tile_rows;         // rows of D per M tile (<= 128; default 128)
     int k_steps;           // number of K steps of the whole reduction (default ceil(K/64))
@@ -243,8 +248,12 @@ cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const flo
 // Sum of squares of g[agent][0..d) -> norm[agent], clip[agent] = min(1, max_norm/(norm+1e-6)).
 // partial: [n_agents][kNormChunks] doubles, ticket: [n_agents] uints (zero before first use).
 constexpr int kNormChunks = 128;
+// A range of g whose sum of squares is already known as partial sums (written by the product that produced it):
+// the norm pass skips reading it and adds the partials in slot order instead.
+struct NormKnown { long off, count; const float* partial; long n_partials, partial_group_stride; };
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
-                             double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st);
+                             double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st,
+                             const NormKnown* known = nullptr);
 cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStream_t st);
 // partial: 592 doubles, ticket: one zeroed unsigned, out: one double (squared distance)
 cudaError_t launch_consensus(const float* x, int n_agents, long d, long d_pad, double* partial, unsigned* ticket,

@@ -201,21 +201,28 @@ cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* c
 // double precision make the result independent of scheduling.
 __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict__ g, long d, long d_pad,
                                                         int agent0, float max_norm, double* partial,
-                                                        unsigned* ticket, float* norm, float* clip) {
+                                                        unsigned* ticket, float* norm, float* clip, NormKnown kn) {
     pdl_wait();
     pdl_launch();
     const int agent = agent0 + blockIdx.y;
     const float* ga = g + (long)agent * d_pad;
-    // chunks are multiples of 4 floats and the padding [d, d_pad) is zero: 16-byte loads throughout
-    const long per = ((d_pad / 4 + kNormChunks - 1) / kNormChunks) * 4;
+    // The elements to read, [0, d_pad) without the range whose sum of squares is already known, are numbered
+    // consecutively and cut into chunks of multiples of 4 floats (the padding [d, d_pad) is zero): 16-byte loads
+    const long total = d_pad - kn.count;
+    const long per = ((total / 4 + kNormChunks - 1) / kNormChunks) * 4;
     const long lo = (long)blockIdx.x * per;
-    long hi = lo + per; if (hi > d_pad) hi = d_pad;
+    long hi = lo + per; if (hi > total) hi = total;
     float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
     for (long i = lo + 4L * threadIdx.x; i < hi; i += 4L * blockDim.x) {
-        const float4 t = __ldcs(reinterpret_cast<const float4*>(ga + i));
+        const float4 t = __ldcs(reinterpret_cast<const float4*>(ga + (i < kn.off ? i : i + kn.count)));
         a0 = fmaf(t.x, t.x, a0); a1 = fmaf(t.y, t.y, a1); a2 = fmaf(t.z, t.z, a2); a3 = fmaf(t.w, t.w, a3);
     }
     double acc = ((double)a0 + (double)a1) + ((double)a2 + (double)a3);
+    if (kn.partial) {   // the known range: its partial sums, shared out over the agent's threads in slot order
+        const float* kp = kn.partial + (long)blockIdx.y * kn.partial_group_stride;
+        for (long k = (long)blockIdx.x * blockDim.x + threadIdx.x; k < kn.n_partials; k += (long)kNormChunks * blockDim.x)
+            acc += (double)kp[k];
+    }
     __shared__ double red[256];
     red[threadIdx.x] = acc;
     __syncthreads();
@@ -245,9 +252,14 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
 }
 
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
-                             double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st) {
+                             double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st,
+                             const NormKnown* known) {
+    NormKnown kn{};
+    if (known) kn = *known;
+    if (!kn.partial) { kn.off = 0; kn.count = 0; kn.n_partials = 0; }
+    if ((kn.off | kn.count) & 3 || kn.off + kn.count > d_pad) return cudaErrorInvalidValue;
     dim3 grid(kNormChunks, n_agents);
-    (void)launch_pdl(grad_norm_kernel, dim3(grid), dim3(256), 0, st, g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip);
+    (void)launch_pdl(grad_norm_kernel, dim3(grid), dim3(256), 0, st, g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip, kn);
     return cudaGetLastError();
 }
 
