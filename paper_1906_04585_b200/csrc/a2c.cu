@@ -215,7 +215,7 @@ cudaError_t launch_heads_fwd(const HeadsArgs& a, int groups, cudaStream_t st) {
     if (bx * groups > 592) bx = (592 + groups - 1) / groups;
     if (bx < 1) bx = 1;
     const size_t smem = (size_t)((a.A + 1) + 8) * a.H * sizeof(float);
-    if (smem > 48 * 1024) {
+    if (smem > 40 * 1024) {   // well below the 48 KiB that need no opt-in
         cudaError_t e = cudaFuncSetAttribute(heads_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
@@ -563,11 +563,13 @@ cudaError_t launch_heads_fused(const HeadsFusedArgs& a0, int groups, cudaStream_
     if (!heads_fused_supported(a.T, a.E, a.A, kHeadsH)) return cudaErrorNotSupported;
     a.ne = heads_fused_envs_per_block(a.T, a.E, groups);
     const size_t smem = heads_fused_smem(a.A, a.ne * (a.T + 1));
-    static size_t attr_set = 0;
-    if (smem > 48 * 1024 && smem > attr_set) {
+    // always opt in: the 48 KiB that need no opt-in include the kernel's static shared memory, so a dynamic size
+    // just below 48 KiB would already be refused
+    static bool attr_set = false;
+    if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(heads_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(160 * 1024));
         if (e != cudaSuccess) return e;
-        attr_set = 160 * 1024;
+        attr_set = true;
     }
     (void)launch_pdl(heads_fused_kernel, dim3((a.E + a.ne - 1) / a.ne, groups), dim3(256), smem, st, a);
     return cudaGetLastError();

@@ -724,6 +724,23 @@ bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint
     return r == CUDA_SUCCESS;
 }
 
+// The same matrix seen as [rows][cols / 256][256] (cols a multiple of 256): a box {256, box_blocks, box_rows} is
+// box_rows x (256 * box_blocks) floats in one copy, past the 256-element limit of a box edge.
+bool make_tensor_map_f32_wide(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
+                              uint32_t box_blocks, uint32_t box_rows) {
+    if (!g_encode) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15) || (row_stride_bytes & 15) || (cols & 255) || box_blocks > 256 || box_rows > 256)
+        return false;
+    cuuint64_t dims[3] = {256, cols / 256, rows};
+    cuuint64_t strides[2] = {1024, row_stride_bytes};
+    cuuint32_t box[3] = {256, box_blocks, box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
                         const uint64_t* strides_bytes, const uint32_t* box, int swizzle) {
     if (!g_encode || rank < 3 || rank > 5) return false;

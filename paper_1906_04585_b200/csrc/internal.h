@@ -133,6 +133,8 @@ bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t
 // rows x cols fp32 matrix, unswizzled box_rows x box_cols tile (gemm_init() first).
 bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
                          uint32_t box_cols, uint32_t box_rows);
+bool make_tensor_map_f32_wide(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
+                              uint32_t box_blocks, uint32_t box_rows);
 // General bf16 tensor map of rank 3..5 (dims/strides innermost first).  swizzle: 0 = 128-byte, 1 = 64-byte
 // (64-byte rows), 2 = 32-byte (32-byte rows).  Dimensions may overlap (a stride smaller than the extent
 // below it); a box may be larger than a dimension (the rest reads as zero).

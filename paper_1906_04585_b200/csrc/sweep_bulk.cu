@@ -48,13 +48,24 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, int* er
 // One instruction moves a [all agents] x [cols] box of a row-major [n_agents][d_pad] fp32 array
 // (column coordinate c0 is a multiple of 4 floats = 16 bytes; columns past d_pad read as zero and
 // are not written).
-__device__ __forceinline__ void tile_load(void* dst, const CUtensorMap* map, int c0, uint64_t* bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(s_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(0), "r"(s_u32(bar)) : "memory");
+// With few agents a 256-column box is small and the copy engine, which is bound by instructions, cannot keep
+// up; the arrays are then seen as [agents][d_pad / 256][256] and a box takes several 256-column blocks
+// (wide = 1: c0 is a multiple of 256 and the coordinates are (0, c0 / 256, 0)).
+__device__ __forceinline__ void tile_load(void* dst, const CUtensorMap* map, int c0, uint64_t* bar, int wide) {
+    if (wide)
+        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                     ::"r"(s_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(c0 >> 8), "r"(0), "r"(s_u32(bar)) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                     ::"r"(s_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(0), "r"(s_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tile_store(const CUtensorMap* map, int c0, const void* src) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(0), "r"(s_u32(src)) : "memory");
+__device__ __forceinline__ void tile_store(const CUtensorMap* map, int c0, const void* src, int wide) {
+    if (wide)
+        asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                     ::"l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(c0 >> 8), "r"(0), "r"(s_u32(src)) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                     ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(0), "r"(s_u32(src)) : "memory");
 }
 
 // sqrt and the quotient use the hardware approximations (about 1e-7 relative each), far inside the
@@ -86,7 +97,7 @@ template <int P>
 __global__ void __launch_bounds__(kConsumers + 32, 1)
 sweep_sync_bulk_kernel(const __grid_constant__ CUtensorMap mx, const __grid_constant__ CUtensorMap mg,
                        const __grid_constant__ CUtensorMap mv, const float* __restrict__ clip, __nv_bfloat16* __restrict__ shadow, int n_agents, long d_pad,
-                       int cols, int kBulkStages, long n_tiles, int off0, int off1, SweepHp hp, int* error_word) {
+                       int cols, int kBulkStages, long n_tiles, int off0, int off1, SweepHp hp, int* error_word, int wide) {
     extern __shared__ __align__(128) float smem[];
     __shared__ __align__(8) uint64_t full[kMaxBulkStages];
     __shared__ __align__(8) uint64_t done[kMaxBulkStages];
@@ -109,16 +120,17 @@ sweep_sync_bulk_kernel(const __grid_constant__ CUtensorMap mx, const __grid_cons
     const long my_tiles = first < n_tiles ? (n_tiles - first + step - 1) / step : 0;
 
     if (warp == kConsumers / 32) {
-        // ---------------- mover warp (one elected lane issues the tensor copies)
+        // ---------------- mover warp (one elected lane issues the tensor copies; issuing the three loads from
+        // three lanes side by side was measured and is no faster)
         if (lane == 0) {
             const uint32_t stage_bytes = (uint32_t)stage_floats * 4u;
             auto issue_loads = [&](long k, int stage) {
                 const int c0 = (int)((first + k * step) * cols);
                 float* sx = smem + (long)stage * stage_floats;
                 bar_expect(&full[stage], stage_bytes);
-                tile_load(sx, &mx, c0, &full[stage]);
-                tile_load(sx + n_agents * cols, &mg, c0, &full[stage]);
-                tile_load(sx + 2 * n_agents * cols, &mv, c0, &full[stage]);
+                tile_load(sx, &mx, c0, &full[stage], wide);
+                tile_load(sx + n_agents * cols, &mg, c0, &full[stage], wide);
+                tile_load(sx + 2 * n_agents * cols, &mv, c0, &full[stage], wide);
             };
             for (int s = 0; s < kBulkStages && s < my_tiles; s++) issue_loads(s, s);
             for (long k = 0; k < my_tiles; k++) {
@@ -126,8 +138,8 @@ sweep_sync_bulk_kernel(const __grid_constant__ CUtensorMap mx, const __grid_cons
                 if (!bar_wait(&done[stage], (uint32_t)(k / kBulkStages) & 1u, error_word)) break;
                 const int c0 = (int)((first + k * step) * cols);
                 const float* sg = smem + (long)stage * stage_floats + n_agents * cols;
-                tile_store(&mx, c0, sg);
-                tile_store(&mv, c0, sg + n_agents * cols);
+                tile_store(&mx, c0, sg, wide);
+                tile_store(&mv, c0, sg + n_agents * cols, wide);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 if (k >= 1 && k - 1 + kBulkStages < my_tiles) {
                     // stage of step k-1: all but the newest group of stores must have left shared memory
@@ -206,17 +218,26 @@ cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const flo
     const long budget = 200L * 1024;
     int cols = (int)(budget / (3L * 12 * n_agents));
     cols = cols / 32 * 32;
-    if (cols > 256) cols = 256;     // box edge limit of a tensor copy
+    // a box edge holds at most 256 elements; wider tiles (few agents) take several 256-column blocks per copy
+    const int wide = cols >= 512 && (d_pad & 255) == 0;
+    if (wide) { cols = cols / 256 * 256; if (cols > 1024) cols = 1024; }
+    else if (cols > 256) cols = 256;
     if (cols < 32) return cudaErrorNotSupported;
     int stages = (int)(budget / ((long)12 * n_agents * cols));
     if (stages > kMaxBulkStages) stages = kMaxBulkStages;
     if (stages < 2) return cudaErrorNotSupported;
     if (gemm_init() != cudaSuccess) return cudaErrorNotSupported;
     CUtensorMap mx, mg, mv;
-    if (!make_tensor_map_f32(&mx, x, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols, n_agents) ||
-        !make_tensor_map_f32(&mg, g, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols, n_agents) ||
-        !make_tensor_map_f32(&mv, v, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols, n_agents))
-        return cudaErrorNotSupported;
+    bool ok;
+    if (wide)
+        ok = make_tensor_map_f32_wide(&mx, x, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols / 256, n_agents) &&
+             make_tensor_map_f32_wide(&mg, g, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols / 256, n_agents) &&
+             make_tensor_map_f32_wide(&mv, v, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols / 256, n_agents);
+    else
+        ok = make_tensor_map_f32(&mx, x, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols, n_agents) &&
+             make_tensor_map_f32(&mg, g, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols, n_agents) &&
+             make_tensor_map_f32(&mv, v, (uint64_t)d_pad, (uint64_t)n_agents, (uint64_t)d_pad * 4, cols, n_agents);
+    if (!ok) return cudaErrorNotSupported;
     const long n_tiles = (d_pad + cols - 1) / cols;
     const size_t smem = (size_t)stages * 3 * n_agents * cols * 4;
     int grid = (int)(n_tiles < 148 ? n_tiles : 148);
@@ -225,7 +246,7 @@ cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const flo
     e = cudaFuncSetAttribute(sweep_sync_bulk_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
     if (e != cudaSuccess) return e;                                                                          \
     (void)launch_pdl(sweep_sync_bulk_kernel<P>, dim3(grid), dim3(kConsumers + 32), smem, st, mx, mg, mv, clip, shadow, n_agents, d_pad, cols, \
-                                                                   stages, n_tiles, o0, o1, hp, error_word);
+                                                                   stages, n_tiles, o0, o1, hp, error_word, wide);
     if (n_peers == 0) { GALA_BULK_LAUNCH(0) }
     else if (n_peers == 1) { GALA_BULK_LAUNCH(1) }
     else if (n_peers == 2) { GALA_BULK_LAUNCH(2) }
