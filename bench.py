@@ -38,7 +38,7 @@ L2_BYTES = 126 * 1024 * 1024
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture of the named kernel
 # class on this workload; None until captured, and again None once that kernel changes.
-NCU_TRAFFIC_BYTES = {"sweep_sync": 239.5e6}   # profiles/hidden_layer_gemm_and_sweep_c2_step.md (8 agents, conv net)
+NCU_TRAFFIC_BYTES = {"sweep_sync": 240.5e6}   # profiles/sweep_sync_bulk_c2_step.md (8 agents, conv net, wide tiles)
 
 
 def peaks():
