@@ -195,7 +195,9 @@ int gala_set_agent_ctas(gala_ctx* ctx, int ctas);
  * to its kernel in csrc/env.cu and restated in gala_inputs.synthetic_env: observations (uint8 frames or float
  * vectors) and the uniform for the action draw depend on the step only, reward = 1 when the action equals a
  * hidden per-step target, done with probability 0.01.  Steps are numbered per agent from 0 and continue over
- * calls.  The rollout buffers belong to the library (allocated by the first call for an agent).  Returns as
+ * calls.  The rollout buffers belong to the library (allocated by the first call for an agent).  Unless graph
+ * replay is off (gala_set_graphs), an agent's iteration without its gossip step is captured on its second run
+ * and replayed as one graph launch from the third on.  Returns as
  * gala_learn / gala_gossip do (GALA_ETIMEOUT from a staleness-bounded gossip step ends the loop early). */
 int gala_actor_loop(gala_ctx* ctx, int agent, int iterations, unsigned long long env_seed);
 /* Waits for the agent's stream and copies the rollout of its last loop iteration to HOST memory (any pointer

@@ -215,9 +215,11 @@ cudaError_t launch_heads_fwd(const HeadsArgs& a, int groups, cudaStream_t st) {
     if (bx * groups > 592) bx = (592 + groups - 1) / groups;
     if (bx < 1) bx = 1;
     const size_t smem = (size_t)((a.A + 1) + 8) * a.H * sizeof(float);
-    if (smem > 40 * 1024) {   // well below the 48 KiB that need no opt-in
+    static size_t opted = 0;   // raised only when a launch needs more (never lowered), so replays of a captured launch need no call
+    if (smem > 40 * 1024 && smem > opted) {   // 40 KiB: well below the 48 KiB that need no opt-in
         cudaError_t e = cudaFuncSetAttribute(heads_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
+        opted = smem;
     }
     (void)launch_pdl(heads_fwd_kernel, dim3(dim3(bx, groups)), dim3(256), smem, st, a);
     return cudaGetLastError();

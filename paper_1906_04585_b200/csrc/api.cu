@@ -17,27 +17,6 @@ constexpr long kFramePix = 84L * 84 * 4;
 
 namespace {
 
-struct Agent {
-    cudaStream_t stream = nullptr, lib_stream = nullptr;
-    cudaEvent_t pub_event[2] = {nullptr, nullptr};  // completion of the sweep that wrote snapshot slot s
-    cudaEvent_t sweep_done = nullptr;               // completion of the agent's latest sweep
-    cudaEvent_t fence = nullptr;                    // scratch event for cross-stream ordering
-    long long version = 0;                          // newest snapshot version enqueued (0: none)
-    long long round = 0;                            // local iteration counter
-    bool pending = false;                           // a gradient waits for its optimiser step
-    long long since_mix = 0;                        // local iterations since the last average with the in-peers
-    std::vector<long long> consumed;                // newest version consumed from each agent
-    std::vector<int> slot_readers[2];               // agents whose sweeps read snapshot slot s
-    long long frames = 0, mixes = 0, skipped = 0, stale_sum = 0, stale_max = 0, stale_waits = 0;
-    // closed actor loop: rollout buffers owned by the library and the environment's step counter
-    void* loop_obs = nullptr; int* loop_actions = nullptr; float* loop_rewards = nullptr;
-    unsigned char* loop_dones = nullptr; float* loop_uniforms = nullptr;
-    long long env_step = 0;
-    int last_n = 0, last_mixed = 0;
-    int last_peers[2] = {0, 0};
-    long long last_versions[2] = {0, 0};
-};
-
 struct Plan {  // one tensor-core product with its descriptors
     GemmOperand A, B;
     GemmArgs args;
@@ -86,6 +65,30 @@ struct StepGraph {
     bool failed = false;            // capture or instantiation did not work: launch directly
     long long launches = 0;         // kernels inside
     long long tag_launches[T_COUNT] = {};
+};
+
+struct Agent {
+    cudaStream_t stream = nullptr, lib_stream = nullptr;
+    cudaEvent_t pub_event[2] = {nullptr, nullptr};  // completion of the sweep that wrote snapshot slot s
+    cudaEvent_t sweep_done = nullptr;               // completion of the agent's latest sweep
+    cudaEvent_t fence = nullptr;                    // scratch event for cross-stream ordering
+    long long version = 0;                          // newest snapshot version enqueued (0: none)
+    long long round = 0;                            // local iteration counter
+    bool pending = false;                           // a gradient waits for its optimiser step
+    long long since_mix = 0;                        // local iterations since the last average with the in-peers
+    std::vector<long long> consumed;                // newest version consumed from each agent
+    std::vector<int> slot_readers[2];               // agents whose sweeps read snapshot slot s
+    long long frames = 0, mixes = 0, skipped = 0, stale_sum = 0, stale_max = 0, stale_waits = 0;
+    // closed actor loop: rollout buffers owned by the library and the environment's step counter
+    void* loop_obs = nullptr; int* loop_actions = nullptr; float* loop_rewards = nullptr;
+    unsigned char* loop_dones = nullptr; float* loop_uniforms = nullptr;
+    long long* env_step_dev = nullptr;              // the step counter the environment kernels read
+    long long env_step = 0;                         // its host mirror (steps enqueued so far)
+    StepGraph loop_graph;                           // one loop iteration (act, environment, learn) as a graph
+    unsigned long long loop_seed = 0; int loop_seen = 0;
+    int last_n = 0, last_mixed = 0;
+    int last_peers[2] = {0, 0};
+    long long last_versions[2] = {0, 0};
 };
 
 }  // namespace
@@ -1236,6 +1239,7 @@ int gala_destroy(gala_ctx* c) {
         if (a.fence) cudaEventDestroy(a.fence);
     }
     for (StepGraph& g : c->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
+    for (Agent& a : c->agents) if (a.loop_graph.exec) cudaGraphExecDestroy(a.loop_graph.exec);
     if (c->side_stream) cudaStreamDestroy(c->side_stream);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
@@ -1266,44 +1270,102 @@ int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int
     return GALA_OK;
 }
 
+// One iteration of the closed loop without the gossip step, enqueued on the agent's stream: the observation the
+// rollout starts from, T x (act, environment step), the learner step, and the advance of the step counter.
+static int actor_iteration(gala_ctx* c, int agent, unsigned long long env_seed) {
+    Agent& ag = c->agents[agent];
+    const int T = c->T, E = c->E;
+    const long obs_elems = c->conv ? kFramePix : c->obs_dim;
+    const long obs_bytes = obs_elems * (c->conv ? 1 : 4);
+    uint8_t* obs = reinterpret_cast<uint8_t*>(ag.loop_obs);
+    EnvArgs ea{};
+    ea.seed = env_seed; ea.agent = agent; ea.n_actions = c->A; ea.step_base = ag.env_step_dev;
+    ea.uniforms = ag.loop_uniforms; ea.obs_elems = obs_elems; ea.frames = c->conv ? 1 : 0;
+    EnvArgs first = ea;   // the environment is a function of the step: the first observation is produced again
+    first.obs_step = 0; first.obs_out = obs;
+    LAUNCH(T_ENV, ag.stream, launch_env(first, E, ag.stream));
+    for (int t = 0; t < T; t++) {
+        int r = gala_act(c, agent, obs + (long)t * E * obs_bytes, ag.loop_uniforms, ag.loop_actions + (long)t * E, nullptr);
+        if (r != GALA_OK) return r;
+        EnvArgs st = ea;
+        st.step = t; st.actions = ag.loop_actions + (long)t * E;
+        st.rewards = ag.loop_rewards + (long)t * E; st.dones = ag.loop_dones + (long)t * E;
+        st.obs_step = t + 1; st.obs_out = obs + (long)(t + 1) * E * obs_bytes;
+        LAUNCH(T_ENV, ag.stream, launch_env(st, E, ag.stream));
+    }
+    gala_rollout ro{obs, ag.loop_actions, ag.loop_rewards, ag.loop_dones};
+    c->cur_ctas = c->agent_ctas;
+    int r = learn_range(c, agent, 1, &ro, ag.stream);
+    c->cur_ctas = 0;
+    if (r != GALA_OK) return r;
+    LAUNCH(T_ENV, ag.stream, launch_env_advance(ag.env_step_dev, T, ag.stream));
+    return GALA_OK;
+}
+
 int gala_actor_loop(gala_ctx* c, int agent, int iterations, unsigned long long env_seed) {
     if (!valid_agent(c, agent) || iterations < 0) return fail(c, GALA_EINVAL, "gala_actor_loop: bad agent or iteration count");
     if (c->topo.kind == GALA_TOPO_COMPLETE)
         return fail(c, GALA_ESTATE, "gala_actor_loop: the complete graph (gradient all-reduce) exists only as gala_step_sync");
     Agent& ag = c->agents[agent];
     const int T = c->T, E = c->E;
-    const long obs_elems = c->conv ? kFramePix : c->obs_dim;
-    const long obs_bytes = obs_elems * (c->conv ? 1 : 4);
+    const long obs_bytes = c->conv ? kFramePix : (long)c->obs_dim * 4;
     if (!ag.loop_obs) {
         uint8_t* ob = nullptr;
         ALLOC(ob, (size_t)(T + 1) * E * obs_bytes);
         ALLOC(ag.loop_actions, (size_t)T * E); ALLOC(ag.loop_rewards, (size_t)T * E);
         ALLOC(ag.loop_dones, (size_t)T * E); ALLOC(ag.loop_uniforms, (size_t)E);
+        ALLOC(ag.env_step_dev, 1);
         ag.loop_obs = ob;
     }
-    uint8_t* obs = reinterpret_cast<uint8_t*>(ag.loop_obs);
-    EnvArgs ea{};
-    ea.seed = env_seed; ea.agent = agent; ea.n_actions = c->A;
-    ea.uniforms = ag.loop_uniforms; ea.obs_elems = obs_elems; ea.frames = c->conv ? 1 : 0;
+    if (ag.loop_seed != env_seed) {   // the captured iteration carries the seed
+        if (ag.loop_graph.exec) { cudaGraphExecDestroy(ag.loop_graph.exec); ag.loop_graph.exec = nullptr; }
+        ag.loop_graph.failed = false;
+        ag.loop_seed = env_seed; ag.loop_seen = 0;
+    }
+    const unsigned long long outside = (1ull << T_SWEEP_SYNC) | (1ull << T_SWEEP_AGENT);
     for (int it = 0; it < iterations; it++) {
-        const long long s0 = ag.env_step;
-        EnvArgs first = ea;   // the observation the rollout starts from (the environment is a function of the step)
-        first.obs_step = s0; first.obs_out = obs;
-        LAUNCH(T_ENV, ag.stream, launch_env(first, E, ag.stream));
-        for (int t = 0; t < T; t++) {
-            int r = gala_act(c, agent, obs + (long)t * E * obs_bytes, ag.loop_uniforms, ag.loop_actions + (long)t * E, nullptr);
-            if (r != GALA_OK) return r;
-            EnvArgs st = ea;
-            st.step = s0 + t; st.actions = ag.loop_actions + (long)t * E;
-            st.rewards = ag.loop_rewards + (long)t * E; st.dones = ag.loop_dones + (long)t * E;
-            st.obs_step = s0 + t + 1; st.obs_out = obs + (long)(t + 1) * E * obs_bytes;
-            LAUNCH(T_ENV, ag.stream, launch_env(st, E, ag.stream));
+        if (ag.pending) {  // a gradient that no gossip step has consumed: apply it without mixing, publish
+            int r0 = sweep_agent(c, agent, false);
+            if (r0 != GALA_OK) return r0;
+            ag.round++;
         }
-        gala_rollout ro{obs, ag.loop_actions, ag.loop_rewards, ag.loop_dones};
-        int r = gala_learn(c, agent, &ro);
-        if (r != GALA_OK) return r;
-        if ((r = gala_gossip(c, agent)) != GALA_OK) return r;
+        StepGraph& g = ag.loop_graph;
+        const bool graphs = c->use_graphs >= 1 && (c->profile_mask & ~outside) == 0 && !c->legacy_conv && !g.failed;
+        int r = GALA_OK;
+        if (graphs && g.exec) {            // third iteration on: one graph launch
+            CK(cudaGraphLaunch(g.exec, ag.stream));
+            c->launches += g.launches;
+            for (int k = 0; k < T_COUNT; k++) c->tag_launches[k] += g.tag_launches[k];
+            ag.pending = true; ag.frames += c->S;
+        } else if (graphs && ag.loop_seen >= 1 && cudaStreamBeginCapture(ag.stream, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
+            const long long l0 = c->launches;   // second iteration: captured, instantiated, launched
+            long long t0[T_COUNT];
+            for (int k = 0; k < T_COUNT; k++) t0[k] = c->tag_launches[k];
+            r = actor_iteration(c, agent, env_seed);
+            cudaGraph_t graph = nullptr;
+            cudaError_t e = cudaStreamEndCapture(ag.stream, &graph);
+            if (r == GALA_OK && e == cudaSuccess && graph) e = cudaGraphInstantiate(&g.exec, graph, 0);
+            if (graph) cudaGraphDestroy(graph);
+            if (r != GALA_OK || e != cudaSuccess || !g.exec) {
+                (void)cudaGetLastError();
+                g.failed = true; g.exec = nullptr;
+                c->launches = l0;
+                for (int k = 0; k < T_COUNT; k++) c->tag_launches[k] = t0[k];
+                if (r != GALA_OK) return r;
+                ag.frames -= c->S;     // counted again by the direct pass
+                if ((r = actor_iteration(c, agent, env_seed)) != GALA_OK) return r;
+            } else {
+                g.launches = c->launches - l0;
+                for (int k = 0; k < T_COUNT; k++) g.tag_launches[k] = c->tag_launches[k] - t0[k];
+                CK(cudaGraphLaunch(g.exec, ag.stream));
+            }
+        } else {                           // first iteration (or no graphs): direct launches
+            (void)cudaGetLastError();
+            if ((r = actor_iteration(c, agent, env_seed)) != GALA_OK) return r;
+        }
+        ag.loop_seen++;
         ag.env_step += T;
+        if ((r = gala_gossip(c, agent)) != GALA_OK) return r;
     }
     return GALA_OK;
 }

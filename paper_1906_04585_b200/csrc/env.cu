@@ -30,6 +30,11 @@ __global__ void __launch_bounds__(256) env_kernel(EnvArgs a) {
     pdl_wait();
     pdl_launch();
     const int e = blockIdx.y;
+    if (a.step_base) {   // steps counted from a counter in device memory (the same launch replayed for every rollout)
+        const long long base = *a.step_base;
+        a.step += base;
+        a.obs_step += base;
+    }
     if (a.actions && blockIdx.x == 0 && threadIdx.x == 0) {
         const uint64_t b = env_base(a.seed, a.agent, e, a.step);
         const uint64_t hr = sm64(b + (1ull << 56)), hd = sm64(b + (2ull << 56));
@@ -48,6 +53,17 @@ __global__ void __launch_bounds__(256) env_kernel(EnvArgs a) {
         for (long j = blockIdx.x * (long)blockDim.x + threadIdx.x; j < a.obs_elems; j += (long)gridDim.x * blockDim.x)
             out[j] = ((float)(sm64(b + (uint64_t)j) >> 40) * 1.1920928955078125e-7f - 1.0f) * 1.7320508f;
     }
+}
+
+// *counter += by, after the last environment step of a rollout
+__global__ void env_advance_kernel(long long* counter, long long by) {
+    pdl_wait();
+    pdl_launch();
+    if (threadIdx.x == 0 && blockIdx.x == 0) *counter += by;
+}
+cudaError_t launch_env_advance(long long* counter, long long by, cudaStream_t st) {
+    (void)launch_pdl(env_advance_kernel, dim3(1), dim3(32), 0, st, counter, by);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_env(const EnvArgs& a, int n_envs, cudaStream_t st) {

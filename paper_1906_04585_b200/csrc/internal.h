@@ -380,6 +380,7 @@ cudaError_t launch_mlp_fused(const MlpFusedArgs& a, int groups, cudaStream_t st)
 struct EnvArgs {
     unsigned long long seed;
     int agent, n_actions;
+    const long long* step_base;  // device counter added to `step` and `obs_step` (null: they are absolute)
     long long step;              // transition whose reward / done flag is produced (if actions != null)
     const int* actions;          // [E] actions taken at `step`, or null
     float* rewards;              // [E]
@@ -391,6 +392,7 @@ struct EnvArgs {
     int frames;                  // 1: uint8 frames, 0: float vectors
 };
 cudaError_t launch_env(const EnvArgs& a, int n_envs, cudaStream_t st);
+cudaError_t launch_env_advance(long long* counter, long long by, cudaStream_t st);
 
 // ---------------------------------------------------------------- conv lowering
 // uint8 frames -> bf16 (exact), per group [samples][84*84*4]
