@@ -5,7 +5,7 @@
 //     D[pixel][n] += X[pixel + offset(tap)][k] * Wtap[k][n] .
 // When the pixels of an image are laid out row after row with a fixed pitch, "pixel + offset" is a
 // constant row shift, so every tap reads the SAME shared-memory image of the input, only from a
-// start address moved by shift * row_bytes.  The input of one work unit (a sample, or five output
+// start address moved by shift * row_bytes.  The input of one work unit (a sample, or six output
 // lines of conv1) is therefore fetched once by TMA - not once per tap - and all weights of the layer
 // stay in shared memory while a CTA works on one agent.  Rows whose pixel falls outside the valid
 // output range (the pitch minus the output width, the tail of the 128-row MMA tile) are computed
@@ -42,27 +42,27 @@ namespace gala {
 
 template <int V> struct ConvTraits;
 template <> struct ConvTraits<CV_CONV1_FWD> {
-    static constexpr int ROWB = 32, LAYOUT = 6, PLANES = 4, PLANE_ROWS = 126, PLANE_STRIDE = 4096, UPS = 4;
-    static constexpr int TAPS = 16, KKN = 1, BN = 32, PITCH = 21, OH = 5, OW = 20;
+    static constexpr int ROWB = 32, LAYOUT = 6, PLANES = 4, PLANE_ROWS = 147, PLANE_STRIDE = 4864;
+    static constexpr int TAPS = 16, KKN = 1, BN = 32, PITCH = 21, OH = 6, OW = 20;
     static constexpr int W_BOXES = 16, W_BOX_BYTES = 1024, B_MN = 0, B_LAYOUT = 6, B_SBO = 256, B_LBO = 16;
 };
 template <> struct ConvTraits<CV_CONV2_FWD> {
-    static constexpr int ROWB = 64, LAYOUT = 4, PLANES = 4, PLANE_ROWS = 100, PLANE_STRIDE = 6656, UPS = 1;
+    static constexpr int ROWB = 64, LAYOUT = 4, PLANES = 4, PLANE_ROWS = 100, PLANE_STRIDE = 6656;
     static constexpr int TAPS = 16, KKN = 2, BN = 64, PITCH = 10, OH = 9, OW = 9;
     static constexpr int W_BOXES = 16, W_BOX_BYTES = 4096, B_MN = 0, B_LAYOUT = 4, B_SBO = 512, B_LBO = 16;
 };
 template <> struct ConvTraits<CV_CONV3_FWD> {
-    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 81, PLANE_STRIDE = 11264, UPS = 1;
+    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 81, PLANE_STRIDE = 11264;
     static constexpr int TAPS = 9, KKN = 4, BN = 64, PITCH = 9, OH = 7, OW = 7;
     static constexpr int W_BOXES = 9, W_BOX_BYTES = 8192, B_MN = 0, B_LAYOUT = 2, B_SBO = 1024, B_LBO = 16;
 };
 template <> struct ConvTraits<CV_CONV2_DGRAD> {
-    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 121, PLANE_STRIDE = 16384, UPS = 1;
+    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 121, PLANE_STRIDE = 16384;
     static constexpr int TAPS = 4, KKN = 4, BN = 128, PITCH = 11, OH = 10, OW = 10;
     static constexpr int W_BOXES = 16, W_BOX_BYTES = 4096, B_MN = 1, B_LAYOUT = 4, B_SBO = 512, B_LBO = 4096;
 };
 template <> struct ConvTraits<CV_CONV3_DGRAD> {
-    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 121, PLANE_STRIDE = 16384, UPS = 1;
+    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 121, PLANE_STRIDE = 16384;
     static constexpr int TAPS = 9, KKN = 4, BN = 64, PITCH = 11, OH = 9, OW = 9;
     static constexpr int W_BOXES = 9, W_BOX_BYTES = 8192, B_MN = 1, B_LAYOUT = 2, B_SBO = 1024, B_LBO = 8192;
 };
@@ -71,11 +71,16 @@ constexpr int kConvMaxStages = 8;
 constexpr int kConvSlack = 8 * 1024;             // rows an MMA reads past the last plane of the ring
 constexpr int kConvEpiWarpBytes = 512;           // an epilogue warp's copy of the layer's bias
 constexpr int kConvSmemMax = 224 * 1024;
-// conv1 reads the uint8 frames themselves: the 24 input lines behind five output lines are one
-// contiguous piece of 24 * 84 * 4 bytes, staged as it is and widened to bf16 planes by four more warps
+// conv1 reads the uint8 frames themselves.  An agent's frames are one long run of groups of four lines
+// (1344 bytes each, 21 per frame), and output line L of that run (frame L / 21, line L % 21; line 20 of a
+// frame does not exist and is dropped) needs groups L and L + 1.  A unit is six consecutive output lines
+// wherever frames begin and end: 126 of the 128 rows of an MMA are pixel slots.  The seven groups behind
+// them are one contiguous piece, staged as it is and widened to bf16 planes by four more warps.
+constexpr int kC1Lines = 6;                          // output lines of a unit
+constexpr int kC1Group = 4 * 336;                    // bytes of four input lines
 constexpr int kU8Stages = 4;
-constexpr int kU8Bytes = 24 * 336;       // 8064
-constexpr int kU8Stride = 8192;
+constexpr int kU8Bytes = (kC1Lines + 1) * kC1Group;  // 9408
+constexpr int kU8Stride = 9728;
 constexpr int kConvThreads = 352, kConv1Threads = 352 + 128;
 
 // plane and row shift of a tap
@@ -97,14 +102,18 @@ template <int V> __device__ __forceinline__ int weight_col(int j) {
     } else return j * 64;
 }
 
-struct UnitCoord { int gz, s, q; };
+// units of one agent: a sample each, except conv1 (six output lines of the agent's run of frames)
+template <int V> __host__ __device__ __forceinline__ int units_per_group(int rows) {
+    if constexpr (V == CV_CONV1_FWD) return (21 * rows + kC1Lines - 1) / kC1Lines;
+    else return rows;
+}
+// gz: agent within the launch; s: sample (conv1: unit within the agent)
+struct UnitCoord { int gz, s; };
 template <int V> __device__ __forceinline__ UnitCoord decode_unit(int u, int rows) {
-    constexpr int UPS = ConvTraits<V>::UPS;
+    const int upg = units_per_group<V>(rows);
     UnitCoord c;
-    c.q = u % UPS;
-    const int r = u / UPS;
-    c.gz = r / rows;
-    c.s = r - c.gz * rows;
+    c.gz = u / upg;
+    c.s = u - c.gz * upg;
     return c;
 }
 
@@ -198,16 +207,18 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (lane == 0) issued_w = wl;
             }
             if constexpr (kU8) {
-                // lines 20q .. 20q+23 of the frame, as stored: one bulk copy of 8064 bytes
+                // groups 6v .. 6v+6 of the agent's frames, as stored: one bulk copy (shorter at the very end)
                 const int su = it % kU8Stages;
                 int go = 1;
                 if (lane == 0) go = mbar_wait(&u8_empty[su], ((uint32_t)(it / kU8Stages) & 1u) ^ 1u, &abort_flag) ? 1 : 0;
                 go = __shfl_sync(0xffffffffu, go, 0);
                 if (!go) break;
                 if (lane == 0) {
-                    mbar_expect_tx(&u8_full[su], (uint32_t)kU8Bytes);
-                    const uint8_t* src = reinterpret_cast<const uint8_t*>(p.obs.p[c.gz]) + (long)c.s * (84 * 336) + c.q * (20 * 336);
-                    bulk_load_1d(smU + su * kU8Stride, src, (uint32_t)kU8Bytes, &u8_full[su]);
+                    const int left = 21 * p.rows - kC1Lines * c.s;   // groups from this unit's first to the last
+                    const uint32_t bytes = (uint32_t)((left < kC1Lines + 1 ? left : kC1Lines + 1) * kC1Group);
+                    mbar_expect_tx(&u8_full[su], bytes);
+                    const uint8_t* src = reinterpret_cast<const uint8_t*>(p.obs.p[c.gz]) + (long)c.s * (kC1Lines * kC1Group);
+                    bulk_load_1d(smU + su * kU8Stride, src, bytes, &u8_full[su]);
                     issued_iters = it + 1;
                 }
                 continue;
@@ -240,7 +251,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             for (int u = u_begin; u < u_end; u++, it++) {
                 // Both issuers follow every change of agent: each reports (through a commit, so only once its
                 // MMAs are complete) that it is done with the old weights, then waits for the new ones.
-                const int gz = (u / T::UPS) / p.rows;
+                const int gz = u / units_per_group<V>(p.rows);
                 if (gz != cur_g) {
                     if (cur_g >= 0) umma_commit(&w_empty);
                     if (!mbar_wait(&w_full, (uint32_t)wl & 1u, &abort_flag)) break;
@@ -280,7 +291,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         }
     } else if (warp >= 11) {
         // ------------------------------------------------ conv1: uint8 lines -> bf16 phase planes
-        // Line yl of the block (y = 20q + yl) belongs to plane yl % 4, row (yl / 4) * 21 + xq for its 16-byte
+        // Line yl of the block (28 lines = 7 groups of 4) belongs to plane yl % 4, row (yl / 4) * 21 + xq for its 16-byte
         // group xq (4 pixels x 4 channels); a row is 32 bytes of bf16 whose two halves swap when bit 7 of
         // its address is set (32-byte swizzle).  0..255 are exact in bf16; 1/255 is applied after the MMAs.
         if constexpr (kU8) {
@@ -293,9 +304,9 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const uint8_t* src = smU + su * kU8Stride;
                 uint8_t* dstage = smX + s * STAGE;
 #pragma unroll
-                for (int k = 0; k < 4; k++) {
-                    const int ch = ct + k * 128;          // 16-byte group of the block, 504 in all
-                    if (ch < 24 * 21) {
+                for (int k = 0; k < 5; k++) {
+                    const int ch = ct + k * 128;          // 16-byte group of the block, 588 in all
+                    if (ch < 4 * (kC1Lines + 1) * 21) {
                         const int yl = ch / 21, xq = ch - yl * 21;
                         const uint4 v = *reinterpret_cast<const uint4*>(src + ch * 16);
                         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -331,10 +342,13 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         float* sbias = reinterpret_cast<float*>(smE + (warp - 2) * kConvEpiWarpBytes);   // this warp's copy of the bias
         const int m = q * 32 + lane;
         const int pa = m / T::PITCH, pb = m - pa * T::PITCH;
-        const bool valid = pa < T::OH && pb < T::OW;
+        const bool in_tile = pa < T::OH && pb < T::OW;
         // element offset of this thread's pixel inside the agent's tensor (pixel (2a, 2b) for the conv2 gradient)
         auto pixel_off = [&](const UnitCoord& c) -> long {
-            if constexpr (V == CV_CONV1_FWD) return ((long)c.s * 400 + (5 * c.q + pa) * 20 + pb) * 32;
+            if constexpr (V == CV_CONV1_FWD) {   // line L of the run = line L % 21 of frame L / 21
+                const int L = kC1Lines * c.s + pa, f = L / 21;
+                return ((long)f * 400 + (L - f * 21) * 20 + pb) * 32;
+            }
             else if constexpr (V == CV_CONV2_FWD) return ((long)c.s * 81 + pa * 9 + pb) * 64;
             else if constexpr (V == CV_CONV3_FWD) return ((long)c.s * 49 + pa * 7 + pb) * 64;
             else if constexpr (V == CV_CONV2_DGRAD) return ((long)c.s * 400 + (2 * pa) * 20 + 2 * pb) * 32;
@@ -348,7 +362,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if constexpr (!kFwd) {
 #pragma unroll
                 for (int ch = 0; ch < NCH; ch++) g[ch] = 0u;
-                if (u < u_end && valid) {
+                if (u < u_end && in_tile) {
                     const UnitCoord c = decode_unit<V>(u, p.rows);
                     const uint32_t* gp = p.gate_in + (long)c.gz * p.gate_group_stride + pixel_off(c) / 32;
                     if constexpr (V == CV_CONV2_DGRAD) {   // words of pixels (2a, 2b), (2a, 2b+1), (2a+1, 2b), (2a+1, 2b+1)
@@ -368,6 +382,11 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         for (int u = u_begin + eg; u < u_end; u += 2, it += 2) {
             const UnitCoord c = decode_unit<V>(u, p.rows);
             const long off = pixel_off(c);
+            bool valid = in_tile;
+            if constexpr (V == CV_CONV1_FWD) {   // not the line between two frames, not past the last frame
+                const int L = kC1Lines * c.s + pa;
+                valid = in_tile && L % 21 < 20 && L < 21 * p.rows;
+            }
             __nv_bfloat16* out = p.out + (long)c.gz * p.out_group_stride + off;
             // column block c0 -> where it goes: forward, conv3 gradient: channels c0.. of the pixel; conv2
             // gradient: block = parity class (py, px) -> pixel (2a + py, 2b + px), all 32 channels
@@ -542,7 +561,7 @@ static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, con
     int nst = (kConvSmemMax - fixed) / STAGE;
     if (nst > kConvMaxStages) nst = kConvMaxStages;
     if (nst < 2) return cudaErrorInvalidValue;
-    const long units = (long)a.groups * a.rows * T::UPS;
+    const long units = (long)a.groups * units_per_group<V>(a.rows);
     if (units <= 0) return cudaSuccess;
     if (units > 0x7fffffffL) return cudaErrorInvalidValue;
     const size_t smem = (size_t)fixed + (size_t)nst * STAGE;
