@@ -802,7 +802,16 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         if ((r = fork()) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_wgrad, agent0, groups, 0, ws)) != GALA_OK) return r;
         if ((r = run_plan(c, c->fc_dgrad, agent0, groups, 0, st)) != GALA_OK) return r;
+        // The chain ends with conv2's data gradient, the second stream is still busy with weight gradients
+        // then: conv1's weight gradient, its slice sum and the column sums follow the chain on `st`.
+        const bool tail_on_chain = side && !c->legacy_conv;
         for (int l = 2; l >= 0; l--) {
+            if (l == 0 && tail_on_chain) {
+                if ((r = flush_pending_reduces(c, agent0, groups, ws)) != GALA_OK) return r;
+                if ((r = run_conv1_wgrad(c, agent0, groups, obs, st)) != GALA_OK) return r;
+                if ((r = flush_pending_reduces(c, agent0, groups, st)) != GALA_OK) return r;
+                break;
+            }
             if ((r = fork()) != GALA_OK) return r;
             r = c->legacy_conv ? run_wgrad(c, c->wgrad[l], agent0, groups, ws)
                 : l > 0        ? run_conv_wgrad(c, c->cwgrad[l], agent0, groups, ws)
@@ -827,10 +836,11 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
                 jobs.j[1 + k] = {c->dy[l] + (long)agent0 * S * P[l] * kConvCout[l], S * P[l] * kConvCout[l], S * P[l],
                                  kConvCout[l], c->cl.b[l]};
             }
-            if ((r = fork()) != GALA_OK) return r;
-            LAUNCH(T_COLSUM, ws, launch_colsum(jobs, c->legacy_conv ? 4 : 2, c->g + (long)agent0 * dp, dp,
+            cudaStream_t cs = tail_on_chain ? st : ws;
+            if (!tail_on_chain && (r = fork()) != GALA_OK) return r;
+            LAUNCH(T_COLSUM, cs, launch_colsum(jobs, c->legacy_conv ? 4 : 2, c->g + (long)agent0 * dp, dp,
                                                c->colsum_partial + (long)agent0 * kColsumJobs * kColsumChunks * 512,
-                                               c->colsum_ticket + (long)agent0 * kColsumJobs, groups, ws));
+                                               c->colsum_ticket + (long)agent0 * kColsumJobs, groups, cs));
         }
         if (side) {   // join: the gradient is complete when both streams are done
             CK(cudaEventRecord(c->ev_join, side));
