@@ -1443,9 +1443,14 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
         CK(cudaStreamWaitEvent(st, c->agents[i].fence, 0));
     }
     if (ros) {
+        // Timing several kernel classes of the step at once: one stream, so that an event pair brackets a kernel
+        // and not its wait for the SMs that the other stream's kernels hold.
+        const unsigned long long outside = (1ull << T_SWEEP_SYNC) | (1ull << T_SWEEP_AGENT) | (1ull << T_SAMPLE);
+        const unsigned long long inside = c->profile_mask & ~outside;
+        cudaStream_t side = (inside & (inside - 1)) != 0 ? nullptr : c->side_stream;
         for (int a0 = 0; a0 < n; a0 += kBatch) {
             const int cnt = n - a0 < kBatch ? n - a0 : kBatch;
-            int r = learn_range_cached(c, a0, cnt, ros + a0, st, c->side_stream);
+            int r = learn_range_cached(c, a0, cnt, ros + a0, st, side);
             if (r != GALA_OK) return r;
         }
     }

@@ -68,13 +68,22 @@ __global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, float* __r
     const int cc = threadIdx.x % cchunks, rl = threadIdx.x / cchunks;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (rl < lanes) {
-        for (long r = lo + rl; r < hi; r += lanes) {
-            const uint4 v = __ldg(src + r * cchunks + cc);
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+        // four rows a step, so that four 16-byte loads are in flight per thread; the sums keep the row order
+        for (long r = lo + rl; r < hi; r += 4L * lanes) {
+            uint4 v[4];
 #pragma unroll
-            for (int q = 0; q < 4; q++) {
-                const float2 f = __bfloat1622float2(h[q]);
-                acc[2 * q] += f.x; acc[2 * q + 1] += f.y;
+            for (int u = 0; u < 4; u++) {
+                const long ru = r + (long)u * lanes;
+                v[u] = ru < hi ? __ldg(src + ru * cchunks + cc) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; u++) {
+                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v[u]);
+#pragma unroll
+                for (int q = 0; q < 4; q++) {
+                    const float2 f = __bfloat1622float2(h[q]);
+                    acc[2 * q] += f.x; acc[2 * q + 1] += f.y;
+                }
             }
         }
     }
