@@ -125,6 +125,8 @@ struct gala_ctx {
     float *clip = nullptr, *norm = nullptr, *losses = nullptr;
     double *norm_partial = nullptr, *colsum_partial = nullptr;
     unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr, *heads_ticket = nullptr;
+    float* c1b = nullptr;                    // bias-gradient slices of conv1, left by conv2's data gradient
+    long c1b_min_samples = 2048;             // ... in launches over at least this many samples
     float* fc_sq = nullptr;                  // [N][1600] sums of squares of the hidden layer's weight gradient, by 32 x 32 block
     float* dzv = nullptr;                    // [N][S][20] rows (dlogits, dvalue, zeros) of the fused heads kernel
     float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
@@ -469,6 +471,7 @@ int build_plans(gala_ctx* c) {
             d.args.gate_in = c->gate[l - 1]; d.args.gate_group_stride = B * in_elems / 32;
             d.args.out = c->dy[l - 1]; d.args.out_group_stride = S * in_elems;
             d.args.error_word = c->error_word;
+            if (l == 1) d.args.bias_partial = c->c1b;   // per-channel sums of dY1 = conv1's bias gradient
             ok &= make_conv_maps(d.args.variant, &d.x, &d.w, c->dy[l], (uint64_t)n * S, c->shadow + c->cl.w[l], n, dp);
             d.built = true;
         }
@@ -570,6 +573,10 @@ int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, c
     a.out += (long)agent0 * a.out_group_stride;
     if (a.gate_out) a.gate_out += (long)agent0 * a.gate_group_stride;
     if (a.gate_in) a.gate_in += (long)agent0 * a.gate_group_stride;
+    if (a.bias_partial) {
+        if ((long)groups * rows < c->c1b_min_samples) a.bias_partial = nullptr;
+        else a.bias_partial += (long)agent0 * kConvBiasSliceStride;
+    }
     LAUNCH(p.tag, st, launch_conv(p.x, p.w, a, st));
     return GALA_OK;
 }
@@ -825,8 +832,8 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         }
         if ((r = flush_pending_reduces(c, agent0, groups, ws)) != GALA_OK) return r;
         // Bias gradients = column sums.  conv2's and conv3's come out of their weight-gradient kernels (summed from
-        // the dY tiles while those are in shared memory); the hidden layer's and conv1's, and in the legacy mode all
-        // four, here.
+        // the dY tiles while those are in shared memory), conv1's out of conv2's data gradient as slices per CTA
+        // and warp that are added here; the hidden layer's, and in the legacy mode all four, are summed here.
         {
             ColsumJobs jobs{};
             jobs.j[0] = {c->dh + (long)agent0 * S * kHidden, S * kHidden, S, kHidden, c->cl.fcb};
@@ -838,9 +845,15 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
             }
             cudaStream_t cs = tail_on_chain ? st : ws;
             if (!tail_on_chain && (r = fork()) != GALA_OK) return r;
-            LAUNCH(T_COLSUM, cs, launch_colsum(jobs, c->legacy_conv ? 4 : 2, c->g + (long)agent0 * dp, dp,
+            ColsumSlices sl{c->c1b + (long)agent0 * kConvBiasSliceStride, c->cl.b[0],
+                            conv_grid((long)groups * S, c->cur_ctas), (int)S};
+            // few samples: the slices' extra work in the epilogue is exposed and the column sums cost a launch's
+            // latency either way, so conv1's bias gradient is summed from dY1 like the hidden layer's
+            const bool slices = !c->legacy_conv && (long)groups * S >= c->c1b_min_samples;
+            LAUNCH(T_COLSUM, cs, launch_colsum(jobs, c->legacy_conv ? 4 : slices ? 1 : 2, c->g + (long)agent0 * dp, dp,
                                                c->colsum_partial + (long)agent0 * kColsumJobs * kColsumChunks * 512,
-                                               c->colsum_ticket + (long)agent0 * kColsumJobs, groups, cs));
+                                               c->colsum_ticket + (long)agent0 * kColsumJobs, groups, cs,
+                                               slices ? &sl : nullptr));
         }
         if (side) {   // join: the gradient is complete when both streams are done
             CK(cudaEventRecord(c->ev_join, side));
@@ -1171,6 +1184,8 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
         ALLOC(c->dzv, (size_t)n * S * 20);
         ALLOC(c->fc_sq, (size_t)n * (kHidden / 128) * ((kFeat + 127) / 128) * 16);
+        ALLOC(c->c1b, (size_t)n * kConvBiasSliceStride);
+        if (const char* e = getenv("GALA_C1B_SLICES")) c->c1b_min_samples = atoi(e) ? 0 : (1L << 60);
         ALLOC(c->shadow, (size_t)n * dp);
         ALLOC(c->colsum_partial, (size_t)n * kColsumJobs * kColsumChunks * 512); ALLOC(c->colsum_ticket, (size_t)n * kColsumJobs);
         for (int l = 0; l < 3; l++) {

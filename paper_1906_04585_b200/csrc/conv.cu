@@ -117,7 +117,24 @@ template <int V> __device__ __forceinline__ UnitCoord decode_unit(int u, int row
     return c;
 }
 
-template <int V>
+// Lane j leaves with the sum over the warp's lanes of their v[j] (v is used up): five exchange steps, each
+// halving the values a lane still holds; the order of the additions is fixed.
+__device__ __forceinline__ float warp_reduce_scatter32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const bool hi = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; i++) {
+            const float send = hi ? v[i] : v[i + s];
+            const float keep = hi ? v[i + s] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+    }
+    return v[0];
+}
+
+// BIAS (conv2 data gradient only): also leave the per-channel sums of the result behind, see ConvArgs::bias_partial.
+template <int V, bool BIAS = false>
 __global__ void __launch_bounds__(V == CV_CONV1_FWD ? kConv1Threads : kConvThreads, 1)
 conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const ConvArgs p,
                      const int nst, const long total_units) {
@@ -379,6 +396,26 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         load_gates(u_begin + eg, gate);
         int cur_g = -1;
         int it = eg;
+        // conv2 data gradient: the sum over pixels of what is stored (= the bias gradient of conv1) is kept per
+        // thread while the CTA stays with an agent and leaves as one slice per agent, CTA and epilogue warp.  A
+        // warp writes a slice for EVERY agent in the CTA's range of units, also where its group had no unit.
+        static_assert(!BIAS || V == CV_CONV2_DGRAD, "bias slices come from conv2's data gradient only");
+        constexpr bool kBias = BIAS;
+        float bacc[kBias ? 32 : 1];
+#pragma unroll
+        for (int j = 0; j < (kBias ? 32 : 1); j++) bacc[j] = 0.0f;
+        const bool bias_on = kBias && u_begin < u_end;
+        int bg = bias_on ? decode_unit<V>(u_begin, p.rows).gz : 0;     // agent that bacc belongs to
+        auto bias_flush = [&](int upto) {      // slices of agents bg .. upto - 1; bacc restarts at zero
+            if constexpr (kBias) {
+                for (; bg < upto; bg++) {
+                    const float sum = warp_reduce_scatter32(bacc, lane);
+                    p.bias_partial[(((long)bg * kConvMaxGrid + blockIdx.x) * 8 + (warp - 2)) * 32 + lane] = sum;
+#pragma unroll
+                    for (int j = 0; j < 32; j++) bacc[j] = 0.0f;
+                }
+            }
+        };
         for (int u = u_begin + eg; u < u_end; u += 2, it += 2) {
             const UnitCoord c = decode_unit<V>(u, p.rows);
             const long off = pixel_off(c);
@@ -395,6 +432,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 else return c0;
             };
             uint32_t gate_next[kFwd ? 1 : NCH];
+            if (bias_on && c.gz != bg) bias_flush(c.gz);
             if constexpr (kFwd) {
                 if (c.gz != cur_g) {
                     const float* bias = p.bias + (long)(p.group0 + c.gz) * p.bias_group_stride;
@@ -429,6 +467,9 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                             if (!((gate[ch] >> (2 * j + 1)) & 1u)) v1 = 0.0f;
                         }
                         o[j] = pack2(v0, v1);
+                        if constexpr (kBias) {
+                            if (valid) { bacc[2 * j] += v0; bacc[2 * j + 1] += v1; }
+                        }
                         if constexpr (kFwd) {   // gate of the stored (rounded) activation
                             if (o[j] & 0x00007fffu) bits |= 1u << (2 * j);
                             if (o[j] & 0x7fff0000u) bits |= 1u << (2 * j + 1);
@@ -451,6 +492,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             tcgen05_fence_before();
             if (lane == 0) mbar_arrive(&acc_empty[ab]);
         }
+        if (bias_on) bias_flush(decode_unit<V>(u_end - 1, p.rows).gz + 1);
     }
 
     // teardown
@@ -497,6 +539,8 @@ cudaError_t conv_init() {
     if ((e = conv_attr<CV_CONV3_FWD>()) != cudaSuccess) return e;
     if ((e = conv_attr<CV_CONV2_DGRAD>()) != cudaSuccess) return e;
     if ((e = conv_attr<CV_CONV3_DGRAD>()) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_resident_kernel<CV_CONV2_DGRAD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kConvSmemMax)) != cudaSuccess) return e;
     done = true;
     return cudaSuccess;
 }
@@ -552,6 +596,12 @@ bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const v
     return ok;
 }
 
+int conv_grid(long units, int max_ctas) {
+    int grid = (int)(units < kConvMaxGrid ? units : kConvMaxGrid);
+    if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;
+    return grid;
+}
+
 template <int V>
 static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, const ConvArgs& a, cudaStream_t st) {
     using T = ConvTraits<V>;
@@ -565,9 +615,15 @@ static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, con
     if (units <= 0) return cudaSuccess;
     if (units > 0x7fffffffL) return cudaErrorInvalidValue;
     const size_t smem = (size_t)fixed + (size_t)nst * STAGE;
-    int grid = (int)(units < 148 ? units : 148);
-    if (a.max_ctas > 0 && grid > a.max_ctas) grid = a.max_ctas;
-    (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), dim3(V == CV_CONV1_FWD ? kConv1Threads : kConvThreads), smem, st, x, w, a, nst, units);
+    const int grid = conv_grid(units, a.max_ctas);
+    const dim3 block(V == CV_CONV1_FWD ? kConv1Threads : kConvThreads);
+    if constexpr (V == CV_CONV2_DGRAD) {
+        if (a.bias_partial) {
+            (void)launch_pdl(conv_resident_kernel<V, true>, dim3(grid), block, smem, st, x, w, a, nst, units);
+            return cudaGetLastError();
+        }
+    }
+    (void)launch_pdl(conv_resident_kernel<V>, dim3(grid), block, smem, st, x, w, a, nst, units);
     return cudaGetLastError();
 }
 

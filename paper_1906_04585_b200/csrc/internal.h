@@ -187,7 +187,15 @@ struct ConvArgs {
     int* error_word;
     int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
     PtrBatch obs;          // conv1 forward: the agents' uint8 frames [rows][84][84][4], 16-byte aligned
+    // conv2 data gradient (may be null): per-channel sums over the pixels of the result, as slices
+    // [agent of the launch][kConvMaxGrid CTAs][8 warps][32 channels].  CTA b (of `grid`) works on samples
+    // [total * b / grid, total * (b + 1) / grid) of the launch's groups * rows and writes the slices of every agent
+    // that range touches; the other slices are left alone and must not be read.
+    float* bias_partial;
 };
+constexpr int kConvMaxGrid = 148;
+constexpr long kConvBiasSliceStride = (long)kConvMaxGrid * 8 * 32;   // floats per agent
+int conv_grid(long units, int max_ctas);   // CTAs of a launch over `units` work units
 cudaError_t conv_init();
 bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const void* x_base, uint64_t samples,
                     const void* w_base, uint64_t groups, uint64_t w_group_stride_elems);
@@ -404,8 +412,12 @@ cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out
 constexpr int kColsumJobs = 4;
 struct ColsumJob { const __nv_bfloat16* dy; long group_stride; long rows; int C; long out_off; };
 struct ColsumJobs { ColsumJob j[kColsumJobs]; };
+// slices: when slices.partial is set, one more block per agent adds the bias slices that a conv2 data-gradient
+// launch of `grid` CTAs over groups * rows samples left behind (ConvArgs::bias_partial), in CTA and warp order,
+// into out_base[g*out_group_stride + out_off + 0..31].
+struct ColsumSlices { const float* partial; long out_off; int grid, rows; };
 cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, long out_group_stride, double* partial,
-                          unsigned* ticket, int groups, cudaStream_t st);
+                          unsigned* ticket, int groups, cudaStream_t st, const ColsumSlices* slices = nullptr);
 constexpr int kColsumChunks = 64;
 
 }  // namespace gala

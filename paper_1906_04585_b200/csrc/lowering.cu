@@ -45,11 +45,43 @@ cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out
 // block that finishes last adds the chunk sums in index order, so the result does not depend on
 // scheduling.  C is a power of two, 8 <= C <= 512.
 // Up to kColsumJobs tensors are reduced by one launch (blockIdx.z picks the tensor).
-__global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, float* __restrict__ out_base, long out_group_stride,
+__global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, int n_jobs, ColsumSlices sl,
+                                                     float* __restrict__ out_base, long out_group_stride,
                                                      double* partial_base, unsigned* ticket_base) {
     pdl_wait();
     pdl_launch();
     const int g = blockIdx.y;
+    __shared__ float red[256 * 8];
+    if ((int)blockIdx.z == n_jobs) {
+        // Bias slices of a conv2 data-gradient launch: CTA b of sl.grid worked on samples
+        // [total * b / grid, total * (b + 1) / grid); those whose range meets agent g's samples left 8 warp slices
+        // of 32 channels each.  Thread (w, c) adds slice w of the CTAs in order, then the 8 sums are added in order.
+        if (blockIdx.x != 0) return;
+        const long total = (long)gridDim.y * sl.rows, lo = (long)g * sl.rows, hi = lo + sl.rows;
+        int b_lo = (int)(lo * sl.grid / total);
+        while (b_lo > 0 && total * b_lo / sl.grid > lo) b_lo--;
+        while (total * (b_lo + 1) / sl.grid <= lo) b_lo++;
+        int b_hi = b_lo;                                   // last CTA whose range starts below hi
+        while (b_hi + 1 < sl.grid && total * (b_hi + 1) / sl.grid < hi) b_hi++;
+        const int w = threadIdx.x >> 5, c = threadIdx.x & 31;
+        const float* src = sl.partial + ((long)g * kConvMaxGrid * 8 + w) * 32 + c;
+        float s = 0.0f;
+        for (int b = b_lo; b <= b_hi; b += 4) {
+            float v[4];
+#pragma unroll
+            for (int u = 0; u < 4; u++) v[u] = b + u <= b_hi ? __ldcg(src + (long)(b + u) * 8 * 32) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < 4; u++) s += v[u];
+        }
+        red[threadIdx.x] = s;
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            float t = 0.0f;
+            for (int k = 0; k < 8; k++) t += red[k * 32 + threadIdx.x];
+            out_base[(long)g * out_group_stride + sl.out_off + threadIdx.x] = t;
+        }
+        return;
+    }
     const ColsumJob job = jobs.j[blockIdx.z];
     const long rows = job.rows;
     const int C = job.C;
@@ -60,7 +92,6 @@ __global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, float* __r
     const long per = (rows + kColsumChunks - 1) / kColsumChunks;
     const long lo = (long)blockIdx.x * per;
     long hi = lo + per; if (hi > rows) hi = rows;
-    __shared__ float red[256 * 8];
     __shared__ bool last;
     double* part = partial + (long)g * kColsumJobs * kColsumChunks * 512 + (long)blockIdx.x * C;
     const int cchunks = C / 8;                    // 16-byte column groups per row
@@ -115,13 +146,19 @@ __global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, float* __r
     }
 }
 cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, long out_group_stride, double* partial,
-                          unsigned* ticket, int groups, cudaStream_t st) {
+                          unsigned* ticket, int groups, cudaStream_t st, const ColsumSlices* slices) {
     if (n_jobs < 1 || n_jobs > kColsumJobs) return cudaErrorInvalidValue;
+    ColsumSlices sl{};
+    if (slices) {
+        sl = *slices;
+        if (!sl.partial || sl.rows < 1 || sl.grid != conv_grid((long)groups * sl.rows, sl.grid)) return cudaErrorInvalidValue;
+    }
     for (int i = 0; i < n_jobs; i++) {
         const int C = jobs.j[i].C;
         if (C > 512 || C < 8 || (C & (C - 1))) return cudaErrorInvalidValue;
     }
-    (void)launch_pdl(colsum_kernel, dim3(dim3(kColsumChunks, groups, n_jobs)), dim3(256), 0, st, jobs, out_base, out_group_stride, partial, ticket);
+    (void)launch_pdl(colsum_kernel, dim3(kColsumChunks, groups, n_jobs + (slices ? 1 : 0)), dim3(256), 0, st, jobs, n_jobs, sl,
+                     out_base, out_group_stride, partial, ticket);
     return cudaGetLastError();
 }
 

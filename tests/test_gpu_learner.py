@@ -340,6 +340,41 @@ def test_conv_sync_round_unfused_heads(monkeypatch):
     _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
 
 
+def test_conv_bias_slices_many_small_agents(monkeypatch):
+    # conv1's bias gradient as per-CTA, per-warp slices out of conv2's data gradient is the path of large batches
+    # (the full-size rounds check it against the oracle).  Here it is forced on for a case of many tiny agents -
+    # 40 agents x 4 samples = 160 work units on 148 CTAs, so CTAs cross agent borders and epilogue warps leave
+    # empty slices for agents their group had no unit of - and compared with the column-sum path, which the
+    # small rounds above check against the oracle: the same sums of fp32 values instead of their bf16 roundings,
+    # everything else bit for bit.
+    B_, LM = _mods()
+    w = GI.WORKLOADS[1].scaled(n_agents=40, n_envs=2, n_steps=2, topo_peers=1)
+    net = oracle_net(w)
+    off = R.param_offsets(net)
+    bounds = sorted(off.values())
+    lo = off["L0.b"]
+    hi = bounds[bounds.index(lo) + 1]
+    ros = [GI.rollout(w, i, 0) for i in range(w.n_agents)]
+    grads = {}
+    for flag in ("0", "1"):
+        monkeypatch.setenv("GALA_C1B_SLICES", flag)
+        L = make_learner(w)
+        seed_identical(L, w, net)
+        L.step_sync([LM.DeviceRollout(r) for r in ros])
+        L.sync()
+        grads[flag] = [L.get_grad(i).copy() for i in range(w.n_agents)]
+        L.close()
+    for i in range(w.n_agents):
+        a, b = grads["0"][i], grads["1"][i]
+        np.testing.assert_array_equal(a[:lo], b[:lo])
+        np.testing.assert_array_equal(a[hi:], b[hi:])
+        assert np.abs(b[lo:hi]).max() > 0
+        err = np.linalg.norm(a[lo:hi].astype(np.float64) - b[lo:hi]) / np.linalg.norm(a[lo:hi].astype(np.float64))
+        # the summands differ by their bf16 rounding (2^-9 relative each) and partly cancel in the sum; a lost or
+        # doubled slice would be an error of 1/16 of the sum or more
+        assert err <= TOL_BF16, (i, err)
+
+
 def test_conv_sync_round_legacy_products(monkeypatch):
     # the previous generation of the convolution products (one TMA box per kernel offset, bf16 frame copies)
     # is kept as an independent cross-check of the resident-input kernels
