@@ -232,7 +232,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (!go) break;
                 if (lane == 0) {
                     const int left = 21 * p.rows - kC1Lines * c.s;   // groups from this unit's first to the last
-                    const uint32_t bytes = (uint32_t)((left < kC1Lines + 1 ? left : kC1Lines + 1) * kC1Group);
+                    const uint32_t bytes = left < kC1Lines + 1 ? (uint32_t)(left * kC1Group) : (uint32_t)kU8Bytes;
                     mbar_expect_tx(&u8_full[su], bytes);
                     const uint8_t* src = reinterpret_cast<const uint8_t*>(p.obs.p[c.gz]) + (long)c.s * (kC1Lines * kC1Group);
                     bulk_load_1d(smU + su * kU8Stride, src, bytes, &u8_full[su]);
@@ -449,39 +449,45 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             tcgen05_fence_after();
             if (q * 32 <= kLastRow) {
                 const uint32_t tmem_acc = tmem_base + (uint32_t)ab * T::BN + ((uint32_t)(q * 32) << 16);
+                // 16 columns (one 32-byte store) at a time, the load of the next 16 in flight meanwhile
+                constexpr int NSUB = 2 * NCH;
+                uint32_t rr[2][16];
+                tmem_ld16_issue(tmem_acc, rr[0]);
+                uint32_t bits = 0u;
 #pragma unroll
-                for (int ch = 0; ch < NCH; ch++) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_acc + (uint32_t)(ch * 32), r);
-                    uint32_t o[16];
-                    uint32_t bits = 0u;
+                for (int sb = 0; sb < NSUB; sb++) {
+                    const int ch = sb >> 1, h = sb & 1;        // 32-column block, half of it
+                    uint32_t (&r)[16] = rr[sb & 1];
+                    tmem_ld16_wait(r);
+                    if (sb + 1 < NSUB) tmem_ld16_issue(tmem_acc + (uint32_t)((sb + 1) * 16), rr[(sb + 1) & 1]);
+                    uint32_t o[8];
 #pragma unroll
-                    for (int j = 0; j < 16; j++) {
+                    for (int j = 0; j < 8; j++) {
                         float v0 = __uint_as_float(r[2 * j]), v1 = __uint_as_float(r[2 * j + 1]);
                         if constexpr (kFwd) {
-                            const float2 bv = *reinterpret_cast<const float2*>(sbias + ch * 32 + 2 * j);
+                            const float2 bv = *reinterpret_cast<const float2*>(sbias + sb * 16 + 2 * j);
                             v0 = fmaxf(fmaf(v0, p.scale, bv.x), 0.0f);
                             v1 = fmaxf(fmaf(v1, p.scale, bv.y), 0.0f);
                         } else {
-                            if (!((gate[ch] >> (2 * j)) & 1u)) v0 = 0.0f;
-                            if (!((gate[ch] >> (2 * j + 1)) & 1u)) v1 = 0.0f;
+                            if (!((gate[ch] >> (16 * h + 2 * j)) & 1u)) v0 = 0.0f;
+                            if (!((gate[ch] >> (16 * h + 2 * j + 1)) & 1u)) v1 = 0.0f;
                         }
                         o[j] = pack2(v0, v1);
                         if constexpr (kBias) {
-                            if (valid) { bacc[2 * j] += v0; bacc[2 * j + 1] += v1; }
+                            if (valid) { bacc[16 * h + 2 * j] += v0; bacc[16 * h + 2 * j + 1] += v1; }
                         }
                         if constexpr (kFwd) {   // gate of the stored (rounded) activation
-                            if (o[j] & 0x00007fffu) bits |= 1u << (2 * j);
-                            if (o[j] & 0x7fff0000u) bits |= 1u << (2 * j + 1);
+                            if (o[j] & 0x00007fffu) bits |= 1u << (16 * h + 2 * j);
+                            if (o[j] & 0x7fff0000u) bits |= 1u << (16 * h + 2 * j + 1);
                         }
                     }
-                    if (valid) {   // two 32-byte stores: every store fills whole sectors
-                        st_global_v8(out + block_add(ch * 32), &o[0]);
-                        st_global_v8(out + block_add(ch * 32) + 16, &o[8]);
+                    if (valid) {   // a 32-byte store fills a whole sector
+                        st_global_v8(out + block_add(ch * 32) + 16 * h, o);
                         if constexpr (kFwd) {
-                            if (p.gate_out) p.gate_out[(long)c.gz * p.gate_group_stride + off / 32 + ch] = bits;
+                            if (h == 1 && p.gate_out) p.gate_out[(long)c.gz * p.gate_group_stride + off / 32 + ch] = bits;
                         }
                     }
+                    if (h == 1) bits = 0u;
                 }
             }
             if constexpr (!kFwd) {
