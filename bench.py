@@ -89,7 +89,10 @@ def round_work(w: GI.Workload, d_pad: int):
     for a in act:
         by += B * a * 2 + B * a * 2 + S * a * 2            # activation written, read forward, read by a weight gradient
         by += B * a / 8 + S * a / 8                        # ReLU gate bits written and read
-        by += S * a * 2 * (4 if a != act[0] else 3)        # dY written; read by data gradient (not conv1), weight gradient, bias sums
+        # dY: written, read by the weight gradient (which also sums conv2's / conv3's bias gradient) and, except
+        # for conv1, by the data gradient; dY1 is read once more by the column sums only in small launches
+        # (larger ones take conv1's bias gradient out of conv2's data gradient)
+        by += S * a * 2 * (3 if a != act[0] else (3 if n * S < 2048 else 2))
     by += B * 512 * 2 * 2 + S * 512 * 2                    # hidden activations: written, read by heads, read by head gradients
     by += S * 512 * 2 * 4                                  # dh: written, read by FC data / weight gradient and bias sums
     by += 2 * (d_pad * 2) + d_pad * 4 + d_pad * 4          # bf16 weights forward + backward, gradient written, read by the norm

@@ -107,7 +107,7 @@ struct gala_ctx {
     std::vector<Agent> agents;
     cudaStream_t main_stream = nullptr;
     cudaEvent_t main_event = nullptr;
-    // second stream of the synchronous mode: weight gradients and bias gradients run beside the chain
+    // second stream of the synchronous mode: the weight gradients of heads, hidden layer, conv3 and conv2 run beside the chain
     // of data gradients they do not depend on
     cudaStream_t side_stream = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
