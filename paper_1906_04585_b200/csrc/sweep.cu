@@ -209,7 +209,8 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
     // The elements to read, [0, d_pad) without the range whose sum of squares is already known, are numbered
     // consecutively and cut into chunks of multiples of 4 floats (the padding [d, d_pad) is zero): 16-byte loads
     const long total = d_pad - kn.count;
-    const long per = ((total / 4 + kNormChunks - 1) / kNormChunks) * 4;
+    const int chunks = gridDim.x;          // <= kNormChunks: fewer when there is little to read
+    const long per = ((total / 4 + chunks - 1) / chunks) * 4;
     const long lo = (long)blockIdx.x * per;
     long hi = lo + per; if (hi > total) hi = total;
     float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
@@ -220,7 +221,7 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
     double acc = ((double)a0 + (double)a1) + ((double)a2 + (double)a3);
     if (kn.partial) {   // the known range: its partial sums, shared out over the agent's threads in slot order
         const float* kp = kn.partial + (long)blockIdx.y * kn.partial_group_stride;
-        for (long k = (long)blockIdx.x * blockDim.x + threadIdx.x; k < kn.n_partials; k += (long)kNormChunks * blockDim.x)
+        for (long k = (long)blockIdx.x * blockDim.x + threadIdx.x; k < kn.n_partials; k += (long)chunks * blockDim.x)
             acc += (double)kp[k];
     }
     __shared__ double red[256];
@@ -235,13 +236,13 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
         partial[(long)agent * kNormChunks + blockIdx.x] = red[0];
         __threadfence();
         unsigned t = atomicAdd(&ticket[agent], 1u);
-        last = (t == kNormChunks - 1);
+        last = (t == (unsigned)chunks - 1);
     }
     __syncthreads();
     if (last && threadIdx.x == 0) {
         __threadfence();
         double s = 0.0;
-        for (int k = 0; k < kNormChunks; k++) s += ((volatile double*)partial)[(long)agent * kNormChunks + k];
+        for (int k = 0; k < chunks; k++) s += ((volatile double*)partial)[(long)agent * kNormChunks + k];
         float nrm = (float)sqrt(s);
         norm[agent] = nrm;
         float c = 1.0f;
@@ -258,7 +259,12 @@ cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int
     if (known) kn = *known;
     if (!kn.partial) { kn.off = 0; kn.count = 0; kn.n_partials = 0; }
     if ((kn.off | kn.count) & 3 || kn.off + kn.count > d_pad) return cudaErrorInvalidValue;
-    dim3 grid(kNormChunks, n_agents);
+    // a chunk is at least 8192 floats (32 bytes per thread of a block, twice): with most of the gradient known
+    // from partial sums a dozen blocks per agent remain, and the last block's sum over chunks is as short
+    long chunks = (d_pad - kn.count + 8191) / 8192;
+    if (chunks < 1) chunks = 1;
+    if (chunks > kNormChunks) chunks = kNormChunks;
+    dim3 grid((unsigned)chunks, n_agents);
     (void)launch_pdl(grad_norm_kernel, dim3(grid), dim3(256), 0, st, g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip, kn);
     return cudaGetLastError();
 }
