@@ -176,6 +176,14 @@ int gala_set_grad(gala_ctx* ctx, int agent, const float* grad, float clip_coef);
 /* Distance of the agents' parameters from their mean, ||X - mean||_F over all agents and
  * parameters (left-hand side of Propositions 1 and 2).  Waits for all work first. */
 int gala_consensus_distance(gala_ctx* ctx, double* out);
+/* Update norms for the bound of Proposition 1, ||X - mean||_F <= alpha * sum_s beta^(k+1-s) ||G(s)||.
+ * gala_track_updates(ctx, 1): every later gala_step_sync also computes, before its optimiser pass and from the same
+ * gradient, clip factor and second-moment estimate, the Frobenius norm over all agents of the step it takes
+ * (row i = lr * c g / (sqrt(v') + eps), i.e. alpha G of that round); one more kernel that reads g and v once,
+ * off by default.  gala_update_norm waits for the main stream and returns the value of the last such round;
+ * GALA_EINVAL when there has been none. */
+int gala_track_updates(gala_ctx* ctx, int on);
+int gala_update_norm(gala_ctx* ctx, double* out);
 /* Longest host wait (ms, default 1000) of a gossip step that is blocked by the staleness bound.
  * When it runs out, or when an in-peer has published nothing newer, gala_gossip returns
  * GALA_ETIMEOUT and has enqueued nothing; the pending gradient stays pending. */

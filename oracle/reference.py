@@ -440,6 +440,24 @@ def consensus_distance(X) -> float:
     return float(np.linalg.norm(X - X.mean(axis=0, keepdims=True)))
 
 
+def prop1_bound(update_norms: Sequence[float], betas) -> np.ndarray:
+    """Right-hand side of Proposition 1 after rounds 0..K-1, for identical initial parameters:
+        bound[k] = sum_{s=0..k} (prod_{r=s..k} beta_r) * ||alpha G(s)||_F ,
+    update_norms[s] = ||alpha G(s)||_F (the step of round s, X - Y of that round), betas a scalar (the
+    proposition's constant beta: bound[k] = alpha sum_s beta^(k+1-s) ||G(s)||) or one contraction factor per round
+    (the second largest singular value of that round's doubly stochastic mixing matrix, which is what the proof's
+    per-round inequality uses).  Written as the double sum of the statement, not as a recursion."""
+    u = _f64(update_norms).ravel()
+    K = u.size
+    be = np.full(K, float(betas)) if np.ndim(betas) == 0 else _f64(betas).ravel()
+    assert be.size == K
+    out = np.zeros(K)
+    for k in range(K):
+        for s0 in range(k + 1):
+            out[k] += np.prod(be[s0:k + 1]) * u[s0]
+    return out
+
+
 # --------------------------------------------------------------------------
 # acting
 # --------------------------------------------------------------------------

@@ -56,7 +56,7 @@ EXPORTS = (
     "gala_get_snapshot", "gala_set_stream", "gala_debug_read", "gala_launch_count",
     "gala_last_error", "gala_gemm_bf16", "gala_sweep_sync", "gala_kernel_classes",
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
-    "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_set_stale_timeout",
+    "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_track_updates", "gala_update_norm", "gala_set_stale_timeout",
     "gala_set_agent_ctas", "gala_set_graphs", "gala_losses_all",
     "gala_actor_loop", "gala_actor_read",
 )
@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
             "gala_gossip": (i, [vp, i]),
             "gala_delay": (i, [vp, i, i]),
             "gala_consensus_distance": (i, [vp, C.POINTER(C.c_double)]),
+            "gala_track_updates": (i, [vp, i]),
+            "gala_update_norm": (i, [vp, C.POINTER(C.c_double)]),
             "gala_set_stale_timeout": (i, [vp, i]),
             "gala_set_agent_ctas": (i, [vp, i]),
             "gala_set_graphs": (i, [vp, i]),
@@ -180,6 +182,16 @@ def gala_delay(ctx, agent: int, usec: int):
 def gala_consensus_distance(ctx) -> float:
     out = C.c_double()
     _check(ctx, lib().gala_consensus_distance(ctx, C.byref(out)))
+    return out.value
+
+
+def gala_track_updates(ctx, on: bool):
+    _check(ctx, lib().gala_track_updates(ctx, 1 if on else 0))
+
+
+def gala_update_norm(ctx) -> float:
+    out = C.c_double()
+    _check(ctx, lib().gala_update_norm(ctx, C.byref(out)))
     return out.value
 
 

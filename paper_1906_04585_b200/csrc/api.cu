@@ -144,6 +144,11 @@ struct gala_ctx {
     int* error_word = nullptr;
     double *cons_partial = nullptr, *cons_out = nullptr;
     unsigned* cons_ticket = nullptr;
+    // update-norm tracking (Proposition 1): ||alpha G||_F^2 of the last synchronous round
+    bool track_updates = false;
+    bool upd_valid = false;
+    double *upd_partial = nullptr, *upd_out = nullptr;
+    unsigned* upd_ticket = nullptr;
     int stale_timeout_ms = 1000;   // longest host wait of a staleness-bounded gossip step
     float *logits = nullptr, *values = nullptr, *returns = nullptr, *adv = nullptr, *dlogits = nullptr,
           *dvalues = nullptr;
@@ -1070,12 +1075,21 @@ int host_wait(gala_ctx* c, cudaStream_t st, int timeout_ms) {
     }
 }
 
+// Copy into device memory that is complete when the call returns.  A plain cudaMemcpy from pageable host memory may
+// return while its last piece is still on the way, and the library's streams are non-blocking, i.e. not ordered
+// behind the default stream that copy runs on: a kernel launched right after it could read the old contents.
+int copy_in(gala_ctx* c, void* dst, const void* src, size_t bytes, cudaStream_t st) {
+    CK(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, st));
+    CK(cudaStreamSynchronize(st));
+    return GALA_OK;
+}
+
 int check_error_word(gala_ctx* c) {
     int w = 0;
     CK(cudaMemcpy(&w, c->error_word, sizeof w, cudaMemcpyDeviceToHost));
     if (w) {
         int z = 0;
-        cudaMemcpy(c->error_word, &z, sizeof z, cudaMemcpyHostToDevice);
+        (void)copy_in(c, c->error_word, &z, sizeof z, c->main_stream);
         return fail(c, GALA_ECUDA, "a bounded device-side wait ran out (tensor-core pipeline)");
     }
     return GALA_OK;
@@ -1165,12 +1179,14 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
     ALLOC(c->norm_partial, (size_t)n * kNormChunks); ALLOC(c->norm_ticket, n);
     ALLOC(c->error_word, 1);
     ALLOC(c->cons_partial, 592); ALLOC(c->cons_out, 1); ALLOC(c->cons_ticket, 1);
+    ALLOC(c->upd_partial, (size_t)n * kUpdateNormChunks); ALLOC(c->upd_out, 1); ALLOC(c->upd_ticket, 1);
     ALLOC(c->logits, (size_t)n * B * A); ALLOC(c->values, (size_t)n * B);
     ALLOC(c->returns, (size_t)n * S); ALLOC(c->adv, (size_t)n * S);
     ALLOC(c->dlogits, (size_t)n * S * A); ALLOC(c->dvalues, (size_t)n * S);
     {   // clip coefficients start at 1
         std::vector<float> ones(n, 1.0f);
-        CK(cudaMemcpy(c->clip, ones.data(), n * sizeof(float), cudaMemcpyHostToDevice));
+        int r = copy_in(c, c->clip, ones.data(), n * sizeof(float), c->main_stream);
+        if (r != GALA_OK) return r;
     }
     if (c->conv) {
         const int P[3] = {400, 81, 49};
@@ -1243,7 +1259,8 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
                     init_tensor(host.data(), c->ml.vb, 1, H, hp->seed, ag);
                 }
             }
-            CK(cudaMemcpy(c->x + (long)i * dp, host.data(), dp * sizeof(float), cudaMemcpyHostToDevice));
+            int r = copy_in(c, c->x + (long)i * dp, host.data(), dp * sizeof(float), c->main_stream);
+            if (r != GALA_OK) return r;
         }
         if (c->conv) {
             LAUNCH(T_CAST, c->main_stream, launch_cast_bf16(c->x, c->shadow, (long)n * dp, c->main_stream));
@@ -1480,6 +1497,11 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
                                                  c->norm_ticket, c->norm, c->clip, st));
     }
     SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
+    if (c->track_updates) {   // the norm of the step this pass is about to take, from the same g, clip and v
+        LAUNCH(T_GRAD_NORM, st, launch_update_norm(c->g, c->v, c->clip, n, c->d_pad, hp, c->upd_partial, c->upd_ticket,
+                                                   c->upd_out, st));
+        c->upd_valid = true;
+    }
     LAUNCH(T_SWEEP_SYNC, st, launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp,
                                             c->error_word, st));
     CK(cudaEventRecord(c->main_event, st));
@@ -1536,13 +1558,17 @@ int gala_set_state(gala_ctx* c, int agent, const float* params, const float* sq_
     CK(cudaStreamSynchronize(ag.stream));
     const size_t bytes = (size_t)c->d * sizeof(float);
     if (params) {
-        CK(cudaMemcpy(c->x + (long)agent * c->d_pad, params, bytes, cudaMemcpyDefault));
+        int r = copy_in(c, c->x + (long)agent * c->d_pad, params, bytes, ag.stream);
+        if (r != GALA_OK) return r;
         if (c->conv) {
             LAUNCH(T_CAST, ag.stream, launch_cast_bf16(c->x + (long)agent * c->d_pad, c->shadow + (long)agent * c->d_pad, c->d_pad, ag.stream));
             CK(cudaStreamSynchronize(ag.stream));
         }
     }
-    if (sq_avg) CK(cudaMemcpy(c->v + (long)agent * c->d_pad, sq_avg, bytes, cudaMemcpyDefault));
+    if (sq_avg) {
+        int r = copy_in(c, c->v + (long)agent * c->d_pad, sq_avg, bytes, ag.stream);
+        if (r != GALA_OK) return r;
+    }
     ag.round = round;
     if (agent == 0) c->sync_round = round;
     return GALA_OK;
@@ -1553,9 +1579,10 @@ int gala_set_grad(gala_ctx* c, int agent, const float* grad, float clip_coef) {
     Agent& ag = c->agents[agent];
     CK(cudaStreamSynchronize(c->main_stream));
     CK(cudaStreamSynchronize(ag.stream));
-    CK(cudaMemcpy(c->g + (long)agent * c->d_pad, grad, (size_t)c->d * sizeof(float), cudaMemcpyDefault));
+    int r = copy_in(c, c->g + (long)agent * c->d_pad, grad, (size_t)c->d * sizeof(float), ag.stream);
+    if (r != GALA_OK) return r;
     if (clip_coef >= 0.0f) {
-        CK(cudaMemcpy(c->clip + agent, &clip_coef, sizeof(float), cudaMemcpyHostToDevice));
+        if ((r = copy_in(c, c->clip + agent, &clip_coef, sizeof(float), ag.stream)) != GALA_OK) return r;
     } else {
         LAUNCH(T_GRAD_NORM, ag.stream, launch_grad_norm(c->g, c->d, c->d_pad, agent, 1, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
                                 c->norm, c->clip, ag.stream));
@@ -1574,6 +1601,24 @@ int gala_consensus_distance(gala_ctx* c, double* out) {
     CK(cudaStreamSynchronize(c->main_stream));
     double sq = 0.0;
     CK(cudaMemcpy(&sq, c->cons_out, sizeof sq, cudaMemcpyDeviceToHost));
+    *out = std::sqrt(sq);
+    return GALA_OK;
+}
+
+int gala_track_updates(gala_ctx* c, int on) {
+    if (!c) return GALA_EINVAL;
+    c->track_updates = on != 0;
+    if (!on) c->upd_valid = false;
+    return GALA_OK;
+}
+
+int gala_update_norm(gala_ctx* c, double* out) {
+    if (!c || !out) return GALA_EINVAL;
+    if (!c->upd_valid) return fail(c, GALA_EINVAL, "gala_update_norm: no synchronous round since gala_track_updates(ctx, 1)");
+    int r = host_wait(c, c->main_stream, -1);
+    if (r != GALA_OK) return r;
+    double sq = 0.0;
+    CK(cudaMemcpy(&sq, c->upd_out, sizeof sq, cudaMemcpyDeviceToHost));
     *out = std::sqrt(sq);
     return GALA_OK;
 }

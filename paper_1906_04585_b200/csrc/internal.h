@@ -266,6 +266,11 @@ cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int
                              const NormKnown* known = nullptr);
 cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStream_t st);
 // partial: 592 doubles, ticket: one zeroed unsigned, out: one double (squared distance)
+// ||alpha G||_F^2 of the coming optimiser pass (see update_norm_kernel).  partial: [n_agents][kUpdateNormChunks]
+// doubles, ticket: one uint (zero before first use), out: one double.
+constexpr int kUpdateNormChunks = 32;
+cudaError_t launch_update_norm(const float* g, const float* v, const float* clip, int n_agents, long d_pad, SweepHp hp,
+                               double* partial, unsigned* ticket, double* out, cudaStream_t st);
 cudaError_t launch_consensus(const float* x, int n_agents, long d, long d_pad, double* partial, unsigned* ticket,
                              double* out, cudaStream_t st);
 cudaError_t launch_delay(unsigned long long usec, cudaStream_t st);

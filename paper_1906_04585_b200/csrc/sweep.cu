@@ -341,6 +341,74 @@ cudaError_t launch_consensus(const float* x, int n_agents, long d, long d_pad, d
     return cudaGetLastError();
 }
 
+// Frobenius norm of the update matrix alpha * G of a synchronous round, the quantity Proposition 1 sums: row i is
+// what the RMSProp step of the next optimiser pass subtracts from agent i's parameters,
+//     u = lr * c g / (sqrt(a v + (1 - a) (c g)^2) + eps),
+// read from the pending gradient, its clip factor and the second-moment estimate BEFORE that pass.  Block partials
+// in double precision, fixed-order final sum by the last block; writes the squared norm over all agents.
+__global__ void __launch_bounds__(256) update_norm_kernel(const float* __restrict__ g, const float* __restrict__ v,
+                                                          const float* __restrict__ clip, long d_pad, SweepHp hp,
+                                                          double* partial, unsigned* ticket, double* out) {
+    pdl_wait();
+    pdl_launch();
+    const int a = blockIdx.y;
+    const float c = clip ? clip[a] : 1.0f;
+    const long n4 = d_pad / 4;
+    const long per = (n4 + gridDim.x - 1) / gridDim.x;
+    const long lo = (long)blockIdx.x * per;
+    long hi = lo + per; if (hi > n4) hi = n4;
+    const float4* g4 = reinterpret_cast<const float4*>(g + (long)a * d_pad);
+    const float4* v4 = reinterpret_cast<const float4*>(v + (long)a * d_pad);
+    double acc = 0.0;
+    for (long i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+        const float4 gg = __ldcs(g4 + i), vv = __ldcs(v4 + i);
+        const float ge[4] = {gg.x, gg.y, gg.z, gg.w}, ve[4] = {vv.x, vv.y, vv.z, vv.w};
+        float s = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+            const float gi = c * ge[e];
+            const float vn = hp.alpha * ve[e] + (1.0f - hp.alpha) * gi * gi;
+            const float u = hp.lr * gi / (sqrtf(vn) + hp.eps);
+            s = fmaf(u, u, s);
+        }
+        acc += (double)s;
+    }
+    __shared__ double red[256];
+    __shared__ bool last;
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    for (int st = 128; st > 0; st >>= 1) {
+        if (threadIdx.x < st) red[threadIdx.x] += red[threadIdx.x + st];
+        __syncthreads();
+    }
+    const unsigned blocks = gridDim.x * gridDim.y;
+    if (threadIdx.x == 0) {
+        partial[blockIdx.y * gridDim.x + blockIdx.x] = red[0];
+        __threadfence();
+        last = atomicAdd(ticket, 1u) == blocks - 1;
+    }
+    __syncthreads();
+    if (last) {
+        __threadfence();
+        double s = 0.0;
+        for (unsigned k = threadIdx.x; k < blocks; k += blockDim.x) s += ((volatile double*)partial)[k];
+        red[threadIdx.x] = s;
+        __syncthreads();
+        for (int st = 128; st > 0; st >>= 1) {
+            if (threadIdx.x < st) red[threadIdx.x] += red[threadIdx.x + st];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) { *out = red[0]; *ticket = 0; }
+    }
+}
+cudaError_t launch_update_norm(const float* g, const float* v, const float* clip, int n_agents, long d_pad, SweepHp hp,
+                               double* partial, unsigned* ticket, double* out, cudaStream_t st) {
+    if (n_agents < 1 || (d_pad & 3)) return cudaErrorInvalidValue;
+    (void)launch_pdl(update_norm_kernel, dim3(kUpdateNormChunks, n_agents), dim3(256), 0, st, g, v, clip, d_pad, hp, partial,
+                     ticket, out);
+    return cudaGetLastError();
+}
+
 // Straggler injection: occupies the stream for about `usec` microseconds (one sleeping thread).
 // Bounded twice: by the requested time (capped by the caller) and by an iteration limit.
 __global__ void delay_kernel(unsigned long long usec) {

@@ -79,6 +79,48 @@ def test_allreduce_a2c_mode_matches_oracle():
     L.close()
 
 
+def test_update_norm_matches_oracle_and_proposition1_bound_holds():
+    # Identical initial parameters, real rollouts, 2-peer ring of 6 agents: the library's ||alpha G(k)||_F of every
+    # round against the oracle's (the norm of X - Y, its own RMSProp steps), and the measured distance from
+    # consensus under the bound of Proposition 1 built from the LIBRARY's norms, with each round's contraction
+    # factor (second singular value of the oracle's dense mixing matrix) and with their maximum as the constant beta
+    from paper_1906_04585_b200 import binding as B
+    from paper_1906_04585_b200 import learner as LM
+    w = GI.WORKLOADS[0].scaled(n_agents=6, topo_kind=R.RING, topo_peers=2)
+    net = oracle_net(w)
+    L = _learner(w)
+    ohp = oracle_hp(L.hp)
+    with pytest.raises(B.GalaError):
+        B.gala_update_norm(L.ctx)                 # nothing tracked yet
+    B.gala_track_updates(L.ctx, True)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    for i in range(w.n_agents):
+        L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32))
+    X = np.tile(p0.astype(np.float64), (w.n_agents, 1))
+    V = np.zeros_like(X)
+    assert B.gala_consensus_distance(L.ctx) == 0.0
+    steps, s2 = [], []
+    for k in range(5):
+        ros = [GI.rollout(w, i, k) for i in range(w.n_agents)]
+        L.step_sync([LM.DeviceRollout(r) for r in ros])
+        G = np.stack([R.learner_grad(net, X[i], ros[i], ohp)["grad"] for i in range(w.n_agents)])
+        Xn, V, Y = R.sweep_sync(X, G, V, ohp, w.topo_kind, w.topo_peers, k)
+        want = np.linalg.norm(Y - X)
+        got = B.gala_update_norm(L.ctx)
+        assert abs(got - want) <= 5 * TOL_FP32_NET * want, (k, got, want)
+        steps.append(got)
+        s2.append(np.linalg.svd(R.mixing_matrix(w.topo_kind, w.topo_peers, w.n_agents, k), compute_uv=False)[1])
+        dist = B.gala_consensus_distance(L.ctx)
+        assert abs(dist - R.consensus_distance(Xn)) <= 5 * TOL_FP32_NET * dist + 1e-7
+        assert 0.0 < dist <= R.prop1_bound(steps, s2)[k] * (1 + 1e-4)
+        assert dist <= R.prop1_bound(steps, max(s2))[k] * (1 + 1e-4)
+        X = Xn
+    B.gala_track_updates(L.ctx, False)
+    with pytest.raises(B.GalaError):
+        B.gala_update_norm(L.ctx)
+    L.close()
+
+
 def test_staleness_bound_waits_for_the_in_peer():
     from paper_1906_04585_b200 import binding as B
     from paper_1906_04585_b200 import learner as LM

@@ -217,3 +217,40 @@ def test_proposition1_bound():
         bound = sum(beta ** (k + 1 - s) * steps[s] for s in range(k + 1))
         assert R.consensus_distance(Xn) <= bound + 1e-12
         X = Xn
+
+
+def test_prop1_bound_closed_forms():
+    # constant step norm u and constant beta: a geometric series, u beta (1 - beta^(k+1)) / (1 - beta)
+    u, beta, K = 0.37, 0.8, 9
+    b = R.prop1_bound([u] * K, beta)
+    for k in range(K):
+        assert abs(b[k] - u * beta * (1 - beta ** (k + 1)) / (1 - beta)) < 1e-14
+    # beta = 0: consensus after every round; beta = 1: the steps just add up
+    steps = [0.5, 0.1, 2.0, 0.0, 0.3]
+    np.testing.assert_array_equal(R.prop1_bound(steps, 0.0), np.zeros(5))
+    np.testing.assert_allclose(R.prop1_bound(steps, 1.0), np.cumsum(steps), rtol=1e-15)
+    # one factor per round: a round that averages exactly (factor 0) forgets everything before it
+    b = R.prop1_bound([1.0, 2.0, 4.0], [0.5, 0.0, 0.25])
+    np.testing.assert_allclose(b, [0.5, 0.0, 1.0], rtol=1e-15)
+
+
+@pytest.mark.parametrize("kind,peers,n", [(R.EXP, 1, 8), (R.EXP, 2, 8), (R.RING, 2, 6)])
+def test_prop1_bound_holds_with_per_round_factors(kind, peers, n):
+    # the bound with every round's own contraction factor sigma_2(W_k) (brute force: SVD of the dense mixing
+    # matrix) holds round by round and is never above the constant-beta bound with beta = max_k sigma_2(W_k)
+    # (which is 1 for the exponential graphs: single rounds with shift n/2 do not contract every direction)
+    rng = np.random.default_rng(11)
+    d, K = 20, 9
+    hp = R.HParams(max_grad_norm=0.5)
+    X = np.tile(rng.normal(size=(1, d)), (n, 1))
+    V = np.zeros((n, d))
+    steps, s2 = [], []
+    for k in range(K):
+        G = rng.normal(size=(n, d)) * (0.0 if 3 <= k < 6 else 1.0 + k % 2)   # three pure-gossip rounds
+        Xn, V, Y = R.sweep_sync(X, G, V, hp, kind, peers, k)
+        steps.append(np.linalg.norm(Y - X))
+        s2.append(np.linalg.svd(R.mixing_matrix(kind, peers, n, k), compute_uv=False)[1])
+        b = R.prop1_bound(steps, s2)
+        assert R.consensus_distance(Xn) <= b[k] * (1 + 1e-12) + 1e-12
+        assert b[k] <= R.prop1_bound(steps, max(s2))[k] + 1e-12
+        X = Xn
