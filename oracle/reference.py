@@ -16,6 +16,9 @@ Algorithm 1 in the paper's order:
                              ``sweep_replay``  (Algorithm 1 gossip steps and
                              its footnote; Eqs. 5-7 of the appendix)
 
+  distance from consensus -> ``consensus_distance``, ``prop1_bound``
+                             (Propositions 1-2)
+
 Topology schedules are integer-only Python.
 
 Parity status: every function here is pinned by tests/test_oracle_*.py to
