@@ -461,6 +461,38 @@ def run_ours(args):
         a2c_ms = e0.elapsed_time(e1) / 20
         L2.close()
         del ext2
+        # Proposition 1 on this workload: identical initial parameters, eight synchronous rounds with the norm of
+        # every round's step tracked; the measured distance from consensus beside the bound
+        # b(k+1) = sigma_2(W_k) * (b(k) + ||alpha G(k)||), W_k the round's mixing matrix built from the library's
+        # in-peers (equal weights over self and in-peers), sigma_2 its second singular value
+        L3 = LM.Learner(w.n_agents, w.topo_kind, w.topo_peers, w.net_kind, w.n_actions, w.n_envs, w.n_steps,
+                        obs_dim=w.obs_dim, hidden=w.hidden)
+        B.gala_track_updates(L3.ctx, True)
+        p1_dist, p1_bound, bnd = [], [], 0.0
+        p1_W, p1_u, p1_prod = [], [], []
+        for k in range(8):
+            Wk = np.zeros((w.n_agents, w.n_agents))
+            for i in range(w.n_agents):
+                peers = [i] + B.gala_in_peers(L3.ctx, k, i)
+                for j in peers:
+                    Wk[i, j] += 1.0 / len(peers)
+            s2 = float(np.linalg.svd(Wk, compute_uv=False)[1]) if w.n_agents > 1 else 0.0
+            L3.step_sync(sets[k % n_sets])
+            p1_u.append(B.gala_update_norm(L3.ctx))
+            bnd = s2 * (bnd + p1_u[-1])
+            p1_dist.append(B.gala_consensus_distance(L3.ctx))
+            p1_bound.append(bnd)
+            # the same bound with the factor of every step taken from the product of the rounds since, as in the
+            # proof: X(k+1) - mean = -sum_s (W_k ... W_s - 11^T/n) alpha G(s); for the exponential graphs a full
+            # cycle of rounds averages exactly, which single-round factors cannot see
+            p1_W.append(Wk)
+            J = np.full_like(Wk, 1.0 / w.n_agents)
+            P, tot = np.eye(w.n_agents), 0.0
+            for s_ in range(k, -1, -1):
+                P = P @ p1_W[s_]
+                tot += float(np.linalg.norm(P - J, 2)) * p1_u[s_]
+            p1_prod.append(tot)
+        L3.close()
         # closed actor loop: every agent acts T times on the synthetic environment, learns and gossips, nothing
         # crosses the host; timed by the host clock between two synchronisations
         loop_iters = 10
@@ -481,6 +513,10 @@ def run_ours(args):
                               consensus_bytes=int(w.n_agents * L.d * 4),
                               allreduce_a2c_ms_per_round=a2c_ms,
                               allreduce_a2c_frames_per_s=w.frames_per_round / (a2c_ms * 1e-3),
+                              prop1=dict(distance=[round(x, 6) for x in p1_dist], bound=[round(x, 6) for x in p1_bound],
+                                         bound_from_products=[round(x, 6) for x in p1_prod],
+                                         holds=all(d_ <= min(b_, c_) * (1 + 1e-4)
+                                                   for d_, b_, c_ in zip(p1_dist, p1_bound, p1_prod))),
                               note="consensus_call_ms is a host-timed call (sync + one kernel + 8-byte read); "
                                    "all-reduce rounds back to back without L2 flush")
     if rank == 0 and world == 1 and not args.no_extras:

@@ -99,7 +99,7 @@ def test_update_norm_matches_oracle_and_proposition1_bound_holds():
     X = np.tile(p0.astype(np.float64), (w.n_agents, 1))
     V = np.zeros_like(X)
     assert B.gala_consensus_distance(L.ctx) == 0.0
-    steps, s2 = [], []
+    steps, s2, Ws = [], [], []
     for k in range(5):
         ros = [GI.rollout(w, i, k) for i in range(w.n_agents)]
         L.step_sync([LM.DeviceRollout(r) for r in ros])
@@ -114,6 +114,13 @@ def test_update_norm_matches_oracle_and_proposition1_bound_holds():
         assert abs(dist - R.consensus_distance(Xn)) <= 5 * TOL_FP32_NET * dist + 1e-7
         assert 0.0 < dist <= R.prop1_bound(steps, s2)[k] * (1 + 1e-4)
         assert dist <= R.prop1_bound(steps, max(s2))[k] * (1 + 1e-4)
+        # the proof's own form: step s weighted by the norm of (W_k ... W_s - 11^T / n)
+        Ws.append(R.mixing_matrix(w.topo_kind, w.topo_peers, w.n_agents, k))
+        P, tot = np.eye(w.n_agents), 0.0
+        for s_ in range(k, -1, -1):
+            P = P @ Ws[s_]
+            tot += np.linalg.norm(P - 1.0 / w.n_agents, 2) * steps[s_]
+        assert dist <= tot * (1 + 1e-4) and tot <= R.prop1_bound(steps, s2)[k] * (1 + 1e-9)
         X = Xn
     B.gala_track_updates(L.ctx, False)
     with pytest.raises(B.GalaError):
