@@ -112,7 +112,14 @@ typedef struct {
 
 /* Create n_agents agents (1..256).  Allocates everything; parameters are
  * initialised from hp->seed (uniform +-1/sqrt(fan_in)), square-average state
- * to 0, round counters to 0.  Uses the current CUDA device. */
+ * to 0, round counters to 0.  Uses the current CUDA device.
+ * Environment variables read here select older or alternative kernels for the same results; they exist so that
+ * two independent implementations can be compared with each other and with the CPU oracle:
+ *   GALA_CONV_LEGACY     convolution products with one tensor copy per kernel offset and bf16 frame copies
+ *   GALA_HEADS_UNFUSED   separate kernels for heads, objective and head gradients
+ *   GALA_MLP_UNFUSED     separate kernels for the small fully connected network
+ *   GALA_C1B_SLICES=0/1  conv1's bias gradient from column sums of dY1 / from conv2's data-gradient kernel
+ *                        (default: the latter for launches over at least 2048 samples) */
 int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* net,
                 const gala_hparams* hp, gala_ctx** out);
 int gala_destroy(gala_ctx* ctx);
