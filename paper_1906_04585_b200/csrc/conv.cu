@@ -179,15 +179,20 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         issued_w = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0 && u_begin < u_end) {
-        // The weights of the first agent are fetched before the wait for the previous kernel: they were
-        // written by the optimiser pass (or a state upload), which lies at least two kernels back.
-        __syncwarp();
-        if (lane == 0) { mbar_expect_tx(&w_full, (uint32_t)W_BYTES); issued_w = 1; }
-        __syncwarp();
-        const int group = p.group0 + decode_unit<V>(u_begin, p.rows).gz;
-        if (lane < T::W_BOXES) tma_load_3d(smW + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
-    }
+    // The weights of the first agent are fetched before the wait for the previous kernel where they were written
+    // at least two kernels back (by the optimiser pass or a state upload, with conv1's forward pass in between).
+    // conv1's forward pass itself may be the very next kernel after a per-agent optimiser pass: it fetches them
+    // after the wait.
+    auto first_weights = [&]() {
+        if (warp == 0 && u_begin < u_end) {
+            __syncwarp();
+            if (lane == 0) { mbar_expect_tx(&w_full, (uint32_t)W_BYTES); issued_w = 1; }
+            __syncwarp();
+            const int group = p.group0 + decode_unit<V>(u_begin, p.rows).gz;
+            if (lane < T::W_BOXES) tma_load_3d(smW + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
+        }
+    };
+    if constexpr (V != CV_CONV1_FWD) first_weights();
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                      "r"(tmem_cols)
@@ -200,6 +205,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const uint32_t tmem_base = tmem_slot;
     pdl_wait();     // set-up above overlaps the previous kernel; its results are read from here on
     pdl_launch();
+    if constexpr (V == CV_CONV1_FWD) first_weights();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
