@@ -81,7 +81,8 @@ constexpr int kC1Group = 4 * 336;                    // bytes of four input line
 constexpr int kU8Stages = 4;
 constexpr int kU8Bytes = (kC1Lines + 1) * kC1Group;  // 9408
 constexpr int kU8Stride = 9728;
-constexpr int kConvThreads = 352, kConv1Threads = 352 + 128;
+constexpr int kC1ConvWarps = 4;                     // conv1: warps that widen the uint8 lines
+constexpr int kConvThreads = 352, kConv1Threads = 352 + 32 * kC1ConvWarps;
 
 // plane and row shift of a tap
 template <int V> __host__ __device__ constexpr void tap_view(int t, int& plane, int& shift) {
@@ -169,8 +170,8 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 
     if (threadIdx.x == 0) {
         // conv1: a stage is filled by the four converting warps, otherwise by TMA (one arrival with a byte count)
-        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], kU8 ? 4 : 1); mbar_init(&empty_bar[s], 1); }
-        for (int s = 0; s < kU8Stages; s++) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], 4); }
+        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], kU8 ? kC1ConvWarps : 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kU8Stages; s++) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kC1ConvWarps); }
         for (int b = 0; b < 4; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
         mbar_init(&w_full, 1);
         mbar_init(&w_empty, 2);
@@ -318,7 +319,8 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         // group xq (4 pixels x 4 channels); a row is 32 bytes of bf16 whose two halves swap when bit 7 of
         // its address is set (32-byte swizzle).  0..255 are exact in bf16; 1/255 is applied after the MMAs.
         if constexpr (kU8) {
-            const int ct = threadIdx.x - 11 * 32;   // 0..127
+            const int ct = threadIdx.x - 11 * 32;   // 0 .. 32 * kC1ConvWarps - 1
+            constexpr int kCT = 32 * kC1ConvWarps, kChunks = 4 * (kC1Lines + 1) * 21;
             int it = 0;
             for (int u = u_begin; u < u_end; u++, it++) {
                 const int su = it % kU8Stages, s = it % nst;
@@ -327,9 +329,9 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const uint8_t* src = smU + su * kU8Stride;
                 uint8_t* dstage = smX + s * STAGE;
 #pragma unroll
-                for (int k = 0; k < 5; k++) {
-                    const int ch = ct + k * 128;          // 16-byte group of the block, 588 in all
-                    if (ch < 4 * (kC1Lines + 1) * 21) {
+                for (int k = 0; k < (kChunks + kCT - 1) / kCT; k++) {
+                    const int ch = ct + k * kCT;          // 16-byte group of the block, 588 in all
+                    if (ch < kChunks) {
                         const int yl = ch / 21, xq = ch - yl * 21;
                         const uint4 v = *reinterpret_cast<const uint4*>(src + ch * 16);
                         const uint32_t w[4] = {v.x, v.y, v.z, v.w};

@@ -37,7 +37,7 @@ constexpr int kW1Stage = kW1XBytes + kW1DyBytes;            // 43008
 constexpr int kW1Stages = 4;
 constexpr int kW1U8Stages = 4, kW1U8Bytes = 24 * 336, kW1U8Stride = 8192;
 constexpr int kW1Smem = kW1Stages * kW1Stage + kW1U8Stages * kW1U8Stride + 1024;
-constexpr int kW1Threads = 320, kW1ConvWarps = 8;
+constexpr int kW1ConvWarps = 8, kW1Threads = 64 + 32 * kW1ConvWarps;
 constexpr int kW1KSteps = 8;                                // 128 pixel rows of 16 (105 of the tile + the 21-row shift)
 
 __global__ void __launch_bounds__(kW1Threads, 1)
@@ -144,7 +144,8 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
         }
     } else {
         // ------------------------------------------------ converters: uint8 lines -> bf16 phase planes, two copies
-        const int ct = threadIdx.x - 64;   // 0..255
+        const int ct = threadIdx.x - 64;   // 0 .. 32 * kW1ConvWarps - 1
+        constexpr int kCT = 32 * kW1ConvWarps, kChunks = 24 * 21;
         bool ok = true;
         for (int it = 0; it < n_it; it++) {
             const int su = it % kW1U8Stages, s = it % kW1Stages;
@@ -153,9 +154,9 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
             const uint8_t* src = smU + su * kW1U8Stride;
             uint8_t* dstage = smem + s * kW1Stage;
 #pragma unroll
-            for (int k = 0; k < 2; k++) {
-                const int ch = ct + k * 256;          // 16-byte group of the block, 504 in all
-                if (ch < 24 * 21) {
+            for (int k = 0; k < (kChunks + kCT - 1) / kCT; k++) {
+                const int ch = ct + k * kCT;          // 16-byte group of the block, 504 in all
+                if (ch < kChunks) {
                     const int yl = ch / 21, xq = ch - yl * 21;
                     const uint4 v = *reinterpret_cast<const uint4*>(src + ch * 16);
                     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
