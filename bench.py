@@ -267,6 +267,8 @@ def run_ours(args):
         B.gala_set_agent_ctas(L.ctx, args.agent_ctas)
     if args.no_graphs:
         B.gala_set_graphs(L.ctx, False)
+    if args.lanes:
+        B.gala_set_group_lanes(L.ctx, args.lanes)
     ext = torch.cuda.ExternalStream(B.gala_get_stream(L.ctx, -1))
     up = torch.cuda.Stream()      # host -> device copies run on a torch stream; the library's stream waits on it
 
@@ -285,6 +287,14 @@ def run_ours(args):
         random order, each preceded by an injected straggler delay, nothing synchronised in between."""
         if not async_mode:
             L.step_sync(cur)
+            return
+        if args.grouped:
+            order = [int(i) for i in rng.permutation(w.n_agents)]
+            gsz = args.grouped
+            for k0 in range(0, len(order), gsz):
+                lst = order[k0:k0 + gsz]
+                L.learn_many(lst, [cur[i] for i in lst])
+                L.gossip_many(lst)
             return
         for i in rng.permutation(w.n_agents):
             i = int(i)
@@ -588,6 +598,8 @@ def main():
     ap.add_argument("--agent-ctas", type=int, default=-1,
                     help="asynchronous mode: thread blocks per kernel of one agent (-1: the library's default)")
     ap.add_argument("--no-graphs", action="store_true", help="launch every kernel of a learner step directly (no graph replay)")
+    ap.add_argument("--grouped", type=int, default=0, help="asynchronous mode through the grouped calls, lists of this many agents")
+    ap.add_argument("--lanes", type=int, default=0)
     ap.add_argument("--no-skew", action="store_true", help="asynchronous mode without the injected straggler delays")
     ap.add_argument("--sweep-only", action="store_true",
                     help="run only the RMSProp + gossip micro-benchmark (32 agents x 1.7M parameters)")

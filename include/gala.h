@@ -148,6 +148,39 @@ int gala_learn(gala_ctx* ctx, int agent, const gala_rollout* rollout);
  * otherwise keep the local result (Eq. 5).  Never waits for a peer. */
 int gala_gossip(gala_ctx* ctx, int agent);
 
+/* The learner step of Algorithm 1 for SEVERAL agents whose rollouts have arrived, as one set of grouped launches
+ * (every kernel of the step works on the whole list; the kernels are those of gala_step_sync), without any of
+ * the listed agents waiting for an agent that is not listed (Sec. 3: agents proceed at their own pace).
+ * agents[m]: distinct agent indices in any order; rollouts[m]: rollouts[k] belongs to agents[k].  Per agent the
+ * call is gala_learn: a gradient that is still pending is first applied without mixing and published.  The work
+ * goes to one of two internal streams; the call orders it behind everything enqueued for the listed agents
+ * before, and later per-agent calls for them behind it.  A host that polls which simulators have delivered and
+ * hands the ready agents to this call amortises the launch cost of a step over all of them.  Networks other
+ * than the conv net (and rollouts too long for the fused heads kernel) are handled as m calls of gala_learn. */
+int gala_learn_many(gala_ctx* ctx, const int* agents, const gala_rollout* rollouts, int m);
+
+/* gala_gossip for several agents in one launch: for every listed agent the RMSProp step with its pending
+ * gradient, the broadcast of the result as its newest snapshot and, where a snapshot newer than the one last
+ * consumed has COMPLETED for each of its in-peers, the equal-weight average (Eqs. 5-6).  Which snapshots are
+ * usable - complete, or published by an earlier grouped call on the same internal stream and therefore complete
+ * before this call's launch runs - is decided for the whole list before anything is enqueued, so a listed agent
+ * never sees a snapshot published by the same call; listed agents that are each other's in-peers are fine (three snapshot slots per
+ * agent: the slot being written is never one that may be read).  Per-agent results, counters and gala_last_mix
+ * are as after m calls of gala_gossip.  GALA_ETIMEOUT from the staleness bound: nothing was enqueued. */
+int gala_gossip_many(gala_ctx* ctx, const int* agents, int m);
+
+/* Streams the grouped calls alternate between: 1 (default) or 2.  With one, grouped calls run on the device in
+ * the order they were made, every kernel's set-up overlapping its predecessor's tail also across calls, and a
+ * gossip step sees every snapshot that an earlier grouped call published (it runs after it).  With two, the
+ * launch sets of consecutive gala_learn_many calls may overlap on the device; a snapshot published on the other
+ * stream counts only once it has completed. */
+int gala_set_group_lanes(gala_ctx* ctx, int lanes);
+
+/* Non-blocking: *busy = 0 when the agent's latest optimiser / gossip step, and whatever was enqueued for the agent
+ * after it, has completed on the device; 1 otherwise.  For hosts that hand the next rollout of an agent to
+ * gala_learn_many only when the parameters it was collected with are in place. */
+int gala_poll_agent(gala_ctx* ctx, int agent, int* busy);
+
 /* Straggler injection for experiments (the slow simulators of Sec. 1 / Sec. 5 "computational
  * performance"): keeps the agent's stream busy for about `usec` microseconds (0..100000) with one
  * sleeping thread before whatever is enqueued next on it.  The wait is bounded on the device. */
@@ -243,7 +276,8 @@ int gala_stats(gala_ctx* ctx, int agent, long long out[8]);
 /* Which snapshot versions the agent's last gala_gossip consumed: versions[j]
  * for in-peer peers[j]; *mixed = 1 if the average was taken. */
 int gala_last_mix(gala_ctx* ctx, int agent, int* peers, long long* versions, int* n, int* mixed);
-/* Read snapshot `version` of an agent if it is still held (the two newest are). */
+/* Read snapshot `version` of an agent if it is still held (the two newest are; an agent has three slots, the
+ * third being the one its next publication goes to). */
 int gala_get_snapshot(gala_ctx* ctx, int agent, long long version, float* out);
 /* Adopt a caller's CUDA stream (cudaStream_t) for the agent; NULL restores the library's. */
 int gala_set_stream(gala_ctx* ctx, int agent, void* cuda_stream);
@@ -276,7 +310,8 @@ const char* gala_last_error(const gala_ctx* ctx);
  * bf16 (A, B) and float (D); K, M, N and the leading dimensions must keep
  * rows 16-byte aligned (multiples of 8 elements).  split_k >= 1 splits the
  * reduction and sums the partials in a fixed order.  Runs on `stream`
- * (cudaStream_t, may be NULL) and returns after enqueueing. */
+ * (cudaStream_t, may be NULL); allocates its scratch with cudaMalloc, waits for
+ * its work and frees the scratch before it returns. */
 int gala_gemm_bf16(const void* A, const void* B, float* D, int groups, int M, int N, int K,
                    int a_mn, int b_mn, int split_k, void* stream);
 
@@ -291,8 +326,10 @@ int gala_gemm_bf16(const void* A, const void* B, float* D, int groups, int M, in
  * load until exit) and calls no allocating routine.
  *   Limit: groups * split_k * M * N <= 2 Mi floats when split_k > 1; beyond that the call is
  *   refused with GALA_EINVAL and a message naming the limit (no limit for split_k == 1).
- *   First call on each device: looks up the array's device address and resolves the tensor-map
- *   encoder; make that first call outside any stream capture.
+ *   First call on each device: looks up the array's device address, resolves the tensor-map
+ *   encoder and opts the kernel in to large shared memory on that device; make that first call
+ *   before any stream capture begins.  Every call waits on `stream` for its own work (and reads
+ *   one status word back on that stream) before it returns; it waits for no other stream.
  *   All calls share the one array, which keeps the previous call's contents (the call clears the
  *   only word that must start at zero).  Two calls whose GPU work overlaps -- different streams,
  *   threads or processes' contexts on the same device and library image -- race on it; this entry
@@ -311,6 +348,27 @@ int gala_gemm_bf16_static(const void* A, const void* B, float* D, int groups, in
 int gala_sweep_sync(float* x, const float* g, float* v, const float* clip, int n_agents,
                     long long d_padded, const gala_topology* topo, long long round,
                     const gala_hparams* hp, void* stream);
+
+/* Stand-alone per-agent form of the fused RMSProp + gossip pass for a list of agents in ONE launch per 64 agents
+ * (Algorithm 1: optimiser step, broadcast, conditional average; Eqs. 5-6), over caller-owned DEVICE arrays:
+ * x, g, v float32 [n_agents][d_padded]; snap float32 [n_agents][n_slots][d_padded] (the agents' published
+ * snapshots); clip float[n_agents] or NULL (= 1).  For item k (distinct agents):
+ *   y = RMSProp(x, clip * g, v) if has_grad, else y = x (v untouched);  snap[agent][out_slot] = y;
+ *   x = (y + sum_j snap[peer[j]][peer_slot[j]]) / (1 + n_peers)     (n_peers = 0: x = y).
+ * No snapshot slot may be both read and written by one call (GALA_EINVAL).  Bytes per parameter and agent:
+ * 24 + 4 n_peers (x, g, v and the peers' snapshots read once; x, v and the own snapshot written once).
+ * d_padded % 4 == 0; every array 16-byte aligned.  Enqueues on `stream` and returns. */
+typedef struct {
+    int agent;
+    int out_slot;
+    int n_peers;      /* 0..2 */
+    int peer[2];
+    int peer_slot[2];
+    int has_grad;
+} gala_sweep_item;
+int gala_sweep_agents(float* x, const float* g, float* v, float* snap, const float* clip, int n_agents, int n_slots,
+                      long long d_padded, const gala_sweep_item* items, int n_items, const gala_hparams* hp,
+                      void* stream);
 
 #ifdef __cplusplus
 }

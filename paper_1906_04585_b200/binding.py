@@ -49,6 +49,11 @@ class gala_rollout(C.Structure):
     _fields_ = [("obs", C.c_void_p), ("actions", C.c_void_p), ("rewards", C.c_void_p), ("dones", C.c_void_p)]
 
 
+class gala_sweep_item(C.Structure):
+    _fields_ = [("agent", C.c_int), ("out_slot", C.c_int), ("n_peers", C.c_int), ("peer", C.c_int * 2),
+                ("peer_slot", C.c_int * 2), ("has_grad", C.c_int)]
+
+
 EXPORTS = (
     "gala_create", "gala_destroy", "gala_act", "gala_learn", "gala_gossip", "gala_step_sync",
     "gala_sync_agent", "gala_sync_all", "gala_in_peers", "gala_get_state", "gala_set_state",
@@ -59,6 +64,7 @@ EXPORTS = (
     "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_track_updates", "gala_update_norm", "gala_set_stale_timeout",
     "gala_set_agent_ctas", "gala_set_graphs", "gala_losses_all",
     "gala_actor_loop", "gala_actor_read",
+    "gala_learn_many", "gala_gossip_many", "gala_poll_agent", "gala_sweep_agents", "gala_set_group_lanes",
 )
 
 _lib = None
@@ -81,6 +87,12 @@ def lib() -> C.CDLL:
             "gala_act": (i, [vp, i, vp, vp, vp, vp]),
             "gala_learn": (i, [vp, i, C.POINTER(gala_rollout)]),
             "gala_gossip": (i, [vp, i]),
+            "gala_learn_many": (i, [vp, C.POINTER(i), C.POINTER(gala_rollout), i]),
+            "gala_gossip_many": (i, [vp, C.POINTER(i), i]),
+            "gala_poll_agent": (i, [vp, i, C.POINTER(i)]),
+            "gala_set_group_lanes": (i, [vp, i]),
+            "gala_sweep_agents": (i, [vp, vp, vp, vp, vp, i, i, ll, C.POINTER(gala_sweep_item), i,
+                                      C.POINTER(gala_hparams), vp]),
             "gala_delay": (i, [vp, i, i]),
             "gala_consensus_distance": (i, [vp, C.POINTER(C.c_double)]),
             "gala_track_updates": (i, [vp, i]),
@@ -173,6 +185,30 @@ def gala_learn(ctx, agent: int, rollout: gala_rollout):
 
 def gala_gossip(ctx, agent: int):
     _check(ctx, lib().gala_gossip(ctx, agent))
+
+
+def gala_learn_many(ctx, agents: Sequence[int], rollouts: Sequence[gala_rollout]):
+    m = len(agents)
+    assert len(rollouts) == m
+    ids = (C.c_int * m)(*agents)
+    arr = rollouts if isinstance(rollouts, C.Array) else (gala_rollout * m)(*rollouts)
+    _check(ctx, lib().gala_learn_many(ctx, ids, arr, m))
+
+
+def gala_gossip_many(ctx, agents: Sequence[int]):
+    m = len(agents)
+    _check(ctx, lib().gala_gossip_many(ctx, (C.c_int * m)(*agents), m))
+
+
+def gala_poll_agent(ctx, agent: int) -> bool:
+    """True while work enqueued for the agent is still running."""
+    busy = C.c_int()
+    _check(ctx, lib().gala_poll_agent(ctx, agent, C.byref(busy)))
+    return bool(busy.value)
+
+
+def gala_set_group_lanes(ctx, lanes: int):
+    _check(ctx, lib().gala_set_group_lanes(ctx, lanes))
 
 
 def gala_delay(ctx, agent: int, usec: int):
@@ -361,6 +397,20 @@ def gala_sweep_sync(x, g, v, clip, n_agents, d_padded, topo: gala_topology, rnd:
                                C.byref(hp), stream)
     if rc < 0:
         raise GalaError(rc, "gala_sweep_sync")
+
+
+def gala_sweep_agents(x, g, v, snap, clip, n_agents: int, n_slots: int, d_padded: int, items, hp: gala_hparams,
+                      stream=None):
+    """items: sequence of (agent, out_slot, [(peer, peer_slot), ...], has_grad)."""
+    arr = (gala_sweep_item * len(items))()
+    for k, (agent, out_slot, peers, has_grad) in enumerate(items):
+        arr[k].agent, arr[k].out_slot, arr[k].n_peers, arr[k].has_grad = agent, out_slot, len(peers), int(has_grad)
+        for j, (pj, sj) in enumerate(peers):
+            arr[k].peer[j], arr[k].peer_slot[j] = pj, sj
+    rc = lib().gala_sweep_agents(_ptr(x), _ptr(g), _ptr(v), _ptr(snap), _ptr(clip), n_agents, n_slots, d_padded, arr,
+                                 len(items), C.byref(hp), stream)
+    if rc < 0:
+        raise GalaError(rc, "gala_sweep_agents")
 
 
 def default_hparams(n_envs: int, n_steps: int, **kw) -> gala_hparams:

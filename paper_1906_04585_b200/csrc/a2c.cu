@@ -301,7 +301,8 @@ constexpr int kHeadsMaxA1 = 19;   // 18 actions + value
 
 __global__ void __launch_bounds__(256) heads_fused_kernel(HeadsFusedArgs p) {
     extern __shared__ __align__(16) unsigned char hf_smem[];
-    const int g = blockIdx.y, bi = blockIdx.x;
+    const int gz = blockIdx.y, bi = blockIdx.x;
+    const int g = agent_slot(p.am, gz);   // the agent's tensors; the rollout pointers come with the launch (gz)
     const int T = p.T, E = p.E, A = p.A, A1 = A + 1, T1 = T + 1;
     const int e0 = bi * p.ne;
     const int ne = min(p.ne, E - e0);
@@ -411,9 +412,9 @@ __global__ void __launch_bounds__(256) heads_fused_kernel(HeadsFusedArgs p) {
             if (k < A) logits[row * A + k] = zsm[i]; else values[row] = zsm[i];
         }
     }
-    const int* actions = reinterpret_cast<const int*>(p.actions.p[g]);
-    const float* rewards = reinterpret_cast<const float*>(p.rewards.p[g]);
-    const unsigned char* dones = reinterpret_cast<const unsigned char*>(p.dones.p[g]);
+    const int* actions = reinterpret_cast<const int*>(p.actions.p[gz]);
+    const float* rewards = reinterpret_cast<const float*>(p.rewards.p[gz]);
+    const unsigned char* dones = reinterpret_cast<const unsigned char*>(p.dones.p[gz]);
     const long S = (long)T * E;
     // returns: a warp per environment, time steps in the lanes, reverse scan of the maps G -> r + gamma (1 - done) G
     for (int el = warp; el < ne; el += 8) {
@@ -587,7 +588,7 @@ __global__ void __launch_bounds__(256) heads_wgrad_tiled_kernel(HeadsBwdArgs a) 
     constexpr int kChunk = 256;
     __shared__ __align__(16) float dzs[kChunk][kHeadsMaxA1 + 1];   // rows of 20 floats; entries from A + 1 on are zero
     __shared__ float part[8][kHeadsMaxA1][32];
-    const int g = blockIdx.y, tile = blockIdx.x;
+    const int g = agent_slot(a.am, blockIdx.y), tile = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int A = a.A, A1 = A + 1, H = a.H;
     const bool bias_tile = tile * 32 >= H;

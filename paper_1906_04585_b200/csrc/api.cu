@@ -67,17 +67,25 @@ struct StepGraph {
     long long tag_launches[T_COUNT] = {};
 };
 
+// Snapshot slots per agent: version w lives in slot w % kSnapSlots.  A reader takes one of the two newest versions,
+// so with three slots the version that is written next never shares a slot with one that a sweep enqueued at the
+// same time may read: agents that are each other's in-peers can publish and average in ONE launch.
+constexpr int kSnapSlots = 3;
+
 struct Agent {
     cudaStream_t stream = nullptr, lib_stream = nullptr;
-    cudaEvent_t pub_event[2] = {nullptr, nullptr};  // completion of the sweep that wrote snapshot slot s
-    cudaEvent_t sweep_done = nullptr;               // completion of the agent's latest sweep
+    cudaEvent_t pub_event[kSnapSlots] = {};         // completion of the sweep that wrote snapshot slot s
     cudaEvent_t fence = nullptr;                    // scratch event for cross-stream ordering
+    cudaStream_t sweep_stream = nullptr;            // stream the agent's latest sweep was enqueued on
+    cudaStream_t pub_stream[kSnapSlots] = {};       // ... and the sweep that wrote slot s
+    bool dirty = false;                             // its own stream carries work no group launch is ordered behind yet
+    int group_lane = -1;                            // group lane whose work its own stream is not ordered behind yet
     long long version = 0;                          // newest snapshot version enqueued (0: none)
     long long round = 0;                            // local iteration counter
     bool pending = false;                           // a gradient waits for its optimiser step
     long long since_mix = 0;                        // local iterations since the last average with the in-peers
     std::vector<long long> consumed;                // newest version consumed from each agent
-    std::vector<int> slot_readers[2];               // agents whose sweeps read snapshot slot s
+    std::vector<int> slot_readers[kSnapSlots];      // agents whose sweeps read snapshot slot s
     long long frames = 0, mixes = 0, skipped = 0, stale_sum = 0, stale_max = 0, stale_waits = 0;
     // closed actor loop: rollout buffers owned by the library and the environment's step counter
     void* loop_obs = nullptr; int* loop_actions = nullptr; float* loop_rewards = nullptr;
@@ -111,6 +119,14 @@ struct gala_ctx {
     // of data gradients they do not depend on
     cudaStream_t side_stream = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // Streams of the grouped per-agent calls (gala_learn_many / gala_gossip_many): a launch set for a list of agents
+    // goes to one lane (its stream, a side stream for the weight gradients); consecutive calls alternate between the
+    // lanes so that the tail of one set overlaps the head of the next.
+    struct Lane { cudaStream_t st = nullptr, side = nullptr; cudaEvent_t fork = nullptr, join = nullptr, done = nullptr; };
+    Lane glane[2];
+    int n_lanes = 1, next_lane = 0;
+    const AgentMap* cur_map = nullptr;       // agent list of the launches being enqueued (null: a range of agents)
+    cudaEvent_t cur_fork = nullptr, cur_join = nullptr;   // fork / join events of the stream pair in use
     long long sync_round = 0;
     long long launches = 0;
     long long tag_launches[T_COUNT] = {};
@@ -283,6 +299,11 @@ void init_tensor(float* p, long off, long count, int fan_in, uint64_t seed, uint
 void fill_batch(PtrBatch& pb, const void* base, long stride_bytes, int agent0, int count) {
     for (int i = 0; i < count; i++) pb.p[i] = reinterpret_cast<const char*>(base) + (long)(agent0 + i) * stride_bytes;
 }
+
+// Agents of the launches being enqueued: k-th agent of a launch over [agent0, agent0 + groups), or of the list in use
+// (then agent0 is 0 and every base pointer is agent 0's).
+inline int sel_agent(const gala_ctx* c, int agent0, int k) { return c->cur_map ? (int)c->cur_map->v[k] : agent0 + k; }
+inline AgentMap sel_map(const gala_ctx* c) { return c->cur_map ? *c->cur_map : AgentMap{}; }
 
 // ------------------------------------------------------------------ GEMM plans (conv net)
 int build_plans(gala_ctx* c) {
@@ -515,7 +536,7 @@ int pick_splits(gala_ctx* c, int groups, int S, long count, int fixed) {
 int run_conv1_wgrad(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, cudaStream_t st) {
     Wgrad1Args a = c->cwgrad1.args;
     const long count = 32 * 256;
-    a.group0 = agent0; a.groups = groups; a.obs = obs;
+    a.group0 = agent0; a.groups = groups; a.obs = obs; a.am = sel_map(c);
     a.splits = pick_splits(c, groups, a.samples, count, 3);
     float* final_out = a.out + (long)agent0 * a.out_group_stride;
     if (a.splits == 1) {
@@ -540,7 +561,7 @@ int run_conv_wgrad(gala_ctx* c, const WgradPlan& p, int agent0, int groups, cuda
     const int S = a.samples;
     const long count = (long)(a.variant == WG_CONV2 ? 64 * 512 : 64 * 576);
     const int best = pick_splits(c, groups, S, count, 6);
-    a.group0 = agent0; a.groups = groups; a.splits = best;
+    a.group0 = agent0; a.groups = groups; a.splits = best; a.am = sel_map(c);
     const int l = a.variant == WG_CONV2 ? 1 : 2;
     if (best == 1) {
         a.out += (long)agent0 * a.out_group_stride;
@@ -566,7 +587,7 @@ int flush_pending_reduces(gala_ctx* c, int agent0, int groups, cudaStream_t st) 
     c->pending.n = 0;
     LAUNCH(T_SPLITK, st, launch_splitk_reduce_multi(c->splitk_ws + (long)agent0 * c->splitk_group_stride,
                                                    c->g + (long)agent0 * c->d_pad, segs, groups, c->splitk_group_stride,
-                                                   c->d_pad, st));
+                                                   c->d_pad, st, c->cur_map));
     return GALA_OK;
 }
 
@@ -574,7 +595,7 @@ int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, c
              const PtrBatch* obs = nullptr) {
     ConvArgs a = p.args;
     if (obs) a.obs = *obs;
-    a.group0 = agent0; a.groups = groups; a.rows = rows; a.max_ctas = c->cur_ctas;
+    a.group0 = agent0; a.groups = groups; a.rows = rows; a.max_ctas = c->cur_ctas; a.am = sel_map(c);
     a.out += (long)agent0 * a.out_group_stride;
     if (a.gate_out) a.gate_out += (long)agent0 * a.gate_group_stride;
     if (a.gate_in) a.gate_in += (long)agent0 * a.gate_group_stride;
@@ -588,7 +609,7 @@ int run_conv(gala_ctx* c, const ConvPlan& p, int agent0, int groups, int rows, c
 
 int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override, cudaStream_t st) {
     GemmArgs a = p.args;
-    a.group0 = agent0; a.groups = groups; a.max_ctas = c->cur_ctas;
+    a.group0 = agent0; a.groups = groups; a.max_ctas = c->cur_ctas; a.am = sel_map(c);
     if (m_override > 0) a.M = m_override;
     const bool bf = a.flags & EPI_OUT_BF16;
     a.out = reinterpret_cast<char*>(a.out) + (long)agent0 * a.out_group_stride * (bf ? 2 : 4);
@@ -610,7 +631,7 @@ int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t s
     if (split == 1) return run_plan(c, p, agent0, groups, 0, st);
     GemmArgs a = p.args;
     const long count = (long)p.args.M * p.args.N;
-    a.group0 = agent0; a.groups = groups; a.split_k = split; a.max_ctas = c->cur_ctas;
+    a.group0 = agent0; a.groups = groups; a.split_k = split; a.max_ctas = c->cur_ctas; a.am = sel_map(c);
     a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
     a.out_group_stride = c->splitk_group_stride;
     a.out_split_stride = count;
@@ -660,7 +681,7 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
             } else {
                 GemmArgs a = p.args;
                 const long count = (long)rows * kHidden;
-                a.group0 = agent0; a.groups = groups; a.M = rows; a.split_k = split; a.max_ctas = c->cur_ctas;
+                a.group0 = agent0; a.groups = groups; a.M = rows; a.split_k = split; a.max_ctas = c->cur_ctas; a.am = sel_map(c);
                 a.flags = 0; a.bias = nullptr;
                 a.out = c->splitk_ws + (long)agent0 * c->splitk_group_stride;
                 a.out_group_stride = c->splitk_group_stride; a.out_split_stride = count;
@@ -722,8 +743,8 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
     cudaStream_t ws = side ? side : st;
     auto fork = [&]() -> int {
         if (!side) return GALA_OK;
-        CK(cudaEventRecord(c->ev_fork, st));
-        CK(cudaStreamWaitEvent(side, c->ev_fork, 0));
+        CK(cudaEventRecord(c->cur_fork, st));
+        CK(cudaStreamWaitEvent(side, c->cur_fork, 0));
         return GALA_OK;
     };
     c->pending.n = 0;
@@ -746,8 +767,9 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         m.ticket = c->heads_ticket + agent0;
         LAUNCH(T_MLP_FUSED, st, launch_mlp_fused(m, groups, st));
         for (int i = 0; i < groups; i++) {
-            c->agents[agent0 + i].pending = true;
-            c->agents[agent0 + i].frames += S;
+            Agent& ag = c->agents[sel_agent(c, agent0, i)];
+            ag.pending = true;
+            ag.frames += S;
         }
         return GALA_OK;
     }
@@ -783,6 +805,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         hf.dh = c->dh + (long)agent0 * S * kHidden; hf.dh_stride = S * kHidden;
         hf.loss_partial = c->heads_partial + (long)agent0 * c->E * 4;
         hf.ticket = c->heads_ticket + agent0;
+        hf.am = sel_map(c);
         LAUNCH(T_HEADS_FUSED, st, launch_heads_fused(hf, groups, st));
     } else {
         LAUNCH(T_LOSS, st, launch_a2c_loss(la, groups, st));
@@ -794,6 +817,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
     hb.dlogits = la.dlogits; hb.dlogits_stride = S * A;
     hb.dvalues = la.dvalues; hb.dvalues_stride = S;
     hb.grad = c->g + (long)agent0 * dp; hb.g_stride = dp;
+    hb.am = sel_map(c);
     if (c->conv) {
         const int P[3] = {400, 81, 49};
         hb.H = kHidden; hb.act = 1;
@@ -858,11 +882,11 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
             LAUNCH(T_COLSUM, cs, launch_colsum(jobs, c->legacy_conv ? 4 : slices ? 1 : 2, c->g + (long)agent0 * dp, dp,
                                                c->colsum_partial + (long)agent0 * kColsumJobs * kColsumChunks * 512,
                                                c->colsum_ticket + (long)agent0 * kColsumJobs, groups, cs,
-                                               slices ? &sl : nullptr));
+                                               slices ? &sl : nullptr, c->cur_map));
         }
         if (side) {   // join: the gradient is complete when both streams are done
-            CK(cudaEventRecord(c->ev_join, side));
-            CK(cudaStreamWaitEvent(st, c->ev_join, 0));
+            CK(cudaEventRecord(c->cur_join, side));
+            CK(cudaStreamWaitEvent(st, c->cur_join, 0));
         }
     } else {
         const int H = c->H;
@@ -897,10 +921,11 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         kn.partial = c->fc_sq + (long)agent0 * kn.n_partials; kn.partial_group_stride = kn.n_partials;
     }
     LAUNCH(T_GRAD_NORM, st, launch_grad_norm(c->g, c->d, dp, agent0, groups, c->hp.max_grad_norm, c->norm_partial, c->norm_ticket,
-                            c->norm, c->clip, st, c->conv ? &kn : nullptr));
+                            c->norm, c->clip, st, c->conv ? &kn : nullptr, c->cur_map));
     for (int i = 0; i < groups; i++) {
-        c->agents[agent0 + i].pending = true;
-        c->agents[agent0 + i].frames += S;
+        Agent& ag = c->agents[sel_agent(c, agent0, i)];
+        ag.pending = true;
+        ag.frames += S;
     }
     return GALA_OK;
 }
@@ -971,91 +996,209 @@ int learn_range_cached(gala_ctx* c, int agent0, int groups, const gala_rollout* 
     return GALA_OK;
 }
 
-// Newest snapshot version of agent j whose writing sweep has completed (0: none usable).
-long long usable_version(gala_ctx* c, int j) {
+// Newest snapshot version of agent j that a sweep enqueued now on stream `st` may read (0: none): its writing
+// sweep has completed, or it was enqueued earlier on the same stream and so completes before the reader runs
+// (the grouped calls share their streams; an agent's own stream carries no other agent's sweeps).
+long long usable_version(gala_ctx* c, int j, cudaStream_t st) {
     Agent& a = c->agents[j];
     for (long long w = a.version; w > 0 && w >= a.version - 1; w--)
-        if (cudaEventQuery(a.pub_event[w & 1]) == cudaSuccess) return w;
+        if (a.pub_stream[w % kSnapSlots] == st || cudaEventQuery(a.pub_event[w % kSnapSlots]) == cudaSuccess) return w;
     return 0;
+}
+
+// What one agent's optimiser / gossip step will do, decided on the host when it is enqueued.
+struct SweepPlan {
+    int np = 0;                    // in-peers of the agent's current round
+    int peers[2] = {0, 0};
+    long long vers[2] = {0, 0};    // snapshot version taken from each
+    bool fresh = false;            // a newer completed snapshot than the one last consumed exists for every in-peer
+    bool waited = false;           // ... after a wait forced by the staleness bound
+    long long w = 0;               // version the agent publishes
+    int slot = 0;                  // and its slot
+};
+
+// Decides (and, under the staleness bound, waits on the host); changes nothing in the context.
+int plan_sweep(gala_ctx* c, int i, bool try_mix, cudaStream_t st, SweepPlan* sp) {
+    Agent& ag = c->agents[i];
+    int off[2] = {0, 0};
+    sp->np = try_mix ? topo_offsets(c->topo, c->n, ag.round, off) : 0;
+    sp->fresh = sp->np > 0;
+    for (int j = 0; j < sp->np; j++) {
+        sp->peers[j] = ((i - off[j]) % c->n + c->n) % c->n;
+        sp->vers[j] = usable_version(c, sp->peers[j], st);
+        if (sp->vers[j] <= ag.consumed[sp->peers[j]]) sp->fresh = false;
+    }
+    // Staleness bound (Sec. 3): if more than tau local iterations have passed since this agent last
+    // averaged, it waits for its in-peers' newest snapshots instead of going on alone.  The wait is a
+    // host wait with a deadline; only snapshots that are already enqueued can complete, so if an
+    // in-peer has nothing newer on its stream the call gives up at once.
+    if (try_mix && sp->np > 0 && !sp->fresh && c->hp.staleness_tau >= 0 && ag.since_mix > c->hp.staleness_tau) {
+        for (int j = 0; j < sp->np; j++) {
+            Agent& pj = c->agents[sp->peers[j]];
+            if (pj.version <= ag.consumed[sp->peers[j]])
+                return fail(c, GALA_ETIMEOUT, "agent %d: %lld iterations without a message and in-peer %d has published "
+                            "nothing newer (tau = %d)", i, ag.since_mix, sp->peers[j], c->hp.staleness_tau);
+        }
+        const auto t0 = std::chrono::steady_clock::now();
+        for (int j = 0; j < sp->np; j++) {
+            Agent& pj = c->agents[sp->peers[j]];
+            for (;;) {
+                cudaError_t e = cudaEventQuery(pj.pub_event[pj.version % kSnapSlots]);
+                if (e == cudaSuccess) break;
+                if (e != cudaErrorNotReady) return fail(c, GALA_ECUDA, "cudaEventQuery: %s", cudaGetErrorString(e));
+                const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+                if (ms >= c->stale_timeout_ms)
+                    return fail(c, GALA_ETIMEOUT, "agent %d: in-peer %d's snapshot still not complete after %d ms", i,
+                                sp->peers[j], c->stale_timeout_ms);
+                std::this_thread::sleep_for(std::chrono::microseconds(20));
+            }
+            sp->vers[j] = pj.version;
+        }
+        sp->fresh = true;
+        sp->waited = true;
+    }
+    sp->w = ag.version + 1;
+    sp->slot = (int)(sp->w % kSnapSlots);
+    return GALA_OK;
+}
+
+// Pairwise back-pressure: sweeps that may still read the slot the agent is about to overwrite go first.
+// `st` is the stream the agent's new sweep goes to; readers whose latest sweep sits on the same stream are
+// ordered already.
+int sweep_backpressure(gala_ctx* c, int i, const SweepPlan& sp, cudaStream_t st) {
+    Agent& ag = c->agents[i];
+    for (int r : ag.slot_readers[sp.slot]) {
+        Agent& rd = c->agents[r];
+        if (rd.version > 0 && rd.sweep_stream != st) CK(cudaStreamWaitEvent(st, rd.pub_event[rd.version % kSnapSlots], 0));
+    }
+    ag.slot_readers[sp.slot].clear();
+    return GALA_OK;
+}
+
+// Host-side record of a sweep that has been enqueued on `st` (its completion event recorded by the caller).
+void commit_sweep(gala_ctx* c, int i, const SweepPlan& sp, cudaStream_t st) {
+    Agent& ag = c->agents[i];
+    if (sp.fresh) {
+        for (int j = 0; j < sp.np; j++) {
+            Agent& pj = c->agents[sp.peers[j]];
+            pj.slot_readers[sp.vers[j] % kSnapSlots].push_back(i);
+            const long long stale = pj.version - sp.vers[j];
+            ag.stale_sum += stale;
+            if (stale > ag.stale_max) ag.stale_max = stale;
+            ag.consumed[sp.peers[j]] = sp.vers[j];
+        }
+        ag.mixes++;
+        ag.since_mix = 0;
+    } else if (sp.np > 0) {
+        ag.skipped++;
+        ag.since_mix++;
+    }
+    if (sp.waited) ag.stale_waits++;
+    ag.version = sp.w;
+    ag.sweep_stream = st;
+    ag.pub_stream[sp.slot] = st;
+    ag.pending = false;
+    ag.last_n = sp.np; ag.last_mixed = sp.fresh ? 1 : 0;
+    for (int j = 0; j < 2; j++) { ag.last_peers[j] = sp.peers[j]; ag.last_versions[j] = sp.fresh ? sp.vers[j] : 0; }
+}
+
+// Orders the agent's own stream behind the group launches that touched the agent, before a per-agent call
+// enqueues on it.
+int own_stream_begin(gala_ctx* c, Agent& ag) {
+    if (ag.group_lane >= 0) {
+        CK(cudaStreamWaitEvent(ag.stream, c->glane[ag.group_lane].done, 0));
+        ag.group_lane = -1;
+    }
+    ag.dirty = true;
+    return GALA_OK;
 }
 
 // Optimiser step + publication (+ conditional average) for one agent on its stream.
 int sweep_agent(gala_ctx* c, int i, bool try_mix) {
     Agent& ag = c->agents[i];
     const long dp = c->d_pad;
-    int off[2] = {0, 0};
-    int np = try_mix ? topo_offsets(c->topo, c->n, ag.round, off) : 0;
-    int peers[2] = {0, 0};
-    long long vers[2] = {0, 0};
-    bool fresh = np > 0;
-    for (int j = 0; j < np; j++) {
-        peers[j] = ((i - off[j]) % c->n + c->n) % c->n;
-        vers[j] = usable_version(c, peers[j]);
-        if (vers[j] <= ag.consumed[peers[j]]) fresh = false;
-    }
-    // Staleness bound (Sec. 3): if more than tau local iterations have passed since this agent last
-    // averaged, it waits for its in-peers' newest snapshots instead of going on alone.  The wait is a
-    // host wait with a deadline; only snapshots that are already enqueued can complete, so if an
-    // in-peer has nothing newer on its stream the call gives up at once.
-    if (try_mix && np > 0 && !fresh && c->hp.staleness_tau >= 0 && ag.since_mix > c->hp.staleness_tau) {
-        for (int j = 0; j < np; j++) {
-            Agent& pj = c->agents[peers[j]];
-            if (pj.version <= ag.consumed[peers[j]])
-                return fail(c, GALA_ETIMEOUT, "agent %d: %lld iterations without a message and in-peer %d has published "
-                            "nothing newer (tau = %d)", i, ag.since_mix, peers[j], c->hp.staleness_tau);
-        }
-        const auto t0 = std::chrono::steady_clock::now();
-        for (int j = 0; j < np; j++) {
-            Agent& pj = c->agents[peers[j]];
-            for (;;) {
-                cudaError_t e = cudaEventQuery(pj.pub_event[pj.version & 1]);
-                if (e == cudaSuccess) break;
-                if (e != cudaErrorNotReady) return fail(c, GALA_ECUDA, "cudaEventQuery: %s", cudaGetErrorString(e));
-                const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
-                if (ms >= c->stale_timeout_ms)
-                    return fail(c, GALA_ETIMEOUT, "agent %d: in-peer %d's snapshot still not complete after %d ms", i,
-                                peers[j], c->stale_timeout_ms);
-                std::this_thread::sleep_for(std::chrono::microseconds(20));
-            }
-            vers[j] = pj.version;
-        }
-        fresh = true;
-        ag.stale_waits++;
-    }
-    const long long w = ag.version + 1;
-    const int slot = (int)(w & 1);
-    // pairwise back-pressure: sweeps that still read the slot we are about to overwrite go first
-    for (int r : ag.slot_readers[slot]) CK(cudaStreamWaitEvent(ag.stream, c->agents[r].sweep_done, 0));
-    ag.slot_readers[slot].clear();
+    SweepPlan sp;
+    int r = plan_sweep(c, i, try_mix, ag.stream, &sp);
+    if (r != GALA_OK) return r;
+    if ((r = own_stream_begin(c, ag)) != GALA_OK) return r;
+    if ((r = sweep_backpressure(c, i, sp, ag.stream)) != GALA_OK) return r;
     const float* p0 = nullptr;
     const float* p1 = nullptr;
-    if (fresh) {
-        for (int j = 0; j < np; j++) {
-            Agent& pj = c->agents[peers[j]];
-            const float* ptr = c->snap + ((long)peers[j] * 2 + (vers[j] & 1)) * dp;
+    if (sp.fresh)
+        for (int j = 0; j < sp.np; j++) {
+            const float* ptr = c->snap + ((long)sp.peers[j] * kSnapSlots + sp.vers[j] % kSnapSlots) * dp;
             if (j == 0) p0 = ptr; else p1 = ptr;
-            pj.slot_readers[vers[j] & 1].push_back(i);
-            const long long stale = pj.version - vers[j];
-            ag.stale_sum += stale;
-            if (stale > ag.stale_max) ag.stale_max = stale;
-            ag.consumed[peers[j]] = vers[j];
         }
-        ag.mixes++;
-        ag.since_mix = 0;
-    } else if (np > 0) {
-        ag.skipped++;
-        ag.since_mix++;
-    }
     SweepHp hp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps};
     LAUNCH(T_SWEEP_AGENT, ag.stream, launch_sweep_agent(c->x + (long)i * dp, ag.pending ? c->g + (long)i * dp : nullptr, c->v + (long)i * dp,
-                              c->snap + ((long)i * 2 + slot) * dp, p0, p1, fresh ? np : 0, c->clip + i,
+                              c->snap + ((long)i * kSnapSlots + sp.slot) * dp, p0, p1, sp.fresh ? sp.np : 0, c->clip + i,
                               c->conv ? c->shadow + (long)i * dp : nullptr, dp, hp, ag.stream));
-    CK(cudaEventRecord(ag.pub_event[slot], ag.stream));
-    CK(cudaEventRecord(ag.sweep_done, ag.stream));
-    ag.version = w;
-    ag.pending = false;
-    ag.last_n = np; ag.last_mixed = fresh ? 1 : 0;
-    for (int j = 0; j < 2; j++) { ag.last_peers[j] = peers[j]; ag.last_versions[j] = fresh ? vers[j] : 0; }
+    CK(cudaEventRecord(ag.pub_event[sp.slot], ag.stream));
+    commit_sweep(c, i, sp, ag.stream);
+    return GALA_OK;
+}
+
+// A group lane becomes ordered behind everything that was enqueued for the listed agents elsewhere: work on their
+// own streams (per-agent calls, the tail of a synchronous round) and launch sets on the other lane.
+int lane_acquire(gala_ctx* c, int lane, const int* agents, int m) {
+    gala_ctx::Lane& L = c->glane[lane];
+    bool other = false;
+    for (int k = 0; k < m; k++) {
+        Agent& ag = c->agents[agents[k]];
+        if (ag.dirty) {
+            CK(cudaEventRecord(ag.fence, ag.stream));
+            CK(cudaStreamWaitEvent(L.st, ag.fence, 0));
+            ag.dirty = false;
+        }
+        if (ag.group_lane >= 0 && ag.group_lane != lane) other = true;
+    }
+    if (other) CK(cudaStreamWaitEvent(L.st, c->glane[lane ^ 1].done, 0));
+    return GALA_OK;
+}
+int lane_release(gala_ctx* c, int lane, const int* agents, int m) {
+    CK(cudaEventRecord(c->glane[lane].done, c->glane[lane].st));
+    for (int k = 0; k < m; k++) c->agents[agents[k]].group_lane = lane;
+    return GALA_OK;
+}
+
+// Optimiser step + publication (+ conditional average) for a list of distinct agents on a group lane, one
+// launch per kBatch agents.  All decisions are taken before anything is enqueued or recorded, so an agent of the
+// list never counts a snapshot of the same call as complete.
+int sweep_group(gala_ctx* c, int lane, const int* agents, int m, bool try_mix) {
+    gala_ctx::Lane& L = c->glane[lane];
+    const long dp = c->d_pad;
+    std::vector<SweepPlan> plans((size_t)m);
+    for (int k = 0; k < m; k++) {
+        int r = plan_sweep(c, agents[k], try_mix, L.st, &plans[k]);
+        if (r != GALA_OK) return r;
+    }
+    for (int k = 0; k < m; k++) {
+        int r = sweep_backpressure(c, agents[k], plans[k], L.st);
+        if (r != GALA_OK) return r;
+    }
+    for (int k0 = 0; k0 < m; k0 += kBatch) {
+        const int cnt = m - k0 < kBatch ? m - k0 : kBatch;
+        SweepManyArgs a{};
+        a.x = c->x; a.g = c->g; a.v = c->v; a.snap = c->snap; a.shadow = c->conv ? c->shadow : nullptr; a.clip = c->clip;
+        a.d_pad = dp; a.hp = SweepHp{c->hp.lr, c->hp.rms_alpha, c->hp.rms_eps}; a.error_word = c->error_word;
+        a.n_items = cnt;
+        for (int e = 0; e < cnt; e++) {
+            const int i = agents[k0 + e];
+            const SweepPlan& sp = plans[k0 + e];
+            SweepItem& it = a.it[e];
+            it.x_row = i;
+            it.out_row = i * kSnapSlots + sp.slot;
+            it.p_row[0] = it.p_row[1] = -1;
+            if (sp.fresh)
+                for (int j = 0; j < sp.np; j++) it.p_row[j] = sp.peers[j] * kSnapSlots + (int)(sp.vers[j] % kSnapSlots);
+            if (c->agents[i].pending) a.has_grad[e >> 5] |= 1u << (e & 31);
+        }
+        LAUNCH(T_SWEEP_AGENT, L.st, launch_sweep_many(a, L.st));
+    }
+    for (int k = 0; k < m; k++) {
+        CK(cudaEventRecord(c->agents[agents[k]].pub_event[plans[k].slot], L.st));
+        commit_sweep(c, agents[k], plans[k], L.st);
+    }
     return GALA_OK;
 }
 
@@ -1096,6 +1239,16 @@ int check_error_word(gala_ctx* c) {
 }
 
 bool valid_agent(const gala_ctx* c, int a) { return c && a >= 0 && a < c->n; }
+
+// Host wait for everything that was enqueued for the agent, wherever it went: the synchronous stream, the lane
+// of the last grouped call that listed it, its own stream.
+int settle_agent(gala_ctx* c, int agent) {
+    Agent& ag = c->agents[agent];
+    CK(cudaStreamSynchronize(c->main_stream));
+    if (ag.group_lane >= 0) CK(cudaStreamSynchronize(c->glane[ag.group_lane].st));
+    CK(cudaStreamSynchronize(ag.stream));
+    return GALA_OK;
+}
 
 }  // namespace
 
@@ -1162,19 +1315,25 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
     CK(cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking));
     CK(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
+    c->cur_fork = c->ev_fork; c->cur_join = c->ev_join;
+    for (gala_ctx::Lane& L : c->glane) {
+        CK(cudaStreamCreateWithFlags(&L.st, cudaStreamNonBlocking));
+        CK(cudaStreamCreateWithFlags(&L.side, cudaStreamNonBlocking));
+        CK(cudaEventCreateWithFlags(&L.fork, cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&L.join, cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&L.done, cudaEventDisableTiming));
+    }
     c->agents.resize(n);
     for (int i = 0; i < n; i++) {
         Agent& a = c->agents[i];
         CK(cudaStreamCreateWithFlags(&a.lib_stream, cudaStreamNonBlocking));
         a.stream = a.lib_stream;
-        CK(cudaEventCreateWithFlags(&a.pub_event[0], cudaEventDisableTiming));
-        CK(cudaEventCreateWithFlags(&a.pub_event[1], cudaEventDisableTiming));
-        CK(cudaEventCreateWithFlags(&a.sweep_done, cudaEventDisableTiming));
+        for (int s = 0; s < kSnapSlots; s++) CK(cudaEventCreateWithFlags(&a.pub_event[s], cudaEventDisableTiming));
         CK(cudaEventCreateWithFlags(&a.fence, cudaEventDisableTiming));
         a.consumed.assign(n, 0);
     }
     ALLOC(c->x, (size_t)n * dp); ALLOC(c->g, (size_t)n * dp); ALLOC(c->v, (size_t)n * dp);
-    ALLOC(c->snap, (size_t)n * 2 * dp);
+    ALLOC(c->snap, (size_t)n * kSnapSlots * dp);
     ALLOC(c->clip, n); ALLOC(c->norm, n); ALLOC(c->losses, (size_t)n * 4);
     ALLOC(c->norm_partial, (size_t)n * kNormChunks); ALLOC(c->norm_ticket, n);
     ALLOC(c->error_word, 1);
@@ -1276,12 +1435,18 @@ int gala_destroy(gala_ctx* c) {
     cudaDeviceSynchronize();
     for (Agent& a : c->agents) {
         if (a.lib_stream) cudaStreamDestroy(a.lib_stream);
-        for (int s = 0; s < 2; s++) if (a.pub_event[s]) cudaEventDestroy(a.pub_event[s]);
-        if (a.sweep_done) cudaEventDestroy(a.sweep_done);
+        for (int s = 0; s < kSnapSlots; s++) if (a.pub_event[s]) cudaEventDestroy(a.pub_event[s]);
         if (a.fence) cudaEventDestroy(a.fence);
     }
     for (StepGraph& g : c->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
     for (Agent& a : c->agents) if (a.loop_graph.exec) cudaGraphExecDestroy(a.loop_graph.exec);
+    for (gala_ctx::Lane& L : c->glane) {
+        if (L.st) cudaStreamDestroy(L.st);
+        if (L.side) cudaStreamDestroy(L.side);
+        if (L.fork) cudaEventDestroy(L.fork);
+        if (L.join) cudaEventDestroy(L.join);
+        if (L.done) cudaEventDestroy(L.done);
+    }
     if (c->side_stream) cudaStreamDestroy(c->side_stream);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
@@ -1300,8 +1465,10 @@ int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int
     Agent& ag = c->agents[agent];
     PtrBatch pb{};
     pb.p[0] = obs;
+    int r = own_stream_begin(c, ag);
+    if (r != GALA_OK) return r;
     c->cur_ctas = c->agent_ctas;
-    int r = forward(c, agent, 1, pb, c->E, ag.stream, c->legacy_conv ? ag.stream : nullptr);
+    r = forward(c, agent, 1, pb, c->E, ag.stream, c->legacy_conv ? ag.stream : nullptr);
     c->cur_ctas = 0;
     if (r != GALA_OK) return r;
     if (actions)
@@ -1365,6 +1532,10 @@ int gala_actor_loop(gala_ctx* c, int agent, int iterations, unsigned long long e
         ag.loop_seed = env_seed; ag.loop_seen = 0;
     }
     const unsigned long long outside = (1ull << T_SWEEP_SYNC) | (1ull << T_SWEEP_AGENT);
+    {
+        int r0 = own_stream_begin(c, ag);
+        if (r0 != GALA_OK) return r0;
+    }
     for (int it = 0; it < iterations; it++) {
         if (ag.pending) {  // a gradient that no gossip step has consumed: apply it without mixing, publish
             int r0 = sweep_agent(c, agent, false);
@@ -1417,7 +1588,7 @@ int gala_actor_read(gala_ctx* c, int agent, void* obs, int* actions, float* rewa
     if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_actor_read: bad agent");
     Agent& ag = c->agents[agent];
     if (!ag.loop_obs) return fail(c, GALA_ESTATE, "gala_actor_read: gala_actor_loop has not run for this agent");
-    CK(cudaStreamSynchronize(ag.stream));
+    { int r = settle_agent(c, agent); if (r != GALA_OK) return r; }
     const long obs_bytes = (c->conv ? kFramePix : (long)c->obs_dim * 4);
     const size_t TE = (size_t)c->T * c->E;
     if (obs) CK(cudaMemcpy(obs, ag.loop_obs, (size_t)(c->T + 1) * c->E * obs_bytes, cudaMemcpyDeviceToHost));
@@ -1437,8 +1608,10 @@ int gala_learn(gala_ctx* c, int agent, const gala_rollout* ro) {
         if (r != GALA_OK) return r;
         ag.round++;
     }
+    int r = own_stream_begin(c, ag);
+    if (r != GALA_OK) return r;
     c->cur_ctas = c->agent_ctas;
-    int r = learn_range_cached(c, agent, 1, ro, ag.stream);
+    r = learn_range_cached(c, agent, 1, ro, ag.stream);
     c->cur_ctas = 0;
     return r;
 }
@@ -1453,11 +1626,100 @@ int gala_gossip(gala_ctx* c, int agent) {
     return GALA_OK;
 }
 
+// A list of distinct, valid agents.
+static int check_agent_list(gala_ctx* c, const int* agents, int m, const char* who) {
+    if (!c) return GALA_EINVAL;
+    if (!agents || m < 0 || m > c->n) return fail(c, GALA_EINVAL, "%s: null list or more entries than agents", who);
+    bool seen[256] = {};
+    for (int k = 0; k < m; k++) {
+        if (!valid_agent(c, agents[k])) return fail(c, GALA_EINVAL, "%s: entry %d is not an agent", who, k);
+        if (seen[agents[k]]) return fail(c, GALA_EINVAL, "%s: agent %d is listed twice", who, agents[k]);
+        seen[agents[k]] = true;
+    }
+    return GALA_OK;
+}
+
+int gala_learn_many(gala_ctx* c, const int* agents, const gala_rollout* ros, int m) {
+    int r = check_agent_list(c, agents, m, "gala_learn_many");
+    if (r != GALA_OK) return r;
+    if (m == 0) return GALA_OK;
+    if (!ros) return fail(c, GALA_EINVAL, "gala_learn_many: null rollouts");
+    for (int k = 0; k < m; k++)
+        if (!ros[k].obs || !ros[k].actions || !ros[k].rewards || !ros[k].dones)
+            return fail(c, GALA_EINVAL, "gala_learn_many: null rollout pointer in entry %d", k);
+    // the grouped kernels are those of the conv net with the fused heads; everything else goes agent by agent
+    if (!c->conv || !c->fused_heads || c->legacy_conv) {
+        for (int k = 0; k < m; k++)
+            if ((r = gala_learn(c, agents[k], &ros[k])) != GALA_OK) return r;
+        return GALA_OK;
+    }
+    const int lane = c->next_lane;
+    c->next_lane = (c->next_lane + 1) % c->n_lanes;
+    gala_ctx::Lane& L = c->glane[lane];
+    if ((r = lane_acquire(c, lane, agents, m)) != GALA_OK) return r;
+    // gradients that no gossip step has consumed are applied without mixing and published first
+    std::vector<int> pend;
+    for (int k = 0; k < m; k++)
+        if (c->agents[agents[k]].pending) pend.push_back(agents[k]);
+    if (!pend.empty()) {
+        if ((r = sweep_group(c, lane, pend.data(), (int)pend.size(), false)) != GALA_OK) return r;
+        for (int i : pend) c->agents[i].round++;
+    }
+    // several kernel classes timed at once: one stream, so that an event pair brackets a kernel
+    const unsigned long long outside = (1ull << T_SWEEP_SYNC) | (1ull << T_SWEEP_AGENT) | (1ull << T_SAMPLE);
+    const unsigned long long inside = c->profile_mask & ~outside;
+    cudaStream_t side = (inside & (inside - 1)) != 0 ? nullptr : L.side;
+    c->cur_fork = L.fork; c->cur_join = L.join;
+    for (int k0 = 0; k0 < m && r == GALA_OK; k0 += kBatch) {
+        const int cnt = m - k0 < kBatch ? m - k0 : kBatch;
+        AgentMap am{};
+        am.on = 1;
+        for (int e = 0; e < cnt; e++) am.v[e] = (unsigned char)agents[k0 + e];
+        c->cur_map = &am;
+        r = learn_range(c, 0, cnt, ros + k0, L.st, side);
+        c->cur_map = nullptr;
+    }
+    c->cur_fork = c->ev_fork; c->cur_join = c->ev_join;
+    const int r2 = lane_release(c, lane, agents, m);
+    return r != GALA_OK ? r : r2;
+}
+
+int gala_gossip_many(gala_ctx* c, const int* agents, int m) {
+    int r = check_agent_list(c, agents, m, "gala_gossip_many");
+    if (r != GALA_OK) return r;
+    if (m == 0) return GALA_OK;
+    if (c->topo.kind == GALA_TOPO_COMPLETE)
+        return fail(c, GALA_ESTATE, "gala_gossip_many: the complete graph (gradient all-reduce) exists only as gala_step_sync");
+    // the lane of the learner steps these agents' gradients come from, so that nothing waits across lanes
+    const int last = c->agents[agents[0]].group_lane;
+    const int lane = last >= 0 ? last : c->next_lane;
+    if ((r = lane_acquire(c, lane, agents, m)) != GALA_OK) return r;
+    if ((r = sweep_group(c, lane, agents, m, true)) != GALA_OK) return r;
+    for (int k = 0; k < m; k++) c->agents[agents[k]].round++;
+    return lane_release(c, lane, agents, m);
+}
+
+int gala_poll_agent(gala_ctx* c, int agent, int* busy) {
+    if (!valid_agent(c, agent) || !busy) return fail(c, GALA_EINVAL, "gala_poll_agent: bad agent or null output");
+    Agent& ag = c->agents[agent];
+    *busy = 0;
+    cudaError_t e = ag.version > 0 ? cudaEventQuery(ag.pub_event[ag.version % kSnapSlots]) : cudaSuccess;
+    if (e == cudaSuccess && (ag.pending || ag.dirty)) {   // work after the last optimiser step: ask the streams
+        if (ag.group_lane >= 0) e = cudaStreamQuery(c->glane[ag.group_lane].st);
+        if (e == cudaSuccess) e = cudaStreamQuery(ag.stream);
+    }
+    if (e == cudaErrorNotReady) { *busy = 1; return GALA_OK; }
+    if (e != cudaSuccess) return fail(c, GALA_ECUDA, "gala_poll_agent: %s", cudaGetErrorString(e));
+    return GALA_OK;
+}
+
 int gala_delay(gala_ctx* c, int agent, int usec) {
     if (!valid_agent(c, agent) || usec < 0 || usec > 100000)
         return fail(c, GALA_EINVAL, "gala_delay: bad agent or delay outside 0..100000 us");
     if (usec == 0) return GALA_OK;
     Agent& ag = c->agents[agent];
+    int r = own_stream_begin(c, ag);
+    if (r != GALA_OK) return r;
     CK(launch_delay((unsigned long long)usec, ag.stream));
     return GALA_OK;
 }
@@ -1471,8 +1733,13 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
                 return fail(c, GALA_EINVAL, "gala_step_sync: null rollout pointer for agent %d", i);
     cudaStream_t st = c->main_stream;
     for (int i = 0; i < n; i++) {  // everything the agents have enqueued goes first
-        CK(cudaEventRecord(c->agents[i].fence, c->agents[i].stream));
-        CK(cudaStreamWaitEvent(st, c->agents[i].fence, 0));
+        Agent& ag = c->agents[i];
+        if (ag.group_lane >= 0) {      // ... also on the lanes of the grouped calls
+            CK(cudaStreamWaitEvent(st, c->glane[ag.group_lane].done, 0));
+            ag.group_lane = -1;
+        }
+        CK(cudaEventRecord(ag.fence, ag.stream));
+        CK(cudaStreamWaitEvent(st, ag.fence, 0));
     }
     if (ros) {
         // Timing several kernel classes of the step at once: one stream, so that an event pair brackets a kernel
@@ -1507,6 +1774,7 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
     CK(cudaEventRecord(c->main_event, st));
     for (int i = 0; i < n; i++) {
         CK(cudaStreamWaitEvent(c->agents[i].stream, c->main_event, 0));
+        c->agents[i].dirty = true;     // a grouped call must be ordered behind this round through the agent's stream
         c->agents[i].pending = false;
         c->agents[i].round++;
     }
@@ -1516,8 +1784,10 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
 
 int gala_sync_agent(gala_ctx* c, int agent, int timeout_ms) {
     if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_sync_agent: bad agent");
-    int r = host_wait(c, c->agents[agent].stream, timeout_ms);
+    Agent& ag = c->agents[agent];
+    int r = ag.group_lane >= 0 ? host_wait(c, c->glane[ag.group_lane].st, timeout_ms) : GALA_OK;
     if (r != GALA_OK) return r;
+    if ((r = host_wait(c, ag.stream, timeout_ms)) != GALA_OK) return r;
     return check_error_word(c);
 }
 
@@ -1525,6 +1795,8 @@ int gala_sync_all(gala_ctx* c, int timeout_ms) {
     if (!c) return GALA_EINVAL;
     int r = host_wait(c, c->main_stream, timeout_ms);
     if (r != GALA_OK) return r;
+    for (gala_ctx::Lane& L : c->glane)
+        if ((r = host_wait(c, L.st, timeout_ms)) != GALA_OK) return r;
     for (int i = 0; i < c->n; i++)
         if ((r = host_wait(c, c->agents[i].stream, timeout_ms)) != GALA_OK) return r;
     return check_error_word(c);
@@ -1541,8 +1813,7 @@ int gala_in_peers(const gala_ctx* c, long long round, int agent, int* peers, int
 
 int gala_get_state(gala_ctx* c, int agent, float* params, float* sq_avg, float* grad, long long* round) {
     if (!valid_agent(c, agent)) return fail(c, GALA_EINVAL, "gala_get_state: bad agent");
-    CK(cudaStreamSynchronize(c->main_stream));
-    CK(cudaStreamSynchronize(c->agents[agent].stream));
+    { int r = settle_agent(c, agent); if (r != GALA_OK) return r; }
     const size_t bytes = (size_t)c->d * sizeof(float);
     if (params) CK(cudaMemcpy(params, c->x + (long)agent * c->d_pad, bytes, cudaMemcpyDefault));
     if (sq_avg) CK(cudaMemcpy(sq_avg, c->v + (long)agent * c->d_pad, bytes, cudaMemcpyDefault));
@@ -1554,8 +1825,7 @@ int gala_get_state(gala_ctx* c, int agent, float* params, float* sq_avg, float* 
 int gala_set_state(gala_ctx* c, int agent, const float* params, const float* sq_avg, long long round) {
     if (!valid_agent(c, agent) || round < 0) return fail(c, GALA_EINVAL, "gala_set_state: bad agent or round");
     Agent& ag = c->agents[agent];
-    CK(cudaStreamSynchronize(c->main_stream));
-    CK(cudaStreamSynchronize(ag.stream));
+    { int r = settle_agent(c, agent); if (r != GALA_OK) return r; }
     const size_t bytes = (size_t)c->d * sizeof(float);
     if (params) {
         int r = copy_in(c, c->x + (long)agent * c->d_pad, params, bytes, ag.stream);
@@ -1577,9 +1847,9 @@ int gala_set_state(gala_ctx* c, int agent, const float* params, const float* sq_
 int gala_set_grad(gala_ctx* c, int agent, const float* grad, float clip_coef) {
     if (!valid_agent(c, agent) || !grad) return fail(c, GALA_EINVAL, "gala_set_grad: bad agent or null gradient");
     Agent& ag = c->agents[agent];
-    CK(cudaStreamSynchronize(c->main_stream));
-    CK(cudaStreamSynchronize(ag.stream));
-    int r = copy_in(c, c->g + (long)agent * c->d_pad, grad, (size_t)c->d * sizeof(float), ag.stream);
+    int r = settle_agent(c, agent);
+    if (r != GALA_OK) return r;
+    r = copy_in(c, c->g + (long)agent * c->d_pad, grad, (size_t)c->d * sizeof(float), ag.stream);
     if (r != GALA_OK) return r;
     if (clip_coef >= 0.0f) {
         if ((r = copy_in(c, c->clip + agent, &clip_coef, sizeof(float), ag.stream)) != GALA_OK) return r;
@@ -1630,6 +1900,13 @@ int gala_set_graphs(gala_ctx* c, int on) {
     return GALA_OK;
 }
 
+int gala_set_group_lanes(gala_ctx* c, int lanes) {
+    if (!c || lanes < 1 || lanes > 2) return fail(c, GALA_EINVAL, "gala_set_group_lanes: 1 or 2");
+    c->n_lanes = lanes;
+    c->next_lane = 0;
+    return GALA_OK;
+}
+
 int gala_set_agent_ctas(gala_ctx* c, int ctas) {
     if (!c || ctas < 0) return fail(c, GALA_EINVAL, "gala_set_agent_ctas: negative budget");
     c->agent_ctas = ctas >= 148 ? 0 : ctas;
@@ -1651,8 +1928,7 @@ int gala_param_count(const gala_ctx* c, long long* d, long long* d_padded) {
 
 int gala_losses(gala_ctx* c, int agent, float out[4]) {
     if (!valid_agent(c, agent) || !out) return fail(c, GALA_EINVAL, "gala_losses: bad argument");
-    CK(cudaStreamSynchronize(c->main_stream));
-    CK(cudaStreamSynchronize(c->agents[agent].stream));
+    { int r = settle_agent(c, agent); if (r != GALA_OK) return r; }
     CK(cudaMemcpy(out, c->losses + (long)agent * 4, 3 * sizeof(float), cudaMemcpyDeviceToHost));
     CK(cudaMemcpy(out + 3, c->norm + agent, sizeof(float), cudaMemcpyDeviceToHost));
     return GALA_OK;
@@ -1661,6 +1937,7 @@ int gala_losses(gala_ctx* c, int agent, float out[4]) {
 int gala_losses_all(gala_ctx* c, float* out) {
     if (!c || !out) return fail(c, GALA_EINVAL, "gala_losses_all: bad argument");
     CK(cudaStreamSynchronize(c->main_stream));
+    for (gala_ctx::Lane& L : c->glane) CK(cudaStreamSynchronize(L.st));
     for (Agent& a : c->agents) CK(cudaStreamSynchronize(a.stream));
     std::vector<float> nrm(c->n);
     CK(cudaMemcpy(out, c->losses, (size_t)c->n * 4 * sizeof(float), cudaMemcpyDeviceToHost));
@@ -1695,8 +1972,8 @@ int gala_get_snapshot(gala_ctx* c, int agent, long long version, float* out) {
     if (version < 1 || version > a.version || version < a.version - 1)
         return fail(c, GALA_ESTATE, "snapshot version %lld of agent %d is not held (newest %lld)", version, agent,
                     a.version);
-    CK(cudaStreamSynchronize(a.stream));
-    CK(cudaMemcpy(out, c->snap + ((long)agent * 2 + (version & 1)) * c->d_pad, (size_t)c->d * sizeof(float),
+    { int r = settle_agent(c, agent); if (r != GALA_OK) return r; }
+    CK(cudaMemcpy(out, c->snap + ((long)agent * kSnapSlots + version % kSnapSlots) * c->d_pad, (size_t)c->d * sizeof(float),
                   cudaMemcpyDefault));
     return GALA_OK;
 }
@@ -1704,15 +1981,14 @@ int gala_get_snapshot(gala_ctx* c, int agent, long long version, float* out) {
 int gala_set_stream(gala_ctx* c, int agent, void* cuda_stream) {
     if (!valid_agent(c, agent)) return GALA_EINVAL;
     Agent& a = c->agents[agent];
-    CK(cudaStreamSynchronize(a.stream));
+    { int r = settle_agent(c, agent); if (r != GALA_OK) return r; }
     a.stream = cuda_stream ? reinterpret_cast<cudaStream_t>(cuda_stream) : a.lib_stream;
     return GALA_OK;
 }
 
 int gala_debug_read(gala_ctx* c, int agent, int what, float* out, long long count) {
     if (!valid_agent(c, agent) || !out || count < 0) return fail(c, GALA_EINVAL, "gala_debug_read: bad argument");
-    CK(cudaStreamSynchronize(c->main_stream));
-    CK(cudaStreamSynchronize(c->agents[agent].stream));
+    { int r = settle_agent(c, agent); if (r != GALA_OK) return r; }
     const long B = c->B, S = c->S;
     const int A = c->A;
     const float* src = nullptr;
@@ -1855,6 +2131,45 @@ int gala_sweep_sync(float* x, const float* g, float* v, const float* clip, int n
     cudaError_t e = launch_sweep_sync(x, g, v, clip, nullptr, n_agents, d_padded, np, off, s, nullptr,
                                       reinterpret_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? GALA_OK : GALA_ECUDA;
+}
+
+int gala_sweep_agents(float* x, const float* g, float* v, float* snap, const float* clip, int n_agents, int n_slots,
+                      long long d_padded, const gala_sweep_item* items, int n_items, const gala_hparams* hp, void* stream) {
+    if (!x || !v || !snap || !items || !hp || n_agents < 1 || n_slots < 1 || n_items < 0 || d_padded < 4 || (d_padded % 4))
+        return GALA_EINVAL;
+    if ((long long)n_agents * n_slots > 0x7fffffffLL) return GALA_EINVAL;
+    std::vector<char> written((size_t)n_agents * n_slots, 0), listed((size_t)n_agents, 0);
+    for (int k = 0; k < n_items; k++) {
+        const gala_sweep_item& it = items[k];
+        if (it.agent < 0 || it.agent >= n_agents || listed[it.agent] || it.out_slot < 0 || it.out_slot >= n_slots ||
+            it.n_peers < 0 || it.n_peers > 2 || (it.has_grad && !g))
+            return GALA_EINVAL;
+        listed[it.agent] = 1;
+        written[(size_t)it.agent * n_slots + it.out_slot] = 1;
+    }
+    for (int k = 0; k < n_items; k++)
+        for (int j = 0; j < items[k].n_peers; j++) {
+            const gala_sweep_item& it = items[k];
+            if (it.peer[j] < 0 || it.peer[j] >= n_agents || it.peer_slot[j] < 0 || it.peer_slot[j] >= n_slots) return GALA_EINVAL;
+            if (written[(size_t)it.peer[j] * n_slots + it.peer_slot[j]]) return GALA_EINVAL;   // read and written in one call
+        }
+    for (int k0 = 0; k0 < n_items; k0 += kBatch) {
+        const int cnt = n_items - k0 < kBatch ? n_items - k0 : kBatch;
+        SweepManyArgs a{};
+        a.x = x; a.g = g; a.v = v; a.snap = snap; a.clip = clip; a.d_pad = d_padded;
+        a.hp = SweepHp{hp->lr, hp->rms_alpha, hp->rms_eps};
+        a.n_items = cnt;
+        for (int e = 0; e < cnt; e++) {
+            const gala_sweep_item& it = items[k0 + e];
+            a.it[e].x_row = it.agent;
+            a.it[e].out_row = it.agent * n_slots + it.out_slot;
+            a.it[e].p_row[0] = it.n_peers > 0 ? it.peer[0] * n_slots + it.peer_slot[0] : -1;
+            a.it[e].p_row[1] = it.n_peers > 1 ? it.peer[1] * n_slots + it.peer_slot[1] : -1;
+            if (it.has_grad) a.has_grad[e >> 5] |= 1u << (e & 31);
+        }
+        if (launch_sweep_many(a, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return GALA_ECUDA;
+    }
+    return GALA_OK;
 }
 
 }  // extern "C"

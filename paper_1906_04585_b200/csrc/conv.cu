@@ -189,7 +189,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             __syncwarp();
             if (lane == 0) { mbar_expect_tx(&w_full, (uint32_t)W_BYTES); issued_w = 1; }
             __syncwarp();
-            const int group = p.group0 + decode_unit<V>(u_begin, p.rows).gz;
+            const int group = p.group0 + agent_slot(p.am, decode_unit<V>(u_begin, p.rows).gz);
             if (lane < T::W_BOXES) tma_load_3d(smW + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
         }
     };
@@ -214,7 +214,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         int cur_g = u_begin < u_end ? decode_unit<V>(u_begin, p.rows).gz : -1;   // already on its way
         for (int u = u_begin; u < u_end; u++, it++) {
             const UnitCoord c = decode_unit<V>(u, p.rows);
-            const int group = p.group0 + c.gz;
+            const int group = p.group0 + agent_slot(p.am, c.gz);
             if (c.gz != cur_g) {
                 // new agent: its weights replace the previous agent's once both issuers have signalled that
                 // every MMA that read those is done
@@ -389,7 +389,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 for (int ch = 0; ch < NCH; ch++) g[ch] = 0u;
                 if (u < u_end && in_tile) {
                     const UnitCoord c = decode_unit<V>(u, p.rows);
-                    const uint32_t* gp = p.gate_in + (long)c.gz * p.gate_group_stride + pixel_off(c) / 32;
+                    const uint32_t* gp = p.gate_in + (long)agent_slot(p.am, c.gz) * p.gate_group_stride + pixel_off(c) / 32;
                     if constexpr (V == CV_CONV2_DGRAD) {   // words of pixels (2a, 2b), (2a, 2b+1), (2a+1, 2b), (2a+1, 2b+1)
                         const uint2 g0 = __ldg(reinterpret_cast<const uint2*>(gp));
                         const uint2 g1 = __ldg(reinterpret_cast<const uint2*>(gp + 20));
@@ -418,7 +418,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if constexpr (kBias) {
                 for (; bg < upto; bg++) {
                     const float sum = warp_reduce_scatter32(bacc, lane);
-                    p.bias_partial[(((long)bg * kConvMaxGrid + blockIdx.x) * 8 + (warp - 2)) * 32 + lane] = sum;
+                    p.bias_partial[(((long)agent_slot(p.am, bg) * kConvMaxGrid + blockIdx.x) * 8 + (warp - 2)) * 32 + lane] = sum;
 #pragma unroll
                     for (int j = 0; j < 32; j++) bacc[j] = 0.0f;
                 }
@@ -432,7 +432,8 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const int L = kC1Lines * c.s + pa;
                 valid = in_tile && L % 21 < 20 && L < 21 * p.rows;
             }
-            __nv_bfloat16* out = p.out + (long)c.gz * p.out_group_stride + off;
+            const int slot = agent_slot(p.am, c.gz);
+            __nv_bfloat16* out = p.out + (long)slot * p.out_group_stride + off;
             // column block c0 -> where it goes: forward, conv3 gradient: channels c0.. of the pixel; conv2
             // gradient: block = parity class (py, px) -> pixel (2a + py, 2b + px), all 32 channels
             auto block_add = [](int c0) -> int {
@@ -443,7 +444,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if (bias_on && c.gz != bg) bias_flush(c.gz);
             if constexpr (kFwd) {
                 if (c.gz != cur_g) {
-                    const float* bias = p.bias + (long)(p.group0 + c.gz) * p.bias_group_stride;
+                    const float* bias = p.bias + (long)(p.group0 + slot) * p.bias_group_stride;
                     __syncwarp();
                     for (int j = lane; j < T::BN; j += 32) sbias[j] = __ldg(bias + j);
                     __syncwarp();
@@ -492,7 +493,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     if (valid) {   // a 32-byte store fills a whole sector
                         st_global_v8(out + block_add(ch * 32) + 16 * h, o);
                         if constexpr (kFwd) {
-                            if (h == 1 && p.gate_out) p.gate_out[(long)c.gz * p.gate_group_stride + off / 32 + ch] = bits;
+                            if (h == 1 && p.gate_out) p.gate_out[(long)slot * p.gate_group_stride + off / 32 + ch] = bits;
                         }
                     }
                     if (h == 1) bits = 0u;

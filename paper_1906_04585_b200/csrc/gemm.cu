@@ -125,7 +125,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         bool ok = true;
         for (long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             const TileCoord t = decode_tile(p, tile, mt, nt);
-            const int group = p.group0 + t.gz;
+            const int group = p.group0 + agent_slot(p.am, t.gz);
             for (int k = 0; k < t.num_k; k++, it++) {
                 const int s = it % nst;
                 const uint32_t ph = (uint32_t)(it / nst) & 1u;
@@ -309,7 +309,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (p.flags & EPI_GATE) {
                 const int m = t.m0 + q * 32 + lane;
                 if (m < p.M) {
-                    const uint32_t* gp = p.gate + (long)t.gz * p.gate_group_stride + (long)m * (p.N >> 5) + (t.n0 >> 5);
+                    const uint32_t* gp = p.gate + (long)agent_slot(p.am, t.gz) * p.gate_group_stride + (long)m * (p.N >> 5) + (t.n0 >> 5);
                     const int nw = (p.N - t.n0) >> 5;
                     if (nw > 0) gw0 = __ldg(gp);
                     if (nw > 1 && BN > 32) gw1 = __ldg(gp + 1);
@@ -320,10 +320,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (!mbar_wait(&acc_full[ab], ((uint32_t)local >> 1) & 1u, &abort_flag)) break;
             tcgen05_fence_after();
             const uint32_t tmem_acc = tmem_base + (uint32_t)ab * acc_cols;
-            const int group = p.group0 + t.gz;
-            const long obase = (long)t.gz * p.out_group_stride + (long)t.split * p.out_split_stride;
+            const int slot = agent_slot(p.am, t.gz);
+            const int group = p.group0 + slot;
+            const long obase = (long)slot * p.out_group_stride + (long)t.split * p.out_split_stride;
+            // block sums of squares are kept per agent: the tile index as it would be in a launch over all agents
+            const long sq_tile = tile + (long)(slot - t.gz) * mt * nt;
             const float* bias = p.bias ? p.bias + (long)group * p.bias_group_stride : nullptr;
-            const __nv_bfloat16* mask = use_mask ? p.mask + (long)t.gz * p.mask_group_stride : nullptr;
+            const __nv_bfloat16* mask = use_mask ? p.mask + (long)slot * p.mask_group_stride : nullptr;
             const int mw = t.m0 + q * 32;   // first row of this warp
             const bool rowmap = p.flags & EPI_ROWMAP_S2;
             // element offset (inside the group) of output row r of this tile
@@ -349,7 +352,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
                 const int nb = t.n0 + c0;
                 if (mw >= p.M || q * 32 >= p.tile_rows || nb >= p.N) {   // warp-uniform
-                    if (p.sq_partial && lane == 0) p.sq_partial[tile * 16 + q * 4 + (c0 >> 5)] = 0.0f;
+                    if (p.sq_partial && lane == 0) p.sq_partial[sq_tile * 16 + q * 4 + (c0 >> 5)] = 0.0f;
                     continue;
                 }
                 if (transpose) {
@@ -424,7 +427,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     }
                     if (p.sq_partial) {   // rows of the block added by a butterfly: the same tree every time
                         for (int o = 16; o > 0; o >>= 1) row_sq += __shfl_xor_sync(0xffffffffu, row_sq, o);
-                        if (lane == 0) p.sq_partial[tile * 16 + q * 4 + (c0 >> 5)] = row_sq;
+                        if (lane == 0) p.sq_partial[sq_tile * 16 + q * 4 + (c0 >> 5)] = row_sq;
                     }
                     continue;
                 }
@@ -587,10 +590,10 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
 // Up to six such reductions in one launch (the conv weight and bias gradients of a step), 16 bytes per thread.
 __global__ void __launch_bounds__(256) splitk_reduce_multi_kernel(const float* __restrict__ ws, float* __restrict__ out,
                                                                   ReduceSegs sg, long total4, long ws_group_stride,
-                                                                  long out_group_stride) {
+                                                                  long out_group_stride, AgentMap am) {
     pdl_wait();
     pdl_launch();
-    const int g = blockIdx.y;
+    const int g = agent_slot(am, blockIdx.y);
     const float* wg = ws + (long)g * ws_group_stride;
     float* og = out + (long)g * out_group_stride;
     for (long j = blockIdx.x * (long)blockDim.x + threadIdx.x; j < total4; j += (long)gridDim.x * blockDim.x) {
@@ -614,7 +617,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_multi_kernel(const float* _
     }
 }
 cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const ReduceSegs& segs, int groups,
-                                       long ws_group_stride, long out_group_stride, cudaStream_t st) {
+                                       long ws_group_stride, long out_group_stride, cudaStream_t st, const AgentMap* am) {
     if (segs.n < 1 || segs.n > 6 || ((ws_group_stride | out_group_stride) & 3)) return cudaErrorInvalidValue;
     long total4 = 0;
     for (int k = 0; k < segs.n; k++) {
@@ -625,7 +628,7 @@ cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const Reduce
     int bx = (int)((total4 + 255) / 256);
     if (bx > 148 * 4) bx = 148 * 4;
     (void)launch_pdl(splitk_reduce_multi_kernel, dim3(bx, groups), dim3(256), 0, st, ws, out, segs, total4, ws_group_stride,
-                     out_group_stride);
+                     out_group_stride, am ? *am : AgentMap{});
     return cudaGetLastError();
 }
 
@@ -684,14 +687,26 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 static EncodeTiledFn g_encode = nullptr;
 
 cudaError_t gemm_init() {
-    if (g_encode) return cudaSuccess;
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (e != cudaSuccess) return e;
-    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
-    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-    return cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e;
+    if (!g_encode) {   // once per process
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    // the opt-in to large dynamic shared memory is a property of the function on ONE device: once per device
+    static bool attr_done[64] = {};
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_done[dev]) {
+        if ((e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess)
+            return e;
+        attr_done[dev] = true;
+    }
+    return cudaSuccess;
 }
 
 bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t groups,

@@ -57,6 +57,20 @@ constexpr int kConvOut[3] = {20, 9, 7};    // output height = width
 constexpr int kConvKK[3] = {256, 512, 576};  // k*k*cin
 constexpr int kFeat = 3136, kHidden = 512;
 
+// Caller-owned per-agent pointers travel in kernel parameters, at most kBatch agents a launch.
+constexpr int kBatch = 64;
+struct PtrBatch { const void* p[kBatch]; };
+
+// Which agents a launch works on.  Group gz of a launch (0 .. groups - 1) addresses the per-agent tensors of the
+// library (parameters, gradients, workspaces) as agent slot(gz): gz itself for the consecutive agents
+// [agent0, agent0 + groups) - every base pointer is then already moved to agent0 - or entry gz of a list of agent
+// indices (base pointers are agent 0's).  Pointers that come with the launch (PtrBatch) are always indexed by gz.
+struct AgentMap {
+    int on;
+    unsigned char v[kBatch];
+};
+__host__ __device__ __forceinline__ int agent_slot(const AgentMap& m, int gz) { return m.on ? (int)m.v[gz] : gz; }
+
 // ---------------------------------------------------------------- GEMM
 // One operand of the grouped tensor-core GEMM, as a TMA descriptor plus what
 // the kernel must know about its shared-memory image.
@@ -96,6 +110,7 @@ struct GemmArgs {
     long gate_group_stride;
     int* error_word;       // device int, set non-zero when a bounded wait runs out
     int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
+    AgentMap am;           // agents behind the groups (operands, outputs, bias, mask, gate, sq_partial)
     // Optional sums of squares of the stored outputs (for a gradient norm without a second pass over this
     // product): slot [tile * 16 + warp quarter * 4 + 32-column block] of sq_partial gets the sum over that
     // 32 x 32 block (0 where the block lies outside the matrix).  Needs block_n = 128, split_k = 1, fp32 row-major
@@ -158,11 +173,8 @@ cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, 
 struct ReduceSeg { long out_off, count, ws_off; int split; };
 struct ReduceSegs { ReduceSeg s[6]; int n; };
 cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const ReduceSegs& segs, int groups,
-                                       long ws_group_stride, long out_group_stride, cudaStream_t st);
-
-// Caller-owned per-agent pointers travel in kernel parameters, at most kBatch agents a launch.
-constexpr int kBatch = 64;
-struct PtrBatch { const void* p[kBatch]; };
+                                       long ws_group_stride, long out_group_stride, cudaStream_t st,
+                                       const AgentMap* am = nullptr);
 
 // ---------------------------------------------------------------- convolutions with a resident input
 // Forward and data-gradient convolutions of the trunk (conv.cu).  Tensors are NHWC bf16; weights
@@ -186,6 +198,7 @@ struct ConvArgs {
     long gate_group_stride;      // words per agent
     int* error_word;
     int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
+    AgentMap am;           // agents behind the groups
     PtrBatch obs;          // conv1 forward: the agents' uint8 frames [rows][84][84][4], 16-byte aligned
     // conv2 data gradient (may be null): per-channel sums over the pixels of the result, as slices
     // [agent of the launch][kConvMaxGrid CTAs][8 warps][32 channels].  CTA b (of `grid`) works on samples
@@ -217,6 +230,7 @@ struct WgradArgs {
     float* bias_out;
     long bias_group_stride, bias_split_stride;
     int* error_word;
+    AgentMap am;           // agents behind the groups
 };
 cudaError_t wgrad_init();
 bool make_wgrad_maps(int variant, CUtensorMap* x_map, CUtensorMap* y_map, const void* x_base, uint64_t x_samples,
@@ -233,6 +247,7 @@ struct Wgrad1Args {
     float* out;            // agent i, slice s at out + i * out_group_stride + s * out_split_stride, as W[32][256]
     long out_group_stride, out_split_stride;
     int* error_word;
+    AgentMap am;           // agents behind the groups
     PtrBatch obs;          // the agents' uint8 frames [..][84][84][4], 16-byte aligned
 };
 cudaError_t wgrad1_init();
@@ -247,6 +262,28 @@ struct SweepHp {
 cudaError_t launch_sweep_agent(float* x, const float* g, float* v, float* snap_out, const float* peer0,
                                const float* peer1, int n_peers, const float* clip, __nv_bfloat16* shadow,
                                long d_pad, SweepHp hp, cudaStream_t st);
+// Per-agent form for up to kBatch agents in one launch (sweep_many.cu).  Rows are indices into row-major arrays of
+// d_pad floats: x_row into x, g, v, clip and shadow (the agent), out_row and p_row into `snap` (agent * slots + slot).
+// No out_row of a launch may equal a p_row of the same launch.
+struct SweepItem {
+    int x_row;
+    int out_row;      // where y, the agent's new snapshot, goes
+    int p_row[2];     // snapshots averaged with y (-1: none; p_row[1] only with p_row[0])
+};
+struct SweepManyArgs {
+    float* x; const float* g; float* v; float* snap;
+    __nv_bfloat16* shadow;      // optional bf16 copy of the new x
+    const float* clip;          // per agent, or null (= 1)
+    long d_pad;
+    SweepHp hp;
+    int* error_word;
+    int n_items;
+    int max_ctas;               // > 0: at most this many CTAs
+    int rows, cols, stages;     // set by the launcher
+    unsigned has_grad[kBatch / 32];   // bit e: item e applies a pending gradient (else y = x, v untouched)
+    SweepItem it[kBatch];
+};
+cudaError_t launch_sweep_many(const SweepManyArgs& a, cudaStream_t st);
 // Synchronous all-agent form.  peer_off[j]: in-peer j of agent i is (i - peer_off[j]) mod n.
 cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* clip,
                               __nv_bfloat16* shadow, int n_agents, long d_pad, int n_peers,
@@ -263,7 +300,7 @@ constexpr int kNormChunks = 128;
 struct NormKnown { long off, count; const float* partial; long n_partials, partial_group_stride; };
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
                              double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st,
-                             const NormKnown* known = nullptr);
+                             const NormKnown* known = nullptr, const AgentMap* am = nullptr);
 cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStream_t st);
 // partial: 592 doubles, ticket: one zeroed unsigned, out: one double (squared distance)
 // ||alpha G||_F^2 of the coming optimiser pass (see update_norm_kernel).  partial: [n_agents][kUpdateNormChunks]
@@ -325,6 +362,7 @@ struct HeadsBwdArgs {
     const float* dzv;                            // optional [g][S][20]: rows (dlogits, dvalue, zeros), 16-byte aligned
     float* grad; long g_stride;                  // flat gradient (same offsets)
     void* dpre; long dpre_stride; int dpre_bf16; // [g][S][H] dL/d(pre-activation of hidden)
+    AgentMap am;                                 // agents behind the groups (tiled weight-gradient kernel only)
 };
 // data part (dpre) and parameter part (gradients of the head weights and biases): independent of each other
 cudaError_t launch_heads_dgrad(const HeadsBwdArgs& a, int groups, cudaStream_t st);
@@ -354,6 +392,7 @@ struct HeadsFusedArgs {
     __nv_bfloat16* dh; long dh_stride;    // [g][S][512]
     float* loss_partial;                  // [g][E][4] scratch
     unsigned* ticket;                     // [g], zero before the first launch
+    AgentMap am;                          // agents behind the groups
 };
 bool heads_fused_supported(int T, int E, int A, int H);
 int heads_fused_blocks(int T, int E, int groups);   // blocks per agent of a launch with `groups` agents
@@ -422,7 +461,8 @@ struct ColsumJobs { ColsumJob j[kColsumJobs]; };
 // into out_base[g*out_group_stride + out_off + 0..31].
 struct ColsumSlices { const float* partial; long out_off; int grid, rows; };
 cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, long out_group_stride, double* partial,
-                          unsigned* ticket, int groups, cudaStream_t st, const ColsumSlices* slices = nullptr);
+                          unsigned* ticket, int groups, cudaStream_t st, const ColsumSlices* slices = nullptr,
+                          const AgentMap* am = nullptr);
 constexpr int kColsumChunks = 64;
 
 }  // namespace gala

@@ -47,17 +47,18 @@ cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out
 // Up to kColsumJobs tensors are reduced by one launch (blockIdx.z picks the tensor).
 __global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, int n_jobs, ColsumSlices sl,
                                                      float* __restrict__ out_base, long out_group_stride,
-                                                     double* partial_base, unsigned* ticket_base) {
+                                                     double* partial_base, unsigned* ticket_base, AgentMap am) {
     pdl_wait();
     pdl_launch();
-    const int g = blockIdx.y;
+    const int gz = blockIdx.y;            // position in the launch
+    const int g = agent_slot(am, gz);     // agent whose tensors are addressed
     __shared__ float red[256 * 8];
     if ((int)blockIdx.z == n_jobs) {
         // Bias slices of a conv2 data-gradient launch: CTA b of sl.grid worked on samples
         // [total * b / grid, total * (b + 1) / grid); those whose range meets agent g's samples left 8 warp slices
         // of 32 channels each.  Thread (w, c) adds slice w of the CTAs in order, then the 8 sums are added in order.
         if (blockIdx.x != 0) return;
-        const long total = (long)gridDim.y * sl.rows, lo = (long)g * sl.rows, hi = lo + sl.rows;
+        const long total = (long)gridDim.y * sl.rows, lo = (long)gz * sl.rows, hi = lo + sl.rows;
         int b_lo = (int)(lo * sl.grid / total);
         while (b_lo > 0 && total * b_lo / sl.grid > lo) b_lo--;
         while (total * (b_lo + 1) / sl.grid <= lo) b_lo++;
@@ -146,7 +147,7 @@ __global__ void __launch_bounds__(256) colsum_kernel(ColsumJobs jobs, int n_jobs
     }
 }
 cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, long out_group_stride, double* partial,
-                          unsigned* ticket, int groups, cudaStream_t st, const ColsumSlices* slices) {
+                          unsigned* ticket, int groups, cudaStream_t st, const ColsumSlices* slices, const AgentMap* am) {
     if (n_jobs < 1 || n_jobs > kColsumJobs) return cudaErrorInvalidValue;
     ColsumSlices sl{};
     if (slices) {
@@ -158,7 +159,7 @@ cudaError_t launch_colsum(const ColsumJobs& jobs, int n_jobs, float* out_base, l
         if (C > 512 || C < 8 || (C & (C - 1))) return cudaErrorInvalidValue;
     }
     (void)launch_pdl(colsum_kernel, dim3(kColsumChunks, groups, n_jobs + (slices ? 1 : 0)), dim3(256), 0, st, jobs, n_jobs, sl,
-                     out_base, out_group_stride, partial, ticket);
+                     out_base, out_group_stride, partial, ticket, am ? *am : AgentMap{});
     return cudaGetLastError();
 }
 

@@ -70,11 +70,11 @@ extern "C" int gala_gemm_bf16_static(const void* A, const void* B, float* D, int
             say(errbuf, errbuf_len, "gala_gemm_bf16_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
             return GALA_ECUDA;
         }
-        if (gemm_init() != cudaSuccess) {
-            say(errbuf, errbuf_len, "gala_gemm_bf16_static: tensor-map encoder not available from the driver");
-            return GALA_ECUDA;
-        }
         g_scratch_addr[dev] = p;
+    }
+    if (gemm_init() != cudaSuccess) {   // encoder once per process, shared-memory opt-in once per device
+        say(errbuf, errbuf_len, "gala_gemm_bf16_static: tensor-map encoder not available from the driver");
+        return GALA_ECUDA;
     }
     float* scratch = g_scratch_addr[dev];
     int* err = reinterpret_cast<int*>(scratch);
@@ -111,12 +111,10 @@ extern "C" int gala_gemm_bf16_static(const void* A, const void* B, float* D, int
         say(errbuf, errbuf_len, "gala_gemm_bf16_static: launch failed: %s", cudaGetErrorString(e));
         return GALA_ECUDA;
     }
-    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) {
-        say(errbuf, errbuf_len, "gala_gemm_bf16_static: %s", cudaGetErrorString(e));
-        return GALA_ECUDA;
-    }
+    // the error word comes back on the caller's stream, so that the one wait below is for this call's work only
     int w = 0;
-    if ((e = cudaMemcpy(&w, err, sizeof w, cudaMemcpyDeviceToHost)) != cudaSuccess || w) {
+    if ((e = cudaMemcpyAsync(&w, err, sizeof w, cudaMemcpyDeviceToHost, st)) == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess || w) {
         say(errbuf, errbuf_len, "gala_gemm_bf16_static: %s",
             e != cudaSuccess ? cudaGetErrorString(e) : "a bounded device-side wait ran out");
         return GALA_ECUDA;

@@ -201,10 +201,11 @@ cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* c
 // double precision make the result independent of scheduling.
 __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict__ g, long d, long d_pad,
                                                         int agent0, float max_norm, double* partial,
-                                                        unsigned* ticket, float* norm, float* clip, NormKnown kn) {
+                                                        unsigned* ticket, float* norm, float* clip, NormKnown kn, AgentMap am) {
     pdl_wait();
     pdl_launch();
-    const int agent = agent0 + blockIdx.y;
+    const int slot = agent_slot(am, blockIdx.y);
+    const int agent = agent0 + slot;
     const float* ga = g + (long)agent * d_pad;
     // The elements to read, [0, d_pad) without the range whose sum of squares is already known, are numbered
     // consecutively and cut into chunks of multiples of 4 floats (the padding [d, d_pad) is zero): 16-byte loads
@@ -220,7 +221,7 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
     }
     double acc = ((double)a0 + (double)a1) + ((double)a2 + (double)a3);
     if (kn.partial) {   // the known range: its partial sums, shared out over the agent's threads in slot order
-        const float* kp = kn.partial + (long)blockIdx.y * kn.partial_group_stride;
+        const float* kp = kn.partial + (long)slot * kn.partial_group_stride;
         for (long k = (long)blockIdx.x * blockDim.x + threadIdx.x; k < kn.n_partials; k += (long)chunks * blockDim.x)
             acc += (double)kp[k];
     }
@@ -254,7 +255,7 @@ __global__ void __launch_bounds__(256) grad_norm_kernel(const float* __restrict_
 
 cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int n_agents, float max_norm,
                              double* partial, unsigned* ticket, float* norm, float* clip, cudaStream_t st,
-                             const NormKnown* known) {
+                             const NormKnown* known, const AgentMap* am) {
     NormKnown kn{};
     if (known) kn = *known;
     if (!kn.partial) { kn.off = 0; kn.count = 0; kn.n_partials = 0; }
@@ -265,7 +266,7 @@ cudaError_t launch_grad_norm(const float* g, long d, long d_pad, int agent0, int
     if (chunks < 1) chunks = 1;
     if (chunks > kNormChunks) chunks = kNormChunks;
     dim3 grid((unsigned)chunks, n_agents);
-    (void)launch_pdl(grad_norm_kernel, dim3(grid), dim3(256), 0, st, g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip, kn);
+    (void)launch_pdl(grad_norm_kernel, dim3(grid), dim3(256), 0, st, g, d, d_pad, agent0, max_norm, partial, ticket, norm, clip, kn, am ? *am : AgentMap{});
     return cudaGetLastError();
 }
 

@@ -70,6 +70,7 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     constexpr uint32_t tmem_cols = T::GROUPS * 64 > 256 ? 512u : 256u;
 
     const int gz = blockIdx.x / p.splits, ss = blockIdx.x - gz * p.splits;
+    const int slot = agent_slot(p.am, gz);
     const int s_begin = (int)((long)p.samples * ss / p.splits), s_end = (int)((long)p.samples * (ss + 1) / p.splits);
     const int n_it = s_end - s_begin;
 
@@ -111,8 +112,8 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             if (!go) break;
             if (lane == 0) mbar_expect_tx(&full_bar[s], (uint32_t)(T::PLANES * T::PLANE_ROWS * T::X_ROWB + T::DY_ROWS * 128));
             __syncwarp();
-            const int sx = (p.group0 + gz) * p.x_samples + s_begin + it;
-            const int sy = (p.group0 + gz) * p.y_samples + s_begin + it;
+            const int sx = (p.group0 + slot) * p.x_samples + s_begin + it;
+            const int sy = (p.group0 + slot) * p.y_samples + s_begin + it;
             uint8_t* dst = smem + s * STAGE;
             if (lane < T::PLANES) {
                 if constexpr (W == WG_CONV2) tma_load_5d(dst + lane * T::PLANE_STRIDE, &tmX, &full_bar[s], 32 * (lane & 1), 0, lane >> 1, 0, sx);
@@ -182,7 +183,7 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             bias_part[wq][2 * lane + 1] = (b1[0] + b1[1]) + (b1[2] + b1[3]);
             asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
             if (wq == 0) {
-                float* bo = p.bias_out + (long)gz * p.bias_group_stride + (long)ss * p.bias_split_stride;
+                float* bo = p.bias_out + (long)slot * p.bias_group_stride + (long)ss * p.bias_split_stride;
                 for (int c0 = lane; c0 < 64; c0 += 32)
                     bo[c0] = ((bias_part[0][c0] + bias_part[1][c0]) + bias_part[2][c0]) + bias_part[3][c0];
             }
@@ -192,7 +193,7 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         if (mbar_wait(&acc_full, 0u, &abort_flag)) {
             tcgen05_fence_after();
             const int m = q * 32 + lane;
-            float* out = p.out + (long)gz * p.out_group_stride + (long)ss * p.out_split_stride;
+            float* out = p.out + (long)slot * p.out_group_stride + (long)ss * p.out_split_stride;
 #pragma unroll 1
             for (int g = 0; g < T::GROUPS; g++) {
                 int col;   // column (tap, ci) of W[co][KK] that row m of group g holds, -1: none

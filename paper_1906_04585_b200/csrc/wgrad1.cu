@@ -58,6 +58,7 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
     constexpr uint32_t tmem_cols = 64;
 
     const int gz = blockIdx.x / p.splits, ss = blockIdx.x - gz * p.splits;
+    const int slot = agent_slot(p.am, gz);
     const int s_begin = (int)((long)p.samples * ss / p.splits), s_end = (int)((long)p.samples * (ss + 1) / p.splits);
     const int n_it = (s_end - s_begin) * 4;
 
@@ -113,7 +114,7 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
             if (lane == 0) {
                 mbar_expect_tx(&full_bar[s], (uint32_t)(kW1DyRows * 64));
                 tma_load_4d(smem + s * kW1Stage + kW1XBytes + kW1DyPad * 64, &tmY, &full_bar[s], 0, 0, 5 * q,
-                            (p.group0 + gz) * p.y_samples + sample);
+                            (p.group0 + slot) * p.y_samples + sample);
                 issued_dy = it + 1;
             }
         }
@@ -196,7 +197,7 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
             const int q = warp & 3;
             const int m = q * 32 + lane;
             const int py = m >> 5, b = (m >> 4) & 1, el = m & 15;
-            float* out = p.out + (long)gz * p.out_group_stride + (long)ss * p.out_split_stride;
+            float* out = p.out + (long)slot * p.out_group_stride + (long)ss * p.out_split_stride;
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const int col = ((4 * h + py) * 8 + 4 * b) * 4 + el;   // (ky, kx, ci) inside W[co][256]

@@ -140,6 +140,12 @@ class Learner:
     def gossip(self, agent: int):
         B.gala_gossip(self.ctx, agent)
 
+    def learn_many(self, agents: Sequence[int], ros: Sequence[DeviceRollout]):
+        B.gala_learn_many(self.ctx, agents, [r.c for r in ros])
+
+    def gossip_many(self, agents: Sequence[int]):
+        B.gala_gossip_many(self.ctx, agents)
+
     def act(self, agent: int, obs: torch.Tensor, uniforms: torch.Tensor):
         torch.cuda.current_stream().synchronize()   # obs / uniforms may still be in flight on torch's stream
         actions = torch.empty(self.E, dtype=torch.int32, device=obs.device)

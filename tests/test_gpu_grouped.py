@@ -1,0 +1,267 @@
+"""GPU parity of the grouped per-agent calls (gala_learn_many / gala_gossip_many: the asynchronous learner and
+gossip steps of Algorithm 1 for a list of ready agents in one launch set) and of the stand-alone per-agent form
+of the fused RMSProp + gossip pass (gala_sweep_agents), against the fp64 oracle through the C ABI."""
+import numpy as np
+import pytest
+
+import gala_inputs as GI
+from oracle import reference as R
+from tests.helpers import TOL_BF16, TOL_FP32_NET, TOL_SWEEP, assert_close, assert_grad_close, oracle_hp, oracle_net
+from tests.test_gpu_learner import check_params, make_learner, seed_identical
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _mods():
+    from paper_1906_04585_b200 import binding, learner
+    return binding, learner
+
+
+# ---------------------------------------------------------------------- stand-alone pass
+def _sweep_agents_case(n, slots, d, items, seed, clip):
+    """items: (agent, out_slot, [(peer, slot), ...], has_grad).  Every listed agent against the oracle's
+    sweep_replay; every row that no item writes must come back bit for bit."""
+    B, _ = _mods()
+    d_pad = (d + 3) // 4 * 4
+    x, g, v = GI.sweep_state(n, d, seed)
+    snap = (np.random.default_rng(seed).standard_normal((n, slots, d)) * 0.01).astype(np.float32)
+    hp = B.default_hparams(1, 1, max_grad_norm=0.0)
+    ohp = R.HParams(lr=float(hp.lr), rms_alpha=float(hp.rms_alpha), rms_eps=float(hp.rms_eps), max_grad_norm=0.0)
+
+    def pad(a):
+        out = np.zeros(a.shape[:-1] + (d_pad,), np.float32)
+        out[..., :d] = a
+        return out
+
+    tx, tg, tv, ts = (torch.from_numpy(pad(t)).cuda() for t in (x, g, v, snap))
+    clips = (0.25 + 0.75 * np.random.default_rng(seed + 1).random(n)).astype(np.float32) if clip else None
+    tclip = torch.from_numpy(clips).cuda() if clip else None
+    B.gala_sweep_agents(tx, tg, tv, ts, tclip, n, slots, d_pad, items, hp, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    gx, gv, gs = tx.cpu().numpy()[:, :d], tv.cpu().numpy()[:, :d], ts.cpu().numpy()[:, :, :d]
+    listed = set()
+    for agent, out_slot, peers, has_grad in items:
+        listed.add(agent)
+        msgs = [snap[pj, sj].astype(np.float64) for pj, sj in peers] or None
+        xn, vn, y = R.sweep_replay(x[agent], g[agent] if has_grad else None, v[agent], ohp, msgs,
+                                   clip=float(clips[agent]) if clip else 1.0)
+        assert_close("x[%d]" % agent, gx[agent], xn, TOL_SWEEP)
+        assert_close("snapshot[%d]" % agent, gs[agent, out_slot], y, TOL_SWEEP)
+        if has_grad:
+            assert_close("v[%d]" % agent, gv[agent], vn, TOL_SWEEP)
+        else:
+            np.testing.assert_array_equal(gv[agent], v[agent])
+        for s in range(slots):
+            if s != out_slot:
+                np.testing.assert_array_equal(gs[agent, s], snap[agent, s])
+    for a in range(n):
+        if a not in listed:
+            np.testing.assert_array_equal(gx[a], x[a])
+            np.testing.assert_array_equal(gv[a], v[a])
+            np.testing.assert_array_equal(gs[a], snap[a])
+
+
+def test_sweep_agents_matches_oracle_mixed_items():
+    # none, one and two in-peers, with and without a pending gradient, in one launch; ragged length
+    items = [(0, 1, [(5, 2)], True), (1, 0, [(0, 0), (2, 2)], True), (2, 1, [], True), (3, 2, [(1, 1)], False),
+             (4, 0, [], False)]
+    _sweep_agents_case(6, 3, 10_007, items, GI.BASE_SEED + 11, clip=True)
+
+
+def test_sweep_agents_many_tiles_and_two_launches():
+    # 70 agents (more than one launch holds), several tiles per agent with a ragged last one; every agent reads
+    # its ring predecessor's slot 0 and writes its own slot 1
+    n = 70
+    items = [(i, 1, [((i - 1) % n, 0)], i % 3 != 0) for i in range(n)]
+    _sweep_agents_case(n, 2, 3 * 4096 + 100, items, GI.BASE_SEED + 12, clip=False)
+
+
+def test_sweep_agents_refuses_a_slot_that_is_read_and_written():
+    B, _ = _mods()
+    n, d = 3, 64
+    t = [torch.zeros((n, d), device="cuda") for _ in range(3)]
+    snap = torch.zeros((n, 2, d), device="cuda")
+    hp = B.default_hparams(1, 1)
+    with pytest.raises(B.GalaError) as ei:
+        B.gala_sweep_agents(t[0], t[1], t[2], snap, None, n, 2, d, [(0, 1, [(1, 0)], True), (1, 0, [], True)], hp,
+                            torch.cuda.current_stream().cuda_stream)
+    assert ei.value.status == B.GALA_EINVAL
+    with pytest.raises(B.GalaError):      # an agent listed twice
+        B.gala_sweep_agents(t[0], t[1], t[2], snap, None, n, 2, d, [(0, 1, [], True), (0, 0, [], True)], hp,
+                            torch.cuda.current_stream().cuda_stream)
+
+
+def test_sweep_agents_full_size_sampled():
+    # the micro-benchmark's size in its per-agent form: 32 agents x 1.7M parameters, one in-peer each (the
+    # 1-peer exponential graph of round 0) and two (rounds 0 and 1 together); the oracle recomputes a sample of
+    # columns, which is exact because the pass is element-wise along the parameter index
+    B, _ = _mods()
+    w = GI.WORKLOADS[3]
+    n, d = w.n_agents, w.sweep_only_d
+    x, g, v = GI.sweep_state(n, d, w.seed)
+    snap0 = (x + np.float32(1e-3)).astype(np.float32)     # snapshots differ from the parameters
+    hp = B.default_hparams(1, 1, max_grad_norm=0.0)
+    ohp = R.HParams(lr=float(hp.lr), rms_alpha=float(hp.rms_alpha), rms_eps=float(hp.rms_eps), max_grad_norm=0.0)
+    rng = np.random.default_rng(9)
+    cols = np.unique(np.concatenate([np.arange(2048), np.arange(d - 2048, d), rng.integers(0, d, 20000)]))
+    for peers in (1, 2):
+        tx, tg, tv = (torch.from_numpy(t).cuda() for t in (x, g, v))
+        ts = torch.zeros((n, 3, d), device="cuda")
+        ts[:, 0] = torch.from_numpy(snap0).cuda()
+        plist = [[(R.in_peers(R.EXP, 1, n, k, i)[0], 0) for k in range(peers)] for i in range(n)]
+        items = [(i, 1, plist[i], True) for i in range(n)]
+        B.gala_sweep_agents(tx, tg, tv, ts, None, n, 3, d, items, hp, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        gx, gv, gy = tx.cpu().numpy()[:, cols], tv.cpu().numpy()[:, cols], ts[:, 1].cpu().numpy()[:, cols]
+        for i in range(n):
+            msgs = [snap0[pj][cols].astype(np.float64) for pj, _ in plist[i]]
+            xn, vn, y = R.sweep_replay(x[i][cols], g[i][cols], v[i][cols], ohp, msgs, clip=1.0)
+            assert_close("x[%d]" % i, gx[i], xn, TOL_SWEEP)
+            assert_close("v[%d]" % i, gv[i], vn, TOL_SWEEP)
+            assert_close("y[%d]" % i, gy[i], y, TOL_SWEEP)
+
+
+# ---------------------------------------------------------------------- grouped learner / gossip steps
+def _grouped_replay(w, steps, tol_net, tol_params, mode="elementwise"):
+    """steps: lists of agents.  Each list gets one gala_learn_many and one gala_gossip_many; the library's own
+    (peer, version) log of every listed agent is then replayed in the oracle, exactly as for the per-agent calls."""
+    B, LM = _mods()
+    net = oracle_net(w)
+    L = make_learner(w)
+    ohp = oracle_hp(L.hp)
+    X, V = seed_identical(L, w, net)
+    n = w.n_agents
+    snaps, version, rnd = {}, [0] * n, [0] * n
+    mixes = same_call_peers = 0
+    rule = "elementwise" if mode == "elementwise" else "norm"
+    for lst in steps:
+        ros = [GI.rollout(w, i, rnd[i]) for i in lst]
+        dev = [LM.DeviceRollout(r) for r in ros]
+        L.learn_many(lst, dev)
+        L.gossip_many(lst)
+        L.sync()
+        new_snaps = {}
+        for i, ro in zip(lst, ros):
+            peers, vers, mixed = B.gala_last_mix(L.ctx, i)
+            assert peers == R.in_peers(w.topo_kind, w.topo_peers, n, rnd[i], i)
+            same_call_peers += sum(1 for pj in peers if pj in lst)
+            info = R.learner_grad(net, X[i], ro, ohp)
+            x_before = X[i].copy()
+            msgs = None
+            if mixed:
+                mixes += 1
+                for pj, vj in zip(peers, vers):
+                    assert 1 <= vj <= version[pj]      # complete before this call: never a snapshot of the same call
+                msgs = [snaps[(pj, vj)] for pj, vj in zip(peers, vers)]
+            xn, vn, y = R.sweep_replay(X[i], info["grad"], V[i], ohp, msgs)
+            assert_grad_close("grad[%d]" % i, L.get_grad(i), info["grad"], net, tol_net, rule)
+            snap = np.empty(L.d, np.float32)
+            B.gala_get_snapshot(L.ctx, i, version[i] + 1, snap)
+            check_params("x[%d]" % i, L.get_params(i), xn, x_before, tol_params, mode)
+            check_params("snapshot[%d]" % i, snap, y, x_before, tol_params, mode)
+            if mode == "elementwise":
+                assert_close("v[%d]" % i, L.get_sq_avg(i), vn, max(tol_params, 2 * tol_net))
+            X[i], V[i] = xn, vn
+            new_snaps[(i, version[i] + 1)] = y
+        for i in lst:
+            version[i] += 1
+            rnd[i] += 1
+            if mode != "elementwise":   # keep both sides on the same trajectory (oracle -> library only)
+                X[i] = X[i].astype(np.float32).astype(np.float64)
+                V[i] = V[i].astype(np.float32).astype(np.float64)
+                new_snaps[(i, version[i])] = new_snaps[(i, version[i])].astype(np.float32).astype(np.float64)
+                L.set_state(i, params=X[i], sq_avg=V[i], rnd=rnd[i])
+            st = B.gala_stats(L.ctx, i)
+            assert st["version"] == version[i] and st["rounds"] == rnd[i]
+        snaps.update(new_snaps)
+    assert mixes > 0 and same_call_peers > 0
+    L.close()
+
+
+def test_grouped_replay_conv():
+    # lists in arbitrary order, of different lengths, with agents that are each other's in-peers in one call
+    w = GI.WORKLOADS[1].scaled(n_agents=5, n_envs=2, n_steps=3)
+    _grouped_replay(w, [[3, 0], [1], [4, 2, 0, 1], [0, 1, 2, 3, 4], [2, 4]], TOL_BF16, TOL_BF16, mode="update")
+
+
+def test_grouped_replay_mlp_falls_back_to_per_agent_kernels():
+    w = GI.WORKLOADS[0]
+    _grouped_replay(w, [[0, 1], [2], [3, 0], [1, 2, 3], [0, 1, 2, 3]], TOL_FP32_NET, TOL_SWEEP)
+
+
+def test_grouped_calls_interleave_with_per_agent_and_synchronous_calls():
+    # The same agent through all three call forms in turn - per-agent calls, grouped calls, a synchronous round -
+    # once with a host wait after every call and once with none: every form must see the state the previous one
+    # left (stream ordering between the forms), so both runs end bit for bit alike.  Agent 1 publishes nothing
+    # before the synchronous round, so agent 0 never averages before it and no decision depends on timing.
+    B, LM = _mods()
+    w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=2, n_steps=2, topo_kind=GI.RING)
+    net = oracle_net(w)
+    ros = [[GI.rollout(w, i, k) for i in range(2)] for k in range(5)]
+    out = []
+    for wait in (True, False):
+        L = make_learner(w)
+        seed_identical(L, w, net)
+        dev = [[LM.DeviceRollout(r) for r in rr] for rr in ros]
+
+        def pause():
+            if wait:
+                L.sync()
+
+        L.learn(0, dev[0][0]); pause()
+        L.gossip(0); pause()
+        L.learn_many([0], [dev[1][0]]); pause()
+        L.gossip_many([0]); pause()
+        L.learn(0, dev[2][0]); pause()
+        L.gossip(0); pause()
+        L.learn_many([0], [dev[3][0]]); pause()
+        L.step_sync(dev[4]); pause()       # applies nothing of the pending gradient twice: it learns anew
+        L.learn_many([1, 0], [dev[0][1], dev[0][0]]); pause()
+        L.gossip_many([0])                 # agent 1 never publishes: nothing here depends on what has completed
+        L.sync()
+        st = [B.gala_stats(L.ctx, i) for i in range(2)]
+        out.append(dict(x=[L.get_params(i) for i in range(2)], v=[L.get_sq_avg(i) for i in range(2)],
+                        g=[L.get_grad(i) for i in range(2)], rounds=[s_["rounds"] for s_ in st],
+                        version=[s_["version"] for s_ in st]))
+        L.close()
+    a, b = out
+    assert a["rounds"] == b["rounds"] == [5, 1] and a["version"] == b["version"] == [4, 0]
+    for key in ("x", "v", "g"):
+        for i in range(2):
+            assert np.isfinite(a[key][i]).all()
+            np.testing.assert_array_equal(a[key][i], b[key][i])
+    assert np.linalg.norm(a["x"][0] - a["x"][1]) > 0
+
+
+def test_grouped_gossip_without_pending_gradient_and_second_learn():
+    # gala_gossip_many with nothing pending publishes and mixes only; a second gala_learn_many applies the
+    # pending gradient without mixing first (as the per-agent calls do)
+    B, LM = _mods()
+    w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=2, n_steps=2)
+    net = oracle_net(w)
+    L = make_learner(w)
+    ohp = oracle_hp(L.hp)
+    X, V = seed_identical(L, w, net)
+    r0, r1 = GI.rollout(w, 0, 0), GI.rollout(w, 0, 1)
+    d0, d1 = LM.DeviceRollout(r0), LM.DeviceRollout(r1)
+    L.learn_many([0], [d0])
+    L.learn_many([0], [d1])
+    L.sync()
+    i0 = R.learner_grad(net, X[0], r0, ohp)
+    x1, v1, _ = R.sweep_replay(X[0], i0["grad"], V[0], ohp, None)
+    check_params("x", L.get_params(0), x1, X[0], TOL_BF16, "update")
+    st = B.gala_stats(L.ctx, 0)
+    assert st["version"] == 1 and st["rounds"] == 1 and st["mixes"] == 0
+    p_before = L.get_params(1).astype(np.float64)
+    v_before = L.get_sq_avg(1)
+    L.gossip_many([1])
+    L.sync()
+    peers, vers, mixed = B.gala_last_mix(L.ctx, 1)
+    assert peers == [0] and vers == [1] and mixed
+    snap = np.empty(L.d, np.float32)
+    B.gala_get_snapshot(L.ctx, 0, 1, snap)
+    assert_close("x1", L.get_params(1), 0.5 * (p_before + snap.astype(np.float64)), TOL_SWEEP)
+    np.testing.assert_array_equal(L.get_sq_avg(1), v_before)
+    L.close()

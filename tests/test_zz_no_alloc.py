@@ -18,8 +18,9 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 # (groups, M, N, K, a_mn, b_mn, split_k): second call is smaller than the first and uses other
-# layouts, so stale partial sums of the first call lie all over its scratch region
-CALLS = [(2, 576, 64, 3920, 1, 1, 4), (1, 256, 40, 200, 1, 0, 2), (3, 300, 72, 136, 0, 0, 1)]
+# layouts, so stale partial sums of the first call lie all over its scratch region; the last call has more
+# splits than K tiles, i.e. a split with nothing to add, which must still overwrite what lies in its region
+CALLS = [(2, 576, 64, 3920, 1, 1, 4), (1, 256, 40, 200, 1, 0, 2), (3, 300, 72, 136, 0, 0, 1), (1, 130, 130, 72, 0, 0, 3)]
 
 
 def _operands(case, seed):
