@@ -284,7 +284,8 @@ int gala_set_stream(gala_ctx* ctx, int agent, void* cuda_stream);
 /* Copy intermediate tensors of the last learn/act of an agent for checks:
  * what = 0 logits [B][A] f32, 1 values [B] f32, 2 returns [S], 3 advantages [S],
  * 4 dlogits [S][A], 5 dvalues [S]; 10+l: output of trunk layer l as float32
- * (B = (T+1)E rows).  out: host or device, `count` floats. */
+ * (B = (T+1)E rows); 20: the bf16 copy of the agent's parameters that the conv
+ * net's products read, as float32 [d].  out: host or device, `count` floats. */
 int gala_debug_read(gala_ctx* ctx, int agent, int what, float* out, long long count);
 /* Number of kernel launches issued by this context so far. */
 long long gala_launch_count(const gala_ctx* ctx);

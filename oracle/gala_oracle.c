@@ -52,6 +52,11 @@ typedef struct {
      * even), as a kernel that stores them in bf16 would; sums stay exact (double).  The caller
      * rounds the trunk weights itself.  0 = exact arithmetic throughout. */
     int round_bf16;
+    /* 1: every pre-activation sum of the trunk is formed in float32, term after term in index order, instead of
+     * exactly.  Not the method: a second, equally valid evaluation of the rounded network, used to measure how far
+     * two implementations that differ only in summation precision drift apart (stored bf16 values one unit in the
+     * last place apart, ReLU gates that fall the other way).  Only meaningful with round_bf16. */
+    int sum_f32;
 } orc_net;
 
 typedef struct {
@@ -134,13 +139,19 @@ static double act_fn(int act, double z) { return act == 0 ? (z > 0.0 ? z : 0.0) 
 static double act_grad(int act, double a) { return act == 0 ? (a > 0.0 ? 1.0 : 0.0) : 1.0 - a * a; }
 
 /* One trunk layer, one sample: y = act(W * x + b). */
-static void layer_forward(const orc_layer *l, int act, int rnd, const double *p, const double *x, double *y) {
+static void layer_forward(const orc_layer *l, int act, int rnd, int f32, const double *p, const double *x, double *y) {
     const double *W = p + l->w_off, *b = p + l->b_off;
     if (!l->conv) {
         for (int o = 0; o < l->oc; o++) {
             double acc = b[o];
             const double *w = W + (long)o * l->in_size;
-            for (long i = 0; i < l->in_size; i++) acc += w[i] * x[i];
+            if (f32) {
+                float a = (float)b[o];
+                for (long i = 0; i < l->in_size; i++) a += (float)w[i] * (float)x[i];
+                acc = (double)a;
+            } else {
+                for (long i = 0; i < l->in_size; i++) acc += w[i] * x[i];
+            }
             y[o] = act_fn(act, acc);
             if (rnd) y[o] = orc_round_bf16(y[o]);
         }
@@ -150,12 +161,15 @@ static void layer_forward(const orc_layer *l, int act, int rnd, const double *p,
         for (int ox = 0; ox < l->ow; ox++)
             for (int o = 0; o < l->oc; o++) {
                 double acc = b[o];
+                float accf = (float)b[o];
                 for (int ky = 0; ky < l->k; ky++)
                     for (int kx = 0; kx < l->k; kx++) {
                         const double *xi = x + ((long)(oy * l->s + ky) * l->iw + (ox * l->s + kx)) * l->ic;
                         const double *w = W + (((long)o * l->k + ky) * l->k + kx) * l->ic;
-                        for (int c = 0; c < l->ic; c++) acc += w[c] * xi[c];
+                        if (f32) for (int c = 0; c < l->ic; c++) accf += (float)w[c] * (float)xi[c];
+                        else for (int c = 0; c < l->ic; c++) acc += w[c] * xi[c];
                     }
+                if (f32) acc = (double)accf;
                 double a = act_fn(act, acc);
                 y[((long)oy * l->ow + ox) * l->oc + o] = rnd ? orc_round_bf16(a) : a;
             }
@@ -225,7 +239,7 @@ int orc_forward(const orc_net *net, const double *params, const double *obs, int
         for (long i = 0; i < L[0].in_size; i++) a0[i] = o[i] * net->in_scale;
         double *x = a0, *y = a1;
         for (int li = 0; li < nl; li++) {
-            layer_forward(&L[li], net->act, net->round_bf16, params, x, y);
+            layer_forward(&L[li], net->act, net->round_bf16, net->sum_f32, params, x, y);
             if (layer_out && li == which_layer)
                 memcpy(layer_out + (long)s * L[li].out_size, y, sizeof(double) * (size_t)L[li].out_size);
             double *t = x; x = y; y = t;
@@ -264,7 +278,7 @@ int orc_backward(const orc_net *net, const double *params, const double *obs, in
     for (int s = 0; s < B; s++) {
         const double *o = obs + (long)s * L[0].in_size;
         for (long i = 0; i < L[0].in_size; i++) acts[0][i] = o[i] * net->in_scale;
-        for (int li = 0; li < nl; li++) layer_forward(&L[li], net->act, net->round_bf16, params, acts[li], acts[li + 1]);
+        for (int li = 0; li < nl; li++) layer_forward(&L[li], net->act, net->round_bf16, net->sum_f32, params, acts[li], acts[li + 1]);
         long H = L[nl - 1].out_size;
         const double *h = acts[nl];
         /* heads */

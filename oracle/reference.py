@@ -53,6 +53,7 @@ class _CNet(C.Structure):
         ("n_actions", C.c_int),
         ("in_scale", C.c_double),
         ("round_bf16", C.c_int),
+        ("sum_f32", C.c_int),
     ]
 
 
@@ -120,9 +121,16 @@ class Net:
     # the ReLU gate, a yes/no decision taken on a stored activation, is taken on the same number
     # by the oracle and by a kernel that stores activations in bf16.  False: exact arithmetic.
     bf16_operands: bool = False
+    # Not the method: the same rounded network with every trunk sum formed in float32, term after term, instead of
+    # exactly - a second valid evaluation, for measuring how far two implementations that differ only in summation
+    # precision drift apart (see gate_flips).
+    sum_f32: bool = False
 
     def with_bf16(self, on: bool = True) -> "Net":
         return replace(self, bf16_operands=on)
+
+    def with_f32_sums(self, on: bool = True) -> "Net":
+        return replace(self, sum_f32=on)
 
     @staticmethod
     def mlp(obs_dim: int = 8, hidden: int = 64, n_actions: int = 4) -> "Net":
@@ -147,6 +155,7 @@ class Net:
         n.n_actions = self.n_actions
         n.in_scale = self.in_scale
         n.round_bf16 = 1 if self.bf16_operands else 0
+        n.sum_f32 = 1 if self.sum_f32 else 0
         return n
 
     @property

@@ -2007,6 +2007,16 @@ int gala_debug_read(gala_ctx* c, int agent, int what, float* out, long long coun
         CK(cudaMemcpy(out, src, (size_t)count * sizeof(float), cudaMemcpyDefault));
         return GALA_OK;
     }
+    if (what == 20) {   // the bf16 copy of the parameters that the trunk products read
+        if (!c->conv) return fail(c, GALA_EINVAL, "gala_debug_read: no bf16 parameter copy for this network");
+        if (count > c->d) return fail(c, GALA_EINVAL, "gala_debug_read: count %lld > %ld", count, c->d);
+        std::vector<__nv_bfloat16> tmp((size_t)count);
+        CK(cudaMemcpy(tmp.data(), c->shadow + (long)agent * c->d_pad, (size_t)count * 2, cudaMemcpyDeviceToHost));
+        std::vector<float> f((size_t)count);
+        for (long long i = 0; i < count; i++) f[i] = __bfloat162float(tmp[i]);
+        CK(cudaMemcpy(out, f.data(), (size_t)count * sizeof(float), cudaMemcpyDefault));
+        return GALA_OK;
+    }
     if (what >= 10 && what <= 13) {
         const int l = what - 10;
         const void* p = nullptr;

@@ -12,16 +12,12 @@ TOL_FP32_NET = 1e-4   # fp32 network (MLP) outputs and gradients
 TOL_BF16 = 2e-2       # bf16-operand GEMM outputs and gradients
 
 
-def assert_close(name, got, want, tol, rule="elementwise"):
-    """Per tensor.  Both rules demand ||a-b||_2 <= tol ||b||_2.
-    rule "elementwise" (fp32 paths) adds |a_i-b_i| <= tol (|b_i| + rms(b)) for every element.
-    rule "norm" (bf16-operand paths) adds max|a_i-b_i| <= 5 tol max|b_i| instead.  Two things make a
-    per-element bound relative to rms(b) meaningless there: a stored bf16 operand that lands one unit
-    in the last place apart on the two sides (fp32 vs exact summation next to a rounding boundary) moves
-    a single product by 0.4 %; and a ReLU input within fp32 summation noise of zero may fall on either
-    side of the gate, which adds or removes that unit's whole contribution (one row of a weight
-    gradient for one sample).  With millions of gated units per step a few such ties are expected; they
-    stay far below tol in l2 but can reach a few % of max|b| on single elements."""
+def assert_close(name, got, want, tol, max_outliers=0):
+    """Per tensor: ||a-b||_2 <= tol ||b||_2, and |a_i-b_i| <= tol (|b_i| + rms(b)) for every element but at most
+    max_outliers of them.  max_outliers is 0 except where the caller has COUNTED, in the oracle alone, how many
+    ReLU gates two valid evaluations of the same bf16 network disagree on (tie_allowance): a gate that falls the
+    other way adds or removes one unit's whole contribution to a row of a weight gradient, which no tolerance on
+    rounding covers.  Returns (relative l2 error, number of elements outside the bound)."""
     a = np.asarray(got, np.float64).ravel()
     b = np.asarray(want, np.float64).ravel()
     assert a.shape == b.shape, (name, a.shape, b.shape)
@@ -30,14 +26,48 @@ def assert_close(name, got, want, tol, rule="elementwise"):
     rel = np.linalg.norm(a - b) / (nb if nb > 0 else 1.0)
     assert rel <= tol, "%s: relative l2 error %.3e > %.1e" % (name, rel, tol)
     if not b.size:
-        return rel
-    if rule == "elementwise":
-        rms = nb / np.sqrt(b.size)
-        worst = np.max(np.abs(a - b) / (np.abs(b) + rms + 1e-30))
-    else:
-        worst = np.max(np.abs(a - b)) / (np.max(np.abs(b)) + 1e-30) / 5.0
-    assert worst <= tol, "%s: worst element error %.3e > %.1e (rel l2 %.3e, rule %s)" % (name, worst, tol, rel, rule)
-    return rel
+        return rel, 0
+    rms = nb / np.sqrt(b.size)
+    ratio = np.abs(a - b) / (np.abs(b) + rms + 1e-30)
+    outliers = int((ratio > tol).sum())
+    assert outliers <= max_outliers, "%s: %d elements beyond %.1e (|b_i| + rms b), %d allowed; worst %.3e (rel l2 %.3e)" % (
+        name, outliers, tol, max_outliers, float(ratio.max()), rel)
+    return rel, outliers
+
+
+# Largest number of gradient elements that one ReLU gate can move beyond rounding: the unit's row of its own
+# layer's weight gradient (3136 for the hidden layer, at most 576 for a convolution) plus what the changed dY
+# does to the rows below through a 4x4 or 3x3 receptive field.
+GATE_FAN_OUT = 4096
+
+
+def tie_allowance(net: R.Net, params, obs) -> int:
+    """Elements of a gradient that may lie outside the per-element bound, counted in the oracle alone: the number of
+    ReLU gates on which two evaluations of the same bf16 network disagree - every sum formed exactly, and every sum
+    formed in float32 term after term - plus one (a third evaluation, the GPU's, disagrees on gates of its own:
+    about one in 10^6 units lies that close to zero, i.e. none to a few per test), times the fan-out of one gate.
+    Nothing here comes from the GPU.  The test in which no gate CAN fall the other way (biases that fix every gate)
+    allows no element at all."""
+    if not net.bf16_operands:
+        return 0
+    from concurrent.futures import ThreadPoolExecutor
+    o = np.asarray(obs).reshape(len(obs), -1)
+    nl = len(net.convs) + len(net.hidden)
+    f32 = net.with_f32_sums()
+
+    def count(chunk):
+        n = 0
+        for li in range(nl):
+            y0 = R.forward(net, params, chunk, which_layer=li)[2]
+            y1 = R.forward(f32, params, chunk, which_layer=li)[2]
+            n += int(((y0 > 0) != (y1 > 0)).sum())
+        return n
+
+    k = max(1, min(8, len(o) // 4))
+    cuts = [len(o) * i // k for i in range(k + 1)]
+    with ThreadPoolExecutor(k) as ex:
+        flips = sum(ex.map(count, [o[cuts[i]:cuts[i + 1]] for i in range(k)]))
+    return (flips + 1) * GATE_FAN_OUT
 
 
 def oracle_net(w: GI.Workload, exact: bool = False) -> R.Net:
@@ -63,9 +93,13 @@ def to_bf16_f64(a: np.ndarray) -> np.ndarray:
     return u.astype(np.uint32).view(np.float32).astype(np.float64)
 
 
-def assert_grad_close(name, got, want, net: R.Net, tol, rule="elementwise"):
-    """The tolerance rule applied per parameter tensor (conv1.W, conv1.b, ..., v.b)."""
+def assert_grad_close(name, got, want, net: R.Net, tol, max_outliers=0):
+    """The tolerance rule applied per parameter tensor (conv1.W, conv1.b, ..., v.b); max_outliers is the budget
+    of the whole gradient.  Returns the number of elements outside the per-element bound."""
     off = R.param_offsets(net)
     bounds = sorted((v, k) for k, v in off.items())
+    total = 0
     for (lo, key), (hi, _) in zip(bounds[:-1], bounds[1:]):
-        assert_close("%s/%s" % (name, key), np.asarray(got)[lo:hi], np.asarray(want)[lo:hi], tol, rule)
+        total += assert_close("%s/%s" % (name, key), np.asarray(got)[lo:hi], np.asarray(want)[lo:hi], tol,
+                              max_outliers=max_outliers - total)[1]
+    return total

@@ -6,7 +6,7 @@ import pytest
 
 import gala_inputs as GI
 from oracle import reference as R
-from tests.helpers import TOL_BF16, assert_close, assert_grad_close, oracle_hp, oracle_net
+from tests.helpers import TOL_BF16, assert_close, assert_grad_close, oracle_hp, oracle_net, tie_allowance
 
 pytestmark = pytest.mark.gpu
 
@@ -31,11 +31,16 @@ def _run_sync_round(w, sampled):
     x0 = p0.astype(np.float64)
     Y = {}
     for i in need:
-        info = R.learner_grad(net, x0, GI.rollout(w, i, 0), ohp, workers=8)
-        assert_close("logits[%d]" % i, L.debug(i, 0, Bn * A), info["logits"], TOL_BF16, "norm")
-        assert_close("values[%d]" % i, L.debug(i, 1, Bn), info["values"], TOL_BF16, "norm")
-        assert_close("returns[%d]" % i, L.debug(i, 2, S), info["G"], TOL_BF16, "norm")
-        assert_grad_close("grad[%d]" % i, L.get_grad(i), info["grad"], net, TOL_BF16, "norm")
+        ro = GI.rollout(w, i, 0)
+        info = R.learner_grad(net, x0, ro, ohp, workers=8)
+        assert_close("logits[%d]" % i, L.debug(i, 0, Bn * A), info["logits"], TOL_BF16)
+        assert_close("values[%d]" % i, L.debug(i, 1, Bn), info["values"], TOL_BF16)
+        assert_close("returns[%d]" % i, L.debug(i, 2, S), info["G"], TOL_BF16)
+        # every gradient element within 2e-2 (|g_i| + rms) of the oracle's, except what the gates that the
+        # oracle's own two evaluations (exact sums, float32 sums) disagree on can move
+        allow = tie_allowance(net, x0, ro["obs"].reshape(Bn, -1)[:S])
+        out = assert_grad_close("grad[%d]" % i, L.get_grad(i), info["grad"], net, TOL_BF16, max_outliers=allow)
+        print("%s agent %d: %d gradient elements outside the per-element bound, %d allowed" % (w.name, i, out, allow))
         ls = B.gala_losses(L.ctx, i)
         for q in range(3):
             assert abs(ls[q] - info["losses"][q]) <= TOL_BF16 * (abs(info["losses"][q]) + 1.0)

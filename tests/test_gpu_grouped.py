@@ -6,7 +6,8 @@ import pytest
 
 import gala_inputs as GI
 from oracle import reference as R
-from tests.helpers import TOL_BF16, TOL_FP32_NET, TOL_SWEEP, assert_close, assert_grad_close, oracle_hp, oracle_net
+from tests.helpers import (TOL_BF16, TOL_FP32_NET, TOL_SWEEP, assert_close, assert_grad_close, oracle_hp, oracle_net,
+                           tie_allowance)
 from tests.test_gpu_learner import check_params, make_learner, seed_identical
 
 pytestmark = pytest.mark.gpu
@@ -135,7 +136,6 @@ def _grouped_replay(w, steps, tol_net, tol_params, mode="elementwise"):
     n = w.n_agents
     snaps, version, rnd = {}, [0] * n, [0] * n
     mixes = same_call_peers = 0
-    rule = "elementwise" if mode == "elementwise" else "norm"
     for lst in steps:
         ros = [GI.rollout(w, i, rnd[i]) for i in lst]
         dev = [LM.DeviceRollout(r) for r in ros]
@@ -156,7 +156,9 @@ def _grouped_replay(w, steps, tol_net, tol_params, mode="elementwise"):
                     assert 1 <= vj <= version[pj]      # complete before this call: never a snapshot of the same call
                 msgs = [snaps[(pj, vj)] for pj, vj in zip(peers, vers)]
             xn, vn, y = R.sweep_replay(X[i], info["grad"], V[i], ohp, msgs)
-            assert_grad_close("grad[%d]" % i, L.get_grad(i), info["grad"], net, tol_net, rule)
+            S_ = w.n_envs * w.n_steps
+            allow = tie_allowance(net, X[i], ro["obs"].reshape(-1, int(np.prod(ro["obs"].shape[2:])))[:S_])
+            assert_grad_close("grad[%d]" % i, L.get_grad(i), info["grad"], net, tol_net, max_outliers=allow)
             snap = np.empty(L.d, np.float32)
             B.gala_get_snapshot(L.ctx, i, version[i] + 1, snap)
             check_params("x[%d]" % i, L.get_params(i), xn, x_before, tol_params, mode)

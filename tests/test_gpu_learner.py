@@ -7,7 +7,7 @@ import pytest
 import gala_inputs as GI
 from oracle import reference as R
 from tests.helpers import (TOL_BF16, TOL_FP32_NET, TOL_SWEEP, assert_close, assert_grad_close, oracle_hp,
-                           oracle_net)
+                           oracle_net, tie_allowance, to_bf16_f64)
 
 pytestmark = pytest.mark.gpu
 
@@ -63,9 +63,14 @@ def test_topology_schedule_bit_exact():
 
 def check_params(name, got, want, before, tol, mode):
     """mode 'elementwise': the fp32 path, every element within tol.
-    mode 'update': the bf16 path.  RMSProp with a tiny epsilon is close to a sign update, so an
-    element whose gradient is smaller than the bf16 noise may step the other way; the parameters are
-    therefore compared in l2 (relative tol), and the update x_new - x_old in l2 with a loose bound."""
+    mode 'update': the bf16 path with the measured workloads' RMSProp epsilon (1e-5).  From v = 0 the step is
+    lr c g / (0.1 |c g| + eps): a sign step of 10 lr for every element whose gradient is above 1e-4.  An element
+    whose gradient is smaller than its bf16 error may therefore step the other way - a difference of 20 lr on an
+    element the method itself does not resolve.  The parameters are compared in l2 (relative tol) and the update
+    x_new - x_old in l2 at 0.3 (about 2 % of the elements may flip); the optimiser pass itself is held to 1e-5 by
+    replaying it in the oracle from the gradient it was given (replay_sweep_from_library_gradient).
+    mode 'smooth': Table 2's epsilon (0.01): the step is proportional to the gradient, so the update must agree
+    with the oracle's to the tolerance of the gradient."""
     if mode == "elementwise":
         assert_close(name, got, want, tol)
         return
@@ -73,7 +78,30 @@ def check_params(name, got, want, before, tol, mode):
     assert np.isfinite(a).all()
     assert np.linalg.norm(a - b) <= tol * np.linalg.norm(b), name
     du = np.linalg.norm((a - x0) - (b - x0)) / max(np.linalg.norm(b - x0), 1e-30)
-    assert du <= 0.3, "%s: update differs by %.3f in l2" % (name, du)
+    bound = tol if mode == "smooth" else 0.3
+    assert du <= bound, "%s: update differs by %.3e in l2 (bound %.1e)" % (name, du, bound)
+
+
+def replay_sweep_from_library_gradient(L, B_, w, X, V, ohp, rnd):
+    """Second stage of a synchronous round on its own: RMSProp + gossip average in the oracle from the state the
+    round started from and the gradient and gradient norm the LIBRARY computed in its first stage (checked against
+    the oracle's separately).  Both sides of this stage then hold the same inputs, so parameters and second-moment
+    estimates must agree to the tolerance of the fp32 pass (1e-5, per element), and the bf16 copy of the
+    parameters that the trunk products read must be the parameters rounded to bf16."""
+    n = w.n_agents
+    G = np.stack([L.get_grad(i).astype(np.float64) for i in range(n)])
+    clips = []
+    for i in range(n):
+        nrm = float(np.float32(B_.gala_losses(L.ctx, i)[3]))
+        mx = float(L.hp.max_grad_norm)
+        clips.append(min(1.0, mx / (nrm + 1e-6)) if mx > 0 else 1.0)
+    Xn, Vn, _ = R.sweep_sync(X, G, V, ohp, w.topo_kind, w.topo_peers, rnd, clips=clips)
+    for i in range(n):
+        x = L.get_params(i)
+        assert_close("sweep stage x[%d]" % i, x, Xn[i], TOL_SWEEP)
+        assert_close("sweep stage v[%d]" % i, L.get_sq_avg(i), Vn[i], TOL_SWEEP)
+        if w.net_kind == "conv":
+            np.testing.assert_array_equal(B_.gala_debug_read(L.ctx, i, 20, L.d).astype(np.float64), to_bf16_f64(x))
 
 
 def _sync_rounds(w, rounds, tol_net, tol_params, mode="elementwise", **hp):
@@ -83,22 +111,26 @@ def _sync_rounds(w, rounds, tol_net, tol_params, mode="elementwise", **hp):
     ohp = oracle_hp(L.hp)
     X, V = seed_identical(L, w, net)
     S, B, A = w.n_envs * w.n_steps, w.n_envs * (w.n_steps + 1), w.n_actions
-    rule = "elementwise" if mode == "elementwise" else "norm"
     for k in range(rounds):
         ros = [GI.rollout(w, i, k) for i in range(w.n_agents)]
         dev = [LM.DeviceRollout(r) for r in ros]
         L.step_sync(dev)
         L.sync()
         Xn, Vn, infos = R.sync_round(net, X, V, ros, ohp, w.topo_kind, w.topo_peers, k, workers=4)
+        if mode != "elementwise":
+            replay_sweep_from_library_gradient(L, B_, w, X, V, ohp, k)
         for i in range(w.n_agents):
             f = infos[i]
-            assert_close("logits[%d]" % i, L.debug(i, 0, B * A), f["logits"], tol_net, rule)
-            assert_close("values[%d]" % i, L.debug(i, 1, B), f["values"], tol_net, rule)
-            assert_close("returns[%d]" % i, L.debug(i, 2, S), f["G"], tol_net, rule)
+            assert_close("logits[%d]" % i, L.debug(i, 0, B * A), f["logits"], tol_net)
+            assert_close("values[%d]" % i, L.debug(i, 1, B), f["values"], tol_net)
+            assert_close("returns[%d]" % i, L.debug(i, 2, S), f["G"], tol_net)
             # advantages are differences of nearly equal numbers: compare on the scale of the returns
             scale = np.abs(f["G"]).max() + np.abs(f["values"]).max() + 1.0
             assert np.abs(L.debug(i, 3, S) - f["adv"].ravel()).max() <= tol_net * scale
-            assert_grad_close("grad[%d]" % i, L.get_grad(i), f["grad"], net, tol_net, rule)
+            allow = tie_allowance(net, X[i], ros[i]["obs"].reshape(B, -1)[:S])
+            out = assert_grad_close("grad[%d]" % i, L.get_grad(i), f["grad"], net, tol_net, max_outliers=allow)
+            if w.net_kind == "conv":
+                print("agent %d round %d: %d gradient elements outside the per-element bound, %d allowed" % (i, k, out, allow))
             ls = B_.gala_losses(L.ctx, i)
             for q in range(3):
                 assert abs(ls[q] - f["losses"][q]) <= tol_net * (abs(f["losses"][q]) + 1.0)
@@ -200,8 +232,9 @@ def _async_replay(w, order, tol_net, tol_params, mode="elementwise", agent_ctas=
         snaps[(i, version[i])] = y
         X[i], V[i] = xn, vn
         rnd[i] += 1
+        S_ = w.n_envs * w.n_steps
         assert_grad_close("grad", L.get_grad(i), info["grad"], net, tol_net,
-                          "elementwise" if mode == "elementwise" else "norm")
+                          max_outliers=tie_allowance(net, x_before, ro["obs"].reshape(-1, int(np.prod(ro["obs"].shape[2:])))[:S_]))
         snap = np.empty(L.d, np.float32)
         B.gala_get_snapshot(L.ctx, i, version[i], snap)
         check_params("x", L.get_params(i), X[i], x_before, tol_params, mode)
@@ -277,7 +310,7 @@ def test_conv_forward_layers():
         for li, shape in enumerate([(20, 20, 32), (9, 9, 64), (7, 7, 64), (512,)]):
             want = R.forward(net, p0, obs, which_layer=li)[2]
             got = L.debug(i, 10 + li, want.size)
-            assert_close("layer%d[%d]" % (li, i), got, want, TOL_BF16, "norm")
+            assert_close("layer%d[%d]" % (li, i), got, want, TOL_BF16)
     L.close()
 
 
@@ -288,10 +321,53 @@ def test_conv_sync_rounds_small():
 
 
 def test_conv_sync_rounds_table2_epsilon():
-    # Table 2's RMSProp epsilon (0.01): the update is smooth in the gradient, so the update itself
-    # must agree to the bf16 tolerance scale
+    # Table 2's RMSProp epsilon (0.01): the update is proportional to the gradient (sqrt(v) << eps), so the update
+    # itself must agree with the oracle's to the tolerance of the gradient, 2e-2 in l2
     w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=2, n_steps=2)
-    _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update", rms_eps=0.01)
+    _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="smooth", rms_eps=0.01)
+
+
+def test_conv_sync_round_with_gates_fixed_by_the_biases_has_no_outlier():
+    # A workload in which no ReLU gate can fall the other way: in every trunk layer the even output channels get a
+    # bias of +2 max|W*x| and the odd ones -2 max|W*x| (the maxima taken from the oracle's own forward pass, layer
+    # after layer), so every unit is open or closed by a margin no rounding reaches, in a pattern that still
+    # exercises every index.  Every gradient element must then lie within 2e-2 (|g_i| + rms): no allowance.
+    B_, LM = _mods()
+    w = GI.WORKLOADS[2].scaled(n_agents=3, n_envs=4, n_steps=5, topo_peers=2)
+    net = oracle_net(w)
+    off = R.param_offsets(net)
+    p = GI.init_params(GI.net_tensors(w), w.seed).astype(np.float64)
+    ros = [GI.rollout(w, i, 0) for i in range(w.n_agents)]
+    Bn, S = w.n_envs * (w.n_steps + 1), w.n_envs * w.n_steps
+    obs_all = np.concatenate([r["obs"].reshape(Bn, -1) for r in ros])
+    widths = [32, 64, 64, 512]
+    for li in range(4):
+        lo = off["L%d.b" % li]
+        p[lo:lo + widths[li]] = 0.0
+        # relu(W*x) with the biases of the layers below set; relu hides the negative side, so also relu(-W*x)
+        exact = oracle_net(w, exact=True)
+        zpos = float(R.forward(exact, p, obs_all, which_layer=li)[2].max())
+        q = p.copy()
+        q[off["L%d.W" % li]:lo] *= -1.0
+        zneg = float(R.forward(exact, q, obs_all, which_layer=li)[2].max())
+        beta = 2.0 * max(zpos, zneg)
+        p[lo:lo + widths[li]] = np.where(np.arange(widths[li]) % 2 == 0, beta, -beta)
+    p = p.astype(np.float32).astype(np.float64)
+    L = make_learner(w)
+    ohp = oracle_hp(L.hp)
+    for i in range(w.n_agents):
+        L.set_state(i, params=p, sq_avg=np.zeros(L.d, np.float32), rnd=0)
+    L.step_sync([LM.DeviceRollout(r) for r in ros])
+    L.sync()
+    for i in range(w.n_agents):
+        info = R.learner_grad(net, p, ros[i], ohp, workers=4)
+        for li in range(4):       # the pattern is what it was built to be: half the channels open, half closed
+            y = R.forward(net, p, ros[i]["obs"].reshape(Bn, -1)[:2], which_layer=li)[2].reshape(2, -1, widths[li])
+            assert (y[..., 0::2] > 0).all() and (y[..., 1::2] == 0).all()
+        assert_close("logits[%d]" % i, L.debug(i, 0, Bn * w.n_actions), info["logits"], TOL_BF16)
+        assert_close("values[%d]" % i, L.debug(i, 1, Bn), info["values"], TOL_BF16)
+        assert assert_grad_close("grad[%d]" % i, L.get_grad(i), info["grad"], net, TOL_BF16, max_outliers=0) == 0
+    L.close()
 
 
 def test_conv_sync_rounds_multi_tile():
@@ -300,23 +376,38 @@ def test_conv_sync_rounds_multi_tile():
     _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
 
 
-def test_conv_gradient_close_to_exact_arithmetic():
-    # against the unrounded fp64 network the bf16 path differs mostly where a ReLU input lies
-    # within bf16 rounding of zero and the gate falls the other way; the gradient as a whole
-    # must still point the same way
-    w = GI.WORKLOADS[1].scaled(n_agents=1, n_envs=3, n_steps=2)
+def test_conv_step_against_exact_fp64_arithmetic():
+    # The stated tolerance (relative 2e-2 on bf16 GEMM outputs and gradients) against the PLAIN fp64 network: no
+    # operand rounded anywhere in the oracle.  Layer outputs, logits and values in l2 (measured 2-4e-3: the bf16
+    # storage of the activations); the gradient in l2 (measured 1.0-1.3e-2 on 8 agents x 96 samples, the same as the
+    # oracle's own bf16-operand evaluation is from exact arithmetic) with twice that as the bound.  The gap is
+    # the sum of the ~0.1 % of ReLU gates that bf16 storage moves, so it needs the workload's own batch to average
+    # (a dozen samples gave 5e-2): 2 agents at the 8-agent workload's 16 environments x 5 steps.
+    w = GI.WORKLOADS[1].scaled(n_agents=2)
     _, LM = _mods()
     L = make_learner(w)
     seed_identical(L, w, oracle_net(w))
+    exact = oracle_net(w, exact=True)
     p0 = GI.init_params(GI.net_tensors(w), w.seed)
-    ro = GI.rollout(w, 0, 0)
-    dev = LM.DeviceRollout(ro)
-    L.step_sync([dev])
+    ros = [GI.rollout(w, i, 0) for i in range(w.n_agents)]
+    L.step_sync([LM.DeviceRollout(r) for r in ros])
     L.sync()
-    g = L.get_grad(0).astype(np.float64)
-    ge = R.learner_grad(oracle_net(w, exact=True), p0, ro, oracle_hp(L.hp), workers=4)["grad"]
-    assert np.linalg.norm(g - ge) <= 0.15 * np.linalg.norm(ge)
-    assert g @ ge >= 0.98 * np.linalg.norm(g) * np.linalg.norm(ge)
+    Bn, A = w.n_envs * (w.n_steps + 1), w.n_actions
+    for i in range(w.n_agents):
+        obs = ros[i]["obs"].reshape(Bn, -1)
+        for li in range(4):
+            want = R.forward(exact, p0, obs, which_layer=li)[2].ravel()
+            got = L.debug(i, 10 + li, want.size).astype(np.float64)
+            assert np.linalg.norm(got - want) <= TOL_BF16 * np.linalg.norm(want), (i, li)
+        info = R.learner_grad(exact, p0, ros[i], oracle_hp(L.hp), workers=4)
+        for what, cnt, key in ((0, Bn * A, "logits"), (1, Bn, "values")):
+            got, want = L.debug(i, what, cnt).astype(np.float64), np.asarray(info[key]).ravel()
+            assert np.linalg.norm(got - want) <= TOL_BF16 * np.linalg.norm(want), (i, key)
+        g, ge = L.get_grad(i).astype(np.float64), info["grad"]
+        gap = np.linalg.norm(g - ge) / np.linalg.norm(ge)
+        print("agent %d: gradient %.3e from exact fp64 arithmetic in l2" % (i, gap))
+        assert gap <= 2.5e-2
+        assert g @ ge >= 0.999 * np.linalg.norm(g) * np.linalg.norm(ge)
     L.close()
 
 
@@ -429,7 +520,8 @@ def _closed_loop(w, iters, tol_net, tol_params, cdf_tol, mode, graphs=1):
         info = R.learner_grad(net, X[0], ro, ohp)
         x_before = X[0].copy()
         xn, vn, _ = R.sweep_replay(X[0], info["grad"], V[0], ohp, None)
-        assert_grad_close("grad", L.get_grad(0), info["grad"], net, tol_net, "elementwise" if mode == "elementwise" else "norm")
+        assert_grad_close("grad", L.get_grad(0), info["grad"], net, tol_net,
+                          max_outliers=tie_allowance(net, X[0], ro["obs"].reshape(-1, int(np.prod(ro["obs"].shape[2:])))[:T * E]))
         check_params("x", L.get_params(0), xn, x_before, tol_params, mode)
         X[0], V[0] = xn, vn
         if mode != "elementwise":   # keep both sides on the same trajectory (oracle -> library only)

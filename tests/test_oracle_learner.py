@@ -372,3 +372,34 @@ def test_bf16_operand_mode_stays_close_to_exact():
     zb, vb = R.forward(net255.with_bf16(), p, obs)
     assert np.linalg.norm(zb - z) <= 2e-2 * np.linalg.norm(z)
     assert np.linalg.norm(vb - v) <= 2e-2 * np.linalg.norm(v)
+
+
+def test_float32_sum_variant_cancellation_and_bound():
+    # The second evaluation of the rounded network (every trunk sum in float32, term after term) that the GPU
+    # tests use to COUNT how many ReLU gates two valid implementations may disagree on.
+    # (1) closed form: weights (2^30, 1, -2^30) on inputs (1, 1, 1), no bias.  Exactly the sum is 1 (gate open);
+    #     in float32, 2^30 + 1 rounds to 2^30, so the running sum ends at 0 (gate closed).
+    net = R.Net(1, 1, 3, (), (1,), "relu", 2, 1.0).with_bf16()
+    p = np.zeros(R.param_count(net))
+    off = R.param_offsets(net)
+    p[off["L0.W"]:off["L0.W"] + 3] = [2.0 ** 30, 1.0, -2.0 ** 30]
+    obs = np.ones((1, 3))
+    assert R.forward(net, p, obs, which_layer=0)[2][0, 0] == 1.0
+    assert R.forward(net.with_f32_sums(), p, obs, which_layer=0)[2][0, 0] == 0.0
+    from tests.helpers import GATE_FAN_OUT, tie_allowance
+    assert tie_allowance(net, p, obs) == 2 * GATE_FAN_OUT      # one gate disagrees (+ the one always granted)
+    assert tie_allowance(net.with_bf16(False), p, obs) == 0     # the exact network has no such question
+    # (2) on ordinary inputs the float32 sums stay within the textbook bound K u sum|w x| of the exact ones
+    #     (u = 2^-24), and so do a conv layer's; the stored bf16 values then agree except for a few that sit on
+    #     a rounding boundary, and no gate differs
+    rng = np.random.default_rng(12)
+    net2 = R.Net(6, 6, 2, ((3, 1, 4),), (16,), "relu", 3, 1.0)
+    p2 = rng.normal(size=R.param_count(net2)) * 0.3
+    o2 = rng.normal(size=(5, net2.in_size))
+    for li, K in ((0, 18), (1, 64)):
+        z = R.forward(net2, p2, o2, which_layer=li)[2]
+        z32 = R.forward(net2.with_f32_sums(), p2, o2, which_layer=li)[2]
+        scale = np.abs(z).max() * K
+        assert np.abs(z32 - z).max() <= (K + 1) * 2.0 ** -24 * scale * 4
+        assert np.abs(z32 - z).max() > 0                        # it really is another evaluation
+    assert tie_allowance(net2.with_bf16(), p2, o2) == GATE_FAN_OUT
