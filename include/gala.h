@@ -287,6 +287,12 @@ int gala_set_stream(gala_ctx* ctx, int agent, void* cuda_stream);
  * (B = (T+1)E rows); 20: the bf16 copy of the agent's parameters that the conv
  * net's products read, as float32 [d].  out: host or device, `count` floats. */
 int gala_debug_read(gala_ctx* ctx, int agent, int what, float* out, long long count);
+/* Failure reporting, exercised without a failure: enqueues on the agent's stream a one-thread kernel that waits,
+ * with the bounded wait of the tensor-core kernels limited to `polls` polls (1..100000, microseconds in all), on a
+ * barrier that nothing arrives at, gives up and raises the context's error word exactly as those kernels do when
+ * a wait of theirs runs out.  The next gala_sync_agent / gala_sync_all / gala_get_state then returns GALA_ECUDA
+ * ("a bounded device-side wait ran out") and clears the word; the context stays usable. */
+int gala_debug_wait_runs_out(gala_ctx* ctx, int agent, int polls);
 /* Number of kernel launches issued by this context so far. */
 long long gala_launch_count(const gala_ctx* ctx);
 /* Kernel classes (im2col, each GEMM, sweeps, ...) for per-class accounting. */

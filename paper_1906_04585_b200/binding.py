@@ -65,6 +65,7 @@ EXPORTS = (
     "gala_set_agent_ctas", "gala_set_graphs", "gala_losses_all",
     "gala_actor_loop", "gala_actor_read",
     "gala_learn_many", "gala_gossip_many", "gala_poll_agent", "gala_sweep_agents", "gala_set_group_lanes",
+    "gala_debug_wait_runs_out",
 )
 
 _lib = None
@@ -91,6 +92,7 @@ def lib() -> C.CDLL:
             "gala_gossip_many": (i, [vp, C.POINTER(i), i]),
             "gala_poll_agent": (i, [vp, i, C.POINTER(i)]),
             "gala_set_group_lanes": (i, [vp, i]),
+            "gala_debug_wait_runs_out": (i, [vp, i, i]),
             "gala_sweep_agents": (i, [vp, vp, vp, vp, vp, i, i, ll, C.POINTER(gala_sweep_item), i,
                                       C.POINTER(gala_hparams), vp]),
             "gala_delay": (i, [vp, i, i]),
@@ -209,6 +211,10 @@ def gala_poll_agent(ctx, agent: int) -> bool:
 
 def gala_set_group_lanes(ctx, lanes: int):
     _check(ctx, lib().gala_set_group_lanes(ctx, lanes))
+
+
+def gala_debug_wait_runs_out(ctx, agent: int, polls: int):
+    _check(ctx, lib().gala_debug_wait_runs_out(ctx, agent, polls))
 
 
 def gala_delay(ctx, agent: int, usec: int):

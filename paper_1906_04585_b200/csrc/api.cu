@@ -1900,6 +1900,16 @@ int gala_set_graphs(gala_ctx* c, int on) {
     return GALA_OK;
 }
 
+int gala_debug_wait_runs_out(gala_ctx* c, int agent, int polls) {
+    if (!valid_agent(c, agent) || polls < 1 || polls > 100000)
+        return fail(c, GALA_EINVAL, "gala_debug_wait_runs_out: bad agent or poll count outside 1..100000");
+    Agent& ag = c->agents[agent];
+    int r = own_stream_begin(c, ag);
+    if (r != GALA_OK) return r;
+    CK(launch_wait_runs_out((unsigned)polls, c->error_word, ag.stream));
+    return GALA_OK;
+}
+
 int gala_set_group_lanes(gala_ctx* c, int lanes) {
     if (!c || lanes < 1 || lanes > 2) return fail(c, GALA_EINVAL, "gala_set_group_lanes: 1 or 2");
     c->n_lanes = lanes;

@@ -311,6 +311,7 @@ cudaError_t launch_update_norm(const float* g, const float* v, const float* clip
 cudaError_t launch_consensus(const float* x, int n_agents, long d, long d_pad, double* partial, unsigned* ticket,
                              double* out, cudaStream_t st);
 cudaError_t launch_delay(unsigned long long usec, cudaStream_t st);
+cudaError_t launch_wait_runs_out(unsigned polls, int* error_word, cudaStream_t st);
 cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st);
 
 // ---------------------------------------------------------------- A2C pieces

@@ -7,6 +7,7 @@
 #include <cstdlib>
 
 #include "internal.h"
+#include "tcgen05.cuh"
 
 namespace gala {
 
@@ -423,6 +424,22 @@ __global__ void delay_kernel(unsigned long long usec) {
         if (t - t0 >= usec * 1000ull) break;
     }
 }
+// The give-up path of the tensor-core kernels on its own: one thread waits, with the kernels' bounded wait and a
+// small limit, on an mbarrier that nothing ever arrives at, and reports as they do - abort flag, then the
+// caller's error word - before it returns.  Nothing is left behind: no copy in flight, no tensor memory.
+__global__ void wait_runs_out_kernel(unsigned polls, int* error_word) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_polls(&bar, 0u, &abort_flag, polls) && abort_flag && error_word) atomicExch(error_word, 1);
+}
+cudaError_t launch_wait_runs_out(unsigned polls, int* error_word, cudaStream_t st) {
+    wait_runs_out_kernel<<<1, 1, 0, st>>>(polls, error_word);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_delay(unsigned long long usec, cudaStream_t st) {
     (void)launch_pdl(delay_kernel, dim3(1), dim3(1), 0, st, usec);
     return cudaGetLastError();

@@ -79,6 +79,44 @@ def test_allreduce_a2c_mode_matches_oracle():
     L.close()
 
 
+def test_allreduce_a2c_mode_conv_net_matches_oracle():
+    # the same mode on the conv net (the path the benchmark's all-reduce leg times): the gradient every agent
+    # holds after the round is the oracle's mean over agents (footnote of Sec. 5: one agent with all simulators),
+    # per element; the common RMSProp step is replayed from that gradient and its norm at the tolerance of the pass
+    from paper_1906_04585_b200 import binding as B
+    from paper_1906_04585_b200 import learner as LM
+    from tests.helpers import TOL_BF16, assert_grad_close, tie_allowance
+    w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=3, n_steps=2, topo_kind=R.COMPLETE, topo_peers=0)
+    net = oracle_net(w)
+    L = _learner(w)
+    ohp = oracle_hp(L.hp)
+    p0 = GI.init_params(GI.net_tensors(w), w.seed)
+    for i in range(w.n_agents):
+        L.set_state(i, params=p0, sq_avg=np.zeros(L.d, np.float32))
+    X = p0.astype(np.float64)
+    ros = [GI.rollout(w, i, 0) for i in range(w.n_agents)]
+    L.step_sync([LM.DeviceRollout(r) for r in ros])
+    L.sync()
+    gm = np.mean([R.learner_grad(net, X, r, ohp)["grad"] for r in ros], axis=0)
+    big = {key: np.concatenate([r[key] for r in ros], axis=1) for key in ros[0]}
+    g_big = R.learner_grad(net, X, big, ohp)["grad"]
+    assert np.linalg.norm(gm - g_big) <= 1e-9 * np.linalg.norm(g_big)
+    S = w.n_envs * w.n_steps
+    allow = sum(tie_allowance(net, X, r["obs"].reshape(-1, 84 * 84 * 4)[:S]) for r in ros)
+    g0 = L.get_grad(0)
+    assert_grad_close("mean gradient", g0, gm, net, TOL_BF16, max_outliers=allow)
+    nrm = float(np.float32(B.gala_losses(L.ctx, 0)[3]))
+    assert abs(nrm - np.linalg.norm(gm)) <= TOL_BF16 * np.linalg.norm(gm)
+    c = min(1.0, ohp.max_grad_norm / (nrm + 1e-6))
+    xn, vn = R.rmsprop(X, g0.astype(np.float64), np.zeros_like(X), c, ohp.lr, ohp.rms_alpha, ohp.rms_eps)
+    for i in range(w.n_agents):
+        np.testing.assert_array_equal(L.get_grad(i), g0)              # every agent holds the same mean
+        assert_close("x[%d]" % i, L.get_params(i), xn, TOL_SWEEP)
+        assert_close("v[%d]" % i, L.get_sq_avg(i), vn, TOL_SWEEP)
+    assert B.gala_consensus_distance(L.ctx) == 0.0
+    L.close()
+
+
 def test_update_norm_matches_oracle_and_proposition1_bound_holds():
     # Identical initial parameters, real rollouts, 2-peer ring of 6 agents: the library's ||alpha G(k)||_F of every
     # round against the oracle's (the norm of X - Y, its own RMSProp steps), and the measured distance from
