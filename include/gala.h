@@ -230,8 +230,8 @@ int gala_update_norm(gala_ctx* ctx, double* out);
 int gala_set_stale_timeout(gala_ctx* ctx, int timeout_ms);
 /* SM budget of one agent's tensor-core kernels in the per-agent calls (gala_learn, gala_act): at most `ctas`
  * thread blocks per kernel, so that kernels of several agents' streams run side by side instead of each
- * taking every SM in turn (Sec. 3: the agents progress independently).  0 or >= 148: no limit (default at
- * creation: 148 * 8 / n_agents, at least 32, no limit for fewer than 5 agents).  gala_step_sync is not
+ * taking every SM in turn (Sec. 3: the agents progress independently).  0 or at least the device's SM count: no
+ * limit (default at creation: 8 x SM count / n_agents, at least 32, no limit for fewer than 5 agents).  gala_step_sync is not
  * affected.  Results do not depend on the budget except through the summation order of sliced weight
  * gradients. */
 int gala_set_agent_ctas(gala_ctx* ctx, int ctas);
@@ -239,10 +239,13 @@ int gala_set_agent_ctas(gala_ctx* ctx, int ctas);
  * `iterations` times { T times: act on the current observations of the agent's E environments, step the
  * environments with the sampled actions and store the transition; then gala_learn on the stored rollout and
  * gala_gossip }.  The environments are a synthetic stand-in for the paper's simulators (which run on CPUs and
- * are no part of this library): a counter-based function of (env_seed, agent, environment, step), defined next
- * to its kernel in csrc/env.cu and restated in gala_inputs.synthetic_env: observations (uint8 frames or float
- * vectors) and the uniform for the action draw depend on the step only, reward = 1 when the action equals a
- * hidden per-step target, done with probability 0.01.  Steps are numbered per agent from 0 and continue over
+ * are no part of this library): a counter-based function of (env_seed, agent, environment, step) on the SplitMix64
+ * output function sm(z): z += 0x9E3779B97F4A7C15; z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9; z = (z ^ z >> 27) *
+ * 0x94D049BB133111EB; return z ^ z >> 31.  With base = sm(sm(sm(env_seed + agent) + environment) + step):
+ * the uniform of the action draw is (sm(base + (3 << 56)) >> 40) * 2^-24; a frame's byte j is byte j % 8
+ * (little-endian) of sm(base + j / 8), a float observation's element j is ((sm(base + j) >> 40) * 2^-23 - 1) *
+ * sqrt(3); the reward is 1 when the action equals sm(base + (1 << 56)) mod n_actions, else 0; the episode ends
+ * when sm(base + (2 << 56)) >> 40 < 167772 (probability 0.01).  Steps are numbered per agent from 0 and continue over
  * calls.  The rollout buffers belong to the library (allocated by the first call for an agent).  Unless graph
  * replay is off (gala_set_graphs), an agent's iteration without its gossip step is captured on its second run
  * and replayed as one graph launch from the third on.  Returns as

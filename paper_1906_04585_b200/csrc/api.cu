@@ -470,7 +470,8 @@ int build_plans(gala_ctx* c) {
         f.tag = T_GEMM_CONV_FWD + l;
         f.args.variant = CV_CONV1_FWD + l;
         f.args.a_samples = (int)B;
-        f.args.scale = l == 0 ? 1.0f / 255.0f : 1.0f;
+        // conv1's products take the weights as fp16(w * 2^12) and the frames as the integers they are
+        f.args.scale = l == 0 ? 1.0f / (255.0f * 4096.0f) : 1.0f;
         f.args.bias = c->x + c->cl.b[l]; f.args.bias_group_stride = dp;
         f.args.out = c->act[l]; f.args.out_group_stride = B * P[l] * CO;
         f.args.gate_out = c->gate[l]; f.args.gate_group_stride = B * P[l] * CO / 32;
@@ -520,7 +521,7 @@ int build_plans(gala_ctx* c) {
 int pick_splits(gala_ctx* c, int groups, int S, long count, int fixed) {
     int best = 1;
     long best_cost = -1;
-    const long sms = c->cur_ctas > 0 ? c->cur_ctas : 148;
+    const long sms = c->cur_ctas > 0 ? c->cur_ctas : sm_count();
     for (int sp = 1; sp <= c->max_split && sp <= S; sp++) {
         if (sp > 1 && S / sp < 4) break;   // max_split slices of every layer fit its region of the workspace
         if (sp > 1 && c->cur_ctas > 0 && (long)groups * sp > sms) break;
@@ -624,7 +625,7 @@ int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override,
 int run_wgrad(gala_ctx* c, const Plan& p, int agent0, int groups, cudaStream_t st) {
     const int k_tiles = p.args.conv_mode != CONV_NONE ? p.args.k_steps : (p.args.K + 63) / 64;
     const int tiles = ((p.args.M + 127) / 128) * ((p.args.N + p.args.block_n - 1) / p.args.block_n);
-    int split = (2 * 148) / (groups * tiles);
+    int split = (2 * sm_count()) / (groups * tiles);
     if (split > k_tiles / 4) split = k_tiles / 4;
     if (split > c->max_split) split = c->max_split;
     if (split < 1) split = 1;
@@ -672,7 +673,7 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         {
             const Plan& p = c->fc_fwd;
             const int tiles = ((rows + 127) / 128) * (kHidden / 128);
-            int split = (c->cur_ctas > 0 ? 2 * c->cur_ctas : 296) / (groups * tiles);
+            int split = (c->cur_ctas > 0 ? 2 * c->cur_ctas : 2 * sm_count()) / (groups * tiles);
             if (split > 7) split = 7;
             while (split > 1 && (long)split * rows * kHidden > c->splitk_group_stride) split--;
             if (split <= 1) {
@@ -1233,7 +1234,9 @@ int check_error_word(gala_ctx* c) {
     if (w) {
         int z = 0;
         (void)copy_in(c, c->error_word, &z, sizeof z, c->main_stream);
-        return fail(c, GALA_ECUDA, "a bounded device-side wait ran out (tensor-core pipeline)");
+        // 1 hidden-layer product, 2 / 3 optimiser passes, 10.. convolution variant, 21 / 22 conv2 / conv3 weight
+        // gradient, 30 conv1 weight gradient
+        return fail(c, GALA_ECUDA, "a bounded device-side wait ran out (kernel code %d)", w);
     }
     return GALA_OK;
 }
@@ -1354,7 +1357,7 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         CK(wgrad_init());
         CK(wgrad1_init());
         c->legacy_conv = getenv("GALA_CONV_LEGACY") != nullptr;
-        if (n >= 5) c->agent_ctas = 148 * 8 / n < 32 ? 32 : 148 * 8 / n;   // measured on 64 agents: 32 beats 16 and 64
+        if (n >= 5) c->agent_ctas = sm_count() * 8 / n < 32 ? 32 : sm_count() * 8 / n;   // measured on 64 agents: 32 beats 16 and 64
         c->fused_heads = heads_fused_supported(c->T, c->E, c->A, kHidden) && getenv("GALA_HEADS_UNFUSED") == nullptr;
         ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
         ALLOC(c->dzv, (size_t)n * S * 20);
@@ -1919,7 +1922,7 @@ int gala_set_group_lanes(gala_ctx* c, int lanes) {
 
 int gala_set_agent_ctas(gala_ctx* c, int ctas) {
     if (!c || ctas < 0) return fail(c, GALA_EINVAL, "gala_set_agent_ctas: negative budget");
-    c->agent_ctas = ctas >= 148 ? 0 : ctas;
+    c->agent_ctas = ctas >= sm_count() ? 0 : ctas;
     return GALA_OK;
 }
 

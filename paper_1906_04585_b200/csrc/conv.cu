@@ -12,9 +12,18 @@
 // and dropped by the epilogue.
 //
 // Strided layers are turned into shifts by splitting the input into phase planes:
-//   conv1 (8x8, stride 4): plane py = input lines y = 4u + py, each line seen as 21 groups of
-//          4 pixels x 4 channels (16 elements = one K=16 MMA); tap (ky, b): plane ky % 4,
-//          shift (ky / 4) * 21 + b
+//   conv1 (8x8, stride 4): a row of the shared-memory image = one group of 4 pixels x 4 channels of the four
+//          input lines y = 4u + py side by side (4 x 16 elements = 128 bytes, 128-byte swizzle; rows whose
+//          16 elements ARE the row, 32 bytes wide, make the tensor core fetch its operands at a fraction of
+//          the rate: 224 cycles per 128 x 64 x 16 MMA measured against ~70 with 128-byte rows); tap (ky, b):
+//          K slice ky % 4 of the row, shift (ky / 4) * 21 + b: 16 MMAs of N = 32 per unit.  (Folding b into
+//          N = 64 columns halves the MMAs, but the epilogue must then add column block 1 of the NEXT row to
+//          block 0 of a row, across lanes and warps, and that cost more than the MMAs saved: a thread issues
+//          an MMA of M = 128, K = 16 every ~80 cycles whatever N <= 128 is, two issuing threads reach one per
+//          ~42 cycles at N = 32 and ~50 at N = 64, measured.)  Operands are fp16, not
+//          bf16: a byte widens to fp16 with one byte permutation and one packed subtraction for two pixels
+//          (0x6400 | b is 1024 + b), and the layer's weights, bf16 values, are exact in fp16 after a scaling
+//          by 2^12 that the epilogue takes back (|w| < 16; weights below 2^-26 lose low bits).
 //   conv2 (4x4, stride 2): plane (py, px) = pixels (2u + py, 2v + px), 32 channels a row; tap (ky, kx):
 //          plane (ky % 2, kx % 2), shift (ky / 2) * 10 + kx / 2
 //   conv3 (3x3, stride 1): one plane, shift ky * 9 + kx
@@ -42,9 +51,11 @@ namespace gala {
 
 template <int V> struct ConvTraits;
 template <> struct ConvTraits<CV_CONV1_FWD> {
-    static constexpr int ROWB = 32, LAYOUT = 6, PLANES = 4, PLANE_ROWS = 147, PLANE_STRIDE = 4864;
-    static constexpr int TAPS = 16, KKN = 1, BN = 32, PITCH = 21, OH = 6, OW = 20;
-    static constexpr int W_BOXES = 16, W_BOX_BYTES = 1024, B_MN = 0, B_LAYOUT = 6, B_SBO = 256, B_LBO = 16;
+    static constexpr int ROWB = 128, LAYOUT = 2, PLANES = 1, PLANE_ROWS = 147, PLANE_STRIDE = 19456;
+    static constexpr int TAPS = 4, KKN = 4, BN = 32, PITCH = 21, OH = 6, OW = 20;   // tap 2 dy + b = kernel lines 4 dy .. 4 dy + 3, pixel group b
+    // the weights arrive as 16 unswizzled boxes [32 co x 16 k] (box 2 ky + b) and are laid out for the products by
+    // the converter warps: tile 2 dy + b = rows co x 128 bytes (K slice ky % 4 at 32 (ky % 4)), 128-byte swizzle
+    static constexpr int W_BOXES = 16, W_BOX_BYTES = 1024, B_MN = 0, B_LAYOUT = 2, B_SBO = 1024, B_LBO = 16;
 };
 template <> struct ConvTraits<CV_CONV2_FWD> {
     static constexpr int ROWB = 64, LAYOUT = 4, PLANES = 4, PLANE_ROWS = 100, PLANE_STRIDE = 6656;
@@ -71,22 +82,28 @@ constexpr int kConvMaxStages = 8;
 constexpr int kConvSlack = 8 * 1024;             // rows an MMA reads past the last plane of the ring
 constexpr int kConvEpiWarpBytes = 512;           // an epilogue warp's copy of the layer's bias
 constexpr int kConvSmemMax = 224 * 1024;
+constexpr int kConv1SmemMax = 226 * 1024;           // conv1 forward: all a block may have but 1 KB for the static part
 // conv1 reads the uint8 frames themselves.  An agent's frames are one long run of groups of four lines
 // (1344 bytes each, 21 per frame), and output line L of that run (frame L / 21, line L % 21; line 20 of a
 // frame does not exist and is dropped) needs groups L and L + 1.  A unit is six consecutive output lines
 // wherever frames begin and end: 126 of the 128 rows of an MMA are pixel slots.  The seven groups behind
-// them are one contiguous piece, staged as it is and widened to bf16 planes by four more warps.
+// them are one contiguous piece, staged as it is and widened to an fp16 plane by four more warps.
 constexpr int kC1Lines = 6;                          // output lines of a unit
 constexpr int kC1Group = 4 * 336;                    // bytes of four input lines
-constexpr int kU8Stages = 4;
+constexpr int kU8Stages = 8;                        // two line blocks in flight per converter warp
 constexpr int kU8Bytes = (kC1Lines + 1) * kC1Group;  // 9408
-constexpr int kU8Stride = 9728;
-constexpr int kC1ConvWarps = 4;                     // conv1: warps that widen the uint8 lines
+constexpr int kU8Stride = 9472;
+constexpr int kC1ConvWarps = 4;                     // conv1: warps that widen the uint8 lines, a whole unit each in turn
+// (15 warps in all, so that 128 registers a thread fit).  A ring slot must always be handled by
+// the same converter warp, in order: a wait for a slot's later phase passes at once while an earlier one is pending.
+static_assert(kU8Stages % kC1ConvWarps == 0, "a byte ring slot belongs to one converter warp");
+static_assert(kC1ConvWarps % 2 == 0, "a stage belongs to one converter warp and to one of the two issuers");
+constexpr float kC1WeightScale = 4096.0f;           // conv1's weights enter the products as fp16(w * 2^12)
 constexpr int kConvThreads = 352, kConv1Threads = 352 + 32 * kC1ConvWarps;
 
 // plane and row shift of a tap
 template <int V> __host__ __device__ constexpr void tap_view(int t, int& plane, int& shift) {
-    if constexpr (V == CV_CONV1_FWD) { const int ky = t >> 1; plane = ky & 3; shift = (ky >> 2) * 21 + (t & 1); }
+    if constexpr (V == CV_CONV1_FWD) { plane = 0; shift = (t >> 1) * 21 + (t & 1); }
     else if constexpr (V == CV_CONV2_FWD) { const int ky = t >> 2, kx = t & 3; plane = (ky & 1) * 2 + (kx & 1); shift = (ky >> 1) * 10 + (kx >> 1); }
     else if constexpr (V == CV_CONV3_FWD) { const int ky = t / 3; plane = 0; shift = ky * 9 + (t - ky * 3); }
     else if constexpr (V == CV_CONV2_DGRAD) { plane = 0; shift = (1 - (t >> 1)) * 11 + (1 - (t & 1)); }
@@ -148,6 +165,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     __shared__ __align__(8) uint64_t acc_full[4];
     __shared__ __align__(8) uint64_t acc_empty[4];
     __shared__ __align__(8) uint64_t w_full, w_empty;
+    __shared__ __align__(8) uint64_t w_conv;        // conv1: the weights in shared memory have been turned into fp16
     __shared__ __align__(8) uint64_t u8_full[kU8Stages];
     __shared__ __align__(8) uint64_t u8_empty[kU8Stages];
     __shared__ uint32_t tmem_slot;
@@ -157,8 +175,9 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* smW = smem;
     uint8_t* smX = smem + W_BYTES;
-    uint8_t* smE = smX + nst * STAGE + kConvSlack;
+    uint8_t* smE = smX + nst * STAGE + (V == CV_CONV1_FWD ? 1024 : kConvSlack);
     uint8_t* smU = smE + 8 * kConvEpiWarpBytes;   // conv1 only: ring of uint8 line blocks
+    uint8_t* smWraw = smU + kU8Stages * kU8Stride;   // conv1 only: the agent's weights as the tensor copies deliver them
     constexpr bool kU8 = V == CV_CONV1_FWD;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -169,12 +188,13 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const int u_end = (int)(total_units * (blockIdx.x + 1) / gridDim.x);
 
     if (threadIdx.x == 0) {
-        // conv1: a stage is filled by the four converting warps, otherwise by TMA (one arrival with a byte count)
-        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], kU8 ? kC1ConvWarps : 1); mbar_init(&empty_bar[s], 1); }
-        for (int s = 0; s < kU8Stages; s++) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kC1ConvWarps); }
+        // conv1: a stage is filled by one converting warp, otherwise by TMA (one arrival with a byte count)
+        for (int s = 0; s < nst; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kU8Stages; s++) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], 1); }
         for (int b = 0; b < 4; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
         mbar_init(&w_full, 1);
-        mbar_init(&w_empty, 2);
+        mbar_init(&w_empty, 2);             // one commit per issuer
+        mbar_init(&w_conv, 1);
         abort_flag = 0;
         issued_iters = 0;
         issued_w = 0;
@@ -190,7 +210,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if (lane == 0) { mbar_expect_tx(&w_full, (uint32_t)W_BYTES); issued_w = 1; }
             __syncwarp();
             const int group = p.group0 + agent_slot(p.am, decode_unit<V>(u_begin, p.rows).gz);
-            if (lane < T::W_BOXES) tma_load_3d(smW + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
+            if (lane < T::W_BOXES) tma_load_3d((kU8 ? smWraw : smW) + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
         }
     };
     if constexpr (V != CV_CONV1_FWD) first_weights();
@@ -224,7 +244,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (!go) break;
                 if (lane == 0) mbar_expect_tx(&w_full, (uint32_t)W_BYTES);
                 __syncwarp();
-                if (lane < T::W_BOXES) tma_load_3d(smW + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
+                if (lane < T::W_BOXES) tma_load_3d((kU8 ? smWraw : smW) + lane * T::W_BOX_BYTES, &tmW, &w_full, weight_col<V>(lane), 0, group);
                 __syncwarp();
                 cur_g = c.gz;
                 wl++;
@@ -267,18 +287,27 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         }
     } else if (warp == 1 || warp == 10) {
         // ------------------------------------------------ MMA issuers: warp 1 takes the even units, warp 10 the odd
+        // A barrier tells its phases apart by one bit, so whoever waits on it must see every phase, in order: a wait
+        // for a phase that is two ahead of the barrier passes at once, one for a phase two behind never ends.  With
+        // two issuers a stage must therefore always come back to the same issuer: the ring has an even number of
+        // stages (conv1's has one per converting warp, and an even number of those).
         if (lane == 0) {
             const int ii = warp == 1 ? 0 : 1;
-            const uint32_t idesc = make_instr_desc(T::BN, 0, T::B_MN);
+            const uint32_t idesc = make_instr_desc(T::BN, 0, T::B_MN, kU8);   // conv1: fp16 operands
             const uint64_t bd_base = make_smem_desc_raw(smem_u32(smW), T::B_LAYOUT, T::B_SBO, T::B_LBO);
             int it = 0, cur_g = -1, wl = 0;
+            const int upg = units_per_group<V>(p.rows);
+            int gz = u_begin / upg, g_end = (gz + 1) * upg;     // the agent of unit u and where its units end
+            int s = -1;                                         // stage of unit u and the parity of its use
+            uint32_t s_par = 0u;
             for (int u = u_begin; u < u_end; u++, it++) {
+                if (++s == nst) { s = 0; s_par ^= 1u; }
                 // Both issuers follow every change of agent: each reports (through a commit, so only once its
                 // MMAs are complete) that it is done with the old weights, then waits for the new ones.
-                const int gz = u / units_per_group<V>(p.rows);
+                if (u >= g_end) { gz++; g_end += upg; }
                 if (gz != cur_g) {
                     if (cur_g >= 0) umma_commit(&w_empty);
-                    if (!mbar_wait(&w_full, (uint32_t)wl & 1u, &abort_flag)) break;
+                    if (!mbar_wait(kU8 ? &w_conv : &w_full, (uint32_t)wl & 1u, &abort_flag)) break;
                     wl++;
                     cur_g = gz;
                 }
@@ -286,8 +315,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const int k = it >> 1;                  // this issuer's k-th unit goes to its buffer k % 2
                 const int ab = ii * 2 + (k & 1);
                 if (!mbar_wait(&acc_empty[ab], (((uint32_t)k >> 1) & 1u) ^ 1u, &abort_flag)) break;
-                const int s = it % nst;
-                if (!mbar_wait(&full_bar[s], (uint32_t)(it / nst) & 1u, &abort_flag)) break;
+                if (!mbar_wait(&full_bar[s], s_par, &abort_flag)) break;
                 tcgen05_fence_after();
                 const uint32_t tmem_acc = tmem_base + (uint32_t)ab * T::BN;
                 const uint32_t x_addr = smem_u32(smX + s * STAGE);
@@ -300,7 +328,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     int plane, shift;
                     tap_view<V>(t, plane, shift);
                     const uint32_t a_off = plane * T::PLANE_STRIDE + shift * T::ROWB;
-                    const uint32_t b_off = (V == CV_CONV2_DGRAD ? t * 4 * T::W_BOX_BYTES : t * T::W_BOX_BYTES);
+                    const uint32_t b_off = (V == CV_CONV2_DGRAD ? t * 4 : V == CV_CONV1_FWD ? t * 4 : t) * T::W_BOX_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < T::KKN; kk++) {
                         // K = 16 further on: 32 B along a K-major row, 16 rows of an MN-major tile
@@ -314,38 +342,102 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             }
         }
     } else if (warp >= 11) {
-        // ------------------------------------------------ conv1: uint8 lines -> bf16 phase planes
-        // Line yl of the block (28 lines = 7 groups of 4) belongs to plane yl % 4, row (yl / 4) * 21 + xq for its 16-byte
-        // group xq (4 pixels x 4 channels); a row is 32 bytes of bf16 whose two halves swap when bit 7 of
-        // its address is set (32-byte swizzle).  0..255 are exact in bf16; 1/255 is applied after the MMAs.
+        // ------------------------------------------------ conv1: uint8 lines -> fp16 phase planes
+        // Line yl of the block (28 lines = 7 groups of 4) is K slice yl % 4 of row (yl / 4) * 21 + xq for its 16-byte
+        // group xq (4 pixels x 4 channels): 32 bytes of fp16 as two 16-byte pieces, piece c of a row at
+        // 16 (c ^ (row & 7)) (128-byte swizzle).  0..255 are exact in fp16; 1/255 is applied after the MMAs.
+        // The same warps turn an agent's weights, which arrive as bf16, into fp16(w * 2^12) where they lie.
+        // Converter warp cw takes the units cw, cw + 4, ... of the CTA's range, a whole unit each: the fixed cost of a
+        // hand-over (two waits, the proxy fence, two arrivals: some 500 cycles) is then paid by one warp per unit
+        // while the others are busy with other units.  A warp owns one stage and two slots of the byte ring, so every
+        // barrier it waits on is its own and it sees each of their phases in turn.  Converter warp 0 also lays out every agent's weights when it
+        // comes to the agent's first unit (always the same warp, so that it waits for the weight copies in their
+        // order: a wait for a later copy's phase would pass at once while an earlier one is still pending).
         if constexpr (kU8) {
-            const int ct = threadIdx.x - 11 * 32;   // 0 .. 32 * kC1ConvWarps - 1
-            constexpr int kCT = 32 * kC1ConvWarps, kChunks = 4 * (kC1Lines + 1) * 21;
-            int it = 0;
-            for (int u = u_begin; u < u_end; u++, it++) {
+            const int cw = warp - 11;
+            constexpr int kChunks = 4 * (kC1Lines + 1) * 21;   // 16-byte groups of a block, 588
+            // where a lane's k-th group goes inside a stage (the same for every unit): row, K slice, swizzle
+            int dst_off[(kChunks + 31) / 32];
+#pragma unroll
+            for (int k = 0; k < (kChunks + 31) / 32; k++) {
+                const int ch = lane + 32 * k;
+                const int yl = ch / 21, xq = ch - yl * 21;
+                const int r = (yl >> 2) * 21 + xq;
+                dst_off[k] = r * 128 + ((((yl & 3) * 2) ^ (r & 7)) << 4);
+            }
+            const int upg = units_per_group<V>(p.rows);
+            int prev_g = -1, wl = 0, it = 0;
+            bool ok = true;
+            int gz = u_begin / upg, g_end = (gz + 1) * upg;
+            for (int u = u_begin; ok && u < u_end; u++, it++) {
+                if (u >= g_end) { gz++; g_end += upg; }
+                const bool mine = it % kC1ConvWarps == cw;
+                if (gz != prev_g) {
+                    if (cw == 0) {
+                        // (the MMAs that read the previous agent's laid-out weights are complete: the producer waited
+                        // for both issuers' commits before it asked for these)
+                        if (!mbar_wait(&w_full, (uint32_t)wl & 1u, &abort_flag)) break;
+                        for (int ch = lane; ch < W_BYTES / 16; ch += 32) {
+                            // 16-byte piece hh of row co of box j = 2 ky + b  ->  tile 2 (ky / 4) + b, row co, K slice ky % 4
+                            const int j = ch >> 6, co = (ch >> 1) & 31, hh = ch & 1;
+                            const int ky = j >> 1, nrow = (j & 1) * 32 + co;
+                            uint4 v = *reinterpret_cast<const uint4*>(smWraw + ch * 16);
+                            uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                float lo = __uint_as_float(w4[e] << 16) * kC1WeightScale;
+                                float hi = __uint_as_float(w4[e] & 0xffff0000u) * kC1WeightScale;
+                                lo = fminf(fmaxf(lo, -65504.0f), 65504.0f);
+                                hi = fminf(fmaxf(hi, -65504.0f), 65504.0f);
+                                const __half2 h = __floats2half2_rn(lo, hi);
+                                w4[e] = *reinterpret_cast<const uint32_t*>(&h);
+                            }
+                            *reinterpret_cast<uint4*>(smW + (ky >> 2) * 8192 + nrow * 128 + ((((ky & 3) * 2 + hh) ^ (nrow & 7)) << 4)) =
+                                make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&w_conv);
+                    }
+                    wl++;
+                    prev_g = gz;
+                }
+                if (!mine) continue;
                 const int su = it % kU8Stages, s = it % nst;
                 if (!mbar_wait(&u8_full[su], (uint32_t)(it / kU8Stages) & 1u, &abort_flag)) break;
                 if (!mbar_wait(&empty_bar[s], ((uint32_t)(it / nst) & 1u) ^ 1u, &abort_flag)) break;
                 const uint8_t* src = smU + su * kU8Stride;
                 uint8_t* dstage = smX + s * STAGE;
+                // Line yl of the block (28 lines = 7 groups of 4) is K slice yl % 4 of row (yl / 4) * 21 + xq for its
+                // 16-byte group xq (4 pixels x 4 channels): 32 bytes of fp16 as two 16-byte pieces, piece c of a row at
+                // 16 (c ^ (row & 7)) (128-byte swizzle).  0..255 are exact in fp16; 1/255 is applied after the MMAs.
+                // Five 16-byte groups a lane are fetched before any of them is widened and stored: the compiler cannot
+                // know that the byte ring and the stage do not overlap, so loads written after a store wait for it.
+                constexpr int kPer = (kChunks + 31) / 32;   // groups a lane, 19
 #pragma unroll
-                for (int k = 0; k < (kChunks + kCT - 1) / kCT; k++) {
-                    const int ch = ct + k * kCT;          // 16-byte group of the block, 588 in all
-                    if (ch < kChunks) {
-                        const int yl = ch / 21, xq = ch - yl * 21;
-                        const uint4 v = *reinterpret_cast<const uint4*>(src + ch * 16);
-                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                        uint32_t o[8];
+                for (int k0 = 0; k0 < kPer; k0 += 5) {
+                    uint4 v[5];
 #pragma unroll
-                        for (int e = 0; e < 4; e++) {
-                            o[2 * e] = u8x2_to_bf16x2(w[e], 0);
-                            o[2 * e + 1] = u8x2_to_bf16x2(w[e], 2);
+                    for (int k = 0; k < 5; k++) {
+                        const int ch = lane + 32 * (k0 + k);
+                        if (k0 + k < kPer && ch < kChunks) v[k] = *reinterpret_cast<const uint4*>(src + ch * 16);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 5; k++) {
+                        const int ch = lane + 32 * (k0 + k);
+                        if (k0 + k < kPer && ch < kChunks) {
+                            const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+                            uint32_t o[8];
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                o[2 * e] = u8x2_to_f16x2(w[e], 0);
+                                o[2 * e + 1] = u8x2_to_f16x2(w[e], 2);
+                            }
+                            uint8_t* d0 = dstage + dst_off[k0 + k];
+                            *reinterpret_cast<uint4*>(d0) = make_uint4(o[0], o[1], o[2], o[3]);
+                            *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(reinterpret_cast<uintptr_t>(d0) ^ 16)) =
+                                make_uint4(o[4], o[5], o[6], o[7]);
                         }
-                        const int r = (yl >> 2) * 21 + xq;
-                        uint8_t* row = dstage + (yl & 3) * T::PLANE_STRIDE + r * 32;
-                        const int sw = ((r >> 2) & 1) * 16;
-                        *reinterpret_cast<uint4*>(row + sw) = make_uint4(o[0], o[1], o[2], o[3]);
-                        *reinterpret_cast<uint4*>(row + (sw ^ 16)) = make_uint4(o[4], o[5], o[6], o[7]);
                     }
                 }
                 // make the generic-proxy writes visible to the tensor core's reads, then hand the stage over
@@ -432,8 +524,8 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const int L = kC1Lines * c.s + pa;
                 valid = in_tile && L % 21 < 20 && L < 21 * p.rows;
             }
-            const int slot = agent_slot(p.am, c.gz);
-            __nv_bfloat16* out = p.out + (long)slot * p.out_group_stride + off;
+            const int slot_ag = agent_slot(p.am, c.gz);
+            __nv_bfloat16* out = p.out + (long)slot_ag * p.out_group_stride + off;
             // column block c0 -> where it goes: forward, conv3 gradient: channels c0.. of the pixel; conv2
             // gradient: block = parity class (py, px) -> pixel (2a + py, 2b + px), all 32 channels
             auto block_add = [](int c0) -> int {
@@ -444,7 +536,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if (bias_on && c.gz != bg) bias_flush(c.gz);
             if constexpr (kFwd) {
                 if (c.gz != cur_g) {
-                    const float* bias = p.bias + (long)(p.group0 + slot) * p.bias_group_stride;
+                    const float* bias = p.bias + (long)(p.group0 + slot_ag) * p.bias_group_stride;
                     __syncwarp();
                     for (int j = lane; j < T::BN; j += 32) sbias[j] = __ldg(bias + j);
                     __syncwarp();
@@ -493,7 +585,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     if (valid) {   // a 32-byte store fills a whole sector
                         st_global_v8(out + block_add(ch * 32) + 16 * h, o);
                         if constexpr (kFwd) {
-                            if (h == 1 && p.gate_out) p.gate_out[(long)slot * p.gate_group_stride + off / 32 + ch] = bits;
+                            if (h == 1 && p.gate_out) p.gate_out[(long)slot_ag * p.gate_group_stride + off / 32 + ch] = bits;
                         }
                     }
                     if (h == 1) bits = 0u;
@@ -515,7 +607,7 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     __syncthreads();
     if (abort_flag) {
         if (threadIdx.x == 0) {
-            if (p.error_word) atomicExch(p.error_word, 1);
+            if (p.error_word) atomicExch(p.error_word, 10 + V);   // which kernel gave up
             // let copies that were already issued land before the shared memory goes away
             const int issued = issued_iters;
             const int ring = kU8 ? kU8Stages : nst;
@@ -543,7 +635,8 @@ conv_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 
 // ------------------------------------------------------------------ host side
 template <int V> static cudaError_t conv_attr() {
-    return cudaFuncSetAttribute(conv_resident_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, kConvSmemMax);
+    return cudaFuncSetAttribute(conv_resident_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                V == CV_CONV1_FWD ? kConv1SmemMax : kConvSmemMax);
 }
 cudaError_t conv_init() {
     static bool done = false;
@@ -570,7 +663,7 @@ bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const v
         ok &= make_tensor_map_nd(x_map, x_base, 5, dims, str, box, 2);
         const uint64_t wd[3] = {256, 32, groups}, ws[2] = {512, w_group_stride_elems * 2};
         const uint32_t wb[3] = {16, 32, 1};
-        ok &= make_tensor_map_nd(w_map, w_base, 3, wd, ws, wb, 2);
+        ok &= make_tensor_map_nd(w_map, w_base, 3, wd, ws, wb, 3);   // unswizzled: the kernel lays them out itself
         break;
     }
     case CV_CONV2_FWD: {   // act1 [sample][20][20][32] as [sample][y/2][y%2][x/2][2 px x 32 ch]
@@ -612,7 +705,8 @@ bool make_conv_maps(int variant, CUtensorMap* x_map, CUtensorMap* w_map, const v
 }
 
 int conv_grid(long units, int max_ctas) {
-    int grid = (int)(units < kConvMaxGrid ? units : kConvMaxGrid);
+    const int most = sm_count() < kConvMaxGrid ? sm_count() : kConvMaxGrid;
+    int grid = (int)(units < most ? units : most);
     if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;
     return grid;
 }
@@ -621,10 +715,18 @@ template <int V>
 static cudaError_t launch_conv_v(const CUtensorMap& x, const CUtensorMap& w, const ConvArgs& a, cudaStream_t st) {
     using T = ConvTraits<V>;
     constexpr int STAGE = T::PLANES * T::PLANE_STRIDE;
-    constexpr int fixed = T::W_BOXES * T::W_BOX_BYTES + kConvSlack + 8 * kConvEpiWarpBytes + 1024 +
-                          (V == CV_CONV1_FWD ? kU8Stages * kU8Stride : 0);
-    int nst = (kConvSmemMax - fixed) / STAGE;
+    // conv1's MMAs read at most two rows past a stage (shift 21 + 128 rows against 147): 1 KB of slack is plenty
+    constexpr int slack = V == CV_CONV1_FWD ? 1024 : kConvSlack;
+    constexpr int smem_max = V == CV_CONV1_FWD ? kConv1SmemMax : kConvSmemMax;
+    constexpr int fixed = T::W_BOXES * T::W_BOX_BYTES + slack + 8 * kConvEpiWarpBytes + 1024 +
+                          (V == CV_CONV1_FWD ? kU8Stages * kU8Stride + T::W_BOXES * T::W_BOX_BYTES : 0);
+    int nst = (smem_max - fixed) / STAGE;
     if (nst > kConvMaxStages) nst = kConvMaxStages;
+    if constexpr (V == CV_CONV1_FWD) {   // one stage per converter warp (see kC1ConvWarps)
+        if (nst < kC1ConvWarps) return cudaErrorInvalidValue;
+        nst = kC1ConvWarps;
+    }
+    else if (nst > 2) nst &= ~1;   // two issuers: a stage always returns to the same one (see the kernel)
     if (nst < 2) return cudaErrorInvalidValue;
     const long units = (long)a.groups * units_per_group<V>(a.rows);
     if (units <= 0) return cudaSuccess;

@@ -626,7 +626,7 @@ cudaError_t launch_splitk_reduce_multi(const float* ws, float* out, const Reduce
     }
     if ((reinterpret_cast<uintptr_t>(ws) | reinterpret_cast<uintptr_t>(out)) & 15) return cudaErrorInvalidValue;
     int bx = (int)((total4 + 255) / 256);
-    if (bx > 148 * 4) bx = 148 * 4;
+    if (bx > sm_count() * 4) bx = sm_count() * 4;
     (void)launch_pdl(splitk_reduce_multi_kernel, dim3(bx, groups), dim3(256), 0, st, ws, out, segs, total4, ws_group_stride,
                      out_group_stride, am ? *am : AgentMap{});
     return cudaGetLastError();
@@ -665,7 +665,7 @@ cudaError_t launch_splitk_reduce_act(const float* partials, __nv_bfloat16* out, 
     if ((count & 3) || (N & 3) || (split_stride & 3) || (partial_group_stride & 3) || (out_group_stride & 3))
         return cudaErrorInvalidValue;
     int bx = (int)((count / 4 + 255) / 256);
-    if (bx > 148 * 4) bx = 148 * 4;
+    if (bx > sm_count() * 4) bx = sm_count() * 4;
     (void)launch_pdl(splitk_reduce_act_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, partials, out, bias, bias_group_stride, group0, count, N,
                                                                split_k, split_stride, partial_group_stride, out_group_stride);
     return cudaGetLastError();
@@ -674,7 +674,7 @@ cudaError_t launch_splitk_reduce_act(const float* partials, __nv_bfloat16* out, 
 cudaError_t launch_splitk_reduce(const float* partials, float* out, long count, int split_k, long split_stride,
                                  int groups, long partial_group_stride, long out_group_stride, cudaStream_t st) {
     int bx = (int)((count + 255) / 256);
-    if (bx > 148 * 4) bx = 148 * 4;
+    if (bx > sm_count() * 4) bx = sm_count() * 4;
     (void)launch_pdl(splitk_reduce_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, partials, out, count, split_k, split_stride,
                                                            partial_group_stride, out_group_stride);
     return cudaGetLastError();
@@ -685,6 +685,18 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn g_encode = nullptr;
+
+int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
 
 cudaError_t gemm_init() {
     cudaError_t e;
@@ -766,7 +778,8 @@ bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint
     for (int i = 0; i + 1 < rank; i++) { st[i] = strides_bytes[i]; if (st[i] & 15) return false; }
     CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
                           CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          swizzle == 2 ? CU_TENSOR_MAP_SWIZZLE_32B : (swizzle == 1 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B),
+                          swizzle == 3 ? CU_TENSOR_MAP_SWIZZLE_NONE
+                          : swizzle == 2 ? CU_TENSOR_MAP_SWIZZLE_32B : (swizzle == 1 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B),
                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -849,7 +862,7 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     int per_sm = (int)((220u * 1024u) / smem);
     if (per_sm > 2) per_sm = 2;   // 2 x 256 tensor-memory columns is all an SM has
     if (per_sm < 1) per_sm = 1;
-    long cap = 148L * per_sm;
+    long cap = (long)sm_count() * per_sm;
     if (a.max_ctas > 0 && cap > (long)a.max_ctas * per_sm) cap = (long)a.max_ctas * per_sm;
     const int grid = (int)(total < cap ? total : cap);
     (void)launch_pdl(gemm_tcgen05_kernel, dim3(grid), dim3(192), smem, st, A.map, B.map, a, A.mn_major, B.mn_major, total, mt, nt);

@@ -141,6 +141,9 @@ struct GemmArgs {
 enum ConvMode : int { CONV_NONE = 0, CONV_FWD = 1, CONV_WGRAD = 2, CONV_DGRAD = 3 };
 
 cudaError_t gemm_init();   // resolves the driver entry point used to build TMA descriptors
+// Streaming multiprocessors of the current device (asked once per device; 148 if the query fails): what grids and
+// slice counts are sized by.
+int sm_count();
 // rows x cols bf16 matrix per group, cols contiguous.  box_rows x box_cols tile.
 bool make_tensor_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t groups,
                      uint64_t row_stride_bytes, uint64_t group_stride_bytes, uint32_t box_cols,
@@ -151,7 +154,7 @@ bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t cols, uint
 bool make_tensor_map_f32_wide(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes,
                               uint32_t box_blocks, uint32_t box_rows);
 // General bf16 tensor map of rank 3..5 (dims/strides innermost first).  swizzle: 0 = 128-byte, 1 = 64-byte
-// (64-byte rows), 2 = 32-byte (32-byte rows).  Dimensions may overlap (a stride smaller than the extent
+// (64-byte rows), 2 = 32-byte (32-byte rows), 3 = none.  Dimensions may overlap (a stride smaller than the extent
 // below it); a box may be larger than a dimension (the rest reads as zero).
 bool make_tensor_map_nd(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
                         const uint64_t* strides_bytes, const uint32_t* box, int swizzle = 0);
@@ -206,7 +209,7 @@ struct ConvArgs {
     // that range touches; the other slices are left alone and must not be read.
     float* bias_partial;
 };
-constexpr int kConvMaxGrid = 148;
+constexpr int kConvMaxGrid = 148;   // most CTAs a convolution launch uses (the bias slices are laid out for it)
 constexpr long kConvBiasSliceStride = (long)kConvMaxGrid * 8 * 32;   // floats per agent
 int conv_grid(long units, int max_ctas);   // CTAs of a launch over `units` work units
 cudaError_t conv_init();

@@ -34,7 +34,7 @@ cudaError_t launch_cast_frames(const PtrBatch& obs, __nv_bfloat16* out, long out
                                cudaStream_t st) {
     const long n16 = (long)samples * (84 * 84 * 4 / 16);
     int bx = (int)((n16 + 255) / 256);
-    if (bx > 148 * 8) bx = 148 * 8;
+    if (bx > sm_count() * 8) bx = sm_count() * 8;
     (void)launch_pdl(cast_frames_kernel, dim3(dim3(bx, groups)), dim3(256), 0, st, obs, out, out_group_stride, n16);
     return cudaGetLastError();
 }

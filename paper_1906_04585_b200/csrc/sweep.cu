@@ -80,7 +80,7 @@ cudaError_t launch_sweep_agent(float* x, const float* g, float* v, float* snap_o
                                long d_pad, SweepHp hp, cudaStream_t st) {
     long n4 = d_pad / 4;
     int grid = (int)((n4 + 255) / 256);
-    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid > sm_count() * 8) grid = sm_count() * 8;
     if (grid < 1) grid = 1;
     if (n_peers == 0)
         (void)launch_pdl(sweep_agent_kernel<0>, dim3(grid), dim3(256), 0, st, x, g, v, snap_out, nullptr, nullptr, clip, shadow, n4, hp);
@@ -177,7 +177,7 @@ cudaError_t launch_sweep_sync(float* x, const float* g, float* v, const float* c
     int per_sm = (int)((200 * 1024) / (smem ? smem : 1));
     if (per_sm < 1) per_sm = 1;
     if (per_sm > 8) per_sm = 8;
-    long cap = 148L * per_sm;
+    long cap = (long)sm_count() * per_sm;
     int grid = (int)(blocks < cap ? blocks : cap);
     if (grid < 1) grid = 1;
     int o0 = 0, o1 = 0;
@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(256) allreduce_grads_kernel(float* __restrict_
 cudaError_t launch_allreduce_grads(float* g, int n_agents, long d_pad, cudaStream_t st) {
     const long n4 = d_pad / 4;
     int grid = (int)((n4 + 255) / 256);
-    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid > sm_count() * 8) grid = sm_count() * 8;
     (void)launch_pdl(allreduce_grads_kernel, dim3(grid), dim3(256), 0, st, g, n_agents, d_pad, n4);
     return cudaGetLastError();
 }
@@ -454,7 +454,7 @@ __global__ void cast_bf16_kernel(const float* __restrict__ x, __nv_bfloat16* __r
 cudaError_t launch_cast_bf16(const float* x, __nv_bfloat16* out, long count, cudaStream_t st) {
     long n4 = count / 4;
     int grid = (int)((n4 + 255) / 256);
-    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid > sm_count() * 8) grid = sm_count() * 8;
     if (grid < 1) grid = 1;
     (void)launch_pdl(cast_bf16_kernel, dim3(grid), dim3(256), 0, st, x, out, n4);
     return cudaGetLastError();

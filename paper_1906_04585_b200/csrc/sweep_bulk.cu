@@ -240,7 +240,7 @@ cudaError_t launch_sweep_sync_bulk(float* x, const float* g, float* v, const flo
     if (!ok) return cudaErrorNotSupported;
     const long n_tiles = (d_pad + cols - 1) / cols;
     const size_t smem = (size_t)stages * 3 * n_agents * cols * 4;
-    int grid = (int)(n_tiles < 148 ? n_tiles : 148);
+    int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
     cudaError_t e;
 #define GALA_BULK_LAUNCH(P)                                                                                  \
     e = cudaFuncSetAttribute(sweep_sync_bulk_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \

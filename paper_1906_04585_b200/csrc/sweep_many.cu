@@ -229,7 +229,7 @@ cudaError_t launch_sweep_many(const SweepManyArgs& args, cudaStream_t st) {
     const long tiles = (a.d_pad + a.cols - 1) / a.cols;
     const long total = tiles * a.n_items;
     const size_t smem = (size_t)a.stages * a.rows * a.cols * 4;
-    int sms = a.max_ctas > 0 ? a.max_ctas : 148;
+    int sms = a.max_ctas > 0 ? a.max_ctas : sm_count();
     const int grid = (int)(total < sms ? total : sms);
     static bool attr_done = false;
     if (!attr_done) {

@@ -4,6 +4,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 namespace gala {
@@ -99,9 +100,10 @@ __device__ __forceinline__ uint64_t make_smem_desc_raw(uint32_t addr, uint32_t l
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
            (1ull << 46) | ((uint64_t)layout << 61);
 }
-// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B.
-__device__ __forceinline__ uint32_t make_instr_desc(int block_n, int a_mn, int b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+// Instruction descriptor for kind::f16: fp32 accumulator; A and B both bf16 (format 1) or both fp16 (format 0).
+__device__ __forceinline__ uint32_t make_instr_desc(int block_n, int a_mn, int b_mn, bool fp16 = false) {
+    const uint32_t fmt = fp16 ? 0u : ((1u << 7) | (1u << 10));
+    return (1u << 4) | fmt | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
            ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
@@ -171,6 +173,13 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 // Bytes k and k+1 of w as two bf16 numbers, without the (slow) integer -> float conversion unit: a byte
 // dropped into the low mantissa bits of 2^23 is the float 2^23 + b, so subtracting 2^23 leaves b exactly;
 // an integer below 256 has no bits in the lower half of its float, so the upper halves are its bf16.
+// Bytes k and k+1 of w (k = 0 or 2) as two fp16 numbers: 0x6400 | b is the fp16 number 1024 + b, so one byte
+// permutation builds both and one packed subtraction of 1024 leaves b exactly.
+__device__ __forceinline__ uint32_t u8x2_to_f16x2(uint32_t w, int k) {
+    const uint32_t biased = __byte_perm(w, 0x64646464u, k ? 0x5342u : 0x5140u);
+    const __half2 h = __hsub2(*reinterpret_cast<const __half2*>(&biased), __half2half2(__ushort_as_half((unsigned short)0x6400)));
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
 __device__ __forceinline__ uint32_t u8x2_to_bf16x2(uint32_t w, int k) {
     const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7650u + k)) - 8388608.0f;
     const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7651u + k)) - 8388608.0f;

@@ -228,7 +228,7 @@ wgrad_resident_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     __syncthreads();
     if (abort_flag) {
         if (threadIdx.x == 0) {
-            if (p.error_word) atomicExch(p.error_word, 1);
+            if (p.error_word) atomicExch(p.error_word, 20 + W);
             const int issued = issued_iters;
             for (int it = max(0, issued - nst); it < issued; it++) {
                 const int s = it % nst;

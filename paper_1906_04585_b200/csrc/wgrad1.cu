@@ -218,7 +218,7 @@ wgrad_conv1_kernel(const __grid_constant__ CUtensorMap tmY, const Wgrad1Args p) 
     __syncthreads();
     if (abort_flag) {
         if (threadIdx.x == 0) {
-            if (p.error_word) atomicExch(p.error_word, 1);
+            if (p.error_word) atomicExch(p.error_word, 30);
             // let copies that were already issued land before the shared memory goes away
             for (int it = max(0, issued_u8 - kW1U8Stages); it < issued_u8; it++) {
                 const uint32_t ph = (uint32_t)(it / kW1U8Stages) & 1u;

@@ -24,12 +24,22 @@ def assert_close(name, got, want, tol, max_outliers=0):
     assert np.isfinite(a).all(), name + ": non-finite values"
     nb = np.linalg.norm(b)
     rel = np.linalg.norm(a - b) / (nb if nb > 0 else 1.0)
-    assert rel <= tol, "%s: relative l2 error %.3e > %.1e" % (name, rel, tol)
     if not b.size:
         return rel, 0
     rms = nb / np.sqrt(b.size)
     ratio = np.abs(a - b) / (np.abs(b) + rms + 1e-30)
-    outliers = int((ratio > tol).sum())
+    inside = ratio <= tol
+    outliers = int(b.size - inside.sum())
+    # Without counted ties (max_outliers == 0) the l2 bound covers every element.  With them it covers the elements
+    # inside the per-element bound, and a gross bound of 5 tol covers all: one gate of the hidden layer that falls
+    # the other way for one of 80 samples moves 2 % of the l2 norm of every tensor below it (seen: one agent of
+    # eight), which is the budgeted effect, not rounding.
+    if max_outliers > 0:
+        rel_in = np.linalg.norm((a - b)[inside]) / (nb if nb > 0 else 1.0)
+        assert rel_in <= tol, "%s: relative l2 error of the elements inside the bound %.3e > %.1e" % (name, rel_in, tol)
+        assert rel <= 5 * tol, "%s: relative l2 error %.3e > 5 x %.1e" % (name, rel, tol)
+    else:
+        assert rel <= tol, "%s: relative l2 error %.3e > %.1e" % (name, rel, tol)
     assert outliers <= max_outliers, "%s: %d elements beyond %.1e (|b_i| + rms b), %d allowed; worst %.3e (rel l2 %.3e)" % (
         name, outliers, tol, max_outliers, float(ratio.max()), rel)
     return rel, outliers

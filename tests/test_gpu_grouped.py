@@ -184,7 +184,12 @@ def _grouped_replay(w, steps, tol_net, tol_params, mode="elementwise"):
 
 def test_grouped_replay_conv():
     # lists in arbitrary order, of different lengths, with agents that are each other's in-peers in one call
-    w = GI.WORKLOADS[1].scaled(n_agents=5, n_envs=2, n_steps=3)
+    # With six samples an agent, one hidden unit whose gate falls the other way for one sample moves every tensor
+    # below it by several per cent, far more elements than one counted tie pays for.  The 8-agent recipe at this
+    # size has such a unit (agent 4, second frame, hidden unit 0: pre-activation 2.4e-6 against an rms of 2e-2 in
+    # the oracle, below the float32 rounding of a 3136-term sum), so this test takes the 16-agent recipe, in which
+    # neither the oracle's two evaluations nor the library's disagree on a gate.
+    w = GI.WORKLOADS[2].scaled(n_agents=5, n_envs=2, n_steps=3)
     _grouped_replay(w, [[3, 0], [1], [4, 2, 0, 1], [0, 1, 2, 3, 4], [2, 4]], TOL_BF16, TOL_BF16, mode="update")
 
 
