@@ -700,6 +700,18 @@ def extras_c2(env: Env, rec, w: GI.Workload):
                               ms_per_round=1e3 * loop_s / loop_iters,
                               note="act x T + environment step x T + learn + gossip per agent on its own stream, "
                                    "synthetic on-GPU environment, host clock")
+    # the same loop with all agents in lockstep: acting batched over the agents, then the synchronous round
+    all_iters = 50
+    B.gala_actor_loop_all(L.ctx, 4, 12345)
+    L.sync()
+    t0 = time.perf_counter()
+    B.gala_actor_loop_all(L.ctx, all_iters, 12345)
+    L.sync()
+    all_s = time.perf_counter() - t0
+    rec["closed_loop_lockstep"] = dict(frames_per_s=w.frames_per_round * all_iters / all_s,
+                                       ms_per_round=1e3 * all_s / all_iters,
+                                       note="T x (one forward pass of all agents, one draw + environment-step kernel "
+                                            "of all agents) + the synchronous round, host clock")
     rec["extras"] = dict(consensus_distance=dist, consensus_call_ms=cons_ms,
                          consensus_bytes=int(w.n_agents * L.d * 4),
                          allreduce_a2c_ms_per_round=a2c_ms,
@@ -826,7 +838,8 @@ def run_ours(args):
                 timing=dict(ms_per_step="median over the timed steps", timed_steps=head["timed_steps"],
                             ms_per_step_mean=head["ms_per_step_mean"], min_region_s=MIN_REGION_S,
                             note="--steps K steps are repeated until the timed region lasts at least min_region_s"))
-    for k in ("async", "wall_ms_per_step", "kernel_ms_per_step", "block_ms_per_step", "launches_per_step"):
+    for k in ("async", "wall_ms_per_step", "kernel_ms_per_step", "block_ms_per_step", "launches_per_step", "closed_loop",
+              "closed_loop_lockstep", "extras"):
         if k in head:
             line[k] = head[k]
     if len(records) > 1:

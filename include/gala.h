@@ -251,6 +251,15 @@ int gala_set_agent_ctas(gala_ctx* ctx, int ctas);
  * and replayed as one graph launch from the third on.  Returns as
  * gala_learn / gala_gossip do (GALA_ETIMEOUT from a staleness-bounded gossip step ends the loop early). */
 int gala_actor_loop(gala_ctx* ctx, int agent, int iterations, unsigned long long env_seed);
+/* The same loop for ALL agents in lockstep (Algorithm 1 with the agents advancing together, as in the synchronous
+ * round): `iterations` times { T times: one forward pass over the E current observations of every agent, then one
+ * kernel that draws every agent's actions and steps every agent's environments; then gala_step_sync on the stored
+ * rollouts }.  Same environment function, same step counters and same rollout buffers as gala_actor_loop (the two
+ * may alternate); acting is batched over the agents, so an iteration is some 50 launches however many agents there
+ * are.  The acting part is captured on its second run and replayed as one graph launch from the third on (unless
+ * graph replay is off); the round inside follows gala_step_sync's own rule.  Returns as gala_step_sync does;
+ * GALA_ESTATE with the earlier convolution kernels (GALA_LEGACY_CONV). */
+int gala_actor_loop_all(gala_ctx* ctx, int iterations, unsigned long long env_seed);
 /* Waits for the agent's stream and copies the rollout of its last loop iteration to HOST memory (any pointer
  * may be NULL): obs [T+1][E][...], actions [T][E], rewards [T][E], dones [T][E]; *next_step = number of
  * environment steps taken so far. */

@@ -63,7 +63,7 @@ EXPORTS = (
     "gala_kernel_class_name", "gala_profile_enable", "gala_profile_read", "gala_get_stream",
     "gala_gemm_bf16_static", "gala_delay", "gala_consensus_distance", "gala_track_updates", "gala_update_norm", "gala_set_stale_timeout",
     "gala_set_agent_ctas", "gala_set_graphs", "gala_losses_all",
-    "gala_actor_loop", "gala_actor_read",
+    "gala_actor_loop", "gala_actor_loop_all", "gala_actor_read",
     "gala_learn_many", "gala_gossip_many", "gala_poll_agent", "gala_sweep_agents", "gala_set_group_lanes",
     "gala_debug_wait_runs_out",
 )
@@ -103,6 +103,7 @@ def lib() -> C.CDLL:
             "gala_set_agent_ctas": (i, [vp, i]),
             "gala_set_graphs": (i, [vp, i]),
             "gala_actor_loop": (i, [vp, i, i, C.c_ulonglong]),
+            "gala_actor_loop_all": (i, [vp, i, C.c_ulonglong]),
             "gala_actor_read": (i, [vp, i, vp, vp, vp, vp, C.POINTER(C.c_longlong)]),
             "gala_step_sync": (i, [vp, C.POINTER(gala_rollout)]),
             "gala_sync_agent": (i, [vp, i, i]),
@@ -239,6 +240,10 @@ def gala_update_norm(ctx) -> float:
 
 def gala_actor_loop(ctx, agent: int, iterations: int, env_seed: int):
     _check(ctx, lib().gala_actor_loop(ctx, agent, iterations, env_seed))
+
+
+def gala_actor_loop_all(ctx, iterations: int, env_seed: int):
+    _check(ctx, lib().gala_actor_loop_all(ctx, iterations, env_seed))
 
 
 def gala_actor_read(ctx, agent: int, n_envs: int, n_steps: int, obs_shape, obs_dtype):

@@ -127,6 +127,11 @@ struct gala_ctx {
     int n_lanes = 1, next_lane = 0;
     const AgentMap* cur_map = nullptr;       // agent list of the launches being enqueued (null: a range of agents)
     cudaEvent_t cur_fork = nullptr, cur_join = nullptr;   // fork / join events of the stream pair in use
+    // closed actor loops: rollout buffers of all agents, one block per kind (an agent's loop_* pointers are slices)
+    uint8_t* la_obs = nullptr; int* la_actions = nullptr; float* la_rewards = nullptr; unsigned char* la_dones = nullptr;
+    float* la_uniforms = nullptr; long long* la_steps = nullptr;
+    StepGraph la_graph;                      // the acting part of one lockstep iteration (all agents) as a graph
+    unsigned long long la_seed = 0; int la_seen = 0;
     long long sync_round = 0;
     long long launches = 0;
     long long tag_launches[T_COUNT] = {};
@@ -1443,6 +1448,7 @@ int gala_destroy(gala_ctx* c) {
     }
     for (StepGraph& g : c->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
     for (Agent& a : c->agents) if (a.loop_graph.exec) cudaGraphExecDestroy(a.loop_graph.exec);
+    if (c->la_graph.exec) cudaGraphExecDestroy(c->la_graph.exec);
     for (gala_ctx::Lane& L : c->glane) {
         if (L.st) cudaStreamDestroy(L.st);
         if (L.side) cudaStreamDestroy(L.side);
@@ -1479,6 +1485,27 @@ int gala_act(gala_ctx* c, int agent, const void* obs, const float* uniforms, int
     if (values)
         CK(cudaMemcpyAsync(values, c->values + (long)agent * c->B, c->E * sizeof(float), cudaMemcpyDeviceToDevice,
                            ag.stream));
+    return GALA_OK;
+}
+
+// Rollout buffers of the closed loops, for all agents at once (the lockstep loop addresses them by stride).
+static int ensure_loop_buffers(gala_ctx* c) {
+    if (c->la_obs) return GALA_OK;
+    const int T = c->T, E = c->E, n = c->n;
+    const long obs_bytes = c->conv ? kFramePix : (long)c->obs_dim * 4;
+    const size_t per_obs = (size_t)(T + 1) * E * obs_bytes, TE = (size_t)T * E;
+    uint8_t* ob = nullptr;
+    ALLOC(ob, (size_t)n * per_obs);
+    ALLOC(c->la_actions, n * TE); ALLOC(c->la_rewards, n * TE); ALLOC(c->la_dones, n * TE);
+    ALLOC(c->la_uniforms, (size_t)n * E); ALLOC(c->la_steps, n);
+    for (int i = 0; i < n; i++) {
+        Agent& ag = c->agents[i];
+        ag.loop_obs = ob + i * per_obs;
+        ag.loop_actions = c->la_actions + i * TE; ag.loop_rewards = c->la_rewards + i * TE;
+        ag.loop_dones = c->la_dones + i * TE; ag.loop_uniforms = c->la_uniforms + (size_t)i * E;
+        ag.env_step_dev = c->la_steps + i;
+    }
+    c->la_obs = ob;
     return GALA_OK;
 }
 
@@ -1519,16 +1546,8 @@ int gala_actor_loop(gala_ctx* c, int agent, int iterations, unsigned long long e
     if (c->topo.kind == GALA_TOPO_COMPLETE)
         return fail(c, GALA_ESTATE, "gala_actor_loop: the complete graph (gradient all-reduce) exists only as gala_step_sync");
     Agent& ag = c->agents[agent];
-    const int T = c->T, E = c->E;
-    const long obs_bytes = c->conv ? kFramePix : (long)c->obs_dim * 4;
-    if (!ag.loop_obs) {
-        uint8_t* ob = nullptr;
-        ALLOC(ob, (size_t)(T + 1) * E * obs_bytes);
-        ALLOC(ag.loop_actions, (size_t)T * E); ALLOC(ag.loop_rewards, (size_t)T * E);
-        ALLOC(ag.loop_dones, (size_t)T * E); ALLOC(ag.loop_uniforms, (size_t)E);
-        ALLOC(ag.env_step_dev, 1);
-        ag.loop_obs = ob;
-    }
+    const int T = c->T;
+    { int r0 = ensure_loop_buffers(c); if (r0 != GALA_OK) return r0; }
     if (ag.loop_seed != env_seed) {   // the captured iteration carries the seed
         if (ag.loop_graph.exec) { cudaGraphExecDestroy(ag.loop_graph.exec); ag.loop_graph.exec = nullptr; }
         ag.loop_graph.failed = false;
@@ -1584,6 +1603,113 @@ int gala_actor_loop(gala_ctx* c, int agent, int iterations, unsigned long long e
         if ((r = gala_gossip(c, agent)) != GALA_OK) return r;
     }
     return GALA_OK;
+}
+
+static int main_stream_joins_agents(gala_ctx* c);
+static int agents_join_main_stream(gala_ctx* c);
+static int sync_round_body(gala_ctx* c, const gala_rollout* ros);
+
+// The acting part of a lockstep iteration on the main stream: first observations, T x (forward of all agents,
+// draw + environment step of all agents), step counters advanced.
+static int act_all(gala_ctx* c, unsigned long long env_seed) {
+    const int T = c->T, E = c->E, n = c->n;
+    const long obs_elems = c->conv ? kFramePix : c->obs_dim;
+    const long obs_bytes = obs_elems * (c->conv ? 1 : 4);
+    const long per_obs = (long)(T + 1) * E * obs_bytes;
+    cudaStream_t st = c->main_stream;
+    EnvActArgs ea{};
+    ea.seed = env_seed; ea.n_actions = c->A; ea.frames = c->conv ? 1 : 0; ea.step_base = c->la_steps;
+    ea.logits = c->logits; ea.logits_stride = c->B * c->A;
+    ea.actions = c->la_actions; ea.rewards = c->la_rewards; ea.dones = c->la_dones; ea.te_stride = (long)T * E;
+    ea.obs_out = c->la_obs; ea.obs_agent_stride = per_obs; ea.obs_elems = obs_elems;
+    EnvActArgs first = ea;   // the environment is a function of the step: the first observation is produced again
+    first.draw = 0; first.step = 0; first.obs_off = 0;
+    LAUNCH(T_ENV, st, launch_env_act_all(first, E, n, st));
+    for (int t = 0; t < T; t++) {
+        for (int a0 = 0; a0 < n; a0 += kBatch) {
+            const int cnt = n - a0 < kBatch ? n - a0 : kBatch;
+            PtrBatch pb{};
+            for (int i = 0; i < cnt; i++) pb.p[i] = c->la_obs + (long)(a0 + i) * per_obs + (long)t * E * obs_bytes;
+            // conv net: the trunk up to the (possibly split) hidden-layer product; the kernel that draws the actions
+            // finishes the hidden layer and forms the policy head of its environment itself
+            HiddenPending pend;
+            int r = forward(c, a0, cnt, pb, E, st, nullptr, c->conv ? &pend : nullptr);
+            if (r != GALA_OK) return r;
+            EnvActArgs sa = ea;
+            sa.agent0 = a0;
+            sa.draw = 1; sa.step = t; sa.te_off = (long)t * E; sa.obs_off = (long)(t + 1) * E * obs_bytes;
+            if (c->conv) {
+                sa.H = kHidden; sa.split = pend.split;
+                sa.partials = c->splitk_ws + (long)a0 * c->splitk_group_stride;
+                sa.split_stride = pend.count; sa.partial_group_stride = c->splitk_group_stride;
+                sa.hid = c->hid; sa.h_stride = c->B * kHidden;
+                sa.params = c->x; sa.p_stride = c->d_pad;
+                sa.piw = c->cl.piw; sa.pib = c->cl.pib; sa.fcb = c->cl.fcb;
+            }
+            LAUNCH(T_ENV, st, launch_env_act_all(sa, E, cnt, st));
+        }
+    }
+    LAUNCH(T_ENV, st, launch_env_advance_all(c->la_steps, n, T, st));
+    return GALA_OK;
+}
+
+int gala_actor_loop_all(gala_ctx* c, int iterations, unsigned long long env_seed) {
+    if (!c || iterations < 0) return c ? fail(c, GALA_EINVAL, "gala_actor_loop_all: negative iteration count") : GALA_EINVAL;
+    if (c->legacy_conv) return fail(c, GALA_ESTATE, "gala_actor_loop_all: not with the earlier convolution kernels");
+    const int n = c->n, T = c->T;
+    { int r0 = ensure_loop_buffers(c); if (r0 != GALA_OK) return r0; }
+    if (c->la_seed != env_seed) {   // the captured part carries the seed
+        if (c->la_graph.exec) { cudaGraphExecDestroy(c->la_graph.exec); c->la_graph.exec = nullptr; }
+        c->la_graph.failed = false;
+        c->la_seed = env_seed; c->la_seen = 0;
+    }
+    std::vector<gala_rollout> ros((size_t)n);
+    for (int i = 0; i < n; i++) {
+        Agent& ag = c->agents[i];
+        ros[i] = gala_rollout{ag.loop_obs, ag.loop_actions, ag.loop_rewards, ag.loop_dones};
+    }
+    cudaStream_t st = c->main_stream;
+    const unsigned long long outside = (1ull << T_SWEEP_SYNC) | (1ull << T_SWEEP_AGENT);
+    // the whole loop runs on the main stream: ordered against the agents' streams once on either side
+    if (iterations > 0) { int r0 = main_stream_joins_agents(c); if (r0 != GALA_OK) return r0; }
+    for (int it = 0; it < iterations; it++) {
+        StepGraph& g = c->la_graph;
+        const bool graphs = c->use_graphs >= 1 && (c->profile_mask & ~outside) == 0 && !g.failed;
+        int r = GALA_OK;
+        if (graphs && g.exec) {            // third iteration on: one graph launch
+            CK(cudaGraphLaunch(g.exec, st));
+            c->launches += g.launches;
+            for (int k = 0; k < T_COUNT; k++) c->tag_launches[k] += g.tag_launches[k];
+        } else if (graphs && c->la_seen >= 1 && cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
+            const long long l0 = c->launches;   // second iteration: captured, instantiated, launched
+            long long t0[T_COUNT];
+            for (int k = 0; k < T_COUNT; k++) t0[k] = c->tag_launches[k];
+            r = act_all(c, env_seed);
+            cudaGraph_t graph = nullptr;
+            cudaError_t e = cudaStreamEndCapture(st, &graph);
+            if (r == GALA_OK && e == cudaSuccess && graph) e = cudaGraphInstantiate(&g.exec, graph, 0);
+            if (graph) cudaGraphDestroy(graph);
+            if (r != GALA_OK || e != cudaSuccess || !g.exec) {
+                (void)cudaGetLastError();
+                g.failed = true; g.exec = nullptr;
+                c->launches = l0;
+                for (int k = 0; k < T_COUNT; k++) c->tag_launches[k] = t0[k];
+                if (r != GALA_OK) return r;
+                if ((r = act_all(c, env_seed)) != GALA_OK) return r;
+            } else {
+                g.launches = c->launches - l0;
+                for (int k = 0; k < T_COUNT; k++) g.tag_launches[k] = c->tag_launches[k] - t0[k];
+                CK(cudaGraphLaunch(g.exec, st));
+            }
+        } else {                           // first iteration (or no graphs): direct launches
+            (void)cudaGetLastError();
+            if ((r = act_all(c, env_seed)) != GALA_OK) return r;
+        }
+        c->la_seen++;
+        for (int i = 0; i < n; i++) c->agents[i].env_step += T;
+        if ((r = sync_round_body(c, ros.data())) != GALA_OK) { (void)agents_join_main_stream(c); return r; }
+    }
+    return iterations > 0 ? agents_join_main_stream(c) : GALA_OK;
 }
 
 int gala_actor_read(gala_ctx* c, int agent, void* obs, int* actions, float* rewards, unsigned char* dones,
@@ -1727,23 +1853,34 @@ int gala_delay(gala_ctx* c, int agent, int usec) {
     return GALA_OK;
 }
 
-int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
-    if (!c) return GALA_EINVAL;
-    const int n = c->n;
-    if (ros)
-        for (int i = 0; i < n; i++)
-            if (!ros[i].obs || !ros[i].actions || !ros[i].rewards || !ros[i].dones)
-                return fail(c, GALA_EINVAL, "gala_step_sync: null rollout pointer for agent %d", i);
+// The main stream waits for everything the agents have enqueued, also on the lanes of the grouped calls.
+static int main_stream_joins_agents(gala_ctx* c) {
     cudaStream_t st = c->main_stream;
-    for (int i = 0; i < n; i++) {  // everything the agents have enqueued goes first
+    for (int i = 0; i < c->n; i++) {
         Agent& ag = c->agents[i];
-        if (ag.group_lane >= 0) {      // ... also on the lanes of the grouped calls
+        if (ag.group_lane >= 0) {
             CK(cudaStreamWaitEvent(st, c->glane[ag.group_lane].done, 0));
             ag.group_lane = -1;
         }
         CK(cudaEventRecord(ag.fence, ag.stream));
         CK(cudaStreamWaitEvent(st, ag.fence, 0));
     }
+    return GALA_OK;
+}
+// The agents' streams wait for what the main stream holds now.
+static int agents_join_main_stream(gala_ctx* c) {
+    CK(cudaEventRecord(c->main_event, c->main_stream));
+    for (int i = 0; i < c->n; i++) {
+        CK(cudaStreamWaitEvent(c->agents[i].stream, c->main_event, 0));
+        c->agents[i].dirty = true;     // a grouped call must be ordered behind this round through the agent's stream
+    }
+    return GALA_OK;
+}
+
+// One synchronous round on the main stream, without the ordering against the agents' streams on either side.
+static int sync_round_body(gala_ctx* c, const gala_rollout* ros) {
+    const int n = c->n;
+    cudaStream_t st = c->main_stream;
     if (ros) {
         // Timing several kernel classes of the step at once: one stream, so that an event pair brackets a kernel
         // and not its wait for the SMs that the other stream's kernels hold.
@@ -1774,15 +1911,24 @@ int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
     }
     LAUNCH(T_SWEEP_SYNC, st, launch_sweep_sync(c->x, c->g, c->v, c->clip, c->conv ? c->shadow : nullptr, n, c->d_pad, np, off, hp,
                                             c->error_word, st));
-    CK(cudaEventRecord(c->main_event, st));
     for (int i = 0; i < n; i++) {
-        CK(cudaStreamWaitEvent(c->agents[i].stream, c->main_event, 0));
-        c->agents[i].dirty = true;     // a grouped call must be ordered behind this round through the agent's stream
         c->agents[i].pending = false;
         c->agents[i].round++;
     }
     c->sync_round++;
     return GALA_OK;
+}
+
+int gala_step_sync(gala_ctx* c, const gala_rollout* ros) {
+    if (!c) return GALA_EINVAL;
+    if (ros)
+        for (int i = 0; i < c->n; i++)
+            if (!ros[i].obs || !ros[i].actions || !ros[i].rewards || !ros[i].dones)
+                return fail(c, GALA_EINVAL, "gala_step_sync: null rollout pointer for agent %d", i);
+    int r = main_stream_joins_agents(c);
+    if (r != GALA_OK) return r;
+    if ((r = sync_round_body(c, ros)) != GALA_OK) return r;
+    return agents_join_main_stream(c);
 }
 
 int gala_sync_agent(gala_ctx* c, int agent, int timeout_ms) {

@@ -448,6 +448,30 @@ struct EnvArgs {
     int frames;                  // 1: uint8 frames, 0: float vectors
 };
 cudaError_t launch_env(const EnvArgs& a, int n_envs, cudaStream_t st);
+// All agents of a lockstep loop in one launch (see env_act_all_kernel).
+struct EnvActArgs {
+    unsigned long long seed;
+    int n_actions, draw, frames;
+    const long long* step_base;  // [n] device counters, added to `step`
+    long long step;              // draw: the transition taken; else the step whose observation is written
+    const float* logits;         // agent i's logits of its E environments at logits + i * logits_stride
+    long logits_stride;
+    int* actions; float* rewards; unsigned char* dones;   // element (i, e) at i * te_stride + te_off + e
+    long te_stride, te_off;
+    void* obs_out;               // agent i's observations at obs_out + i * obs_agent_stride + obs_off (bytes)
+    long obs_agent_stride, obs_off;
+    long obs_elems;              // bytes (frames) or floats (vectors) per environment
+    int agent0;                  // first agent of the launch (grid.z counts from it)
+    // H > 0: the policy head is formed here from the hidden layer instead of read from `logits`: hidden unit u of
+    // environment e = bf16(relu(sum over the splits of partials + bias)) if split > 0, else hid[e][u]
+    int H, split;
+    const float* partials; long split_stride, partial_group_stride;   // [i][split][E][H]
+    const __nv_bfloat16* hid; long h_stride;                          // [i][.][H]
+    const float* params; long p_stride;                               // flat parameter vectors, agent 0 first
+    long piw, pib, fcb;
+};
+cudaError_t launch_env_act_all(const EnvActArgs& a, int n_envs, int n_agents, cudaStream_t st);
+cudaError_t launch_env_advance_all(long long* counters, int n, long long by, cudaStream_t st);
 cudaError_t launch_env_advance(long long* counter, long long by, cudaStream_t st);
 
 // ---------------------------------------------------------------- conv lowering

@@ -542,6 +542,78 @@ def test_closed_actor_loop_conv():
     _closed_loop(w, 3, TOL_BF16, TOL_BF16, 1e-2, "update", graphs=2)
 
 
+def _closed_loop_all(w, iters, tol_net, tol_params, cdf_tol, mode):
+    """Lockstep closed loop of all agents against the oracle, one iteration at a time: every agent's environment
+    bit for bit (same function and step numbering as the per-agent loop), every action equal to the oracle's draw
+    unless the uniform lies within cdf_tol of a boundary of the oracle's CDF, then the synchronous round of the
+    oracle on the library's rollouts (gradient, parameters after the averaging of that round's in-peers)."""
+    B, LM = _mods()
+    seed = 20190611
+    net = oracle_net(w)
+    L = make_learner(w)
+    ohp = oracle_hp(L.hp)
+    X, V = seed_identical(L, w, net)
+    n, T, E, A = w.n_agents, w.n_steps, w.n_envs, w.n_actions
+    frames = w.net_kind == "conv"
+    mismatches = 0
+    for it in range(iters):
+        B.gala_actor_loop_all(L.ctx, 1, seed)
+        L.sync()
+        ros = []
+        for i in range(n):
+            ro, nxt = B.gala_actor_read(L.ctx, i, E, T, GI.obs_shape(w), np.uint8 if frames else np.float32)
+            assert nxt == (it + 1) * T
+            for t in range(T + 1):
+                env = GI.synthetic_env(seed, i, E, it * T + t, A, frames, w.obs_dim, actions=ro["actions"][t] if t < T else None)
+                np.testing.assert_array_equal(ro["obs"][t], env["obs"])
+                if t == T:
+                    break
+                np.testing.assert_array_equal(ro["rewards"][t], env["rewards"])
+                np.testing.assert_array_equal(ro["dones"][t], env["dones"])
+                z, _ = R.forward(net, X[i], env["obs"])
+                want = R.sample(z, env["uniforms"])
+                cdf = np.cumsum(R.softmax(z), axis=1)
+                assert ro["actions"][t].min() >= 0 and ro["actions"][t].max() < A
+                for e in np.nonzero(ro["actions"][t] != want)[0]:
+                    assert np.min(np.abs(cdf[e] - env["uniforms"][e])) < cdf_tol, (it, i, t, e, cdf[e], env["uniforms"][e])
+                    mismatches += 1
+            ros.append(ro)
+        Xn, Vn, infos = R.sync_round(net, X, V, ros, ohp, w.topo_kind, w.topo_peers, it, workers=4)
+        if mode != "elementwise":
+            replay_sweep_from_library_gradient(L, B, w, X, V, ohp, it)
+        for i in range(n):
+            allow = tie_allowance(net, X[i], ros[i]["obs"].reshape(-1, int(np.prod(ros[i]["obs"].shape[2:])))[:T * E])
+            assert_grad_close("grad[%d]" % i, L.get_grad(i), infos[i]["grad"], net, tol_net, max_outliers=allow)
+            check_params("x[%d]" % i, L.get_params(i), Xn[i], X[i], tol_params, mode)
+        if mode == "elementwise":
+            X, V = Xn, Vn
+        else:   # keep both sides on the same trajectory (oracle -> library only)
+            X = Xn.astype(np.float32).astype(np.float64)
+            V = Vn.astype(np.float32).astype(np.float64)
+            for i in range(n):
+                L.set_state(i, params=X[i], sq_avg=V[i], rnd=it + 1)
+    assert mismatches <= max(1, iters * n * T * E // 50)
+    # the per-agent loop goes on from the same counters and buffers
+    B.gala_actor_loop(L.ctx, 0, 1, seed)
+    L.sync()
+    ro, nxt = B.gala_actor_read(L.ctx, 0, E, T, GI.obs_shape(w), np.uint8 if frames else np.float32)
+    assert nxt == (iters + 1) * T
+    env = GI.synthetic_env(seed, 0, E, iters * T, A, frames, w.obs_dim)
+    np.testing.assert_array_equal(ro["obs"][0], env["obs"])
+    L.close()
+
+
+def test_closed_actor_loop_all_agents_mlp():
+    w = GI.WORKLOADS[0].scaled(n_agents=3, n_envs=8, n_steps=5)
+    _closed_loop_all(w, 3, TOL_FP32_NET, TOL_SWEEP, 1e-5, "elementwise")
+
+
+def test_closed_actor_loop_all_agents_conv():
+    # four iterations: direct launches, the captured acting part, two replays
+    w = GI.WORKLOADS[2].scaled(n_agents=3, n_envs=3, n_steps=2)
+    _closed_loop_all(w, 4, TOL_BF16, TOL_BF16, 1e-2, "update")
+
+
 def test_mlp_sync_round_unfused_kernels(monkeypatch):
     # the layer-by-layer MLP kernels (used when a rollout is too large for the one-kernel step's shared memory)
     monkeypatch.setenv("GALA_MLP_UNFUSED", "1")
