@@ -148,6 +148,7 @@ struct gala_ctx {
     unsigned *norm_ticket = nullptr, *colsum_ticket = nullptr, *heads_ticket = nullptr;
     float* c1b = nullptr;                    // bias-gradient slices of conv1, left by conv2's data gradient
     long c1b_min_samples = 2048;             // ... in launches over at least this many samples
+    int fc_bn = 128;                         // columns of a tile of the hidden layer's forward product
     float* fc_sq = nullptr;                  // [N][1600] sums of squares of the hidden layer's weight gradient, by 32 x 32 block
     float* dzv = nullptr;                    // [N][S][20] rows (dlogits, dvalue, zeros) of the fused heads kernel
     float* heads_partial = nullptr;          // [N][E][4] objective sums per block of the fused heads kernel
@@ -437,9 +438,13 @@ int build_plans(gala_ctx* c) {
         Plan& f = c->fc_fwd;
         zero_args(f);
         f.tag = T_GEMM_FC_FWD;
+        // forward: 128 x 256 tiles (one CTA an SM; a quarter less operand traffic from L2, which bounds this product
+        // with its 3136-long reduction) once an agent's batch fills several row tiles; 128 x 128 below that, where
+        // the number of CTAs matters more
+        const int fbn = c->fc_bn;
         ok &= make_operand(&f.A, c->act[2], 0, B, kFeat, n, kFeat, (uint64_t)B * kFeat, 128);
-        ok &= make_operand(&f.B, c->shadow + c->cl.fcw, 0, kHidden, kFeat, n, kFeat, dp, 128);
-        f.args.M = (int)B; f.args.N = kHidden; f.args.K = kFeat; f.args.block_n = 128;
+        ok &= make_operand(&f.B, c->shadow + c->cl.fcw, 0, kHidden, kFeat, n, kFeat, dp, fbn);
+        f.args.M = (int)B; f.args.N = kHidden; f.args.K = kFeat; f.args.block_n = fbn;
         f.args.flags = EPI_OUT_BF16 | EPI_RELU;
         f.args.bias = c->x + c->cl.fcb; f.args.bias_group_stride = dp;
         f.args.out = c->hid; f.args.out_group_stride = B * kHidden; f.args.ldc = kHidden;
@@ -449,7 +454,7 @@ int build_plans(gala_ctx* c) {
         w.tag = T_GEMM_FC_WGRAD;
         ok &= make_operand(&w.A, c->dh, 1, kHidden, S, n, kHidden, (uint64_t)S * kHidden, 128);
         ok &= make_operand(&w.B, c->act[2], 1, kFeat, S, n, kFeat, (uint64_t)B * kFeat, 128);
-        w.args.M = kHidden; w.args.N = kFeat; w.args.K = (int)S; w.args.block_n = 128;
+        w.args.M = kHidden; w.args.N = kFeat; w.args.K = (int)S; w.args.block_n = 128;   // (bound by its epilogue: no gain from wider tiles)
         w.args.out = c->g + c->cl.fcw; w.args.out_group_stride = dp; w.args.ldc = kFeat;
         w.args.sq_partial = c->fc_sq;   // so that the norm pass need not read these 95 % of the gradient again
         // data gradient: dh [S][512] x Wfc [512][3136] -> dY3 [S][3136], masked by act3 > 0
@@ -621,7 +626,7 @@ int run_plan(gala_ctx* c, const Plan& p, int agent0, int groups, int m_override,
     a.out = reinterpret_cast<char*>(a.out) + (long)agent0 * a.out_group_stride * (bf ? 2 : 4);
     if (a.mask) a.mask += (long)agent0 * a.mask_group_stride;
     if (a.gate) a.gate += (long)agent0 * a.gate_group_stride;
-    if (a.sq_partial) a.sq_partial += (long)agent0 * ((a.M + 127) / 128) * ((a.N + a.block_n - 1) / a.block_n) * 16;
+    if (a.sq_partial) a.sq_partial += (long)agent0 * ((a.M + 127) / 128) * ((a.N + a.block_n - 1) / a.block_n) * (a.block_n / 8);
     LAUNCH(p.tag, st, launch_gemm(p.A, p.B, a, st));
     return GALA_OK;
 }
@@ -677,7 +682,7 @@ int forward(gala_ctx* c, int agent0, int groups, const PtrBatch& obs, int rows, 
         int r;
         {
             const Plan& p = c->fc_fwd;
-            const int tiles = ((rows + 127) / 128) * (kHidden / 128);
+            const int tiles = ((rows + 127) / 128) * (kHidden / p.args.block_n);
             int split = (c->cur_ctas > 0 ? 2 * c->cur_ctas : 2 * sm_count()) / (groups * tiles);
             if (split > 7) split = 7;
             while (split > 1 && (long)split * rows * kHidden > c->splitk_group_stride) split--;
@@ -1366,6 +1371,8 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         c->fused_heads = heads_fused_supported(c->T, c->E, c->A, kHidden) && getenv("GALA_HEADS_UNFUSED") == nullptr;
         ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
         ALLOC(c->dzv, (size_t)n * S * 20);
+        c->fc_bn = c->B >= 256 ? 256 : 128;
+        if (const char* e = getenv("GALA_FC_BN")) { const int v = atoi(e); if (v == 128 || v == 256) c->fc_bn = v; }
         ALLOC(c->fc_sq, (size_t)n * (kHidden / 128) * ((kFeat + 127) / 128) * 16);
         ALLOC(c->c1b, (size_t)n * kConvBiasSliceStride);
         if (const char* e = getenv("GALA_C1B_SLICES")) c->c1b_min_samples = atoi(e) ? 0 : (1L << 60);
@@ -2255,7 +2262,7 @@ int gala_gemm_bf16(const void* A, const void* B, float* D, int groups, int M, in
     if ((K % 8) || (a_mn && (M % 8)) || (b_mn && (N % 8))) return GALA_EINVAL;
     if (gemm_init() != cudaSuccess) return GALA_ECUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const int bn = b_mn ? (N > 64 ? 128 : 64) : (N > 64 ? 128 : (N > 32 ? 64 : 32));
+    const int bn = N >= 512 ? 256 : b_mn ? (N > 64 ? 128 : 64) : (N > 64 ? 128 : (N > 32 ? 64 : 32));
     GemmOperand oa, ob;
     if (!make_operand(&oa, A, a_mn, M, K, groups, a_mn ? M : K, (uint64_t)M * K, 128)) return GALA_ECUDA;
     if (!make_operand(&ob, B, b_mn, N, K, groups, b_mn ? N : K, (uint64_t)N * K, bn)) return GALA_ECUDA;

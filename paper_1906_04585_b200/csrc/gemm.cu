@@ -28,7 +28,7 @@ constexpr int BK = 64;           // K per stage = one 128-byte swizzle atom of b
 constexpr int kStages = 4;
 constexpr int kStageA = BM * BK * 2;    // 16 KiB
 constexpr int kStageB = 128 * BK * 2;   // room for block_n = 128
-constexpr int kSmemBytes = 200 * 1024;   // most dynamic shared memory a launch may ask for
+constexpr int kSmemBytes = 216 * 1024;   // most dynamic shared memory a launch may ask for (four stages of a 128 x 256 tile)
 
 // ------------------------------------------------------------------ kernel
 // Work decomposition shared by the three roles: tile index -> (group, split, m-tile, n-tile), n fastest
@@ -214,7 +214,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (lane < 2) {          // A: one box (K-major) or two 64-wide boxes (MN-major)
                         if (!a_mn) { if (lane == 0) tma_load_3d(a, &tmA, &full_bar[s], k0, t.m0, group); }
                         else tma_load_3d(a + lane * 8192, &tmA, &full_bar[s], t.m0 + 64 * lane, k0, group);
-                    } else if (lane < 4) {   // B likewise
+                    } else if (lane < 6) {   // B likewise (up to four boxes for 256 columns)
                         const int j = lane - 2;
                         if (!b_mn) { if (j == 0) tma_load_3d(b, &tmB, &full_bar[s], k0, t.n0, group); }
                         else if (j < BN / 64) tma_load_3d(b + j * 8192, &tmB, &full_bar[s], t.n0 + 64 * j, k0, group);
@@ -305,16 +305,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int ab = local & 1;
             // gate words of this thread's row (one per 32 columns): they depend only on the tile, so they are
             // fetched before the wait for the MMAs
-            uint32_t gw0 = 0xffffffffu, gw1 = 0xffffffffu, gw2 = 0xffffffffu, gw3 = 0xffffffffu;
+            uint32_t gws[8];
+#pragma unroll
+            for (int j = 0; j < 8; j++) gws[j] = 0xffffffffu;
             if (p.flags & EPI_GATE) {
                 const int m = t.m0 + q * 32 + lane;
                 if (m < p.M) {
                     const uint32_t* gp = p.gate + (long)agent_slot(p.am, t.gz) * p.gate_group_stride + (long)m * (p.N >> 5) + (t.n0 >> 5);
                     const int nw = (p.N - t.n0) >> 5;
-                    if (nw > 0) gw0 = __ldg(gp);
-                    if (nw > 1 && BN > 32) gw1 = __ldg(gp + 1);
-                    if (nw > 2 && BN > 64) gw2 = __ldg(gp + 2);
-                    if (nw > 3 && BN > 96) gw3 = __ldg(gp + 3);
+#pragma unroll
+                    for (int j = 0; j < 8; j++)
+                        if (j < nw && 32 * j < BN) gws[j] = __ldg(gp + j);
                 }
             }
             if (!mbar_wait(&acc_full[ab], ((uint32_t)local >> 1) & 1u, &abort_flag)) break;
@@ -345,14 +346,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     for (int j = 0; j < 32; j++) r[j] = 0u;
                 }
                 if (p.flags & EPI_GATE) {
-                    const uint32_t gw = c0 == 0 ? gw0 : c0 == 32 ? gw1 : c0 == 64 ? gw2 : gw3;
+                    uint32_t gw = gws[0];
+#pragma unroll
+                    for (int j = 1; j < 8; j++)
+                        if (c0 == 32 * j) gw = gws[j];
 #pragma unroll
                     for (int j = 0; j < 32; j++)
                         if (!((gw >> j) & 1u)) r[j] = 0u;
                 }
                 const int nb = t.n0 + c0;
                 if (mw >= p.M || q * 32 >= p.tile_rows || nb >= p.N) {   // warp-uniform
-                    if (p.sq_partial && lane == 0) p.sq_partial[sq_tile * 16 + q * 4 + (c0 >> 5)] = 0.0f;
+                    if (p.sq_partial && lane == 0) p.sq_partial[sq_tile * (BN >> 3) + q * (BN >> 5) + (c0 >> 5)] = 0.0f;
                     continue;
                 }
                 if (transpose) {
@@ -427,7 +431,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     }
                     if (p.sq_partial) {   // rows of the block added by a butterfly: the same tree every time
                         for (int o = 16; o > 0; o >>= 1) row_sq += __shfl_xor_sync(0xffffffffu, row_sq, o);
-                        if (lane == 0) p.sq_partial[sq_tile * 16 + q * 4 + (c0 >> 5)] = row_sq;
+                        if (lane == 0) p.sq_partial[sq_tile * (BN >> 3) + q * (BN >> 5) + (c0 >> 5)] = row_sq;
                     }
                     continue;
                 }
@@ -794,10 +798,12 @@ bool make_operand(GemmOperand* op, const void* base, int mn_major, uint64_t mn_e
 }
 
 cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, cudaStream_t st) {
-    if (args.block_n != 32 && args.block_n != 64 && args.block_n != 128) return cudaErrorInvalidValue;
+    if (args.block_n != 32 && args.block_n != 64 && args.block_n != 128 &&
+        !(args.block_n == 256 && args.conv_mode == CONV_NONE))
+        return cudaErrorInvalidValue;
     if (B.mn_major && args.block_n < 64 && !(args.conv_mode != CONV_NONE && args.conv_layer == 0)) return cudaErrorInvalidValue;
     if (args.split_k < 1 || args.groups < 1 || args.M < 1 || args.N < 1 || args.K < 1) return cudaErrorInvalidValue;
-    if (args.sq_partial && (args.block_n != 128 || args.split_k != 1 || (args.N & 31) || (args.ldc & 7) ||
+    if (args.sq_partial && ((args.block_n != 128 && args.block_n != 256) || args.split_k != 1 || (args.N & 31) || (args.ldc & 7) ||
                             (args.flags & (EPI_OUT_BF16 | EPI_TRANSPOSE | EPI_MASK | EPI_ROWMAP_S2)) ||
                             (reinterpret_cast<uintptr_t>(args.out) & 31) || (args.out_group_stride & 7) ||
                             args.conv_mode != CONV_NONE))
@@ -850,7 +856,7 @@ cudaError_t launch_gemm(const GemmOperand& A, const GemmOperand& B, const GemmAr
     size_t smem = (size_t)a.stages * (a.stage_a_bytes + a.stage_b_bytes) + 4 * kEpiWarpBytes + 1024;
     // two resident CTAs per SM (two producers, two MMA issuers, eight epilogue warps) beat one CTA
     // with a deeper ring: shrink the ring until two fit
-    while (smem > (size_t)(110 * 1024) && a.stages > 2) {
+    while (a.block_n < 256 && smem > (size_t)(110 * 1024) && a.stages > 2) {
         a.stages--;
         smem = (size_t)a.stages * (a.stage_a_bytes + a.stage_b_bytes) + 4 * kEpiWarpBytes + 1024;
     }

@@ -112,7 +112,7 @@ struct GemmArgs {
     int max_ctas;          // > 0: at most this many CTAs (leaves SMs to kernels of other streams)
     AgentMap am;           // agents behind the groups (operands, outputs, bias, mask, gate, sq_partial)
     // Optional sums of squares of the stored outputs (for a gradient norm without a second pass over this
-    // product): slot [tile * 16 + warp quarter * 4 + 32-column block] of sq_partial gets the sum over that
+    // product): slot [tile * (block_n / 8) + warp quarter * (block_n / 32) + 32-column block] of sq_partial gets the sum over that
     // 32 x 32 block (0 where the block lies outside the matrix).  Needs block_n = 128, split_k = 1, fp32 row-major
     // output with 32-byte aligned rows and N a multiple of 32; tile = (group * m_tiles + m_tile) * n_tiles + n_tile.
     float* sq_partial;

@@ -81,7 +81,7 @@ extern "C" int gala_gemm_bf16_static(const void* A, const void* B, float* D, int
     float* ws = scratch + kHeaderFloats;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
-    const int bn = b_mn ? (N > 64 ? 128 : 64) : (N > 64 ? 128 : (N > 32 ? 64 : 32));
+    const int bn = N >= 512 ? 256 : b_mn ? (N > 64 ? 128 : 64) : (N > 64 ? 128 : (N > 32 ? 64 : 32));
     GemmOperand oa, ob;
     if (!make_operand(&oa, A, a_mn, M, K, groups, a_mn ? M : K, (uint64_t)M * K, 128) ||
         !make_operand(&ob, B, b_mn, N, K, groups, b_mn ? N : K, (uint64_t)N * K, bn)) {

@@ -32,6 +32,8 @@ GEMM_CASES = [
     (1, 256, 32, 6400, 1, 1, 7),      # conv1 weight gradient: N = 32 inside a 64-wide box
     (1, 256, 40, 200, 1, 0, 2),       # mixed: A stored [K][M], B stored [N][K]
     (1, 130, 130, 72, 0, 0, 3),       # more splits than K tiles
+    (2, 300, 640, 200, 0, 0, 1),      # 256-column tiles (N >= 512): ragged M, N = 2.5 tiles, K tail
+    (1, 264, 768, 520, 1, 0, 3),      # 256-column tiles with split reduction, A stored [K][M]
 ]
 
 
