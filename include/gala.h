@@ -115,11 +115,13 @@ typedef struct {
  * to 0, round counters to 0.  Uses the current CUDA device.
  * Environment variables read here select older or alternative kernels for the same results; they exist so that
  * two independent implementations can be compared with each other and with the CPU oracle:
- *   GALA_CONV_LEGACY     convolution products with one tensor copy per kernel offset and bf16 frame copies
  *   GALA_HEADS_UNFUSED   separate kernels for heads, objective and head gradients
  *   GALA_MLP_UNFUSED     separate kernels for the small fully connected network
  *   GALA_C1B_SLICES=0/1  conv1's bias gradient from column sums of dY1 / from conv2's data-gradient kernel
- *                        (default: the latter for launches over at least 2048 samples) */
+ *                        (default: the latter for launches over at least 2048 samples)
+ *   GALA_FC_BN=128/256   columns of an output tile of the hidden layer's forward product
+ * A build of the same sources with GALA_CROSS_CHECK defined (libgala_check.so, loaded by one test only) also knows
+ *   GALA_CONV_LEGACY     convolution products with one tensor copy per kernel offset and bf16 frame copies */
 int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* net,
                 const gala_hparams* hp, gala_ctx** out);
 int gala_destroy(gala_ctx* ctx);
@@ -258,7 +260,7 @@ int gala_actor_loop(gala_ctx* ctx, int agent, int iterations, unsigned long long
  * may alternate); acting is batched over the agents, so an iteration is some 50 launches however many agents there
  * are.  The acting part is captured on its second run and replayed as one graph launch from the third on (unless
  * graph replay is off); the round inside follows gala_step_sync's own rule.  Returns as gala_step_sync does;
- * GALA_ESTATE with the earlier convolution kernels (GALA_LEGACY_CONV). */
+ * GALA_ESTATE with the earlier convolution kernels (cross-check build only). */
 int gala_actor_loop_all(gala_ctx* ctx, int iterations, unsigned long long env_seed);
 /* Waits for the agent's stream and copies the rollout of its last loop iteration to HOST memory (any pointer
  * may be NULL): obs [T+1][E][...], actions [T][E], rewards [T][E], dones [T][E]; *next_step = number of

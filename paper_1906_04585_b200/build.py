@@ -12,6 +12,10 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgala.so")
+# The same sources with GALA_CROSS_CHECK defined: the only library in which the environment variable
+# GALA_CONV_LEGACY selects the earlier convolution products (a second implementation that one test compares
+# with the oracle).  Nothing but that test loads it.
+CHECK_LIB = os.path.join(HERE, "libgala_check.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 
 FLAGS = [
@@ -26,9 +30,9 @@ def sources():
 
 
 def _stale() -> bool:
-    if not os.path.exists(LIB):
+    if not os.path.exists(LIB) or not os.path.exists(CHECK_LIB):
         return True
-    t = os.path.getmtime(LIB)
+    t = min(os.path.getmtime(LIB), os.path.getmtime(CHECK_LIB))
     deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
     return any(os.path.getmtime(p) > t for p in deps)
 
@@ -44,6 +48,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         objs.append(obj)
         cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+    api_src = os.path.join(CSRC, "api.cu")
+    api_check = os.path.join(HERE, "_build", "api.cu.check.o")
+    procs.append((api_src + " (cross-check)", subprocess.Popen(
+        [NVCC] + FLAGS + ["-DGALA_CROSS_CHECK", "-c", api_src, "-o", api_check],
+        stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for src, p in procs:
         out, _ = p.communicate()
@@ -55,6 +64,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + ".tmp.%d" % os.getpid()
     subprocess.check_call([NVCC, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
     os.replace(tmp, LIB)
+    check_objs = [api_check if os.path.basename(o) == "api.cu.o" else o for o in objs]
+    tmp = CHECK_LIB + ".tmp.%d" % os.getpid()
+    subprocess.check_call([NVCC, "-shared", "-o", tmp] + check_objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
+    os.replace(tmp, CHECK_LIB)
     return LIB
 
 

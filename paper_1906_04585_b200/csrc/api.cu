@@ -118,6 +118,10 @@ struct gala_ctx {
     // second stream of the synchronous mode: the weight gradients of heads, hidden layer, conv3 and conv2 run beside the chain
     // of data gradients they do not depend on
     cudaStream_t side_stream = nullptr;
+    // third stream of the synchronous mode: the column sums (bias gradients) run beside conv1's weight gradient, both
+    // behind the last data gradient
+    cudaStream_t tail_stream = nullptr;
+    cudaEvent_t ev_tail_fork = nullptr, ev_tail_join = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // Streams of the grouped per-agent calls (gala_learn_many / gala_gossip_many): a launch set for a list of agents
     // goes to one lane (its stream, a side stream for the weight gradients); consecutive calls alternate between the
@@ -852,9 +856,15 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
         // The chain ends with conv2's data gradient, the second stream is still busy with weight gradients
         // then: conv1's weight gradient, its slice sum and the column sums follow the chain on `st`.
         const bool tail_on_chain = side && !c->legacy_conv;
+        // ... the column sums on a third stream beside conv1's weight gradient (synchronous round only)
+        const bool tail_third = tail_on_chain && st == c->main_stream && side == c->side_stream;
         for (int l = 2; l >= 0; l--) {
             if (l == 0 && tail_on_chain) {
                 if ((r = flush_pending_reduces(c, agent0, groups, ws)) != GALA_OK) return r;
+                if (tail_third) {   // the column sums need dh and dY1, both complete here
+                    CK(cudaEventRecord(c->ev_tail_fork, st));
+                    CK(cudaStreamWaitEvent(c->tail_stream, c->ev_tail_fork, 0));
+                }
                 if ((r = run_conv1_wgrad(c, agent0, groups, obs, st)) != GALA_OK) return r;
                 if ((r = flush_pending_reduces(c, agent0, groups, st)) != GALA_OK) return r;
                 break;
@@ -883,7 +893,7 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
                 jobs.j[1 + k] = {c->dy[l] + (long)agent0 * S * P[l] * kConvCout[l], S * P[l] * kConvCout[l], S * P[l],
                                  kConvCout[l], c->cl.b[l]};
             }
-            cudaStream_t cs = tail_on_chain ? st : ws;
+            cudaStream_t cs = tail_third ? c->tail_stream : tail_on_chain ? st : ws;
             if (!tail_on_chain && (r = fork()) != GALA_OK) return r;
             ColsumSlices sl{c->c1b + (long)agent0 * kConvBiasSliceStride, c->cl.b[0],
                             conv_grid((long)groups * S, c->cur_ctas), (int)S};
@@ -895,9 +905,13 @@ int learn_range(gala_ctx* c, int agent0, int groups, const gala_rollout* ro, cud
                                                c->colsum_ticket + (long)agent0 * kColsumJobs, groups, cs,
                                                slices ? &sl : nullptr, c->cur_map));
         }
-        if (side) {   // join: the gradient is complete when both streams are done
+        if (side) {   // join: the gradient is complete when all streams are done
             CK(cudaEventRecord(c->cur_join, side));
             CK(cudaStreamWaitEvent(st, c->cur_join, 0));
+            if (tail_third) {
+                CK(cudaEventRecord(c->ev_tail_join, c->tail_stream));
+                CK(cudaStreamWaitEvent(st, c->ev_tail_join, 0));
+            }
         }
     } else {
         const int H = c->H;
@@ -1326,6 +1340,9 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
     CK(cudaStreamCreateWithFlags(&c->main_stream, cudaStreamNonBlocking));
     CK(cudaEventCreateWithFlags(&c->main_event, cudaEventDisableTiming));
     CK(cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking));
+    CK(cudaStreamCreateWithFlags(&c->tail_stream, cudaStreamNonBlocking));
+    CK(cudaEventCreateWithFlags(&c->ev_tail_fork, cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&c->ev_tail_join, cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
     c->cur_fork = c->ev_fork; c->cur_join = c->ev_join;
@@ -1366,7 +1383,11 @@ int gala_create(int n_agents, const gala_topology* topo, const gala_net_spec* ne
         CK(conv_init());
         CK(wgrad_init());
         CK(wgrad1_init());
+#ifdef GALA_CROSS_CHECK
+        // Only in the cross-check build of the library (libgala_check.so, loaded by one test): the previous generation
+        // of the convolution products, one tensor copy per kernel offset, as an independent second implementation.
         c->legacy_conv = getenv("GALA_CONV_LEGACY") != nullptr;
+#endif
         if (n >= 5) c->agent_ctas = sm_count() * 8 / n < 32 ? 32 : sm_count() * 8 / n;   // measured on 64 agents: 32 beats 16 and 64
         c->fused_heads = heads_fused_supported(c->T, c->E, c->A, kHidden) && getenv("GALA_HEADS_UNFUSED") == nullptr;
         ALLOC(c->heads_partial, (size_t)n * c->E * 4); ALLOC(c->heads_ticket, n);
@@ -1464,6 +1485,9 @@ int gala_destroy(gala_ctx* c) {
         if (L.done) cudaEventDestroy(L.done);
     }
     if (c->side_stream) cudaStreamDestroy(c->side_stream);
+    if (c->tail_stream) cudaStreamDestroy(c->tail_stream);
+    if (c->ev_tail_fork) cudaEventDestroy(c->ev_tail_fork);
+    if (c->ev_tail_join) cudaEventDestroy(c->ev_tail_join);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->main_stream) cudaStreamDestroy(c->main_stream);

@@ -469,6 +469,10 @@ def test_conv_bias_slices_many_small_agents(monkeypatch):
 def test_conv_sync_round_legacy_products(monkeypatch):
     # the previous generation of the convolution products (one TMA box per kernel offset, bf16 frame copies)
     # is kept as an independent cross-check of the resident-input kernels
+    # (only the cross-check build of the library knows the switch; the product build ignores it)
+    from paper_1906_04585_b200 import binding as B_, build as BLD
+    monkeypatch.setattr(B_, "LIB_PATH", BLD.CHECK_LIB)
+    monkeypatch.setattr(B_, "_lib", None)
     monkeypatch.setenv("GALA_CONV_LEGACY", "1")
     w = GI.WORKLOADS[1].scaled(n_agents=2, n_envs=3, n_steps=2)
     _sync_rounds(w, rounds=1, tol_net=TOL_BF16, tol_params=TOL_BF16, mode="update")
