@@ -48,7 +48,15 @@ MIN_REGION_S = 0.3           # every timed region lasts at least this long (the 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture of the kernel class named, on the
 # workload named, taken on the kernels as they are now; an entry is removed when its kernel changes.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # all-agent optimiser / gossip pass inside the c2 round (kernel unchanged since the capture): 162.1 MB read +
+    # 78.4 MB written against 297.2 MB algorithmic; part of the output is still in L2 when the kernel ends
+    ("c2_conv_exp_n8", "sweep_sync"): 240.5e6,
+}
+# For classes whose launches differ in size (the grouped optimiser / gossip pass takes the agents that were ready):
+# dram bytes / algorithmic bytes from an ncu capture of the same kernel (32 agents x 1.7 M parameters, every agent
+# averaging with one in-peer: 1 472.9 MB against 1 523.2 MB); its traffic is proportional to agents x parameters.
+NCU_TRAFFIC_RATIO = {"sweep_agent": 1472.9 / 1523.2}
 
 
 def peaks():
@@ -524,6 +532,8 @@ def measure(env: Env, w: GI.Workload, mode: str, key: str, e2e: bool = True):
         achieved = amount / (per_step_ms * 1e-3) / 1e12 if per_step_ms > 0 else 0.0
         peak, unit = pk["tensor"], "TFLOP/s"
     traffic = NCU_TRAFFIC_BYTES.get((w.name, dominant))
+    if traffic is None and dominant in NCU_TRAFFIC_RATIO and launches_per_step > 0:
+        traffic = NCU_TRAFFIC_RATIO[dominant] * amount / launches_per_step   # per launch, like `achieved`
     roofline = dict(kernel=dominant, bound=bound, achieved=achieved, peak=peak, unit=unit, frac=achieved / peak,
                     peak_source=pk["source"], traffic=traffic,
                     algorithmic_per_step=amount, ms_per_step=per_step_ms, ms_per_launch=per_launch_ms,
