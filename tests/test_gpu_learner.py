@@ -423,6 +423,15 @@ def test_async_replay_conv_with_sm_budget():
     _async_replay(w, [0, 1, 0, 2, 3, 1, 0, 3], TOL_BF16, TOL_BF16, mode="update", agent_ctas=5)
 
 
+def test_async_replay_conv_many_units_per_block():
+    # Two thread blocks per kernel: a block of conv1's forward pass takes 42 units, one of the other convolution
+    # kernels 10-12 samples, so every ring of stages, every byte-ring slot and every accumulator buffer is reused
+    # many times by every role (a barrier's phases must be seen in order by its one waiter: with few units a block,
+    # as in the other small cases, a role that skips or repeats a phase would go unnoticed).
+    w = GI.WORKLOADS[2].scaled(n_agents=2, n_envs=4, n_steps=5)
+    _async_replay(w, [0, 1, 0, 1], TOL_BF16, TOL_BF16, mode="update", agent_ctas=2)
+
+
 def test_conv_sync_round_unfused_heads(monkeypatch):
     # the separate heads / objective / head-gradient kernels (used when a rollout is too long for the fused
     # kernel's shared memory) against the same oracle
