@@ -26,6 +26,12 @@ def _run_sync_round(w, sampled):
     L.step_sync(dev)
     L.sync()
     S, Bn, A = w.n_envs * w.n_steps, w.n_envs * (w.n_steps + 1), w.n_actions
+    if w.n_agents <= 16:
+        # the optimiser / gossip stage of the full-size launch on its own: replayed in the oracle from the gradient
+        # and norm the library computed, all agents, parameters and second moments to 1e-5, bf16 copy bit for bit
+        from tests.test_gpu_learner import replay_sweep_from_library_gradient
+        X0 = np.tile(p0.astype(np.float64), (w.n_agents, 1))
+        replay_sweep_from_library_gradient(L, B, w, X0, np.zeros_like(X0), ohp, 0)
     # the oracle recomputes the sampled agents and their in-peers of round 0
     need = sorted(set(sampled) | {j for i in sampled for j in R.in_peers(w.topo_kind, w.topo_peers, w.n_agents, 0, i)})
     x0 = p0.astype(np.float64)
