@@ -52,6 +52,8 @@ NCU_TRAFFIC_BYTES = {
     # all-agent optimiser / gossip pass inside the c2 round (kernel unchanged since the capture): 162.1 MB read +
     # 78.4 MB written against 297.2 MB algorithmic; part of the output is still in L2 when the kernel ends
     ("c2_conv_exp_n8", "sweep_sync"): 240.5e6,
+    # conv1 forward at c3: 304.2 MB read (the uint8 frames, once) + 250.3 MB written (act1 and gate words)
+    ("c3_conv_exp_n16", "gemm_conv1_fwd"): 554.5e6,
 }
 # For classes whose launches differ in size (the grouped optimiser / gossip pass takes the agents that were ready):
 # dram bytes / algorithmic bytes from an ncu capture of the same kernel (32 agents x 1.7 M parameters, every agent
